@@ -1,0 +1,208 @@
+/*
+ * ebs.h -- C ABI of the binary-decomposition (BD) mixed-precision convolution
+ * library for NVIDIA B200 (sm_100a).
+ *
+ * The operation (paper Sec. 4.3, Eq. 12-15, built on Eq. 2): a convolution between
+ * M-bit weights and K-bit activations is computed by splitting both operands into
+ * binary bit-planes; stage 1 is a binary convolution (AND + bitcount) between every
+ * weight plane m and activation plane k, stage 2 recombines the M*K partial results
+ * with powers of two 2^(m+k).  Every layer may use its own (M, K).  In this header
+ * M is `w_bits` and K is `a_bits`.
+ *
+ * Number formats.  Activation codes are unsigned, 0 .. 2^a_bits-1 (Eq. 1b: the
+ * activation is a_scale * code with a_scale = alpha / (2^a_bits-1)).  Weight codes
+ * are signed two's complement, -2^(w_bits-1) .. 2^(w_bits-1)-1, real value w_scale *
+ * code; the top weight plane therefore carries the coefficient -2^(w_bits-1).
+ * Rounding is "round half up" (text after Eq. 1c): code = floor(x * (1/scale) + 0.5),
+ * evaluated in fp32 with 1/scale rounded once and every operation rounded on its own.
+ *
+ * Conventions for every entry point
+ *  - Pointers named *_dev are DEVICE pointers on the current CUDA device; pointers
+ *    named *_host are host pointers.  All buffers are owned by the caller; the library
+ *    keeps no state between calls and allocates nothing (the one exception is the
+ *    measurement helper ebs_probe_pipe, which allocates and frees a small scratch).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *    Work is enqueued on it and the call returns without waiting.
+ *  - Device buffers must be 16-byte aligned (buffers from cudaMalloc / torch are).
+ *  - Return value: an ebs_status (0 = success, negative = error).  Arguments are
+ *    validated on the host before anything is launched; on error nothing has been
+ *    enqueued.  No call aborts, throws or traps.
+ *
+ * Packed bit-plane layouts (little-endian 32-bit words, CW = ceil(C/32)):
+ *  - activations  u32 [N][H][W][CW][a_bits]: bit (c % 32) of word [n][h][w][c/32][k]
+ *    is bit k of the code of channel c at pixel (n,h,w);
+ *  - weights      u32 [kh][kw][CW][C_out][w_bits]: bit (c % 32) of word
+ *    [r][s][c/32][co][m] is bit m of the two's-complement code of W[co][c][r][s];
+ *  - bits of channels >= C are zero in both.
+ */
+#ifndef EBS_H_
+#define EBS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum ebs_status {
+    EBS_OK = 0,
+    EBS_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, bitwidth outside 1..8, misalignment */
+    EBS_ERR_UNSUPPORTED = -2, /* valid request this build has no kernel for */
+    EBS_ERR_OVERFLOW = -3,    /* c_in*kh*kw*2^(w_bits-1)*(2^a_bits-1) >= 2^31, or an index would overflow */
+    EBS_ERR_CUDA = -4,        /* a CUDA runtime call failed (launch error, bad device pointer, ...) */
+    EBS_ERR_TIMEOUT = -5      /* a bounded device-side wait gave up (reserved) */
+} ebs_status;
+
+typedef enum ebs_layout {
+    EBS_NCHW = 0, /* activations [N][C][H][W]; weights [C_out][C_in][kh][kw] */
+    EBS_NHWC = 1  /* activations [N][H][W][C]; weights [C_out][kh][kw][C_in] */
+} ebs_layout;
+
+typedef enum ebs_dtype {
+    EBS_F32 = 0,      /* real values; quantized inside the call (Eq. 1b / 1c) */
+    EBS_I8_CODES = 1, /* signed 8-bit integer codes (weights) */
+    EBS_U8_CODES = 2  /* unsigned 8-bit integer codes (activations) */
+} ebs_dtype;
+
+/* One convolution layer (Sec. 3: weight tensor c_i x c_o x k x k; Sec. 4.3: per-layer M and K). */
+typedef struct ebs_conv_desc {
+    int c_in, c_out;
+    int kh, kw;
+    int stride_h, stride_w;
+    int pad_h, pad_w;   /* zero padding: a padded tap is the real value 0 */
+    int w_bits, a_bits; /* M and K of the paper, 1..8 each */
+    float w_scale;      /* real weight  = w_scale * code */
+    float a_scale;      /* real input   = a_scale * code */
+} ebs_conv_desc;
+
+/*
+ * Optional epilogue after the integer accumulator (scale merge of Sec. 4.3, clip and
+ * round of Eq. 1b-1c / Eq. 16a-16c), each step a separately rounded fp32 operation:
+ *   y = float(acc) * S                 S = fl32(w_scale * a_scale)
+ *   y = y * ch_scale[co]               if ch_scale_dev
+ *   y = y + ch_bias[co]                if ch_bias_dev
+ *   y = y + residual[n][ho][wo][co]    if residual_dev   (fp32, NHWC, output shape)
+ *   y = max(y, 0)                      if relu
+ *   q = clamp(floor(y * (1/next_a_scale) + 0.5), 0, 2^next_a_bits - 1)   (packed output only)
+ * A NULL epilogue means: no per-channel terms, no residual, no ReLU, y in NHWC.
+ */
+typedef struct ebs_epilogue {
+    const float *ch_scale_dev; /* nullable, length c_out */
+    const float *ch_bias_dev;  /* nullable, length c_out */
+    const float *residual_dev; /* nullable */
+    int relu;                  /* 0 / 1 */
+    int next_a_bits;           /* bitwidth of packed_next (1..8); ignored if packed_next is NULL */
+    float next_a_scale;        /* step of the next layer's activation quantizer */
+    int y_layout;              /* ebs_layout of y_out */
+} ebs_epilogue;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int ebs_version(void);
+
+/* Human-readable text for an ebs_status; never NULL. */
+const char *ebs_status_string(int status);
+
+/* Text of the last CUDA error seen by this thread's failing call ("" if none). */
+const char *ebs_last_cuda_error(void);
+
+/* Output height/width of the img2col convolution (Sec. 4.3): floor((in + 2 pad - k)/stride) + 1.
+ * Returns EBS_ERR_INVALID_ARG if the kernel is larger than the padded input. */
+int ebs_conv_out_shape(const ebs_conv_desc *desc, int h, int w, int *h_out, int *w_out);
+
+/* Size in bytes of the packed weight planes of a layer: kh*kw*ceil(c_in/32)*c_out*w_bits*4.
+ * "BD incurs the same memory cost as the weights before BD" (Sec. 4.3, complexity).  0 on bad input. */
+size_t ebs_packed_weight_bytes(const ebs_conv_desc *desc);
+
+/* Size in bytes of packed activation planes: n*h*w*ceil(c/32)*a_bits*4.  0 on bad input. */
+size_t ebs_packed_act_bytes(int n, int h, int w, int c, int a_bits);
+
+/*
+ * Weight quantization and bit-plane expansion B_w (Eq. 12, Eq. 15; quantizer Eq. 1c).
+ *   w_dev       c_out*c_in*kh*kw values in `layout`; EBS_F32 (quantized with desc->w_scale to
+ *               signed desc->w_bits codes) or EBS_I8_CODES (taken as they are; must be in range).
+ *   packed_w_dev  ebs_packed_weight_bytes(desc) bytes, fully overwritten.
+ * Done once per layer, off the inference path.
+ */
+int ebs_pack_weights(const void *w_dev, int dtype, int layout, const ebs_conv_desc *desc,
+                     void *packed_w_dev, void *stream);
+
+/*
+ * Activation quantization (Eq. 1b: clip to [0, alpha], round half up) and bit-plane expansion B_x
+ * (Sec. 4.3).  x_dev holds n*c*h*w values in `layout`; EBS_F32 (quantized with a_scale) or
+ * EBS_U8_CODES (only the low a_bits bits of each code are used).  packed_x_dev receives
+ * ebs_packed_act_bytes(n,h,w,c,a_bits) bytes, fully overwritten.
+ */
+int ebs_pack_acts(const void *x_dev, int dtype, int layout, int n, int c, int h, int w, int a_bits,
+                  float a_scale, void *packed_x_dev, void *stream);
+
+/*
+ * The mixed-precision convolution by binary decomposition (Eq. 13-14): for every output
+ * (n, ho, wo, co)
+ *   acc = sum_{m<M} sum_{k<K} c_m 2^(m+k) * sum_{taps, channel words} popcount(A_k AND W_m),
+ *   c_m = -1 for m = M-1 (signed weights), +1 otherwise,
+ * with taps outside the image contributing zero.  The M*K partial sums (the paper's matrix P)
+ * never leave the chip.  Any subset of the three outputs may be requested (at least one):
+ *   acc_out_dev     int32 [N][Ho][Wo][C_out]                      exact accumulators
+ *   y_out_dev       fp32, epilogue applied, layout epi->y_layout  (NHWC if epi is NULL)
+ *   packed_next_dev u32 [N][Ho][Wo][ceil(C_out/32)][next_a_bits]  requantized, ready to be the
+ *                   packed_x_dev of the next layer (requires epi)
+ * packed_x_dev: activations [n][h][w] with desc->c_in channels and desc->a_bits planes;
+ * packed_w_dev: weights of `desc`.  Both as produced by the pack calls (or a previous layer).
+ */
+int ebs_conv2d_mixed(const void *packed_x_dev, int n, int h, int w, const void *packed_w_dev,
+                     const ebs_conv_desc *desc, const ebs_epilogue *epi, int32_t *acc_out_dev,
+                     float *y_out_dev, void *packed_next_dev, void *stream);
+
+/*
+ * The same call with the tile variant forced (0 .. ebs_num_conv_variants()-1) instead of chosen by
+ * the built-in heuristic (-1); the result is identical for every variant, only the speed differs.
+ * For tuning and for tests that must cover every kernel instantiation.  Returns
+ * EBS_ERR_UNSUPPORTED if the variant cannot produce the requested packed output.
+ */
+int ebs_num_conv_variants(void);
+int ebs_conv2d_mixed_variant(const void *packed_x_dev, int n, int h, int w, const void *packed_w_dev,
+                             const ebs_conv_desc *desc, const ebs_epilogue *epi, int32_t *acc_out_dev,
+                             float *y_out_dev, void *packed_next_dev, void *stream, int variant);
+
+/*
+ * Stand-alone de-quantization of accumulators ("quantize_b includes the de-quantize process",
+ * text after Eq. 1c): y = float(acc) * scale, then * ch_scale[co], + ch_bias[co], ReLU, each
+ * optional, over n_pixels * c_out values stored pixel-major (NHWC).
+ */
+int ebs_dequant(const int32_t *acc_dev, size_t n_pixels, int c_out, float scale,
+                const float *ch_scale_dev, const float *ch_bias_dev, int relu, float *y_dev,
+                void *stream);
+
+/*
+ * One layer from HOST buffers, for callers whose data lives on the host: copies the activations
+ * to the device, packs them, runs ebs_conv2d_mixed and copies the requested outputs back, all
+ * enqueued on `stream` (host buffers should be pinned for the copies to be asynchronous; the
+ * caller synchronizes the stream before reading the outputs).
+ *   x_host            n*c_in*h*w values, dtype EBS_F32 or EBS_U8_CODES, in `layout`
+ *   packed_w_dev      packed weights already on the device
+ *   workspace_dev     caller-provided device scratch of at least ebs_host_workspace_bytes(...)
+ *   acc_out_host / y_out_host / packed_next_host   any subset, same shapes as the device call
+ * epi's pointers are still DEVICE pointers.
+ */
+size_t ebs_host_workspace_bytes(const ebs_conv_desc *desc, int n, int h, int w, int dtype, int next_a_bits);
+int ebs_conv2d_mixed_host(const void *x_host, int dtype, int layout, int n, int h, int w,
+                          const void *packed_w_dev, const ebs_conv_desc *desc, const ebs_epilogue *epi,
+                          void *workspace_dev, size_t workspace_bytes, int32_t *acc_out_host,
+                          float *y_out_host, void *packed_next_host, void *stream);
+
+/*
+ * Register-resident throughput probe of the execution pipes the convolution can use; the
+ * measured rate is the denominator of the kernel's arithmetic roofline.  Runs `iters` loop
+ * iterations on every SM, synchronizes the device, and writes the measured rate.
+ *   kind 0: AND + POPC + accumulate on the integer pipes        -> bit-AND-popcounts per second
+ *   kind 1: mma.sync m16n8k256 b1 AND.POPC                      -> bit-AND-popcounts per second
+ *   kind 2: POPC alone                                          -> bit-popcounts per second
+ * The paper has no counterpart; this is measurement support.
+ */
+int ebs_probe_pipe(int kind, int iters, double *bit_ops_per_second);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EBS_H_ */

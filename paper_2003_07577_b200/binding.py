@@ -1,0 +1,190 @@
+"""Thin ctypes binding of libebs.so: argument marshalling only.
+
+Every function has the name and argument order of its C entry point in ``include/ebs.h`` and
+does no arithmetic of its own.  Tensors are ``torch.Tensor`` objects used purely as device (or
+pinned host) memory: the binding passes ``tensor.data_ptr()`` and the current CUDA stream.
+There is no CPU fallback: if the shared library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libebs.so")
+
+EBS_OK, EBS_ERR_INVALID_ARG, EBS_ERR_UNSUPPORTED, EBS_ERR_OVERFLOW, EBS_ERR_CUDA, EBS_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+EBS_NCHW, EBS_NHWC = 0, 1
+EBS_F32, EBS_I8_CODES, EBS_U8_CODES = 0, 1, 2
+
+EXPORTS = [
+    "ebs_version", "ebs_status_string", "ebs_last_cuda_error", "ebs_conv_out_shape", "ebs_packed_weight_bytes",
+    "ebs_packed_act_bytes", "ebs_pack_weights", "ebs_pack_acts", "ebs_conv2d_mixed", "ebs_num_conv_variants",
+    "ebs_conv2d_mixed_variant", "ebs_dequant", "ebs_host_workspace_bytes", "ebs_conv2d_mixed_host",
+    "ebs_probe_pipe",
+]
+
+
+class ebs_conv_desc(ctypes.Structure):
+    _fields_ = [("c_in", ctypes.c_int), ("c_out", ctypes.c_int), ("kh", ctypes.c_int), ("kw", ctypes.c_int),
+                ("stride_h", ctypes.c_int), ("stride_w", ctypes.c_int), ("pad_h", ctypes.c_int),
+                ("pad_w", ctypes.c_int), ("w_bits", ctypes.c_int), ("a_bits", ctypes.c_int),
+                ("w_scale", ctypes.c_float), ("a_scale", ctypes.c_float)]
+
+
+class ebs_epilogue(ctypes.Structure):
+    _fields_ = [("ch_scale_dev", ctypes.c_void_p), ("ch_bias_dev", ctypes.c_void_p),
+                ("residual_dev", ctypes.c_void_p), ("relu", ctypes.c_int), ("next_a_bits", ctypes.c_int),
+                ("next_a_scale", ctypes.c_float), ("y_layout", ctypes.c_int)]
+
+
+class EbsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        text = lib().ebs_status_string(status).decode()
+        cuda = lib().ebs_last_cuda_error().decode() if status == EBS_ERR_CUDA else ""
+        super().__init__(f"{where}: {text} ({status})" + (f": {cuda}" if cuda else ""))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libebs.so (built by ``paper_2003_07577_b200.build``); raises if it is not there."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2003_07577_b200.build` "
+                              "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        i, f, p, z = ctypes.c_int, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t
+        D, E = ctypes.POINTER(ebs_conv_desc), ctypes.POINTER(ebs_epilogue)
+        L.ebs_version.restype = i
+        L.ebs_status_string.argtypes = [i]
+        L.ebs_status_string.restype = ctypes.c_char_p
+        L.ebs_last_cuda_error.restype = ctypes.c_char_p
+        L.ebs_conv_out_shape.argtypes = [D, i, i, ctypes.POINTER(i), ctypes.POINTER(i)]
+        L.ebs_packed_weight_bytes.argtypes = [D]
+        L.ebs_packed_weight_bytes.restype = z
+        L.ebs_packed_act_bytes.argtypes = [i, i, i, i, i]
+        L.ebs_packed_act_bytes.restype = z
+        L.ebs_pack_weights.argtypes = [p, i, i, D, p, p]
+        L.ebs_pack_acts.argtypes = [p, i, i, i, i, i, i, i, f, p, p]
+        L.ebs_conv2d_mixed.argtypes = [p, i, i, i, p, D, E, p, p, p, p]
+        L.ebs_num_conv_variants.restype = i
+        L.ebs_conv2d_mixed_variant.argtypes = [p, i, i, i, p, D, E, p, p, p, p, i]
+        L.ebs_dequant.argtypes = [p, z, i, f, p, p, i, p, p]
+        L.ebs_host_workspace_bytes.argtypes = [D, i, i, i, i, i]
+        L.ebs_host_workspace_bytes.restype = z
+        L.ebs_conv2d_mixed_host.argtypes = [p, i, i, i, i, i, p, D, E, p, z, p, p, p, p]
+        L.ebs_probe_pipe.argtypes = [i, i, ctypes.POINTER(ctypes.c_double)]
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _check(rc: int, where: str):
+    if rc != EBS_OK:
+        raise EbsError(rc, where)
+
+
+def conv_desc(c_in, c_out, kh, kw, stride_h, stride_w, pad_h, pad_w, w_bits, a_bits, w_scale, a_scale) -> ebs_conv_desc:
+    return ebs_conv_desc(c_in, c_out, kh, kw, stride_h, stride_w, pad_h, pad_w, w_bits, a_bits, w_scale, a_scale)
+
+
+def epilogue(ch_scale=None, ch_bias=None, residual=None, relu=False, next_a_bits=0, next_a_scale=1.0,
+             y_layout=EBS_NHWC) -> ebs_epilogue:
+    e = ebs_epilogue(None if ch_scale is None else ch_scale.data_ptr(),
+                     None if ch_bias is None else ch_bias.data_ptr(),
+                     None if residual is None else residual.data_ptr(),
+                     int(bool(relu)), int(next_a_bits), float(next_a_scale), int(y_layout))
+    e._keepalive = (ch_scale, ch_bias, residual)
+    return e
+
+
+def ebs_version() -> int:
+    return lib().ebs_version()
+
+
+def ebs_status_string(status: int) -> str:
+    return lib().ebs_status_string(status).decode()
+
+
+def ebs_conv_out_shape(desc: ebs_conv_desc, h: int, w: int):
+    ho, wo = ctypes.c_int(0), ctypes.c_int(0)
+    _check(lib().ebs_conv_out_shape(ctypes.byref(desc), h, w, ctypes.byref(ho), ctypes.byref(wo)), "ebs_conv_out_shape")
+    return ho.value, wo.value
+
+
+def ebs_packed_weight_bytes(desc: ebs_conv_desc) -> int:
+    return lib().ebs_packed_weight_bytes(ctypes.byref(desc))
+
+
+def ebs_packed_act_bytes(n: int, h: int, w: int, c: int, a_bits: int) -> int:
+    return lib().ebs_packed_act_bytes(n, h, w, c, a_bits)
+
+
+def ebs_pack_weights(w_dev: torch.Tensor, dtype: int, layout: int, desc: ebs_conv_desc, packed_w_dev: torch.Tensor,
+                     stream=None) -> None:
+    _check(lib().ebs_pack_weights(_ptr(w_dev), dtype, layout, ctypes.byref(desc), _ptr(packed_w_dev), _stream(stream)),
+           "ebs_pack_weights")
+
+
+def ebs_pack_acts(x_dev: torch.Tensor, dtype: int, layout: int, n: int, c: int, h: int, w: int, a_bits: int,
+                  a_scale: float, packed_x_dev: torch.Tensor, stream=None) -> None:
+    _check(lib().ebs_pack_acts(_ptr(x_dev), dtype, layout, n, c, h, w, a_bits, a_scale, _ptr(packed_x_dev),
+                               _stream(stream)), "ebs_pack_acts")
+
+
+def ebs_conv2d_mixed(packed_x_dev, n, h, w, packed_w_dev, desc, epi=None, acc_out_dev=None, y_out_dev=None,
+                     packed_next_dev=None, stream=None, variant: int = -1) -> None:
+    e = None if epi is None else ctypes.byref(epi)
+    if variant < 0:
+        rc = lib().ebs_conv2d_mixed(_ptr(packed_x_dev), n, h, w, _ptr(packed_w_dev), ctypes.byref(desc), e,
+                                    _ptr(acc_out_dev), _ptr(y_out_dev), _ptr(packed_next_dev), _stream(stream))
+    else:
+        rc = lib().ebs_conv2d_mixed_variant(_ptr(packed_x_dev), n, h, w, _ptr(packed_w_dev), ctypes.byref(desc), e,
+                                            _ptr(acc_out_dev), _ptr(y_out_dev), _ptr(packed_next_dev),
+                                            _stream(stream), variant)
+    _check(rc, "ebs_conv2d_mixed")
+
+
+def ebs_num_conv_variants() -> int:
+    return lib().ebs_num_conv_variants()
+
+
+def ebs_dequant(acc_dev, n_pixels: int, c_out: int, scale: float, ch_scale_dev=None, ch_bias_dev=None,
+                relu=False, y_dev=None, stream=None) -> None:
+    _check(lib().ebs_dequant(_ptr(acc_dev), n_pixels, c_out, scale, _ptr(ch_scale_dev), _ptr(ch_bias_dev),
+                             int(bool(relu)), _ptr(y_dev), _stream(stream)), "ebs_dequant")
+
+
+def ebs_host_workspace_bytes(desc, n, h, w, dtype, next_a_bits=0) -> int:
+    return lib().ebs_host_workspace_bytes(ctypes.byref(desc), n, h, w, dtype, next_a_bits)
+
+
+def ebs_conv2d_mixed_host(x_host, dtype, layout, n, h, w, packed_w_dev, desc, epi, workspace_dev,
+                          acc_out_host=None, y_out_host=None, packed_next_host=None, stream=None) -> None:
+    e = None if epi is None else ctypes.byref(epi)
+    rc = lib().ebs_conv2d_mixed_host(_ptr(x_host), dtype, layout, n, h, w, _ptr(packed_w_dev), ctypes.byref(desc), e,
+                                     _ptr(workspace_dev), workspace_dev.numel() * workspace_dev.element_size(),
+                                     _ptr(acc_out_host), _ptr(y_out_host), _ptr(packed_next_host), _stream(stream))
+    _check(rc, "ebs_conv2d_mixed_host")
+
+
+def ebs_probe_pipe(kind: int, iters: int = 2000) -> float:
+    out = ctypes.c_double(0.0)
+    _check(lib().ebs_probe_pipe(kind, iters, ctypes.byref(out)), "ebs_probe_pipe")
+    return out.value

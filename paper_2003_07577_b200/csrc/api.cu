@@ -1,0 +1,282 @@
+// C ABI of libebs: host-side validation, kernel selection, launches.  See include/ebs.h.
+#include <string.h>
+
+#include "ebs_internal.cuh"
+
+namespace ebs {
+
+static thread_local char g_cuda_error[256] = "";
+
+int check_cuda(cudaError_t e) {
+    if (e == cudaSuccess) return EBS_OK;
+    strncpy(g_cuda_error, cudaGetErrorString(e), sizeof(g_cuda_error) - 1);
+    g_cuda_error[sizeof(g_cuda_error) - 1] = '\0';
+    return EBS_ERR_CUDA;
+}
+
+const ConvVariant* conv_popc_variant(int w_bits, int a_bits, int variant) {
+    switch (w_bits) {
+        case 1: return conv_popc_variant_w1(a_bits, variant);
+        case 2: return conv_popc_variant_w2(a_bits, variant);
+        case 3: return conv_popc_variant_w3(a_bits, variant);
+        case 4: return conv_popc_variant_w4(a_bits, variant);
+        case 5: return conv_popc_variant_w5(a_bits, variant);
+        case 6: return conv_popc_variant_w6(a_bits, variant);
+        case 7: return conv_popc_variant_w7(a_bits, variant);
+        case 8: return conv_popc_variant_w8(a_bits, variant);
+        default: return nullptr;
+    }
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int out_dim(int in, int pad, int k, int stride) {
+    const int span = in + 2 * pad - k;
+    return span < 0 ? 0 : span / stride + 1;
+}
+
+static int validate_desc(const ebs_conv_desc* d) {
+    if (!d) return EBS_ERR_INVALID_ARG;
+    if (d->c_in <= 0 || d->c_out <= 0 || d->kh <= 0 || d->kw <= 0 || d->stride_h <= 0 || d->stride_w <= 0 ||
+        d->pad_h < 0 || d->pad_w < 0)
+        return EBS_ERR_INVALID_ARG;
+    if (d->w_bits < 1 || d->w_bits > 8 || d->a_bits < 1 || d->a_bits > 8) return EBS_ERR_INVALID_ARG;
+    if (d->kh > 255 || d->kw > 255 || d->c_in > (1 << 20) || d->c_out > (1 << 20)) return EBS_ERR_UNSUPPORTED;
+    if (!(d->w_scale > 0.0f) || !(d->a_scale > 0.0f)) return EBS_ERR_INVALID_ARG;
+    // largest |acc| = c_in*kh*kw * 2^(w_bits-1) * (2^a_bits - 1) must fit int32
+    const long long s = (long long)d->c_in * d->kh * d->kw;
+    const long long worst = s * (1LL << (d->w_bits - 1)) * ((1LL << d->a_bits) - 1);
+    if (worst >= (1LL << 31)) return EBS_ERR_OVERFLOW;
+    return EBS_OK;
+}
+
+static int sm_count() {
+    int dev = 0, n = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    return n > 0 ? n : 148;
+}
+
+// Picks the tile variant: tile_c from c_out, then the largest pixel tile that still gives every SM
+// about two CTAs; problems too small for that use the small tile.
+static int choose_variant(int w_bits, int a_bits, int P, int Co, bool want_packed, int sms) {
+    const int tc_idx = Co <= 16 ? 0 : (Co <= 32 ? 1 : 2);
+    for (int tp_idx = 2; tp_idx >= 0; --tp_idx) {
+        const ConvVariant* v = conv_popc_variant(w_bits, a_bits, tc_idx * 3 + tp_idx);
+        const long long ctas = (long long)((P + v->tile_p - 1) / v->tile_p) * ((Co + v->tile_c - 1) / v->tile_c);
+        if (ctas >= 2LL * sms) return tc_idx * 3 + tp_idx;
+    }
+    const ConvVariant* v1 = conv_popc_variant(w_bits, a_bits, tc_idx * 3);
+    const long long ctas1 = (long long)((P + v1->tile_p - 1) / v1->tile_p) * ((Co + v1->tile_c - 1) / v1->tile_c);
+    if (ctas1 >= sms) return tc_idx * 3;
+    // the small tile has 16 channels: a packed output word needs all 32 channels of a word in one CTA
+    if (want_packed && Co > 16) return tc_idx * 3;
+    return CONV_VARIANT_SMALL;
+}
+
+static int conv_impl(const void* packed_x, int n, int h, int w, const void* packed_w, const ebs_conv_desc* d,
+                     const ebs_epilogue* epi, int32_t* acc_out, float* y_out, void* packed_next, void* stream,
+                     int variant) {
+    int rc = validate_desc(d);
+    if (rc) return rc;
+    if (!packed_x || !packed_w || n <= 0 || h <= 0 || w <= 0) return EBS_ERR_INVALID_ARG;
+    if (!acc_out && !y_out && !packed_next) return EBS_ERR_INVALID_ARG;
+    if (!aligned16(packed_x) || !aligned16(packed_w) || !aligned16(acc_out) || !aligned16(y_out) ||
+        !aligned16(packed_next))
+        return EBS_ERR_INVALID_ARG;
+    if (h > 32000 || w > 32000) return EBS_ERR_UNSUPPORTED;
+    const int Ho = out_dim(h, d->pad_h, d->kh, d->stride_h), Wo = out_dim(w, d->pad_w, d->kw, d->stride_w);
+    if (Ho <= 0 || Wo <= 0) return EBS_ERR_INVALID_ARG;
+    const long long P = (long long)n * Ho * Wo, in_pixels = (long long)n * h * w;
+    if (P >= (1LL << 31) || in_pixels >= (1LL << 31) || P * d->c_out >= (1LL << 40)) return EBS_ERR_OVERFLOW;
+    if (packed_next) {
+        if (!epi || epi->next_a_bits < 1 || epi->next_a_bits > 8 || !(epi->next_a_scale > 0.0f))
+            return EBS_ERR_INVALID_ARG;
+    }
+    if (epi) {
+        if (epi->y_layout != EBS_NCHW && epi->y_layout != EBS_NHWC) return EBS_ERR_INVALID_ARG;
+        if (!aligned16(epi->residual_dev)) return EBS_ERR_INVALID_ARG;
+    }
+    if (variant >= NUM_CONV_VARIANTS) return EBS_ERR_INVALID_ARG;
+
+    ConvParams p;
+    memset(&p, 0, sizeof(p));
+    p.x = static_cast<const uint32_t*>(packed_x);
+    p.w = static_cast<const uint32_t*>(packed_w);
+    p.N = n; p.H = h; p.W = w; p.CW = (d->c_in + 31) / 32;
+    p.Co = d->c_out; p.Ho = Ho; p.Wo = Wo; p.CWo = (d->c_out + 31) / 32;
+    p.kh = d->kh; p.kw = d->kw; p.sh = d->stride_h; p.sw = d->stride_w; p.ph = d->pad_h; p.pw = d->pad_w;
+    p.KK = d->kh * d->kw * p.CW;
+    p.P = (int)P;
+    p.acc = acc_out; p.y = y_out; p.packed_next = static_cast<uint32_t*>(packed_next);
+    p.S = d->w_scale * d->a_scale;       // one rounded fp32 multiply
+    p.next_bits = 1;
+    if (epi) {
+        p.ch_scale = epi->ch_scale_dev; p.ch_bias = epi->ch_bias_dev; p.residual = epi->residual_dev;
+        p.relu = epi->relu ? 1 : 0;
+        p.y_nchw = epi->y_layout == EBS_NCHW;
+        if (packed_next) { p.next_bits = epi->next_a_bits; p.inv_next = 1.0f / epi->next_a_scale; }
+    }
+    if (variant < 0) variant = choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
+    const ConvVariant* v = conv_popc_variant(d->w_bits, d->a_bits, variant);
+    if (!v) return EBS_ERR_UNSUPPORTED;
+    if (packed_next && (v->tile_c % 32) != 0 && v->tile_c < p.Co) return EBS_ERR_UNSUPPORTED;
+    const long long gx = (P + v->tile_p - 1) / v->tile_p, gy = (p.Co + v->tile_c - 1) / v->tile_c;
+    if (gy > 65535) return EBS_ERR_UNSUPPORTED;
+    v->launch(p, dim3((unsigned)gx, (unsigned)gy, 1), static_cast<cudaStream_t>(stream));
+    return check_cuda(cudaGetLastError());
+}
+
+}  // namespace ebs
+
+using namespace ebs;
+
+extern "C" {
+
+int ebs_version(void) { return 100; }
+
+const char* ebs_status_string(int status) {
+    switch (status) {
+        case EBS_OK: return "ok";
+        case EBS_ERR_INVALID_ARG: return "invalid argument";
+        case EBS_ERR_UNSUPPORTED: return "unsupported configuration";
+        case EBS_ERR_OVERFLOW: return "accumulator or index would overflow";
+        case EBS_ERR_CUDA: return "CUDA runtime error";
+        case EBS_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+const char* ebs_last_cuda_error(void) { return g_cuda_error; }
+
+int ebs_conv_out_shape(const ebs_conv_desc* d, int h, int w, int* h_out, int* w_out) {
+    int rc = validate_desc(d);
+    if (rc) return rc;
+    if (h <= 0 || w <= 0 || !h_out || !w_out) return EBS_ERR_INVALID_ARG;
+    const int Ho = out_dim(h, d->pad_h, d->kh, d->stride_h), Wo = out_dim(w, d->pad_w, d->kw, d->stride_w);
+    if (Ho <= 0 || Wo <= 0) return EBS_ERR_INVALID_ARG;
+    *h_out = Ho;
+    *w_out = Wo;
+    return EBS_OK;
+}
+
+size_t ebs_packed_weight_bytes(const ebs_conv_desc* d) {
+    if (validate_desc(d)) return 0;
+    return (size_t)d->kh * d->kw * ((d->c_in + 31) / 32) * d->c_out * d->w_bits * sizeof(uint32_t);
+}
+
+size_t ebs_packed_act_bytes(int n, int h, int w, int c, int a_bits) {
+    if (n <= 0 || h <= 0 || w <= 0 || c <= 0 || a_bits < 1 || a_bits > 8) return 0;
+    return (size_t)n * h * w * ((c + 31) / 32) * a_bits * sizeof(uint32_t);
+}
+
+int ebs_pack_weights(const void* w_dev, int dtype, int layout, const ebs_conv_desc* d, void* packed_w_dev,
+                     void* stream) {
+    int rc = validate_desc(d);
+    if (rc) return rc;
+    if (!w_dev || !packed_w_dev || !aligned16(w_dev) || !aligned16(packed_w_dev)) return EBS_ERR_INVALID_ARG;
+    if (dtype != EBS_F32 && dtype != EBS_I8_CODES) return EBS_ERR_INVALID_ARG;
+    if (layout != EBS_NCHW && layout != EBS_NHWC) return EBS_ERR_INVALID_ARG;
+    return launch_pack_weights(w_dev, dtype, layout, *d, 1.0f / d->w_scale, static_cast<uint32_t*>(packed_w_dev),
+                               static_cast<cudaStream_t>(stream));
+}
+
+int ebs_pack_acts(const void* x_dev, int dtype, int layout, int n, int c, int h, int w, int a_bits, float a_scale,
+                  void* packed_x_dev, void* stream) {
+    if (!x_dev || !packed_x_dev || n <= 0 || c <= 0 || h <= 0 || w <= 0) return EBS_ERR_INVALID_ARG;
+    if (a_bits < 1 || a_bits > 8) return EBS_ERR_INVALID_ARG;
+    if (dtype != EBS_F32 && dtype != EBS_U8_CODES) return EBS_ERR_INVALID_ARG;
+    if (layout != EBS_NCHW && layout != EBS_NHWC) return EBS_ERR_INVALID_ARG;
+    if (dtype == EBS_F32 && !(a_scale > 0.0f)) return EBS_ERR_INVALID_ARG;
+    if (!aligned16(x_dev) || !aligned16(packed_x_dev)) return EBS_ERR_INVALID_ARG;
+    if ((long long)n * h * w >= (1LL << 31)) return EBS_ERR_OVERFLOW;
+    const float inv = dtype == EBS_F32 ? 1.0f / a_scale : 1.0f;
+    return launch_pack_acts(x_dev, dtype, layout, n, c, h, w, a_bits, inv, static_cast<uint32_t*>(packed_x_dev),
+                            static_cast<cudaStream_t>(stream));
+}
+
+int ebs_conv2d_mixed(const void* packed_x_dev, int n, int h, int w, const void* packed_w_dev,
+                     const ebs_conv_desc* desc, const ebs_epilogue* epi, int32_t* acc_out_dev, float* y_out_dev,
+                     void* packed_next_dev, void* stream) {
+    return conv_impl(packed_x_dev, n, h, w, packed_w_dev, desc, epi, acc_out_dev, y_out_dev, packed_next_dev,
+                     stream, -1);
+}
+
+int ebs_num_conv_variants(void) { return NUM_CONV_VARIANTS; }
+
+int ebs_conv2d_mixed_variant(const void* packed_x_dev, int n, int h, int w, const void* packed_w_dev,
+                             const ebs_conv_desc* desc, const ebs_epilogue* epi, int32_t* acc_out_dev,
+                             float* y_out_dev, void* packed_next_dev, void* stream, int variant) {
+    return conv_impl(packed_x_dev, n, h, w, packed_w_dev, desc, epi, acc_out_dev, y_out_dev, packed_next_dev,
+                     stream, variant);
+}
+
+int ebs_dequant(const int32_t* acc_dev, size_t n_pixels, int c_out, float scale, const float* ch_scale_dev,
+                const float* ch_bias_dev, int relu, float* y_dev, void* stream) {
+    if (!acc_dev || !y_dev || n_pixels == 0 || c_out <= 0) return EBS_ERR_INVALID_ARG;
+    if (!aligned16(acc_dev) || !aligned16(y_dev)) return EBS_ERR_INVALID_ARG;
+    if (n_pixels >= ((size_t)1 << 40) / (size_t)c_out) return EBS_ERR_OVERFLOW;
+    return launch_dequant(acc_dev, n_pixels, c_out, scale, ch_scale_dev, ch_bias_dev, relu ? 1 : 0, y_dev,
+                          static_cast<cudaStream_t>(stream));
+}
+
+static size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+size_t ebs_host_workspace_bytes(const ebs_conv_desc* d, int n, int h, int w, int dtype, int next_a_bits) {
+    if (validate_desc(d) || n <= 0 || h <= 0 || w <= 0) return 0;
+    const int Ho = out_dim(h, d->pad_h, d->kh, d->stride_h), Wo = out_dim(w, d->pad_w, d->kw, d->stride_w);
+    if (Ho <= 0 || Wo <= 0) return 0;
+    const size_t elems_in = (size_t)n * h * w * d->c_in, outs = (size_t)n * Ho * Wo * d->c_out;
+    size_t total = round256(elems_in * (dtype == EBS_F32 ? 4 : 1));
+    total += round256(ebs_packed_act_bytes(n, h, w, d->c_in, d->a_bits));
+    total += round256(outs * 4) * 2;                                   // acc and y
+    if (next_a_bits >= 1 && next_a_bits <= 8) total += round256(ebs_packed_act_bytes(n, Ho, Wo, d->c_out, next_a_bits));
+    return total;
+}
+
+int ebs_conv2d_mixed_host(const void* x_host, int dtype, int layout, int n, int h, int w, const void* packed_w_dev,
+                          const ebs_conv_desc* d, const ebs_epilogue* epi, void* workspace_dev, size_t workspace_bytes,
+                          int32_t* acc_out_host, float* y_out_host, void* packed_next_host, void* stream) {
+    int rc = validate_desc(d);
+    if (rc) return rc;
+    if (!x_host || !workspace_dev || !aligned16(workspace_dev) || n <= 0 || h <= 0 || w <= 0) return EBS_ERR_INVALID_ARG;
+    if (dtype != EBS_F32 && dtype != EBS_U8_CODES) return EBS_ERR_INVALID_ARG;
+    if (!acc_out_host && !y_out_host && !packed_next_host) return EBS_ERR_INVALID_ARG;
+    if (packed_next_host && (!epi || epi->next_a_bits < 1 || epi->next_a_bits > 8)) return EBS_ERR_INVALID_ARG;
+    const int next_bits = packed_next_host ? epi->next_a_bits : 0;
+    const size_t need = ebs_host_workspace_bytes(d, n, h, w, dtype, next_bits);
+    if (need == 0 || workspace_bytes < need) return EBS_ERR_INVALID_ARG;
+    const int Ho = out_dim(h, d->pad_h, d->kh, d->stride_h), Wo = out_dim(w, d->pad_w, d->kw, d->stride_w);
+    const size_t elems_in = (size_t)n * h * w * d->c_in, outs = (size_t)n * Ho * Wo * d->c_out;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    char* ws = static_cast<char*>(workspace_dev);
+    void* x_dev = ws;                 ws += round256(elems_in * (dtype == EBS_F32 ? 4 : 1));
+    void* px_dev = ws;                ws += round256(ebs_packed_act_bytes(n, h, w, d->c_in, d->a_bits));
+    int32_t* acc_dev = (int32_t*)ws;  ws += round256(outs * 4);
+    float* y_dev = (float*)ws;        ws += round256(outs * 4);
+    void* pn_dev = ws;
+
+    rc = check_cuda(cudaMemcpyAsync(x_dev, x_host, elems_in * (dtype == EBS_F32 ? 4 : 1), cudaMemcpyHostToDevice, st));
+    if (rc) return rc;
+    rc = ebs_pack_acts(x_dev, dtype, layout, n, d->c_in, h, w, d->a_bits, d->a_scale, px_dev, stream);
+    if (rc) return rc;
+    rc = conv_impl(px_dev, n, h, w, packed_w_dev, d, epi, acc_out_host ? acc_dev : nullptr,
+                   y_out_host ? y_dev : nullptr, packed_next_host ? pn_dev : nullptr, stream, -1);
+    if (rc) return rc;
+    if (acc_out_host) {
+        rc = check_cuda(cudaMemcpyAsync(acc_out_host, acc_dev, outs * 4, cudaMemcpyDeviceToHost, st));
+        if (rc) return rc;
+    }
+    if (y_out_host) {
+        rc = check_cuda(cudaMemcpyAsync(y_out_host, y_dev, outs * 4, cudaMemcpyDeviceToHost, st));
+        if (rc) return rc;
+    }
+    if (packed_next_host) {
+        rc = check_cuda(cudaMemcpyAsync(packed_next_host, pn_dev, ebs_packed_act_bytes(n, Ho, Wo, d->c_out, next_bits),
+                                        cudaMemcpyDeviceToHost, st));
+        if (rc) return rc;
+    }
+    return EBS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,6 @@
+// Popcount-path convolution kernels for 5-bit weights (all activation bitwidths, all tile families).
+#include "conv_popc.cuh"
+
+namespace ebs {
+EBS_DEFINE_WB_TABLE(5)
+}  // namespace ebs

@@ -1,0 +1,57 @@
+// Stand-alone de-quantization of int32 accumulators (the "de-quantize process" of Eq. 1c and the
+// scale merge of Sec. 4.3).  Pure streaming: 4 bytes read + 4 bytes written per element.
+#include "ebs_internal.cuh"
+
+namespace ebs {
+
+__device__ __forceinline__ float dequant_one(int a, int co, float scale, const float* __restrict__ ch_scale,
+                                             const float* __restrict__ ch_bias, int relu) {
+    float y = __fmul_rn((float)a, scale);
+    if (ch_scale) y = __fmul_rn(y, __ldg(ch_scale + co));
+    if (ch_bias) y = __fadd_rn(y, __ldg(ch_bias + co));
+    if (relu && !(y > 0.0f)) y = 0.0f;
+    return y;
+}
+
+// VEC = 4: c_out % 4 == 0, so a 16-byte vector never straddles a pixel and its channels are co..co+3.
+template <int VEC>
+__global__ void __launch_bounds__(256) dequant_kernel(const int32_t* __restrict__ acc, size_t total, int c_out,
+                                                      float scale, const float* __restrict__ ch_scale,
+                                                      const float* __restrict__ ch_bias, int relu,
+                                                      float* __restrict__ y) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    if constexpr (VEC == 4) {
+        const size_t nvec = total / 4;
+        for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += stride) {
+            const int4 a = __ldg(reinterpret_cast<const int4*>(acc) + v);
+            const int co = (int)((v * 4) % (size_t)c_out);
+            float4 o;
+            o.x = dequant_one(a.x, co, scale, ch_scale, ch_bias, relu);
+            o.y = dequant_one(a.y, co + 1, scale, ch_scale, ch_bias, relu);
+            o.z = dequant_one(a.z, co + 2, scale, ch_scale, ch_bias, relu);
+            o.w = dequant_one(a.w, co + 3, scale, ch_scale, ch_bias, relu);
+            reinterpret_cast<float4*>(y)[v] = o;
+        }
+    } else {
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride)
+            y[i] = dequant_one(acc[i], (int)(i % (size_t)c_out), scale, ch_scale, ch_bias, relu);
+    }
+}
+
+int launch_dequant(const int32_t* acc, size_t n_pixels, int c_out, float scale, const float* ch_scale,
+                   const float* ch_bias, int relu, float* y, cudaStream_t st) {
+    const size_t total = n_pixels * (size_t)c_out;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const bool vec = (c_out % 4) == 0;
+    const size_t work = vec ? total / 4 : total;
+    size_t blocks = (work + 255) / 256;
+    const size_t cap = (size_t)sms * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    if (vec) dequant_kernel<4><<<(int)blocks, 256, 0, st>>>(acc, total, c_out, scale, ch_scale, ch_bias, relu, y);
+    else dequant_kernel<1><<<(int)blocks, 256, 0, st>>>(acc, total, c_out, scale, ch_scale, ch_bias, relu, y);
+    return check_cuda(cudaGetLastError());
+}
+
+}  // namespace ebs

@@ -1,0 +1,72 @@
+// Internal declarations shared by the translation units of libebs (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ebs.h"
+
+namespace ebs {
+
+// Everything the convolution kernels need, passed by value as a kernel argument.
+struct ConvParams {
+    const uint32_t* __restrict__ x;   // packed activations [N][H][W][CW][AB]
+    const uint32_t* __restrict__ w;   // packed weights     [kh][kw][CW][Co][WB]
+    int N, H, W, CW;
+    int Co, Ho, Wo, CWo;              // CWo = ceil(Co/32)
+    int kh, kw, sh, sw, ph, pw;
+    int KK;                           // kh*kw*CW reduction words per plane pair
+    int P;                            // N*Ho*Wo output pixels
+    int32_t* __restrict__ acc;        // nullable, [P][Co]
+    float* __restrict__ y;            // nullable
+    uint32_t* __restrict__ packed_next;  // nullable, [P][CWo][next_bits]
+    float S;                          // fl32(w_scale * a_scale)
+    const float* __restrict__ ch_scale;
+    const float* __restrict__ ch_bias;
+    const float* __restrict__ residual;
+    int relu;
+    int next_bits;
+    float inv_next;
+    int y_nchw;
+};
+
+// One instantiation of the popcount kernel: launch function + its tile geometry.
+struct ConvVariant {
+    void (*launch)(const ConvParams&, dim3 grid, cudaStream_t);
+    int tile_p, tile_c, threads;
+};
+
+// Number of tile variants per (w_bits, a_bits); see VariantGeom in conv_popc.cuh.
+enum { NUM_CONV_VARIANTS = 10, CONV_VARIANT_SMALL = 9 };
+
+// Filled by the per-bitwidth translation units (conv_popc_w1.cu .. conv_popc_w8.cu).
+const ConvVariant* conv_popc_variant(int w_bits, int a_bits, int variant);
+#define EBS_DECLARE_WB(WB) const ConvVariant* conv_popc_variant_w##WB(int a_bits, int variant);
+EBS_DECLARE_WB(1) EBS_DECLARE_WB(2) EBS_DECLARE_WB(3) EBS_DECLARE_WB(4)
+EBS_DECLARE_WB(5) EBS_DECLARE_WB(6) EBS_DECLARE_WB(7) EBS_DECLARE_WB(8)
+#undef EBS_DECLARE_WB
+
+// pack.cu
+int launch_pack_acts(const void* x, int dtype, int layout, int n, int c, int h, int w, int a_bits,
+                     float inv_scale, uint32_t* out, cudaStream_t st);
+int launch_pack_weights(const void* wt, int dtype, int layout, const ebs_conv_desc& d, float inv_scale,
+                        uint32_t* out, cudaStream_t st);
+// dequant.cu
+int launch_dequant(const int32_t* acc, size_t n_pixels, int c_out, float scale, const float* ch_scale,
+                   const float* ch_bias, int relu, float* y, cudaStream_t st);
+
+// Records a CUDA error for ebs_last_cuda_error() and returns EBS_ERR_CUDA (or EBS_OK).
+int check_cuda(cudaError_t e);
+
+// quantize_b of Eq. 1c in code form: round half up, every fp32 operation rounded on its own.
+__device__ __forceinline__ int quantize_code(float x, float inv_scale, int lo, int hi) {
+    float v = __fmul_rn(x, inv_scale);
+    float f = floorf(__fadd_rn(v, 0.5f));
+    int q;
+    if (!(f >= (float)lo)) q = lo;       // NaN lands here too
+    else if (f > (float)hi) q = hi;
+    else q = (int)f;
+    return q;
+}
+
+}  // namespace ebs
