@@ -1,0 +1,355 @@
+#!/usr/bin/env python
+"""Benchmark of the bit-plane mixed-precision convolution path on the CIFAR ResNet-20 stack.
+
+A step is one pass of the whole path over one batch of 128 synthetic images: for each of the 20
+quantized convolution layers, activation quantize+pack (ebs_pack_acts), the bit-plane convolution
+with fused epilogue writing int32 accumulators and the next layer's packed planes
+(ebs_conv2d_mixed), and the stand-alone de-quantization (ebs_dequant).  Weight packing is done once
+before timing (it is off the inference path).  Prints one JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from workloads import gen  # noqa: E402
+
+METRIC = "effective binary TOPS (2*MACs*Wb*Ab per second), ResNet-20 CIFAR quantized conv stack"
+UNIT = "TOPS"
+WORKLOAD = "config2: ResNet-20 CIFAR-shaped stack, 20 quantized convs, batch 128, (Wb,Ab) in {1..4}^2, seed 0"
+SM_COUNT, POPC_LANES_PER_CLK_SM = 148, 16
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+def popc_pipe_peak_tops(sm_max_mhz: float) -> float:
+    """Binary TOPS of the POPC pipe: 16 lanes/clk/SM x 32 bit x 148 SMs x clock, 2 ops per bit pair."""
+    return 2.0 * SM_COUNT * POPC_LANES_PER_CLK_SM * 32 * sm_max_mhz * 1e6 / 1e12
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        super().__init__(daemon=True)
+        self.index, self.period, self.samples, self.reasons, self.max_mhz = index, period_s, [], set(), None
+        self._stop_evt = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or nv.nvmlDeviceGetCurrentClocksThrottleReasons
+                mask = get(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------- GPU arm
+
+class Layer:
+    """Device buffers and descriptors of one layer (plumbing only)."""
+
+    def __init__(self, ebs, spec, next_bits, dev):
+        L = spec.layer
+        self.spec, self.n, self.next_bits = spec, spec.batch, next_bits
+        self.d = ebs.conv_desc(L.c_in, L.c_out, L.k, L.k, L.stride, L.stride, L.pad, L.pad, spec.w_bits, spec.a_bits,
+                               spec.w_scale, spec.a_scale)
+        qa = gen.act_codes(spec).astype(np.uint8)
+        self.x_host = torch.from_numpy(np.ascontiguousarray(qa.transpose(0, 2, 3, 1))).pin_memory()   # NHWC codes
+        self.x = self.x_host.to(dev)
+        qw = torch.from_numpy(gen.weight_codes(spec).astype(np.int8)).to(dev)
+        self.pw = torch.empty(ebs.ebs_packed_weight_bytes(self.d) // 4, dtype=torch.int32, device=dev)
+        ebs.ebs_pack_weights(qw, ebs.EBS_I8_CODES, ebs.EBS_NCHW, self.d, self.pw)
+        self.px = torch.empty(ebs.ebs_packed_act_bytes(self.n, L.h_in, L.w_in, L.c_in, spec.a_bits) // 4,
+                              dtype=torch.int32, device=dev)
+        ho, wo = L.h_out, L.w_out
+        self.pixels = self.n * ho * wo
+        self.acc = torch.empty((self.n, ho, wo, L.c_out), dtype=torch.int32, device=dev)
+        self.y = torch.empty((self.n, ho, wo, L.c_out), dtype=torch.float32, device=dev)
+        self.pn_bytes = ebs.ebs_packed_act_bytes(self.n, ho, wo, L.c_out, next_bits)
+        self.pn = torch.empty(self.pn_bytes // 4, dtype=torch.int32, device=dev)
+        self.pn_host = torch.empty(self.pn_bytes // 4, dtype=torch.int32).pin_memory()
+        self.epi = ebs.epilogue(relu=True, next_a_bits=next_bits, next_a_scale=4.0 * spec.w_scale * spec.a_scale * L.c_in)
+        self.S = float(np.float32(spec.w_scale) * np.float32(spec.a_scale))
+        self.ops = gen.binary_ops(spec)
+        self.ws_bytes = ebs.ebs_host_workspace_bytes(self.d, self.n, L.h_in, L.w_in, ebs.EBS_U8_CODES, next_bits)
+
+    def run(self, ebs):
+        L = self.spec.layer
+        ebs.ebs_pack_acts(self.x, ebs.EBS_U8_CODES, ebs.EBS_NHWC, self.n, L.c_in, L.h_in, L.w_in, self.spec.a_bits,
+                          self.spec.a_scale, self.px)
+        ebs.ebs_conv2d_mixed(self.px, self.n, L.h_in, L.w_in, self.pw, self.d, self.epi, self.acc, None, self.pn)
+        ebs.ebs_dequant(self.acc, self.pixels, L.c_out, self.S, None, None, True, self.y)
+
+    def run_conv_only(self, ebs):
+        L = self.spec.layer
+        ebs.ebs_conv2d_mixed(self.px, self.n, L.h_in, L.w_in, self.pw, self.d, self.epi, self.acc, None, self.pn)
+
+    def run_host(self, ebs, ws):
+        L = self.spec.layer
+        ebs.ebs_conv2d_mixed_host(self.x_host, ebs.EBS_U8_CODES, ebs.EBS_NHWC, self.n, L.h_in, L.w_in, self.pw, self.d,
+                                  self.epi, ws, None, None, self.pn_host)
+
+
+def dist_setup(n_gpus: int):
+    """One process per GPU under torchrun; returns (rank, world, local_rank)."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        if not dist.is_initialized():
+            dist.init_process_group(backend=backend)
+        return dist.get_rank(), world, int(os.environ.get("LOCAL_RANK", "0"))
+    return 0, 1, 0
+
+
+def max_over_ranks(value: float, device=None) -> float:
+    """MAX all-reduce of a scalar (the only collective: the data path itself shards with none)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device if dist.get_backend() == "nccl" else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.barrier()
+
+
+class OracleWorkload:
+    """The CPU oracle on (a batch slice of) the same workload; codes are generated outside the timing."""
+
+    def __init__(self, batch: int):
+        import oracle
+        oracle.build()
+        self.oracle, self.batch = oracle, batch
+        self.specs = [s for s in gen.config2(0) if s.layer.quantized]
+        self.data = [(gen.act_codes(s, batch=batch), gen.weight_codes(s)) for s in self.specs]
+        self.ops = sum(gen.binary_ops(s, batch=batch) for s in self.specs)
+
+    def step(self) -> float:
+        t0 = time.perf_counter()
+        for s, (qa, qw) in zip(self.specs, self.data):
+            L = s.layer
+            acc = self.oracle.conv2d_codes(qa, qw, (L.stride, L.stride), (L.pad, L.pad))
+            self.oracle.epilogue(acc, self.oracle.combined_scale(s.w_scale, s.a_scale), relu=True)
+        return time.perf_counter() - t0
+
+
+def oracle_batch_for(budget_s: float, n_steps: int) -> int:
+    """Largest batch (<= 128) for which n_steps oracle passes fit the time budget."""
+    probe = OracleWorkload(2)
+    probe.step()
+    per_image = probe.step() / 2
+    return int(max(1, min(128, budget_s / max(n_steps, 1) / per_image)))
+
+
+def cpu_baseline_sample(budget_s: float = 15.0):
+    """The oracle, as it stands, timed on this host's cores on a bounded sample (a reported baseline)."""
+    wl = OracleWorkload(oracle_batch_for(budget_s, 3))
+    wl.step()
+    times = [wl.step() for _ in range(2)]
+    dt = float(np.mean(times))
+    return {"value": wl.ops / dt / 1e12, "unit": UNIT, "cores": wl.oracle.num_threads(), "kind": "oracle",
+            "sample": f"all 20 quantized layers at batch {wl.batch} of 128 (direct integer conv + fp32 epilogue), "
+                      f"mean of 2 passes of {dt:.2f} s"}
+
+
+def run_reference(args):
+    rank, world, _ = dist_setup(args.gpus)
+    if rank != 0:
+        return
+    wl = OracleWorkload(oracle_batch_for(150.0, args.steps + args.warmup))
+    for _ in range(args.warmup):
+        wl.step()
+    times = [wl.step() for _ in range(args.steps)]
+    dt = float(np.mean(times))
+    value = wl.ops / dt / 1e12
+    base = {"value": value, "unit": UNIT, "cores": wl.oracle.num_threads(), "kind": "oracle",
+            "sample": f"each step: all 20 quantized layers at batch {wl.batch} of 128"}
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample_batch": wl.batch},
+            "cpu_baseline": base,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def run_gpu(args):
+    from paper_2003_07577_b200 import binding as ebs
+    ebs.lib()
+    rank, world, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    peaks, peak_kind = measured_peaks()
+
+    specs = [s for s in gen.config2(0) if s.layer.quantized]        # every rank: one full batch (weak scaling)
+    if args.only:                                                   # profiling aid: a subset of the layers
+        specs = [s for s in specs if s.layer.name in args.only.split(",")]
+    layers = [Layer(ebs, s, specs[(i + 1) % len(specs)].a_bits, dev) for i, s in enumerate(specs)]
+    ws = torch.empty(max(L.ws_bytes for L in layers), dtype=torch.uint8, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
+    total_ops = sum(L.ops for L in layers)
+    stream = torch.cuda.current_stream()
+
+    def one_step():
+        for L in layers:
+            L.run(ebs)
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    wall0 = time.perf_counter()
+    for e0, e1 in ev:
+        flush.zero_()                                               # cold L2 for every timed step
+        e0.record(stream)
+        one_step()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - wall0
+    barrier()
+    step_ms = [e0.elapsed_time(e1) for e0, e1 in ev]
+    total_ms = max_over_ranks(float(sum(step_ms)), dev)
+    ms_per_step = total_ms / args.steps
+
+    # dominant kernel (the bit-plane convolution) alone: events around each launch, cold L2 per step
+    conv_ms = np.zeros(len(layers))
+    reps = max(3, min(args.steps, 20))
+    for _ in range(reps):
+        flush.zero_()
+        pairs = []
+        for L in layers:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            L.run_conv_only(ebs)
+            b.record(stream)
+            pairs.append((a, b))
+        torch.cuda.synchronize()
+        conv_ms += np.array([a.elapsed_time(b) for a, b in pairs])
+    clocks = sampler.stop()
+    conv_ms /= reps
+    conv_total_ms = float(conv_ms.sum())
+
+    # end to end through the host entry point: pinned host codes in, packed planes out, every step
+    e2e_steps = max(3, min(args.steps, 10))
+    for L in layers:
+        L.run_host(ebs, ws)
+    torch.cuda.synchronize()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        for L in layers:
+            L.run_host(ebs, ws)
+        torch.cuda.synchronize()
+    e2e_s = max_over_ranks(time.perf_counter() - t0, dev) / e2e_steps
+
+    if rank != 0:
+        return
+    sm_max = float(clocks.get("sm_max_mhz") or peaks.get("sm_max_mhz", 1965.0))
+    peak_tops = popc_pipe_peak_tops(sm_max)
+    achieved = total_ops / (conv_total_ms * 1e-3) / 1e12
+    per_layer = [{"name": L.spec.layer.name, "wb": L.spec.w_bits, "ab": L.spec.a_bits, "us": round(float(t) * 1e3, 2),
+                  "tops": round(L.ops / (t * 1e-3) / 1e12, 2), "frac": round(L.ops / (t * 1e-3) / 1e12 / peak_tops, 3)}
+                 for L, t in zip(layers, conv_ms)]
+    cpu = cpu_baseline_sample() if world == 1 and not args.no_cpu_baseline else None
+    line = {
+        "metric": METRIC, "value": world * total_ops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": WORKLOAD + (f" [only {args.only}]" if args.only else ""), "global_batch": 128 * world, "imgs_per_s": world * 128 / (ms_per_step * 1e-3),
+                   "l2": "256 MB buffer rewritten before every timed step (cold L2)",
+                   "step": "per layer: ebs_pack_acts(u8 NHWC) + ebs_conv2d_mixed(acc + packed_next) + ebs_dequant",
+                   "parallelism": f"dp{world} (batch replicas, no data-path collective)"},
+        "clocks": clocks,
+        "e2e": {"value": world * total_ops / e2e_s / 1e12, "unit": UNIT,
+                "h2d_bytes_per_step": int(sum(L.x_host.numel() for L in layers)),
+                "d2h_bytes_per_step": int(sum(L.pn_bytes for L in layers)),
+                "note": "ebs_conv2d_mixed_host per layer: pinned u8 codes in, packed next-layer planes out; wall clock"},
+        "gpu_launches": 3 * len(layers) * args.steps,
+        "roofline": {"bound": "alu", "kernel": "conv_popc_kernel", "achieved": achieved, "peak": peak_tops,
+                     "unit": "TOPS (binary)", "frac": achieved / peak_tops, "traffic": None,
+                     "peak_source": f"POPC pipe: 148 SMs x 16 lanes/clk x 32 bit x {sm_max:.0f} MHz x 2 ops",
+                     "conv_ms_per_step": conv_total_ms, "hbm_peak_gbs": peaks.get("hbm_gbs"), "hbm_peak_kind": peak_kind,
+                     "per_layer": per_layer},
+        "wall_s_timed_region": wall,
+    }
+    if cpu is not None:
+        line["cpu_baseline"] = cpu
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default="", help="comma-separated layer names: restrict the step to these layers (for profiling)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
