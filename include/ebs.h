@@ -51,7 +51,8 @@ typedef enum ebs_status {
     EBS_ERR_UNSUPPORTED = -2, /* valid request this build has no kernel for */
     EBS_ERR_OVERFLOW = -3,    /* c_in*kh*kw*2^(w_bits-1)*(2^a_bits-1) >= 2^31, or an index would overflow */
     EBS_ERR_CUDA = -4,        /* a CUDA runtime call failed (launch error, bad device pointer, ...) */
-    EBS_ERR_TIMEOUT = -5      /* a bounded device-side wait gave up (reserved) */
+    EBS_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (reserved) */
+    EBS_ERR_SCRATCH_TOO_SMALL = -6 /* the request needs more than the built-in scratch of the no-allocation call */
 } ebs_status;
 
 typedef enum ebs_layout {
@@ -190,6 +191,34 @@ int ebs_conv2d_mixed_host(const void *x_host, int dtype, int layout, int n, int 
                           const void *packed_w_dev, const ebs_conv_desc *desc, const ebs_epilogue *epi,
                           void *workspace_dev, size_t workspace_bytes, int32_t *acc_out_host,
                           float *y_out_host, void *packed_next_host, void *stream);
+
+/*
+ * ebs_conv2d_mixed_host for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this is an integration aid.)  Some hosts of this library are not allowed to call
+ * cudaMalloc at all: code running inside a framework whose memory pool owns the whole device,
+ * plug-ins that are handed a context with a fixed memory budget, real-time loops in which an
+ * allocation could block or fail.  They cannot supply the `workspace_dev` scratch the ordinary
+ * host call wants.  This variant takes the same arguments without the workspace and keeps the
+ * scratch in a fixed array of EBS_NOALLOC_SCRATCH_BYTES (32 MiB) that is part of the library
+ * image: every GPU context that loads the library holds those bytes until the process exits.
+ *  - It calls no allocating routine (no cudaMalloc / cudaFree, no library that allocates).
+ *  - A layer whose ebs_host_workspace_bytes(...) exceeds EBS_NOALLOC_SCRATCH_BYTES is rejected with
+ *    EBS_ERR_SCRATCH_TOO_SMALL before anything is enqueued; ebs_noalloc_scratch_bytes() returns the limit.
+ *  - The first call on each device looks up the device address of the array (a one-time,
+ *    synchronous runtime query made with that device current); make that first call outside any
+ *    stream capture.  Later calls on that device only enqueue work.
+ *  - All calls on a device share the one array, and it keeps whatever the previous call left in
+ *    it.  Every byte the path reads is written earlier in the same call, so nothing needs to be
+ *    cleared; but two calls whose GPU work overlaps (different streams, or the same stream from
+ *    two threads) race on it.  Run them one after the other on one stream.
+ * Inputs, outputs, epilogue and results are exactly those of ebs_conv2d_mixed_host.
+ */
+#define EBS_NOALLOC_SCRATCH_BYTES (32u << 20)
+size_t ebs_noalloc_scratch_bytes(void);
+int ebs_conv2d_mixed_host_noalloc(const void *x_host, int dtype, int layout, int n, int h, int w,
+                                  const void *packed_w_dev, const ebs_conv_desc *desc, const ebs_epilogue *epi,
+                                  int32_t *acc_out_host, float *y_out_host, void *packed_next_host,
+                                  void *stream);
 
 /*
  * Register-resident throughput probe of the execution pipes the convolution can use; the

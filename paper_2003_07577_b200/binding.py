@@ -17,6 +17,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libebs.so")
 
 EBS_OK, EBS_ERR_INVALID_ARG, EBS_ERR_UNSUPPORTED, EBS_ERR_OVERFLOW, EBS_ERR_CUDA, EBS_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+EBS_ERR_SCRATCH_TOO_SMALL = -6
 EBS_NCHW, EBS_NHWC = 0, 1
 EBS_F32, EBS_I8_CODES, EBS_U8_CODES = 0, 1, 2
 
@@ -24,7 +25,7 @@ EXPORTS = [
     "ebs_version", "ebs_status_string", "ebs_last_cuda_error", "ebs_conv_out_shape", "ebs_packed_weight_bytes",
     "ebs_packed_act_bytes", "ebs_pack_weights", "ebs_pack_acts", "ebs_conv2d_mixed", "ebs_num_conv_variants",
     "ebs_conv2d_mixed_variant", "ebs_dequant", "ebs_host_workspace_bytes", "ebs_conv2d_mixed_host",
-    "ebs_probe_pipe",
+    "ebs_probe_pipe", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
 ]
 
 
@@ -81,6 +82,8 @@ def lib() -> ctypes.CDLL:
         L.ebs_host_workspace_bytes.restype = z
         L.ebs_conv2d_mixed_host.argtypes = [p, i, i, i, i, i, p, D, E, p, z, p, p, p, p]
         L.ebs_probe_pipe.argtypes = [i, i, ctypes.POINTER(ctypes.c_double)]
+        L.ebs_noalloc_scratch_bytes.restype = z
+        L.ebs_conv2d_mixed_host_noalloc.argtypes = [p, i, i, i, i, i, p, D, E, p, p, p, p]
         _lib = L
     return _lib
 
@@ -188,3 +191,17 @@ def ebs_probe_pipe(kind: int, iters: int = 2000) -> float:
     out = ctypes.c_double(0.0)
     _check(lib().ebs_probe_pipe(kind, iters, ctypes.byref(out)), "ebs_probe_pipe")
     return out.value
+
+
+def ebs_noalloc_scratch_bytes() -> int:
+    return lib().ebs_noalloc_scratch_bytes()
+
+
+def ebs_conv2d_mixed_host_noalloc(x_host, dtype, layout, n, h, w, packed_w_dev, desc, epi, acc_out_host=None,
+                                  y_out_host=None, packed_next_host=None, stream=None) -> None:
+    """Same as ebs_conv2d_mixed_host, for callers that may not allocate device memory: no workspace argument."""
+    e = None if epi is None else ctypes.byref(epi)
+    rc = lib().ebs_conv2d_mixed_host_noalloc(_ptr(x_host), dtype, layout, n, h, w, _ptr(packed_w_dev),
+                                             ctypes.byref(desc), e, _ptr(acc_out_host), _ptr(y_out_host),
+                                             _ptr(packed_next_host), _stream(stream))
+    _check(rc, "ebs_conv2d_mixed_host_noalloc")

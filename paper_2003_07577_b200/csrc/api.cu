@@ -142,6 +142,7 @@ const char* ebs_status_string(int status) {
         case EBS_ERR_OVERFLOW: return "accumulator or index would overflow";
         case EBS_ERR_CUDA: return "CUDA runtime error";
         case EBS_ERR_TIMEOUT: return "device-side wait timed out";
+        case EBS_ERR_SCRATCH_TOO_SMALL: return "request exceeds the built-in scratch of the no-allocation call";
         default: return "unknown status";
     }
 }
