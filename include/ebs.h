@@ -156,8 +156,10 @@ int ebs_conv2d_mixed(const void *packed_x_dev, int n, int h, int w, const void *
                      float *y_out_dev, void *packed_next_dev, void *stream);
 
 /*
- * The same call with the tile variant forced (0 .. ebs_num_conv_variants()-1) instead of chosen by
+ * The same call with the kernel variant forced (0 .. ebs_num_conv_variants()-1) instead of chosen by
  * the built-in heuristic (-1); the result is identical for every variant, only the speed differs.
+ * Variants 0..9 are the integer-pipe kernels (AND + POPC), variants 10..18 the tensor-pipe kernels
+ * (int8 MMA on bit planes expanded to bytes).
  * For tuning and for tests that must cover every kernel instantiation.  Returns
  * EBS_ERR_UNSUPPORTED if the variant cannot produce the requested packed output.
  */

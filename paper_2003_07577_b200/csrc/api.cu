@@ -28,6 +28,20 @@ const ConvVariant* conv_popc_variant(int w_bits, int a_bits, int variant) {
     }
 }
 
+const ConvVariant* conv_mma_variant(int w_bits, int a_bits, int variant) {
+    switch (w_bits) {
+        case 1: return conv_mma_variant_w1(a_bits, variant);
+        case 2: return conv_mma_variant_w2(a_bits, variant);
+        case 3: return conv_mma_variant_w3(a_bits, variant);
+        case 4: return conv_mma_variant_w4(a_bits, variant);
+        case 5: return conv_mma_variant_w5(a_bits, variant);
+        case 6: return conv_mma_variant_w6(a_bits, variant);
+        case 7: return conv_mma_variant_w7(a_bits, variant);
+        case 8: return conv_mma_variant_w8(a_bits, variant);
+        default: return nullptr;
+    }
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static int out_dim(int in, int pad, int k, int stride) {
@@ -73,6 +87,25 @@ static int choose_variant(int w_bits, int a_bits, int P, int Co, bool want_packe
     return CONV_VARIANT_SMALL;
 }
 
+// The tensor-pipe kernels keep a table of the reduction words in shared memory, masks of valid taps
+// in 32-bit words and word offsets in int: layers outside those limits use the popcount kernels.
+static bool mma_path_supported(const ConvParams& p, const ebs_conv_desc* d) {
+    const long long x_words = (long long)p.N * p.H * p.W * p.CW * d->a_bits;
+    return p.KK <= CONV_MMA_MAX_KK && d->kh <= 32 && d->kw <= 32 && x_words < (1LL << 31);
+}
+
+// Tensor-pipe variant: tile_c from c_out; the largest warp tile that still gives every SM about a
+// dozen warps (smaller layers need more, smaller tiles to hide latency).
+static int choose_mma_variant(int w_bits, int a_bits, int P, int Co, int sms) {
+    const int tc_idx = Co <= 16 ? 0 : (Co <= 32 ? 1 : 2);
+    for (int cls = 0; cls < 2; ++cls) {
+        const ConvVariant* v = conv_mma_variant(w_bits, a_bits, cls * 3 + tc_idx);
+        const long long ctas = (long long)((P + v->tile_p - 1) / v->tile_p) * ((Co + v->tile_c - 1) / v->tile_c);
+        if (ctas * (v->threads / 32) >= 12LL * sms) return cls * 3 + tc_idx;
+    }
+    return 6 + tc_idx;
+}
+
 static int conv_impl(const void* packed_x, int n, int h, int w, const void* packed_w, const ebs_conv_desc* d,
                      const ebs_epilogue* epi, int32_t* acc_out, float* y_out, void* packed_next, void* stream,
                      int variant) {
@@ -96,7 +129,7 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
         if (epi->y_layout != EBS_NCHW && epi->y_layout != EBS_NHWC) return EBS_ERR_INVALID_ARG;
         if (!aligned16(epi->residual_dev)) return EBS_ERR_INVALID_ARG;
     }
-    if (variant >= NUM_CONV_VARIANTS) return EBS_ERR_INVALID_ARG;
+    if (variant >= NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS) return EBS_ERR_INVALID_ARG;
 
     ConvParams p;
     memset(&p, 0, sizeof(p));
@@ -116,8 +149,15 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
         p.y_nchw = epi->y_layout == EBS_NCHW;
         if (packed_next) { p.next_bits = epi->next_a_bits; p.inv_next = 1.0f / epi->next_a_scale; }
     }
-    if (variant < 0) variant = choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
-    const ConvVariant* v = conv_popc_variant(d->w_bits, d->a_bits, variant);
+    const bool mma_ok = mma_path_supported(p, d);
+    if (variant < 0) {
+        variant = mma_ok ? NUM_CONV_VARIANTS + choose_mma_variant(d->w_bits, d->a_bits, p.P, p.Co, sm_count())
+                         : choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
+    }
+    if (variant >= NUM_CONV_VARIANTS && !mma_ok) return EBS_ERR_UNSUPPORTED;
+    const ConvVariant* v = variant >= NUM_CONV_VARIANTS
+                               ? conv_mma_variant(d->w_bits, d->a_bits, variant - NUM_CONV_VARIANTS)
+                               : conv_popc_variant(d->w_bits, d->a_bits, variant);
     if (!v) return EBS_ERR_UNSUPPORTED;
     if (packed_next && (v->tile_c % 32) != 0 && v->tile_c < p.Co) return EBS_ERR_UNSUPPORTED;
     const long long gx = (P + v->tile_p - 1) / v->tile_p, gy = (p.Co + v->tile_c - 1) / v->tile_c;
@@ -202,7 +242,7 @@ int ebs_conv2d_mixed(const void* packed_x_dev, int n, int h, int w, const void* 
                      stream, -1);
 }
 
-int ebs_num_conv_variants(void) { return NUM_CONV_VARIANTS; }
+int ebs_num_conv_variants(void) { return NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS; }
 
 int ebs_conv2d_mixed_variant(const void* packed_x_dev, int n, int h, int w, const void* packed_w_dev,
                              const ebs_conv_desc* desc, const ebs_epilogue* epi, int32_t* acc_out_dev,

@@ -1,0 +1,400 @@
+// Implicit-GEMM bit-plane convolution on the int8 tensor pipe (mma.sync m16n8k32), sm_100a.
+//
+// sm_100a has no native 1-bit AND+POPC matrix instruction: the toolchain expands
+// mma.sync...b1.and.popc into ~110 instructions that turn bits into bytes and issue eight int8
+// MMAs.  This kernel does that expansion itself, once per operand fragment instead of once per
+// MMA: a bit plane is turned into bytes that are 0 where the bit is clear and the plane's
+// coefficient where it is set (2^k for activation plane k, 2^m for weight plane m, -2^(M-1) for the
+// top weight plane), so that one int8 MMA of activation plane k against weight plane m adds
+// c_m 2^(m+k) * bitcount(AND(plane k, plane m)) -- stage 1 (Eq. 13) and stage 2 (Eq. 14) of the
+// binary decomposition at once -- into ONE int32 accumulator per output.  Every plane pair is still
+// its own binary contraction (M*K MMAs per 32 reduction bits); the matrix P never exists.
+//
+// Fragments are built in registers straight from the packed 32-bit words: thread (g, tq) of a warp
+// owns reduction bits {8b + tq, 8b + 4 + tq : b = 0..3} of a word, so "rotate right by (tq - k), AND
+// with 0x01010101 << k" yields a fragment register (two instructions per register).  The same bit
+// assignment is used for both operands, which is all the MMA needs.
+//
+// Work split: a CTA owns TILE_P consecutive output pixels x TILE_C channels; a warp owns
+// 16*MT pixels x 8*NT channels.  Packed words of KSTEP reduction words are staged with cp.async
+// (zero fill for taps outside the image), double buffered.
+#pragma once
+
+#include "ebs_internal.cuh"
+
+namespace ebs {
+
+constexpr int MMA_KTAB = 256;   // reduction words (kh*kw*CW) the in-kernel tap table can hold
+
+__device__ __forceinline__ void cp_async_bytes(void* smem_dst, const void* gsrc, int bytes, bool valid) {
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    const int src_size = valid ? bytes : 0;        // src_size 0: nothing is read, the destination is zero filled
+    if (bytes == 16)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(gsrc), "r"(src_size));
+    else if (bytes == 8)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;\n" ::"r"(dst), "l"(gsrc), "r"(src_size));
+    else
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(dst), "l"(gsrc), "r"(src_size));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+// Largest of 16/8/4 bytes that divides a run of `words` 32-bit words (and hence its alignment).
+__host__ __device__ constexpr int chunk_bytes(int words) { return (words % 4 == 0) ? 16 : ((words % 2 == 0) ? 8 : 4); }
+
+// Reads NWORDS consecutive shared-memory words whose address is aligned to chunk_bytes(NWORDS).
+template <int NWORDS>
+__device__ __forceinline__ void load_words_shared(const uint32_t* src, uint32_t (&dst)[NWORDS]) {
+    if constexpr (NWORDS % 4 == 0) {
+#pragma unroll
+        for (int v = 0; v < NWORDS / 4; ++v) {
+            const uint4 t = reinterpret_cast<const uint4*>(src)[v];
+            dst[4 * v] = t.x; dst[4 * v + 1] = t.y; dst[4 * v + 2] = t.z; dst[4 * v + 3] = t.w;
+        }
+    } else if constexpr (NWORDS % 2 == 0) {
+#pragma unroll
+        for (int v = 0; v < NWORDS / 2; ++v) {
+            const uint2 t = reinterpret_cast<const uint2*>(src)[v];
+            dst[2 * v] = t.x; dst[2 * v + 1] = t.y;
+        }
+    } else {
+#pragma unroll
+        for (int v = 0; v < NWORDS; ++v) dst[v] = src[v];
+    }
+}
+
+__device__ __forceinline__ void mma_u8s8(int (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+template <int WB, int AB, int MT, int NT, int WARPS_P, int WARPS_C>
+struct MmaTile {
+    static constexpr int NTHREADS = 32 * WARPS_P * WARPS_C;
+    static constexpr int TILE_P = 16 * MT * WARPS_P;
+    static constexpr int TILE_C = 8 * NT * WARPS_C;
+    static constexpr int KW_WORDS = TILE_P * AB + TILE_C * WB;          // words per staged reduction word
+    static constexpr int KSTEP_RAW = 2048 / KW_WORDS;                    // about 8 KB per stage
+    static constexpr int KSTEP = KSTEP_RAW < 1 ? 1 : (KSTEP_RAW > 8 ? 8 : KSTEP_RAW);
+    static constexpr int STAGE_WORDS = KSTEP * KW_WORDS;
+    static constexpr int OUT_WORDS = TILE_P * TILE_C / 4;
+    static constexpr int SMEM_WORDS = 2 * STAGE_WORDS > OUT_WORDS ? 2 * STAGE_WORDS : OUT_WORDS;
+    static constexpr int PPT = TILE_P > NTHREADS ? TILE_P / NTHREADS : 1;       // pixels staged per thread
+    static constexpr int QSTRIDE = NTHREADS > TILE_P ? NTHREADS / TILE_P : 1;   // threads sharing a pixel
+    static_assert(TILE_P % NTHREADS == 0 || NTHREADS % TILE_P == 0, "staging map needs a power-of-two ratio");
+    static_assert(SMEM_WORDS * 4 + MMA_KTAB * 8 <= 47 * 1024, "static shared memory budget");
+};
+
+template <int WB, int AB, int MT, int NT, int WARPS_P, int WARPS_C>
+__global__ void __launch_bounds__(32 * WARPS_P * WARPS_C)
+conv_mma_kernel(const ConvParams p) {
+    using T = MmaTile<WB, AB, MT, NT, WARPS_P, WARPS_C>;
+    constexpr int NTH = T::NTHREADS, TILE_P = T::TILE_P, TILE_C = T::TILE_C, KSTEP = T::KSTEP;
+    constexpr int PPT = T::PPT, QSTRIDE = T::QSTRIDE;
+    constexpr int A_CH = chunk_bytes(AB), W_CH = chunk_bytes(WB);
+
+    __shared__ __align__(16) uint32_t smem[T::SMEM_WORDS];
+    __shared__ int2 ktab[MMA_KTAB];            // per reduction word: {word offset of the tap, r | s << 8}
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, tq = lane & 3;
+    const int wp = warp % WARPS_P, wc = warp / WARPS_P;
+    const int tile_p0 = blockIdx.x * TILE_P;
+    const int co0 = blockIdx.y * TILE_C;
+
+    // ---- tap table (kk = tap * CW + cw)
+    for (int kk = tid; kk < p.KK; kk += NTH) {
+        const int tap = kk / p.CW, cw = kk - tap * p.CW;
+        const int r = tap / p.kw, s = tap - r * p.kw;
+        ktab[kk] = make_int2(((r * p.W + s) * p.CW + cw) * AB, r | (s << 8));
+    }
+
+    // ---- the pixels this thread stages: word offset of (n, h0, w0) and which taps stay inside the image
+    int pix_off[PPT];
+    uint32_t row_ok[PPT], col_ok[PPT];
+#pragma unroll
+    for (int u = 0; u < PPT; ++u) {
+        const int pl = (tid % TILE_P) + u * NTH;
+        const int gp = tile_p0 + pl;
+        pix_off[u] = 0; row_ok[u] = 0u; col_ok[u] = 0u;
+        if (gp < p.P) {
+            const int hw = p.Ho * p.Wo;
+            const int n = gp / hw, rem = gp - n * hw;
+            const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
+            const int h0 = ho * p.sh - p.ph, w0 = wo * p.sw - p.pw;
+            pix_off[u] = ((n * p.H + h0) * p.W + w0) * p.CW * AB;
+            for (int r = 0; r < p.kh; ++r) row_ok[u] |= ((unsigned)(h0 + r) < (unsigned)p.H ? 1u : 0u) << r;
+            for (int s = 0; s < p.kw; ++s) col_ok[u] |= ((unsigned)(w0 + s) < (unsigned)p.W ? 1u : 0u) << s;
+        }
+    }
+    const bool w_vec_ok = ((p.Co * WB) % (W_CH / 4)) == 0;      // weight rows keep the chunk alignment
+
+    auto stage = [&](int kk0, int buf) {
+        uint32_t* A_s = smem + buf * T::STAGE_WORDS;                       // [KSTEP][TILE_P][AB]
+        uint32_t* W_s = A_s + KSTEP * TILE_P * AB;                         // [KSTEP][TILE_C][WB]
+#pragma unroll
+        for (int qq = 0; qq < (KSTEP + QSTRIDE - 1) / QSTRIDE; ++qq) {
+            const int q = qq * QSTRIDE + (QSTRIDE > 1 ? tid / TILE_P : 0);
+            if (QSTRIDE > 1 && q >= KSTEP) break;
+            const int kk = kk0 + q;
+            const bool kvalid = kk < p.KK;
+            const int2 info = kvalid ? ktab[kk] : make_int2(0, 0);
+            const int r = info.y & 0xff, s = info.y >> 8;
+#pragma unroll
+            for (int u = 0; u < PPT; ++u) {
+                const int pl = (tid % TILE_P) + u * NTH;
+                const bool valid = kvalid && ((row_ok[u] >> r) & (col_ok[u] >> s) & 1u);
+                const uint32_t* src = valid ? p.x + (pix_off[u] + info.x) : p.x;
+                uint32_t* dst = A_s + (q * TILE_P + pl) * AB;
+#pragma unroll
+                for (int c = 0; c < AB * 4 / A_CH; ++c)
+                    cp_async_bytes(dst + c * (A_CH / 4), src + c * (A_CH / 4), A_CH, valid);
+            }
+        }
+        // weights: per reduction word a contiguous run of TILE_C*WB words (channels co0 .. co0+TILE_C)
+        if (w_vec_ok) {
+            constexpr int CHUNKS = TILE_C * WB * 4 / W_CH;
+            for (int e = tid; e < KSTEP * CHUNKS; e += NTH) {
+                const int q = e / CHUNKS, ch = e - q * CHUNKS;
+                const int word = ch * (W_CH / 4), c = word / WB;
+                const int kk = kk0 + q;
+                const bool valid = kk < p.KK && co0 + c < p.Co;
+                const uint32_t* src = valid ? p.w + ((size_t)kk * p.Co + co0) * WB + word : p.w;
+                cp_async_bytes(W_s + q * TILE_C * WB + word, src, W_CH, valid);
+            }
+        } else {
+            for (int e = tid; e < KSTEP * TILE_C * WB; e += NTH) {
+                const int q = e / (TILE_C * WB), word = e - q * (TILE_C * WB), c = word / WB;
+                const int kk = kk0 + q;
+                const bool valid = kk < p.KK && co0 + c < p.Co;
+                const uint32_t* src = valid ? p.w + ((size_t)kk * p.Co + co0) * WB + word : p.w;
+                cp_async_bytes(W_s + q * TILE_C * WB + word, src, 4, valid);
+            }
+        }
+    };
+
+    int acc[MT][NT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0;
+
+    __syncthreads();                                   // tap table ready
+    const int nsteps = (p.KK + KSTEP - 1) / KSTEP;
+    stage(0, 0);
+    cp_async_commit();
+
+    for (int st = 0; st < nsteps; ++st) {
+        const int buf = st & 1;
+        if (st + 1 < nsteps) {
+            stage((st + 1) * KSTEP, buf ^ 1);
+            cp_async_commit();
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+
+        const uint32_t* A_s = smem + buf * T::STAGE_WORDS;
+        const uint32_t* W_s = A_s + KSTEP * TILE_P * AB;
+#pragma unroll
+        for (int q = 0; q < KSTEP; ++q) {
+            if (st * KSTEP + q < p.KK) {
+                // activation fragments: byte = 2^k where bit k-plane is set
+                uint32_t af[MT][AB][4];
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    const int r0 = (wp * MT + mt) * 16 + g;
+                    const uint32_t* row0 = A_s + (q * TILE_P + r0) * AB;
+                    const uint32_t* row1 = row0 + 8 * AB;
+                    uint32_t wr0[AB], wr1[AB];
+                    load_words_shared<AB>(row0, wr0);
+                    load_words_shared<AB>(row1, wr1);
+#pragma unroll
+                    for (int k = 0; k < AB; ++k) {
+                        const uint32_t w0 = wr0[k], w1 = wr1[k];
+                        const uint32_t mask = 0x01010101u << k;
+                        af[mt][k][0] = __funnelshift_r(w0, w0, tq - k) & mask;
+                        af[mt][k][1] = __funnelshift_r(w1, w1, tq - k) & mask;
+                        af[mt][k][2] = __funnelshift_r(w0, w0, tq + 4 - k) & mask;
+                        af[mt][k][3] = __funnelshift_r(w1, w1, tq + 4 - k) & mask;
+                    }
+                }
+                // weight fragments: byte = 2^m, or -2^(WB-1) (two's complement byte) for the top plane
+                uint32_t bf[NT][WB][2];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint32_t* row = W_s + (q * TILE_C + (wc * NT + nt) * 8 + g) * WB;
+                    uint32_t wr[WB];
+                    load_words_shared<WB>(row, wr);
+#pragma unroll
+                    for (int m = 0; m < WB; ++m) {
+                        const uint32_t w = wr[m];
+                        const uint32_t mask = 0x01010101u << m;
+                        uint32_t b0 = __funnelshift_r(w, w, tq - m) & mask;
+                        uint32_t b1 = __funnelshift_r(w, w, tq + 4 - m) & mask;
+                        if (m == WB - 1 && WB < 8) {              // 2^(WB-1) * (2^(9-WB) - 1) = 256 - 2^(WB-1)
+                            b0 *= (1u << (9 - WB)) - 1u;
+                            b1 *= (1u << (9 - WB)) - 1u;
+                        }
+                        bf[nt][m][0] = b0;
+                        bf[nt][m][1] = b1;
+                    }
+                }
+#pragma unroll
+                for (int m = 0; m < WB; ++m)
+#pragma unroll
+                    for (int k = 0; k < AB; ++k)
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) mma_u8s8(acc[mt][nt], af[mt][k], bf[nt][m][0], bf[nt][m][1]);
+            }
+        }
+        __syncthreads();
+    }
+
+    // ---- epilogue.  Fragment element e of (mt, nt): pixel row (e >> 1) * 8 + g, channel 2 * tq + (e & 1).
+    const bool want_y = p.y != nullptr, want_q = p.packed_next != nullptr;
+    uint8_t* out_s = reinterpret_cast<uint8_t*>(smem);      // [TILE_P][TILE_C] requantized codes
+    const int qmax = (1 << p.next_bits) - 1;
+    const bool pair_ok = (p.Co & 1) == 0;                   // two adjacent channels form an aligned 8-byte pair
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int pl = (wp * MT + mt) * 16 + half * 8 + g;
+            const int gp = tile_p0 + pl;
+            const bool pvalid = gp < p.P;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const int cl = (wc * NT + nt) * 8 + 2 * tq, co = co0 + cl;
+                const int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
+                int code0 = 0, code1 = 0;
+                if (pvalid && co < p.Co) {
+                    const size_t o = (size_t)gp * p.Co + co;
+                    const bool two = co + 1 < p.Co;
+                    if (p.acc) {
+                        if (pair_ok) *reinterpret_cast<int2*>(p.acc + o) = make_int2(a0, a1);
+                        else { p.acc[o] = a0; if (two) p.acc[o + 1] = a1; }
+                    }
+                    if (want_y || want_q) {
+                        float y0 = __fmul_rn((float)a0, p.S), y1 = __fmul_rn((float)a1, p.S);
+                        if (p.ch_scale) {
+                            y0 = __fmul_rn(y0, __ldg(p.ch_scale + co));
+                            if (two) y1 = __fmul_rn(y1, __ldg(p.ch_scale + co + 1));
+                        }
+                        if (p.ch_bias) {
+                            y0 = __fadd_rn(y0, __ldg(p.ch_bias + co));
+                            if (two) y1 = __fadd_rn(y1, __ldg(p.ch_bias + co + 1));
+                        }
+                        if (p.residual) {
+                            y0 = __fadd_rn(y0, __ldg(p.residual + o));
+                            if (two) y1 = __fadd_rn(y1, __ldg(p.residual + o + 1));
+                        }
+                        if (p.relu) {
+                            if (!(y0 > 0.0f)) y0 = 0.0f;
+                            if (!(y1 > 0.0f)) y1 = 0.0f;
+                        }
+                        if (want_y) {
+                            if (p.y_nchw) {
+                                const int hw = p.Ho * p.Wo;
+                                const int n = gp / hw, rem = gp - n * hw;
+                                p.y[((size_t)n * p.Co + co) * hw + rem] = y0;
+                                if (two) p.y[((size_t)n * p.Co + co + 1) * hw + rem] = y1;
+                            } else if (pair_ok) {
+                                *reinterpret_cast<float2*>(p.y + o) = make_float2(y0, y1);
+                            } else {
+                                p.y[o] = y0;
+                                if (two) p.y[o + 1] = y1;
+                            }
+                        }
+                        if (want_q) {
+                            code0 = quantize_code(y0, p.inv_next, 0, qmax);
+                            if (two) code1 = quantize_code(y1, p.inv_next, 0, qmax);
+                        }
+                    }
+                }
+                if (want_q) *reinterpret_cast<uint16_t*>(out_s + pl * TILE_C + cl) = (uint16_t)(code0 | (code1 << 8));
+            }
+        }
+    }
+    if (want_q) {
+        __syncthreads();
+        constexpr int CWL = (TILE_C + 31) / 32;
+        for (int item = warp; item < TILE_P * CWL; item += NTH / 32) {
+            const int pl = item / CWL, cwl = item - pl * CWL;
+            const int gp = tile_p0 + pl;
+            if (gp >= p.P) continue;                              // uniform per warp
+            const int cl = cwl * 32 + lane;
+            const uint32_t code = (cl < TILE_C) ? out_s[pl * TILE_C + cl] : 0u;
+            const int cwg = (co0 >> 5) + cwl;
+            if (cwg >= p.CWo) continue;
+            uint32_t mine = 0u;
+            for (int j = 0; j < p.next_bits; ++j) {
+                const uint32_t word = __ballot_sync(0xffffffffu, (code >> j) & 1u);
+                if (lane == j) mine = word;
+            }
+            if (lane < p.next_bits) p.packed_next[((size_t)gp * p.CWo + cwg) * p.next_bits + lane] = mine;
+        }
+    }
+}
+
+template <int WB, int AB, int MT, int NT, int WARPS_P, int WARPS_C>
+void launch_conv_mma(const ConvParams& p, dim3 grid, cudaStream_t st) {
+    conv_mma_kernel<WB, AB, MT, NT, WARPS_P, WARPS_C><<<grid, 32 * WARPS_P * WARPS_C, 0, st>>>(p);
+}
+
+// Variants: variant = size_class * 3 + tile_c_index, tile_c in {16, 32, 64}.
+//   class 0 (large)  the biggest warp tile the plane-pair count allows (fewest fragment rebuilds), 8 warps
+//   class 1 (medium) 32 pixels x 16 channels per warp, 8 warps
+//   class 2 (small)  16 pixels x 16 channels per warp, 4 warps -- for layers that otherwise leave SMs idle
+// Every plane pair is one MMA per 16x8 output block per reduction word, so the large warp tile
+// shrinks as the pair count grows.
+template <int WB, int AB, int VARIANT>
+struct MmaGeom {
+    static constexpr int PAIRS = WB * AB;
+    static constexpr int CLASS = VARIANT / 3;
+    static constexpr int TILE_C = 16 << (VARIANT % 3);
+    static constexpr int WARPS = CLASS == 2 ? 4 : 8;
+    static constexpr int NT_PREF = (CLASS == 0 && PAIRS <= 4) ? 4 : 2;
+    static constexpr int NT = (TILE_C / 8) < NT_PREF ? (TILE_C / 8) : NT_PREF;
+    static constexpr int WARPS_C_RAW = TILE_C / (8 * NT);
+    static constexpr int WARPS_C = WARPS_C_RAW > WARPS ? WARPS : WARPS_C_RAW;
+    static constexpr int WARPS_P = WARPS / WARPS_C;
+    static constexpr int ACC_BUDGET = PAIRS == 1 ? 64 : (PAIRS <= 4 ? 32 : (PAIRS <= 16 ? 16 : 8));
+    static constexpr int MT_RAW = ACC_BUDGET / (4 * NT);
+    static constexpr int MT_AB = AB <= 2 ? 4 : (AB <= 4 ? 2 : 1);      // activation fragments: MT*AB*4 registers
+    static constexpr int MT_LARGE = MT_RAW < 1 ? 1 : (MT_RAW > MT_AB ? MT_AB : MT_RAW);
+    static constexpr int MT = CLASS == 0 ? MT_LARGE : (CLASS == 1 ? (MT_AB < 2 ? MT_AB : 2) : 1);
+};
+
+constexpr int NUM_MMA_VARIANTS = 9;
+
+template <int WB, int AB, int VARIANT>
+constexpr ConvVariant make_mma_variant() {
+    using G = MmaGeom<WB, AB, VARIANT>;
+    return ConvVariant{&launch_conv_mma<WB, AB, G::MT, G::NT, G::WARPS_P, G::WARPS_C>, 16 * G::MT * G::WARPS_P,
+                       8 * G::NT * G::WARPS_C, 32 * G::WARPS_P * G::WARPS_C};
+}
+
+#define EBS_MMA_ROW(WB, AB)                                                                             \
+    {make_mma_variant<WB, AB, 0>(), make_mma_variant<WB, AB, 1>(), make_mma_variant<WB, AB, 2>(),       \
+     make_mma_variant<WB, AB, 3>(), make_mma_variant<WB, AB, 4>(), make_mma_variant<WB, AB, 5>(),       \
+     make_mma_variant<WB, AB, 6>(), make_mma_variant<WB, AB, 7>(), make_mma_variant<WB, AB, 8>()}
+
+#define EBS_DEFINE_MMA_TABLE(WB)                                                                        \
+    const ConvVariant* conv_mma_variant_w##WB(int a_bits, int variant) {                                \
+        static const ConvVariant table[8][NUM_MMA_VARIANTS] = {                                         \
+            EBS_MMA_ROW(WB, 1), EBS_MMA_ROW(WB, 2), EBS_MMA_ROW(WB, 3), EBS_MMA_ROW(WB, 4),             \
+            EBS_MMA_ROW(WB, 5), EBS_MMA_ROW(WB, 6), EBS_MMA_ROW(WB, 7), EBS_MMA_ROW(WB, 8)};            \
+        if (a_bits < 1 || a_bits > 8 || variant < 0 || variant >= NUM_MMA_VARIANTS) return nullptr;     \
+        return &table[a_bits - 1][variant];                                                             \
+    }
+
+}  // namespace ebs

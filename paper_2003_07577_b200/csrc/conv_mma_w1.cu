@@ -1,0 +1,7 @@
+// Tensor-pipe (int8 MMA on bit planes) convolution kernels for 1-bit weights.
+#include "conv_mma.cuh"
+
+namespace ebs {
+static_assert(NUM_MMA_VARIANTS == NUM_CONV_MMA_VARIANTS && MMA_KTAB == CONV_MMA_MAX_KK, "tables out of sync");
+EBS_DEFINE_MMA_TABLE(1)
+}  // namespace ebs

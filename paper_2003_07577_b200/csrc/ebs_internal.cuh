@@ -46,6 +46,14 @@ EBS_DECLARE_WB(1) EBS_DECLARE_WB(2) EBS_DECLARE_WB(3) EBS_DECLARE_WB(4)
 EBS_DECLARE_WB(5) EBS_DECLARE_WB(6) EBS_DECLARE_WB(7) EBS_DECLARE_WB(8)
 #undef EBS_DECLARE_WB
 
+// Tensor-pipe kernels (conv_mma_w1.cu .. conv_mma_w8.cu); variant 0 .. NUM_CONV_MMA_VARIANTS-1.
+enum { NUM_CONV_MMA_VARIANTS = 9, CONV_MMA_MAX_KK = 256 };
+const ConvVariant* conv_mma_variant(int w_bits, int a_bits, int variant);
+#define EBS_DECLARE_WB(WB) const ConvVariant* conv_mma_variant_w##WB(int a_bits, int variant);
+EBS_DECLARE_WB(1) EBS_DECLARE_WB(2) EBS_DECLARE_WB(3) EBS_DECLARE_WB(4)
+EBS_DECLARE_WB(5) EBS_DECLARE_WB(6) EBS_DECLARE_WB(7) EBS_DECLARE_WB(8)
+#undef EBS_DECLARE_WB
+
 // pack.cu
 int launch_pack_acts(const void* x, int dtype, int layout, int n, int c, int h, int w, int a_bits,
                      float inv_scale, uint32_t* out, cudaStream_t st);
