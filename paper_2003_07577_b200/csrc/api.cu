@@ -143,6 +143,8 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
     p.acc = acc_out; p.y = y_out; p.packed_next = static_cast<uint32_t*>(packed_next);
     p.S = d->w_scale * d->a_scale;       // one rounded fp32 multiply
     p.next_bits = 1;
+    p.fold = d->c_in <= 4 ? 8 : (d->c_in <= 8 ? 4 : (d->c_in <= 16 ? 2 : 1));
+    p.fold_bits = 32 / p.fold;
     if (epi) {
         p.ch_scale = epi->ch_scale_dev; p.ch_bias = epi->ch_bias_dev; p.residual = epi->residual_dev;
         p.relu = epi->relu ? 1 : 0;

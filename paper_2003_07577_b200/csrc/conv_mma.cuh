@@ -15,6 +15,10 @@
 // with 0x01010101 << k" yields a fragment register (two instructions per register).  The same bit
 // assignment is used for both operands, which is all the MMA needs.
 //
+// Layers with at most 16 input channels use only the low bits of each word; there 2, 4 or 8 staged
+// taps are OR-ed into one word (shifted by 16, 8 or 4 bits) while the fragments are built, for both
+// operands alike, so a 32-bit MMA step is filled with real reduction bits.
+//
 // Work split: a CTA owns TILE_P consecutive output pixels x TILE_C channels; a warp owns
 // 16*MT pixels x 8*NT channels.  Packed words of KSTEP reduction words are staged with cp.async
 // (zero fill for taps outside the image), double buffered.
@@ -80,7 +84,7 @@ struct MmaTile {
     static constexpr int KSTEP_RAW = 2048 / KW_WORDS;                    // about 8 KB per stage
     static constexpr int KSTEP = KSTEP_RAW < 1 ? 1 : (KSTEP_RAW > 8 ? 8 : KSTEP_RAW);
     static constexpr int STAGE_WORDS = KSTEP * KW_WORDS;
-    static constexpr int OUT_WORDS = TILE_P * TILE_C / 4;
+    static constexpr int OUT_WORDS = TILE_P * code_row_bytes(TILE_C) / 4;
     static constexpr int SMEM_WORDS = 2 * STAGE_WORDS > OUT_WORDS ? 2 * STAGE_WORDS : OUT_WORDS;
     static constexpr int PPT = TILE_P > NTHREADS ? TILE_P / NTHREADS : 1;       // pixels staged per thread
     static constexpr int QSTRIDE = NTHREADS > TILE_P ? NTHREADS / TILE_P : 1;   // threads sharing a pixel
@@ -204,7 +208,7 @@ conv_mma_kernel(const ConvParams p) {
         const uint32_t* W_s = A_s + KSTEP * TILE_P * AB;
 #pragma unroll
         for (int q = 0; q < KSTEP; ++q) {
-            if (st * KSTEP + q < p.KK) {
+            if ((q & (p.fold - 1)) == 0 && st * KSTEP + q < p.KK) {
                 // activation fragments: byte = 2^k where bit k-plane is set
                 uint32_t af[MT][AB][4];
 #pragma unroll
@@ -215,6 +219,18 @@ conv_mma_kernel(const ConvParams p) {
                     uint32_t wr0[AB], wr1[AB];
                     load_words_shared<AB>(row0, wr0);
                     load_words_shared<AB>(row1, wr1);
+                    if (p.fold > 1) {                     // few input channels: several taps share one word
+                        for (int f = 1; f < p.fold && q + f < KSTEP; ++f) {
+                            uint32_t t0[AB], t1[AB];
+                            load_words_shared<AB>(row0 + f * TILE_P * AB, t0);
+                            load_words_shared<AB>(row1 + f * TILE_P * AB, t1);
+#pragma unroll
+                            for (int k = 0; k < AB; ++k) {
+                                wr0[k] |= t0[k] << (f * p.fold_bits);
+                                wr1[k] |= t1[k] << (f * p.fold_bits);
+                            }
+                        }
+                    }
 #pragma unroll
                     for (int k = 0; k < AB; ++k) {
                         const uint32_t w0 = wr0[k], w1 = wr1[k];
@@ -232,6 +248,14 @@ conv_mma_kernel(const ConvParams p) {
                     const uint32_t* row = W_s + (q * TILE_C + (wc * NT + nt) * 8 + g) * WB;
                     uint32_t wr[WB];
                     load_words_shared<WB>(row, wr);
+                    if (p.fold > 1) {
+                        for (int f = 1; f < p.fold && q + f < KSTEP; ++f) {
+                            uint32_t t[WB];
+                            load_words_shared<WB>(row + f * TILE_C * WB, t);
+#pragma unroll
+                            for (int m = 0; m < WB; ++m) wr[m] |= t[m] << (f * p.fold_bits);
+                        }
+                    }
 #pragma unroll
                     for (int m = 0; m < WB; ++m) {
                         const uint32_t w = wr[m];
@@ -261,7 +285,7 @@ conv_mma_kernel(const ConvParams p) {
 
     // ---- epilogue.  Fragment element e of (mt, nt): pixel row (e >> 1) * 8 + g, channel 2 * tq + (e & 1).
     const bool want_y = p.y != nullptr, want_q = p.packed_next != nullptr;
-    uint8_t* out_s = reinterpret_cast<uint8_t*>(smem);      // [TILE_P][TILE_C] requantized codes
+    uint8_t* out_s = reinterpret_cast<uint8_t*>(smem);      // [TILE_P][TILE_C + 4] requantized codes
     const int qmax = (1 << p.next_bits) - 1;
     const bool pair_ok = (p.Co & 1) == 0;                   // two adjacent channels form an aligned 8-byte pair
 #pragma unroll
@@ -320,28 +344,13 @@ conv_mma_kernel(const ConvParams p) {
                         }
                     }
                 }
-                if (want_q) *reinterpret_cast<uint16_t*>(out_s + pl * TILE_C + cl) = (uint16_t)(code0 | (code1 << 8));
+                if (want_q) *reinterpret_cast<uint16_t*>(out_s + pl * code_row_bytes(TILE_C) + cl) = (uint16_t)(code0 | (code1 << 8));
             }
         }
     }
     if (want_q) {
         __syncthreads();
-        constexpr int CWL = (TILE_C + 31) / 32;
-        for (int item = warp; item < TILE_P * CWL; item += NTH / 32) {
-            const int pl = item / CWL, cwl = item - pl * CWL;
-            const int gp = tile_p0 + pl;
-            if (gp >= p.P) continue;                              // uniform per warp
-            const int cl = cwl * 32 + lane;
-            const uint32_t code = (cl < TILE_C) ? out_s[pl * TILE_C + cl] : 0u;
-            const int cwg = (co0 >> 5) + cwl;
-            if (cwg >= p.CWo) continue;
-            uint32_t mine = 0u;
-            for (int j = 0; j < p.next_bits; ++j) {
-                const uint32_t word = __ballot_sync(0xffffffffu, (code >> j) & 1u);
-                if (lane == j) mine = word;
-            }
-            if (lane < p.next_bits) p.packed_next[((size_t)gp * p.CWo + cwg) * p.next_bits + lane] = mine;
-        }
+        pack_code_tile<TILE_P, TILE_C, NTH>(out_s, p, tile_p0, co0);
     }
 }
 

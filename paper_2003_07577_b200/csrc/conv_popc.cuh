@@ -46,7 +46,7 @@ struct PopcTile {
     static constexpr int KSTEP_RAW = (16 * 1024 / 4) / KK_WORDS;
     static constexpr int KSTEP = KSTEP_RAW < 1 ? 1 : (KSTEP_RAW > 8 ? 8 : KSTEP_RAW);
     static constexpr int STAGE_WORDS = KSTEP * KK_WORDS;
-    static constexpr int OUT_WORDS = TILE_P * TILE_C / 4;   // u8 codes of the tile for the packed output
+    static constexpr int OUT_WORDS = TILE_P * code_row_bytes(TILE_C) / 4;   // u8 codes of the tile for the packed output
     static constexpr int SMEM_WORDS = STAGE_WORDS > OUT_WORDS ? STAGE_WORDS : OUT_WORDS;
 };
 
@@ -203,27 +203,12 @@ conv_popc_kernel(const ConvParams p) {
                     if (want_q) code = quantize_code(yv, p.inv_next, 0, qmax);
                 }
             }
-            if (want_q) out_s[pl * TILE_C + cl] = (uint8_t)code;
+            if (want_q) out_s[pl * code_row_bytes(TILE_C) + cl] = (uint8_t)code;
         }
     }
     if (want_q) {
         __syncthreads();
-        constexpr int CWL = (TILE_C + 31) / 32;
-        for (int item = warp; item < TILE_P * CWL; item += NT / 32) {
-            const int pl = item / CWL, cwl = item - pl * CWL;
-            const int gp = tile_p0 + pl;
-            if (gp >= p.P) continue;                              // uniform per warp
-            const int cl = cwl * 32 + lane;
-            const uint32_t code = (cl < TILE_C) ? out_s[pl * TILE_C + cl] : 0u;
-            const int cwg = (co0 >> 5) + cwl;
-            if (cwg >= p.CWo) continue;
-            uint32_t mine = 0u;
-            for (int j = 0; j < p.next_bits; ++j) {
-                const uint32_t word = __ballot_sync(0xffffffffu, (code >> j) & 1u);
-                if (lane == j) mine = word;
-            }
-            if (lane < p.next_bits) p.packed_next[((size_t)gp * p.CWo + cwg) * p.next_bits + lane] = mine;
-        }
+        pack_code_tile<TILE_P, TILE_C, NT>(out_s, p, tile_p0, co0);
     }
 }
 

@@ -28,6 +28,8 @@ struct ConvParams {
     int next_bits;
     float inv_next;
     int y_nchw;
+    int fold;                         // taps OR-ed into one reduction word by the tensor-pipe kernels: 1, 2, 4, 8
+    int fold_bits;                    // 32 / fold: bits each folded tap occupies (>= c_in)
 };
 
 // One instantiation of the popcount kernel: launch function + its tile geometry.
@@ -75,6 +77,40 @@ __device__ __forceinline__ int quantize_code(float x, float inv_scale, int lo, i
     else if (f > (float)hi) q = hi;
     else q = (int)f;
     return q;
+}
+
+// Row pitch (bytes) of the tile of requantized codes kept in shared memory: 4 bytes of padding make
+// consecutive pixels start in different banks.
+__host__ __device__ constexpr int code_row_bytes(int tile_c) { return tile_c + 4; }
+
+// Packs a CTA's tile of requantized codes (one byte per output, [TILE_P][code_row_bytes(TILE_C)] in
+// shared memory) into the next layer's bit-plane words.  One thread per (pixel, 32-channel word):
+// four code bytes at a time, plane j of the four codes is gathered into a nibble with one multiply
+// ((x >> j) & 0x01010101) * 0x01020408 >> 24.
+template <int TILE_P, int TILE_C, int NTHREADS>
+__device__ __forceinline__ void pack_code_tile(const uint8_t* out_s, const ConvParams& p, int tile_p0, int co0) {
+    constexpr int ROWB = code_row_bytes(TILE_C);
+    constexpr int CWL = (TILE_C + 31) / 32;
+    constexpr int NW = TILE_C >= 32 ? 8 : TILE_C / 4;           // code words per 32-channel group
+    for (int item = threadIdx.x; item < TILE_P * CWL; item += NTHREADS) {
+        const int cwl = item / TILE_P, pl = item - cwl * TILE_P;
+        const int gp = tile_p0 + pl, cwg = (co0 >> 5) + cwl;
+        if (gp >= p.P || cwg >= p.CWo) continue;
+        const uint32_t* row = reinterpret_cast<const uint32_t*>(out_s + pl * ROWB + cwl * 32);
+        uint32_t codes[NW];
+#pragma unroll
+        for (int k = 0; k < NW; ++k) codes[k] = row[k];
+        uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + cwg) * p.next_bits;
+        for (int j = 0; j < p.next_bits; ++j) {
+            uint32_t word = 0u;
+#pragma unroll
+            for (int k = 0; k < NW; ++k) {
+                const uint32_t t = (codes[k] >> j) & 0x01010101u;
+                word |= ((t * 0x01020408u) >> 24) << (4 * k);
+            }
+            dst[j] = word;
+        }
+    }
 }
 
 }  // namespace ebs
