@@ -44,6 +44,53 @@ __global__ void __launch_bounds__(256) pack_acts_nhwc_kernel(const T* __restrict
     }
 }
 
+// NHWC integer codes: one thread per (pixel, 32-channel word).  The thread reads its 32 code bytes
+// as 16-byte vectors and gathers plane j of four codes at a time into a nibble with one multiply
+// (((x >> j) & 0x01010101) * 0x01020408) >> 24, so no cross-lane traffic is needed and a warp moves
+// 1 KB per load instruction.
+__global__ void __launch_bounds__(256) pack_acts_nhwc_u8_kernel(const uint8_t* __restrict__ x, long long items, int C,
+                                                                int CW, int AB, uint32_t* __restrict__ out) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const bool vec16 = (C % 16) == 0;
+    for (long long item = (long long)blockIdx.x * blockDim.x + threadIdx.x; item < items; item += stride) {
+        const long long pix = item / CW;
+        const int cw = (int)(item - pix * CW);
+        const int c0 = cw * 32;
+        const int nvalid = C - c0 < 32 ? C - c0 : 32;
+        const uint8_t* src = x + pix * C + c0;
+        uint32_t codes[8];
+        if (vec16) {
+            const uint4 lo = __ldg(reinterpret_cast<const uint4*>(src));
+            codes[0] = lo.x; codes[1] = lo.y; codes[2] = lo.z; codes[3] = lo.w;
+            if (nvalid > 16) {
+                const uint4 hi = __ldg(reinterpret_cast<const uint4*>(src) + 1);
+                codes[4] = hi.x; codes[5] = hi.y; codes[6] = hi.z; codes[7] = hi.w;
+            } else {
+                codes[4] = codes[5] = codes[6] = codes[7] = 0u;
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                uint32_t wv = 0u;
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+                    if (4 * k + b < nvalid) wv |= (uint32_t)__ldg(src + 4 * k + b) << (8 * b);
+                codes[k] = wv;
+            }
+        }
+        uint32_t* dst = out + item * AB;
+        for (int j = 0; j < AB; ++j) {
+            uint32_t word = 0u;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t t = (codes[k] >> j) & 0x01010101u;
+                word |= ((t * 0x01020408u) >> 24) << (4 * k);
+            }
+            dst[j] = word;
+        }
+    }
+}
+
 // NCHW input: a CTA transposes a [32 channels][32 pixels] tile through shared memory so that
 // global reads run along the contiguous pixel axis and the ballot still sees lane = channel.
 template <typename T>
@@ -141,8 +188,12 @@ int launch_pack_acts(const void* x, int dtype, int layout, int n, int c, int h, 
         const int grid = grid_for(pixels * CW, sms);
         if (dtype == EBS_F32)
             pack_acts_nhwc_kernel<float><<<grid, 256, 0, st>>>((const float*)x, pixels, c, CW, a_bits, inv_scale, out);
-        else
-            pack_acts_nhwc_kernel<uint8_t><<<grid, 256, 0, st>>>((const uint8_t*)x, pixels, c, CW, a_bits, inv_scale, out);
+        else {
+            const long long items = pixels * CW;
+            long long blocks = (items + 255) / 256;
+            if (blocks > (long long)sms * 32) blocks = (long long)sms * 32;
+            pack_acts_nhwc_u8_kernel<<<(int)blocks, 256, 0, st>>>((const uint8_t*)x, items, c, CW, a_bits, out);
+        }
     } else {
         const long long tiles = (long long)n * CW * ((h * w + 31) / 32);
         long long grid = tiles < (long long)sms * 16 ? tiles : (long long)sms * 16;
