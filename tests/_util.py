@@ -76,3 +76,32 @@ def rand_codes(rng, shape, bits, signed):
     if signed:
         return rng.integers(-(1 << (bits - 1)), (1 << (bits - 1)), size=shape, dtype=np.int32)
     return rng.integers(0, 1 << bits, size=shape, dtype=np.int32)
+
+
+def spec_desc(spec):
+    L = spec.layer
+    return ebs.conv_desc(L.c_in, L.c_out, L.k, L.k, L.stride, L.stride, L.pad, L.pad, spec.w_bits, spec.a_bits,
+                         spec.w_scale, spec.a_scale)
+
+
+def conv_on_device(px, n, h, w, pw, d, epi=None, want_acc=True, want_y=False, next_bits=0):
+    """ebs_conv2d_mixed on already packed device operands; returns device tensors (acc NHWC, y, packed_next)."""
+    ho, wo = ebs.ebs_conv_out_shape(d, h, w)
+    acc = torch.empty((n, ho, wo, d.c_out), dtype=torch.int32, device=dev()) if want_acc else None
+    y = torch.empty((n, ho, wo, d.c_out), dtype=torch.float32, device=dev()) if want_y else None
+    pn = None
+    if next_bits:
+        pn = torch.empty(ebs.ebs_packed_act_bytes(n, ho, wo, d.c_out, next_bits) // 4, dtype=torch.int32, device=dev())
+    ebs.ebs_conv2d_mixed(px, n, h, w, pw, d, epi, acc, y, pn)
+    return acc, y, pn
+
+
+def images_nchw(t: torch.Tensor, idx):
+    """Selected images of an NHWC device tensor as a numpy [len(idx), C, H, W] array."""
+    return t[idx].cpu().numpy().transpose(0, 3, 1, 2)
+
+
+def packed_images(pn: torch.Tensor, n, ho, wo, co, bits, idx):
+    """Selected images of a packed activation tensor as uint32 [len(idx), ho, wo, CW, bits]."""
+    v = pn.view(n, ho, wo, (co + 31) // 32, bits)
+    return v[idx].cpu().numpy().view(np.uint32)
