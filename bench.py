@@ -31,6 +31,9 @@ METRIC = "effective binary TOPS (2*MACs*Wb*Ab per second), ResNet-20 CIFAR quant
 UNIT = "TOPS"
 WORKLOAD = "config2: ResNet-20 CIFAR-shaped stack, 20 quantized convs, batch 128, (Wb,Ab) in {1..4}^2, seed 0"
 SM_COUNT, POPC_LANES_PER_CLK_SM = 148, 16
+# dram__bytes_read.sum + dram__bytes_write.sum per conv launch, mean over the 20 layers, from the ncu
+# capture summarised in profiles/ (outputs stay in the 126 MB L2 while ncu replays a launch)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
 
 
 def measured_peaks():
@@ -39,6 +42,11 @@ def measured_peaks():
         with open(path) as f:
             return json.load(f), "measured"
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+def int8_tensor_peak_tops(peaks: dict) -> float:
+    """Dense int8 tensor peak in TOPS: the measured bf16 burst figure times the nominal int8:bf16 ratio (2)."""
+    return 2.0 * float(peaks.get("bf16_tflops", 1590.0))
 
 
 def popc_pipe_peak_tops(sm_max_mhz: float) -> float:
@@ -328,11 +336,28 @@ def run_gpu(args):
     if rank != 0:
         return
     sm_max = float(clocks.get("sm_max_mhz") or peaks.get("sm_max_mhz", 1965.0))
-    peak_tops = popc_pipe_peak_tops(sm_max)
+    peak_tops = int8_tensor_peak_tops(peaks)                 # 1 bit-pair AND+bitcount = 1 byte MAC = 2 ops
+    hbm_gbs = float(peaks.get("hbm_gbs", 6650.0))
     achieved = total_ops / (conv_total_ms * 1e-3) / 1e12
-    per_layer = [{"name": L.spec.layer.name, "wb": L.spec.w_bits, "ab": L.spec.a_bits, "us": round(float(t) * 1e3, 2),
-                  "tops": round(L.ops / (t * 1e-3) / 1e12, 2), "frac": round(L.ops / (t * 1e-3) / 1e12 / peak_tops, 3)}
-                 for L, t in zip(layers, conv_ms)]
+    probes = {}
+    if world == 1:
+        try:
+            probes = {"imma_mma_sync_tops": 2 * ebs.ebs_probe_pipe(3, 500) / 1e12,
+                      "b1_mma_sync_tops": 2 * ebs.ebs_probe_pipe(1, 200) / 1e12,
+                      "and_popc_add_tops": 2 * ebs.ebs_probe_pipe(0, 500) / 1e12}
+        except Exception as exc:                                 # the probes are context, never fatal
+            probes = {"error": str(exc)}
+    per_layer, roof_ms = [], 0.0
+    for L, t in zip(layers, conv_ms):
+        lay = L.spec.layer
+        bytes_alg = (L.px.numel() * 4 + L.pw.numel() * 4 + L.acc.numel() * 4 + L.pn_bytes)
+        t_tensor, t_hbm = L.ops / (peak_tops * 1e12), bytes_alg / (hbm_gbs * 1e9)
+        roof = max(t_tensor, t_hbm)
+        roof_ms += roof * 1e3
+        per_layer.append({"name": lay.name, "wb": L.spec.w_bits, "ab": L.spec.a_bits, "us": round(float(t) * 1e3, 2),
+                          "tops": round(L.ops / (t * 1e-3) / 1e12, 1), "bytes": int(bytes_alg),
+                          "roof_us": round(roof * 1e6, 2), "roof": "tensor" if t_tensor >= t_hbm else "hbm",
+                          "frac_of_roof": round(roof * 1e3 / float(t), 3)})
     cpu = cpu_baseline_sample() if world == 1 and not args.no_cpu_baseline else None
     line = {
         "metric": METRIC, "value": world * total_ops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
@@ -349,10 +374,18 @@ def run_gpu(args):
                 "d2h_bytes_per_step": int(sum(L.pn_bytes for L in layers)),
                 "note": "ebs_conv2d_mixed_host per layer: pinned u8 codes in, packed next-layer planes out; wall clock"},
         "gpu_launches": 3 * len(layers) * args.steps,
-        "roofline": {"bound": "alu", "kernel": "conv_popc_kernel", "achieved": achieved, "peak": peak_tops,
-                     "unit": "TOPS (binary)", "frac": achieved / peak_tops, "traffic": None,
-                     "peak_source": f"POPC pipe: 148 SMs x 16 lanes/clk x 32 bit x {sm_max:.0f} MHz x 2 ops",
-                     "conv_ms_per_step": conv_total_ms, "per_layer_note": "per-layer times are L2-warm (10 back-to-back launches)", "hbm_peak_gbs": peaks.get("hbm_gbs"), "hbm_peak_kind": peak_kind,
+        "roofline": {"bound": "tensor", "kernel": "conv_mma_kernel (int8 mma.sync on bit planes)",
+                     "achieved": achieved, "peak": peak_tops, "unit": "TOPS", "frac": achieved / peak_tops,
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                     "peak_source": f"int8 dense = 2 x bf16 burst ({peaks.get('bf16_tflops')} TFLOP/s, {peak_kind}); "
+                                    "one bit-pair AND+bitcount is one byte multiply-accumulate = 2 ops",
+                     "conv_ms_per_step": conv_total_ms, "conv_launches_per_step": len(layers),
+                     "algorithmic_bytes_per_launch": int(np.mean([pl["bytes"] for pl in per_layer])),
+                     "sum_layer_roofs_ms": roof_ms, "frac_of_layer_roofs": roof_ms / float(conv_ms.sum()),
+                     "hbm_peak_gbs": hbm_gbs, "hbm_peak_kind": peak_kind,
+                     "other_pipes": dict(probes, popc_pipe_unit_count_tops=popc_pipe_peak_tops(sm_max)),
+                     "per_layer_note": "per-layer times are L2-warm (10 back-to-back launches in a graph); "
+                                       "roof = max(ops / tensor peak, algorithmic bytes / HBM peak)",
                      "per_layer": per_layer},
         "wall_s_timed_region": wall,
     }

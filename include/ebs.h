@@ -229,6 +229,7 @@ int ebs_conv2d_mixed_host_noalloc(const void *x_host, int dtype, int layout, int
  *   kind 0: AND + POPC + accumulate on the integer pipes        -> bit-AND-popcounts per second
  *   kind 1: mma.sync m16n8k256 b1 AND.POPC                      -> bit-AND-popcounts per second
  *   kind 2: POPC alone                                          -> bit-popcounts per second
+ *   kind 3: mma.sync m16n8k32 u8 x s8 (one byte per bit)        -> byte multiply-accumulates per second
  * The paper has no counterpart; this is measurement support.
  */
 int ebs_probe_pipe(int kind, int iters, double *bit_ops_per_second);

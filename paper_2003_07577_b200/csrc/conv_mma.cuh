@@ -206,7 +206,7 @@ conv_mma_kernel(const ConvParams p) {
 
         const uint32_t* A_s = smem + buf * T::STAGE_WORDS;
         const uint32_t* W_s = A_s + KSTEP * TILE_P * AB;
-#pragma unroll
+#pragma unroll 1
         for (int q = 0; q < KSTEP; ++q) {
             if ((q & (p.fold - 1)) == 0 && st * KSTEP + q < p.KK) {
                 // activation fragments: byte = 2^k where bit k-plane is set
@@ -286,8 +286,11 @@ conv_mma_kernel(const ConvParams p) {
     // ---- epilogue.  Fragment element e of (mt, nt): pixel row (e >> 1) * 8 + g, channel 2 * tq + (e & 1).
     const bool want_y = p.y != nullptr, want_q = p.packed_next != nullptr;
     uint8_t* out_s = reinterpret_cast<uint8_t*>(smem);      // [TILE_P][TILE_C + 4] requantized codes
+    constexpr int ROWB = code_row_bytes(TILE_C);
     const int qmax = (1 << p.next_bits) - 1;
     const bool pair_ok = (p.Co & 1) == 0;                   // two adjacent channels form an aligned 8-byte pair
+    // common case: even c_out, no per-channel terms, no residual, NHWC -> straight-line code
+    const bool simple = pair_ok && !p.ch_scale && !p.ch_bias && !p.residual && !p.y_nchw;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
@@ -295,6 +298,29 @@ conv_mma_kernel(const ConvParams p) {
             const int pl = (wp * MT + mt) * 16 + half * 8 + g;
             const int gp = tile_p0 + pl;
             const bool pvalid = gp < p.P;
+            const size_t row_o = (size_t)gp * p.Co + co0 + wc * NT * 8 + 2 * tq;
+            uint8_t* code_row = out_s + pl * ROWB + wc * NT * 8 + 2 * tq;
+            if (simple) {
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
+                    const int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
+                    const bool valid = pvalid && co < p.Co;
+                    int code0 = 0, code1 = 0;
+                    if (valid && p.acc) *reinterpret_cast<int2*>(p.acc + row_o + nt * 8) = make_int2(a0, a1);
+                    if (want_y || want_q) {
+                        float y0 = __fmul_rn((float)a0, p.S), y1 = __fmul_rn((float)a1, p.S);
+                        if (p.relu) { y0 = y0 > 0.0f ? y0 : 0.0f; y1 = y1 > 0.0f ? y1 : 0.0f; }
+                        if (valid && want_y) *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
+                        if (valid && want_q) {
+                            code0 = quantize_act_code(y0, p.inv_next, qmax);
+                            code1 = quantize_act_code(y1, p.inv_next, qmax);
+                        }
+                    }
+                    if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
+                }
+                continue;
+            }
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 const int cl = (wc * NT + nt) * 8 + 2 * tq, co = co0 + cl;
@@ -339,12 +365,12 @@ conv_mma_kernel(const ConvParams p) {
                             }
                         }
                         if (want_q) {
-                            code0 = quantize_code(y0, p.inv_next, 0, qmax);
-                            if (two) code1 = quantize_code(y1, p.inv_next, 0, qmax);
+                            code0 = quantize_act_code(y0, p.inv_next, qmax);
+                            if (two) code1 = quantize_act_code(y1, p.inv_next, qmax);
                         }
                     }
                 }
-                if (want_q) *reinterpret_cast<uint16_t*>(out_s + pl * code_row_bytes(TILE_C) + cl) = (uint16_t)(code0 | (code1 << 8));
+                if (want_q) *reinterpret_cast<uint16_t*>(out_s + pl * ROWB + cl) = (uint16_t)(code0 | (code1 << 8));
             }
         }
     }

@@ -79,6 +79,13 @@ __device__ __forceinline__ int quantize_code(float x, float inv_scale, int lo, i
     return q;
 }
 
+// The same quantizer for activation codes (lo = 0): floor and float->int in one conversion
+// (round toward -inf, saturating; NaN converts to 0), then an integer clamp.
+__device__ __forceinline__ int quantize_act_code(float y, float inv_scale, int qmax) {
+    const float r = __fadd_rn(__fmul_rn(y, inv_scale), 0.5f);
+    return min(max(__float2int_rd(r), 0), qmax);
+}
+
 // Row pitch (bytes) of the tile of requantized codes kept in shared memory: 4 bytes of padding make
 // consecutive pixels start in different banks.
 __host__ __device__ constexpr int code_row_bytes(int tile_c) { return tile_c + 4; }

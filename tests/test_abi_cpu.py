@@ -75,7 +75,7 @@ def test_validation_rejects_bad_requests_without_launching(ebs):
     assert L.ebs_pack_acts(fake, ebs.EBS_F32, 0, 1, 3, 4, 4, 2, 0.0, fake, None) == ebs.EBS_ERR_INVALID_ARG
     assert L.ebs_pack_weights(None, ebs.EBS_I8_CODES, 0, ref(good), fake, None) == ebs.EBS_ERR_INVALID_ARG
     assert L.ebs_dequant(fake, 0, 4, 1.0, None, None, 0, fake, None) == ebs.EBS_ERR_INVALID_ARG
-    assert L.ebs_probe_pipe(5, 10, ref(ctypes.c_double())) == ebs.EBS_ERR_INVALID_ARG
+    assert L.ebs_probe_pipe(9, 10, ref(ctypes.c_double())) == ebs.EBS_ERR_INVALID_ARG
     with pytest.raises(ebs.EbsError):
         ebs.ebs_conv_out_shape(ebs.conv_desc(64, 64, 9, 9, 1, 1, 0, 0, 2, 2, 0.05, 0.05), 4, 4)
 
