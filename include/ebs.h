@@ -158,8 +158,9 @@ int ebs_conv2d_mixed(const void *packed_x_dev, int n, int h, int w, const void *
 /*
  * The same call with the kernel variant forced (0 .. ebs_num_conv_variants()-1) instead of chosen by
  * the built-in heuristic (-1); the result is identical for every variant, only the speed differs.
- * Variants 0..9 are the integer-pipe kernels (AND + POPC), variants 10..18 the tensor-pipe kernels
- * (int8 MMA on bit planes expanded to bytes).
+ * Variants 0..9 are the integer-pipe kernels (AND + POPC), variants 10..18 the warp-level tensor-pipe
+ * kernels (int8 mma.sync on bit planes expanded to bytes), variants 19..22 the tcgen05 kernels (same
+ * product, 128 pixels x 16/32/64/128 channels per CTA, accumulator in tensor memory).
  * For tuning and for tests that must cover every kernel instantiation.  Returns
  * EBS_ERR_UNSUPPORTED if the variant cannot produce the requested packed output.
  */
@@ -167,6 +168,13 @@ int ebs_num_conv_variants(void);
 int ebs_conv2d_mixed_variant(const void *packed_x_dev, int n, int h, int w, const void *packed_w_dev,
                              const ebs_conv_desc *desc, const ebs_epilogue *epi, int32_t *acc_out_dev,
                              float *y_out_dev, void *packed_next_dev, void *stream, int variant);
+
+/*
+ * Number of thread blocks that gave up a bounded device-side wait (on the tensor core's completion
+ * barrier) since the library was loaded; such a block skips its outputs.  0 in a healthy run.
+ * Synchronizes the device.  The paper has no counterpart.
+ */
+long long ebs_device_wait_timeouts(void);
 
 /*
  * Stand-alone de-quantization of accumulators ("quantize_b includes the de-quantize process",

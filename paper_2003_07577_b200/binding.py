@@ -25,7 +25,7 @@ EXPORTS = [
     "ebs_version", "ebs_status_string", "ebs_last_cuda_error", "ebs_conv_out_shape", "ebs_packed_weight_bytes",
     "ebs_packed_act_bytes", "ebs_pack_weights", "ebs_pack_acts", "ebs_conv2d_mixed", "ebs_num_conv_variants",
     "ebs_conv2d_mixed_variant", "ebs_dequant", "ebs_host_workspace_bytes", "ebs_conv2d_mixed_host",
-    "ebs_probe_pipe", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
+    "ebs_probe_pipe", "ebs_device_wait_timeouts", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
 ]
 
 
@@ -83,6 +83,7 @@ def lib() -> ctypes.CDLL:
         L.ebs_conv2d_mixed_host.argtypes = [p, i, i, i, i, i, p, D, E, p, z, p, p, p, p]
         L.ebs_probe_pipe.argtypes = [i, i, ctypes.POINTER(ctypes.c_double)]
         L.ebs_noalloc_scratch_bytes.restype = z
+        L.ebs_device_wait_timeouts.restype = ctypes.c_longlong
         L.ebs_conv2d_mixed_host_noalloc.argtypes = [p, i, i, i, i, i, p, D, E, p, p, p, p]
         _lib = L
     return _lib
@@ -191,6 +192,10 @@ def ebs_probe_pipe(kind: int, iters: int = 2000) -> float:
     out = ctypes.c_double(0.0)
     _check(lib().ebs_probe_pipe(kind, iters, ctypes.byref(out)), "ebs_probe_pipe")
     return out.value
+
+
+def ebs_device_wait_timeouts() -> int:
+    return int(lib().ebs_device_wait_timeouts())
 
 
 def ebs_noalloc_scratch_bytes() -> int:

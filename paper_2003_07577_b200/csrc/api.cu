@@ -42,6 +42,25 @@ const ConvVariant* conv_mma_variant(int w_bits, int a_bits, int variant) {
     }
 }
 
+const ConvVariant* conv_umma_variant(int w_bits, int a_bits, int variant) {
+    switch (w_bits) {
+        case 1: return conv_umma_variant_w1(a_bits, variant);
+        case 2: return conv_umma_variant_w2(a_bits, variant);
+        case 3: return conv_umma_variant_w3(a_bits, variant);
+        case 4: return conv_umma_variant_w4(a_bits, variant);
+        case 5: return conv_umma_variant_w5(a_bits, variant);
+        case 6: return conv_umma_variant_w6(a_bits, variant);
+        case 7: return conv_umma_variant_w7(a_bits, variant);
+        case 8: return conv_umma_variant_w8(a_bits, variant);
+        default: return nullptr;
+    }
+}
+
+unsigned long long conv_umma_timeouts() {
+    return conv_umma_timeouts_w1() + conv_umma_timeouts_w2() + conv_umma_timeouts_w3() + conv_umma_timeouts_w4() +
+           conv_umma_timeouts_w5() + conv_umma_timeouts_w6() + conv_umma_timeouts_w7() + conv_umma_timeouts_w8();
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static int out_dim(int in, int pad, int k, int stride) {
@@ -129,7 +148,7 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
         if (epi->y_layout != EBS_NCHW && epi->y_layout != EBS_NHWC) return EBS_ERR_INVALID_ARG;
         if (!aligned16(epi->residual_dev)) return EBS_ERR_INVALID_ARG;
     }
-    if (variant >= NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS) return EBS_ERR_INVALID_ARG;
+    if (variant >= NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS) return EBS_ERR_INVALID_ARG;
 
     ConvParams p;
     memset(&p, 0, sizeof(p));
@@ -157,9 +176,11 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
                          : choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
     }
     if (variant >= NUM_CONV_VARIANTS && !mma_ok) return EBS_ERR_UNSUPPORTED;
-    const ConvVariant* v = variant >= NUM_CONV_VARIANTS
-                               ? conv_mma_variant(d->w_bits, d->a_bits, variant - NUM_CONV_VARIANTS)
-                               : conv_popc_variant(d->w_bits, d->a_bits, variant);
+    const ConvVariant* v =
+        variant >= NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS
+            ? conv_umma_variant(d->w_bits, d->a_bits, variant - NUM_CONV_VARIANTS - NUM_CONV_MMA_VARIANTS)
+            : (variant >= NUM_CONV_VARIANTS ? conv_mma_variant(d->w_bits, d->a_bits, variant - NUM_CONV_VARIANTS)
+                                            : conv_popc_variant(d->w_bits, d->a_bits, variant));
     if (!v) return EBS_ERR_UNSUPPORTED;
     if (packed_next && (v->tile_c % 32) != 0 && v->tile_c < p.Co) return EBS_ERR_UNSUPPORTED;
     const long long gx = (P + v->tile_p - 1) / v->tile_p, gy = (p.Co + v->tile_c - 1) / v->tile_c;
@@ -244,7 +265,9 @@ int ebs_conv2d_mixed(const void* packed_x_dev, int n, int h, int w, const void* 
                      stream, -1);
 }
 
-int ebs_num_conv_variants(void) { return NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS; }
+int ebs_num_conv_variants(void) { return NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS; }
+
+long long ebs_device_wait_timeouts(void) { return (long long)conv_umma_timeouts(); }
 
 int ebs_conv2d_mixed_variant(const void* packed_x_dev, int n, int h, int w, const void* packed_w_dev,
                              const ebs_conv_desc* desc, const ebs_epilogue* epi, int32_t* acc_out_dev,

@@ -16,27 +16,6 @@
 
 namespace ebs {
 
-template <int NWORDS>
-__device__ __forceinline__ void load_words_global(const uint32_t* __restrict__ src, uint32_t (&dst)[NWORDS]) {
-    // src is aligned to 4*NWORDS bytes when NWORDS is a power of two (plane-minor layout).
-    if constexpr (NWORDS % 4 == 0) {
-#pragma unroll
-        for (int v = 0; v < NWORDS / 4; ++v) {
-            uint4 t = __ldg(reinterpret_cast<const uint4*>(src) + v);
-            dst[4 * v] = t.x; dst[4 * v + 1] = t.y; dst[4 * v + 2] = t.z; dst[4 * v + 3] = t.w;
-        }
-    } else if constexpr (NWORDS % 2 == 0) {
-#pragma unroll
-        for (int v = 0; v < NWORDS / 2; ++v) {
-            uint2 t = __ldg(reinterpret_cast<const uint2*>(src) + v);
-            dst[2 * v] = t.x; dst[2 * v + 1] = t.y;
-        }
-    } else {
-#pragma unroll
-        for (int v = 0; v < NWORDS; ++v) dst[v] = __ldg(src + v);
-    }
-}
-
 template <int WB, int AB, int TP, int TC, int WARPS_P, int WARPS_C>
 struct PopcTile {
     static constexpr int NT = 32 * WARPS_P * WARPS_C;

@@ -1,0 +1,393 @@
+// Implicit-GEMM bit-plane convolution on the 5th-generation tensor cores (tcgen05.mma kind::i8,
+// accumulator in tensor memory), sm_100a.
+//
+// Same arithmetic as conv_mma_kernel: activation plane k is expanded to bytes 2^k * bit, weight plane m
+// to bytes 2^m * bit (the top plane to -2^(M-1) * bit), and one int8 MMA of plane k against plane m adds
+// c_m 2^(m+k) * bitcount(AND(plane k, plane m)) -- Eq. 13 and Eq. 14 at once -- into ONE int32
+// accumulator per output.  Here an MMA covers 128 output pixels x TILE_N channels x 32 reduction bits,
+// reads both operands from shared memory and accumulates in tensor memory (TMEM).
+//
+// A CTA (128 threads) owns 128 consecutive output pixels x TILE_N channels.  Per reduction word:
+//   1. every thread expands the packed words of "its" pixel row (all Ab planes) and its share of the
+//      weight rows into 32-byte rows of a K-major, 32-byte-swizzled shared tile (one tile per plane);
+//      the bit -> byte map (byte 4b+i of a row <- bit 8i+b of the word) is the same for both operands;
+//   2. fence.proxy.async + __syncthreads hand the tiles to the tensor core;
+//   3. one thread issues Wb*Ab tcgen05.mma (one per plane pair) and a tcgen05.commit that arrives on
+//      the stage's mbarrier when the tensor core has finished reading the stage.
+// Two stages: the expansion of the next reduction words overlaps the MMAs of the current ones.
+// Epilogue: tcgen05.ld gives every thread the TILE_N accumulators of its pixel; it stores them,
+// applies the fp32 steps and packs the requantized codes of its pixel into plane words in registers.
+//
+// Every wait on an mbarrier is bounded; on a timeout the CTA records it in a device counter, skips
+// its remaining work, frees its tensor memory and returns.
+#pragma once
+
+#include "ebs_internal.cuh"
+
+namespace ebs {
+
+constexpr int UMMA_KTAB = 256;          // reduction words the in-kernel tap table can hold
+constexpr int UMMA_M = 128;             // pixels per CTA = TMEM lanes
+constexpr unsigned UMMA_WAIT_LIMIT = 1u << 20;
+
+static __device__ unsigned long long g_umma_timeouts = 0ull;   // CTAs that gave up waiting (0 in a healthy run)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(count));
+}
+// Bounded wait for the phase with the given parity; false = gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    for (unsigned it = 0; it < UMMA_WAIT_LIMIT; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}\n"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// Shared-memory matrix descriptor: K-major operand, 32-byte swizzle, rows of 32 bytes (K = 32 int8),
+// 8-row groups 256 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_sw32(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);     // start address, 16-byte units
+    d |= (uint64_t)1u << 16;                         // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(256u >> 4) << 32;                // stride byte offset between 8-row groups
+    d |= (uint64_t)1u << 46;                         // descriptor version of this architecture
+    d |= (uint64_t)6u << 61;                         // layout type: 32-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: D = s32, A = u8 (activations), B = s8 (weights), both K-major, M = 128.
+__host__ __device__ constexpr uint32_t umma_idesc_i8(int n) {
+    return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(UMMA_M >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                        uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}\n"
+        :: "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+}
+
+// One packed word -> one 32-byte row (two 16-byte chunks) of plane-coefficient bytes.
+// Byte 4b+i of the row is (bit 8i+b of the word) * coefficient; `scale` = 1, or 2^(9-Wb)-1 for the
+// top weight plane so that its byte is the two's-complement byte of -2^(Wb-1).
+__device__ __forceinline__ void expand_word_to_row(uint32_t word, int plane, uint32_t scale, uint4& lo, uint4& hi) {
+    const uint32_t mask = 0x01010101u << plane;
+    uint32_t r[8];
+#pragma unroll
+    for (int b = 0; b < 8; ++b) r[b] = (__funnelshift_r(word, word, b - plane) & mask) * scale;
+    lo = make_uint4(r[0], r[1], r[2], r[3]);
+    hi = make_uint4(r[4], r[5], r[6], r[7]);
+}
+// Address of 16-byte chunk c (0/1) of row `row` in a 32-byte-swizzled tile (tile base 256-byte aligned).
+__device__ __forceinline__ uint8_t* sw32_chunk(uint8_t* tile, int row, int c) {
+    return tile + row * 32 + ((c ^ ((row >> 2) & 1)) << 4);
+}
+
+template <int WB, int AB, int TILE_N>
+struct UmmaTile {
+    static constexpr int A_PLANE_BYTES = UMMA_M * 32;                   // one activation plane, one reduction word
+    static constexpr int B_PLANE_BYTES = TILE_N * 32;
+    static constexpr int KW_BYTES = AB * A_PLANE_BYTES + WB * B_PLANE_BYTES;
+    static constexpr int KS_RAW = (24 * 1024) / KW_BYTES;               // reduction words per stage
+    static constexpr int KS = KS_RAW < 1 ? 1 : (KS_RAW > 4 ? 4 : KS_RAW);
+    static constexpr int STAGE_BYTES = KS * KW_BYTES;
+    static constexpr int SMEM_BYTES = 2 * STAGE_BYTES + 1024;           // + slack to align the tiles to 1 KB
+    static constexpr int TMEM_COLS = TILE_N < 32 ? 32 : TILE_N;
+    static_assert(TILE_N % 16 == 0 && TILE_N >= 16 && TILE_N <= 256, "tcgen05.mma N for M = 128");
+    static_assert((STAGE_BYTES % 256) == 0, "tiles keep the swizzle alignment");
+};
+
+template <int WB, int AB, int TILE_N>
+__global__ void __launch_bounds__(UMMA_M) conv_umma_kernel(const ConvParams p) {
+    using T = UmmaTile<WB, AB, TILE_N>;
+    constexpr int KS = T::KS;
+    extern __shared__ uint8_t dyn_smem[];
+    __shared__ int2 ktab[UMMA_KTAB];
+    __shared__ __align__(8) uint64_t mbar[2];
+    __shared__ uint32_t tmem_slot;
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tile_p0 = blockIdx.x * UMMA_M;
+    const int co0 = blockIdx.y * TILE_N;
+    uint8_t* tiles = dyn_smem + ((1024u - (smem_u32(dyn_smem) & 1023u)) & 1023u);
+
+    // ---- set-up: tap table, barriers, tensor memory
+    for (int kk = tid; kk < p.KK; kk += UMMA_M) {
+        const int tap = kk / p.CW, cw = kk - tap * p.CW;
+        const int r = tap / p.kw, s = tap - r * p.kw;
+        ktab[kk] = make_int2(((r * p.W + s) * p.CW + cw) * AB, r | (s << 8));
+    }
+    if (tid == 0) {
+        mbar_init(&mbar[0], 1);
+        mbar_init(&mbar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&tmem_slot)),
+                     "r"((uint32_t)T::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    const uint32_t tmem_base = tmem_slot;
+
+    // ---- this thread's pixel row
+    const int gp = tile_p0 + tid;
+    int pix_off = 0;
+    uint32_t row_ok = 0u, col_ok = 0u;
+    if (gp < p.P) {
+        const int hw = p.Ho * p.Wo;
+        const int n = gp / hw, rem = gp - n * hw;
+        const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
+        const int h0 = ho * p.sh - p.ph, w0 = wo * p.sw - p.pw;
+        pix_off = ((n * p.H + h0) * p.W + w0) * p.CW * AB;
+        for (int r = 0; r < p.kh; ++r) row_ok |= ((unsigned)(h0 + r) < (unsigned)p.H ? 1u : 0u) << r;
+        for (int s = 0; s < p.kw; ++s) col_ok |= ((unsigned)(w0 + s) < (unsigned)p.W ? 1u : 0u) << s;
+    }
+
+    const int kwords = (p.KK + p.fold - 1) / p.fold;          // reduction words after tap folding
+    const int nchunks = (kwords + KS - 1) / KS;
+    constexpr uint32_t IDESC = umma_idesc_i8(TILE_N);
+    bool aborted = false;
+
+    for (int ch = 0; ch < nchunks; ++ch) {
+        const int st = ch & 1;
+        uint8_t* A_st = tiles + st * T::STAGE_BYTES;               // [KS][AB] planes of 128 rows x 32 B
+        uint8_t* B_st = A_st + KS * AB * T::A_PLANE_BYTES;         // [KS][WB] planes of TILE_N rows x 32 B
+        if (ch >= 2) {                                             // the MMAs of chunk ch-2 must have read the stage
+            bool ok = true;
+            if (tid == 0) ok = mbar_wait_bounded(&mbar[st], (uint32_t)(((ch >> 1) - 1) & 1));
+            if (__syncthreads_or(!ok)) { aborted = true; break; }
+        }
+        // ---- expand
+#pragma unroll 1
+        for (int q = 0; q < KS; ++q) {
+            const int kw = ch * KS + q;
+            // activations: row = this thread's pixel, all planes
+            uint32_t aw[AB];
+#pragma unroll
+            for (int k = 0; k < AB; ++k) aw[k] = 0u;
+            if (kw < kwords) {
+                for (int f = 0; f < p.fold; ++f) {
+                    const int kk = kw * p.fold + f;
+                    if (kk >= p.KK) break;
+                    const int2 info = ktab[kk];
+                    if ((row_ok >> (info.y & 0xff)) & (col_ok >> (info.y >> 8)) & 1u) {
+                        uint32_t t[AB];
+                        load_words_global<AB>(p.x + (pix_off + info.x), t);
+#pragma unroll
+                        for (int k = 0; k < AB; ++k) aw[k] |= t[k] << (f * p.fold_bits);
+                    }
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < AB; ++k) {
+                uint4 lo, hi;
+                expand_word_to_row(aw[k], k, 1u, lo, hi);
+                uint8_t* tile = A_st + (q * AB + k) * T::A_PLANE_BYTES;
+                *reinterpret_cast<uint4*>(sw32_chunk(tile, tid, 0)) = lo;
+                *reinterpret_cast<uint4*>(sw32_chunk(tile, tid, 1)) = hi;
+            }
+            // weights: TILE_N * WB rows shared out over the threads
+            for (int item = tid; item < TILE_N * WB; item += UMMA_M) {
+                const int m = item / TILE_N, nrow = item - m * TILE_N;
+                uint32_t ww = 0u;
+                if (kw < kwords && co0 + nrow < p.Co) {
+                    for (int f = 0; f < p.fold; ++f) {
+                        const int kk = kw * p.fold + f;
+                        if (kk >= p.KK) break;
+                        ww |= __ldg(p.w + ((size_t)kk * p.Co + co0 + nrow) * WB + m) << (f * p.fold_bits);
+                    }
+                }
+                const uint32_t scale = (m == WB - 1 && WB < 8) ? ((1u << (9 - WB)) - 1u) : 1u;
+                uint4 lo, hi;
+                expand_word_to_row(ww, m, scale, lo, hi);
+                uint8_t* tile = B_st + (q * WB + m) * T::B_PLANE_BYTES;
+                *reinterpret_cast<uint4*>(sw32_chunk(tile, nrow, 0)) = lo;
+                *reinterpret_cast<uint4*>(sw32_chunk(tile, nrow, 1)) = hi;
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");     // generic writes -> tensor-core reads
+        asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+        __syncthreads();
+        // ---- issue the MMAs of this chunk
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            const uint32_t a_base = smem_u32(A_st), b_base = smem_u32(B_st);
+#pragma unroll 1
+            for (int q = 0; q < KS; ++q) {
+                if (ch * KS + q >= kwords) break;
+#pragma unroll 1
+                for (int m = 0; m < WB; ++m) {
+                    const uint64_t db = umma_desc_sw32(b_base + (q * WB + m) * T::B_PLANE_BYTES);
+#pragma unroll 1
+                    for (int k = 0; k < AB; ++k) {
+                        const uint64_t da = umma_desc_sw32(a_base + (q * AB + k) * T::A_PLANE_BYTES);
+                        const uint32_t accumulate = (ch | q | m | k) != 0 ? 1u : 0u;
+                        umma_i8(tmem_base, da, db, IDESC, accumulate);
+                    }
+                }
+            }
+            umma_commit(&mbar[st]);
+        }
+    }
+
+    // ---- wait for the last MMAs, then the epilogue straight out of tensor memory
+    if (!aborted) {
+        const int last = nchunks - 1;
+        bool ok = true;
+        if (tid == 0) ok = mbar_wait_bounded(&mbar[last & 1], (uint32_t)((last >> 1) & 1));
+        if (__syncthreads_or(!ok)) aborted = true;
+    }
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+
+    if (!aborted) {
+        const bool want_y = p.y != nullptr, want_q = p.packed_next != nullptr;
+        const int qmax = (1 << p.next_bits) - 1;
+        const bool pvalid = gp < p.P;
+        const bool vec_ok = (p.Co & 3) == 0;                        // 16-byte aligned groups of four channels
+        const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
+        const int hw = p.Ho * p.Wo;
+        const int img = pvalid ? gp / hw : 0, rem = pvalid ? gp - img * hw : 0;
+        uint32_t planes[8];
+#pragma unroll 1
+        for (int c0 = 0; c0 < TILE_N; c0 += 16) {
+            uint32_t v[16];
+            tmem_ld16(trow + (uint32_t)c0, v);                       // whole warp, also for rows past the end
+            if ((c0 & 31) == 0) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) planes[j] = 0u;
+            }
+#pragma unroll
+            for (int gq = 0; gq < 4; ++gq) {                          // four channels at a time
+                const int co = co0 + c0 + 4 * gq;
+                uint32_t code4 = 0u;
+                float yv[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int a = (int)v[4 * gq + e];
+                    float y = __fmul_rn((float)a, p.S);
+                    if (co + e < p.Co) {
+                        if (p.ch_scale) y = __fmul_rn(y, __ldg(p.ch_scale + co + e));
+                        if (p.ch_bias) y = __fadd_rn(y, __ldg(p.ch_bias + co + e));
+                        if (p.residual && pvalid) y = __fadd_rn(y, __ldg(p.residual + (size_t)gp * p.Co + co + e));
+                    }
+                    if (p.relu && !(y > 0.0f)) y = 0.0f;
+                    yv[e] = y;
+                    if (want_q && co + e < p.Co) code4 |= (uint32_t)quantize_act_code(y, p.inv_next, qmax) << (8 * e);
+                }
+                if (pvalid && co < p.Co) {
+                    const size_t o = (size_t)gp * p.Co + co;
+                    if (p.acc) {
+                        if (vec_ok) *reinterpret_cast<int4*>(p.acc + o) =
+                            make_int4((int)v[4 * gq], (int)v[4 * gq + 1], (int)v[4 * gq + 2], (int)v[4 * gq + 3]);
+                        else
+                            for (int e = 0; e < 4 && co + e < p.Co; ++e) p.acc[o + e] = (int)v[4 * gq + e];
+                    }
+                    if (want_y) {
+                        if (p.y_nchw) {
+                            for (int e = 0; e < 4 && co + e < p.Co; ++e)
+                                p.y[((size_t)img * p.Co + co + e) * hw + rem] = yv[e];
+                        } else if (vec_ok) {
+                            *reinterpret_cast<float4*>(p.y + o) = make_float4(yv[0], yv[1], yv[2], yv[3]);
+                        } else {
+                            for (int e = 0; e < 4 && co + e < p.Co; ++e) p.y[o + e] = yv[e];
+                        }
+                    }
+                }
+                if (want_q) {
+                    const int nib_pos = ((c0 & 16) >> 2) + gq;          // which nibble of the 32-channel word
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (j < p.next_bits)
+                            planes[j] |= ((((code4 >> j) & 0x01010101u) * 0x01020408u) >> 24) << (4 * nib_pos);
+                }
+            }
+            const bool word_done = ((c0 & 16) != 0) || (c0 + 16 >= TILE_N);
+            if (want_q && word_done && pvalid) {
+                const int cwg = (co0 + c0) >> 5;
+                if (cwg < p.CWo) {
+                    uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + cwg) * p.next_bits;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (j < p.next_bits) dst[j] = planes[j];
+                }
+            }
+        }
+    } else if (tid == 0) {
+        atomicAdd(&g_umma_timeouts, 1ull);
+    }
+
+    // ---- release tensor memory (every path reaches this)
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"((uint32_t)T::TMEM_COLS)
+                     : "memory");
+    }
+}
+
+template <int WB, int AB, int TILE_N>
+void launch_conv_umma(const ConvParams& p, dim3 grid, cudaStream_t st) {
+    using T = UmmaTile<WB, AB, TILE_N>;
+    static bool attr_set = false;              // raising the dynamic shared-memory limit is a one-time attribute
+    if (!attr_set) {
+        cudaFuncSetAttribute(conv_umma_kernel<WB, AB, TILE_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             T::SMEM_BYTES);
+        attr_set = true;
+    }
+    conv_umma_kernel<WB, AB, TILE_N><<<grid, UMMA_M, T::SMEM_BYTES, st>>>(p);
+}
+
+constexpr int NUM_UMMA_VARIANTS = 4;           // TILE_N = 16, 32, 64, 128
+
+template <int WB, int AB, int VARIANT>
+constexpr ConvVariant make_umma_variant() {
+    constexpr int TILE_N = 16 << VARIANT;
+    return ConvVariant{&launch_conv_umma<WB, AB, TILE_N>, UMMA_M, TILE_N, UMMA_M};
+}
+
+#define EBS_UMMA_ROW(WB, AB)                                                                              \
+    {make_umma_variant<WB, AB, 0>(), make_umma_variant<WB, AB, 1>(), make_umma_variant<WB, AB, 2>(),      \
+     make_umma_variant<WB, AB, 3>()}
+
+#define EBS_DEFINE_UMMA_TABLE(WB)                                                                         \
+    const ConvVariant* conv_umma_variant_w##WB(int a_bits, int variant) {                                 \
+        static const ConvVariant table[8][NUM_UMMA_VARIANTS] = {                                          \
+            EBS_UMMA_ROW(WB, 1), EBS_UMMA_ROW(WB, 2), EBS_UMMA_ROW(WB, 3), EBS_UMMA_ROW(WB, 4),           \
+            EBS_UMMA_ROW(WB, 5), EBS_UMMA_ROW(WB, 6), EBS_UMMA_ROW(WB, 7), EBS_UMMA_ROW(WB, 8)};          \
+        if (a_bits < 1 || a_bits > 8 || variant < 0 || variant >= NUM_UMMA_VARIANTS) return nullptr;      \
+        return &table[a_bits - 1][variant];                                                               \
+    }                                                                                                     \
+    unsigned long long conv_umma_timeouts_w##WB() {                                                       \
+        unsigned long long v = 0;                                                                         \
+        cudaMemcpyFromSymbol(&v, g_umma_timeouts, sizeof(v));                                             \
+        return v;                                                                                         \
+    }
+
+}  // namespace ebs

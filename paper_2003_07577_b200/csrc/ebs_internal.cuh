@@ -56,6 +56,17 @@ EBS_DECLARE_WB(1) EBS_DECLARE_WB(2) EBS_DECLARE_WB(3) EBS_DECLARE_WB(4)
 EBS_DECLARE_WB(5) EBS_DECLARE_WB(6) EBS_DECLARE_WB(7) EBS_DECLARE_WB(8)
 #undef EBS_DECLARE_WB
 
+// 5th-generation tensor-core kernels (conv_umma_w1.cu .. conv_umma_w8.cu); variant = log2(tile_n / 16).
+enum { NUM_CONV_UMMA_VARIANTS = 4 };
+const ConvVariant* conv_umma_variant(int w_bits, int a_bits, int variant);
+unsigned long long conv_umma_timeouts();
+#define EBS_DECLARE_WB(WB)                                                   \
+    const ConvVariant* conv_umma_variant_w##WB(int a_bits, int variant);     \
+    unsigned long long conv_umma_timeouts_w##WB();
+EBS_DECLARE_WB(1) EBS_DECLARE_WB(2) EBS_DECLARE_WB(3) EBS_DECLARE_WB(4)
+EBS_DECLARE_WB(5) EBS_DECLARE_WB(6) EBS_DECLARE_WB(7) EBS_DECLARE_WB(8)
+#undef EBS_DECLARE_WB
+
 // pack.cu
 int launch_pack_acts(const void* x, int dtype, int layout, int n, int c, int h, int w, int a_bits,
                      float inv_scale, uint32_t* out, cudaStream_t st);
@@ -67,6 +78,28 @@ int launch_dequant(const int32_t* acc, size_t n_pixels, int c_out, float scale, 
 
 // Records a CUDA error for ebs_last_cuda_error() and returns EBS_ERR_CUDA (or EBS_OK).
 int check_cuda(cudaError_t e);
+
+// Reads NWORDS consecutive packed words from global memory through the read-only path.
+template <int NWORDS>
+__device__ __forceinline__ void load_words_global(const uint32_t* __restrict__ src, uint32_t (&dst)[NWORDS]) {
+    // src is aligned to 4*NWORDS bytes when NWORDS is a power of two (plane-minor layout).
+    if constexpr (NWORDS % 4 == 0) {
+#pragma unroll
+        for (int v = 0; v < NWORDS / 4; ++v) {
+            uint4 t = __ldg(reinterpret_cast<const uint4*>(src) + v);
+            dst[4 * v] = t.x; dst[4 * v + 1] = t.y; dst[4 * v + 2] = t.z; dst[4 * v + 3] = t.w;
+        }
+    } else if constexpr (NWORDS % 2 == 0) {
+#pragma unroll
+        for (int v = 0; v < NWORDS / 2; ++v) {
+            uint2 t = __ldg(reinterpret_cast<const uint2*>(src) + v);
+            dst[2 * v] = t.x; dst[2 * v + 1] = t.y;
+        }
+    } else {
+#pragma unroll
+        for (int v = 0; v < NWORDS; ++v) dst[v] = __ldg(src + v);
+    }
+}
 
 // quantize_b of Eq. 1c in code form: round half up, every fp32 operation rounded on its own.
 __device__ __forceinline__ int quantize_code(float x, float inv_scale, int lo, int hi) {
