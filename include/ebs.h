@@ -159,8 +159,8 @@ int ebs_conv2d_mixed(const void *packed_x_dev, int n, int h, int w, const void *
  * The same call with the kernel variant forced (0 .. ebs_num_conv_variants()-1) instead of chosen by
  * the built-in heuristic (-1); the result is identical for every variant, only the speed differs.
  * Variants 0..9 are the integer-pipe kernels (AND + POPC), variants 10..18 the warp-level tensor-pipe
- * kernels (int8 mma.sync on bit planes expanded to bytes), variants 19..22 the tcgen05 kernels (same
- * product, 128 pixels x 16/32/64/128 channels per CTA, accumulator in tensor memory).
+ * kernels (int8 mma.sync on bit planes expanded to bytes), variants 19..23 the tcgen05 kernels (same
+ * product, 128 pixels x 16/32/64/128/256 channels per CTA, accumulator in tensor memory).
  * For tuning and for tests that must cover every kernel instantiation.  Returns
  * EBS_ERR_UNSUPPORTED if the variant cannot produce the requested packed output.
  */

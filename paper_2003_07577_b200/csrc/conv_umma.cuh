@@ -7,19 +7,22 @@
 // accumulator per output.  Here an MMA covers 128 output pixels x TILE_N channels x 32 reduction bits,
 // reads both operands from shared memory and accumulates in tensor memory (TMEM).
 //
-// A CTA (128 threads) owns 128 consecutive output pixels x TILE_N channels.  Per reduction word:
-//   1. every thread expands the packed words of "its" pixel row (all Ab planes) and its share of the
-//      weight rows into 32-byte rows of a K-major, 32-byte-swizzled shared tile (one tile per plane);
-//      the bit -> byte map (byte 4b+i of a row <- bit 8i+b of the word) is the same for both operands;
-//   2. fence.proxy.async + __syncthreads hand the tiles to the tensor core;
-//   3. one thread issues Wb*Ab tcgen05.mma (one per plane pair) and a tcgen05.commit that arrives on
-//      the stage's mbarrier when the tensor core has finished reading the stage.
-// Two stages: the expansion of the next reduction words overlaps the MMAs of the current ones.
-// Epilogue: tcgen05.ld gives every thread the TILE_N accumulators of its pixel; it stores them,
-// applies the fp32 steps and packs the requantized codes of its pixel into plane words in registers.
+// A CTA owns 128 consecutive output pixels x TILE_N channels and has 9 warps:
+//   warps 0-7 (expanders)  load packed words one stage ahead into registers, expand them -- the
+//      thread's pixel row for its share of the activation planes and its share of the weight rows --
+//      into 32-byte rows of K-major, 32-byte-swizzled shared tiles (one tile per plane and reduction
+//      word; byte 4b+i of a row <- bit 8i+b of the word, the same map for both operands), then
+//      fence.proxy.async and arrive on the stage's "full" mbarrier;
+//   warp 8 (issuer)        waits for "full", issues Wb*Ab tcgen05.mma per reduction word (one per
+//      plane pair) and a tcgen05.commit that arrives on the stage's "empty" mbarrier once the tensor
+//      core has read the stage.
+// Two stages, so expansion of the next reduction words overlaps the MMAs of the current ones.
+// Epilogue: tcgen05.ld gives every expander thread accumulators of its pixel (warps w and w+4 split
+// the channels); it stores them, applies the fp32 steps and packs the requantized codes of its pixel
+// into plane words in registers.
 //
-// Every wait on an mbarrier is bounded; on a timeout the CTA records it in a device counter, skips
-// its remaining work, frees its tensor memory and returns.
+// Every wait on an mbarrier is bounded; on a timeout the CTA raises a shared abort flag, all its
+// loops end, it records the event in a device counter, frees its tensor memory and returns.
 #pragma once
 
 #include "ebs_internal.cuh"
@@ -37,8 +40,11 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(count));
 }
-// Bounded wait for the phase with the given parity; false = gave up.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait for the phase with the given parity; false = gave up (or another thread already had).
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     const uint32_t addr = smem_u32(bar);
     for (unsigned it = 0; it < UMMA_WAIT_LIMIT; ++it) {
         uint32_t done;
@@ -48,7 +54,9 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
             "selp.u32 %0, 1, 0, p;\n\t}\n"
             : "=r"(done) : "r"(addr), "r"(parity) : "memory");
         if (done) return true;
+        if (*abort_flag) return false;
     }
+    *abort_flag = 1;
     return false;
 }
 
@@ -107,6 +115,9 @@ __device__ __forceinline__ uint8_t* sw32_chunk(uint8_t* tile, int row, int c) {
     return tile + row * 32 + ((c ^ ((row >> 2) & 1)) << 4);
 }
 
+constexpr int UMMA_EXPANDERS = 256;     // threads of warps 0-7
+constexpr int UMMA_THREADS = UMMA_EXPANDERS + 32;
+
 template <int WB, int AB, int TILE_N>
 struct UmmaTile {
     static constexpr int A_PLANE_BYTES = UMMA_M * 32;                   // one activation plane, one reduction word
@@ -117,36 +128,45 @@ struct UmmaTile {
     static constexpr int STAGE_BYTES = KS * KW_BYTES;
     static constexpr int SMEM_BYTES = 2 * STAGE_BYTES + 1024;           // + slack to align the tiles to 1 KB
     static constexpr int TMEM_COLS = TILE_N < 32 ? 32 : TILE_N;
+    static constexpr int A_ITEMS = KS * AB;                              // (reduction word, plane) per pixel row
+    static constexpr int B_ITEMS = (KS * WB * TILE_N + UMMA_EXPANDERS - 1) / UMMA_EXPANDERS;   // weight rows per thread
     static_assert(TILE_N % 16 == 0 && TILE_N >= 16 && TILE_N <= 256, "tcgen05.mma N for M = 128");
     static_assert((STAGE_BYTES % 256) == 0, "tiles keep the swizzle alignment");
+    static_assert(SMEM_BYTES <= 220 * 1024, "shared memory per CTA");
 };
 
 template <int WB, int AB, int TILE_N>
-__global__ void __launch_bounds__(UMMA_M) conv_umma_kernel(const ConvParams p) {
+__global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParams p) {
     using T = UmmaTile<WB, AB, TILE_N>;
     constexpr int KS = T::KS;
     extern __shared__ uint8_t dyn_smem[];
     __shared__ int2 ktab[UMMA_KTAB];
-    __shared__ __align__(8) uint64_t mbar[2];
+    __shared__ __align__(8) uint64_t full_bar[2];
+    __shared__ __align__(8) uint64_t empty_bar[2];
     __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int tile_p0 = blockIdx.x * UMMA_M;
     const int co0 = blockIdx.y * TILE_N;
     uint8_t* tiles = dyn_smem + ((1024u - (smem_u32(dyn_smem) & 1023u)) & 1023u);
+    volatile int* abortp = &abort_flag;
 
     // ---- set-up: tap table, barriers, tensor memory
-    for (int kk = tid; kk < p.KK; kk += UMMA_M) {
+    for (int kk = tid; kk < p.KK; kk += UMMA_THREADS) {
         const int tap = kk / p.CW, cw = kk - tap * p.CW;
         const int r = tap / p.kw, s = tap - r * p.kw;
         ktab[kk] = make_int2(((r * p.W + s) * p.CW + cw) * AB, r | (s << 8));
     }
     if (tid == 0) {
-        mbar_init(&mbar[0], 1);
-        mbar_init(&mbar[1], 1);
+        abort_flag = 0;
+        mbar_init(&full_bar[0], UMMA_EXPANDERS);
+        mbar_init(&full_bar[1], UMMA_EXPANDERS);
+        mbar_init(&empty_bar[0], 1);
+        mbar_init(&empty_bar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    if (warp == 0) {
+    if (warp == 8) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&tmem_slot)),
                      "r"((uint32_t)T::TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
@@ -156,127 +176,165 @@ __global__ void __launch_bounds__(UMMA_M) conv_umma_kernel(const ConvParams p) {
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const uint32_t tmem_base = tmem_slot;
 
-    // ---- this thread's pixel row
-    const int gp = tile_p0 + tid;
-    int pix_off = 0;
-    uint32_t row_ok = 0u, col_ok = 0u;
-    if (gp < p.P) {
-        const int hw = p.Ho * p.Wo;
-        const int n = gp / hw, rem = gp - n * hw;
-        const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
-        const int h0 = ho * p.sh - p.ph, w0 = wo * p.sw - p.pw;
-        pix_off = ((n * p.H + h0) * p.W + w0) * p.CW * AB;
-        for (int r = 0; r < p.kh; ++r) row_ok |= ((unsigned)(h0 + r) < (unsigned)p.H ? 1u : 0u) << r;
-        for (int s = 0; s < p.kw; ++s) col_ok |= ((unsigned)(w0 + s) < (unsigned)p.W ? 1u : 0u) << s;
-    }
-
     const int kwords = (p.KK + p.fold - 1) / p.fold;          // reduction words after tap folding
     const int nchunks = (kwords + KS - 1) / KS;
-    constexpr uint32_t IDESC = umma_idesc_i8(TILE_N);
-    bool aborted = false;
+    const int row = tid & (UMMA_M - 1);                        // pixel row of an expander thread
+    const int gp = tile_p0 + row;
 
-    for (int ch = 0; ch < nchunks; ++ch) {
-        const int st = ch & 1;
-        uint8_t* A_st = tiles + st * T::STAGE_BYTES;               // [KS][AB] planes of 128 rows x 32 B
-        uint8_t* B_st = A_st + KS * AB * T::A_PLANE_BYTES;         // [KS][WB] planes of TILE_N rows x 32 B
-        if (ch >= 2) {                                             // the MMAs of chunk ch-2 must have read the stage
-            bool ok = true;
-            if (tid == 0) ok = mbar_wait_bounded(&mbar[st], (uint32_t)(((ch >> 1) - 1) & 1));
-            if (__syncthreads_or(!ok)) { aborted = true; break; }
+    if (warp < 8) {
+        // =========================== expanders ===========================
+        const int half = tid >> 7;                             // which share of the activation items
+        int pix_off = 0;
+        uint32_t row_ok = 0u, col_ok = 0u;
+        if (gp < p.P) {
+            const int hw = p.Ho * p.Wo;
+            const int n = gp / hw, rem = gp - n * hw;
+            const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
+            const int h0 = ho * p.sh - p.ph, w0 = wo * p.sw - p.pw;
+            pix_off = ((n * p.H + h0) * p.W + w0) * p.CW * AB;
+            for (int r = 0; r < p.kh; ++r) row_ok |= ((unsigned)(h0 + r) < (unsigned)p.H ? 1u : 0u) << r;
+            for (int s = 0; s < p.kw; ++s) col_ok |= ((unsigned)(w0 + s) < (unsigned)p.W ? 1u : 0u) << s;
         }
-        // ---- expand
-#pragma unroll 1
-        for (int q = 0; q < KS; ++q) {
-            const int kw = ch * KS + q;
-            // activations: row = this thread's pixel, all planes
-            uint32_t aw[AB];
+        uint32_t a_nxt[KS][AB], b_nxt[T::B_ITEMS];
+
+        // packed words of chunk `ch` -> registers (zero past the end, outside the image, past c_out)
+        auto load_chunk = [&](int ch) {
 #pragma unroll
-            for (int k = 0; k < AB; ++k) aw[k] = 0u;
-            if (kw < kwords) {
-                for (int f = 0; f < p.fold; ++f) {
-                    const int kk = kw * p.fold + f;
-                    if (kk >= p.KK) break;
-                    const int2 info = ktab[kk];
-                    if ((row_ok >> (info.y & 0xff)) & (col_ok >> (info.y >> 8)) & 1u) {
-                        uint32_t t[AB];
-                        load_words_global<AB>(p.x + (pix_off + info.x), t);
+            for (int q = 0; q < KS; ++q) {
+                const int kw = ch * KS + q;
 #pragma unroll
-                        for (int k = 0; k < AB; ++k) aw[k] |= t[k] << (f * p.fold_bits);
+                for (int k = 0; k < AB; ++k) a_nxt[q][k] = 0u;
+                if (((q * AB) & 1) == half || AB > 1) {           // this half uses at least one plane of word q
+                    if (kw < kwords) {
+                        for (int f = 0; f < p.fold; ++f) {
+                            const int kk = kw * p.fold + f;
+                            if (kk >= p.KK) break;
+                            const int2 info = ktab[kk];
+                            if ((row_ok >> (info.y & 0xff)) & (col_ok >> (info.y >> 8)) & 1u) {
+                                uint32_t t[AB];
+                                load_words_global<AB>(p.x + (pix_off + info.x), t);
+#pragma unroll
+                                for (int k = 0; k < AB; ++k) a_nxt[q][k] |= t[k] << (f * p.fold_bits);
+                            }
+                        }
                     }
                 }
             }
 #pragma unroll
-            for (int k = 0; k < AB; ++k) {
-                uint4 lo, hi;
-                expand_word_to_row(aw[k], k, 1u, lo, hi);
-                uint8_t* tile = A_st + (q * AB + k) * T::A_PLANE_BYTES;
-                *reinterpret_cast<uint4*>(sw32_chunk(tile, tid, 0)) = lo;
-                *reinterpret_cast<uint4*>(sw32_chunk(tile, tid, 1)) = hi;
-            }
-            // weights: TILE_N * WB rows shared out over the threads
-            for (int item = tid; item < TILE_N * WB; item += UMMA_M) {
-                const int m = item / TILE_N, nrow = item - m * TILE_N;
+            for (int i = 0; i < T::B_ITEMS; ++i) {
+                const int item = tid + i * UMMA_EXPANDERS;
+                const int q = item / (WB * TILE_N), rem = item - q * (WB * TILE_N);
+                const int m = rem / TILE_N, nrow = rem - m * TILE_N;
+                const int kw = ch * KS + q;
                 uint32_t ww = 0u;
-                if (kw < kwords && co0 + nrow < p.Co) {
+                if (q < KS && kw < kwords && co0 + nrow < p.Co) {
                     for (int f = 0; f < p.fold; ++f) {
                         const int kk = kw * p.fold + f;
                         if (kk >= p.KK) break;
                         ww |= __ldg(p.w + ((size_t)kk * p.Co + co0 + nrow) * WB + m) << (f * p.fold_bits);
                     }
                 }
-                const uint32_t scale = (m == WB - 1 && WB < 8) ? ((1u << (9 - WB)) - 1u) : 1u;
-                uint4 lo, hi;
-                expand_word_to_row(ww, m, scale, lo, hi);
-                uint8_t* tile = B_st + (q * WB + m) * T::B_PLANE_BYTES;
-                *reinterpret_cast<uint4*>(sw32_chunk(tile, nrow, 0)) = lo;
-                *reinterpret_cast<uint4*>(sw32_chunk(tile, nrow, 1)) = hi;
+                b_nxt[i] = ww;
             }
-        }
-        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");     // generic writes -> tensor-core reads
-        asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-        __syncthreads();
-        // ---- issue the MMAs of this chunk
-        if (tid == 0) {
-            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-            const uint32_t a_base = smem_u32(A_st), b_base = smem_u32(B_st);
-#pragma unroll 1
+        };
+
+        load_chunk(0);
+        for (int ch = 0; ch < nchunks; ++ch) {
+            const int st = ch & 1;
+            uint8_t* A_st = tiles + st * T::STAGE_BYTES;               // [KS][AB] planes of 128 rows x 32 B
+            uint8_t* B_st = A_st + KS * AB * T::A_PLANE_BYTES;         // [KS][WB] planes of TILE_N rows x 32 B
+            uint32_t a_cur[KS][AB], b_cur[T::B_ITEMS];
+#pragma unroll
+            for (int q = 0; q < KS; ++q)
+#pragma unroll
+                for (int k = 0; k < AB; ++k) a_cur[q][k] = a_nxt[q][k];
+#pragma unroll
+            for (int i = 0; i < T::B_ITEMS; ++i) b_cur[i] = b_nxt[i];
+            if (ch + 1 < nchunks) load_chunk(ch + 1);                   // in flight while this chunk is expanded
+            if (ch >= 2) {                                             // the MMAs of chunk ch-2 must have read the stage
+                if (!mbar_wait_bounded(&empty_bar[st], (uint32_t)(((ch >> 1) - 1) & 1), abortp)) break;
+            }
+#pragma unroll
             for (int q = 0; q < KS; ++q) {
-                if (ch * KS + q >= kwords) break;
-#pragma unroll 1
-                for (int m = 0; m < WB; ++m) {
-                    const uint64_t db = umma_desc_sw32(b_base + (q * WB + m) * T::B_PLANE_BYTES);
-#pragma unroll 1
-                    for (int k = 0; k < AB; ++k) {
-                        const uint64_t da = umma_desc_sw32(a_base + (q * AB + k) * T::A_PLANE_BYTES);
-                        const uint32_t accumulate = (ch | q | m | k) != 0 ? 1u : 0u;
-                        umma_i8(tmem_base, da, db, IDESC, accumulate);
-                    }
+#pragma unroll
+                for (int k = 0; k < AB; ++k) {
+                    if (((q * AB + k) & 1) != half) continue;
+                    uint4 lo, hi;
+                    expand_word_to_row(a_cur[q][k], k, 1u, lo, hi);
+                    uint8_t* tile = A_st + (q * AB + k) * T::A_PLANE_BYTES;
+                    *reinterpret_cast<uint4*>(sw32_chunk(tile, row, 0)) = lo;
+                    *reinterpret_cast<uint4*>(sw32_chunk(tile, row, 1)) = hi;
                 }
             }
-            umma_commit(&mbar[st]);
+#pragma unroll
+            for (int i = 0; i < T::B_ITEMS; ++i) {
+                const int item = tid + i * UMMA_EXPANDERS;
+                const int q = item / (WB * TILE_N), rem = item - q * (WB * TILE_N);
+                const int m = rem / TILE_N, nrow = rem - m * TILE_N;
+                if (q < KS) {
+                    const uint32_t scale = (m == WB - 1 && WB < 8) ? ((1u << (9 - WB)) - 1u) : 1u;
+                    uint4 lo, hi;
+                    expand_word_to_row(b_cur[i], m, scale, lo, hi);
+                    uint8_t* tile = B_st + (q * WB + m) * T::B_PLANE_BYTES;
+                    *reinterpret_cast<uint4*>(sw32_chunk(tile, nrow, 0)) = lo;
+                    *reinterpret_cast<uint4*>(sw32_chunk(tile, nrow, 1)) = hi;
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");     // generic writes -> tensor-core reads
+            mbar_arrive(&full_bar[st]);
+        }
+        // all MMAs done (the last commit covers every earlier one)
+        if (!*abortp) mbar_wait_bounded(&empty_bar[(nchunks - 1) & 1], (uint32_t)(((nchunks - 1) >> 1) & 1), abortp);
+    } else {
+        // =========================== issuer ===========================
+        constexpr uint32_t IDESC = umma_idesc_i8(TILE_N);
+        for (int ch = 0; ch < nchunks; ++ch) {
+            const int st = ch & 1;
+            if (!mbar_wait_bounded(&full_bar[st], (uint32_t)((ch >> 1) & 1), abortp)) break;
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            if ((tid & 31) == 0) {
+                const uint32_t a_base = smem_u32(tiles + st * T::STAGE_BYTES);
+                const uint32_t b_base = a_base + KS * AB * T::A_PLANE_BYTES;
+                const uint64_t da0 = umma_desc_sw32(a_base), db0 = umma_desc_sw32(b_base);
+#pragma unroll 1
+                for (int q = 0; q < KS; ++q) {
+                    if (ch * KS + q >= kwords) break;
+#pragma unroll 1
+                    for (int m = 0; m < WB; ++m) {
+                        const uint64_t db = db0 + (uint64_t)(((q * WB + m) * T::B_PLANE_BYTES) >> 4);
+#pragma unroll
+                        for (int k = 0; k < AB; ++k) {
+                            const uint64_t da = da0 + (uint64_t)(((q * AB + k) * T::A_PLANE_BYTES) >> 4);
+                            umma_i8(tmem_base, da, db, IDESC, (ch | q | m | k) != 0 ? 1u : 0u);
+                        }
+                    }
+                }
+                umma_commit(&empty_bar[st]);
+            }
+            __syncwarp();
         }
     }
 
-    // ---- wait for the last MMAs, then the epilogue straight out of tensor memory
-    if (!aborted) {
-        const int last = nchunks - 1;
-        bool ok = true;
-        if (tid == 0) ok = mbar_wait_bounded(&mbar[last & 1], (uint32_t)((last >> 1) & 1));
-        if (__syncthreads_or(!ok)) aborted = true;
-    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    const bool aborted = abort_flag != 0;
 
-    if (!aborted) {
+    // ---- epilogue straight out of tensor memory: warps w and w+4 own the same 32 pixels and split the channels
+    constexpr int EPI_WARPS = TILE_N >= 64 ? 8 : 4;
+    constexpr int COLS_PER_WARP = TILE_N >= 64 ? TILE_N / 2 : TILE_N;
+    if (!aborted && warp < EPI_WARPS) {
         const bool want_y = p.y != nullptr, want_q = p.packed_next != nullptr;
         const int qmax = (1 << p.next_bits) - 1;
         const bool pvalid = gp < p.P;
         const bool vec_ok = (p.Co & 3) == 0;                        // 16-byte aligned groups of four channels
-        const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
+        const uint32_t trow = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
         const int hw = p.Ho * p.Wo;
         const int img = pvalid ? gp / hw : 0, rem = pvalid ? gp - img * hw : 0;
+        const int cbeg = (warp >> 2) * COLS_PER_WARP;
         uint32_t planes[8];
 #pragma unroll 1
-        for (int c0 = 0; c0 < TILE_N; c0 += 16) {
+        for (int c0 = cbeg; c0 < cbeg + COLS_PER_WARP; c0 += 16) {
             uint32_t v[16];
             tmem_ld16(trow + (uint32_t)c0, v);                       // whole warp, also for rows past the end
             if ((c0 & 31) == 0) {
@@ -339,14 +397,13 @@ __global__ void __launch_bounds__(UMMA_M) conv_umma_kernel(const ConvParams p) {
                 }
             }
         }
-    } else if (tid == 0) {
-        atomicAdd(&g_umma_timeouts, 1ull);
     }
+    if (aborted && tid == 0) atomicAdd(&g_umma_timeouts, 1ull);
 
     // ---- release tensor memory (every path reaches this)
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 8) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"((uint32_t)T::TMEM_COLS)
                      : "memory");
     }
@@ -361,20 +418,20 @@ void launch_conv_umma(const ConvParams& p, dim3 grid, cudaStream_t st) {
                              T::SMEM_BYTES);
         attr_set = true;
     }
-    conv_umma_kernel<WB, AB, TILE_N><<<grid, UMMA_M, T::SMEM_BYTES, st>>>(p);
+    conv_umma_kernel<WB, AB, TILE_N><<<grid, UMMA_THREADS, T::SMEM_BYTES, st>>>(p);
 }
 
-constexpr int NUM_UMMA_VARIANTS = 4;           // TILE_N = 16, 32, 64, 128
+constexpr int NUM_UMMA_VARIANTS = 5;           // TILE_N = 16, 32, 64, 128, 256
 
 template <int WB, int AB, int VARIANT>
 constexpr ConvVariant make_umma_variant() {
     constexpr int TILE_N = 16 << VARIANT;
-    return ConvVariant{&launch_conv_umma<WB, AB, TILE_N>, UMMA_M, TILE_N, UMMA_M};
+    return ConvVariant{&launch_conv_umma<WB, AB, TILE_N>, UMMA_M, TILE_N, UMMA_THREADS};
 }
 
 #define EBS_UMMA_ROW(WB, AB)                                                                              \
     {make_umma_variant<WB, AB, 0>(), make_umma_variant<WB, AB, 1>(), make_umma_variant<WB, AB, 2>(),      \
-     make_umma_variant<WB, AB, 3>()}
+     make_umma_variant<WB, AB, 3>(), make_umma_variant<WB, AB, 4>()}
 
 #define EBS_DEFINE_UMMA_TABLE(WB)                                                                         \
     const ConvVariant* conv_umma_variant_w##WB(int a_bits, int variant) {                                 \

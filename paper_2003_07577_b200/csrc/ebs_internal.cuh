@@ -57,7 +57,7 @@ EBS_DECLARE_WB(5) EBS_DECLARE_WB(6) EBS_DECLARE_WB(7) EBS_DECLARE_WB(8)
 #undef EBS_DECLARE_WB
 
 // 5th-generation tensor-core kernels (conv_umma_w1.cu .. conv_umma_w8.cu); variant = log2(tile_n / 16).
-enum { NUM_CONV_UMMA_VARIANTS = 4 };
+enum { NUM_CONV_UMMA_VARIANTS = 5 };
 const ConvVariant* conv_umma_variant(int w_bits, int a_bits, int variant);
 unsigned long long conv_umma_timeouts();
 #define EBS_DECLARE_WB(WB)                                                   \

@@ -90,7 +90,7 @@ def test_conv_all_bitwidth_pairs(ebs, U, oracle, wb, ab):
     d = U.desc_for(40, 21, 3, 1, 1, wb, ab)
     ref = oracle.conv2d_codes(qa, qw, (1, 1), (1, 1))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
-    for variant in (-1, 0, 4, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22):
+    for variant in (-1, 0, 4, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23):
         got = U.run_conv(qa, qw, d, variant=variant, px=px, pw=pw)["acc"]
         assert np.array_equal(got, ref), f"variant {variant}"
 
@@ -181,7 +181,7 @@ def test_fused_epilogue_and_requantized_planes(ebs, U, oracle, next_bits, co):
     res_nhwc = to(res.transpose(0, 2, 3, 1))
     for y_layout in (ebs.EBS_NHWC, ebs.EBS_NCHW):
         epi = ebs.epilogue(to(cs), to(cb), res_nhwc, True, next_bits, float(next_scale), y_layout)
-        for variant in (-1, 3, 6, 7, 11, 12, 14, 15, 17, 18, 20, 21, 22):
+        for variant in (-1, 3, 6, 7, 11, 12, 14, 15, 17, 18, 20, 21, 22, 23):
             out = U.run_conv(qa, qw, d, epi, want_acc=True, want_y=True, next_bits=next_bits, variant=variant)
             assert np.array_equal(out["acc"], ref_acc)
             assert np.allclose(out["y"], y_ref, rtol=RTOL, atol=0.0)
