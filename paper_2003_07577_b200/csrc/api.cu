@@ -125,6 +125,19 @@ static int choose_mma_variant(int w_bits, int a_bits, int P, int Co, int sms) {
     return 6 + tc_idx;
 }
 
+// tcgen05 kernels pay off when a CTA's 128 x tile_n accumulator sees many MMAs (deep reduction, several
+// plane pairs), the channel tile is wide enough to amortise the activation expansion, and the layer
+// has enough output tiles; smaller layers run faster on the warp-level kernels.  (Rule fitted to
+// per-variant timings of the ResNet-18/20/50 layer shapes.)  Returns the umma variant or -1.
+static int choose_umma_variant(const ConvParams& p, const ebs_conv_desc* d) {
+    const int kwords = (p.KK + p.fold - 1) / p.fold;
+    const long long mmas_per_tile = (long long)kwords * d->w_bits * d->a_bits;
+    const long long outputs = (long long)p.P * p.Co;
+    if (p.Co < 64 || mmas_per_tile < 48) return -1;
+    if (outputs < (1LL << 20) && kwords < 72) return -1;
+    return p.Co >= 128 ? 3 : 2;             // tile_n 128 or 64
+}
+
 static int conv_impl(const void* packed_x, int n, int h, int w, const void* packed_w, const ebs_conv_desc* d,
                      const ebs_epilogue* epi, int32_t* acc_out, float* y_out, void* packed_next, void* stream,
                      int variant) {
@@ -172,8 +185,10 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
     }
     const bool mma_ok = mma_path_supported(p, d);
     if (variant < 0) {
-        variant = mma_ok ? NUM_CONV_VARIANTS + choose_mma_variant(d->w_bits, d->a_bits, p.P, p.Co, sm_count())
-                         : choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
+        const int umma = mma_ok ? choose_umma_variant(p, d) : -1;
+        if (umma >= 0) variant = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + umma;
+        else variant = mma_ok ? NUM_CONV_VARIANTS + choose_mma_variant(d->w_bits, d->a_bits, p.P, p.Co, sm_count())
+                              : choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
     }
     if (variant >= NUM_CONV_VARIANTS && !mma_ok) return EBS_ERR_UNSUPPORTED;
     const ConvVariant* v =
