@@ -30,6 +30,16 @@ from workloads import gen  # noqa: E402
 METRIC = "effective binary TOPS (2*MACs*Wb*Ab per second), ResNet-20 CIFAR quantized conv stack"
 UNIT = "TOPS"
 WORKLOAD = "config2: ResNet-20 CIFAR-shaped stack, 20 quantized convs, batch 128, (Wb,Ab) in {1..4}^2, seed 0"
+# other workloads of the same path, for profiling and for the results table (the default is config2)
+WORKLOADS = {
+    "config2": (WORKLOAD, lambda: [s for s in gen.config2(0) if s.layer.quantized]),
+    "config1": ("config1: one 3x3 conv 64->64, 32x32, batch 1, W2A2, seed 0", lambda: gen.config1(0)),
+    "config3": ("config3: ResNet-18 ImageNet-shaped quantized convs, batch 64, (Wb,Ab) in {2..6}^2, seed 0",
+                lambda: gen.config3(0)),
+    "config5": ("config5: ResNet-50 ImageNet-shaped bottleneck stack, batch 256, (Wb,Ab) in {2..8}^2, seed 0 "
+                "(layers run with independent inputs here; the chained run is a parity test)",
+                lambda: gen.config5(0)),
+}
 SM_COUNT, POPC_LANES_PER_CLK_SM = 148, 16
 # dram__bytes_read.sum + dram__bytes_write.sum per conv launch, mean over the 20 layers, from the ncu
 # capture summarised in profiles/ (outputs stay in the 126 MB L2 while ncu replays a launch)
@@ -243,7 +253,8 @@ def run_gpu(args):
     torch.cuda.set_device(dev)
     peaks, peak_kind = measured_peaks()
 
-    specs = [s for s in gen.config2(0) if s.layer.quantized]        # every rank: one full batch (weak scaling)
+    workload_text, make_specs = WORKLOADS[args.workload]
+    specs = make_specs()                                            # every rank: one full batch (weak scaling)
     if args.only:                                                   # profiling aid: a subset of the layers
         specs = [s for s in specs if s.layer.name in args.only.split(",")]
     layers = [Layer(ebs, s, specs[(i + 1) % len(specs)].a_bits, dev) for i, s in enumerate(specs)]
@@ -363,7 +374,8 @@ def run_gpu(args):
         "metric": METRIC, "value": world * total_ops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-        "config": {"workload": WORKLOAD + (f" [only {args.only}]" if args.only else ""), "global_batch": 128 * world, "imgs_per_s": world * 128 / (ms_per_step * 1e-3),
+        "config": {"workload": workload_text + (f" [only {args.only}]" if args.only else ""), "global_batch": specs[0].batch * world,
+                   "imgs_per_s": world * specs[0].batch / (ms_per_step * 1e-3),
                    "l2": "256 MB buffer rewritten before every timed step (cold L2)",
                    "launch": "each step is one CUDA-graph replay of its 60 kernel launches",
                    "step": "per layer: ebs_pack_acts(u8 NHWC) + ebs_conv2d_mixed(acc + packed_next) + ebs_dequant",
@@ -373,10 +385,11 @@ def run_gpu(args):
                 "h2d_bytes_per_step": int(sum(L.x_host.numel() for L in layers)),
                 "d2h_bytes_per_step": int(sum(L.pn_bytes for L in layers)),
                 "note": "ebs_conv2d_mixed_host per layer: pinned u8 codes in, packed next-layer planes out; wall clock"},
-        "gpu_launches": 3 * len(layers) * args.steps,
-        "roofline": {"bound": "tensor", "kernel": "conv_mma_kernel (int8 mma.sync on bit planes)",
+        "gpu_launches": 3 * len(layers) * args.steps, "device_wait_timeouts": ebs.ebs_device_wait_timeouts(),
+        "roofline": {"bound": "tensor",
+                     "kernel": "bit-plane conv on the int8 tensor pipe (conv_mma_kernel: mma.sync; conv_umma_kernel: tcgen05)",
                      "achieved": achieved, "peak": peak_tops, "unit": "TOPS", "frac": achieved / peak_tops,
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if args.workload == "config2" and not args.only else None,
                      "peak_source": f"int8 dense = 2 x bf16 burst ({peaks.get('bf16_tflops')} TFLOP/s, {peak_kind}); "
                                     "one bit-pair AND+bitcount is one byte multiply-accumulate = 2 ops",
                      "conv_ms_per_step": conv_total_ms, "conv_launches_per_step": len(layers),
@@ -401,6 +414,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS), help="default: the bench workload")
     ap.add_argument("--only", default="", help="comma-separated layer names: restrict the step to these layers (for profiling)")
     args = ap.parse_args()
     if args.impl == "reference":
