@@ -197,6 +197,24 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
         }
         uint32_t a_nxt[KS][AB], b_nxt[T::B_ITEMS];
 
+        // per-thread constants of the weight rows it expands: which (reduction word, plane, channel row),
+        // where that row starts in global memory (for reduction word 0) and in the stage
+        int b_q[T::B_ITEMS], b_m[T::B_ITEMS], b_goff[T::B_ITEMS], b_soff[T::B_ITEMS];
+#pragma unroll
+        for (int i = 0; i < T::B_ITEMS; ++i) {
+            const int item = tid + i * UMMA_EXPANDERS;
+            const int q = item / (WB * TILE_N), rem = item - q * (WB * TILE_N);
+            const int m = rem / TILE_N, nrow = rem - m * TILE_N;
+            const bool live = q < KS && co0 + nrow < p.Co;
+            b_q[i] = q < KS ? q : -1;                            // -1: no row (more threads than rows)
+            b_m[i] = m;
+            b_goff[i] = live ? (co0 + nrow) * WB + m : -1;        // -1: channel past c_out -> zero row
+            b_soff[i] = KS * AB * T::A_PLANE_BYTES + (q * WB + m) * T::B_PLANE_BYTES + nrow * 32;
+        }
+        const int sw = ((row >> 2) & 1) << 4;                     // 32-byte swizzle of this thread's pixel row
+        const int a_soff0 = row * 32 + sw, a_soff1 = row * 32 + (sw ^ 16);
+        const int co_wb = p.Co * WB;                              // weight words per reduction word
+
         // packed words of chunk `ch` -> registers (zero past the end, outside the image, past c_out)
         auto load_chunk = [&](int ch) {
 #pragma unroll
@@ -204,8 +222,12 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
                 const int kw = ch * KS + q;
 #pragma unroll
                 for (int k = 0; k < AB; ++k) a_nxt[q][k] = 0u;
-                if (((q * AB) & 1) == half || AB > 1) {           // this half uses at least one plane of word q
-                    if (kw < kwords) {
+                if ((((q * AB) & 1) == half || AB > 1) && kw < kwords) {     // this half uses a plane of word q
+                    if (p.fold == 1) {
+                        const int2 info = ktab[kw];
+                        if ((row_ok >> (info.y & 0xff)) & (col_ok >> (info.y >> 8)) & 1u)
+                            load_words_global<AB>(p.x + (pix_off + info.x), a_nxt[q]);
+                    } else {
                         for (int f = 0; f < p.fold; ++f) {
                             const int kk = kw * p.fold + f;
                             if (kk >= p.KK) break;
@@ -222,16 +244,17 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
             }
 #pragma unroll
             for (int i = 0; i < T::B_ITEMS; ++i) {
-                const int item = tid + i * UMMA_EXPANDERS;
-                const int q = item / (WB * TILE_N), rem = item - q * (WB * TILE_N);
-                const int m = rem / TILE_N, nrow = rem - m * TILE_N;
-                const int kw = ch * KS + q;
                 uint32_t ww = 0u;
-                if (q < KS && kw < kwords && co0 + nrow < p.Co) {
-                    for (int f = 0; f < p.fold; ++f) {
-                        const int kk = kw * p.fold + f;
-                        if (kk >= p.KK) break;
-                        ww |= __ldg(p.w + ((size_t)kk * p.Co + co0 + nrow) * WB + m) << (f * p.fold_bits);
+                const int kw = ch * KS + b_q[i];
+                if (b_q[i] >= 0 && b_goff[i] >= 0 && kw < kwords) {
+                    if (p.fold == 1) {
+                        ww = __ldg(p.w + (size_t)kw * co_wb + b_goff[i]);
+                    } else {
+                        for (int f = 0; f < p.fold; ++f) {
+                            const int kk = kw * p.fold + f;
+                            if (kk >= p.KK) break;
+                            ww |= __ldg(p.w + (size_t)kk * co_wb + b_goff[i]) << (f * p.fold_bits);
+                        }
                     }
                 }
                 b_nxt[i] = ww;
@@ -241,8 +264,8 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
         load_chunk(0);
         for (int ch = 0; ch < nchunks; ++ch) {
             const int st = ch & 1;
-            uint8_t* A_st = tiles + st * T::STAGE_BYTES;               // [KS][AB] planes of 128 rows x 32 B
-            uint8_t* B_st = A_st + KS * AB * T::A_PLANE_BYTES;         // [KS][WB] planes of TILE_N rows x 32 B
+            uint8_t* A_st = tiles + st * T::STAGE_BYTES;               // [KS][AB] planes of 128 rows x 32 B, then
+                                                                       // [KS][WB] planes of TILE_N rows x 32 B
             uint32_t a_cur[KS][AB], b_cur[T::B_ITEMS];
 #pragma unroll
             for (int q = 0; q < KS; ++q)
@@ -262,22 +285,25 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
                     uint4 lo, hi;
                     expand_word_to_row(a_cur[q][k], k, 1u, lo, hi);
                     uint8_t* tile = A_st + (q * AB + k) * T::A_PLANE_BYTES;
-                    *reinterpret_cast<uint4*>(sw32_chunk(tile, row, 0)) = lo;
-                    *reinterpret_cast<uint4*>(sw32_chunk(tile, row, 1)) = hi;
+                    *reinterpret_cast<uint4*>(tile + a_soff0) = lo;
+                    *reinterpret_cast<uint4*>(tile + a_soff1) = hi;
                 }
             }
 #pragma unroll
             for (int i = 0; i < T::B_ITEMS; ++i) {
-                const int item = tid + i * UMMA_EXPANDERS;
-                const int q = item / (WB * TILE_N), rem = item - q * (WB * TILE_N);
-                const int m = rem / TILE_N, nrow = rem - m * TILE_N;
-                if (q < KS) {
+                if (b_q[i] >= 0) {
+                    const int m = b_m[i];
+                    // rotate once by the plane, then the eight byte groups are fixed rotations of that
+                    const uint32_t wrot = __funnelshift_l(b_cur[i], b_cur[i], m);
+                    const uint32_t mask = 0x01010101u << m;
                     const uint32_t scale = (m == WB - 1 && WB < 8) ? ((1u << (9 - WB)) - 1u) : 1u;
-                    uint4 lo, hi;
-                    expand_word_to_row(b_cur[i], m, scale, lo, hi);
-                    uint8_t* tile = B_st + (q * WB + m) * T::B_PLANE_BYTES;
-                    *reinterpret_cast<uint4*>(sw32_chunk(tile, nrow, 0)) = lo;
-                    *reinterpret_cast<uint4*>(sw32_chunk(tile, nrow, 1)) = hi;
+                    uint32_t r[8];
+#pragma unroll
+                    for (int bb = 0; bb < 8; ++bb) r[bb] = (__funnelshift_r(wrot, wrot, bb) & mask) * scale;
+                    uint8_t* dst = A_st + b_soff[i];
+                    const int bsw = (b_soff[i] >> 3) & 16;               // ((row >> 2) & 1) << 4 with row = offset / 32
+                    *reinterpret_cast<uint4*>(dst + bsw) = make_uint4(r[0], r[1], r[2], r[3]);
+                    *reinterpret_cast<uint4*>(dst + (bsw ^ 16)) = make_uint4(r[4], r[5], r[6], r[7]);
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");     // generic writes -> tensor-core reads
