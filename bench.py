@@ -59,6 +59,10 @@ def int8_tensor_peak_tops(peaks: dict) -> float:
     return 2.0 * float(peaks.get("bf16_tflops", 1590.0))
 
 
+def hbm_gbs_for_streaming(peaks: dict) -> float:
+    return float(peaks.get("hbm_gbs", 6650.0))
+
+
 def popc_pipe_peak_tops(sm_max_mhz: float) -> float:
     """Binary TOPS of the POPC pipe: 16 lanes/clk/SM x 32 bit x 148 SMs x clock, 2 ops per bit pair."""
     return 2.0 * SM_COUNT * POPC_LANES_PER_CLK_SM * 32 * sm_max_mhz * 1e6 / 1e12
@@ -331,6 +335,42 @@ def run_gpu(args):
         torch.cuda.synchronize()
         conv_ms[i] = e0.elapsed_time(e1) / 10.0
 
+    # the streaming kernels (rows a2 and a6) on a tensor far larger than L2: achieved GB/s of algorithmic bytes
+    streaming = {}
+    if world == 1:
+        sn, sh, sc, sab = 256, 56, 64, 4                                   # ResNet-50 layer-1 activations: 51 M values, inputs > L2
+        vals = sn * sh * sh * sc
+        xf = torch.rand((sn, sh, sh, sc), dtype=torch.float32, device=dev)
+        xu = torch.randint(0, 16, (sn, sh, sh, sc), dtype=torch.uint8, device=dev)
+        pk = torch.empty(ebs.ebs_packed_act_bytes(sn, sh, sh, sc, sab) // 4, dtype=torch.int32, device=dev)
+        ai = torch.randint(-1000, 1000, (sn * sh * sh, sc), dtype=torch.int32, device=dev)
+        yo = torch.empty((sn * sh * sh, sc), dtype=torch.float32, device=dev)
+
+        def gbs(fn, nbytes, reps=10):
+            fn()
+            tot = 0.0
+            for _ in range(reps):                                       # inputs are larger than L2: no flush needed
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                torch.cuda.synchronize()
+                tot += a.elapsed_time(b)
+            return nbytes / (tot / reps * 1e-3) / 1e9
+
+        out_b = vals * sab // 8
+        streaming = {
+            "tensor": f"{sn}x{sh}x{sh}x{sc} NHWC, {sab} planes", "hbm_peak_gbs": hbm_gbs_for_streaming(peaks),
+            "pack_acts_fp32_gbs": gbs(lambda: ebs.ebs_pack_acts(xf, ebs.EBS_F32, ebs.EBS_NHWC, sn, sc, sh, sh, sab, 0.07, pk),
+                                      vals * 4 + out_b),
+            "pack_acts_u8_gbs": gbs(lambda: ebs.ebs_pack_acts(xu, ebs.EBS_U8_CODES, ebs.EBS_NHWC, sn, sc, sh, sh, sab, 1.0, pk),
+                                    vals + out_b),
+            "pack_acts_fp32_nchw_gbs": gbs(lambda: ebs.ebs_pack_acts(xf, ebs.EBS_F32, ebs.EBS_NCHW, sn, sc, sh, sh, sab, 0.07, pk),
+                                           vals * 4 + out_b),
+            "dequant_gbs": gbs(lambda: ebs.ebs_dequant(ai, sn * sh * sh, sc, 0.01, None, None, True, yo), vals * 8),
+        }
+        del xf, xu, pk, ai, yo
+
     # end to end through the host entry point: pinned host codes in, packed planes out, every step
     e2e_steps = max(3, min(args.steps, 10))
     for L in layers:
@@ -400,6 +440,7 @@ def run_gpu(args):
                      "per_layer_note": "per-layer times are L2-warm (10 back-to-back launches in a graph); "
                                        "roof = max(ops / tensor peak, algorithmic bytes / HBM peak)",
                      "per_layer": per_layer},
+        "streaming_kernels": streaming,
         "wall_s_timed_region": wall,
     }
     if cpu is not None:

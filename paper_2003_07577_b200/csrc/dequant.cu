@@ -22,15 +22,25 @@ __global__ void __launch_bounds__(256) dequant_kernel(const int32_t* __restrict_
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     if constexpr (VEC == 4) {
         const size_t nvec = total / 4;
-        for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += stride) {
-            const int4 a = __ldg(reinterpret_cast<const int4*>(acc) + v);
-            const int co = (int)((v * 4) % (size_t)c_out);
-            float4 o;
-            o.x = dequant_one(a.x, co, scale, ch_scale, ch_bias, relu);
-            o.y = dequant_one(a.y, co + 1, scale, ch_scale, ch_bias, relu);
-            o.z = dequant_one(a.z, co + 2, scale, ch_scale, ch_bias, relu);
-            o.w = dequant_one(a.w, co + 3, scale, ch_scale, ch_bias, relu);
-            reinterpret_cast<float4*>(y)[v] = o;
+        constexpr int U = 4;                                   // independent 16-byte loads in flight per thread
+        for (size_t v0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v0 < nvec; v0 += stride * U) {
+            int4 a[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (v0 + u * stride < nvec) a[u] = __ldg(reinterpret_cast<const int4*>(acc) + v0 + u * stride);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const size_t v = v0 + u * stride;
+                if (v < nvec) {
+                    const int co = (int)((v * 4) % (size_t)c_out);
+                    float4 o;
+                    o.x = dequant_one(a[u].x, co, scale, ch_scale, ch_bias, relu);
+                    o.y = dequant_one(a[u].y, co + 1, scale, ch_scale, ch_bias, relu);
+                    o.z = dequant_one(a[u].z, co + 2, scale, ch_scale, ch_bias, relu);
+                    o.w = dequant_one(a[u].w, co + 3, scale, ch_scale, ch_bias, relu);
+                    reinterpret_cast<float4*>(y)[v] = o;
+                }
+            }
         }
     } else {
         for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride)
@@ -46,7 +56,7 @@ int launch_dequant(const int32_t* acc, size_t n_pixels, int c_out, float scale, 
     const bool vec = (c_out % 4) == 0;
     const size_t work = vec ? total / 4 : total;
     size_t blocks = (work + 255) / 256;
-    const size_t cap = (size_t)sms * 8;
+    const size_t cap = (size_t)sms * 16;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     if (vec) dequant_kernel<4><<<(int)blocks, 256, 0, st>>>(acc, total, c_out, scale, ch_scale, ch_bias, relu, y);

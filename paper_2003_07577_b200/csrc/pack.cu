@@ -1,9 +1,10 @@
 // Quantize + bit-plane packing kernels (Eq. 1b/1c quantizer; B_x and B_w of Eq. 12/15).
 //
-// A warp turns 32 consecutive channels of one pixel into a_bits words with one __ballot_sync per
-// plane: lane = channel, so bit (c % 32) of a plane word is that plane's bit of channel c.  The
-// kernels are pure streaming (HBM-bound): 4 bytes (fp32) or 1 byte (codes) read per element,
-// a_bits/8 bytes written.
+// The activation kernels give one thread the 32 codes of a (pixel, 32-channel word), four code bytes
+// to a register, and gather plane j of four codes into a nibble with one multiply; bit (c % 32) of a
+// plane word is that plane's bit of channel c.  They are pure streaming (HBM-bound): 4 bytes (fp32)
+// or 1 byte (codes) read per element, a_bits/8 bytes written.  The weight kernel (off the inference
+// path) uses one warp per word and a __ballot_sync per plane.
 #include "ebs_internal.cuh"
 
 namespace ebs {
@@ -19,30 +20,7 @@ __device__ __forceinline__ uint32_t act_code<uint8_t>(uint8_t v, float, int qmax
     return (uint32_t)v & (uint32_t)qmax;
 }
 
-// NHWC input: items are (pixel, channel word); one warp per item, grid-stride.
-template <typename T>
-__global__ void __launch_bounds__(256) pack_acts_nhwc_kernel(const T* __restrict__ x, long long pixels, int C,
-                                                             int CW, int AB, float inv_scale,
-                                                             uint32_t* __restrict__ out) {
-    const int lane = threadIdx.x & 31;
-    const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
-    const long long items = pixels * CW;
-    const int qmax = (1 << AB) - 1;
-    for (long long item = warp0; item < items; item += nwarps) {
-        const long long pix = item / CW;
-        const int cw = (int)(item - pix * CW);
-        const int c = cw * 32 + lane;
-        uint32_t code = 0u;
-        if (c < C) code = act_code<T>(x[pix * C + c], inv_scale, qmax);
-        uint32_t mine = 0u;
-        for (int j = 0; j < AB; ++j) {
-            const uint32_t word = __ballot_sync(0xffffffffu, (code >> j) & 1u);
-            if (lane == j) mine = word;
-        }
-        if (lane < AB) out[item * AB + lane] = mine;
-    }
-}
+__device__ __forceinline__ void store_planes(const uint32_t (&codes)[8], int AB, uint32_t* __restrict__ dst);
 
 // NHWC integer codes: one thread per (pixel, 32-channel word).  The thread reads its 32 code bytes
 // as 16-byte vectors and gathers plane j of four codes at a time into a nibble with one multiply
@@ -78,53 +56,187 @@ __global__ void __launch_bounds__(256) pack_acts_nhwc_u8_kernel(const uint8_t* _
                 codes[k] = wv;
             }
         }
-        uint32_t* dst = out + item * AB;
-        for (int j = 0; j < AB; ++j) {
-            uint32_t word = 0u;
+        store_planes(codes, AB, out + item * AB);
+    }
+}
+
+// Plane words of 32 codes held as eight words of four code bytes each.
+__device__ __forceinline__ void store_planes(const uint32_t (&codes)[8], int AB, uint32_t* __restrict__ dst) {
+    uint32_t w[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        uint32_t word = 0u;
+        if (j < AB) {
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 const uint32_t t = (codes[k] >> j) & 0x01010101u;
                 word |= ((t * 0x01020408u) >> 24) << (4 * k);
             }
-            dst[j] = word;
         }
+        w[j] = word;
+    }
+    if (AB == 4) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+    else if (AB == 8) {
+        *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(dst + 4) = make_uint4(w[4], w[5], w[6], w[7]);
+    } else if (AB == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
+    else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (j < AB) dst[j] = w[j];
     }
 }
 
-// NCHW input: a CTA transposes a [32 channels][32 pixels] tile through shared memory so that
-// global reads run along the contiguous pixel axis and the ballot still sees lane = channel.
+// NHWC, channels a multiple of 32: a warp takes 32 consecutive (pixel, 32-channel word) items, i.e.
+// 1024 consecutive values.  Loads are fully coalesced (lane l reads 16-byte chunk i*32+l of the run),
+// each chunk is quantized (fp32) and reduced to one word of four code bytes, the words are regrouped
+// through shared memory so that lane l holds the eight code words of item l, and the lane builds the
+// plane words with the multiply-gather.
+__global__ void __launch_bounds__(256) pack_acts_nhwc_f32_coalesced_kernel(const float* __restrict__ x, long long items, int AB,
+                                                                       float inv_scale, uint32_t* __restrict__ out) {
+    __shared__ uint32_t regroup[8][32][9];                    // [warp][item][code word], padded
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    const int qmax = (1 << AB) - 1;
+    const long long groups = (items + 31) / 32;
+    for (long long grp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; grp < groups; grp += nwarps) {
+        const long long item0 = grp * 32;
+        const long long left = items - item0;
+        const int nitems = left < 32 ? (int)left : 32;
+        {
+            const float4* src = reinterpret_cast<const float4*>(x + item0 * 32);
+            float4 v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int chunk = i * 32 + lane;                  // 16-byte chunk of the run: item chunk/8, word chunk%8
+                v[i] = (chunk >> 3) < nitems ? __ldg(src + chunk) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int chunk = i * 32 + lane;
+                regroup[warp][chunk >> 3][chunk & 7] =
+                    (uint32_t)quantize_act_code(v[i].x, inv_scale, qmax) | ((uint32_t)quantize_act_code(v[i].y, inv_scale, qmax) << 8) |
+                    ((uint32_t)quantize_act_code(v[i].z, inv_scale, qmax) << 16) | ((uint32_t)quantize_act_code(v[i].w, inv_scale, qmax) << 24);
+            }
+        }
+        __syncwarp();
+        if (lane < nitems) {
+            uint32_t codes[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) codes[k] = regroup[warp][lane][k];
+            store_planes(codes, AB, out + (item0 + lane) * AB);
+        }
+        __syncwarp();
+    }
+}
+
+// Same for integer codes; a warp takes 128 items (4 KB) per iteration so that enough loads are in flight.
+__global__ void __launch_bounds__(256) pack_acts_nhwc_u8_coalesced_kernel(const uint8_t* __restrict__ x, long long items,
+                                                                          int AB, uint32_t* __restrict__ out) {
+    constexpr int G = 4;                                       // groups of 32 items per warp iteration
+    __shared__ uint32_t regroup[8][G * 32][9];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    const long long groups = (items + G * 32 - 1) / (G * 32);
+    for (long long grp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; grp < groups; grp += nwarps) {
+        const long long item0 = grp * (G * 32);
+        const long long left = items - item0;
+        const int nitems = left < G * 32 ? (int)left : G * 32;
+        const uint4* src = reinterpret_cast<const uint4*>(x + item0 * 32);
+        uint4 v[2 * G];
+#pragma unroll
+        for (int i = 0; i < 2 * G; ++i) {
+            const int chunk = i * 32 + lane;                      // 16-byte chunk: item chunk/2, code words 4*(chunk%2)..
+            v[i] = (chunk >> 1) < nitems ? __ldg(src + chunk) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int i = 0; i < 2 * G; ++i) {
+            const int chunk = i * 32 + lane;
+            uint32_t* dst = &regroup[warp][chunk >> 1][(chunk & 1) * 4];
+            dst[0] = v[i].x; dst[1] = v[i].y; dst[2] = v[i].z; dst[3] = v[i].w;
+        }
+        __syncwarp();
+#pragma unroll
+        for (int gq = 0; gq < G; ++gq) {
+            const int it = gq * 32 + lane;
+            if (it < nitems) {
+                uint32_t codes[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) codes[k] = regroup[warp][it][k];
+                store_planes(codes, AB, out + (item0 + it) * AB);
+            }
+        }
+        __syncwarp();
+    }
+}
+
+// NHWC fp32, any channel count: one thread per (pixel, 32-channel word).
+__global__ void __launch_bounds__(256) pack_acts_nhwc_f32_kernel(const float* __restrict__ x, long long items, int C,
+                                                                 int CW, int AB, float inv_scale,
+                                                                 uint32_t* __restrict__ out) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const int qmax = (1 << AB) - 1;
+    const bool vec = (C % 4) == 0;
+    for (long long item = (long long)blockIdx.x * blockDim.x + threadIdx.x; item < items; item += stride) {
+        const long long pix = item / CW;
+        const int cw = (int)(item - pix * CW);
+        const int c0 = cw * 32;
+        const int nvalid = C - c0 < 32 ? C - c0 : 32;
+        const float* src = x + pix * C + c0;
+        uint32_t codes[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            uint32_t wv = 0u;
+            if (vec) {
+                if (4 * k < nvalid) {
+                    const float4 v = __ldg(reinterpret_cast<const float4*>(src) + k);
+                    wv = (uint32_t)quantize_act_code(v.x, inv_scale, qmax) | ((uint32_t)quantize_act_code(v.y, inv_scale, qmax) << 8) |
+                         ((uint32_t)quantize_act_code(v.z, inv_scale, qmax) << 16) | ((uint32_t)quantize_act_code(v.w, inv_scale, qmax) << 24);
+                }
+            } else {
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+                    if (4 * k + b < nvalid)
+                        wv |= (uint32_t)quantize_act_code(__ldg(src + 4 * k + b), inv_scale, qmax) << (8 * b);
+            }
+            codes[k] = wv;
+        }
+        store_planes(codes, AB, out + item * AB);
+    }
+}
+
+// NCHW input (fp32 or codes): a CTA takes 32 channels x 128 pixels; global reads run along the
+// contiguous pixel axis, the codes are transposed through shared memory (one byte each), then one
+// thread per pixel gathers its 32 codes and builds the plane words.
 template <typename T>
-__global__ void __launch_bounds__(256) pack_acts_nchw_kernel(const T* __restrict__ x, int N, int C, int HW,
+__global__ void __launch_bounds__(128) pack_acts_nchw_kernel(const T* __restrict__ x, int N, int C, int HW,
                                                              int CW, int AB, float inv_scale,
                                                              uint32_t* __restrict__ out) {
-    __shared__ uint32_t tile[32][33];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int ptiles = (HW + 31) / 32;
+    constexpr int PT = 128, ROWB = 36;                       // pixels per tile; bytes per pixel row (32 codes + pad)
+    __shared__ __align__(16) uint8_t tile[PT * ROWB];
+    const int ptiles = (HW + PT - 1) / PT;
     const long long tiles = (long long)N * CW * ptiles;
     const int qmax = (1 << AB) - 1;
     for (long long tix = blockIdx.x; tix < tiles; tix += gridDim.x) {
         const int pt = (int)(tix % ptiles);
         const long long rest = tix / ptiles;
         const int cw = (int)(rest % CW), n = (int)(rest / CW);
-        const int p0 = pt * 32;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int cl = warp * 4 + k, c = cw * 32 + cl, pp = p0 + lane;
+        const int p0 = pt * PT;
+        for (int e = threadIdx.x; e < 32 * PT; e += 128) {   // e -> (channel, pixel): consecutive threads, consecutive pixels
+            const int cl = e / PT, pl = e - cl * PT;
+            const int c = cw * 32 + cl, pp = p0 + pl;
             uint32_t code = 0u;
             if (c < C && pp < HW) code = act_code<T>(x[((long long)n * C + c) * HW + pp], inv_scale, qmax);
-            tile[cl][lane] = code;
+            tile[pl * ROWB + cl] = (uint8_t)code;
         }
         __syncthreads();
+        const int pp = p0 + threadIdx.x;
+        if (pp < HW) {
+            const uint32_t* row = reinterpret_cast<const uint32_t*>(tile + threadIdx.x * ROWB);
+            uint32_t codes[8];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int pl = warp * 4 + k, pp = p0 + pl;
-            const uint32_t code = tile[lane][pl];
-            uint32_t mine = 0u;
-            for (int j = 0; j < AB; ++j) {
-                const uint32_t word = __ballot_sync(0xffffffffu, (code >> j) & 1u);
-                if (lane == j) mine = word;
-            }
-            if (pp < HW && lane < AB) out[(((long long)n * HW + pp) * CW + cw) * AB + lane] = mine;
+            for (int k = 0; k < 8; ++k) codes[k] = row[k];
+            store_planes(codes, AB, out + (((long long)n * HW + pp) * CW + cw) * AB);
         }
         __syncthreads();
     }
@@ -186,22 +298,34 @@ int launch_pack_acts(const void* x, int dtype, int layout, int n, int c, int h, 
     const int sms = sm_count();
     if (layout == EBS_NHWC) {
         const int grid = grid_for(pixels * CW, sms);
-        if (dtype == EBS_F32)
-            pack_acts_nhwc_kernel<float><<<grid, 256, 0, st>>>((const float*)x, pixels, c, CW, a_bits, inv_scale, out);
-        else {
-            const long long items = pixels * CW;
-            long long blocks = (items + 255) / 256;
-            if (blocks > (long long)sms * 32) blocks = (long long)sms * 32;
+        const long long items = pixels * CW;
+        long long blocks = (items + 255) / 256;
+        if (blocks > (long long)sms * 32) blocks = (long long)sms * 32;
+        (void)grid;
+        if (c % 32 == 0 && (dtype == EBS_F32 || items >= (1LL << 20))) {   // full, aligned runs of 32 values; small
+                                                                             // code tensors are latency-bound and
+                                                                             // do better with a thread per word
+            long long wblocks = ((items + 31) / 32 + 7) / 8;
+            if (wblocks > (long long)sms * 32) wblocks = (long long)sms * 32;
+            if (dtype == EBS_F32)
+                pack_acts_nhwc_f32_coalesced_kernel<<<(int)wblocks, 256, 0, st>>>((const float*)x, items, a_bits, inv_scale, out);
+            else {
+                long long ublocks = ((items + 127) / 128 + 7) / 8;
+                if (ublocks > (long long)sms * 16) ublocks = (long long)sms * 16;
+                pack_acts_nhwc_u8_coalesced_kernel<<<(int)ublocks, 256, 0, st>>>((const uint8_t*)x, items, a_bits, out);
+            }
+        } else if (dtype == EBS_F32)
+            pack_acts_nhwc_f32_kernel<<<(int)blocks, 256, 0, st>>>((const float*)x, items, c, CW, a_bits, inv_scale, out);
+        else
             pack_acts_nhwc_u8_kernel<<<(int)blocks, 256, 0, st>>>((const uint8_t*)x, items, c, CW, a_bits, out);
-        }
     } else {
-        const long long tiles = (long long)n * CW * ((h * w + 31) / 32);
+        const long long tiles = (long long)n * CW * ((h * w + 127) / 128);
         long long grid = tiles < (long long)sms * 16 ? tiles : (long long)sms * 16;
         if (grid < 1) grid = 1;
         if (dtype == EBS_F32)
-            pack_acts_nchw_kernel<float><<<(int)grid, 256, 0, st>>>((const float*)x, n, c, h * w, CW, a_bits, inv_scale, out);
+            pack_acts_nchw_kernel<float><<<(int)grid, 128, 0, st>>>((const float*)x, n, c, h * w, CW, a_bits, inv_scale, out);
         else
-            pack_acts_nchw_kernel<uint8_t><<<(int)grid, 256, 0, st>>>((const uint8_t*)x, n, c, h * w, CW, a_bits, inv_scale, out);
+            pack_acts_nchw_kernel<uint8_t><<<(int)grid, 128, 0, st>>>((const uint8_t*)x, n, c, h * w, CW, a_bits, inv_scale, out);
     }
     return check_cuda(cudaGetLastError());
 }

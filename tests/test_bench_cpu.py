@@ -1,0 +1,72 @@
+"""CPU-only checks of bench.py: the reference arm's JSON line, and the multi-process plumbing
+(rendezvous, barrier, MAX all-reduce of the timing) with two gloo ranks."""
+import json
+import os
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def run(args, env_extra=None, timeout=300):
+    env = dict(os.environ)
+    env.update(env_extra or {})
+    return subprocess.run([sys.executable, os.path.join(ROOT, "bench.py")] + args, capture_output=True, text=True,
+                          env=env, timeout=timeout, cwd=ROOT)
+
+
+def test_reference_arm_prints_one_json_line():
+    res = run(["--impl", "reference", "--steps", "1", "--warmup", "0"])
+    assert res.returncode == 0, res.stderr
+    lines = [ln for ln in res.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["unit"] == "TOPS" and d["higher_is_better"] is True
+    assert d["value"] > 0 and d["ms_per_step"] > 0 and d["vs_baseline"] is None
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0
+    assert d["config"]["workload"].startswith("config2")
+
+
+WORKER = r"""
+import os, sys
+sys.path.insert(0, {root!r})
+import bench
+rank, world, local = bench.dist_setup(2)
+assert world == 2 and rank == int(os.environ["RANK"])
+bench.barrier()
+m = bench.max_over_ranks(10.0 + rank)          # rank 1 is the slow one
+assert m == 11.0, m
+bench.barrier()
+print("rank", rank, "ok", m)
+"""
+
+
+def test_two_gloo_ranks_agree_on_the_max_time(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER.format(root=ROOT))
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT="29541", CUDA_VISIBLE_DEVICES="")
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.PIPE, text=True))
+    outs = [p.communicate(timeout=180) for p in procs]
+    for p, (out, err) in zip(procs, outs):
+        assert p.returncode == 0, err
+        assert "ok 11.0" in out
+
+
+def test_reference_arm_under_two_ranks_prints_once():
+    """Under torchrun-style launch only rank 0 runs the oracle; the other rank exits 0 without output."""
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT="29542", CUDA_VISIBLE_DEVICES="")
+        procs.append(subprocess.Popen([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                                       "--steps", "1", "--warmup", "0"], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.PIPE, text=True, cwd=ROOT))
+    outs = [p.communicate(timeout=300) for p in procs]
+    assert all(p.returncode == 0 for p in procs), [o[1] for o in outs]
+    printed = [o[0].strip() for o in outs if o[0].strip()]
+    assert len(printed) == 1 and json.loads(printed[0])["impl"] == "reference"
