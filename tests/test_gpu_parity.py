@@ -262,3 +262,52 @@ def test_host_entry_point(ebs, U, oracle):
     ebs.ebs_conv2d_mixed_host(xf_host, ebs.EBS_F32, ebs.EBS_NCHW, 3, 12, 9, pw, d, None, ws2, acc_h, None, None)
     torch.cuda.synchronize()
     assert np.array_equal(acc_h.numpy().transpose(0, 3, 1, 2), ref)
+
+
+# ------------------------------------------------------------------ edge cases
+
+EDGE = [
+    # c_in, c_out, k, stride, pad, h, w, n, wb, ab        what it stresses
+    (1, 1, 1, 1, 0, 1, 1, 1, 1, 1),                      # a single bit pair
+    (5, 3, 3, 1, 1, 1, 1, 2, 2, 3),                      # 1x1 image: only the centre tap is inside
+    (7, 9, 3, 1, 0, 3, 3, 1, 3, 2),                      # kernel covers the whole input: one output pixel
+    (33, 2, 1, 3, 0, 7, 8, 1, 4, 4),                     # stride larger than the kernel
+    (40, 70, 3, 1, 2, 4, 4, 1, 2, 2),                    # padding larger than needed: border outputs see few taps
+    (64, 64, 3, 1, 1, 12, 11, 1, 8, 8),                  # widest codes
+    (16, 16, 3, 2, 1, 33, 31, 3, 1, 8),                  # folded taps, odd sizes, stride 2
+    (8, 24, 5, 1, 2, 9, 9, 2, 3, 3),                     # four taps per word
+    (3, 16, 7, 2, 3, 21, 20, 2, 8, 8),                   # eight taps per word (first-layer shape)
+    (257, 5, 1, 1, 0, 3, 130, 1, 5, 6),                  # one image row longer than a pixel tile, ragged channels
+]
+
+
+@pytest.mark.parametrize("case", EDGE)
+def test_conv_edge_cases_all_variants(ebs, U, oracle, case):
+    c, co, k, s, pad, h, w, n, wb, ab = case
+    rng = np.random.default_rng(sum(case))
+    qa = U.rand_codes(rng, (n, c, h, w), ab, False)
+    qw = U.rand_codes(rng, (co, c, k, k), wb, True)
+    d = U.desc_for(c, co, k, s, pad, wb, ab)
+    ref = oracle.conv2d_codes(qa, qw, (s, s), (pad, pad))
+    px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
+    for variant in range(-1, ebs.ebs_num_conv_variants()):
+        got = U.run_conv(qa, qw, d, variant=variant, px=px, pw=pw)["acc"]
+        assert got.shape == ref.shape and np.array_equal(got, ref), f"variant {variant}"
+    assert ebs.ebs_device_wait_timeouts() == 0
+
+
+def test_conv_at_the_int32_limit(ebs, U, oracle):
+    """The largest reduction 8x8 bits allow (|acc| just below 2^31) with saturated codes, and one more channel refused."""
+    c = 65793                                               # 65793 * 128 * 255 = 2^31 - 2^15 - ... < 2^31
+    assert c * 128 * 255 < 2 ** 31 <= (c + 1) * 128 * 255
+    qa = np.full((1, c, 1, 2), 255, dtype=np.int32)
+    qw = np.full((2, c, 1, 1), -128, dtype=np.int32)
+    qw[1] = 127
+    d = U.desc_for(c, 2, 1, 1, 0, 8, 8)
+    got = U.run_conv(qa, qw, d)["acc"]
+    assert got[0, 0, 0, 0] == -128 * 255 * c and got[0, 1, 0, 1] == 127 * 255 * c
+    assert np.array_equal(got, oracle.conv2d_codes(qa, qw))
+    with pytest.raises(ebs.EbsError) as err:
+        ebs.ebs_packed_weight_bytes(U.desc_for(c + 1, 2, 1, 1, 0, 8, 8)) or ebs.ebs_conv_out_shape(
+            U.desc_for(c + 1, 2, 1, 1, 0, 8, 8), 1, 2)
+    assert err.value.status == ebs.EBS_ERR_OVERFLOW
