@@ -49,7 +49,8 @@ typedef enum ebs_status {
     EBS_OK = 0,
     EBS_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, bitwidth outside 1..8, misalignment */
     EBS_ERR_UNSUPPORTED = -2, /* valid request this build has no kernel for */
-    EBS_ERR_OVERFLOW = -3,    /* c_in*kh*kw*2^(w_bits-1)*(2^a_bits-1) >= 2^31, or an index would overflow */
+    EBS_ERR_OVERFLOW = -3,    /* c_in*kh*kw*2^(w_bits-1)*(2^a_bits-1) >= 2^31 (w_levels = 1: c_in*kh*kw*(2^w_bits-1)*
+                                 (2^a_bits-1)), or an index would overflow */
     EBS_ERR_CUDA = -4,        /* a CUDA runtime call failed (launch error, bad device pointer, ...) */
     EBS_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (reserved) */
     EBS_ERR_SCRATCH_TOO_SMALL = -6 /* the request needs more than the built-in scratch of the no-allocation call */
@@ -73,8 +74,15 @@ typedef struct ebs_conv_desc {
     int stride_h, stride_w;
     int pad_h, pad_w;   /* zero padding: a padded tap is the real value 0 */
     int w_bits, a_bits; /* M and K of the paper, 1..8 each */
-    float w_scale;      /* real weight  = w_scale * code */
+    float w_scale;      /* real weight  = w_scale * code (w_levels = 0) or w_scale * (2*code + 1) (w_levels = 1) */
     float a_scale;      /* real input   = a_scale * code */
+    int w_levels;       /* 0: two's-complement weights, real weight = w_scale * code.
+                           1: the paper's own weight levels (Eq. 1a): the 2^b levels 2*q_u - (2^b - 1), q_u = 0 .. 2^b-1,
+                              symmetric about zero; stored as the signed code q_u - 2^(b-1), so the level is
+                              2*code + 1 and w_scale = 1/(2^b - 1) gives the paper's range [-1, 1].  The accumulator
+                              is then sum (2*code + 1) * activation code = 2 * (bit-plane sum) + (sum of the
+                              activation codes under the filter window); the window sum is taken from the
+                              activation planes inside the same kernel. */
 } ebs_conv_desc;
 
 /*
@@ -121,7 +129,9 @@ size_t ebs_packed_act_bytes(int n, int h, int w, int c, int a_bits);
 /*
  * Weight quantization and bit-plane expansion B_w (Eq. 12, Eq. 15; quantizer Eq. 1c).
  *   w_dev       c_out*c_in*kh*kw values in `layout`; EBS_F32 (quantized with desc->w_scale to
- *               signed desc->w_bits codes) or EBS_I8_CODES (taken as they are; must be in range).
+ *               signed desc->w_bits codes: code = floor(w/w_scale + 0.5), or with w_levels = 1 the
+ *               nearest level, code = floor((w/w_scale + 2^b - 1)/2 + 0.5) - 2^(b-1), clamped) or
+ *               EBS_I8_CODES (signed codes taken as they are; must be in range).
  *   packed_w_dev  ebs_packed_weight_bytes(desc) bytes, fully overwritten.
  * Done once per layer, off the inference path.
  */
@@ -142,7 +152,8 @@ int ebs_pack_acts(const void *x_dev, int dtype, int layout, int n, int c, int h,
  * (n, ho, wo, co)
  *   acc = sum_{m<M} sum_{k<K} c_m 2^(m+k) * sum_{taps, channel words} popcount(A_k AND W_m),
  *   c_m = -1 for m = M-1 (signed weights), +1 otherwise,
- * with taps outside the image contributing zero.  The M*K partial sums (the paper's matrix P)
+ * with taps outside the image contributing zero; with desc->w_levels = 1 the accumulator is
+ * 2 * acc + sum_{k<K} 2^k * sum_{taps, channel words} popcount(A_k) (see ebs_conv_desc).  The M*K partial sums (the paper's matrix P)
  * never leave the chip.  Any subset of the three outputs may be requested (at least one):
  *   acc_out_dev     int32 [N][Ho][Wo][C_out]                      exact accumulators
  *   y_out_dev       fp32, epilogue applied, layout epi->y_layout  (NHWC if epi is NULL)

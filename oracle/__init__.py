@@ -46,6 +46,10 @@ def _load():
         lib.oracle_quantize.restype = None
         lib.oracle_conv2d_codes.argtypes = [p, p] + [i] * 11 + [p]
         lib.oracle_conv2d_codes.restype = i
+        lib.oracle_conv2d_levels.argtypes = [p, p] + [i] * 11 + [p]
+        lib.oracle_conv2d_levels.restype = i
+        lib.oracle_quantize_weight_levels.argtypes = [p, z, f, i, p]
+        lib.oracle_quantize_weight_levels.restype = None
         lib.oracle_conv2d_bitplanes.argtypes = [p, p] + [i] * 14 + [p]
         lib.oracle_conv2d_bitplanes.restype = i
         lib.oracle_epilogue.argtypes = [p, i, i, i, i, f, p, p, p, i, p, i, f, p]
@@ -115,6 +119,32 @@ def conv2d_codes(qa, qw, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
     if rc != OK:
         raise ValueError(f"oracle_conv2d_codes: bad arguments ({rc})")
     return acc
+
+
+def conv2d_levels(qa, qw, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
+    """Convolution with the paper's weight levels 2*qw + 1 (Eq. 1a), qw the signed code q_u - 2^(b-1)."""
+    qa, qw = _i32(qa), _i32(qw)
+    n, c, h, w = qa.shape
+    co, c2, kh, kw = qw.shape
+    assert c == c2
+    ho, wo = out_dim(h, pad[0], kh, stride[0]), out_dim(w, pad[1], kw, stride[1])
+    acc = np.empty((n, co, ho, wo), dtype=np.int32)
+    rc = _load().oracle_conv2d_levels(_ptr(qa), _ptr(qw), n, c, h, w, co, kh, kw, stride[0], stride[1],
+                                      pad[0], pad[1], _ptr(acc))
+    if rc == ERR_OVERFLOW:
+        raise OverflowError("accumulator does not fit int32")
+    if rc != OK:
+        raise ValueError(f"oracle_conv2d_levels: bad arguments ({rc})")
+    return acc
+
+
+def quantize_weight_levels(w, w_scale: float, w_bits: int) -> np.ndarray:
+    """Eq. 1a: nearest of the levels w_scale*(2 q_u - (2^b-1)); returns the signed code q_u - 2^(b-1)."""
+    w = _f32(w)
+    q = np.empty(w.shape, dtype=np.int32)
+    inv = np.float32(1.0) / np.float32(w_scale)
+    _load().oracle_quantize_weight_levels(_ptr(w), w.size, inv, w_bits, _ptr(q))
+    return q
 
 
 def conv2d_bitplanes(qa, qw, w_bits, a_bits, stride=(1, 1), pad=(0, 0), signed_w=True) -> np.ndarray:

@@ -115,6 +115,69 @@ int oracle_conv2d_codes(const int32_t *qa, const int32_t *qw, int N, int C, int 
 }
 
 /*
+ * The paper's own weight format (Eq. 1a): b-bit weights take the 2^b levels 2*q_u - (2^b - 1),
+ * q_u = 0 .. 2^b - 1 (times 1/(2^b - 1)).  With the signed code qw = q_u - 2^(b-1) the level is
+ * 2*qw + 1, and the convolution of levels with activation codes is
+ *   acc[n][co][ho][wo] = sum (2*qw + 1) * qa        (direct definition, taps outside the image skipped).
+ */
+int oracle_conv2d_levels(const int32_t *qa, const int32_t *qw, int N, int C, int H, int W, int Co,
+                         int kh, int kw, int sh, int sw, int ph, int pw, int32_t *acc) {
+    if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || Co <= 0 || kh <= 0 || kw <= 0 || sh <= 0 || sw <= 0 ||
+        ph < 0 || pw < 0)
+        return ORACLE_ERR_ARG;
+    const int Ho = out_dim(H, ph, kh, sh), Wo = out_dim(W, pw, kw, sw);
+    if (Ho <= 0 || Wo <= 0) return ORACLE_ERR_ARG;
+    int overflow = 0;
+#pragma omp parallel for collapse(2) schedule(static) reduction(| : overflow)
+    for (int n = 0; n < N; ++n) {
+        for (int co = 0; co < Co; ++co) {
+            for (int ho = 0; ho < Ho; ++ho) {
+                for (int wo = 0; wo < Wo; ++wo) {
+                    int64_t sum = 0;
+                    for (int ci = 0; ci < C; ++ci)
+                        for (int r = 0; r < kh; ++r) {
+                            const int hi = ho * sh + r - ph;
+                            if (hi < 0 || hi >= H) continue;
+                            for (int s = 0; s < kw; ++s) {
+                                const int wi = wo * sw + s - pw;
+                                if (wi < 0 || wi >= W) continue;
+                                const int64_t a = qa[(((size_t)n * C + ci) * H + hi) * W + wi];
+                                const int64_t level = 2 * (int64_t)qw[(((size_t)co * C + ci) * kh + r) * kw + s] + 1;
+                                sum += a * level;
+                            }
+                        }
+                    if (sum > INT32_MAX || sum < INT32_MIN) overflow = 1;
+                    acc[(((size_t)n * Co + co) * Ho + ho) * Wo + wo] = (int32_t)sum;
+                }
+            }
+        }
+    }
+    return overflow ? ORACLE_ERR_OVERFLOW : ORACLE_OK;
+}
+
+/*
+ * Weight quantizer of Eq. 1a in code form: the nearest level w_step * (2*q_u - L), L = 2^b - 1,
+ * round half up; returns the signed code q_u - 2^(b-1).
+ *   v = fl(w * inv_step);  u = fl(fl(v + L) * 0.5);  q_u = clamp(floor(fl(u + 0.5)), 0, L).
+ * With w = w_n (normalised to [-1, 1]) and w_step = 1/L this is q_u = round(L * (w_n/2 + 1/2)).
+ */
+void oracle_quantize_weight_levels(const float *w, size_t count, float inv_step, int bits, int32_t *q) {
+    const int L = (1 << bits) - 1;
+    for (size_t t = 0; t < count; ++t) {
+        volatile float v = w[t] * inv_step;
+        volatile float s = v + (float)L;
+        volatile float u = s * 0.5f;
+        volatile float r = u + 0.5f;
+        float f = floorf(r);
+        int32_t qu;
+        if (!(f >= 0.0f)) qu = 0;
+        else if (f > (float)L) qu = L;
+        else qu = (int32_t)f;
+        q[t] = qu - (1 << (bits - 1));
+    }
+}
+
+/*
  * The same result by the bit-plane route of Eq. 2, one bit at a time and without
  * any packing:  sum_m sum_k c_m 2^(m+k) bitcount(AND(bit m of w, bit k of x)).
  * Weights are Wb-bit two's-complement codes, so the coefficient of the top

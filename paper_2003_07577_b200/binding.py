@@ -33,7 +33,7 @@ class ebs_conv_desc(ctypes.Structure):
     _fields_ = [("c_in", ctypes.c_int), ("c_out", ctypes.c_int), ("kh", ctypes.c_int), ("kw", ctypes.c_int),
                 ("stride_h", ctypes.c_int), ("stride_w", ctypes.c_int), ("pad_h", ctypes.c_int),
                 ("pad_w", ctypes.c_int), ("w_bits", ctypes.c_int), ("a_bits", ctypes.c_int),
-                ("w_scale", ctypes.c_float), ("a_scale", ctypes.c_float)]
+                ("w_scale", ctypes.c_float), ("a_scale", ctypes.c_float), ("w_levels", ctypes.c_int)]
 
 
 class ebs_epilogue(ctypes.Structure):
@@ -104,8 +104,10 @@ def _check(rc: int, where: str):
         raise EbsError(rc, where)
 
 
-def conv_desc(c_in, c_out, kh, kw, stride_h, stride_w, pad_h, pad_w, w_bits, a_bits, w_scale, a_scale) -> ebs_conv_desc:
-    return ebs_conv_desc(c_in, c_out, kh, kw, stride_h, stride_w, pad_h, pad_w, w_bits, a_bits, w_scale, a_scale)
+def conv_desc(c_in, c_out, kh, kw, stride_h, stride_w, pad_h, pad_w, w_bits, a_bits, w_scale, a_scale,
+              w_levels=0) -> ebs_conv_desc:
+    return ebs_conv_desc(c_in, c_out, kh, kw, stride_h, stride_w, pad_h, pad_w, w_bits, a_bits, w_scale, a_scale,
+                         int(w_levels))
 
 
 def epilogue(ch_scale=None, ch_bias=None, residual=None, relu=False, next_a_bits=0, next_a_scale=1.0,

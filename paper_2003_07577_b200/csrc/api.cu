@@ -78,7 +78,9 @@ static int validate_desc(const ebs_conv_desc* d) {
     if (!(d->w_scale > 0.0f) || !(d->a_scale > 0.0f)) return EBS_ERR_INVALID_ARG;
     // largest |acc| = c_in*kh*kw * 2^(w_bits-1) * (2^a_bits - 1) must fit int32
     const long long s = (long long)d->c_in * d->kh * d->kw;
-    const long long worst = s * (1LL << (d->w_bits - 1)) * ((1LL << d->a_bits) - 1);
+    if (d->w_levels != 0 && d->w_levels != 1) return EBS_ERR_INVALID_ARG;
+    const long long wmax = d->w_levels ? (1LL << d->w_bits) - 1 : (1LL << (d->w_bits - 1));   // largest |weight level|
+    const long long worst = s * wmax * ((1LL << d->a_bits) - 1);
     if (worst >= (1LL << 31)) return EBS_ERR_OVERFLOW;
     return EBS_OK;
 }
@@ -175,6 +177,7 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
     p.acc = acc_out; p.y = y_out; p.packed_next = static_cast<uint32_t*>(packed_next);
     p.S = d->w_scale * d->a_scale;       // one rounded fp32 multiply
     p.next_bits = 1;
+    p.w_levels = d->w_levels;
     p.fold = d->c_in <= 4 ? 8 : (d->c_in <= 8 ? 4 : (d->c_in <= 16 ? 2 : 1));
     p.fold_bits = 32 / p.fold;
     if (epi) {

@@ -181,12 +181,15 @@ conv_mma_kernel(const ConvParams p) {
     };
 
     int acc[MT][NT][4];
+    int wsum[MT][2];           // sum of the activation codes under the filter window, rows g and g+8 (w_levels)
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+    for (int mt = 0; mt < MT; ++mt) {
+        wsum[mt][0] = 0; wsum[mt][1] = 0;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0;
+    }
 
     __syncthreads();                                   // tap table ready
     const int nsteps = (p.KK + KSTEP - 1) / KSTEP;
@@ -234,6 +237,10 @@ conv_mma_kernel(const ConvParams p) {
 #pragma unroll
                     for (int k = 0; k < AB; ++k) {
                         const uint32_t w0 = wr0[k], w1 = wr1[k];
+                        if (p.w_levels) {                   // every lane holds the whole word of its two rows
+                            wsum[mt][0] += __popc(w0) << k;
+                            wsum[mt][1] += __popc(w1) << k;
+                        }
                         const uint32_t mask = 0x01010101u << k;
                         af[mt][k][0] = __funnelshift_r(w0, w0, tq - k) & mask;
                         af[mt][k][1] = __funnelshift_r(w1, w1, tq - k) & mask;
@@ -304,7 +311,8 @@ conv_mma_kernel(const ConvParams p) {
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
-                    const int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
+                    int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
+                    if (p.w_levels) { a0 = 2 * a0 + wsum[mt][half]; a1 = 2 * a1 + wsum[mt][half]; }
                     const bool valid = pvalid && co < p.Co;
                     int code0 = 0, code1 = 0;
                     if (valid && p.acc) *reinterpret_cast<int2*>(p.acc + row_o + nt * 8) = make_int2(a0, a1);
@@ -324,7 +332,8 @@ conv_mma_kernel(const ConvParams p) {
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 const int cl = (wc * NT + nt) * 8 + 2 * tq, co = co0 + cl;
-                const int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
+                int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
+                if (p.w_levels) { a0 = 2 * a0 + wsum[mt][half]; a1 = 2 * a1 + wsum[mt][half]; }
                 int code0 = 0, code1 = 0;
                 if (pvalid && co < p.Co) {
                     const size_t o = (size_t)gp * p.Co + co;

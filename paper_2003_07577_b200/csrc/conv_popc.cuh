@@ -75,10 +75,13 @@ conv_popc_kernel(const ConvParams p) {
     if (tid < KSTEP) kinfo[0][tid] = decode_kk(tid);
 
     int acc[TP][TC];
+    int wsum[TP];              // sum of the activation codes under the filter window (w_levels)
 #pragma unroll
-    for (int t = 0; t < TP; ++t)
+    for (int t = 0; t < TP; ++t) {
+        wsum[t] = 0;
 #pragma unroll
         for (int c = 0; c < TC; ++c) acc[t][c] = 0;
+    }
 
     __syncthreads();
 
@@ -122,7 +125,10 @@ conv_popc_kernel(const ConvParams p) {
 #pragma unroll
                 for (int t = 0; t < TP; ++t)
 #pragma unroll
-                    for (int j = 0; j < AB; ++j) a[t][j] = A_s[q][j][(wp * TP + t) * 32 + lane];
+                    for (int j = 0; j < AB; ++j) {
+                        a[t][j] = A_s[q][j][(wp * TP + t) * 32 + lane];
+                        if (p.w_levels) wsum[t] += __popc(a[t][j]) << j;
+                    }
                 const uint4* wv = reinterpret_cast<const uint4*>(&W_s[q][wc * TC][0]);
                 uint32_t* wflat = &w[0][0];
 #pragma unroll
@@ -163,9 +169,10 @@ conv_popc_kernel(const ConvParams p) {
             int code = 0;
             if (valid) {
                 const size_t o = (size_t)gp * p.Co + co;
-                if (p.acc) p.acc[o] = acc[t][c];
+                const int av = p.w_levels ? 2 * acc[t][c] + wsum[t] : acc[t][c];
+                if (p.acc) p.acc[o] = av;
                 if (want_y || want_q) {
-                    float yv = __fmul_rn((float)acc[t][c], p.S);
+                    float yv = __fmul_rn((float)av, p.S);
                     if (p.ch_scale) yv = __fmul_rn(yv, __ldg(p.ch_scale + co));
                     if (p.ch_bias) yv = __fadd_rn(yv, __ldg(p.ch_bias + co));
                     if (p.residual) yv = __fadd_rn(yv, __ldg(p.residual + o));

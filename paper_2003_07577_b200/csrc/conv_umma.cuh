@@ -145,6 +145,7 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
     __shared__ __align__(8) uint64_t empty_bar[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ int wsum_s[2][UMMA_M];          // per pixel row: window sum of the activation codes, one part per half
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int tile_p0 = blockIdx.x * UMMA_M;
@@ -195,7 +196,7 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
             for (int r = 0; r < p.kh; ++r) row_ok |= ((unsigned)(h0 + r) < (unsigned)p.H ? 1u : 0u) << r;
             for (int s = 0; s < p.kw; ++s) col_ok |= ((unsigned)(w0 + s) < (unsigned)p.W ? 1u : 0u) << s;
         }
-        uint32_t a_nxt[KS][AB], b_nxt[T::B_ITEMS];
+        uint32_t a_set[3][KS][AB], b_set[3][T::B_ITEMS];   // packed words of three consecutive chunks (ring)
 
         // per-thread constants of the weight rows it expands: which (reduction word, plane, channel row),
         // where that row starts in global memory (for reduction word 0) and in the stage
@@ -216,7 +217,9 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
         const int co_wb = p.Co * WB;                              // weight words per reduction word
 
         // packed words of chunk `ch` -> registers (zero past the end, outside the image, past c_out)
-        auto load_chunk = [&](int ch) {
+        auto load_chunk = [&](int ch, int set) {
+            uint32_t (&a_nxt)[KS][AB] = a_set[set];
+            uint32_t (&b_nxt)[T::B_ITEMS] = b_set[set];
 #pragma unroll
             for (int q = 0; q < KS; ++q) {
                 const int kw = ch * KS + q;
@@ -261,54 +264,64 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
             }
         };
 
-        load_chunk(0);
-        for (int ch = 0; ch < nchunks; ++ch) {
-            const int st = ch & 1;
-            uint8_t* A_st = tiles + st * T::STAGE_BYTES;               // [KS][AB] planes of 128 rows x 32 B, then
+        // the words of chunks ch+1 and ch+2 are in flight while chunk ch is expanded; the ring index is a
+        // compile-time constant after unrolling, so the three sets stay in registers and no pending load is moved
+        load_chunk(0, 0);
+        if (nchunks > 1) load_chunk(1, 1);
+        bool expanders_ok = true;
+        int wsum = 0;                                              // this thread's share of its row's window sum
+        for (int ch0 = 0; ch0 < nchunks && expanders_ok; ch0 += 3) {
+#pragma unroll
+            for (int u = 0; u < 3; ++u) {
+                const int ch = ch0 + u;
+                if (ch >= nchunks) break;
+                const int st = ch & 1;
+                uint8_t* A_st = tiles + st * T::STAGE_BYTES;           // [KS][AB] planes of 128 rows x 32 B, then
                                                                        // [KS][WB] planes of TILE_N rows x 32 B
-            uint32_t a_cur[KS][AB], b_cur[T::B_ITEMS];
-#pragma unroll
-            for (int q = 0; q < KS; ++q)
-#pragma unroll
-                for (int k = 0; k < AB; ++k) a_cur[q][k] = a_nxt[q][k];
-#pragma unroll
-            for (int i = 0; i < T::B_ITEMS; ++i) b_cur[i] = b_nxt[i];
-            if (ch + 1 < nchunks) load_chunk(ch + 1);                   // in flight while this chunk is expanded
-            if (ch >= 2) {                                             // the MMAs of chunk ch-2 must have read the stage
-                if (!mbar_wait_bounded(&empty_bar[st], (uint32_t)(((ch >> 1) - 1) & 1), abortp)) break;
-            }
-#pragma unroll
-            for (int q = 0; q < KS; ++q) {
-#pragma unroll
-                for (int k = 0; k < AB; ++k) {
-                    if (((q * AB + k) & 1) != half) continue;
-                    uint4 lo, hi;
-                    expand_word_to_row(a_cur[q][k], k, 1u, lo, hi);
-                    uint8_t* tile = A_st + (q * AB + k) * T::A_PLANE_BYTES;
-                    *reinterpret_cast<uint4*>(tile + a_soff0) = lo;
-                    *reinterpret_cast<uint4*>(tile + a_soff1) = hi;
+                if (ch + 2 < nchunks) load_chunk(ch + 2, (u + 2) % 3);
+                if (ch >= 2) {                                         // the MMAs of chunk ch-2 must have read the stage
+                    if (!mbar_wait_bounded(&empty_bar[st], (uint32_t)(((ch >> 1) - 1) & 1), abortp)) {
+                        expanders_ok = false;
+                        break;
+                    }
                 }
-            }
+                const uint32_t (&a_cur)[KS][AB] = a_set[u];
+                const uint32_t (&b_cur)[T::B_ITEMS] = b_set[u];
 #pragma unroll
-            for (int i = 0; i < T::B_ITEMS; ++i) {
-                if (b_q[i] >= 0) {
-                    const int m = b_m[i];
-                    // rotate once by the plane, then the eight byte groups are fixed rotations of that
-                    const uint32_t wrot = __funnelshift_l(b_cur[i], b_cur[i], m);
-                    const uint32_t mask = 0x01010101u << m;
-                    const uint32_t scale = (m == WB - 1 && WB < 8) ? ((1u << (9 - WB)) - 1u) : 1u;
-                    uint32_t r[8];
+                for (int q = 0; q < KS; ++q) {
 #pragma unroll
-                    for (int bb = 0; bb < 8; ++bb) r[bb] = (__funnelshift_r(wrot, wrot, bb) & mask) * scale;
-                    uint8_t* dst = A_st + b_soff[i];
-                    const int bsw = (b_soff[i] >> 3) & 16;               // ((row >> 2) & 1) << 4 with row = offset / 32
-                    *reinterpret_cast<uint4*>(dst + bsw) = make_uint4(r[0], r[1], r[2], r[3]);
-                    *reinterpret_cast<uint4*>(dst + (bsw ^ 16)) = make_uint4(r[4], r[5], r[6], r[7]);
+                    for (int k = 0; k < AB; ++k) {
+                        if (((q * AB + k) & 1) != half) continue;
+                        if (p.w_levels) wsum += __popc(a_cur[q][k]) << k;
+                        uint4 lo, hi;
+                        expand_word_to_row(a_cur[q][k], k, 1u, lo, hi);
+                        uint8_t* tile = A_st + (q * AB + k) * T::A_PLANE_BYTES;
+                        *reinterpret_cast<uint4*>(tile + a_soff0) = lo;
+                        *reinterpret_cast<uint4*>(tile + a_soff1) = hi;
+                    }
                 }
+#pragma unroll
+                for (int i = 0; i < T::B_ITEMS; ++i) {
+                    if (b_q[i] >= 0) {
+                        const int m = b_m[i];
+                        // rotate once by the plane, then the eight byte groups are fixed rotations of that
+                        const uint32_t wrot = __funnelshift_l(b_cur[i], b_cur[i], m);
+                        const uint32_t mask = 0x01010101u << m;
+                        const uint32_t scale = (m == WB - 1 && WB < 8) ? ((1u << (9 - WB)) - 1u) : 1u;
+                        uint32_t r[8];
+#pragma unroll
+                        for (int bb = 0; bb < 8; ++bb) r[bb] = (__funnelshift_r(wrot, wrot, bb) & mask) * scale;
+                        uint8_t* dst = A_st + b_soff[i];
+                        const int bsw = (b_soff[i] >> 3) & 16;           // ((row >> 2) & 1) << 4 with row = offset / 32
+                        *reinterpret_cast<uint4*>(dst + bsw) = make_uint4(r[0], r[1], r[2], r[3]);
+                        *reinterpret_cast<uint4*>(dst + (bsw ^ 16)) = make_uint4(r[4], r[5], r[6], r[7]);
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");  // generic writes -> tensor-core reads
+                mbar_arrive(&full_bar[st]);
             }
-            asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");     // generic writes -> tensor-core reads
-            mbar_arrive(&full_bar[st]);
         }
+        wsum_s[half][row] = wsum;
         // all MMAs done (the last commit covers every earlier one)
         if (!*abortp) mbar_wait_bounded(&empty_bar[(nchunks - 1) & 1], (uint32_t)(((nchunks - 1) >> 1) & 1), abortp);
     } else {
@@ -358,11 +371,17 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
         const int hw = p.Ho * p.Wo;
         const int img = pvalid ? gp / hw : 0, rem = pvalid ? gp - img * hw : 0;
         const int cbeg = (warp >> 2) * COLS_PER_WARP;
+        const int erow = (warp & 3) * 32 + (tid & 31);             // the pixel row whose accumulators this thread reads
+        const int wsum_row = p.w_levels ? wsum_s[0][erow] + wsum_s[1][erow] : 0;
         uint32_t planes[8];
 #pragma unroll 1
         for (int c0 = cbeg; c0 < cbeg + COLS_PER_WARP; c0 += 16) {
             uint32_t v[16];
             tmem_ld16(trow + (uint32_t)c0, v);                       // whole warp, also for rows past the end
+            if (p.w_levels) {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = (uint32_t)(2 * (int)v[e] + wsum_row);
+            }
             if ((c0 & 31) == 0) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j) planes[j] = 0u;
@@ -438,11 +457,14 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
 template <int WB, int AB, int TILE_N>
 void launch_conv_umma(const ConvParams& p, dim3 grid, cudaStream_t st) {
     using T = UmmaTile<WB, AB, TILE_N>;
-    static bool attr_set = false;              // raising the dynamic shared-memory limit is a one-time attribute
-    if (!attr_set) {
+    // raising the dynamic shared-memory limit is a per-device attribute of the kernel: set it once per device
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
         cudaFuncSetAttribute(conv_umma_kernel<WB, AB, TILE_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              T::SMEM_BYTES);
-        attr_set = true;
+        attr_set[dev] = true;
     }
     conv_umma_kernel<WB, AB, TILE_N><<<grid, UMMA_THREADS, T::SMEM_BYTES, st>>>(p);
 }

@@ -28,6 +28,7 @@ struct ConvParams {
     int next_bits;
     float inv_next;
     int y_nchw;
+    int w_levels;                     // 1: accumulator = 2 * plane sum + window sum of the activation codes
     int fold;                         // taps OR-ed into one reduction word by the tensor-pipe kernels: 1, 2, 4, 8
     int fold_bits;                    // 32 / fold: bits each folded tap occupies (>= c_in)
 };
@@ -110,6 +111,20 @@ __device__ __forceinline__ int quantize_code(float x, float inv_scale, int lo, i
     else if (f > (float)hi) q = hi;
     else q = (int)f;
     return q;
+}
+
+// Nearest of the paper's weight levels w_scale * (2 q_u - (2^b - 1)), q_u = 0 .. 2^b-1 (Eq. 1a), returned
+// as the signed code q_u - 2^(b-1).  (v + L)/2 is exact in fp32 for the magnitudes that survive the clamp.
+__device__ __forceinline__ int quantize_weight_level(float w, float inv_scale, int bits) {
+    const int L = (1 << bits) - 1;
+    const float v = __fmul_rn(w, inv_scale);
+    const float u = __fmul_rn(__fadd_rn(v, (float)L), 0.5f);
+    const float f = floorf(__fadd_rn(u, 0.5f));
+    int qu;
+    if (!(f >= 0.0f)) qu = 0;
+    else if (f > (float)L) qu = L;
+    else qu = (int)f;
+    return qu - (1 << (bits - 1));
 }
 
 // The same quantizer for activation codes (lo = 0): floor and float->int in one conversion

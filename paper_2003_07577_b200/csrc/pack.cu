@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(128) pack_acts_nchw_kernel(const T* __restrict
 template <typename T>
 __global__ void __launch_bounds__(256) pack_weights_kernel(const T* __restrict__ wt, int layout, int Co, int C,
                                                            int kh, int kw, int CW, int WB, float inv_scale,
-                                                           uint32_t* __restrict__ out) {
+                                                           int w_levels, uint32_t* __restrict__ out) {
     const int lane = threadIdx.x & 31;
     const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -264,7 +264,8 @@ __global__ void __launch_bounds__(256) pack_weights_kernel(const T* __restrict__
             const long long idx = layout == EBS_NCHW ? (((long long)co * C + c) * kh + r) * kw + s
                                                      : (((long long)co * kh + r) * kw + s) * C + c;
             int q;
-            if constexpr (sizeof(T) == 4) q = quantize_code((float)wt[idx], inv_scale, lo, hi);
+            if constexpr (sizeof(T) == 4)
+                q = w_levels ? quantize_weight_level((float)wt[idx], inv_scale, WB) : quantize_code((float)wt[idx], inv_scale, lo, hi);
             else q = (int)wt[idx];
             code = (uint32_t)q & ((1u << WB) - 1u);      // two's-complement bit pattern
         }
@@ -337,10 +338,10 @@ int launch_pack_weights(const void* wt, int dtype, int layout, const ebs_conv_de
     const int grid = grid_for(items, sm_count());
     if (dtype == EBS_F32)
         pack_weights_kernel<float><<<grid, 256, 0, st>>>((const float*)wt, layout, d.c_out, d.c_in, d.kh, d.kw, CW,
-                                                         d.w_bits, inv_scale, out);
+                                                         d.w_bits, inv_scale, d.w_levels, out);
     else
         pack_weights_kernel<int8_t><<<grid, 256, 0, st>>>((const int8_t*)wt, layout, d.c_out, d.c_in, d.kh, d.kw, CW,
-                                                          d.w_bits, inv_scale, out);
+                                                          d.w_bits, inv_scale, d.w_levels, out);
     return check_cuda(cudaGetLastError());
 }
 

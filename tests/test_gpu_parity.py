@@ -311,3 +311,42 @@ def test_conv_at_the_int32_limit(ebs, U, oracle):
         ebs.ebs_packed_weight_bytes(U.desc_for(c + 1, 2, 1, 1, 0, 8, 8)) or ebs.ebs_conv_out_shape(
             U.desc_for(c + 1, 2, 1, 1, 0, 8, 8), 1, 2)
     assert err.value.status == ebs.EBS_ERR_OVERFLOW
+
+
+# ------------------------------------------------------------------ the paper's own weight levels (w_levels = 1)
+
+@pytest.mark.parametrize("wb,ab,c,co,k,s,pad", [(1, 1, 16, 16, 3, 1, 1), (1, 2, 64, 64, 3, 1, 1), (2, 3, 40, 21, 3, 2, 1),
+                                                (4, 4, 128, 70, 1, 1, 0), (8, 8, 33, 9, 3, 1, 0), (3, 5, 8, 130, 5, 1, 2)])
+def test_conv_with_paper_weight_levels_all_variants(ebs, U, oracle, wb, ab, c, co, k, s, pad):
+    rng = np.random.default_rng(wb * 100 + ab * 10 + k)
+    qa = U.rand_codes(rng, (2, c, 10, 9), ab, False)
+    qs = U.rand_codes(rng, (co, c, k, k), wb, True)
+    L = (1 << wb) - 1
+    d = ebs.conv_desc(c, co, k, k, s, s, pad, pad, wb, ab, 1.0 / L, 0.05, w_levels=1)
+    ref = oracle.conv2d_levels(qa, qs, (s, s), (pad, pad))
+    S = oracle.combined_scale(1.0 / L, 0.05)
+    y_ref, q_ref = oracle.epilogue(ref, S, relu=True, next_bits=3, inv_next=np.float32(1.0) / np.float32(0.4))
+    px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qs, d)
+    epi = ebs.epilogue(relu=True, next_a_bits=3, next_a_scale=0.4)
+    for variant in range(-1, ebs.ebs_num_conv_variants()):
+        try:
+            out = U.run_conv(qa, qs, d, epi, want_acc=True, want_y=True, next_bits=3, variant=variant, px=px, pw=pw)
+        except ebs.EbsError as exc:                      # 16-channel tiles cannot produce packed words of wider layers
+            assert exc.status == ebs.EBS_ERR_UNSUPPORTED
+            continue
+        assert np.array_equal(out["acc"], ref), f"variant {variant}"
+        assert np.array_equal(out["y"], y_ref), f"variant {variant}"
+        assert np.array_equal(oracle.unpack_acts(out["packed"], co), q_ref), f"variant {variant}"
+
+
+def test_pack_weights_fp32_to_paper_levels(ebs, U, oracle):
+    rng = np.random.default_rng(5)
+    wb, c, co, k = 3, 20, 12, 3
+    L = (1 << wb) - 1
+    w = rng.uniform(-1.1, 1.1, size=(co, c, k, k)).astype(np.float32)
+    qs = oracle.quantize_weight_levels(w, 1.0 / L, wb)
+    assert qs.min() == -(1 << (wb - 1)) and qs.max() == (1 << (wb - 1)) - 1
+    d = ebs.conv_desc(c, co, k, k, 1, 1, 1, 1, wb, 2, 1.0 / L, 0.05, w_levels=1)
+    out = torch.empty(ebs.ebs_packed_weight_bytes(d) // 4, dtype=torch.int32, device=U.dev())
+    ebs.ebs_pack_weights(torch.from_numpy(w).to(U.dev()), ebs.EBS_F32, ebs.EBS_NCHW, d, out)
+    assert np.array_equal(U.as_u32(out).reshape(k, k, 1, co, wb), oracle.pack_weights(qs, wb))

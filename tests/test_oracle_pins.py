@@ -337,3 +337,43 @@ def test_generators_are_seeded_and_in_range():
         assert np.array_equal(qw, gen.weight_codes(s))
     c1 = gen.config1()[0]
     assert (c1.w_bits, c1.a_bits, c1.batch) == (2, 2, 1) and 0.01 <= c1.w_scale <= 0.1
+
+
+# ---------------------------------------------------------------- the paper's own weight levels (Eq. 1a)
+
+def test_levels_conv_equals_brute_force_and_the_unsigned_bitplane_route(oracle):
+    rng = np.random.default_rng(41)
+    wb, ab = 3, 2
+    L = (1 << wb) - 1
+    qa = rand_codes(rng, (2, 5, 6, 5), ab, False)
+    qs = rand_codes(rng, (3, 5, 3, 3), wb, True)                 # signed code = q_u - 2^(b-1)
+    qu = qs + (1 << (wb - 1))                                    # the paper's unsigned level index
+    levels = 2 * qu - L                                          # Eq. 1a numerator: 2*round(L x) - L
+    assert levels.min() >= -L and levels.max() <= L and np.all(levels % 2 != 0) and np.array_equal(levels, 2 * qs + 1)
+    got = oracle.conv2d_levels(qa, qs, (1, 1), (1, 1))
+    assert np.array_equal(got, brute_conv(qa, levels, (1, 1), (1, 1)))
+    # Eq. 2 with the paper's unsigned codes: sum (2 q_u - L) a = 2 * bitplane_sum(q_u, a) - L * window_sum(a)
+    ones = np.ones_like(qs)
+    window = brute_conv(qa, ones, (1, 1), (1, 1))
+    unsigned_route = 2 * oracle.conv2d_bitplanes(qa, qu, wb, ab, (1, 1), (1, 1), signed_w=False).astype(np.int64) - L * window
+    assert np.array_equal(got, unsigned_route)
+    # and the form the GPU uses: 2 * (signed bit-plane sum) + window sum
+    assert np.array_equal(got, 2 * oracle.conv2d_codes(qa, qs, (1, 1), (1, 1)).astype(np.int64) + window)
+
+
+def test_weight_level_quantizer_is_eq1a(oracle):
+    """q_u = round_half_up(L * (w_n/2 + 1/2)) for normalised weights w_n in [-1, 1], step 1/L."""
+    for b in (1, 2, 3, 4, 8):
+        L = (1 << b) - 1
+        wn = np.linspace(-1.2, 1.2, 481).astype(np.float32)
+        x = L * (wn.astype(np.float64) / 2 + 0.5)
+        safe = np.abs(x - np.floor(x) - 0.5) > 1e-4
+        ref_qu = np.clip(np.floor(x + 0.5), 0, L).astype(np.int32)
+        got = oracle.quantize_weight_levels(wn, 1.0 / L, b) + (1 << (b - 1))
+        assert np.array_equal(got[safe], ref_qu[safe]), b
+        hat = (2 * got - L) / L                                  # the de-quantized weight of Eq. 1a
+        assert hat.min() == -1.0 and hat.max() == 1.0
+    # exact ties with a power-of-two step go up
+    q = oracle.quantize_weight_levels(np.array([0.0, -2.0, 2.0, -0.5, 100.0, -100.0], np.float32), 1.0, 2)
+    #   v=0: (0+3)/2=1.5 -> 2 ; v=-2: 0.5 -> 1 ; v=2: 2.5 -> 3 ; v=-.5: 1.25 -> 1 ; clamp 3 ; clamp 0     (q_u)
+    assert (q + 2).tolist() == [2, 1, 3, 1, 3, 0]
