@@ -212,6 +212,22 @@ conv_mma_kernel(const ConvParams p) {
 #pragma unroll 1
         for (int q = 0; q < KSTEP; ++q) {
             if ((q & (p.fold - 1)) == 0 && st * KSTEP + q < p.KK) {
+                if (p.w_levels) {            // window sum of the activation codes: every lane reads the whole
+                                             // words of its rows g and g+8, so it can count them itself
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt) {
+                        const int r0 = (wp * MT + mt) * 16 + g;
+                        for (int f = 0; f < p.fold && q + f < KSTEP; ++f) {
+                            const uint32_t* row0 = A_s + ((q + f) * TILE_P + r0) * AB;
+                            const uint32_t* row1 = row0 + 8 * AB;
+#pragma unroll
+                            for (int k = 0; k < AB; ++k) {
+                                wsum[mt][0] += __popc(row0[k]) << k;
+                                wsum[mt][1] += __popc(row1[k]) << k;
+                            }
+                        }
+                    }
+                }
                 // activation fragments: byte = 2^k where bit k-plane is set
                 uint32_t af[MT][AB][4];
 #pragma unroll
@@ -237,10 +253,6 @@ conv_mma_kernel(const ConvParams p) {
 #pragma unroll
                     for (int k = 0; k < AB; ++k) {
                         const uint32_t w0 = wr0[k], w1 = wr1[k];
-                        if (p.w_levels) {                   // every lane holds the whole word of its two rows
-                            wsum[mt][0] += __popc(w0) << k;
-                            wsum[mt][1] += __popc(w1) << k;
-                        }
                         const uint32_t mask = 0x01010101u << k;
                         af[mt][k][0] = __funnelshift_r(w0, w0, tq - k) & mask;
                         af[mt][k][1] = __funnelshift_r(w1, w1, tq - k) & mask;
@@ -297,6 +309,14 @@ conv_mma_kernel(const ConvParams p) {
     const int qmax = (1 << p.next_bits) - 1;
     const bool pair_ok = (p.Co & 1) == 0;                   // two adjacent channels form an aligned 8-byte pair
     // common case: even c_out, no per-channel terms, no residual, NHWC -> straight-line code
+    if (p.w_levels) {                                       // accumulator = 2 * plane sum + window sum
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 2 * acc[mt][nt][e] + wsum[mt][e >> 1];
+    }
     const bool simple = pair_ok && !p.ch_scale && !p.ch_bias && !p.residual && !p.y_nchw;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
@@ -311,8 +331,7 @@ conv_mma_kernel(const ConvParams p) {
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
-                    int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
-                    if (p.w_levels) { a0 = 2 * a0 + wsum[mt][half]; a1 = 2 * a1 + wsum[mt][half]; }
+                    const int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
                     const bool valid = pvalid && co < p.Co;
                     int code0 = 0, code1 = 0;
                     if (valid && p.acc) *reinterpret_cast<int2*>(p.acc + row_o + nt * 8) = make_int2(a0, a1);
@@ -332,8 +351,7 @@ conv_mma_kernel(const ConvParams p) {
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 const int cl = (wc * NT + nt) * 8 + 2 * tq, co = co0 + cl;
-                int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
-                if (p.w_levels) { a0 = 2 * a0 + wsum[mt][half]; a1 = 2 * a1 + wsum[mt][half]; }
+                const int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
                 int code0 = 0, code1 = 0;
                 if (pvalid && co < p.Co) {
                     const size_t o = (size_t)gp * p.Co + co;
