@@ -4,6 +4,8 @@ Full sizes run on the GPU exactly as bench.py launches them (heuristic kernel ch
 checks every output where it finishes in seconds (configs 1 and 2) and otherwise every output of
 sampled images / sampled GEMM rows, which it computes one by one.
 """
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -16,7 +18,10 @@ RTOL = 1e-5
 def ebs():
     if not torch.cuda.is_available():
         pytest.skip("needs a CUDA device")
+    import paper_2003_07577_b200 as pkg
     from paper_2003_07577_b200 import binding
+    if not os.path.exists(binding.LIB_PATH):
+        pkg.build()
     binding.lib()
     return binding
 

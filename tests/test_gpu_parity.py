@@ -5,6 +5,8 @@ relative (they are in fact computed with the same individually rounded operation
 """
 import itertools
 
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -18,7 +20,10 @@ RTOL = 1e-5
 def ebs():
     if not torch.cuda.is_available():
         pytest.skip("needs a CUDA device")
+    import paper_2003_07577_b200 as pkg
     from paper_2003_07577_b200 import binding
+    if not os.path.exists(binding.LIB_PATH):
+        pkg.build()
     binding.lib()
     return binding
 
