@@ -92,6 +92,9 @@ typedef struct ebs_conv_desc {
  *   y = y * ch_scale[co]               if ch_scale_dev
  *   y = y + ch_bias[co]                if ch_bias_dev
  *   y = y + residual[n][ho][wo][co]    if residual_dev   (fp32, NHWC, output shape)
+ *   y = y + res_scale * code           if res_packed_dev (the shortcut of a residual block given as packed
+ *                                      activation planes u32 [N][Ho][Wo][ceil(C_out/32)][res_bits], e.g. the block's
+ *                                      own packed input: it is de-quantized on the fly, one rounded multiply)
  *   y = max(y, 0)                      if relu
  *   q = clamp(floor(y * (1/next_a_scale) + 0.5), 0, 2^next_a_bits - 1)   (packed output only)
  * A NULL epilogue means: no per-channel terms, no residual, no ReLU, y in NHWC.
@@ -104,6 +107,9 @@ typedef struct ebs_epilogue {
     int next_a_bits;           /* bitwidth of packed_next (1..8); ignored if packed_next is NULL */
     float next_a_scale;        /* step of the next layer's activation quantizer */
     int y_layout;              /* ebs_layout of y_out */
+    const void *res_packed_dev; /* nullable; packed planes with the output's pixel grid and c_out channels */
+    int res_bits;              /* planes of res_packed_dev (1..8) */
+    float res_scale;           /* real value of a residual code */
 } ebs_epilogue;
 
 /* Library version (major*10000 + minor*100 + patch). */
@@ -195,6 +201,14 @@ long long ebs_device_wait_timeouts(void);
 int ebs_dequant(const int32_t *acc_dev, size_t n_pixels, int c_out, float scale,
                 const float *ch_scale_dev, const float *ch_bias_dev, int relu, float *y_dev,
                 void *stream);
+
+/*
+ * Global average pooling between the last residual block and the classifier of the ResNets the
+ * paper evaluates (Sec. 5); not part of the binary decomposition itself.  y_dev is fp32 NHWC
+ * [n][hw][c]; out_dev receives [n][c]: the pixels are added in order 0 .. hw-1 in fp32 and the
+ * sum is multiplied by fl(1/hw).
+ */
+int ebs_global_avgpool(const float *y_dev, int n, int hw, int c, float *out_dev, void *stream);
 
 /*
  * One layer from HOST buffers, for callers whose data lives on the host: copies the activations

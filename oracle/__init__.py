@@ -179,6 +179,23 @@ def epilogue(acc, S, ch_scale=None, ch_bias=None, residual=None, relu=False, nex
     return y, q
 
 
+def dequant_codes(q, step) -> np.ndarray:
+    """The value a code stands for: fl32(step * code) (Eq. 1b's second line, one fp32 product)."""
+    return (np.float32(step) * np.asarray(q).astype(np.float32)).astype(np.float32)
+
+
+def global_avgpool(y) -> np.ndarray:
+    """Average over the pixels of [N, C, H, W] fp32 values, as the ResNets of Sec. 5 do before the
+    classifier: pixels are added one by one in row-major order in fp32, then multiplied by fl32(1/HW)."""
+    y = np.asarray(y, dtype=np.float32)
+    n, c, h, w = y.shape
+    acc = np.zeros((n, c), dtype=np.float32)
+    for i in range(h):
+        for j in range(w):
+            acc = (acc + y[:, :, i, j]).astype(np.float32)
+    return (acc * (np.float32(1.0) / np.float32(h * w))).astype(np.float32)
+
+
 def pack_acts(qa, a_bits: int) -> np.ndarray:
     """uint32 [N, H, W, ceil(C/32), Ab] bit-plane words, built bit by bit."""
     qa = _i32(qa)

@@ -25,7 +25,7 @@ EXPORTS = [
     "ebs_version", "ebs_status_string", "ebs_last_cuda_error", "ebs_conv_out_shape", "ebs_packed_weight_bytes",
     "ebs_packed_act_bytes", "ebs_pack_weights", "ebs_pack_acts", "ebs_conv2d_mixed", "ebs_num_conv_variants",
     "ebs_conv2d_mixed_variant", "ebs_dequant", "ebs_host_workspace_bytes", "ebs_conv2d_mixed_host",
-    "ebs_probe_pipe", "ebs_device_wait_timeouts", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
+    "ebs_probe_pipe", "ebs_device_wait_timeouts", "ebs_global_avgpool", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
 ]
 
 
@@ -39,7 +39,8 @@ class ebs_conv_desc(ctypes.Structure):
 class ebs_epilogue(ctypes.Structure):
     _fields_ = [("ch_scale_dev", ctypes.c_void_p), ("ch_bias_dev", ctypes.c_void_p),
                 ("residual_dev", ctypes.c_void_p), ("relu", ctypes.c_int), ("next_a_bits", ctypes.c_int),
-                ("next_a_scale", ctypes.c_float), ("y_layout", ctypes.c_int)]
+                ("next_a_scale", ctypes.c_float), ("y_layout", ctypes.c_int), ("res_packed_dev", ctypes.c_void_p),
+                ("res_bits", ctypes.c_int), ("res_scale", ctypes.c_float)]
 
 
 class EbsError(RuntimeError):
@@ -82,6 +83,7 @@ def lib() -> ctypes.CDLL:
         L.ebs_host_workspace_bytes.restype = z
         L.ebs_conv2d_mixed_host.argtypes = [p, i, i, i, i, i, p, D, E, p, z, p, p, p, p]
         L.ebs_probe_pipe.argtypes = [i, i, ctypes.POINTER(ctypes.c_double)]
+        L.ebs_global_avgpool.argtypes = [p, i, i, i, p, p]
         L.ebs_noalloc_scratch_bytes.restype = z
         L.ebs_device_wait_timeouts.restype = ctypes.c_longlong
         L.ebs_conv2d_mixed_host_noalloc.argtypes = [p, i, i, i, i, i, p, D, E, p, p, p, p]
@@ -111,12 +113,13 @@ def conv_desc(c_in, c_out, kh, kw, stride_h, stride_w, pad_h, pad_w, w_bits, a_b
 
 
 def epilogue(ch_scale=None, ch_bias=None, residual=None, relu=False, next_a_bits=0, next_a_scale=1.0,
-             y_layout=EBS_NHWC) -> ebs_epilogue:
+             y_layout=EBS_NHWC, res_packed=None, res_bits=0, res_scale=0.0) -> ebs_epilogue:
     e = ebs_epilogue(None if ch_scale is None else ch_scale.data_ptr(),
                      None if ch_bias is None else ch_bias.data_ptr(),
                      None if residual is None else residual.data_ptr(),
-                     int(bool(relu)), int(next_a_bits), float(next_a_scale), int(y_layout))
-    e._keepalive = (ch_scale, ch_bias, residual)
+                     int(bool(relu)), int(next_a_bits), float(next_a_scale), int(y_layout),
+                     None if res_packed is None else res_packed.data_ptr(), int(res_bits), float(res_scale))
+    e._keepalive = (ch_scale, ch_bias, residual, res_packed)
     return e
 
 
@@ -194,6 +197,10 @@ def ebs_probe_pipe(kind: int, iters: int = 2000) -> float:
     out = ctypes.c_double(0.0)
     _check(lib().ebs_probe_pipe(kind, iters, ctypes.byref(out)), "ebs_probe_pipe")
     return out.value
+
+
+def ebs_global_avgpool(y_dev, n: int, hw: int, c: int, out_dev, stream=None) -> None:
+    _check(lib().ebs_global_avgpool(_ptr(y_dev), n, hw, c, _ptr(out_dev), _stream(stream)), "ebs_global_avgpool")
 
 
 def ebs_device_wait_timeouts() -> int:

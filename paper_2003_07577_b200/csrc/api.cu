@@ -161,7 +161,8 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
     }
     if (epi) {
         if (epi->y_layout != EBS_NCHW && epi->y_layout != EBS_NHWC) return EBS_ERR_INVALID_ARG;
-        if (!aligned16(epi->residual_dev)) return EBS_ERR_INVALID_ARG;
+        if (!aligned16(epi->residual_dev) || !aligned16(epi->res_packed_dev)) return EBS_ERR_INVALID_ARG;
+        if (epi->res_packed_dev && (epi->res_bits < 1 || epi->res_bits > 8)) return EBS_ERR_INVALID_ARG;
     }
     if (variant >= NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS) return EBS_ERR_INVALID_ARG;
 
@@ -182,6 +183,7 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
     p.fold_bits = 32 / p.fold;
     if (epi) {
         p.ch_scale = epi->ch_scale_dev; p.ch_bias = epi->ch_bias_dev; p.residual = epi->residual_dev;
+        p.res_packed = static_cast<const uint32_t*>(epi->res_packed_dev); p.res_bits = epi->res_bits; p.res_scale = epi->res_scale;
         p.relu = epi->relu ? 1 : 0;
         p.y_nchw = epi->y_layout == EBS_NCHW;
         if (packed_next) { p.next_bits = epi->next_a_bits; p.inv_next = 1.0f / epi->next_a_scale; }
@@ -301,6 +303,12 @@ int ebs_dequant(const int32_t* acc_dev, size_t n_pixels, int c_out, float scale,
     if (n_pixels >= ((size_t)1 << 40) / (size_t)c_out) return EBS_ERR_OVERFLOW;
     return launch_dequant(acc_dev, n_pixels, c_out, scale, ch_scale_dev, ch_bias_dev, relu ? 1 : 0, y_dev,
                           static_cast<cudaStream_t>(stream));
+}
+
+int ebs_global_avgpool(const float* y_dev, int n, int hw, int c, float* out_dev, void* stream) {
+    if (!y_dev || !out_dev || n <= 0 || hw <= 0 || c <= 0) return EBS_ERR_INVALID_ARG;
+    if ((long long)n * c >= (1LL << 31)) return EBS_ERR_OVERFLOW;
+    return launch_avgpool(y_dev, n, hw, c, out_dev, static_cast<cudaStream_t>(stream));
 }
 
 static size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }

@@ -317,7 +317,7 @@ conv_mma_kernel(const ConvParams p) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 2 * acc[mt][nt][e] + wsum[mt][e >> 1];
     }
-    const bool simple = pair_ok && !p.ch_scale && !p.ch_bias && !p.residual && !p.y_nchw;
+    const bool simple = pair_ok && !p.ch_scale && !p.ch_bias && !p.residual && !p.res_packed && !p.y_nchw;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
@@ -373,6 +373,10 @@ conv_mma_kernel(const ConvParams p) {
                         if (p.residual) {
                             y0 = __fadd_rn(y0, __ldg(p.residual + o));
                             if (two) y1 = __fadd_rn(y1, __ldg(p.residual + o + 1));
+                        }
+                        if (p.res_packed) {
+                            y0 = __fadd_rn(y0, packed_residual(p, gp, co));
+                            if (two) y1 = __fadd_rn(y1, packed_residual(p, gp, co + 1));
                         }
                         if (p.relu) {
                             if (!(y0 > 0.0f)) y0 = 0.0f;

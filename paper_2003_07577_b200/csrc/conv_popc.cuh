@@ -176,6 +176,7 @@ conv_popc_kernel(const ConvParams p) {
                     if (p.ch_scale) yv = __fmul_rn(yv, __ldg(p.ch_scale + co));
                     if (p.ch_bias) yv = __fadd_rn(yv, __ldg(p.ch_bias + co));
                     if (p.residual) yv = __fadd_rn(yv, __ldg(p.residual + o));
+                    if (p.res_packed) yv = __fadd_rn(yv, packed_residual(p, gp, co));
                     if (p.relu && !(yv > 0.0f)) yv = 0.0f;
                     if (want_y) {
                         if (p.y_nchw) {

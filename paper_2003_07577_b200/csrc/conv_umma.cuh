@@ -399,6 +399,7 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
                         if (p.ch_scale) y = __fmul_rn(y, __ldg(p.ch_scale + co + e));
                         if (p.ch_bias) y = __fadd_rn(y, __ldg(p.ch_bias + co + e));
                         if (p.residual && pvalid) y = __fadd_rn(y, __ldg(p.residual + (size_t)gp * p.Co + co + e));
+                        if (p.res_packed && pvalid) y = __fadd_rn(y, packed_residual(p, gp, co + e));
                     }
                     if (p.relu && !(y > 0.0f)) y = 0.0f;
                     yv[e] = y;

@@ -48,6 +48,26 @@ __global__ void __launch_bounds__(256) dequant_kernel(const int32_t* __restrict_
     }
 }
 
+// Global average pooling of an NHWC fp32 tensor: one thread per (image, channel) adds the pixels in
+// order p = 0 .. hw-1 (a fixed order, so the result is reproducible bit for bit) and multiplies by
+// fl(1/hw).  Consecutive threads read consecutive channels, so every load is coalesced.
+__global__ void __launch_bounds__(256) avgpool_kernel(const float* __restrict__ y, int n, int hw, int c, float inv_hw,
+                                                      float* __restrict__ out) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= n * c) return;
+    const int img = idx / c, ch = idx - img * c;
+    const float* src = y + (size_t)img * hw * c + ch;
+    float acc = 0.0f;
+    for (int p = 0; p < hw; ++p) acc = __fadd_rn(acc, __ldg(src + (size_t)p * c));
+    out[idx] = __fmul_rn(acc, inv_hw);
+}
+
+int launch_avgpool(const float* y, int n, int hw, int c, float* out, cudaStream_t st) {
+    const int total = n * c;
+    avgpool_kernel<<<(total + 255) / 256, 256, 0, st>>>(y, n, hw, c, 1.0f / (float)hw, out);
+    return check_cuda(cudaGetLastError());
+}
+
 int launch_dequant(const int32_t* acc, size_t n_pixels, int c_out, float scale, const float* ch_scale,
                    const float* ch_bias, int relu, float* y, cudaStream_t st) {
     const size_t total = n_pixels * (size_t)c_out;

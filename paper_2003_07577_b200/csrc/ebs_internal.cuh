@@ -24,6 +24,9 @@ struct ConvParams {
     const float* __restrict__ ch_scale;
     const float* __restrict__ ch_bias;
     const float* __restrict__ residual;
+    const uint32_t* __restrict__ res_packed;   // nullable: shortcut as packed planes [P][CWo][res_bits]
+    int res_bits;
+    float res_scale;
     int relu;
     int next_bits;
     float inv_next;
@@ -76,6 +79,8 @@ int launch_pack_weights(const void* wt, int dtype, int layout, const ebs_conv_de
 // dequant.cu
 int launch_dequant(const int32_t* acc, size_t n_pixels, int c_out, float scale, const float* ch_scale,
                    const float* ch_bias, int relu, float* y, cudaStream_t st);
+
+int launch_avgpool(const float* y, int n, int hw, int c, float* out, cudaStream_t st);
 
 // Records a CUDA error for ebs_last_cuda_error() and returns EBS_ERR_CUDA (or EBS_OK).
 int check_cuda(cudaError_t e);
@@ -132,6 +137,15 @@ __device__ __forceinline__ int quantize_weight_level(float w, float inv_scale, i
 __device__ __forceinline__ int quantize_act_code(float y, float inv_scale, int qmax) {
     const float r = __fadd_rn(__fmul_rn(y, inv_scale), 0.5f);
     return min(max(__float2int_rd(r), 0), qmax);
+}
+
+// Shortcut of a residual block kept as packed planes: real value res_scale * code of channel co at
+// output pixel gp (one rounded multiply).
+__device__ __forceinline__ float packed_residual(const ConvParams& p, int gp, int co) {
+    const uint32_t* w = p.res_packed + ((size_t)gp * p.CWo + (co >> 5)) * p.res_bits;
+    uint32_t code = 0u;
+    for (int j = 0; j < p.res_bits; ++j) code |= ((__ldg(w + j) >> (co & 31)) & 1u) << j;
+    return __fmul_rn(p.res_scale, (float)code);
 }
 
 // Row pitch (bytes) of the tile of requantized codes kept in shared memory: 4 bytes of padding make

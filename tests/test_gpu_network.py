@@ -1,0 +1,179 @@
+"""GPU parity of the whole-network wiring: the shortcut taken from packed codes inside the epilogue,
+global average pooling, and a complete ResNet-20 forward pass chained through the C ABI, each against
+the CPU oracle on the same seeded inputs."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ebs():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import paper_2003_07577_b200 as pkg
+    from paper_2003_07577_b200 import binding
+    if not os.path.exists(binding.LIB_PATH):
+        pkg.build()
+    binding.lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def U(ebs):
+    from tests import _util
+    return _util
+
+
+@pytest.fixture(scope="module")
+def gen():
+    from workloads import gen as g
+    return g
+
+
+def _to(a, U):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(U.dev())
+
+
+@pytest.mark.parametrize("res_bits,co,next_bits", [(1, 16, 2), (2, 32, 3), (3, 64, 1), (4, 21, 4), (8, 70, 8), (5, 130, 2)])
+def test_shortcut_from_packed_codes(ebs, U, oracle, res_bits, co, next_bits):
+    """y += fl32(res_scale * code) with the codes read from packed planes, every kernel family."""
+    rng = np.random.default_rng(res_bits * 1000 + co)
+    wb, ab, c = 2, 3, 40
+    qa = U.rand_codes(rng, (2, c, 9, 7), ab, False)
+    qw = U.rand_codes(rng, (co, c, 3, 3), wb, True)
+    q_res = U.rand_codes(rng, (2, co, 9, 7), res_bits, False)
+    w_scale, a_scale, res_scale = 0.021, 0.04, 0.37 / ((1 << res_bits) - 1)
+    d = U.desc_for(c, co, 3, 1, 1, wb, ab, w_scale, a_scale)
+    acc = oracle.conv2d_codes(qa, qw, (1, 1), (1, 1))
+    S = oracle.combined_scale(w_scale, a_scale)
+    cb = rng.uniform(-0.2, 0.2, co).astype(np.float32)
+    res = oracle.dequant_codes(q_res, res_scale)
+    step = np.float32(0.9 / ((1 << next_bits) - 1))
+    y_ref, q_ref = oracle.epilogue(acc, S, None, cb, res, relu=True, next_bits=next_bits,
+                                   inv_next=np.float32(1.0) / step)
+    p_res = U.pack_acts_codes(q_res, res_bits)
+    epi = ebs.epilogue(None, _to(cb, U), None, True, next_bits, float(step), ebs.EBS_NHWC, res_packed=p_res,
+                       res_bits=res_bits, res_scale=res_scale)
+    for variant in (-1, 3, 6, 7, 11, 12, 14, 15, 17, 18, 20, 21, 22, 23):
+        out = U.run_conv(qa, qw, d, epi, want_acc=False, want_y=True, next_bits=next_bits, variant=variant)
+        assert np.array_equal(out["y"], y_ref), f"variant {variant}"
+        assert np.array_equal(oracle.unpack_acts(out["packed"], co), q_ref), f"variant {variant}"
+    assert 0 < q_ref.mean() < (1 << next_bits) - 1
+    # packed-only output (no fp32 tensor written) takes the same shortcut
+    out = U.run_conv(qa, qw, d, epi, want_acc=False, want_y=False, next_bits=next_bits)
+    assert np.array_equal(oracle.unpack_acts(out["packed"], co), q_ref)
+
+
+def test_shortcut_argument_checks(ebs, U):
+    d = U.desc_for(16, 16, 3, 1, 1, 2, 2)
+    px = torch.zeros(ebs.ebs_packed_act_bytes(1, 4, 4, 16, 2) // 4, dtype=torch.int32, device=U.dev())
+    pw = torch.zeros(ebs.ebs_packed_weight_bytes(d) // 4, dtype=torch.int32, device=U.dev())
+    y = torch.empty(1 * 4 * 4 * 16, dtype=torch.float32, device=U.dev())
+    for bits in (0, 9):
+        epi = ebs.epilogue(res_packed=px, res_bits=bits, res_scale=0.1)
+        with pytest.raises(RuntimeError):
+            ebs.ebs_conv2d_mixed(px, 1, 4, 4, pw, d, epi, None, y, None)
+
+
+@pytest.mark.parametrize("n,hw,c", [(3, 64, 64), (1, 49, 2048), (5, 7, 21), (128, 64, 64)])
+def test_global_avgpool(ebs, U, oracle, n, hw, c):
+    rng = np.random.default_rng(n + hw + c)
+    y = rng.standard_normal((n, c, hw, 1)).astype(np.float32) * 3.0
+    out = torch.empty((n, c), dtype=torch.float32, device=U.dev())
+    ebs.ebs_global_avgpool(_to(y.transpose(0, 2, 3, 1), U), n, hw, c, out)
+    assert np.array_equal(out.cpu().numpy(), oracle.global_avgpool(y))
+
+
+def _oracle_network(oracle, gen, specs, imgs, sample):
+    """The ResNet-20 forward pass in oracle calls on the sampled images.  Also fixes, per layer, the
+    folded-BatchNorm shift and the step of the next quantizer (a calibration: any positive values
+    would serve the comparison, these keep the codes spread over their range)."""
+    x = imgs[sample]
+    a0 = 1.0 / 255.0
+    plan, trace = {}, {}
+    by_name = {s.layer.name: s for s in specs}
+    order = [s.layer.name for s in specs]
+
+    def conv(spec, src, a_scale, residual=None, relu=True, nb=0):
+        L = spec.layer
+        acc = oracle.conv2d_codes(src, gen.weight_codes(spec), (L.stride, L.stride), (L.pad, L.pad))
+        S = oracle.combined_scale(spec.w_scale, a_scale)
+        gain = 1.0 / max(float(np.std(acc)) * float(S), 1e-12)          # folded BatchNorm: unit variance, zero mean
+        cs = np.full(L.c_out, gain, np.float32)
+        bias = np.full(L.c_out, -float(np.mean(acc)) * float(S) * gain, np.float32)
+        y0, _ = oracle.epilogue(acc, S, cs, bias, residual, relu=relu)
+        step = 0.0
+        q = None
+        if nb:
+            step = float(np.float32(max(np.percentile(y0, 99.5), 1e-6) / ((1 << nb) - 1)))
+            _, q = oracle.epilogue(acc, S, cs, bias, residual, relu=relu, next_bits=nb,
+                                   inv_next=np.float32(1.0) / np.float32(step))
+        plan[L.name] = dict(a_scale=a_scale, bias=bias, scale=cs, out_bits=nb, out_step=step)
+        trace[L.name] = q
+        return y0, q, step
+
+    blocks = [nm[:-2] for nm in order if nm.endswith("c1")]
+    first = by_name["conv1"]
+    nb = by_name[blocks[0] + "c1"].a_bits
+    _, qx, sx = conv(first, x, a0, nb=nb)
+    y_last = None
+    for bi, tag in enumerate(blocks):
+        c1, c2, ds = by_name[tag + "c1"], by_name[tag + "c2"], by_name.get(tag + "ds")
+        _, qt, st = conv(c1, qx, sx, nb=c2.a_bits)
+        if ds is not None:
+            res, _, _ = conv(ds, qx, sx, relu=False)
+        else:
+            res = oracle.dequant_codes(qx, sx)
+        nb = by_name[blocks[bi + 1] + "c1"].a_bits if bi + 1 < len(blocks) else 0
+        y_last, qx, sx = conv(c2, qt, st, residual=res, nb=nb)
+    pooled = oracle.global_avgpool(y_last)
+    fc = by_name["fc"]
+    s_fc = float(np.float32(max(float(pooled.max()), 1e-6) / 255.0))
+    qp = oracle.quantize_acts(pooled.reshape(len(sample), -1, 1, 1), s_fc, 8)
+    logits, _, _ = conv(fc, qp, s_fc, relu=False)
+    return plan, trace, logits.reshape(len(sample), -1), qp
+
+
+def _gpu_network(ebs, U, gen, specs, plan):
+    from paper_2003_07577_b200.network import BasicBlockNet, ConvPlan
+    plans = []
+    for spec in specs:
+        L, pl = spec.layer, plan[spec.layer.name]
+        d = ebs.conv_desc(L.c_in, L.c_out, L.k, L.k, L.stride, L.stride, L.pad, L.pad, spec.w_bits, spec.a_bits,
+                          spec.w_scale, pl["a_scale"])
+        plans.append(ConvPlan(L.name, L.role, d, L.h_in, L.w_in, U.pack_weight_codes(gen.weight_codes(spec), d),
+                              ch_bias=_to(pl["bias"], U), ch_scale=_to(pl["scale"], U), out_bits=pl["out_bits"], out_step=pl["out_step"]))
+    return BasicBlockNet(plans, U.dev())
+
+
+def test_resnet20_forward_matches_the_oracle(ebs, U, oracle, gen):
+    """Whole network at batch 32: every layer's packed output and the logits of the sampled images
+    equal the oracle's, bit for bit."""
+    n = 32
+    sample = [0, 13, 31]
+    specs = gen.resnet20_network(0, n)
+    imgs = gen.images_u8(0, n)
+    plan, trace, logits_ref, qp_ref = _oracle_network(oracle, gen, specs, imgs, sample)
+    net = _gpu_network(ebs, U, gen, specs, plan)
+    x = _to(imgs.astype(np.uint8).transpose(0, 2, 3, 1), U)
+    for _ in range(2):                                    # second pass reuses every buffer
+        logits = net.forward(x)
+        torch.cuda.synchronize()
+    for spec in specs:
+        L, q_ref = spec.layer, trace[spec.layer.name]
+        if q_ref is None:
+            continue
+        bits = plan[L.name]["out_bits"]
+        got = oracle.unpack_acts(U.packed_images(net._buf[(L.name, "q")], n, L.h_out, L.w_out, L.c_out, bits, sample),
+                                 L.c_out)
+        assert np.array_equal(got, q_ref), f"{L.name} W{spec.w_bits}A{spec.a_bits}"
+        assert 0 < q_ref.mean() < (1 << bits) - 1
+    got_p = oracle.unpack_acts(U.packed_images(net._buf[("pool", "q")], n, 1, 1, 64, 8, sample), 64)
+    assert np.array_equal(got_p, qp_ref)
+    assert np.array_equal(logits[sample].cpu().numpy(), logits_ref)
+    assert np.unique(logits_ref.argmax(axis=1)).size >= 1 and np.isfinite(logits_ref).all()
+    assert ebs.ebs_device_wait_timeouts() == 0

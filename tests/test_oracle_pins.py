@@ -377,3 +377,27 @@ def test_weight_level_quantizer_is_eq1a(oracle):
     q = oracle.quantize_weight_levels(np.array([0.0, -2.0, 2.0, -0.5, 100.0, -100.0], np.float32), 1.0, 2)
     #   v=0: (0+3)/2=1.5 -> 2 ; v=-2: 0.5 -> 1 ; v=2: 2.5 -> 3 ; v=-.5: 1.25 -> 1 ; clamp 3 ; clamp 0     (q_u)
     assert (q + 2).tolist() == [2, 1, 3, 1, 3, 0]
+
+
+def test_global_avgpool_pins(oracle):
+    """Exact where the mathematics fixes it (integers with a power-of-two pixel count, constants);
+    within fp32 summation error of the float64 mean elsewhere; order of axes checked by a ramp."""
+    rng = np.random.default_rng(5)
+    yi = rng.integers(-100, 100, size=(3, 5, 8, 8)).astype(np.float32)
+    assert np.array_equal(oracle.global_avgpool(yi), yi.astype(np.float64).mean(axis=(2, 3)).astype(np.float32))
+    y = rng.standard_normal((2, 7, 6, 5)).astype(np.float32)
+    ref = y.astype(np.float64).mean(axis=(2, 3))
+    got = oracle.global_avgpool(y)
+    assert got.dtype == np.float32 and got.shape == (2, 7)
+    assert np.allclose(got, ref, rtol=0, atol=30 * 2.0 ** -24 * np.abs(y).sum(axis=(2, 3)).max() / 30)
+    ramp = np.zeros((2, 3, 4, 4), np.float32)
+    ramp[1, 2] = 16.0
+    assert np.array_equal(oracle.global_avgpool(ramp), np.array([[0, 0, 0], [0, 0, 16]], np.float32))
+
+
+def test_dequant_codes_is_one_fp32_product(oracle):
+    q = np.arange(0, 256)
+    step = np.float32(0.0371)
+    got = oracle.dequant_codes(q, step)
+    assert got.dtype == np.float32
+    assert np.array_equal(got, np.array([np.float32(float(step) * int(v)) for v in q], np.float32))

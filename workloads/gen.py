@@ -137,3 +137,29 @@ def binary_ops(spec: LayerSpec, batch: Optional[int] = None) -> int:
     """2 * MACs * Wb * Ab: one AND and one bitcount-accumulate per bit pair (Sec. 4.3, complexity)."""
     n = spec.batch if batch is None else batch
     return 2 * n * spec.layer.macs * spec.w_bits * spec.a_bits
+
+
+def resnet20_network(seed: int = 0, batch: int = 128) -> List[LayerSpec]:
+    """The ResNet-20 stack of config2 wired as a network: a projection shortcut reads the same
+    tensor as its block's first convolution, so it takes that layer's activation bitwidth."""
+    specs = config2(seed, batch)
+    by_name = {s.layer.name: s for s in specs}
+    out = []
+    for s in specs:
+        if s.layer.role == "shortcut":
+            first = by_name[s.layer.name[:-2] + "c1"]
+            s = LayerSpec(s.index, s.layer, s.w_bits, first.a_bits, s.w_scale, first.a_scale, s.batch, s.dist, s.seed)
+        out.append(s)
+    return out
+
+
+def images_u8(seed: int, batch: int, h: int = 32, w: int = 32, c: int = 3) -> np.ndarray:
+    """Synthetic 8-bit images [N, C, H, W]: smooth per-image gradients plus noise, so that pixel
+    statistics differ between images and channels the way natural images' do."""
+    rng = np.random.default_rng([int(seed), 4242])
+    yy, xx = np.meshgrid(np.linspace(0, 1, h), np.linspace(0, 1, w), indexing="ij")
+    gx = rng.uniform(-1, 1, size=(batch, c, 1, 1))
+    gy = rng.uniform(-1, 1, size=(batch, c, 1, 1))
+    base = rng.uniform(0.2, 0.8, size=(batch, c, 1, 1))
+    img = base + 0.3 * gx * xx + 0.3 * gy * yy + 0.08 * rng.standard_normal(size=(batch, c, h, w))
+    return np.clip(np.floor(img * 255.0 + 0.5), 0, 255).astype(np.int32)
