@@ -228,8 +228,8 @@ conv_mma_kernel(const ConvParams p) {
                         }
                     }
                 }
-                // activation fragments: byte = 2^k where bit k-plane is set
-                uint32_t af[MT][AB][4];
+                // activation fragments: the planes of a channel merged back into its code, byte = sum_k 2^k bit_k
+                uint32_t af[MT][4];
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     const int r0 = (wp * MT + mt) * 16 + g;
@@ -250,18 +250,20 @@ conv_mma_kernel(const ConvParams p) {
                             }
                         }
                     }
+                    af[mt][0] = af[mt][1] = af[mt][2] = af[mt][3] = 0u;
 #pragma unroll
                     for (int k = 0; k < AB; ++k) {
                         const uint32_t w0 = wr0[k], w1 = wr1[k];
                         const uint32_t mask = 0x01010101u << k;
-                        af[mt][k][0] = __funnelshift_r(w0, w0, tq - k) & mask;
-                        af[mt][k][1] = __funnelshift_r(w1, w1, tq - k) & mask;
-                        af[mt][k][2] = __funnelshift_r(w0, w0, tq + 4 - k) & mask;
-                        af[mt][k][3] = __funnelshift_r(w1, w1, tq + 4 - k) & mask;
+                        af[mt][0] |= __funnelshift_r(w0, w0, tq - k) & mask;
+                        af[mt][1] |= __funnelshift_r(w1, w1, tq - k) & mask;
+                        af[mt][2] |= __funnelshift_r(w0, w0, tq + 4 - k) & mask;
+                        af[mt][3] |= __funnelshift_r(w1, w1, tq + 4 - k) & mask;
                     }
                 }
-                // weight fragments: byte = 2^m, or -2^(WB-1) (two's complement byte) for the top plane
-                uint32_t bf[NT][WB][2];
+                // weight fragments: the planes merged into the two's-complement code, byte = sum_m c_m 2^m bit_m.
+                // The top plane contributes -2^(WB-1) = the byte with bits WB-1 .. 7 set (sign extension).
+                uint32_t bf[NT][2];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     const uint32_t* row = W_s + (q * TILE_C + (wc * NT + nt) * 8 + g) * WB;
@@ -275,6 +277,7 @@ conv_mma_kernel(const ConvParams p) {
                             for (int m = 0; m < WB; ++m) wr[m] |= t[m] << (f * p.fold_bits);
                         }
                     }
+                    bf[nt][0] = bf[nt][1] = 0u;
 #pragma unroll
                     for (int m = 0; m < WB; ++m) {
                         const uint32_t w = wr[m];
@@ -285,18 +288,14 @@ conv_mma_kernel(const ConvParams p) {
                             b0 *= (1u << (9 - WB)) - 1u;
                             b1 *= (1u << (9 - WB)) - 1u;
                         }
-                        bf[nt][m][0] = b0;
-                        bf[nt][m][1] = b1;
+                        bf[nt][0] |= b0;
+                        bf[nt][1] |= b1;
                     }
                 }
 #pragma unroll
-                for (int m = 0; m < WB; ++m)
+                for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-                    for (int k = 0; k < AB; ++k)
-#pragma unroll
-                        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                            for (int nt = 0; nt < NT; ++nt) mma_u8s8(acc[mt][nt], af[mt][k], bf[nt][m][0], bf[nt][m][1]);
+                    for (int nt = 0; nt < NT; ++nt) mma_u8s8(acc[mt][nt], af[mt], bf[nt][0], bf[nt][1]);
             }
         }
         __syncthreads();

@@ -1,21 +1,25 @@
 // Implicit-GEMM bit-plane convolution on the 5th-generation tensor cores (tcgen05.mma kind::i8,
 // accumulator in tensor memory), sm_100a.
 //
-// Same arithmetic as conv_mma_kernel: activation plane k is expanded to bytes 2^k * bit, weight plane m
-// to bytes 2^m * bit (the top plane to -2^(M-1) * bit), and one int8 MMA of plane k against plane m adds
-// c_m 2^(m+k) * bitcount(AND(plane k, plane m)) -- Eq. 13 and Eq. 14 at once -- into ONE int32
-// accumulator per output.  Here an MMA covers 128 output pixels x TILE_N channels x 32 reduction bits,
-// reads both operands from shared memory and accumulates in tensor memory (TMEM).
+// Same arithmetic as conv_mma_kernel.  The plane-pair sum of the binary decomposition,
+//     sum_m sum_k c_m 2^(m+k) * bitcount(AND(activation plane k, weight plane m)),
+// regroups channel by channel into (sum_k 2^k a_k) * (sum_m c_m 2^m w_m): the expanders merge the
+// planes of a packed word back into one byte per channel (the activation code as u8, the weight code
+// as two's-complement s8, the top plane supplying the sign extension), and ONE int8 MMA per reduction
+// word then retires all Wb*Ab plane pairs of its 32 channels into one int32 accumulator per output.
+// An MMA covers 128 output pixels x TILE_N channels x 32 channels of one tap, reads both operands
+// from shared memory and accumulates in tensor memory (TMEM).  Operands stay bit planes in global
+// memory; bytes exist only in shared memory.
 //
 // A CTA owns 128 consecutive output pixels x TILE_N channels and has 9 warps:
-//   warps 0-7 (expanders)  load packed words one stage ahead into registers, expand them -- the
-//      thread's pixel row for its share of the activation planes and its share of the weight rows --
-//      into 32-byte rows of K-major, 32-byte-swizzled shared tiles (one tile per plane and reduction
-//      word; byte 4b+i of a row <- bit 8i+b of the word, the same map for both operands), then
+//   warps 0-7 (expanders)  load packed words ahead into registers and expand them into 32-byte rows of
+//      K-major, 32-byte-swizzled shared tiles (one tile per reduction word; byte 4b+i of a row <- bit
+//      8i+b of the words, the same map for both operands): threads t and t+128 build the two 16-byte
+//      halves of pixel row t, and the weight rows are dealt out over all 256 threads; then
 //      fence.proxy.async and arrive on the stage's "full" mbarrier;
-//   warp 8 (issuer)        waits for "full", issues Wb*Ab tcgen05.mma per reduction word (one per
-//      plane pair) and a tcgen05.commit that arrives on the stage's "empty" mbarrier once the tensor
-//      core has read the stage.
+//   warp 8 (issuer)        waits for "full", issues one tcgen05.mma per reduction word and a
+//      tcgen05.commit that arrives on the stage's "empty" mbarrier once the tensor core has read the
+//      stage.
 // Two stages, so expansion of the next reduction words overlaps the MMAs of the current ones.
 // Epilogue: tcgen05.ld gives every expander thread accumulators of its pixel (warps w and w+4 split
 // the channels); it stores them, applies the fp32 steps and packs the requantized codes of its pixel
@@ -99,17 +103,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 }
 
-// One packed word -> one 32-byte row (two 16-byte chunks) of plane-coefficient bytes.
-// Byte 4b+i of the row is (bit 8i+b of the word) * coefficient; `scale` = 1, or 2^(9-Wb)-1 for the
-// top weight plane so that its byte is the two's-complement byte of -2^(Wb-1).
-__device__ __forceinline__ void expand_word_to_row(uint32_t word, int plane, uint32_t scale, uint4& lo, uint4& hi) {
-    const uint32_t mask = 0x01010101u << plane;
-    uint32_t r[8];
-#pragma unroll
-    for (int b = 0; b < 8; ++b) r[b] = (__funnelshift_r(word, word, b - plane) & mask) * scale;
-    lo = make_uint4(r[0], r[1], r[2], r[3]);
-    hi = make_uint4(r[4], r[5], r[6], r[7]);
-}
 // Address of 16-byte chunk c (0/1) of row `row` in a 32-byte-swizzled tile (tile base 256-byte aligned).
 __device__ __forceinline__ uint8_t* sw32_chunk(uint8_t* tile, int row, int c) {
     return tile + row * 32 + ((c ^ ((row >> 2) & 1)) << 4);
@@ -118,18 +111,24 @@ __device__ __forceinline__ uint8_t* sw32_chunk(uint8_t* tile, int row, int c) {
 constexpr int UMMA_EXPANDERS = 256;     // threads of warps 0-7
 constexpr int UMMA_THREADS = UMMA_EXPANDERS + 32;
 
+constexpr int umma_min(int a, int b) { return a < b ? a : b; }
+
 template <int WB, int AB, int TILE_N>
 struct UmmaTile {
-    static constexpr int A_PLANE_BYTES = UMMA_M * 32;                   // one activation plane, one reduction word
-    static constexpr int B_PLANE_BYTES = TILE_N * 32;
-    static constexpr int KW_BYTES = AB * A_PLANE_BYTES + WB * B_PLANE_BYTES;
-    static constexpr int KS_RAW = (24 * 1024) / KW_BYTES;               // reduction words per stage
-    static constexpr int KS = KS_RAW < 1 ? 1 : (KS_RAW > 4 ? 4 : KS_RAW);
+    static constexpr int A_TILE_BYTES = UMMA_M * 32;                    // activation codes of one reduction word
+    static constexpr int B_TILE_BYTES = TILE_N * 32;                    // weight codes of one reduction word
+    static constexpr int KW_BYTES = A_TILE_BYTES + B_TILE_BYTES;
+    // reduction words per stage: bounded by shared memory (32 KB a stage) and by the registers that hold
+    // the packed words of three chunks in flight (about 16 activation and 16 weight words per chunk)
+    static constexpr int KS_SMEM = (32 * 1024) / KW_BYTES;
+    static constexpr int KS_A = 16 / AB;
+    static constexpr int KS_B = (16 * UMMA_EXPANDERS) / (WB * TILE_N);
+    static constexpr int KS_MIN = umma_min(umma_min(KS_SMEM, KS_A), umma_min(KS_B, 4));
+    static constexpr int KS = KS_MIN < 1 ? 1 : KS_MIN;
     static constexpr int STAGE_BYTES = KS * KW_BYTES;
     static constexpr int SMEM_BYTES = 2 * STAGE_BYTES + 1024;           // + slack to align the tiles to 1 KB
     static constexpr int TMEM_COLS = TILE_N < 32 ? 32 : TILE_N;
-    static constexpr int A_ITEMS = KS * AB;                              // (reduction word, plane) per pixel row
-    static constexpr int B_ITEMS = (KS * WB * TILE_N + UMMA_EXPANDERS - 1) / UMMA_EXPANDERS;   // weight rows per thread
+    static constexpr int B_ITEMS = (KS * TILE_N + UMMA_EXPANDERS - 1) / UMMA_EXPANDERS;   // weight rows per thread
     static_assert(TILE_N % 16 == 0 && TILE_N >= 16 && TILE_N <= 256, "tcgen05.mma N for M = 128");
     static_assert((STAGE_BYTES % 256) == 0, "tiles keep the swizzle alignment");
     static_assert(SMEM_BYTES <= 220 * 1024, "shared memory per CTA");
@@ -184,7 +183,7 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
 
     if (warp < 8) {
         // =========================== expanders ===========================
-        const int half = tid >> 7;                             // which share of the activation items
+        const int half = tid >> 7;                             // which 16-byte half of its pixel row it builds
         int pix_off = 0;
         uint32_t row_ok = 0u, col_ok = 0u;
         if (gp < p.P) {
@@ -196,36 +195,33 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
             for (int r = 0; r < p.kh; ++r) row_ok |= ((unsigned)(h0 + r) < (unsigned)p.H ? 1u : 0u) << r;
             for (int s = 0; s < p.kw; ++s) col_ok |= ((unsigned)(w0 + s) < (unsigned)p.W ? 1u : 0u) << s;
         }
-        uint32_t a_set[3][KS][AB], b_set[3][T::B_ITEMS];   // packed words of three consecutive chunks (ring)
+        uint32_t a_set[3][KS][AB], b_set[3][T::B_ITEMS][WB];   // packed words of three consecutive chunks (ring)
 
-        // per-thread constants of the weight rows it expands: which (reduction word, plane, channel row),
-        // where that row starts in global memory (for reduction word 0) and in the stage
-        int b_q[T::B_ITEMS], b_m[T::B_ITEMS], b_goff[T::B_ITEMS], b_soff[T::B_ITEMS];
+        // per-thread constants of the weight rows it expands: which (reduction word, channel row), where
+        // that row starts in global memory (for reduction word 0) and in the stage
+        int b_q[T::B_ITEMS], b_goff[T::B_ITEMS], b_soff[T::B_ITEMS];
 #pragma unroll
         for (int i = 0; i < T::B_ITEMS; ++i) {
             const int item = tid + i * UMMA_EXPANDERS;
-            const int q = item / (WB * TILE_N), rem = item - q * (WB * TILE_N);
-            const int m = rem / TILE_N, nrow = rem - m * TILE_N;
+            const int q = item / TILE_N, nrow = item - q * TILE_N;
             const bool live = q < KS && co0 + nrow < p.Co;
             b_q[i] = q < KS ? q : -1;                            // -1: no row (more threads than rows)
-            b_m[i] = m;
-            b_goff[i] = live ? (co0 + nrow) * WB + m : -1;        // -1: channel past c_out -> zero row
-            b_soff[i] = KS * AB * T::A_PLANE_BYTES + (q * WB + m) * T::B_PLANE_BYTES + nrow * 32;
+            b_goff[i] = live ? (co0 + nrow) * WB : -1;            // -1: channel past c_out -> zero row
+            b_soff[i] = KS * T::A_TILE_BYTES + q * T::B_TILE_BYTES + nrow * 32;
         }
-        const int sw = ((row >> 2) & 1) << 4;                     // 32-byte swizzle of this thread's pixel row
-        const int a_soff0 = row * 32 + sw, a_soff1 = row * 32 + (sw ^ 16);
+        const int a_soff = row * 32 + ((half ^ ((row >> 2) & 1)) << 4);   // this thread's chunk, 32-byte swizzle
         const int co_wb = p.Co * WB;                              // weight words per reduction word
 
         // packed words of chunk `ch` -> registers (zero past the end, outside the image, past c_out)
         auto load_chunk = [&](int ch, int set) {
             uint32_t (&a_nxt)[KS][AB] = a_set[set];
-            uint32_t (&b_nxt)[T::B_ITEMS] = b_set[set];
+            uint32_t (&b_nxt)[T::B_ITEMS][WB] = b_set[set];
 #pragma unroll
             for (int q = 0; q < KS; ++q) {
                 const int kw = ch * KS + q;
 #pragma unroll
                 for (int k = 0; k < AB; ++k) a_nxt[q][k] = 0u;
-                if ((((q * AB) & 1) == half || AB > 1) && kw < kwords) {     // this half uses a plane of word q
+                if (kw < kwords) {
                     if (p.fold == 1) {
                         const int2 info = ktab[kw];
                         if ((row_ok >> (info.y & 0xff)) & (col_ok >> (info.y >> 8)) & 1u)
@@ -247,20 +243,23 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
             }
 #pragma unroll
             for (int i = 0; i < T::B_ITEMS; ++i) {
-                uint32_t ww = 0u;
+#pragma unroll
+                for (int m = 0; m < WB; ++m) b_nxt[i][m] = 0u;
                 const int kw = ch * KS + b_q[i];
                 if (b_q[i] >= 0 && b_goff[i] >= 0 && kw < kwords) {
                     if (p.fold == 1) {
-                        ww = __ldg(p.w + (size_t)kw * co_wb + b_goff[i]);
+                        load_words_global<WB>(p.w + ((size_t)kw * co_wb + b_goff[i]), b_nxt[i]);
                     } else {
                         for (int f = 0; f < p.fold; ++f) {
                             const int kk = kw * p.fold + f;
                             if (kk >= p.KK) break;
-                            ww |= __ldg(p.w + (size_t)kk * co_wb + b_goff[i]) << (f * p.fold_bits);
+                            uint32_t t[WB];
+                            load_words_global<WB>(p.w + ((size_t)kk * co_wb + b_goff[i]), t);
+#pragma unroll
+                            for (int m = 0; m < WB; ++m) b_nxt[i][m] |= t[m] << (f * p.fold_bits);
                         }
                     }
                 }
-                b_nxt[i] = ww;
             }
         };
 
@@ -276,8 +275,8 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
                 const int ch = ch0 + u;
                 if (ch >= nchunks) break;
                 const int st = ch & 1;
-                uint8_t* A_st = tiles + st * T::STAGE_BYTES;           // [KS][AB] planes of 128 rows x 32 B, then
-                                                                       // [KS][WB] planes of TILE_N rows x 32 B
+                uint8_t* A_st = tiles + st * T::STAGE_BYTES;           // [KS] tiles of 128 rows x 32 B, then
+                                                                       // [KS] tiles of TILE_N rows x 32 B
                 if (ch + 2 < nchunks) load_chunk(ch + 2, (u + 2) % 3);
                 if (ch >= 2) {                                         // the MMAs of chunk ch-2 must have read the stage
                     if (!mbar_wait_bounded(&empty_bar[st], (uint32_t)(((ch >> 1) - 1) & 1), abortp)) {
@@ -286,31 +285,35 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
                     }
                 }
                 const uint32_t (&a_cur)[KS][AB] = a_set[u];
-                const uint32_t (&b_cur)[T::B_ITEMS] = b_set[u];
+                const uint32_t (&b_cur)[T::B_ITEMS][WB] = b_set[u];
 #pragma unroll
                 for (int q = 0; q < KS; ++q) {
+                    // activation codes: register b of the row holds channels {b, 8+b, 16+b, 24+b}
+                    uint32_t r[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
                     for (int k = 0; k < AB; ++k) {
-                        if (((q * AB + k) & 1) != half) continue;
-                        if (p.w_levels) wsum += __popc(a_cur[q][k]) << k;
-                        uint4 lo, hi;
-                        expand_word_to_row(a_cur[q][k], k, 1u, lo, hi);
-                        uint8_t* tile = A_st + (q * AB + k) * T::A_PLANE_BYTES;
-                        *reinterpret_cast<uint4*>(tile + a_soff0) = lo;
-                        *reinterpret_cast<uint4*>(tile + a_soff1) = hi;
+                        const uint32_t w = a_cur[q][k];
+                        if (p.w_levels && (k & 1) == half) wsum += __popc(w) << k;
+                        const uint32_t mask = 0x01010101u << k;
+#pragma unroll
+                        for (int bb = 0; bb < 4; ++bb) r[bb] |= __funnelshift_r(w, w, 4 * half + bb - k) & mask;
                     }
+                    *reinterpret_cast<uint4*>(A_st + q * T::A_TILE_BYTES + a_soff) = make_uint4(r[0], r[1], r[2], r[3]);
                 }
 #pragma unroll
                 for (int i = 0; i < T::B_ITEMS; ++i) {
                     if (b_q[i] >= 0) {
-                        const int m = b_m[i];
-                        // rotate once by the plane, then the eight byte groups are fixed rotations of that
-                        const uint32_t wrot = __funnelshift_l(b_cur[i], b_cur[i], m);
-                        const uint32_t mask = 0x01010101u << m;
-                        const uint32_t scale = (m == WB - 1 && WB < 8) ? ((1u << (9 - WB)) - 1u) : 1u;
-                        uint32_t r[8];
+                        // weight codes: planes below the top one give the low bits, the top plane the byte
+                        // 256 - 2^(WB-1) (bits WB-1 .. 7 set): two's-complement sign extension
+                        uint32_t r[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
 #pragma unroll
-                        for (int bb = 0; bb < 8; ++bb) r[bb] = (__funnelshift_r(wrot, wrot, bb) & mask) * scale;
+                        for (int m = 0; m < WB; ++m) {
+                            const uint32_t w = b_cur[i][m];
+                            const uint32_t mask = 0x01010101u << m;
+                            const uint32_t scale = (m == WB - 1 && WB < 8) ? ((1u << (9 - WB)) - 1u) : 1u;
+#pragma unroll
+                            for (int bb = 0; bb < 8; ++bb) r[bb] |= (__funnelshift_r(w, w, bb - m) & mask) * scale;
+                        }
                         uint8_t* dst = A_st + b_soff[i];
                         const int bsw = (b_soff[i] >> 3) & 16;           // ((row >> 2) & 1) << 4 with row = offset / 32
                         *reinterpret_cast<uint4*>(dst + bsw) = make_uint4(r[0], r[1], r[2], r[3]);
@@ -333,20 +336,13 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
             if ((tid & 31) == 0) {
                 const uint32_t a_base = smem_u32(tiles + st * T::STAGE_BYTES);
-                const uint32_t b_base = a_base + KS * AB * T::A_PLANE_BYTES;
+                const uint32_t b_base = a_base + KS * T::A_TILE_BYTES;
                 const uint64_t da0 = umma_desc_sw32(a_base), db0 = umma_desc_sw32(b_base);
-#pragma unroll 1
+#pragma unroll
                 for (int q = 0; q < KS; ++q) {
                     if (ch * KS + q >= kwords) break;
-#pragma unroll 1
-                    for (int m = 0; m < WB; ++m) {
-                        const uint64_t db = db0 + (uint64_t)(((q * WB + m) * T::B_PLANE_BYTES) >> 4);
-#pragma unroll
-                        for (int k = 0; k < AB; ++k) {
-                            const uint64_t da = da0 + (uint64_t)(((q * AB + k) * T::A_PLANE_BYTES) >> 4);
-                            umma_i8(tmem_base, da, db, IDESC, (ch | q | m | k) != 0 ? 1u : 0u);
-                        }
-                    }
+                    umma_i8(tmem_base, da0 + (uint64_t)((q * T::A_TILE_BYTES) >> 4),
+                            db0 + (uint64_t)((q * T::B_TILE_BYTES) >> 4), IDESC, (ch | q) != 0 ? 1u : 0u);
                 }
                 umma_commit(&empty_bar[st]);
             }

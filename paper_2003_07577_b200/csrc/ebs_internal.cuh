@@ -140,12 +140,19 @@ __device__ __forceinline__ int quantize_act_code(float y, float inv_scale, int q
 }
 
 // Shortcut of a residual block kept as packed planes: real value res_scale * code of channel co at
-// output pixel gp (one rounded multiply).
-__device__ __forceinline__ float packed_residual(const ConvParams& p, int gp, int co) {
-    const uint32_t* w = p.res_packed + ((size_t)gp * p.CWo + (co >> 5)) * p.res_bits;
+// output pixel gp (one rounded multiply).  Deliberately not inlined: only the epilogue of a layer
+// with such a shortcut calls it, and inlining it raised the register count of every kernel (and so
+// lowered the occupancy of layers that never take this path).  Arguments are scalars so that the
+// kernel parameter block is not copied to local memory.
+static __device__ __noinline__ float packed_residual_at(const uint32_t* __restrict__ res_packed, int CWo, int res_bits,
+                                                 float res_scale, int gp, int co) {
+    const uint32_t* w = res_packed + ((size_t)gp * CWo + (co >> 5)) * res_bits;
     uint32_t code = 0u;
-    for (int j = 0; j < p.res_bits; ++j) code |= ((__ldg(w + j) >> (co & 31)) & 1u) << j;
-    return __fmul_rn(p.res_scale, (float)code);
+    for (int j = 0; j < res_bits; ++j) code |= ((__ldg(w + j) >> (co & 31)) & 1u) << j;
+    return __fmul_rn(res_scale, (float)code);
+}
+__device__ __forceinline__ float packed_residual(const ConvParams& p, int gp, int co) {
+    return packed_residual_at(p.res_packed, p.CWo, p.res_bits, p.res_scale, gp, co);
 }
 
 // Row pitch (bytes) of the tile of requantized codes kept in shared memory: 4 bytes of padding make
