@@ -459,7 +459,7 @@ def run_gpu(args):
     per_layer, roof_ms = [], 0.0
     for L, t in zip(layers, conv_ms):
         lay = L.spec.layer
-        bytes_alg = (L.px.numel() * 4 + L.pw.numel() * 4 + L.acc.numel() * 4 + L.pn_bytes)
+        bytes_alg = (L.px.numel() * 4 + ebs.ebs_packed_weight_plane_bytes(L.d) + L.acc.numel() * 4 + L.pn_bytes)
         t_tensor, t_hbm = L.ops / (peak_tops * 1e12), bytes_alg / (hbm_gbs * 1e9)
         roof = max(t_tensor, t_hbm)
         roof_ms += roof * 1e3

@@ -125,9 +125,18 @@ const char *ebs_last_cuda_error(void);
  * Returns EBS_ERR_INVALID_ARG if the kernel is larger than the padded input. */
 int ebs_conv_out_shape(const ebs_conv_desc *desc, int h, int w, int *h_out, int *w_out);
 
-/* Size in bytes of the packed weight planes of a layer: kh*kw*ceil(c_in/32)*c_out*w_bits*4.
- * "BD incurs the same memory cost as the weights before BD" (Sec. 4.3, complexity).  0 on bad input. */
+/* Size in bytes of the packed weight buffer of a layer.  It has two parts:
+ *   1. the bit planes B_w, kh*kw*ceil(c_in/32)*c_out*w_bits 32-bit words laid out
+ *      [kh][kw][ceil(c_in/32)][c_out][w_bits], the same memory as the weights before decomposition
+ *      (Sec. 4.3, complexity), rounded up to a multiple of 256 bytes
+ *      (ebs_packed_weight_plane_bytes);
+ *   2. the same codes once more as one signed byte per (tap, channel, output channel) in the
+ *      order the tensor-core kernels read them, kh*kw*ceil(c_in/32)*roundup(c_out,16)*32 bytes.
+ *      The paper has no counterpart for part 2: it is a prepared copy of a static operand, written
+ *      once by ebs_pack_weights, so that those kernels do not rebuild it in every thread block.
+ * 0 on bad input. */
 size_t ebs_packed_weight_bytes(const ebs_conv_desc *desc);
+size_t ebs_packed_weight_plane_bytes(const ebs_conv_desc *desc);
 
 /* Size in bytes of packed activation planes: n*h*w*ceil(c/32)*a_bits*4.  0 on bad input. */
 size_t ebs_packed_act_bytes(int n, int h, int w, int c, int a_bits);

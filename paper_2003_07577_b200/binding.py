@@ -25,7 +25,7 @@ EXPORTS = [
     "ebs_version", "ebs_status_string", "ebs_last_cuda_error", "ebs_conv_out_shape", "ebs_packed_weight_bytes",
     "ebs_packed_act_bytes", "ebs_pack_weights", "ebs_pack_acts", "ebs_conv2d_mixed", "ebs_num_conv_variants",
     "ebs_conv2d_mixed_variant", "ebs_dequant", "ebs_host_workspace_bytes", "ebs_conv2d_mixed_host",
-    "ebs_probe_pipe", "ebs_device_wait_timeouts", "ebs_global_avgpool", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
+    "ebs_probe_pipe", "ebs_device_wait_timeouts", "ebs_global_avgpool", "ebs_packed_weight_plane_bytes", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
 ]
 
 
@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.ebs_conv_out_shape.argtypes = [D, i, i, ctypes.POINTER(i), ctypes.POINTER(i)]
         L.ebs_packed_weight_bytes.argtypes = [D]
         L.ebs_packed_weight_bytes.restype = z
+        L.ebs_packed_weight_plane_bytes.argtypes = [D]
+        L.ebs_packed_weight_plane_bytes.restype = z
         L.ebs_packed_act_bytes.argtypes = [i, i, i, i, i]
         L.ebs_packed_act_bytes.restype = z
         L.ebs_pack_weights.argtypes = [p, i, i, D, p, p]
@@ -139,6 +141,10 @@ def ebs_conv_out_shape(desc: ebs_conv_desc, h: int, w: int):
 
 def ebs_packed_weight_bytes(desc: ebs_conv_desc) -> int:
     return lib().ebs_packed_weight_bytes(ctypes.byref(desc))
+
+
+def ebs_packed_weight_plane_bytes(desc: ebs_conv_desc) -> int:
+    return lib().ebs_packed_weight_plane_bytes(ctypes.byref(desc))
 
 
 def ebs_packed_act_bytes(n: int, h: int, w: int, c: int, a_bits: int) -> int:

@@ -58,7 +58,8 @@ const ConvVariant* conv_umma_variant(int w_bits, int a_bits, int variant) {
 
 unsigned long long conv_umma_timeouts() {
     return conv_umma_timeouts_w1() + conv_umma_timeouts_w2() + conv_umma_timeouts_w3() + conv_umma_timeouts_w4() +
-           conv_umma_timeouts_w5() + conv_umma_timeouts_w6() + conv_umma_timeouts_w7() + conv_umma_timeouts_w8();
+           conv_umma_timeouts_w5() + conv_umma_timeouts_w6() + conv_umma_timeouts_w7() + conv_umma_timeouts_w8() +
+           conv_umma_strip_timeouts();
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -127,15 +128,30 @@ static int choose_mma_variant(int w_bits, int a_bits, int P, int Co, int sms) {
     return 6 + tc_idx;
 }
 
-// tcgen05 kernels pay off when a CTA's 128 x tile_n accumulator sees many MMAs (deep reduction, several
-// plane pairs), the channel tile is wide enough to amortise the activation expansion, and the layer
-// has enough output tiles; smaller layers run faster on the warp-level kernels.  (Rule fitted to
-// per-variant timings of the ResNet-18/20/50 layer shapes.)  Returns the umma variant or -1.
+// Stride-1 layers with at least 64 output channels and enough outputs to fill the GPU run on the strip
+// kernel (every input pixel expanded once per CTA, weights fetched as bytes).  The channel tile is the
+// largest of 256/128/64 that divides c_out, so that every tile is whole and takes the straight-line
+// epilogue; failing that the largest not above c_out.  (Rule fitted to per-variant timings of the
+// ResNet-18/20/50 layer shapes.)  Returns the strip variant or -1.
+static int choose_strip_variant(const ConvParams& p) {
+    if (p.Co < 64 || (long long)p.P * p.Co < (1LL << 20)) return -1;
+    int pick = -1;
+    for (int v = 4; v >= 2; --v)
+        if (p.Co % (16 << v) == 0) { pick = v; break; }
+    if (pick < 0) pick = p.Co >= 256 ? 4 : (p.Co >= 128 ? 3 : 2);
+    for (; pick >= 2; --pick)
+        if (conv_umma_strip_applies(p, pick)) return pick;
+    return -1;
+}
+
+// The per-tap tcgen05 kernels (any stride) pay off when a CTA's 128 x tile_n accumulator sees a deep
+// reduction, the channel tile is wide enough to amortise the activation expansion, and the layer has
+// enough output tiles; smaller layers run faster on the warp-level kernels.  Returns the variant or -1.
 static int choose_umma_variant(const ConvParams& p, const ebs_conv_desc* d) {
     const int kwords = (p.KK + p.fold - 1) / p.fold;
-    const long long mmas_per_tile = (long long)kwords * d->w_bits * d->a_bits;
     const long long outputs = (long long)p.P * p.Co;
-    if (p.Co < 64 || mmas_per_tile < 48) return -1;
+    (void)d;
+    if (p.Co < 64 || kwords < 8) return -1;
     if (outputs < (1LL << 20) && kwords < 72) return -1;
     return p.Co >= 128 ? 3 : 2;             // tile_n 128 or 64
 }
@@ -164,12 +180,15 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
         if (!aligned16(epi->residual_dev) || !aligned16(epi->res_packed_dev)) return EBS_ERR_INVALID_ARG;
         if (epi->res_packed_dev && (epi->res_bits < 1 || epi->res_bits > 8)) return EBS_ERR_INVALID_ARG;
     }
-    if (variant >= NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS) return EBS_ERR_INVALID_ARG;
+    constexpr int STRIP_BASE = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS;
+    if (variant >= STRIP_BASE + NUM_CONV_STRIP_VARIANTS) return EBS_ERR_INVALID_ARG;
 
     ConvParams p;
     memset(&p, 0, sizeof(p));
     p.x = static_cast<const uint32_t*>(packed_x);
     p.w = static_cast<const uint32_t*>(packed_w);
+    p.w8 = static_cast<const uint8_t*>(packed_w) + packed_weight_plane_bytes(*d);
+    p.Co16 = (d->c_out + 15) & ~15;
     p.N = n; p.H = h; p.W = w; p.CW = (d->c_in + 31) / 32;
     p.Co = d->c_out; p.Ho = Ho; p.Wo = Wo; p.CWo = (d->c_out + 31) / 32;
     p.kh = d->kh; p.kw = d->kw; p.sh = d->stride_h; p.sw = d->stride_w; p.ph = d->pad_h; p.pw = d->pad_w;
@@ -190,13 +209,17 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
     }
     const bool mma_ok = mma_path_supported(p, d);
     if (variant < 0) {
-        const int umma = mma_ok ? choose_umma_variant(p, d) : -1;
-        if (umma >= 0) variant = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + umma;
+        const int strip = mma_ok ? choose_strip_variant(p) : -1;
+        const int umma = (mma_ok && strip < 0) ? choose_umma_variant(p, d) : -1;
+        if (strip >= 0) variant = STRIP_BASE + strip;
+        else if (umma >= 0) variant = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + umma;
         else variant = mma_ok ? NUM_CONV_VARIANTS + choose_mma_variant(d->w_bits, d->a_bits, p.P, p.Co, sm_count())
                               : choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
     }
     if (variant >= NUM_CONV_VARIANTS && !mma_ok) return EBS_ERR_UNSUPPORTED;
+    if (variant >= STRIP_BASE && !conv_umma_strip_applies(p, variant - STRIP_BASE)) return EBS_ERR_UNSUPPORTED;
     const ConvVariant* v =
+        variant >= STRIP_BASE ? conv_umma_strip_variant(d->a_bits, variant - STRIP_BASE) :
         variant >= NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS
             ? conv_umma_variant(d->w_bits, d->a_bits, variant - NUM_CONV_VARIANTS - NUM_CONV_MMA_VARIANTS)
             : (variant >= NUM_CONV_VARIANTS ? conv_mma_variant(d->w_bits, d->a_bits, variant - NUM_CONV_VARIANTS)
@@ -245,7 +268,12 @@ int ebs_conv_out_shape(const ebs_conv_desc* d, int h, int w, int* h_out, int* w_
 
 size_t ebs_packed_weight_bytes(const ebs_conv_desc* d) {
     if (validate_desc(d)) return 0;
-    return (size_t)d->kh * d->kw * ((d->c_in + 31) / 32) * d->c_out * d->w_bits * sizeof(uint32_t);
+    return packed_weight_plane_bytes(*d) + packed_weight_image_bytes(*d);
+}
+
+size_t ebs_packed_weight_plane_bytes(const ebs_conv_desc* d) {
+    if (validate_desc(d)) return 0;
+    return packed_weight_plane_bytes(*d);
 }
 
 size_t ebs_packed_act_bytes(int n, int h, int w, int c, int a_bits) {
@@ -285,7 +313,9 @@ int ebs_conv2d_mixed(const void* packed_x_dev, int n, int h, int w, const void* 
                      stream, -1);
 }
 
-int ebs_num_conv_variants(void) { return NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS; }
+int ebs_num_conv_variants(void) {
+    return NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS + NUM_CONV_STRIP_VARIANTS;
+}
 
 long long ebs_device_wait_timeouts(void) { return (long long)conv_umma_timeouts(); }
 

@@ -108,6 +108,175 @@ __device__ __forceinline__ uint8_t* sw32_chunk(uint8_t* tile, int row, int c) {
     return tile + row * 32 + ((c ^ ((row >> 2) & 1)) << 4);
 }
 
+// Epilogue straight out of tensor memory.  Warp w reads TMEM lanes 32 * (w % 4) .. + 31: thread `lane`
+// of it owns the accumulators of one pixel row (global output pixel gp; pvalid false = row without an
+// output).  Warps w and w + 4 split the channels when the tile is wide enough.  The thread stores the
+// accumulators, applies the fp32 steps and packs the requantized codes of its pixel into plane words.
+template <int TILE_N>
+__device__ __forceinline__ void umma_epilogue(const ConvParams& p, uint32_t tmem_base, int warp, int gp, bool pvalid,
+                                              int wsum_row, int co0) {
+    constexpr int EPI_WARPS = TILE_N >= 64 ? 8 : 4;
+    constexpr int COLS_PER_WARP = TILE_N >= 64 ? TILE_N / 2 : TILE_N;
+    if (warp < EPI_WARPS) {
+        const bool want_y = p.y != nullptr, want_q = p.packed_next != nullptr;
+        const int qmax = (1 << p.next_bits) - 1;
+        const bool vec_ok = (p.Co & 3) == 0;                        // 16-byte aligned groups of four channels
+        const uint32_t trow = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+        const int hw = p.Ho * p.Wo;
+        const int img = pvalid ? gp / hw : 0, rem = pvalid ? gp - img * hw : 0;
+        const int cbeg = (warp >> 2) * COLS_PER_WARP;
+        // Common case -- the whole channel tile exists, channels in aligned groups of four, no per-channel
+        // terms, no shortcut, NHWC: straight-line code, 32 channels (one packed output word) per round.
+        if (COLS_PER_WARP % 32 == 0 && co0 + TILE_N <= p.Co && vec_ok && !p.ch_scale && !p.ch_bias && !p.residual &&
+            !p.res_packed && !p.y_nchw) {
+            const int nb = want_q ? p.next_bits : 0;
+            const float S = p.S, inv_next = p.inv_next;
+            const bool relu = p.relu != 0, w_levels = p.w_levels != 0;
+#pragma unroll 1
+            for (int c0 = cbeg; c0 < cbeg + COLS_PER_WARP; c0 += 32) {
+                uint32_t planes[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    uint32_t v[16];
+                    tmem_ld16(trow + (uint32_t)(c0 + 16 * hf), v);   // whole warp, also for rows past the end
+                    if (w_levels) {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) v[e] = (uint32_t)(2 * (int)v[e] + wsum_row);
+                    }
+                    const size_t o = (size_t)gp * p.Co + co0 + c0 + 16 * hf;
+                    if (p.acc && pvalid) {
+#pragma unroll
+                        for (int gq = 0; gq < 4; ++gq)
+                            *reinterpret_cast<int4*>(p.acc + o + 4 * gq) =
+                                make_int4((int)v[4 * gq], (int)v[4 * gq + 1], (int)v[4 * gq + 2], (int)v[4 * gq + 3]);
+                    }
+                    if (want_y || want_q) {
+                        float y[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            y[e] = __fmul_rn((float)(int)v[e], S);
+                            if (relu) y[e] = y[e] > 0.0f ? y[e] : 0.0f;
+                        }
+                        if (want_y && pvalid) {
+#pragma unroll
+                            for (int gq = 0; gq < 4; ++gq)
+                                *reinterpret_cast<float4*>(p.y + o + 4 * gq) =
+                                    make_float4(y[4 * gq], y[4 * gq + 1], y[4 * gq + 2], y[4 * gq + 3]);
+                        }
+                        if (want_q) {
+                            uint32_t c4[4];
+#pragma unroll
+                            for (int gq = 0; gq < 4; ++gq) {
+                                c4[gq] = 0u;
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    c4[gq] |= (uint32_t)quantize_act_code(y[4 * gq + e], inv_next, qmax) << (8 * e);
+                            }
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                if (j >= nb) break;
+                                uint32_t bits16 = 0u;                 // plane j of these 16 channels
+#pragma unroll
+                                for (int gq = 0; gq < 4; ++gq)
+                                    bits16 |= ((((c4[gq] >> j) & 0x01010101u) * 0x01020408u) >> 24) << (4 * gq);
+                                planes[j] |= bits16 << (16 * hf);
+                            }
+                        }
+                    }
+                }
+                if (want_q && pvalid) {
+                    uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + ((co0 + c0) >> 5)) * nb;
+                    if (nb == 4) {
+                        *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
+                    } else if (nb == 8) {
+                        *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
+                        *reinterpret_cast<uint4*>(dst + 4) = make_uint4(planes[4], planes[5], planes[6], planes[7]);
+                    } else if (nb == 2) {
+                        *reinterpret_cast<uint2*>(dst) = make_uint2(planes[0], planes[1]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (j >= nb) break;
+                            dst[j] = planes[j];
+                        }
+                    }
+                }
+            }
+            return;
+        }
+        uint32_t planes[8];
+#pragma unroll 1
+        for (int c0 = cbeg; c0 < cbeg + COLS_PER_WARP; c0 += 16) {
+            uint32_t v[16];
+            tmem_ld16(trow + (uint32_t)c0, v);                       // whole warp, also for rows past the end
+            if (p.w_levels) {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = (uint32_t)(2 * (int)v[e] + wsum_row);
+            }
+            if ((c0 & 31) == 0) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) planes[j] = 0u;
+            }
+#pragma unroll
+            for (int gq = 0; gq < 4; ++gq) {                          // four channels at a time
+                const int co = co0 + c0 + 4 * gq;
+                uint32_t code4 = 0u;
+                float yv[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int a = (int)v[4 * gq + e];
+                    float y = __fmul_rn((float)a, p.S);
+                    if (co + e < p.Co) {
+                        if (p.ch_scale) y = __fmul_rn(y, __ldg(p.ch_scale + co + e));
+                        if (p.ch_bias) y = __fadd_rn(y, __ldg(p.ch_bias + co + e));
+                        if (p.residual && pvalid) y = __fadd_rn(y, __ldg(p.residual + (size_t)gp * p.Co + co + e));
+                        if (p.res_packed && pvalid) y = __fadd_rn(y, packed_residual(p, gp, co + e));
+                    }
+                    if (p.relu && !(y > 0.0f)) y = 0.0f;
+                    yv[e] = y;
+                    if (want_q && co + e < p.Co) code4 |= (uint32_t)quantize_act_code(y, p.inv_next, qmax) << (8 * e);
+                }
+                if (pvalid && co < p.Co) {
+                    const size_t o = (size_t)gp * p.Co + co;
+                    if (p.acc) {
+                        if (vec_ok) *reinterpret_cast<int4*>(p.acc + o) =
+                            make_int4((int)v[4 * gq], (int)v[4 * gq + 1], (int)v[4 * gq + 2], (int)v[4 * gq + 3]);
+                        else
+                            for (int e = 0; e < 4 && co + e < p.Co; ++e) p.acc[o + e] = (int)v[4 * gq + e];
+                    }
+                    if (want_y) {
+                        if (p.y_nchw) {
+                            for (int e = 0; e < 4 && co + e < p.Co; ++e)
+                                p.y[((size_t)img * p.Co + co + e) * hw + rem] = yv[e];
+                        } else if (vec_ok) {
+                            *reinterpret_cast<float4*>(p.y + o) = make_float4(yv[0], yv[1], yv[2], yv[3]);
+                        } else {
+                            for (int e = 0; e < 4 && co + e < p.Co; ++e) p.y[o + e] = yv[e];
+                        }
+                    }
+                }
+                if (want_q) {
+                    const int nib_pos = ((c0 & 16) >> 2) + gq;          // which nibble of the 32-channel word
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (j < p.next_bits)
+                            planes[j] |= ((((code4 >> j) & 0x01010101u) * 0x01020408u) >> 24) << (4 * nib_pos);
+                }
+            }
+            const bool word_done = ((c0 & 16) != 0) || (c0 + 16 >= TILE_N);
+            if (want_q && word_done && pvalid) {
+                const int cwg = (co0 + c0) >> 5;
+                if (cwg < p.CWo) {
+                    uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + cwg) * p.next_bits;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (j < p.next_bits) dst[j] = planes[j];
+                }
+            }
+        }
+    }
+}
+
 constexpr int UMMA_EXPANDERS = 256;     // threads of warps 0-7
 constexpr int UMMA_THREADS = UMMA_EXPANDERS + 32;
 
@@ -355,90 +524,10 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const bool aborted = abort_flag != 0;
 
-    // ---- epilogue straight out of tensor memory: warps w and w+4 own the same 32 pixels and split the channels
-    constexpr int EPI_WARPS = TILE_N >= 64 ? 8 : 4;
-    constexpr int COLS_PER_WARP = TILE_N >= 64 ? TILE_N / 2 : TILE_N;
-    if (!aborted && warp < EPI_WARPS) {
-        const bool want_y = p.y != nullptr, want_q = p.packed_next != nullptr;
-        const int qmax = (1 << p.next_bits) - 1;
-        const bool pvalid = gp < p.P;
-        const bool vec_ok = (p.Co & 3) == 0;                        // 16-byte aligned groups of four channels
-        const uint32_t trow = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-        const int hw = p.Ho * p.Wo;
-        const int img = pvalid ? gp / hw : 0, rem = pvalid ? gp - img * hw : 0;
-        const int cbeg = (warp >> 2) * COLS_PER_WARP;
-        const int erow = (warp & 3) * 32 + (tid & 31);             // the pixel row whose accumulators this thread reads
-        const int wsum_row = p.w_levels ? wsum_s[0][erow] + wsum_s[1][erow] : 0;
-        uint32_t planes[8];
-#pragma unroll 1
-        for (int c0 = cbeg; c0 < cbeg + COLS_PER_WARP; c0 += 16) {
-            uint32_t v[16];
-            tmem_ld16(trow + (uint32_t)c0, v);                       // whole warp, also for rows past the end
-            if (p.w_levels) {
-#pragma unroll
-                for (int e = 0; e < 16; ++e) v[e] = (uint32_t)(2 * (int)v[e] + wsum_row);
-            }
-            if ((c0 & 31) == 0) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) planes[j] = 0u;
-            }
-#pragma unroll
-            for (int gq = 0; gq < 4; ++gq) {                          // four channels at a time
-                const int co = co0 + c0 + 4 * gq;
-                uint32_t code4 = 0u;
-                float yv[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int a = (int)v[4 * gq + e];
-                    float y = __fmul_rn((float)a, p.S);
-                    if (co + e < p.Co) {
-                        if (p.ch_scale) y = __fmul_rn(y, __ldg(p.ch_scale + co + e));
-                        if (p.ch_bias) y = __fadd_rn(y, __ldg(p.ch_bias + co + e));
-                        if (p.residual && pvalid) y = __fadd_rn(y, __ldg(p.residual + (size_t)gp * p.Co + co + e));
-                        if (p.res_packed && pvalid) y = __fadd_rn(y, packed_residual(p, gp, co + e));
-                    }
-                    if (p.relu && !(y > 0.0f)) y = 0.0f;
-                    yv[e] = y;
-                    if (want_q && co + e < p.Co) code4 |= (uint32_t)quantize_act_code(y, p.inv_next, qmax) << (8 * e);
-                }
-                if (pvalid && co < p.Co) {
-                    const size_t o = (size_t)gp * p.Co + co;
-                    if (p.acc) {
-                        if (vec_ok) *reinterpret_cast<int4*>(p.acc + o) =
-                            make_int4((int)v[4 * gq], (int)v[4 * gq + 1], (int)v[4 * gq + 2], (int)v[4 * gq + 3]);
-                        else
-                            for (int e = 0; e < 4 && co + e < p.Co; ++e) p.acc[o + e] = (int)v[4 * gq + e];
-                    }
-                    if (want_y) {
-                        if (p.y_nchw) {
-                            for (int e = 0; e < 4 && co + e < p.Co; ++e)
-                                p.y[((size_t)img * p.Co + co + e) * hw + rem] = yv[e];
-                        } else if (vec_ok) {
-                            *reinterpret_cast<float4*>(p.y + o) = make_float4(yv[0], yv[1], yv[2], yv[3]);
-                        } else {
-                            for (int e = 0; e < 4 && co + e < p.Co; ++e) p.y[o + e] = yv[e];
-                        }
-                    }
-                }
-                if (want_q) {
-                    const int nib_pos = ((c0 & 16) >> 2) + gq;          // which nibble of the 32-channel word
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        if (j < p.next_bits)
-                            planes[j] |= ((((code4 >> j) & 0x01010101u) * 0x01020408u) >> 24) << (4 * nib_pos);
-                }
-            }
-            const bool word_done = ((c0 & 16) != 0) || (c0 + 16 >= TILE_N);
-            if (want_q && word_done && pvalid) {
-                const int cwg = (co0 + c0) >> 5;
-                if (cwg < p.CWo) {
-                    uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + cwg) * p.next_bits;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        if (j < p.next_bits) dst[j] = planes[j];
-                }
-            }
-        }
+    // ---- epilogue: expander threads read the accumulators of their own pixel row
+    if (!aborted) {
+        const int wsum_row = (p.w_levels && warp < 8) ? wsum_s[0][row] + wsum_s[1][row] : 0;
+        umma_epilogue<TILE_N>(p, tmem_base, warp, gp, gp < p.P, wsum_row, co0);
     }
     if (aborted && tid == 0) atomicAdd(&g_umma_timeouts, 1ull);
 

@@ -12,6 +12,8 @@ namespace ebs {
 struct ConvParams {
     const uint32_t* __restrict__ x;   // packed activations [N][H][W][CW][AB]
     const uint32_t* __restrict__ w;   // packed weights     [kh][kw][CW][Co][WB]
+    const uint8_t* __restrict__ w8;   // byte image of the weights [kh*kw*CW][Co16][32] (second part of the buffer)
+    int Co16;                         // c_out rounded up to 16
     int N, H, W, CW;
     int Co, Ho, Wo, CWo;              // CWo = ceil(Co/32)
     int kh, kw, sh, sw, ph, pw;
@@ -34,6 +36,7 @@ struct ConvParams {
     int w_levels;                     // 1: accumulator = 2 * plane sum + window sum of the activation codes
     int fold;                         // taps OR-ed into one reduction word by the tensor-pipe kernels: 1, 2, 4, 8
     int fold_bits;                    // 32 / fold: bits each folded tap occupies (>= c_in)
+    int strip_pix, strip_ks;          // strip kernel only (set by its launcher): pixels of a strip, words per stage
 };
 
 // One instantiation of the popcount kernel: launch function + its tile geometry.
@@ -61,7 +64,11 @@ EBS_DECLARE_WB(5) EBS_DECLARE_WB(6) EBS_DECLARE_WB(7) EBS_DECLARE_WB(8)
 #undef EBS_DECLARE_WB
 
 // 5th-generation tensor-core kernels (conv_umma_w1.cu .. conv_umma_w8.cu); variant = log2(tile_n / 16).
-enum { NUM_CONV_UMMA_VARIANTS = 5 };
+enum { NUM_CONV_UMMA_VARIANTS = 5, NUM_CONV_STRIP_VARIANTS = 5 };
+// Stride-1 strip kernel (conv_umma_strip.cu): variants by channel tile 16 << variant.
+const ConvVariant* conv_umma_strip_variant(int a_bits, int variant);
+bool conv_umma_strip_applies(const ConvParams& p, int variant);
+unsigned long long conv_umma_strip_timeouts();
 const ConvVariant* conv_umma_variant(int w_bits, int a_bits, int variant);
 unsigned long long conv_umma_timeouts();
 #define EBS_DECLARE_WB(WB)                                                   \
@@ -80,6 +87,8 @@ int launch_pack_weights(const void* wt, int dtype, int layout, const ebs_conv_de
 int launch_dequant(const int32_t* acc, size_t n_pixels, int c_out, float scale, const float* ch_scale,
                    const float* ch_bias, int relu, float* y, cudaStream_t st);
 
+size_t packed_weight_plane_bytes(const ebs_conv_desc& d);   // bit-plane words, rounded up to 256 bytes
+size_t packed_weight_image_bytes(const ebs_conv_desc& d);   // byte image that follows them
 int launch_avgpool(const float* y, int n, int hw, int c, float* out, cudaStream_t st);
 
 // Records a CUDA error for ebs_last_cuda_error() and returns EBS_ERR_CUDA (or EBS_OK).

@@ -331,6 +331,44 @@ int launch_pack_acts(const void* x, int dtype, int layout, int n, int c, int h, 
     return check_cuda(cudaGetLastError());
 }
 
+// Byte image of the packed weights for the tcgen05 strip kernel: per reduction word kk = tap * CW + cw
+// and output channel co one 32-byte row of two's-complement codes (the planes merged, top plane as sign
+// extension), laid out [kk][Co16][32] with Co16 = c_out rounded up to 16.  Byte 4b + i of a row is
+// channel 8i + b of the word and the two 16-byte halves of row co are swapped when (co >> 2) & 1: the
+// order and the 32-byte swizzle the kernel's shared-memory operand tiles use, so that a tile is one
+// contiguous copy.  Rows co >= c_out are zero.
+__global__ void __launch_bounds__(256) weight_byte_image_kernel(const uint32_t* __restrict__ planes, long long rows,
+                                                                int Co, int Co16, int WB, uint4* __restrict__ out) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x; r < rows; r += stride) {
+        const long long kk = r / Co16;
+        const int co = (int)(r - kk * Co16);
+        uint32_t reg[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+        if (co < Co) {
+            const uint32_t* src = planes + ((size_t)kk * Co + co) * WB;
+            for (int m = 0; m < WB; ++m) {
+                const uint32_t w = __ldg(src + m);
+                const uint32_t mask = 0x01010101u << m;
+                const uint32_t scale = (m == WB - 1 && WB < 8) ? ((1u << (9 - WB)) - 1u) : 1u;
+#pragma unroll
+                for (int b = 0; b < 8; ++b) reg[b] |= (__funnelshift_r(w, w, b - m) & mask) * scale;
+            }
+        }
+        const int sw = (co >> 2) & 1;
+        out[r * 2 + sw] = make_uint4(reg[0], reg[1], reg[2], reg[3]);
+        out[r * 2 + (sw ^ 1)] = make_uint4(reg[4], reg[5], reg[6], reg[7]);
+    }
+}
+
+size_t packed_weight_plane_bytes(const ebs_conv_desc& d) {
+    const size_t raw = (size_t)d.kh * d.kw * ((d.c_in + 31) / 32) * d.c_out * d.w_bits * sizeof(uint32_t);
+    return (raw + 255) & ~(size_t)255;
+}
+size_t packed_weight_image_bytes(const ebs_conv_desc& d) {
+    const size_t co16 = ((size_t)d.c_out + 15) & ~(size_t)15;
+    return (size_t)d.kh * d.kw * ((d.c_in + 31) / 32) * co16 * 32;
+}
+
 int launch_pack_weights(const void* wt, int dtype, int layout, const ebs_conv_desc& d, float inv_scale,
                         uint32_t* out, cudaStream_t st) {
     const int CW = (d.c_in + 31) / 32;
@@ -342,6 +380,12 @@ int launch_pack_weights(const void* wt, int dtype, int layout, const ebs_conv_de
     else
         pack_weights_kernel<int8_t><<<grid, 256, 0, st>>>((const int8_t*)wt, layout, d.c_out, d.c_in, d.kh, d.kw, CW,
                                                           d.w_bits, inv_scale, d.w_levels, out);
+    if (check_cuda(cudaGetLastError())) return EBS_ERR_CUDA;
+    // second part of the buffer: the byte image, built from the plane words just written
+    const int Co16 = (d.c_out + 15) & ~15;
+    const long long rows = (long long)d.kh * d.kw * CW * Co16;
+    uint4* image = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(out) + packed_weight_plane_bytes(d));
+    weight_byte_image_kernel<<<grid_for(rows, sm_count()), 256, 0, st>>>(out, rows, d.c_out, Co16, d.w_bits, image);
     return check_cuda(cudaGetLastError());
 }
 

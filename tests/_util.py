@@ -40,6 +40,30 @@ def pack_weight_codes(qw: np.ndarray, d, layout=ebs.EBS_NCHW) -> torch.Tensor:
     return out
 
 
+def weight_planes(buf: torch.Tensor, d) -> np.ndarray:
+    """First part of a packed weight buffer: the plane words [kh][kw][CW][c_out][w_bits]."""
+    cw = (d.c_in + 31) // 32
+    n = d.kh * d.kw * cw * d.c_out * d.w_bits
+    return as_u32(buf)[:n].reshape(d.kh, d.kw, cw, d.c_out, d.w_bits)
+
+
+def weight_byte_image(buf: torch.Tensor, d) -> np.ndarray:
+    """Second part of a packed weight buffer decoded back to signed codes [c_out16, CW*32, kh, kw]:
+    undoes the half swap of rows with (co >> 2) & 1 and the byte order 4b + i <- channel 8i + b."""
+    cw = (d.c_in + 31) // 32
+    co16 = (d.c_out + 15) // 16 * 16
+    raw = buf.cpu().numpy().view(np.uint8)[ebs.ebs_packed_weight_plane_bytes(d):]
+    rows = raw[: d.kh * d.kw * cw * co16 * 32].reshape(d.kh, d.kw, cw, co16, 2, 16).copy()
+    swap = ((np.arange(co16) >> 2) & 1).astype(bool)
+    rows[:, :, :, swap] = rows[:, :, :, swap][..., ::-1, :]
+    rows = rows.reshape(d.kh, d.kw, cw, co16, 32)
+    j = np.arange(32)
+    chan = 8 * (j % 4) + j // 4                       # byte j = 4b + i holds channel 8i + b
+    out = np.zeros((d.kh, d.kw, cw, co16, 32), np.int8)
+    out[..., chan] = rows.view(np.int8)
+    return out.transpose(3, 2, 4, 0, 1).reshape(co16, cw * 32, d.kh, d.kw)
+
+
 def as_u32(t: torch.Tensor) -> np.ndarray:
     return t.cpu().numpy().view(np.uint32)
 
@@ -70,6 +94,27 @@ def run_conv(qa, qw, d, epi=None, want_acc=True, want_y=False, next_bits=0, vari
     if pn is not None:
         out["packed"] = as_u32(pn).reshape(n, ho, wo, (co + 31) // 32, next_bits)
     return out
+
+
+N_STRIP = 5     # the last variants are the stride-1 strip kernels
+
+
+def strip_variant_applies(d, w, tile_n):
+    """Host-side rule of the strip kernel: stride 1 (or a 1x1 layer without padding), a strip of at most 512 pixels, and two
+    stages of (strip + kh*kw weight tiles) within 200 KB of shared memory."""
+    pointwise = d.kh == 1 and d.kw == 1 and d.pad_h == 0 and d.pad_w == 0    # 1x1 without padding: any stride
+    if (d.stride_h != 1 or d.stride_w != 1) and not pointwise:
+        return False
+    strip = 128 + (d.kh - 1) * (w + 2 * d.pad_w) + d.kw - 1
+    pad = (strip + 7) // 8 * 8
+    return strip <= 512 and 2 * (pad * 32 + d.kh * d.kw * tile_n * 32) + 1024 + pad * 4 <= 200 * 1024
+
+
+def all_variants(d, w=16):
+    """Every kernel variant that applies to descriptor d on images of width w (-1 = the library's own choice)."""
+    n = ebs.ebs_num_conv_variants()
+    strip = [n - N_STRIP + i for i in range(N_STRIP) if strip_variant_applies(d, w, 16 << i)]
+    return list(range(-1, n - N_STRIP)) + strip
 
 
 def rand_codes(rng, shape, bits, signed):

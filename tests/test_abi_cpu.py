@@ -36,14 +36,17 @@ def test_library_exports_every_declared_symbol(ebs):
 
 def test_sizes_and_shapes(ebs):
     d = ebs.conv_desc(64, 64, 3, 3, 1, 1, 1, 1, 2, 2, 0.05, 0.05)
-    assert ebs.ebs_packed_weight_bytes(d) == 3 * 3 * 2 * 64 * 2 * 4       # same bits as the unpacked weights
-    assert ebs.ebs_packed_weight_bytes(d) * 8 == 64 * 64 * 9 * 2
+    assert ebs.ebs_packed_weight_plane_bytes(d) == 3 * 3 * 2 * 64 * 2 * 4   # same bits as the unpacked weights
+    assert ebs.ebs_packed_weight_plane_bytes(d) * 8 == 64 * 64 * 9 * 2
+    assert ebs.ebs_packed_weight_bytes(d) == 3 * 3 * 2 * 64 * 2 * 4 + 3 * 3 * 2 * 64 * 32   # + one byte per weight
+    d5 = ebs.conv_desc(3, 5, 1, 1, 1, 1, 0, 0, 3, 2, 0.05, 0.05)
+    assert ebs.ebs_packed_weight_plane_bytes(d5) == 256 and ebs.ebs_packed_weight_bytes(d5) == 256 + 16 * 32
     assert ebs.ebs_packed_act_bytes(1, 32, 32, 64, 2) == 32 * 32 * 2 * 2 * 4
     assert ebs.ebs_packed_act_bytes(2, 5, 5, 33, 3) == 2 * 25 * 2 * 3 * 4
     assert ebs.ebs_conv_out_shape(d, 32, 32) == (32, 32)
     d2 = ebs.conv_desc(3, 64, 7, 7, 2, 2, 3, 3, 8, 8, 0.05, 0.05)
     assert ebs.ebs_conv_out_shape(d2, 224, 224) == (112, 112)
-    assert ebs.ebs_version() >= 100 and ebs.ebs_num_conv_variants() == 24
+    assert ebs.ebs_version() >= 100 and ebs.ebs_num_conv_variants() == 29
     assert ebs.ebs_status_string(0) == "ok" and "overflow" in ebs.ebs_status_string(-3)
     assert ebs.ebs_host_workspace_bytes(d, 1, 32, 32, ebs.EBS_U8_CODES, 2) >= 65536 + 16384 + 2 * 262144 + 16384
 

@@ -71,8 +71,11 @@ def test_pack_weights(ebs, U, oracle, co, c, k, wb, layout):
     rng = np.random.default_rng(co + c + wb)
     qw = U.rand_codes(rng, (co, c, k, k), wb, True)
     d = U.desc_for(c, co, k, 1, k // 2, wb, 2)
-    got = U.as_u32(U.pack_weight_codes(qw, d, layout)).reshape(k, k, (c + 31) // 32, co, wb)
+    buf = U.pack_weight_codes(qw, d, layout)
+    got = U.weight_planes(buf, d)
     assert np.array_equal(got, oracle.pack_weights(qw, wb))
+    image = U.weight_byte_image(buf, d)                    # the byte copy of the same codes, zero padded
+    assert np.array_equal(image[:co, :c], qw) and not image[co:].any() and not image[:, c:].any()
     # fp32 weights go through the quantizer first
     scale = np.float32(0.043)
     wf = ((qw + rng.uniform(-0.4, 0.4, qw.shape)) * scale).astype(np.float32)
@@ -81,7 +84,8 @@ def test_pack_weights(ebs, U, oracle, co, c, k, wb, layout):
     src = np.ascontiguousarray(wf.transpose(0, 2, 3, 1)) if layout == ebs.EBS_NHWC else wf
     out = torch.empty(ebs.ebs_packed_weight_bytes(d2) // 4, dtype=torch.int32, device=U.dev())
     ebs.ebs_pack_weights(torch.from_numpy(src).to(U.dev()), ebs.EBS_F32, layout, d2, out)
-    assert np.array_equal(U.as_u32(out).reshape(got.shape), oracle.pack_weights(qref, wb))
+    assert np.array_equal(U.weight_planes(out, d2), oracle.pack_weights(qref, wb))
+    assert np.array_equal(U.weight_byte_image(out, d2)[:co, :c], qref)
 
 
 # ------------------------------------------------------------------ contraction + recombination (rows a3, a4)
@@ -95,7 +99,7 @@ def test_conv_all_bitwidth_pairs(ebs, U, oracle, wb, ab):
     d = U.desc_for(40, 21, 3, 1, 1, wb, ab)
     ref = oracle.conv2d_codes(qa, qw, (1, 1), (1, 1))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
-    for variant in (-1, 0, 4, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23):
+    for variant in (-1, 0, 4, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28):
         got = U.run_conv(qa, qw, d, variant=variant, px=px, pw=pw)["acc"]
         assert np.array_equal(got, ref), f"variant {variant}"
 
@@ -118,9 +122,16 @@ def test_conv_geometries_all_variants(ebs, U, oracle, geom):
     d = U.desc_for(c, co, k, s, pad, wb, ab)
     ref = oracle.conv2d_codes(qa, qw, (s, s), (pad, pad))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
-    for variant in range(-1, ebs.ebs_num_conv_variants()):
+    for variant in U.all_variants(d, w):
         got = U.run_conv(qa, qw, d, variant=variant, px=px, pw=pw)["acc"]
         assert got.shape == ref.shape and np.array_equal(got, ref), f"variant {variant}"
+
+
+def test_strip_kernel_refuses_strided_layers(ebs, U):
+    d = U.desc_for(32, 32, 3, 2, 1, 2, 2)
+    qa, qw = np.zeros((1, 32, 8, 8), np.int32), np.zeros((32, 32, 3, 3), np.int32)
+    with pytest.raises(RuntimeError):
+        U.run_conv(qa, qw, d, variant=ebs.ebs_num_conv_variants() - 1)
 
 
 def test_no_device_wait_timed_out(ebs):
@@ -186,7 +197,7 @@ def test_fused_epilogue_and_requantized_planes(ebs, U, oracle, next_bits, co):
     res_nhwc = to(res.transpose(0, 2, 3, 1))
     for y_layout in (ebs.EBS_NHWC, ebs.EBS_NCHW):
         epi = ebs.epilogue(to(cs), to(cb), res_nhwc, True, next_bits, float(next_scale), y_layout)
-        for variant in (-1, 3, 6, 7, 11, 12, 14, 15, 17, 18, 20, 21, 22, 23):
+        for variant in (-1, 3, 6, 7, 11, 12, 14, 15, 17, 18, 20, 21, 22, 23, 25, 26, 27, 28):
             out = U.run_conv(qa, qw, d, epi, want_acc=True, want_y=True, next_bits=next_bits, variant=variant)
             assert np.array_equal(out["acc"], ref_acc)
             assert np.allclose(out["y"], y_ref, rtol=RTOL, atol=0.0)
@@ -295,7 +306,7 @@ def test_conv_edge_cases_all_variants(ebs, U, oracle, case):
     d = U.desc_for(c, co, k, s, pad, wb, ab)
     ref = oracle.conv2d_codes(qa, qw, (s, s), (pad, pad))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
-    for variant in range(-1, ebs.ebs_num_conv_variants()):
+    for variant in U.all_variants(d, w):
         got = U.run_conv(qa, qw, d, variant=variant, px=px, pw=pw)["acc"]
         assert got.shape == ref.shape and np.array_equal(got, ref), f"variant {variant}"
     assert ebs.ebs_device_wait_timeouts() == 0
@@ -333,7 +344,7 @@ def test_conv_with_paper_weight_levels_all_variants(ebs, U, oracle, wb, ab, c, c
     y_ref, q_ref = oracle.epilogue(ref, S, relu=True, next_bits=3, inv_next=np.float32(1.0) / np.float32(0.4))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qs, d)
     epi = ebs.epilogue(relu=True, next_a_bits=3, next_a_scale=0.4)
-    for variant in range(-1, ebs.ebs_num_conv_variants()):
+    for variant in U.all_variants(d, 9):
         try:
             out = U.run_conv(qa, qs, d, epi, want_acc=True, want_y=True, next_bits=3, variant=variant, px=px, pw=pw)
         except ebs.EbsError as exc:                      # 16-channel tiles cannot produce packed words of wider layers
@@ -354,4 +365,4 @@ def test_pack_weights_fp32_to_paper_levels(ebs, U, oracle):
     d = ebs.conv_desc(c, co, k, k, 1, 1, 1, 1, wb, 2, 1.0 / L, 0.05, w_levels=1)
     out = torch.empty(ebs.ebs_packed_weight_bytes(d) // 4, dtype=torch.int32, device=U.dev())
     ebs.ebs_pack_weights(torch.from_numpy(w).to(U.dev()), ebs.EBS_F32, ebs.EBS_NCHW, d, out)
-    assert np.array_equal(U.as_u32(out).reshape(k, k, 1, co, wb), oracle.pack_weights(qs, wb))
+    assert np.array_equal(U.weight_planes(out, d), oracle.pack_weights(qs, wb))
