@@ -148,9 +148,10 @@ class Layer:
         ebs.ebs_conv2d_mixed(self.px, self.n, L.h_in, L.w_in, self.pw, self.d, self.epi, self.acc, None, self.pn)
         ebs.ebs_dequant(self.acc, self.pixels, L.c_out, self.S, None, None, True, self.y)
 
-    def run_conv_only(self, ebs):
+    def run_conv_only(self, ebs, variant=-1):
         L = self.spec.layer
-        ebs.ebs_conv2d_mixed(self.px, self.n, L.h_in, L.w_in, self.pw, self.d, self.epi, self.acc, None, self.pn)
+        ebs.ebs_conv2d_mixed(self.px, self.n, L.h_in, L.w_in, self.pw, self.d, self.epi, self.acc, None, self.pn,
+                             variant=variant)
 
     def run_host(self, ebs, ws, stream=None):
         L = self.spec.layer
@@ -376,6 +377,22 @@ def run_gpu(args):
         torch.cuda.synchronize()
         conv_ms[i] = e0.elapsed_time(e1) / 10.0
 
+    # the same 20 conv launches on the integer-pipe kernels only: the plane-pair double sum evaluated
+    # literally (AND + POPC + shift-add per plane pair), held against the POPC pipe's peak
+    literal = {}
+    if world == 1:
+        lit_graph = capture(lambda: [L.run_conv_only(ebs, -2) for L in layers])
+        lev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for e0, e1 in lev:
+            flush.zero_()
+            e0.record(stream)
+            lit_graph.replay()
+            e1.record(stream)
+        torch.cuda.synchronize()
+        lit_ms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in lev]))
+        literal = {"kernel": "conv_popc_kernel (variant -2: the library's choice among the integer-pipe kernels)",
+                   "conv_ms_per_step": lit_ms, "binary_tops": total_ops / (lit_ms * 1e-3) / 1e12}
+
     # the streaming kernels (rows a2 and a6) on a tensor far larger than L2: achieved GB/s of algorithmic bytes
     streaming = {}
     if world == 1:
@@ -517,6 +534,11 @@ def run_gpu(args):
                      "per_layer_note": "per-layer times are L2-warm (10 back-to-back launches in a graph); "
                                        "roof = max(2*MACs / int8 tensor peak, algorithmic bytes / HBM peak)",
                      "per_layer": per_layer},
+        "literal_bitplane_path": dict(literal, popc_pipe_peak_tops=popc_pipe_peak_tops(sm_max),
+                                      frac_of_popc_pipe=(literal["binary_tops"] / popc_pipe_peak_tops(sm_max)
+                                                         if literal else None),
+                                      note="every bit pair is one AND+POPC lane-op here, so binary ops are what this "
+                                           "pipe executes; the default path above retires Wb*Ab of them per int8 MAC"),
         "streaming_kernels": streaming,
         "network": network,
         "wall_s_timed_region": wall,

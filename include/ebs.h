@@ -184,11 +184,19 @@ int ebs_conv2d_mixed(const void *packed_x_dev, int n, int h, int w, const void *
 /*
  * The same call with the kernel variant forced (0 .. ebs_num_conv_variants()-1) instead of chosen by
  * the built-in heuristic (-1); the result is identical for every variant, only the speed differs.
- * Variants 0..9 are the integer-pipe kernels (AND + POPC), variants 10..18 the warp-level tensor-pipe
- * kernels (int8 mma.sync on bit planes expanded to bytes), variants 19..23 the tcgen05 kernels (same
- * product, 128 pixels x 16/32/64/128/256 channels per CTA, accumulator in tensor memory).
+ *   0..9    integer-pipe kernels: the plane-pair double sum of Eq. 13-14 evaluated literally
+ *           (AND + POPC + shift-add per plane pair);
+ *   10..18  warp-level tensor-pipe kernels (int8 mma.sync; the planes of a channel merged into
+ *           its byte in registers, one MMA per 32 channels of a tap);
+ *   19..23  tcgen05 kernels, any stride (same product, 128 pixels x 16/32/64/128/256 channels
+ *           per CTA, accumulator in tensor memory);
+ *   24..28  tcgen05 strip kernels for stride-1 layers and strided 1x1 layers (every input
+ *           pixel expanded once per CTA; weights read from the byte image).
+ * variant = -2 lets the library choose among the integer-pipe kernels only (the literal
+ * bit-plane evaluation), for comparison runs.
  * For tuning and for tests that must cover every kernel instantiation.  Returns
- * EBS_ERR_UNSUPPORTED if the variant cannot produce the requested packed output.
+ * EBS_ERR_UNSUPPORTED if the variant does not apply to the layer or cannot produce the requested
+ * packed output.
  */
 int ebs_num_conv_variants(void);
 int ebs_conv2d_mixed_variant(const void *packed_x_dev, int n, int h, int w, const void *packed_w_dev,

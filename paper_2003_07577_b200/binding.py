@@ -166,7 +166,7 @@ def ebs_pack_acts(x_dev: torch.Tensor, dtype: int, layout: int, n: int, c: int, 
 def ebs_conv2d_mixed(packed_x_dev, n, h, w, packed_w_dev, desc, epi=None, acc_out_dev=None, y_out_dev=None,
                      packed_next_dev=None, stream=None, variant: int = -1) -> None:
     e = None if epi is None else ctypes.byref(epi)
-    if variant < 0:
+    if variant == -1:
         rc = lib().ebs_conv2d_mixed(_ptr(packed_x_dev), n, h, w, _ptr(packed_w_dev), ctypes.byref(desc), e,
                                     _ptr(acc_out_dev), _ptr(y_out_dev), _ptr(packed_next_dev), _stream(stream))
     else:

@@ -208,7 +208,9 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
         if (packed_next) { p.next_bits = epi->next_a_bits; p.inv_next = 1.0f / epi->next_a_scale; }
     }
     const bool mma_ok = mma_path_supported(p, d);
-    if (variant < 0) {
+    if (variant == -2) {
+        variant = choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
+    } else if (variant < 0) {
         const int strip = mma_ok ? choose_strip_variant(p) : -1;
         const int umma = (mma_ok && strip < 0) ? choose_umma_variant(p, d) : -1;
         if (strip >= 0) variant = STRIP_BASE + strip;
