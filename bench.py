@@ -427,6 +427,15 @@ def run_gpu(args):
                                            vals * 4 + out_b),
             "dequant_gbs": gbs(lambda: ebs.ebs_dequant(ai, sn * sh * sh, sc, 0.01, None, None, True, yo), vals * 8),
         }
+        # search-stage forward (Eq. 6-7), five candidate bitwidths: 4 B in + 4 B out per value; the weight form
+        # reads the tensor once more for max|w|
+        cand_bits, cand_coeff = [1, 2, 3, 4, 5], [0.1, 0.15, 0.4, 0.25, 0.1]
+        scratch = torch.zeros(4, dtype=torch.int32, device=dev)
+        xo = torch.empty_like(xf)
+        streaming["search_act_forward_gbs"] = gbs(lambda: ebs.ebs_search_act_forward(xf, 6.0, cand_bits, cand_coeff, xo), vals * 8)
+        streaming["search_weight_forward_gbs"] = gbs(
+            lambda: ebs.ebs_search_weight_forward(xf, cand_bits, cand_coeff, xo, scratch), vals * 12)
+        del xo
         del xf, xu, pk, ai, yo
 
     # whole-network inference (the ResNet-20 of this workload wired with its shortcuts, pooling and

@@ -220,6 +220,35 @@ int ebs_dequant(const int32_t *acc_dev, size_t n_pixels, int c_out, float scale,
                 void *stream);
 
 /*
+ * Search-stage forward of the bitwidth search (Sec. 4.1; next-row kernels, not on the deployment
+ * path).  The full-precision meta tensor is quantized at every candidate bitwidth and the results
+ * are blended in one pass:
+ *   weights (Eq. 1a, Eq. 6):  u = tanh(w) / (2 max|tanh(w)|) + 1/2,
+ *                             w_hat = sum_i coeff[i] * (2 quantize_b[i](u) - 1)
+ *   activations (Eq. 1b, Eq. 7):  u = clip(x, 0, alpha) * fl32(1/alpha),
+ *                             x_hat = alpha * sum_j coeff[j] * quantize_b[j](u)
+ *   quantize_b(u) = fl32(1/(2^b - 1)) * floor((2^b - 1) u + 0.5)   (Eq. 1c, round half up)
+ * `bits` (each 1..16) and `coeff` are HOST arrays of n_cand <= EBS_MAX_CANDIDATES entries; coeff is
+ * the softmax of the strengths (deterministic search) or the Gumbel-softmax sample (stochastic
+ * search, Eq. 8), computed by the caller.  Every fp32 operation is rounded on its own, candidates
+ * are accumulated in array order.  src/dst are device tensors of n floats (16-byte aligned; dst
+ * may alias src); scratch_dev is 16 bytes of device memory the weight call uses for max|w|.
+ */
+#define EBS_MAX_CANDIDATES 8
+int ebs_search_weight_forward(const float *w_dev, size_t n, const int *bits, const float *coeff, int n_cand,
+                              float *w_hat_dev, void *scratch_dev, void *stream);
+int ebs_search_act_forward(const float *x_dev, size_t n, float alpha, const int *bits, const float *coeff,
+                           int n_cand, float *x_hat_dev, void *stream);
+
+/*
+ * Expected operation count of a layer during the search (Eq. 11):
+ * FLOP(sum_i coeff_w[i] bits_w[i], sum_j coeff_x[j] bits_x[j]) with FLOP(M, K) = macs * M * K
+ * (Sec. 4.3: s n c_o M K AND operations).  Host arithmetic in double; negative on bad arguments.
+ */
+double ebs_expected_flops(double macs, const int *bits_w, const float *coeff_w, int n_w, const int *bits_x,
+                          const float *coeff_x, int n_x);
+
+/*
  * Global average pooling between the last residual block and the classifier of the ResNets the
  * paper evaluates (Sec. 5); not part of the binary decomposition itself.  y_dev is fp32 NHWC
  * [n][hw][c]; out_dev receives [n][c]: the pixels are added in order 0 .. hw-1 in fp32 and the

@@ -196,6 +196,64 @@ def global_avgpool(y) -> np.ndarray:
     return (acc * (np.float32(1.0) / np.float32(h * w))).astype(np.float32)
 
 
+# ---------------------------------------------------------------- search stage (Sec. 4.1), plain numpy
+
+def softmax_strengths(r) -> np.ndarray:
+    """Coefficients of the deterministic search: softmax of the strengths (Eq. 5-6), evaluated in
+    float64 and rounded to the fp32 values both sides are given."""
+    r = np.asarray(r, dtype=np.float64)
+    e = np.exp(r - r.max())
+    return (e / e.sum()).astype(np.float32)
+
+
+def quantize_unit(u, bits: int) -> np.ndarray:
+    """quantize_b of Eq. 1c on fp32 values in [0, 1]: (1 / (2^b - 1)) * floor((2^b - 1) u + 0.5), the
+    reciprocal rounded to fp32 once, every operation rounded to fp32 on its own (round half up)."""
+    u = np.asarray(u, dtype=np.float32)
+    L = np.float32((1 << bits) - 1)
+    code = np.floor((u * L).astype(np.float32) + np.float32(0.5)).astype(np.float32)
+    return ((np.float32(1.0) / L) * code).astype(np.float32)
+
+
+def search_act_forward(x, alpha, bits, coeff) -> np.ndarray:
+    """Eq. 1b per candidate bitwidth, blended as in Eq. 7:
+    x_hat = alpha * sum_j coeff_j * quantize_{b_j}(clip(x, 0, alpha) * (1/alpha)), fp32, the reciprocal
+    rounded once, candidates in order."""
+    x = np.asarray(x, dtype=np.float32)
+    a = np.float32(alpha)
+    u = (np.minimum(np.maximum(x, np.float32(0.0)), a) * (np.float32(1.0) / a)).astype(np.float32)
+    acc = np.zeros_like(u)
+    for b, c in zip(bits, coeff):
+        acc = (acc + (np.float32(c) * quantize_unit(u, int(b))).astype(np.float32)).astype(np.float32)
+    return (a * acc).astype(np.float32)
+
+
+def search_weight_forward(w, bits, coeff):
+    """Eq. 1a per candidate bitwidth, blended as in Eq. 6, in float64:
+    u = tanh(w) / (2 max|tanh(w)|) + 1/2;  w_hat = sum_i coeff_i * (2 quantize_{b_i}(u) - 1).
+    Also returns, per element, the smallest distance of (2^b - 1) u + 0.5 to an integer over the
+    candidates: where it is tiny, a float32 evaluation may legitimately round to the other level."""
+    w = np.asarray(w, dtype=np.float64)
+    t = np.tanh(w)
+    u = t / (2.0 * np.abs(t).max()) + 0.5
+    out = np.zeros_like(u)
+    margin = np.full(u.shape, 1.0)
+    for b, c in zip(bits, coeff):
+        L = float((1 << int(b)) - 1)
+        v = L * u + 0.5
+        code = np.clip(np.floor(v), 0.0, L)
+        margin = np.minimum(margin, np.abs(v - np.round(v)))
+        out += float(c) * (2.0 * code / L - 1.0)
+    return out, margin
+
+
+def expected_flops(macs, bits_w, coeff_w, bits_x, coeff_x) -> float:
+    """Eq. 11: FLOP(sum_i f(r)_i b_i, sum_j f(s)_j b_j) with FLOP(M, K) = macs * M * K (Sec. 4.3)."""
+    m = sum(float(c) * int(b) for b, c in zip(bits_w, coeff_w))
+    k = sum(float(c) * int(b) for b, c in zip(bits_x, coeff_x))
+    return float(macs) * m * k
+
+
 def pack_acts(qa, a_bits: int) -> np.ndarray:
     """uint32 [N, H, W, ceil(C/32), Ab] bit-plane words, built bit by bit."""
     qa = _i32(qa)

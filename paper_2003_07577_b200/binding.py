@@ -25,7 +25,8 @@ EXPORTS = [
     "ebs_version", "ebs_status_string", "ebs_last_cuda_error", "ebs_conv_out_shape", "ebs_packed_weight_bytes",
     "ebs_packed_act_bytes", "ebs_pack_weights", "ebs_pack_acts", "ebs_conv2d_mixed", "ebs_num_conv_variants",
     "ebs_conv2d_mixed_variant", "ebs_dequant", "ebs_host_workspace_bytes", "ebs_conv2d_mixed_host",
-    "ebs_probe_pipe", "ebs_device_wait_timeouts", "ebs_global_avgpool", "ebs_packed_weight_plane_bytes", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
+    "ebs_probe_pipe", "ebs_device_wait_timeouts", "ebs_global_avgpool", "ebs_packed_weight_plane_bytes", "ebs_search_weight_forward",
+    "ebs_search_act_forward", "ebs_expected_flops", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
 ]
 
 
@@ -86,6 +87,11 @@ def lib() -> ctypes.CDLL:
         L.ebs_conv2d_mixed_host.argtypes = [p, i, i, i, i, i, p, D, E, p, z, p, p, p, p]
         L.ebs_probe_pipe.argtypes = [i, i, ctypes.POINTER(ctypes.c_double)]
         L.ebs_global_avgpool.argtypes = [p, i, i, i, p, p]
+        ip, fp = ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_float)
+        L.ebs_search_weight_forward.argtypes = [p, z, ip, fp, i, p, p, p]
+        L.ebs_search_act_forward.argtypes = [p, z, ctypes.c_float, ip, fp, i, p, p]
+        L.ebs_expected_flops.argtypes = [ctypes.c_double, ip, fp, i, ip, fp, i]
+        L.ebs_expected_flops.restype = ctypes.c_double
         L.ebs_noalloc_scratch_bytes.restype = z
         L.ebs_device_wait_timeouts.restype = ctypes.c_longlong
         L.ebs_conv2d_mixed_host_noalloc.argtypes = [p, i, i, i, i, i, p, D, E, p, p, p, p]
@@ -207,6 +213,29 @@ def ebs_probe_pipe(kind: int, iters: int = 2000) -> float:
 
 def ebs_global_avgpool(y_dev, n: int, hw: int, c: int, out_dev, stream=None) -> None:
     _check(lib().ebs_global_avgpool(_ptr(y_dev), n, hw, c, _ptr(out_dev), _stream(stream)), "ebs_global_avgpool")
+
+
+def _cand(bits, coeff):
+    n = len(bits)
+    return (ctypes.c_int * n)(*[int(b) for b in bits]), (ctypes.c_float * n)(*[float(c) for c in coeff]), n
+
+
+def ebs_search_weight_forward(w_dev, bits, coeff, w_hat_dev, scratch_dev, stream=None) -> None:
+    b, c, n = _cand(bits, coeff)
+    _check(lib().ebs_search_weight_forward(_ptr(w_dev), w_dev.numel(), b, c, n, _ptr(w_hat_dev), _ptr(scratch_dev),
+                                           _stream(stream)), "ebs_search_weight_forward")
+
+
+def ebs_search_act_forward(x_dev, alpha: float, bits, coeff, x_hat_dev, stream=None) -> None:
+    b, c, n = _cand(bits, coeff)
+    _check(lib().ebs_search_act_forward(_ptr(x_dev), x_dev.numel(), alpha, b, c, n, _ptr(x_hat_dev), _stream(stream)),
+           "ebs_search_act_forward")
+
+
+def ebs_expected_flops(macs: float, bits_w, coeff_w, bits_x, coeff_x) -> float:
+    bw, cw, nw = _cand(bits_w, coeff_w)
+    bx, cx, nx = _cand(bits_x, coeff_x)
+    return lib().ebs_expected_flops(float(macs), bw, cw, nw, bx, cx, nx)
 
 
 def ebs_device_wait_timeouts() -> int:

@@ -337,6 +337,29 @@ int ebs_dequant(const int32_t* acc_dev, size_t n_pixels, int c_out, float scale,
                           static_cast<cudaStream_t>(stream));
 }
 
+int ebs_search_weight_forward(const float* w_dev, size_t n, const int* bits, const float* coeff, int n_cand,
+                              float* w_hat_dev, void* scratch_dev, void* stream) {
+    if (!w_dev || !w_hat_dev || !scratch_dev || n == 0) return EBS_ERR_INVALID_ARG;
+    if (!aligned16(w_dev) || !aligned16(w_hat_dev) || !aligned16(scratch_dev)) return EBS_ERR_INVALID_ARG;
+    return launch_search_weights(w_dev, n, bits, coeff, n_cand, w_hat_dev, scratch_dev, static_cast<cudaStream_t>(stream));
+}
+
+int ebs_search_act_forward(const float* x_dev, size_t n, float alpha, const int* bits, const float* coeff, int n_cand,
+                           float* x_hat_dev, void* stream) {
+    if (!x_dev || !x_hat_dev || n == 0 || !(alpha > 0.0f)) return EBS_ERR_INVALID_ARG;
+    if (!aligned16(x_dev) || !aligned16(x_hat_dev)) return EBS_ERR_INVALID_ARG;
+    return launch_search_acts(x_dev, n, alpha, bits, coeff, n_cand, x_hat_dev, static_cast<cudaStream_t>(stream));
+}
+
+double ebs_expected_flops(double macs, const int* bits_w, const float* coeff_w, int n_w, const int* bits_x,
+                          const float* coeff_x, int n_x) {
+    if (!bits_w || !coeff_w || !bits_x || !coeff_x || n_w < 1 || n_x < 1 || !(macs >= 0.0)) return -1.0;
+    double m = 0.0, k = 0.0;
+    for (int i = 0; i < n_w; ++i) m += (double)coeff_w[i] * bits_w[i];
+    for (int j = 0; j < n_x; ++j) k += (double)coeff_x[j] * bits_x[j];
+    return macs * m * k;
+}
+
 int ebs_global_avgpool(const float* y_dev, int n, int hw, int c, float* out_dev, void* stream) {
     if (!y_dev || !out_dev || n <= 0 || hw <= 0 || c <= 0) return EBS_ERR_INVALID_ARG;
     if ((long long)n * c >= (1LL << 31)) return EBS_ERR_OVERFLOW;

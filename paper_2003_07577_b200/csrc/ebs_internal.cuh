@@ -89,6 +89,10 @@ int launch_dequant(const int32_t* acc, size_t n_pixels, int c_out, float scale, 
 
 size_t packed_weight_plane_bytes(const ebs_conv_desc& d);   // bit-plane words, rounded up to 256 bytes
 size_t packed_weight_image_bytes(const ebs_conv_desc& d);   // byte image that follows them
+int launch_search_weights(const float* w, size_t n, const int* bits, const float* coeff, int n_cand, float* w_hat,
+                          void* scratch, cudaStream_t st);
+int launch_search_acts(const float* x, size_t n, float alpha, const int* bits, const float* coeff, int n_cand,
+                       float* x_hat, cudaStream_t st);
 int launch_avgpool(const float* y, int n, int hw, int c, float* out, cudaStream_t st);
 
 // Records a CUDA error for ebs_last_cuda_error() and returns EBS_ERR_CUDA (or EBS_OK).

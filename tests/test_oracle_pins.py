@@ -401,3 +401,68 @@ def test_dequant_codes_is_one_fp32_product(oracle):
     got = oracle.dequant_codes(q, step)
     assert got.dtype == np.float32
     assert np.array_equal(got, np.array([np.float32(float(step) * int(v)) for v in q], np.float32))
+
+
+# ------------------------------------------------------------------ search stage (Eq. 1a-c, 6, 7, 11)
+
+def test_quantize_unit_levels_half_up_and_idempotent(oracle):
+    for b in (1, 2, 3, 5, 8):
+        L = (1 << b) - 1
+        grid = (np.arange(L + 1, dtype=np.float32) * (np.float32(1.0) / np.float32(L))).astype(np.float32)
+        assert np.array_equal(oracle.quantize_unit(grid, b), grid)                   # levels are fixed points
+        u = np.linspace(0, 1, 4001, dtype=np.float32)
+        q = oracle.quantize_unit(u, b)
+        assert np.all(np.diff(q) >= 0) and set(np.unique(q)) <= set(grid)             # monotone, on the grid
+        assert np.all(np.abs(q.astype(np.float64) - u) <= 0.5 / L + 1e-6)              # nearest level
+    assert oracle.quantize_unit(np.float32(0.5), 1) == 1.0                            # the tie goes up
+    assert oracle.quantize_unit(np.float32(0.25), 2) == np.float32(1.0) / np.float32(3.0)   # 0.75 + 0.5 -> floor 1
+    assert oracle.quantize_unit(np.float32(1.0), 3) == np.float32(7.0) * (np.float32(1.0) / np.float32(7.0))
+
+
+def test_softmax_strengths_closed_forms(oracle):
+    assert np.allclose(oracle.softmax_strengths([0, 0]), [0.5, 0.5])                  # the text's two-candidate example
+    p = oracle.softmax_strengths([-1, 1])
+    assert np.allclose(p, [1 / (1 + np.e ** 2), np.e ** 2 / (1 + np.e ** 2)], atol=1e-7) and p[1] > 0.88
+    assert np.allclose(oracle.softmax_strengths(np.zeros(5)), 0.2) and oracle.softmax_strengths([3, 3, 3]).dtype == np.float32
+
+
+def test_search_act_forward_special_cases(oracle):
+    rng = np.random.default_rng(3)
+    x = rng.uniform(-1, 8, 5000).astype(np.float32)
+    alpha = 6.0
+    one = oracle.search_act_forward(x, alpha, [3], [1.0])                             # one candidate: plain Eq. 1b
+    ref = alpha * np.round(np.clip(x.astype(np.float64), 0, alpha) / alpha * 7 + 1e-12) / 7
+    assert np.allclose(one, ref, atol=1e-5) and one.min() == 0 and one.max() == np.float32(alpha)
+    assert set(np.unique(np.round(one / alpha * 7).astype(int))) == set(range(8))
+    two = oracle.search_act_forward(x, alpha, [2, 3], [0.5, 0.5])                     # equal blend of two bitwidths
+    a2, a3 = oracle.search_act_forward(x, alpha, [2], [1.0]), oracle.search_act_forward(x, alpha, [3], [1.0])
+    assert np.allclose(two, 0.5 * a2.astype(np.float64) + 0.5 * a3, atol=1e-6)
+    sharp = oracle.search_act_forward(x, alpha, [2, 3], [0.0, 1.0])                   # softmax -> max selects one branch
+    assert np.array_equal(sharp, a3)
+
+
+def test_search_weight_forward_special_cases(oracle):
+    rng = np.random.default_rng(4)
+    w = rng.standard_normal(4000) * 0.7
+    for b in (1, 2, 4):
+        L = (1 << b) - 1
+        out, _ = oracle.search_weight_forward(w, [b], [1.0])
+        lv = np.unique(np.round((out + 1) * L / 2).astype(int))
+        assert np.allclose((out + 1) * L / 2, np.round((out + 1) * L / 2), atol=1e-9)   # on the level grid of [-1, 1]
+        assert lv.min() == 0 and lv.max() == L and np.abs(out).max() == 1.0            # the largest weight maps to +-1
+    out1, _ = oracle.search_weight_forward(w, [1], [1.0])
+    assert np.array_equal(out1, np.where(w >= 0, 1.0, -1.0))                          # one bit: the sign
+    out8, _ = oracle.search_weight_forward(w, [8], [1.0])
+    assert np.abs(out8 - np.tanh(w) / np.abs(np.tanh(w)).max()).max() <= 1.0 / 255 + 1e-12   # fine grid: the normalized tanh
+    blend, margin = oracle.search_weight_forward(w, [2, 3], [0.5, 0.5])
+    o2, _ = oracle.search_weight_forward(w, [2], [1.0])
+    o3, _ = oracle.search_weight_forward(w, [3], [1.0])
+    assert np.allclose(blend, 0.5 * o2 + 0.5 * o3) and np.unique(np.round(blend, 9)).size > 4 and (margin >= 0).all()
+
+
+def test_expected_flops_eq11(oracle):
+    bits = [1, 2, 3, 4, 5]
+    uniform = oracle.softmax_strengths(np.zeros(5))
+    assert abs(oracle.expected_flops(1e6, bits, uniform, bits, uniform) - 9e6) < 1.0   # mean bitwidth 3 on both sides
+    onehot = [0, 0, 1, 0, 0]
+    assert oracle.expected_flops(40.81e6, bits, onehot, bits, [0, 1, 0, 0, 0]) == 40.81e6 * 3 * 2
