@@ -109,6 +109,14 @@ __device__ __forceinline__ uint8_t* sw32_chunk(uint8_t* tile, int row, int c) {
     return tile + row * 32 + ((c ^ ((row >> 2) & 1)) << 4);
 }
 
+// Four integers -> four bytes a | b << 8 | c << 16 | d << 24, each saturated to 0 .. 255.
+__device__ __forceinline__ uint32_t pack_sat_u8x4(int a, int b, int c, int d) {
+    uint32_t hi, out;
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;\n" : "=r"(hi) : "r"(d), "r"(c), "r"(0));
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;\n" : "=r"(out) : "r"(b), "r"(a), "r"(hi));
+    return out;
+}
+
 // Epilogue straight out of tensor memory.  Warp w reads TMEM lanes 32 * (w % 4) .. + 31: thread `lane`
 // of it owns the accumulators of one pixel row (global output pixel gp; pvalid false = row without an
 // output).  Warps w and w + 4 split the channels when the tile is wide enough.  The thread stores the
@@ -137,7 +145,7 @@ __device__ __forceinline__ void umma_epilogue(const ConvParams& p, uint32_t tmem
             for (int c0 = cbeg; c0 < cbeg + COLS_PER_WARP; c0 += 32) {
                 uint32_t planes[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
 #pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
+                for (int hf = 1; hf >= 0; --hf) {                    // upper 16 channels first: planes grow by shifting left
                     uint32_t v[16];
                     tmem_ld16(trow + (uint32_t)(c0 + 16 * hf), v);   // whole warp, also for rows past the end
                     if (w_levels) {
@@ -165,22 +173,23 @@ __device__ __forceinline__ void umma_epilogue(const ConvParams& p, uint32_t tmem
                                     make_float4(y[4 * gq], y[4 * gq + 1], y[4 * gq + 2], y[4 * gq + 3]);
                         }
                         if (want_q) {
-                            uint32_t c4[4];
 #pragma unroll
-                            for (int gq = 0; gq < 4; ++gq) {
-                                c4[gq] = 0u;
+                            for (int gq = 3; gq >= 0; --gq) {
+                                // codes of four channels as bytes: floor(y / step + 0.5), at most qmax; the pack
+                                // instruction saturates at 0 (negative values, and NaN converts to 0)
+                                int q[4];
 #pragma unroll
                                 for (int e = 0; e < 4; ++e)
-                                    c4[gq] |= (uint32_t)quantize_act_code(y[4 * gq + e], inv_next, qmax) << (8 * e);
-                            }
+                                    q[e] = min(__float2int_rd(__fadd_rn(__fmul_rn(y[4 * gq + e], inv_next), 0.5f)), qmax);
+                                const uint32_t c4 = pack_sat_u8x4(q[0], q[1], q[2], q[3]);
+                                // plane j of the four codes -> the top nibble of a product, shifted into the plane word
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                if (j >= nb) break;
-                                uint32_t bits16 = 0u;                 // plane j of these 16 channels
-#pragma unroll
-                                for (int gq = 0; gq < 4; ++gq)
-                                    bits16 |= ((((c4[gq] >> j) & 0x01010101u) * 0x01020408u) >> 24) << (4 * gq);
-                                planes[j] |= bits16 << (16 * hf);
+                                for (int j = 0; j < 8; ++j) {
+                                    if (j >= nb) break;
+                                    const uint32_t bits = j <= 4 ? (c4 & (0x01010101u << j)) * (0x10204080u >> j)
+                                                                 : ((c4 >> j) & 0x01010101u) * 0x10204080u;
+                                    planes[j] = __funnelshift_l(bits, planes[j], 4);
+                                }
                             }
                         }
                     }
