@@ -191,7 +191,10 @@ int ebs_conv2d_mixed(const void *packed_x_dev, int n, int h, int w, const void *
  *   19..23  tcgen05 kernels, any stride (same product, 128 pixels x 16/32/64/128/256 channels
  *           per CTA, accumulator in tensor memory);
  *   24..28  tcgen05 strip kernels for stride-1 layers and strided 1x1 layers (every input
- *           pixel expanded once per CTA; weights read from the byte image).
+ *           pixel expanded once per CTA; weights read from the byte image);
+ *   29..33  the same as persistent CTAs that keep the weight bytes of their channel tile in
+ *           shared memory and overlap expansion, MMAs and epilogue of consecutive pixel tiles
+ *           (layers whose weight tiles fit in 150 KB, w_levels = 0).
  * variant = -2 lets the library choose among the integer-pipe kernels only (the literal
  * bit-plane evaluation), for comparison runs.
  * For tuning and for tests that must cover every kernel instantiation.  Returns

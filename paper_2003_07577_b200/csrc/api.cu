@@ -59,7 +59,7 @@ const ConvVariant* conv_umma_variant(int w_bits, int a_bits, int variant) {
 unsigned long long conv_umma_timeouts() {
     return conv_umma_timeouts_w1() + conv_umma_timeouts_w2() + conv_umma_timeouts_w3() + conv_umma_timeouts_w4() +
            conv_umma_timeouts_w5() + conv_umma_timeouts_w6() + conv_umma_timeouts_w7() + conv_umma_timeouts_w8() +
-           conv_umma_strip_timeouts();
+           conv_umma_strip_timeouts() + conv_umma_resident_timeouts();
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -181,7 +181,8 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
         if (epi->res_packed_dev && (epi->res_bits < 1 || epi->res_bits > 8)) return EBS_ERR_INVALID_ARG;
     }
     constexpr int STRIP_BASE = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS;
-    if (variant >= STRIP_BASE + NUM_CONV_STRIP_VARIANTS) return EBS_ERR_INVALID_ARG;
+    constexpr int RES_BASE = STRIP_BASE + NUM_CONV_STRIP_VARIANTS;
+    if (variant >= RES_BASE + NUM_CONV_RESIDENT_VARIANTS) return EBS_ERR_INVALID_ARG;
 
     ConvParams p;
     memset(&p, 0, sizeof(p));
@@ -213,14 +214,21 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
     } else if (variant < 0) {
         const int strip = mma_ok ? choose_strip_variant(p) : -1;
         const int umma = (mma_ok && strip < 0) ? choose_umma_variant(p, d) : -1;
-        if (strip >= 0) variant = STRIP_BASE + strip;
+        // deep reductions whose weight tiles fit in shared memory: the persistent form of the same tile
+        if (strip >= 0 && p.CW * d->kh * d->kw >= 8 && conv_umma_resident_applies(p, strip)) variant = RES_BASE + strip;
+        else if (strip >= 0) variant = STRIP_BASE + strip;
         else if (umma >= 0) variant = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + umma;
         else variant = mma_ok ? NUM_CONV_VARIANTS + choose_mma_variant(d->w_bits, d->a_bits, p.P, p.Co, sm_count())
                               : choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
     }
     if (variant >= NUM_CONV_VARIANTS && !mma_ok) return EBS_ERR_UNSUPPORTED;
-    if (variant >= STRIP_BASE && !conv_umma_strip_applies(p, variant - STRIP_BASE)) return EBS_ERR_UNSUPPORTED;
+    if (variant >= RES_BASE) {
+        if (!conv_umma_resident_applies(p, variant - RES_BASE)) return EBS_ERR_UNSUPPORTED;
+    } else if (variant >= STRIP_BASE && !conv_umma_strip_applies(p, variant - STRIP_BASE)) {
+        return EBS_ERR_UNSUPPORTED;
+    }
     const ConvVariant* v =
+        variant >= RES_BASE ? conv_umma_resident_variant(d->a_bits, variant - RES_BASE) :
         variant >= STRIP_BASE ? conv_umma_strip_variant(d->a_bits, variant - STRIP_BASE) :
         variant >= NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS
             ? conv_umma_variant(d->w_bits, d->a_bits, variant - NUM_CONV_VARIANTS - NUM_CONV_MMA_VARIANTS)
@@ -316,7 +324,8 @@ int ebs_conv2d_mixed(const void* packed_x_dev, int n, int h, int w, const void* 
 }
 
 int ebs_num_conv_variants(void) {
-    return NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS + NUM_CONV_STRIP_VARIANTS;
+    return NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS + NUM_CONV_STRIP_VARIANTS +
+           NUM_CONV_RESIDENT_VARIANTS;
 }
 
 long long ebs_device_wait_timeouts(void) { return (long long)conv_umma_timeouts(); }

@@ -109,6 +109,22 @@ __device__ __forceinline__ uint8_t* sw32_chunk(uint8_t* tile, int row, int c) {
     return tile + row * 32 + ((c ^ ((row >> 2) & 1)) << 4);
 }
 
+// The two halves of a tensor-memory load: issue, and later wait.  The wait names the destination registers
+// as read-write operands so that no use of them is scheduled before it.
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld16_wait(uint32_t (&v)[16]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;\n"
+                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                   "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+                 :: "memory");
+}
+
 // Four integers -> four bytes a | b << 8 | c << 16 | d << 24, each saturated to 0 .. 255.
 __device__ __forceinline__ uint32_t pack_sat_u8x4(int a, int b, int c, int d) {
     uint32_t hi, out;
@@ -141,59 +157,67 @@ __device__ __forceinline__ void umma_epilogue(const ConvParams& p, uint32_t tmem
             const int nb = want_q ? p.next_bits : 0;
             const float S = p.S, inv_next = p.inv_next;
             const bool relu = p.relu != 0, w_levels = p.w_levels != 0;
-#pragma unroll 1
-            for (int c0 = cbeg; c0 < cbeg + COLS_PER_WARP; c0 += 32) {
-                uint32_t planes[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+            // 16 channels of this thread's pixel: store, requantize, shift their plane bits into `planes`
+            auto process16 = [&](uint32_t (&v)[16], int cbase, uint32_t (&planes)[8]) {
+                if (w_levels) {
 #pragma unroll
-                for (int hf = 1; hf >= 0; --hf) {                    // upper 16 channels first: planes grow by shifting left
-                    uint32_t v[16];
-                    tmem_ld16(trow + (uint32_t)(c0 + 16 * hf), v);   // whole warp, also for rows past the end
-                    if (w_levels) {
+                    for (int e = 0; e < 16; ++e) v[e] = (uint32_t)(2 * (int)v[e] + wsum_row);
+                }
+                const size_t o = (size_t)gp * p.Co + co0 + cbase;
+                if (p.acc && pvalid) {
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) v[e] = (uint32_t)(2 * (int)v[e] + wsum_row);
+                    for (int gq = 0; gq < 4; ++gq)
+                        *reinterpret_cast<int4*>(p.acc + o + 4 * gq) =
+                            make_int4((int)v[4 * gq], (int)v[4 * gq + 1], (int)v[4 * gq + 2], (int)v[4 * gq + 3]);
+                }
+                if (want_y || want_q) {
+                    float y[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        y[e] = __fmul_rn((float)(int)v[e], S);
+                        if (relu) y[e] = y[e] > 0.0f ? y[e] : 0.0f;
                     }
-                    const size_t o = (size_t)gp * p.Co + co0 + c0 + 16 * hf;
-                    if (p.acc && pvalid) {
+                    if (want_y && pvalid) {
 #pragma unroll
                         for (int gq = 0; gq < 4; ++gq)
-                            *reinterpret_cast<int4*>(p.acc + o + 4 * gq) =
-                                make_int4((int)v[4 * gq], (int)v[4 * gq + 1], (int)v[4 * gq + 2], (int)v[4 * gq + 3]);
+                            *reinterpret_cast<float4*>(p.y + o + 4 * gq) =
+                                make_float4(y[4 * gq], y[4 * gq + 1], y[4 * gq + 2], y[4 * gq + 3]);
                     }
-                    if (want_y || want_q) {
-                        float y[16];
+                    if (want_q) {
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            y[e] = __fmul_rn((float)(int)v[e], S);
-                            if (relu) y[e] = y[e] > 0.0f ? y[e] : 0.0f;
-                        }
-                        if (want_y && pvalid) {
+                        for (int gq = 3; gq >= 0; --gq) {
+                            // codes of four channels as bytes: floor(y / step + 0.5), at most qmax; the pack
+                            // instruction saturates at 0 (negative values, and NaN converts to 0)
+                            int q[4];
 #pragma unroll
-                            for (int gq = 0; gq < 4; ++gq)
-                                *reinterpret_cast<float4*>(p.y + o + 4 * gq) =
-                                    make_float4(y[4 * gq], y[4 * gq + 1], y[4 * gq + 2], y[4 * gq + 3]);
-                        }
-                        if (want_q) {
+                            for (int e = 0; e < 4; ++e)
+                                q[e] = min(__float2int_rd(__fadd_rn(__fmul_rn(y[4 * gq + e], inv_next), 0.5f)), qmax);
+                            const uint32_t c4 = pack_sat_u8x4(q[0], q[1], q[2], q[3]);
+                            // plane j of the four codes -> the top nibble of a product, shifted into the plane word
 #pragma unroll
-                            for (int gq = 3; gq >= 0; --gq) {
-                                // codes of four channels as bytes: floor(y / step + 0.5), at most qmax; the pack
-                                // instruction saturates at 0 (negative values, and NaN converts to 0)
-                                int q[4];
-#pragma unroll
-                                for (int e = 0; e < 4; ++e)
-                                    q[e] = min(__float2int_rd(__fadd_rn(__fmul_rn(y[4 * gq + e], inv_next), 0.5f)), qmax);
-                                const uint32_t c4 = pack_sat_u8x4(q[0], q[1], q[2], q[3]);
-                                // plane j of the four codes -> the top nibble of a product, shifted into the plane word
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) {
-                                    if (j >= nb) break;
-                                    const uint32_t bits = j <= 4 ? (c4 & (0x01010101u << j)) * (0x10204080u >> j)
-                                                                 : ((c4 >> j) & 0x01010101u) * 0x10204080u;
-                                    planes[j] = __funnelshift_l(bits, planes[j], 4);
-                                }
+                            for (int j = 0; j < 8; ++j) {
+                                if (j >= nb) break;
+                                const uint32_t bits = j <= 4 ? (c4 & (0x01010101u << j)) * (0x10204080u >> j)
+                                                             : ((c4 >> j) & 0x01010101u) * 0x10204080u;
+                                planes[j] = __funnelshift_l(bits, planes[j], 4);
                             }
                         }
                     }
                 }
+            };
+            // the load of the next 16 channels is in flight while the current ones are processed; the upper
+            // half of a 32-channel word comes first because the plane words grow by shifting left
+            uint32_t va[16], vb[16];
+            tmem_ld16_issue(trow + (uint32_t)(cbeg + 16), va);     // whole warp, also for rows past the end
+#pragma unroll 1
+            for (int c0 = cbeg; c0 < cbeg + COLS_PER_WARP; c0 += 32) {
+                uint32_t planes[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+                tmem_ld16_wait(va);
+                tmem_ld16_issue(trow + (uint32_t)c0, vb);
+                process16(va, c0 + 16, planes);
+                tmem_ld16_wait(vb);
+                if (c0 + 32 < cbeg + COLS_PER_WARP) tmem_ld16_issue(trow + (uint32_t)(c0 + 48), va);
+                process16(vb, c0, planes);
                 if (want_q && pvalid) {
                     uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + ((co0 + c0) >> 5)) * nb;
                     if (nb == 4) {

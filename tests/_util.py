@@ -96,12 +96,13 @@ def run_conv(qa, qw, d, epi=None, want_acc=True, want_y=False, next_bits=0, vari
     return out
 
 
-N_STRIP = 5     # the last variants are the stride-1 strip kernels
+N_STRIP = 5       # variants n-10 .. n-6: the strip kernels
+N_RESIDENT = 5    # variants n-5 .. n-1: the persistent weight-resident strip kernels
 
 
 def strip_variant_applies(d, w, tile_n):
-    """Host-side rule of the strip kernel: stride 1 (or a 1x1 layer without padding), a strip of at most 512 pixels, and two
-    stages of (strip + kh*kw weight tiles) within 200 KB of shared memory."""
+    """Host-side rule of the strip kernel: stride 1 (or a 1x1 layer without padding), a strip
+    of at most 512 pixels, and two stages of (strip + kh*kw weight tiles) within 200 KB of shared memory."""
     pointwise = d.kh == 1 and d.kw == 1 and d.pad_h == 0 and d.pad_w == 0    # 1x1 without padding: any stride
     if (d.stride_h != 1 or d.stride_w != 1) and not pointwise:
         return False
@@ -110,11 +111,21 @@ def strip_variant_applies(d, w, tile_n):
     return strip <= 512 and 2 * (pad * 32 + d.kh * d.kw * tile_n * 32) + 1024 + pad * 4 <= 200 * 1024
 
 
+def resident_variant_applies(d, w, tile_n):
+    """Host-side rule of the persistent kernel: the strip rule, no window-sum term, and all weight tiles
+    of a channel tile (ceil(c_in/32) * kh*kw * tile_n * 32 bytes) within 150 KB."""
+    cw = (d.c_in + 31) // 32
+    return (strip_variant_applies(d, w, tile_n) and not d.w_levels
+            and cw * d.kh * d.kw * tile_n * 32 <= 150 * 1024)
+
+
 def all_variants(d, w=16):
     """Every kernel variant that applies to descriptor d on images of width w (-1 = the library's own choice)."""
     n = ebs.ebs_num_conv_variants()
-    strip = [n - N_STRIP + i for i in range(N_STRIP) if strip_variant_applies(d, w, 16 << i)]
-    return list(range(-1, n - N_STRIP)) + strip
+    base = n - N_STRIP - N_RESIDENT
+    strip = [base + i for i in range(N_STRIP) if strip_variant_applies(d, w, 16 << i)]
+    resident = [base + N_STRIP + i for i in range(N_RESIDENT) if resident_variant_applies(d, w, 16 << i)]
+    return list(range(-1, base)) + strip + resident
 
 
 def rand_codes(rng, shape, bits, signed):

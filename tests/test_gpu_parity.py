@@ -99,7 +99,7 @@ def test_conv_all_bitwidth_pairs(ebs, U, oracle, wb, ab):
     d = U.desc_for(40, 21, 3, 1, 1, wb, ab)
     ref = oracle.conv2d_codes(qa, qw, (1, 1), (1, 1))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
-    for variant in (-1, 0, 4, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28):
+    for variant in (-1, 0, 4, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28, 29, 30, 31, 32, 33):
         got = U.run_conv(qa, qw, d, variant=variant, px=px, pw=pw)["acc"]
         assert np.array_equal(got, ref), f"variant {variant}"
 
@@ -131,7 +131,36 @@ def test_strip_kernel_refuses_strided_layers(ebs, U):
     d = U.desc_for(32, 32, 3, 2, 1, 2, 2)
     qa, qw = np.zeros((1, 32, 8, 8), np.int32), np.zeros((32, 32, 3, 3), np.int32)
     with pytest.raises(RuntimeError):
+        U.run_conv(qa, qw, d, variant=ebs.ebs_num_conv_variants() - 6)
+    with pytest.raises(RuntimeError):
         U.run_conv(qa, qw, d, variant=ebs.ebs_num_conv_variants() - 1)
+
+
+@pytest.mark.parametrize("c,co,k,s,pad,h,n,wb,ab", [(32, 64, 3, 1, 1, 30, 48, 2, 3), (64, 48, 1, 2, 0, 40, 64, 4, 2),
+                                                    (96, 16, 3, 1, 0, 24, 60, 3, 8)])
+def test_persistent_kernel_walks_several_tiles_per_cta(ebs, U, oracle, c, co, k, s, pad, h, n, wb, ab):
+    """More pixel tiles than thread blocks: both accumulators, both stages and the tile loop wrap around."""
+    rng = np.random.default_rng(c + co + k + n)
+    qa = U.rand_codes(rng, (n, c, h, h), ab, False)
+    qw = U.rand_codes(rng, (co, c, k, k), wb, True)
+    d = U.desc_for(c, co, k, s, pad, wb, ab, 0.03, 0.07)
+    ref = oracle.conv2d_codes(qa, qw, (s, s), (pad, pad))
+    y_ref, q_ref = oracle.epilogue(ref, oracle.combined_scale(0.03, 0.07), relu=True, next_bits=4,
+                                   inv_next=np.float32(1.0) / np.float32(0.9))
+    px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
+    epi = ebs.epilogue(relu=True, next_a_bits=4, next_a_scale=0.9)
+    nv = ebs.ebs_num_conv_variants()
+    ran = 0
+    for variant in range(nv - U.N_RESIDENT, nv):
+        if not U.resident_variant_applies(d, h, 16 << (variant - (nv - U.N_RESIDENT))):
+            continue
+        if (16 << (variant - (nv - U.N_RESIDENT))) < min(co, 32):
+            continue                                          # 16-channel tiles cannot write packed words of wider layers
+        out = U.run_conv(qa, qw, d, epi, want_acc=True, want_y=True, next_bits=4, variant=variant, px=px, pw=pw)
+        assert np.array_equal(out["acc"], ref), f"variant {variant}"
+        assert np.array_equal(out["y"], y_ref) and np.array_equal(oracle.unpack_acts(out["packed"], co), q_ref)
+        ran += 1
+    assert ran >= 2 and ebs.ebs_device_wait_timeouts() == 0
 
 
 def test_no_device_wait_timed_out(ebs):
@@ -197,7 +226,7 @@ def test_fused_epilogue_and_requantized_planes(ebs, U, oracle, next_bits, co):
     res_nhwc = to(res.transpose(0, 2, 3, 1))
     for y_layout in (ebs.EBS_NHWC, ebs.EBS_NCHW):
         epi = ebs.epilogue(to(cs), to(cb), res_nhwc, True, next_bits, float(next_scale), y_layout)
-        for variant in (-1, 3, 6, 7, 11, 12, 14, 15, 17, 18, 20, 21, 22, 23, 25, 26, 27, 28):
+        for variant in (-1, 3, 6, 7, 11, 12, 14, 15, 17, 18, 20, 21, 22, 23, 25, 26, 27, 28, 30, 31, 32, 33):
             out = U.run_conv(qa, qw, d, epi, want_acc=True, want_y=True, next_bits=next_bits, variant=variant)
             assert np.array_equal(out["acc"], ref_acc)
             assert np.allclose(out["y"], y_ref, rtol=RTOL, atol=0.0)
