@@ -316,7 +316,42 @@ conv_mma_kernel(const ConvParams p) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 2 * acc[mt][nt][e] + wsum[mt][e >> 1];
     }
-    const bool simple = pair_ok && !p.ch_scale && !p.ch_bias && !p.residual && !p.res_packed && !p.y_nchw;
+    // common case: even c_out and NHWC -> two-channel vectors, per-channel terms kept in registers, the
+    // shortcut codes (if the shortcut comes as packed planes) staged as bytes in the code tile
+    const bool simple = pair_ok && !p.y_nchw;
+    const bool plain = simple && !p.ch_scale && !p.ch_bias && !p.residual && !p.res_packed;
+    if (simple && p.res_packed) {
+        constexpr int GROUPS = TILE_C / 8;
+        for (int e = tid; e < TILE_P * GROUPS; e += NTH) {
+            const int pl = e / GROUPS, grp = e - pl * GROUPS;
+            const int gp = tile_p0 + pl, c = co0 + 8 * grp;
+            uint32_t lo = 0u, hi = 0u;                          // codes of channels c .. c+3 and c+4 .. c+7, one per byte
+            if (gp < p.P && c < p.Co) {
+                const uint32_t* w = p.res_packed + ((size_t)gp * p.CWo + (c >> 5)) * p.res_bits;
+                for (int j = 0; j < p.res_bits; ++j) {
+                    const uint32_t byte = (__ldg(w + j) >> (c & 31)) & 0xFFu;         // plane j of the eight channels
+                    lo |= (((byte & 0xFu) * 0x00204081u) & 0x01010101u) << j;          // bit i -> bit 8 i
+                    hi |= (((byte >> 4) * 0x00204081u) & 0x01010101u) << j;
+                }
+            }
+            uint32_t* dst = reinterpret_cast<uint32_t*>(out_s + pl * ROWB + 8 * grp);
+            dst[0] = lo;
+            dst[1] = hi;
+        }
+        __syncthreads();
+    }
+    float cs[NT][2], cb[NT][2];
+    if (simple && !plain) {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
+            const bool in = co < p.Co;                          // c_out is even here: co + 1 exists with co
+            cs[nt][0] = (p.ch_scale && in) ? __ldg(p.ch_scale + co) : 1.0f;
+            cs[nt][1] = (p.ch_scale && in) ? __ldg(p.ch_scale + co + 1) : 1.0f;
+            cb[nt][0] = (p.ch_bias && in) ? __ldg(p.ch_bias + co) : 0.0f;
+            cb[nt][1] = (p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : 0.0f;
+        }
+    }
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
@@ -326,6 +361,27 @@ conv_mma_kernel(const ConvParams p) {
             const bool pvalid = gp < p.P;
             const size_t row_o = (size_t)gp * p.Co + co0 + wc * NT * 8 + 2 * tq;
             uint8_t* code_row = out_s + pl * ROWB + wc * NT * 8 + 2 * tq;
+            if (plain) {                                        // no per-channel terms, no shortcut
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
+                    const int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
+                    const bool valid = pvalid && co < p.Co;
+                    int code0 = 0, code1 = 0;
+                    if (valid && p.acc) *reinterpret_cast<int2*>(p.acc + row_o + nt * 8) = make_int2(a0, a1);
+                    if (want_y || want_q) {
+                        float y0 = __fmul_rn((float)a0, p.S), y1 = __fmul_rn((float)a1, p.S);
+                        if (p.relu) { y0 = y0 > 0.0f ? y0 : 0.0f; y1 = y1 > 0.0f ? y1 : 0.0f; }
+                        if (valid && want_y) *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
+                        if (valid && want_q) {
+                            code0 = quantize_act_code(y0, p.inv_next, qmax);
+                            code1 = quantize_act_code(y1, p.inv_next, qmax);
+                        }
+                    }
+                    if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
+                }
+                continue;
+            }
             if (simple) {
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
@@ -336,6 +392,18 @@ conv_mma_kernel(const ConvParams p) {
                     if (valid && p.acc) *reinterpret_cast<int2*>(p.acc + row_o + nt * 8) = make_int2(a0, a1);
                     if (want_y || want_q) {
                         float y0 = __fmul_rn((float)a0, p.S), y1 = __fmul_rn((float)a1, p.S);
+                        if (p.ch_scale) { y0 = __fmul_rn(y0, cs[nt][0]); y1 = __fmul_rn(y1, cs[nt][1]); }
+                        if (p.ch_bias) { y0 = __fadd_rn(y0, cb[nt][0]); y1 = __fadd_rn(y1, cb[nt][1]); }
+                        if (p.residual && valid) {
+                            const float2 r = __ldg(reinterpret_cast<const float2*>(p.residual + row_o + nt * 8));
+                            y0 = __fadd_rn(y0, r.x);
+                            y1 = __fadd_rn(y1, r.y);
+                        }
+                        if (p.res_packed) {
+                            const uint32_t rc = *reinterpret_cast<const uint16_t*>(code_row + nt * 8);
+                            y0 = __fadd_rn(y0, __fmul_rn(p.res_scale, (float)(rc & 0xFFu)));
+                            y1 = __fadd_rn(y1, __fmul_rn(p.res_scale, (float)(rc >> 8)));
+                        }
                         if (p.relu) { y0 = y0 > 0.0f ? y0 : 0.0f; y1 = y1 > 0.0f ? y1 : 0.0f; }
                         if (valid && want_y) *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
                         if (valid && want_q) {
