@@ -137,7 +137,10 @@ __device__ __forceinline__ uint32_t pack_sat_u8x4(int a, int b, int c, int d) {
 // of it owns the accumulators of one pixel row (global output pixel gp; pvalid false = row without an
 // output).  Warps w and w + 4 split the channels when the tile is wide enough.  The thread stores the
 // accumulators, applies the fp32 steps and packs the requantized codes of its pixel into plane words.
-template <int TILE_N>
+// AFFINE = false compiles the straight-line path without per-channel terms and shortcuts (layers that have
+// them then take the general path); kernels that are built in both forms pick the form on the host, so the
+// extra registers of the terms do not lower the occupancy of layers without them.
+template <int TILE_N, bool AFFINE = false>
 __device__ __forceinline__ void umma_epilogue(const ConvParams& p, uint32_t tmem_base, int warp, int gp, bool pvalid,
                                               int wsum_row, int co0) {
     constexpr int EPI_WARPS = TILE_N >= 64 ? 8 : 4;
@@ -152,12 +155,15 @@ __device__ __forceinline__ void umma_epilogue(const ConvParams& p, uint32_t tmem
         const int cbeg = (warp >> 2) * COLS_PER_WARP;
         // Common case -- the whole channel tile exists, channels in aligned groups of four, no per-channel
         // terms, no shortcut, NHWC: straight-line code, 32 channels (one packed output word) per round.
-        if (COLS_PER_WARP % 32 == 0 && co0 + TILE_N <= p.Co && vec_ok && !p.ch_scale && !p.ch_bias && !p.residual &&
-            !p.res_packed && !p.y_nchw) {
+        const bool terms_aligned = (((uintptr_t)p.ch_scale | (uintptr_t)p.ch_bias) & 15u) == 0;
+        const bool no_terms = !p.ch_scale && !p.ch_bias && !p.residual && !p.res_packed;
+        if (COLS_PER_WARP % 32 == 0 && co0 + TILE_N <= p.Co && vec_ok && !p.y_nchw &&
+            (AFFINE ? terms_aligned : no_terms)) {
             const int nb = want_q ? p.next_bits : 0;
             const float S = p.S, inv_next = p.inv_next;
             const bool relu = p.relu != 0, w_levels = p.w_levels != 0;
-            // 16 channels of this thread's pixel: store, requantize, shift their plane bits into `planes`
+            // 16 channels of this thread's pixel: store, fp32 steps, requantize, shift their plane bits into `planes`
+            uint32_t resw[8];                                   // shortcut planes of the current 32-channel word
             auto process16 = [&](uint32_t (&v)[16], int cbase, uint32_t (&planes)[8]) {
                 if (w_levels) {
 #pragma unroll
@@ -173,9 +179,50 @@ __device__ __forceinline__ void umma_epilogue(const ConvParams& p, uint32_t tmem
                 if (want_y || want_q) {
                     float y[16];
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        y[e] = __fmul_rn((float)(int)v[e], S);
-                        if (relu) y[e] = y[e] > 0.0f ? y[e] : 0.0f;
+                    for (int e = 0; e < 16; ++e) y[e] = __fmul_rn((float)(int)v[e], S);
+                    if (AFFINE && p.ch_scale) {                 // the same 16 values for every lane: broadcast vector loads
+#pragma unroll
+                        for (int gq = 0; gq < 4; ++gq) {
+                            const float4 t = __ldg(reinterpret_cast<const float4*>(p.ch_scale + co0 + cbase) + gq);
+                            y[4 * gq] = __fmul_rn(y[4 * gq], t.x); y[4 * gq + 1] = __fmul_rn(y[4 * gq + 1], t.y);
+                            y[4 * gq + 2] = __fmul_rn(y[4 * gq + 2], t.z); y[4 * gq + 3] = __fmul_rn(y[4 * gq + 3], t.w);
+                        }
+                    }
+                    if (AFFINE && p.ch_bias) {
+#pragma unroll
+                        for (int gq = 0; gq < 4; ++gq) {
+                            const float4 t = __ldg(reinterpret_cast<const float4*>(p.ch_bias + co0 + cbase) + gq);
+                            y[4 * gq] = __fadd_rn(y[4 * gq], t.x); y[4 * gq + 1] = __fadd_rn(y[4 * gq + 1], t.y);
+                            y[4 * gq + 2] = __fadd_rn(y[4 * gq + 2], t.z); y[4 * gq + 3] = __fadd_rn(y[4 * gq + 3], t.w);
+                        }
+                    }
+                    if (AFFINE && p.residual && pvalid) {
+#pragma unroll
+                        for (int gq = 0; gq < 4; ++gq) {
+                            const float4 t = __ldg(reinterpret_cast<const float4*>(p.residual + o) + gq);
+                            y[4 * gq] = __fadd_rn(y[4 * gq], t.x); y[4 * gq + 1] = __fadd_rn(y[4 * gq + 1], t.y);
+                            y[4 * gq + 2] = __fadd_rn(y[4 * gq + 2], t.z); y[4 * gq + 3] = __fadd_rn(y[4 * gq + 3], t.w);
+                        }
+                    }
+                    if (AFFINE && p.res_packed) {               // shortcut codes from packed planes: bit i of a nibble -> byte i
+                        const int sh = cbase & 16;
+#pragma unroll
+                        for (int gq = 0; gq < 4; ++gq) {
+                            uint32_t c4r = 0u;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                if (j >= p.res_bits) break;
+                                c4r |= ((((resw[j] >> (sh + 4 * gq)) & 0xFu) * 0x00204081u) & 0x01010101u) << j;
+                            }
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                y[4 * gq + e] = __fadd_rn(y[4 * gq + e],
+                                                          __fmul_rn(p.res_scale, (float)((c4r >> (8 * e)) & 0xFFu)));
+                        }
+                    }
+                    if (relu) {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) y[e] = y[e] > 0.0f ? y[e] : 0.0f;
                     }
                     if (want_y && pvalid) {
 #pragma unroll
@@ -212,6 +259,11 @@ __device__ __forceinline__ void umma_epilogue(const ConvParams& p, uint32_t tmem
 #pragma unroll 1
             for (int c0 = cbeg; c0 < cbeg + COLS_PER_WARP; c0 += 32) {
                 uint32_t planes[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+                if (AFFINE && p.res_packed) {
+                    const uint32_t* rw = p.res_packed + ((size_t)gp * p.CWo + ((co0 + c0) >> 5)) * p.res_bits;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) resw[j] = (pvalid && j < p.res_bits) ? __ldg(rw + j) : 0u;
+                }
                 tmem_ld16_wait(va);
                 tmem_ld16_issue(trow + (uint32_t)c0, vb);
                 process16(va, c0 + 16, planes);

@@ -56,7 +56,7 @@ inline ResidentGeom resident_geometry(const ConvParams& p, int tile_n, int sms) 
     return g;
 }
 
-template <int AB, int TILE_N>
+template <int AB, int TILE_N, bool AFFINE>
 __global__ void __launch_bounds__(RES_THREADS, 1) conv_umma_resident_kernel(const ConvParams p) {
     constexpr int TMEM_COLS = 2 * TILE_N < 32 ? 32 : 2 * TILE_N;     // two accumulators
     constexpr int B_TILE_BYTES = TILE_N * 32;
@@ -245,7 +245,7 @@ __global__ void __launch_bounds__(RES_THREADS, 1) conv_umma_resident_kernel(cons
                 pvalid = hp < p.Ho && wp < p.Wo;
                 gp = (n * p.Ho + hp) * p.Wo + wp;
             }
-            umma_epilogue<TILE_N>(p, tmem_base + (uint32_t)(buf * TILE_N), vwarp, gp, pvalid, 0, co0);
+            umma_epilogue<TILE_N, AFFINE>(p, tmem_base + (uint32_t)(buf * TILE_N), vwarp, gp, pvalid, 0, co0);
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
             mbar_arrive(&acc_empty[buf]);
         }
@@ -273,11 +273,15 @@ void launch_conv_umma_resident(const ConvParams& p0, dim3 /*grid*/, cudaStream_t
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaFuncSetAttribute(conv_umma_resident_kernel<AB, TILE_N>, cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024);
+        cudaFuncSetAttribute(conv_umma_resident_kernel<AB, TILE_N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024);
+        cudaFuncSetAttribute(conv_umma_resident_kernel<AB, TILE_N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024);
         attr_set[dev] = true;
     }
     const dim3 grid((unsigned)g.grid_x, (unsigned)((p.Co + TILE_N - 1) / TILE_N), 1);
-    conv_umma_resident_kernel<AB, TILE_N><<<grid, RES_THREADS, g.smem_bytes, st>>>(p);
+    if (p.ch_scale || p.ch_bias || p.residual || p.res_packed)
+        conv_umma_resident_kernel<AB, TILE_N, true><<<grid, RES_THREADS, g.smem_bytes, st>>>(p);
+    else
+        conv_umma_resident_kernel<AB, TILE_N, false><<<grid, RES_THREADS, g.smem_bytes, st>>>(p);
 }
 
 constexpr int NUM_UMMA_RESIDENT_VARIANTS = 5;      // TILE_N = 16, 32, 64, 128, 256

@@ -95,7 +95,7 @@ __device__ long long g_strip_trace[4][16];
 #define STRIP_TRACE(i, cond) do { } while (0)
 #endif
 
-template <int AB, int TILE_N>
+template <int AB, int TILE_N, bool AFFINE>
 __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const ConvParams p) {
     constexpr int TMEM_COLS = TILE_N < 32 ? 32 : TILE_N;
     constexpr int B_TILE_BYTES = TILE_N * 32;
@@ -290,7 +290,7 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
         if (p.w_levels)
             for (int r = 0; r < p.kh; ++r)
                 for (int s = 0; s < p.kw; ++s) wsum_row += csum_s[row + r * Wp + s];
-        umma_epilogue<TILE_N>(p, tmem_base, warp, gp, pvalid, wsum_row, co0);
+        umma_epilogue<TILE_N, AFFINE>(p, tmem_base, warp, gp, pvalid, wsum_row, co0);
     }
     if (aborted && tid == 0) atomicAdd(&g_umma_timeouts, 1ull);
     STRIP_TRACE(10, tid == 0);
@@ -312,16 +312,19 @@ void launch_conv_umma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st
     if (!g.ok) return;                                        // callers check strip_geometry first
     p.strip_pix = g.strip_pix;
     p.strip_ks = g.ks;
-    static int attr_bytes[64] = {};                           // largest dynamic shared memory enabled, per device
+    const bool affine = p.ch_scale || p.ch_bias || p.residual || p.res_packed;
+    static bool attr_set[64] = {};                            // dynamic shared memory limit raised, per device
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && attr_bytes[dev] < g.smem_bytes) {
-        cudaFuncSetAttribute(conv_umma_strip_kernel<AB, TILE_N>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        attr_bytes[dev] = 200 * 1024;
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        cudaFuncSetAttribute(conv_umma_strip_kernel<AB, TILE_N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        cudaFuncSetAttribute(conv_umma_strip_kernel<AB, TILE_N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        attr_set[dev] = true;
     }
     const long long frame = (long long)p.N * strip_frame_h(p) * strip_frame_w(p);
     const dim3 grid((unsigned)((frame + UMMA_M - 1) / UMMA_M), (unsigned)((p.Co + TILE_N - 1) / TILE_N), 1);
-    conv_umma_strip_kernel<AB, TILE_N><<<grid, UMMA_THREADS, g.smem_bytes, st>>>(p);
+    if (affine) conv_umma_strip_kernel<AB, TILE_N, true><<<grid, UMMA_THREADS, g.smem_bytes, st>>>(p);
+    else conv_umma_strip_kernel<AB, TILE_N, false><<<grid, UMMA_THREADS, g.smem_bytes, st>>>(p);
 }
 
 constexpr int NUM_UMMA_STRIP_VARIANTS = 5;      // TILE_N = 16, 32, 64, 128, 256
