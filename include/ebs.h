@@ -252,6 +252,61 @@ double ebs_expected_flops(double macs, const int *bits_w, const float *coeff_w, 
                           const float *coeff_x, int n_x);
 
 /*
+ * Whole-network inference of a basic-block CIFAR ResNet (Sec. 5, Table 1) in ONE launch: a thread
+ * block carries one image through every layer with its activation codes resident in shared memory
+ * as bytes (no bit planes, no global traffic and no launch between layers); the arithmetic of every
+ * layer is that of ebs_conv2d_mixed with a fused epilogue, so the logits equal those of the
+ * layer-by-layer calls bit for bit.  The paper has no counterpart (it runs layer by layer).
+ *
+ * Layers are described by ebs_fused_layer records in execution order:
+ *   w8         the byte image of the layer's weights: packed_w + ebs_packed_weight_plane_bytes(desc)
+ *   k, stride  3x3 (stride 1 or 2, padding 1) or the 1x1 stride-2 projection shortcut (hold = 1)
+ *   src, dst   activation strips 0..2 in shared memory; the image is loaded into strip 0; dst = -1
+ *              on the last layer sends its fp32 result to pooling
+ *   res        0 none; 1 identity shortcut: res_step * code read from strip res_buf; 2 projection:
+ *              the previous record (hold = 1) kept its accumulators in tensor memory and this
+ *              epilogue adds fl(fl(acc * S) * ch_scale + ch_bias) of that record
+ *   zero_dst   clear strip dst first (set whenever the strip last held another geometry)
+ *   S          fl32(w_scale * a_scale); out_inv_step = fl32(1 / step of the output codes)
+ *   trace_off  byte offset of this layer's output codes (u8, [Ho][Wo][c_out]) inside each image's
+ *              slice of the trace buffer, or -1
+ * Limits: c_in, c_out <= 64, (h_in + 2) * (w_in + 2) <= 1156 frame pixels (32 x 32 images).
+ * ebs_fused_plan_upload validates the records (host array) and copies them to layers_dev
+ * (n_layers * sizeof(ebs_fused_layer) bytes of device memory); ebs_resnet_cifar_forward takes that
+ * device array, u8 NHWC images [n][img_h][img_w][3] and writes fp32 logits [n][head.c_out].
+ * The head is global average pooling (pixels added in order, times fl32(1/HW)), quantization of the
+ * pooled features to 8 bits (a_inv_step = fl32(1 / a_scale)) and the classifier as an integer dot
+ * product with its byte image, scaled by S and the per-channel terms.
+ */
+typedef struct ebs_fused_layer {
+    const unsigned char *w8;
+    const float *ch_scale;
+    const float *ch_bias;
+    int c_in, c_out, k, stride;
+    int h_in, w_in;
+    int src, dst;
+    int res;
+    int relu, out_bits, hold;
+    int zero_dst;
+    int trace_off;
+    float S, out_inv_step, res_step;
+    int res_buf;
+} ebs_fused_layer;
+
+typedef struct ebs_fused_head {
+    const unsigned char *w8;
+    const float *ch_scale;
+    const float *ch_bias;
+    int c_in, c_out;
+    float a_inv_step, S;
+} ebs_fused_head;
+
+int ebs_fused_plan_upload(const ebs_fused_layer *layers_host, int n_layers, void *layers_dev, void *stream);
+int ebs_resnet_cifar_forward(const unsigned char *images_dev, int n, int img_h, int img_w, const void *layers_dev,
+                             int n_layers, const ebs_fused_head *head_host, float *logits_dev,
+                             unsigned char *trace_dev, long long trace_stride, void *stream);
+
+/*
  * Global average pooling between the last residual block and the classifier of the ResNets the
  * paper evaluates (Sec. 5); not part of the binary decomposition itself.  y_dev is fp32 NHWC
  * [n][hw][c]; out_dev receives [n][c]: the pixels are added in order 0 .. hw-1 in fp32 and the

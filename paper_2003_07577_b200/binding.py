@@ -26,7 +26,7 @@ EXPORTS = [
     "ebs_packed_act_bytes", "ebs_pack_weights", "ebs_pack_acts", "ebs_conv2d_mixed", "ebs_num_conv_variants",
     "ebs_conv2d_mixed_variant", "ebs_dequant", "ebs_host_workspace_bytes", "ebs_conv2d_mixed_host",
     "ebs_probe_pipe", "ebs_device_wait_timeouts", "ebs_global_avgpool", "ebs_packed_weight_plane_bytes", "ebs_search_weight_forward",
-    "ebs_search_act_forward", "ebs_expected_flops", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
+    "ebs_search_act_forward", "ebs_expected_flops", "ebs_fused_plan_upload", "ebs_resnet_cifar_forward", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
 ]
 
 
@@ -92,6 +92,8 @@ def lib() -> ctypes.CDLL:
         L.ebs_search_act_forward.argtypes = [p, z, ctypes.c_float, ip, fp, i, p, p]
         L.ebs_expected_flops.argtypes = [ctypes.c_double, ip, fp, i, ip, fp, i]
         L.ebs_expected_flops.restype = ctypes.c_double
+        L.ebs_fused_plan_upload.argtypes = [ctypes.c_void_p, i, p, p]
+        L.ebs_resnet_cifar_forward.argtypes = [p, i, i, i, p, i, ctypes.c_void_p, p, p, ctypes.c_longlong, p]
         L.ebs_noalloc_scratch_bytes.restype = z
         L.ebs_device_wait_timeouts.restype = ctypes.c_longlong
         L.ebs_conv2d_mixed_host_noalloc.argtypes = [p, i, i, i, i, i, p, D, E, p, p, p, p]
@@ -213,6 +215,34 @@ def ebs_probe_pipe(kind: int, iters: int = 2000) -> float:
 
 def ebs_global_avgpool(y_dev, n: int, hw: int, c: int, out_dev, stream=None) -> None:
     _check(lib().ebs_global_avgpool(_ptr(y_dev), n, hw, c, _ptr(out_dev), _stream(stream)), "ebs_global_avgpool")
+
+
+class ebs_fused_layer(ctypes.Structure):
+    _fields_ = [("w8", ctypes.c_void_p), ("ch_scale", ctypes.c_void_p), ("ch_bias", ctypes.c_void_p),
+                ("c_in", ctypes.c_int), ("c_out", ctypes.c_int), ("k", ctypes.c_int), ("stride", ctypes.c_int),
+                ("h_in", ctypes.c_int), ("w_in", ctypes.c_int), ("src", ctypes.c_int), ("dst", ctypes.c_int),
+                ("res", ctypes.c_int), ("relu", ctypes.c_int), ("out_bits", ctypes.c_int), ("hold", ctypes.c_int),
+                ("zero_dst", ctypes.c_int), ("trace_off", ctypes.c_int), ("S", ctypes.c_float),
+                ("out_inv_step", ctypes.c_float), ("res_step", ctypes.c_float), ("res_buf", ctypes.c_int)]
+
+
+class ebs_fused_head(ctypes.Structure):
+    _fields_ = [("w8", ctypes.c_void_p), ("ch_scale", ctypes.c_void_p), ("ch_bias", ctypes.c_void_p),
+                ("c_in", ctypes.c_int), ("c_out", ctypes.c_int), ("a_inv_step", ctypes.c_float), ("S", ctypes.c_float)]
+
+
+def ebs_fused_plan_upload(layers, layers_dev: torch.Tensor, stream=None) -> None:
+    """layers: list of ebs_fused_layer; layers_dev: uint8 device tensor of len(layers) * sizeof(ebs_fused_layer) bytes."""
+    arr = (ebs_fused_layer * len(layers))(*layers)
+    _check(lib().ebs_fused_plan_upload(arr, len(layers), _ptr(layers_dev), _stream(stream)), "ebs_fused_plan_upload")
+    torch.cuda.current_stream().synchronize()          # the host array may be released after the copy
+
+
+def ebs_resnet_cifar_forward(images_dev, n, img_h, img_w, layers_dev, n_layers, head: ebs_fused_head, logits_dev,
+                             trace_dev=None, trace_stride: int = 0, stream=None) -> None:
+    _check(lib().ebs_resnet_cifar_forward(_ptr(images_dev), n, img_h, img_w, _ptr(layers_dev), n_layers,
+                                          ctypes.byref(head), _ptr(logits_dev), _ptr(trace_dev), trace_stride,
+                                          _stream(stream)), "ebs_resnet_cifar_forward")
 
 
 def _cand(bits, coeff):

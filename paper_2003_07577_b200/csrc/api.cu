@@ -59,7 +59,7 @@ const ConvVariant* conv_umma_variant(int w_bits, int a_bits, int variant) {
 unsigned long long conv_umma_timeouts() {
     return conv_umma_timeouts_w1() + conv_umma_timeouts_w2() + conv_umma_timeouts_w3() + conv_umma_timeouts_w4() +
            conv_umma_timeouts_w5() + conv_umma_timeouts_w6() + conv_umma_timeouts_w7() + conv_umma_timeouts_w8() +
-           conv_umma_strip_timeouts() + conv_umma_resident_timeouts();
+           conv_umma_strip_timeouts() + conv_umma_resident_timeouts() + fused_net_timeouts();
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -367,6 +367,22 @@ double ebs_expected_flops(double macs, const int* bits_w, const float* coeff_w, 
     for (int i = 0; i < n_w; ++i) m += (double)coeff_w[i] * bits_w[i];
     for (int j = 0; j < n_x; ++j) k += (double)coeff_x[j] * bits_x[j];
     return macs * m * k;
+}
+
+int ebs_fused_plan_upload(const ebs_fused_layer* layers_host, int n_layers, void* layers_dev, void* stream) {
+    if (!layers_host || !layers_dev || n_layers < 1 || n_layers > 4096) return EBS_ERR_INVALID_ARG;
+    return fused_plan_upload(layers_host, n_layers, layers_dev, static_cast<cudaStream_t>(stream));
+}
+
+int ebs_resnet_cifar_forward(const unsigned char* images_dev, int n, int img_h, int img_w, const void* layers_dev,
+                             int n_layers, const ebs_fused_head* head_host, float* logits_dev, unsigned char* trace_dev,
+                             long long trace_stride, void* stream) {
+    if (!images_dev || !layers_dev || !head_host || !logits_dev || n < 1 || n_layers < 1) return EBS_ERR_INVALID_ARG;
+    if (img_h < 1 || img_w < 1 || (img_h + 2) * (img_w + 2) > 1156) return EBS_ERR_UNSUPPORTED;
+    if (!head_host->w8 || head_host->c_in < 1 || head_host->c_in > 64 || head_host->c_out < 1 || head_host->c_out > 256)
+        return EBS_ERR_INVALID_ARG;
+    return launch_fused_resnet(images_dev, n, img_h, img_w, layers_dev, n_layers, head_host, logits_dev, trace_dev,
+                               trace_stride, static_cast<cudaStream_t>(stream));
 }
 
 int ebs_global_avgpool(const float* y_dev, int n, int hw, int c, float* out_dev, void* stream) {

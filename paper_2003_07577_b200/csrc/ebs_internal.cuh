@@ -97,6 +97,10 @@ int launch_search_weights(const float* w, size_t n, const int* bits, const float
                           void* scratch, cudaStream_t st);
 int launch_search_acts(const float* x, size_t n, float alpha, const int* bits, const float* coeff, int n_cand,
                        float* x_hat, cudaStream_t st);
+int fused_plan_upload(const void* layers_host, int n_layers, void* layers_dev, cudaStream_t st);
+int launch_fused_resnet(const uint8_t* images, int n, int img_h, int img_w, const void* layers_dev, int n_layers,
+                        const void* head_host, float* logits, uint8_t* trace, long long trace_stride, cudaStream_t st);
+unsigned long long fused_net_timeouts();
 int launch_avgpool(const float* y, int n, int hw, int c, float* out, cudaStream_t st);
 
 // Records a CUDA error for ebs_last_cuda_error() and returns EBS_ERR_CUDA (or EBS_OK).

@@ -1,0 +1,353 @@
+// Whole-network kernel for basic-block CIFAR ResNets: one CTA carries one image through every layer
+// with its activations resident in shared memory.
+//
+// The per-layer kernels spend most of a ResNet-20 layer's 5-18 us on launch, prologue and moving 4-37 KB
+// of activations per image through L2.  Here the activation codes of an image live in shared memory as
+// BYTES, already in the un-swizzled K-major strip layout the tcgen05 operand descriptors read
+// ([16-byte half][frame pixel][16 bytes] per 32-channel word, frame = zero-padded image), so between
+// layers there is no bit-to-byte expansion, no global traffic and no launch.  Per layer the CTA
+//   1. has the layer's weight byte image (the second part of an ebs_pack_weights buffer) fetched into one
+//      of two shared buffers by cp.async.bulk while the previous layer runs,
+//   2. lets one thread issue all MMAs of the layer -- every 128-row tile of the frame x every tap x every
+//      32-channel word, a tap being a shifted descriptor -- into tensor-memory accumulators (tile t at
+//      columns 32 t or 64 t), then tcgen05.commit onto an mbarrier,
+//   3. runs the fp32 steps of the epilogue out of tensor memory (scale, per-channel scale/shift, shortcut,
+//      ReLU, requantize: the same individually rounded operations as the per-layer kernels) and writes the
+//      codes as bytes at frame position f + Wp + 1 of the destination strip: outputs that do not exist
+//      (frame columns >= Wo, rows >= Ho) land exactly on padding positions and are written as zero.
+// Stride-2 3x3 layers are computed at stride 1 and subsampled in the epilogue (4x the MMAs of two or three
+// layers, no phase logic); a 1x1 stride-2 projection runs on a subsampled copy of its input laid out in the
+// output frame, keeps its accumulators in tensor memory, and the next layer's epilogue adds them as the
+// shortcut.  The identity shortcut is read from the destination strip (the block input) just before it is
+// overwritten in place.  After the last block: average pooling (pixels added in order), 8-bit
+// quantization, and the classifier as a plain integer dot product.
+// Every wait is bounded; on a timeout the CTA sets its abort flag, skips the rest, frees tensor memory.
+#include "conv_umma_strip.cuh"
+
+namespace ebs {
+
+constexpr int FUSED_THREADS = 256;
+constexpr int FUSED_ACT_PIX = 1360;                    // pixels an activation strip holds (34 x 34 frame + halo, 128-row tiles)
+constexpr int FUSED_ACT_BYTES = FUSED_ACT_PIX * 32;    // one 32-channel word
+constexpr int FUSED_W_BYTES = 37 * 1024;               // largest weight image (3x3 64->64)
+constexpr int FUSED_SMEM = 3 * FUSED_ACT_BYTES + 2 * FUSED_W_BYTES + 1024;
+constexpr int FUSED_HOLD_COL = 320;                    // accumulator columns of a held projection
+
+using FusedLayer = ebs_fused_layer;
+using FusedHead = ebs_fused_head;
+
+__device__ __forceinline__ uint8_t* strip_ptr(uint8_t* acts, int buf) { return acts + buf * FUSED_ACT_BYTES; }
+// A strip holds one 32-channel word of up to 1360 frame pixels or two words of up to 680: pixels per word.
+__host__ __device__ inline int strip_cap(int channels) { return channels > 32 ? FUSED_ACT_PIX / 2 : FUSED_ACT_PIX; }
+
+__global__ void __launch_bounds__(FUSED_THREADS, 1)
+fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, const FusedLayer* __restrict__ layers,
+                    int n_layers, const FusedHead head, float* __restrict__ logits, uint8_t* __restrict__ trace,
+                    long long trace_stride) {
+    extern __shared__ uint8_t dyn_smem[];
+    __shared__ __align__(8) uint64_t w_bar[2], mma_bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ int fc_codes[64];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int img = blockIdx.x;
+    uint8_t* base = dyn_smem + ((1024u - (smem_u32(dyn_smem) & 1023u)) & 1023u);
+    uint8_t* acts = base;                                        // three strips
+    uint8_t* wbuf = base + 3 * FUSED_ACT_BYTES;                  // two weight images
+    volatile int* abortp = &abort_flag;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(&w_bar[0], 1);
+        mbar_init(&w_bar[1], 1);
+        mbar_init(&mma_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&tmem_slot)),
+                     "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    // all strips start as zeros (padding positions are never written with anything else)
+    for (int i = tid; i < 3 * FUSED_ACT_BYTES / 16; i += FUSED_THREADS) reinterpret_cast<uint4*>(acts)[i] = make_uint4(0, 0, 0, 0);
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    const uint32_t tmem_base = tmem_slot;
+
+    auto fetch_weights = [&](int li) {                           // one thread: the whole byte image of layer li
+        const FusedLayer& L = layers[li];
+        const int cw = (L.c_in + 31) >> 5, co16 = (L.c_out + 15) & ~15;
+        const uint32_t bytes = (uint32_t)(L.k * L.k * cw * co16 * 32);
+        mbar_arrive_expect_tx(&w_bar[li & 1], bytes);
+        bulk_copy_g2s(wbuf + (li & 1) * FUSED_W_BYTES, L.w8, bytes, &w_bar[li & 1]);
+    };
+    if (tid == 0 && n_layers > 0) fetch_weights(0);
+
+    // ---- the image: u8 NHWC, 3 channels -> bytes of strip 0 in the padded frame (channel c is byte 4c of word 0)
+    {
+        const int Wp = img_w + 2;
+        const uint8_t* src = images + (size_t)img * img_h * img_w * 3;
+        for (int pix = tid; pix < img_h * img_w; pix += FUSED_THREADS) {
+            const int h = pix / img_w, w = pix - h * img_w;
+            const uint32_t r = src[pix * 3], g = src[pix * 3 + 1], b = src[pix * 3 + 2];
+            uint32_t* dst = reinterpret_cast<uint32_t*>(strip_ptr(acts, 0) + ((h + 1) * Wp + (w + 1)) * 16);
+            dst[0] = r; dst[1] = g; dst[2] = b;                   // words 0..2 of the first 16-byte half: channels 0, 1, 2
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    __syncthreads();
+
+    bool ok = true;
+    int mma_phase = 0;
+    float* pool_scratch = reinterpret_cast<float*>(strip_ptr(acts, 0));      // [pixels][c_out] of the last layer
+
+    for (int li = 0; li < n_layers && ok; ++li) {
+        const FusedLayer L = layers[li];
+        const int cw = (L.c_in + 31) >> 5, co16 = (L.c_out + 15) & ~15;
+        const int Ho = L.stride == 2 ? L.h_in / 2 : L.h_in, Wo = L.stride == 2 ? L.w_in / 2 : L.w_in;
+        // frame in which the MMAs run: the padded input for a 3x3 layer, the padded OUTPUT frame for the projection
+        const int Hf = L.k == 3 ? L.h_in + 2 : Ho + 2, Wf = L.k == 3 ? L.w_in + 2 : Wo + 2;
+        const int frame = Hf * Wf;
+        const int tiles = (frame + UMMA_M - 1) / UMMA_M;
+        const int acc_stride = co16 > 32 ? co16 : 32;
+        const int col0 = L.hold ? FUSED_HOLD_COL : 0;
+        const int Wp_out = Wo + 2;                                 // frame of the destination strip
+        const int cap_in = strip_cap(L.c_in), cap_out = strip_cap(L.c_out);   // pixels per word of the strips read / written
+        uint8_t* src_strip = strip_ptr(acts, L.src);
+        uint8_t* dst_strip = L.dst >= 0 ? strip_ptr(acts, L.dst) : nullptr;
+
+        if (tid == 0 && li + 1 < n_layers) fetch_weights(li + 1);  // its buffer was last read by layer li-1, finished
+
+        if (L.k == 1) {
+            // projection: its input is the stride-2 subsample of strip src, copied into strip dst in the output frame
+            for (int i = tid; i < FUSED_ACT_BYTES / 16; i += FUSED_THREADS)
+                reinterpret_cast<uint4*>(dst_strip)[i] = make_uint4(0, 0, 0, 0);
+            __syncthreads();
+            const int Wp_in = L.w_in + 2;
+            for (int e = tid; e < Ho * Wo * cw * 2; e += FUSED_THREADS) {
+                const int half = e & 1, rest = e >> 1, wd = rest % cw, pix = rest / cw;
+                const int ho = pix / Wo, wo = pix - ho * Wo;
+                const uint8_t* s = src_strip + wd * cap_in * 32 + half * cap_in * 16 + ((2 * ho + 1) * Wp_in + 2 * wo + 1) * 16;
+                uint8_t* d = dst_strip + wd * cap_in * 32 + half * cap_in * 16 + ((ho + 1) * Wf + wo + 1) * 16;
+                *reinterpret_cast<uint4*>(d) = *reinterpret_cast<const uint4*>(s);
+            }
+        } else if (L.zero_dst && dst_strip) {
+            for (int i = tid; i < FUSED_ACT_BYTES / 16; i += FUSED_THREADS)
+                reinterpret_cast<uint4*>(dst_strip)[i] = make_uint4(0, 0, 0, 0);
+        }
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+        __syncthreads();
+
+        // ---- MMAs of the whole layer
+        if (!mbar_wait_bounded(&w_bar[li & 1], (uint32_t)((li >> 1) & 1), abortp)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        if (tid == 0) {
+            const uint32_t idesc = umma_idesc_i8(co16);
+            const uint8_t* a_src = L.k == 1 ? dst_strip : src_strip;   // the projection reads its subsampled copy
+            const uint32_t a_base = smem_u32(a_src), b_base = smem_u32(wbuf + (li & 1) * FUSED_W_BYTES);
+            for (int t = 0; t < tiles; ++t) {
+                const uint32_t tmem_d = tmem_base + (uint32_t)(col0 + t * acc_stride);
+                int first = 1;
+                for (int wd = 0; wd < cw; ++wd) {
+                    for (int tap = 0; tap < L.k * L.k; ++tap) {
+                        const int r = tap / L.k, s = tap - r * L.k;
+                        const int shift = L.k == 3 ? r * Wf + s : Wf + 1;    // 1x1: the centre of the output frame
+                        const uint64_t da = umma_desc_interleaved(a_base + wd * cap_in * 32 + (t * UMMA_M + shift) * 16,
+                                                                  (uint32_t)(cap_in * 16));
+                        const uint64_t db = umma_desc_sw32(b_base + (tap * cw + wd) * co16 * 32);
+                        umma_i8(tmem_d, da, db, idesc, first ? 0u : 1u);
+                        first = 0;
+                    }
+                }
+            }
+            umma_commit(&mma_bar);
+        }
+        if (!mbar_wait_bounded(&mma_bar, (uint32_t)(mma_phase & 1), abortp)) { ok = false; break; }
+        ++mma_phase;
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+
+        // ---- epilogue (a held projection has none: the next layer reads its accumulators)
+        if (!L.hold) {
+            const FusedLayer P = L.res == 2 ? layers[li - 1] : L;   // the projection whose accumulators are held
+            const int qmax = (1 << L.out_bits) - 1;
+            const int quarter = warp & 3;
+            for (int t = warp >> 2; t < tiles; t += 2) {
+                const int f = t * UMMA_M + quarter * 32 + lane;
+                const int hp = f / Wf, wp = f - hp * Wf;
+                // does this frame row have an output, and where does it go in the destination frame
+                bool valid = f < frame;
+                int ho = hp, wo = wp;
+                if (L.stride == 2) { valid = valid && !(hp & 1) && !(wp & 1); ho = hp >> 1; wo = wp >> 1; }
+                valid = valid && ho < Ho && wo < Wo;
+                const int target = L.stride == 2 ? (ho + 1) * Wp_out + wo + 1 : f + Wf + 1;
+                const bool in_frame = f < frame && (L.stride == 1 || valid);   // stride 1 also writes the zeros of the padding
+                const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(col0 + t * acc_stride);
+                const uint32_t prow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(FUSED_HOLD_COL + t * acc_stride);
+#pragma unroll 1
+                for (int c0 = 0; c0 < co16; c0 += 32) {
+                    int q[32];
+                    uint32_t res_lo[4] = {0, 0, 0, 0}, res_hi[4] = {0, 0, 0, 0};
+                    if (L.res == 1 && valid) {
+                        const uint8_t* rp = strip_ptr(acts, L.res_buf) + (c0 >> 5) * cap_out * 32 + target * 16;
+                        const uint4 a = *reinterpret_cast<const uint4*>(rp), b = *reinterpret_cast<const uint4*>(rp + cap_out * 16);
+                        res_lo[0] = a.x; res_lo[1] = a.y; res_lo[2] = a.z; res_lo[3] = a.w;
+                        res_hi[0] = b.x; res_hi[1] = b.y; res_hi[2] = b.z; res_hi[3] = b.w;
+                    }
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf) {
+                        uint32_t v[16], pv[16];
+                        if (c0 + 16 * hf < co16) tmem_ld16(trow + (uint32_t)(c0 + 16 * hf), v);
+                        else {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) v[e] = 0u;
+                        }
+                        if (L.res == 2 && c0 + 16 * hf < co16) tmem_ld16(prow + (uint32_t)(c0 + 16 * hf), pv);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const int c = c0 + 16 * hf + e;
+                            float y = __fmul_rn((float)(int)v[e], L.S);
+                            if (c < L.c_out) {
+                                if (L.ch_scale) y = __fmul_rn(y, __ldg(L.ch_scale + c));
+                                if (L.ch_bias) y = __fadd_rn(y, __ldg(L.ch_bias + c));
+                                if (L.res == 2) {                   // projection shortcut: its own scale and per-channel terms
+                                    float r = __fmul_rn((float)(int)pv[e], P.S);
+                                    if (P.ch_scale) r = __fmul_rn(r, __ldg(P.ch_scale + c));
+                                    if (P.ch_bias) r = __fadd_rn(r, __ldg(P.ch_bias + c));
+                                    y = __fadd_rn(y, r);
+                                }
+                                if (L.res == 1) {                   // identity shortcut: byte (c / 8) of word (c % 8)
+                                    const int cc = c & 31, k8 = cc & 7;
+                                    const uint32_t wv = k8 < 4 ? res_lo[k8] : res_hi[k8 - 4];
+                                    y = __fadd_rn(y, __fmul_rn(L.res_step, (float)((wv >> (8 * (cc >> 3))) & 0xFFu)));
+                                }
+                            }
+                            if (L.relu && !(y > 0.0f)) y = 0.0f;
+                            int code = 0;
+                            if (valid && c < L.c_out) {
+                                if (L.dst < 0) pool_scratch[(ho * Wo + wo) * L.c_out + c] = y;
+                                else code = quantize_act_code(y, L.out_inv_step, qmax);
+                            }
+                            q[16 * hf + e] = code;
+                        }
+                    }
+                    if (L.dst >= 0 && in_frame) {
+                        // word k of the pixel = channels k, 8+k, 16+k, 24+k as bytes
+                        uint32_t w8v[8];
+#pragma unroll
+                        for (int k8 = 0; k8 < 8; ++k8) w8v[k8] = pack_sat_u8x4(q[k8], q[8 + k8], q[16 + k8], q[24 + k8]);
+                        uint8_t* wp_ = dst_strip + (c0 >> 5) * cap_out * 32 + target * 16;
+                        *reinterpret_cast<uint4*>(wp_) = make_uint4(w8v[0], w8v[1], w8v[2], w8v[3]);
+                        *reinterpret_cast<uint4*>(wp_ + cap_out * 16) = make_uint4(w8v[4], w8v[5], w8v[6], w8v[7]);
+                        if (trace && L.trace_off >= 0 && valid) {
+                            uint8_t* tp = trace + (size_t)img * trace_stride + L.trace_off + (size_t)(ho * Wo + wo) * L.c_out + c0;
+                            for (int e = 0; e < 32 && c0 + e < L.c_out; ++e) tp[e] = (uint8_t)q[e];
+                        }
+                    }
+                }
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+        __syncthreads();
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    }
+
+    // ---- pooling, 8-bit quantization, classifier
+    if (ok && !abort_flag && n_layers > 0) {
+        const FusedLayer L = layers[n_layers - 1];
+        const int Ho = L.stride == 2 ? L.h_in / 2 : L.h_in, Wo = L.stride == 2 ? L.w_in / 2 : L.w_in;
+        const int hw = Ho * Wo, C = L.c_out;
+        if (tid < C && tid < 64) {
+            float acc = 0.0f;
+            for (int p = 0; p < hw; ++p) acc = __fadd_rn(acc, pool_scratch[p * C + tid]);
+            const float m = __fmul_rn(acc, 1.0f / (float)hw);
+            fc_codes[tid] = quantize_act_code(m, head.a_inv_step, 255);
+        }
+        __syncthreads();
+        if (tid < head.c_out) {
+            const int co16 = (head.c_out + 15) & ~15, cwf = (head.c_in + 31) >> 5;
+            int acc = 0;
+            for (int c = 0; c < head.c_in; ++c) {
+                const int wd = c >> 5, cc = c & 31, j = 4 * (cc & 7) + (cc >> 3);      // byte 4b + i of the row
+                const int jj = j ^ (((tid >> 2) & 1) << 4);                               // halves swapped for these rows
+                const int8_t wv = (int8_t)head.w8[((size_t)wd * co16 + tid) * 32 + jj];
+                acc += (int)wv * fc_codes[c];
+            }
+            (void)cwf;
+            float y = __fmul_rn((float)acc, head.S);
+            if (head.ch_scale) y = __fmul_rn(y, __ldg(head.ch_scale + tid));
+            if (head.ch_bias) y = __fadd_rn(y, __ldg(head.ch_bias + tid));
+            logits[(size_t)img * head.c_out + tid] = y;
+        }
+    }
+    if (abort_flag != 0 && tid == 0) atomicAdd(&g_umma_timeouts, 1ull);
+
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+// Limits of the kernel for one layer; returns EBS_OK or the reason it cannot run.
+static int check_layer(const FusedLayer& L, const FusedLayer* prev) {
+    if (!L.w8 || (L.k != 1 && L.k != 3) || (L.stride != 1 && L.stride != 2)) return EBS_ERR_INVALID_ARG;
+    if (L.c_in < 1 || L.c_in > 64 || L.c_out < 1 || L.c_out > 64 || L.h_in < 1 || L.w_in < 1) return EBS_ERR_UNSUPPORTED;
+    if (L.k == 1 && (L.stride != 2 || !L.hold)) return EBS_ERR_UNSUPPORTED;        // 1x1 only as the strided projection
+    if (L.stride == 2 && ((L.h_in | L.w_in) & 1)) return EBS_ERR_UNSUPPORTED;
+    if (L.src < 0 || L.src > 2 || L.dst < -1 || L.dst > 2 || (L.hold && L.dst < 0)) return EBS_ERR_INVALID_ARG;
+    if (L.res < 0 || L.res > 2 || (L.res == 1 && (L.res_buf < 0 || L.res_buf > 2))) return EBS_ERR_INVALID_ARG;
+    if (L.res == 2 && (!prev || !prev->hold || prev->c_out != L.c_out)) return EBS_ERR_INVALID_ARG;
+    if (L.dst >= 0 && !L.hold && (L.out_bits < 1 || L.out_bits > 8 || !(L.out_inv_step > 0.0f))) return EBS_ERR_INVALID_ARG;
+    const int Ho = L.stride == 2 ? L.h_in / 2 : L.h_in, Wo = L.stride == 2 ? L.w_in / 2 : L.w_in;
+    const int Hf = L.k == 3 ? L.h_in + 2 : Ho + 2, Wf = L.k == 3 ? L.w_in + 2 : Wo + 2;
+    const int tiles = (Hf * Wf + UMMA_M - 1) / UMMA_M, co16 = (L.c_out + 15) & ~15, cw = (L.c_in + 31) >> 5;
+    if (tiles * UMMA_M + 2 * Wf + 2 > strip_cap(L.c_in)) return EBS_ERR_UNSUPPORTED;          // rows the MMAs read
+    if (L.dst >= 0 && !L.hold && (Ho + 2) * (Wo + 2) + Wo + 3 > strip_cap(L.c_out)) return EBS_ERR_UNSUPPORTED;   // rows written
+    if ((L.hold ? FUSED_HOLD_COL : 0) + tiles * (co16 > 32 ? co16 : 32) > (L.hold ? 512 : FUSED_HOLD_COL)) return EBS_ERR_UNSUPPORTED;
+    if (L.k * L.k * cw * co16 * 32 > FUSED_W_BYTES) return EBS_ERR_UNSUPPORTED;
+    if (L.dst < 0 && Ho * Wo * L.c_out * 4 > FUSED_ACT_BYTES) return EBS_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(L.w8) & 15u) != 0) return EBS_ERR_INVALID_ARG;
+    return EBS_OK;
+}
+
+int fused_plan_upload(const void* layers_host, int n_layers, void* layers_dev, cudaStream_t st) {
+    const FusedLayer* L = static_cast<const FusedLayer*>(layers_host);
+    for (int i = 0; i < n_layers; ++i) {
+        const int rc = check_layer(L[i], i > 0 ? &L[i - 1] : nullptr);
+        if (rc) return rc;
+    }
+    if (L[0].c_in > 4 || L[0].src != 0) return EBS_ERR_UNSUPPORTED;                   // the image goes to strip 0, <= 4 channels
+    if (L[n_layers - 1].dst != -1 || L[n_layers - 1].c_out > 64) return EBS_ERR_INVALID_ARG;
+    return check_cuda(cudaMemcpyAsync(layers_dev, layers_host, (size_t)n_layers * sizeof(FusedLayer), cudaMemcpyHostToDevice, st));
+}
+
+int launch_fused_resnet(const uint8_t* images, int n, int img_h, int img_w, const void* layers_dev, int n_layers,
+                        const void* head_host, float* logits, uint8_t* trace, long long trace_stride, cudaStream_t st) {
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        if (check_cuda(cudaFuncSetAttribute(fused_resnet_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FUSED_SMEM)))
+            return EBS_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    FusedHead head;
+    memcpy(&head, head_host, sizeof(head));
+    fused_resnet_kernel<<<n, FUSED_THREADS, FUSED_SMEM, st>>>(images, img_h, img_w, static_cast<const FusedLayer*>(layers_dev),
+                                                               n_layers, head, logits, trace, trace_stride);
+    return check_cuda(cudaGetLastError());
+}
+
+unsigned long long fused_net_timeouts() {
+    unsigned long long v = 0;
+    cudaMemcpyFromSymbol(&v, g_umma_timeouts, sizeof(v));
+    return v;
+}
+
+int fused_layer_bytes() { return (int)sizeof(FusedLayer); }
+int fused_head_bytes() { return (int)sizeof(FusedHead); }
+
+}  // namespace ebs

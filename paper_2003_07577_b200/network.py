@@ -182,3 +182,87 @@ def calibrated_plans(layers, weight_codes, images_u8_nhwc: torch.Tensor, device=
     run(fc, pq, s_fc, 0, relu=False)
     torch.cuda.synchronize(device)
     return [plans[L.name] for L in layers]
+
+
+class FusedBasicBlockNet:
+    """The same network as BasicBlockNet through ebs_resnet_cifar_forward: one launch per batch, one thread
+    block per image, activations resident in shared memory.  Built from the same ConvPlan list."""
+
+    def __init__(self, plans: List[ConvPlan], device=None, trace: bool = False):
+        self.device = torch.device("cuda:0") if device is None else device
+        self.plans = plans
+        first, fc = plans[0], plans[-1]
+        by_name = {p.name: p for p in plans}
+        blocks = [(p, by_name[p.name[:-2] + "c2"], by_name.get(p.name[:-2] + "ds")) for p in plans[1:-1]
+                  if p.name.endswith("c1")]
+        self._keep = []
+        self.trace_offsets: Dict[str, int] = {}
+        trace_bytes = 0
+
+        def record(p: ConvPlan, src, dst, *, res=0, res_buf=0, res_step=0.0, hold=0, zero_dst=0, relu=1, last=False):
+            nonlocal trace_bytes
+            d = p.desc
+            ho, wo = ebs.ebs_conv_out_shape(d, p.h_in, p.w_in)
+            off = -1
+            if trace and not hold and not last:
+                off = trace_bytes
+                self.trace_offsets[p.name] = off
+                trace_bytes += ho * wo * d.c_out
+            S = torch.tensor(d.w_scale, dtype=torch.float32) * torch.tensor(d.a_scale, dtype=torch.float32)
+            inv = float(torch.tensor(1.0, dtype=torch.float32) / torch.tensor(p.out_step, dtype=torch.float32)) if p.out_bits else 0.0
+            self._keep.append((p.packed_w, p.ch_scale, p.ch_bias))
+            return ebs.ebs_fused_layer(
+                p.packed_w.data_ptr() + ebs.ebs_packed_weight_plane_bytes(d),
+                None if p.ch_scale is None else p.ch_scale.data_ptr(), None if p.ch_bias is None else p.ch_bias.data_ptr(),
+                d.c_in, d.c_out, d.kh, d.stride_h, p.h_in, p.w_in, src, -1 if last else dst, res, relu, p.out_bits, hold,
+                zero_dst, off, float(S), inv, float(res_step), res_buf)
+
+        X, T, XS = 1, 2, 0
+        layers = [record(first, 0, X)]
+        x_step = first.out_step
+        for bi, (c1, c2, ds) in enumerate(blocks):
+            last = bi == len(blocks) - 1
+            if ds is not None:
+                layers.append(record(c1, X, T, zero_dst=1))
+                layers.append(record(ds, X, XS, hold=1, relu=0))
+                layers.append(record(c2, T, X, res=2, zero_dst=1, last=last))
+            else:
+                layers.append(record(c1, X, T))
+                layers.append(record(c2, T, X, res=1, res_buf=X, res_step=x_step, last=last))
+            x_step = c2.out_step
+        self.n_layers = len(layers)
+        self.layers_dev = torch.empty(self.n_layers * ctypes_sizeof(ebs.ebs_fused_layer), dtype=torch.uint8, device=self.device)
+        ebs.ebs_fused_plan_upload(layers, self.layers_dev)
+        fd = fc.desc
+        S_fc = torch.tensor(fd.w_scale, dtype=torch.float32) * torch.tensor(fd.a_scale, dtype=torch.float32)
+        a_inv = torch.tensor(1.0, dtype=torch.float32) / torch.tensor(fd.a_scale, dtype=torch.float32)
+        self.head = ebs.ebs_fused_head(fc.packed_w.data_ptr() + ebs.ebs_packed_weight_plane_bytes(fd),
+                                       None if fc.ch_scale is None else fc.ch_scale.data_ptr(),
+                                       None if fc.ch_bias is None else fc.ch_bias.data_ptr(), fd.c_in, fd.c_out,
+                                       float(a_inv), float(S_fc))
+        self.classes = fd.c_out
+        self.img_h, self.img_w = first.h_in, first.w_in
+        self.trace_bytes = trace_bytes
+        self._logits = None
+        self._trace = None
+
+    def forward(self, images_u8_nhwc: torch.Tensor, stream=None) -> torch.Tensor:
+        n = images_u8_nhwc.shape[0]
+        if self._logits is None or self._logits.shape[0] != n:
+            self._logits = torch.empty((n, self.classes), dtype=torch.float32, device=self.device)
+            self._trace = (torch.zeros((n, self.trace_bytes), dtype=torch.uint8, device=self.device)
+                           if self.trace_bytes else None)
+        ebs.ebs_resnet_cifar_forward(images_u8_nhwc, n, self.img_h, self.img_w, self.layers_dev, self.n_layers,
+                                     self.head, self._logits, self._trace, self.trace_bytes, stream=stream)
+        return self._logits
+
+    def traced_codes(self, name: str, plan: ConvPlan) -> torch.Tensor:
+        """Output codes of layer `name` of the last forward pass, uint8 [N, Ho, Wo, C] (trace=True only)."""
+        ho, wo = ebs.ebs_conv_out_shape(plan.desc, plan.h_in, plan.w_in)
+        off = self.trace_offsets[name]
+        return self._trace[:, off: off + ho * wo * plan.desc.c_out].reshape(-1, ho, wo, plan.desc.c_out)
+
+
+def ctypes_sizeof(t) -> int:
+    import ctypes
+    return ctypes.sizeof(t)

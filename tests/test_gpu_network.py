@@ -177,3 +177,47 @@ def test_resnet20_forward_matches_the_oracle(ebs, U, oracle, gen):
     assert np.array_equal(logits[sample].cpu().numpy(), logits_ref)
     assert np.unique(logits_ref.argmax(axis=1)).size >= 1 and np.isfinite(logits_ref).all()
     assert ebs.ebs_device_wait_timeouts() == 0
+
+
+def test_fused_network_kernel_matches_the_oracle(ebs, U, oracle, gen):
+    """The one-launch whole-network kernel: every layer's codes (trace) and the logits of the sampled
+    images equal the oracle's chain bit for bit, and the logits equal the layer-by-layer run's for all images."""
+    from paper_2003_07577_b200.network import FusedBasicBlockNet
+    n = 40
+    sample = [0, 17, 39]
+    specs = gen.resnet20_network(0, n)
+    imgs = gen.images_u8(0, n)
+    plan, trace, logits_ref, _ = _oracle_network(oracle, gen, specs, imgs, sample)
+    net = _gpu_network(ebs, U, gen, specs, plan)
+    fused = FusedBasicBlockNet(net.plans, U.dev(), trace=True)
+    x = _to(imgs.astype(np.uint8).transpose(0, 2, 3, 1), U)
+    for _ in range(2):
+        logits = fused.forward(x)
+        torch.cuda.synchronize()
+    assert ebs.ebs_device_wait_timeouts() == 0
+    by_name = {p.name: p for p in net.plans}
+    for spec in specs:
+        name, q_ref = spec.layer.name, trace[spec.layer.name]
+        if q_ref is None or name not in fused.trace_offsets:
+            continue
+        got = fused.traced_codes(name, by_name[name])[sample].cpu().numpy().transpose(0, 3, 1, 2)
+        assert np.array_equal(got, q_ref), f"{name} W{spec.w_bits}A{spec.a_bits}"
+    assert np.array_equal(logits[sample].cpu().numpy(), logits_ref)
+    layerwise = net.forward(x)
+    torch.cuda.synchronize()
+    assert np.array_equal(logits.cpu().numpy(), layerwise.cpu().numpy())
+
+
+def test_fused_network_plan_is_validated(ebs, U):
+    from paper_2003_07577_b200 import binding
+    d = U.desc_for(3, 16, 3, 1, 1, 8, 8)
+    pw = torch.zeros(ebs.ebs_packed_weight_bytes(d) // 4, dtype=torch.int32, device=U.dev())
+    w8 = pw.data_ptr() + ebs.ebs_packed_weight_plane_bytes(d)
+    ok = binding.ebs_fused_layer(w8, None, None, 3, 16, 3, 1, 16, 16, 0, -1, 0, 1, 0, 0, 0, -1, 0.01, 0.0, 0.0, 0)
+    dev = torch.empty(4096, dtype=torch.uint8, device=U.dev())
+    ebs.ebs_fused_plan_upload([ok], dev)
+    for field, value in (("k", 5), ("c_out", 128), ("h_in", 64), ("src", 1), ("dst", 1)):
+        bad = binding.ebs_fused_layer.from_buffer_copy(ok)
+        setattr(bad, field, value)
+        with pytest.raises(RuntimeError):
+            ebs.ebs_fused_plan_upload([bad], dev)
