@@ -26,7 +26,7 @@
 
 namespace ebs {
 
-constexpr int FUSED_THREADS = 256;
+constexpr int FUSED_THREADS = 512;
 constexpr int FUSED_ACT_PIX = 1360;                    // pixels an activation strip holds (34 x 34 frame + halo, 128-row tiles)
 constexpr int FUSED_ACT_BYTES = FUSED_ACT_PIX * 32;    // one 32-channel word
 constexpr int FUSED_W_BYTES = 37 * 1024;               // largest weight image (3x3 64->64)
@@ -40,6 +40,13 @@ __device__ __forceinline__ uint8_t* strip_ptr(uint8_t* acts, int buf) { return a
 // A strip holds one 32-channel word of up to 1360 frame pixels or two words of up to 680: pixels per word.
 __host__ __device__ inline int strip_cap(int channels) { return channels > 32 ? FUSED_ACT_PIX / 2 : FUSED_ACT_PIX; }
 
+#ifdef EBS_FUSED_TRACE
+__device__ long long g_fused_clk[72][4];
+#define FUSED_CLK(li, k) do { if (blockIdx.x == 0 && tid == 0) g_fused_clk[li][k] = clock64(); } while (0)
+#else
+#define FUSED_CLK(li, k) do { } while (0)
+#endif
+
 __global__ void __launch_bounds__(FUSED_THREADS, 1)
 fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, const FusedLayer* __restrict__ layers,
                     int n_layers, const FusedHead head, float* __restrict__ logits, uint8_t* __restrict__ trace,
@@ -49,6 +56,9 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int fc_codes[64];
+    __shared__ float s_cs[64], s_cb[64], s_pcs[64], s_pcb[64];    // per-channel terms of the layer / of the held projection
+    __shared__ float s_proj_S;
+    __shared__ int s_proj_flags;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int img = blockIdx.x;
@@ -104,6 +114,7 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
     float* pool_scratch = reinterpret_cast<float*>(strip_ptr(acts, 0));      // [pixels][c_out] of the last layer
 
     for (int li = 0; li < n_layers && ok; ++li) {
+        FUSED_CLK(li, 0);
         const FusedLayer L = layers[li];
         const int cw = (L.c_in + 31) >> 5, co16 = (L.c_out + 15) & ~15;
         const int Ho = L.stride == 2 ? L.h_in / 2 : L.h_in, Wo = L.stride == 2 ? L.w_in / 2 : L.w_in;
@@ -113,12 +124,24 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
         const int tiles = (frame + UMMA_M - 1) / UMMA_M;
         const int acc_stride = co16 > 32 ? co16 : 32;
         const int col0 = L.hold ? FUSED_HOLD_COL : 0;
+
         const int Wp_out = Wo + 2;                                 // frame of the destination strip
         const int cap_in = strip_cap(L.c_in), cap_out = strip_cap(L.c_out);   // pixels per word of the strips read / written
         uint8_t* src_strip = strip_ptr(acts, L.src);
         uint8_t* dst_strip = L.dst >= 0 ? strip_ptr(acts, L.dst) : nullptr;
 
         if (tid == 0 && li + 1 < n_layers) fetch_weights(li + 1);  // its buffer was last read by layer li-1, finished
+        if (tid < 64) {                                            // per-channel terms -> shared memory (read by every row)
+            const bool in = tid < L.c_out;
+            s_cs[tid] = (L.ch_scale && in) ? __ldg(L.ch_scale + tid) : 1.0f;
+            s_cb[tid] = (L.ch_bias && in) ? __ldg(L.ch_bias + tid) : 0.0f;
+            if (L.res == 2) {
+                const FusedLayer& P = layers[li - 1];              // the projection whose accumulators are held
+                s_pcs[tid] = (P.ch_scale && in) ? __ldg(P.ch_scale + tid) : 1.0f;
+                s_pcb[tid] = (P.ch_bias && in) ? __ldg(P.ch_bias + tid) : 0.0f;
+                if (tid == 0) { s_proj_S = P.S; s_proj_flags = (P.ch_scale ? 1 : 0) | (P.ch_bias ? 2 : 0); }
+            }
+        }
 
         if (L.k == 1) {
             // projection: its input is the stride-2 subsample of strip src, copied into strip dst in the output frame
@@ -141,24 +164,24 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
         __syncthreads();
 
         // ---- MMAs of the whole layer
+        FUSED_CLK(li, 1);
         if (!mbar_wait_bounded(&w_bar[li & 1], (uint32_t)((li >> 1) & 1), abortp)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
         if (tid == 0) {
             const uint32_t idesc = umma_idesc_i8(co16);
             const uint8_t* a_src = L.k == 1 ? dst_strip : src_strip;   // the projection reads its subsampled copy
             const uint32_t a_base = smem_u32(a_src), b_base = smem_u32(wbuf + (li & 1) * FUSED_W_BYTES);
-            for (int t = 0; t < tiles; ++t) {
-                const uint32_t tmem_d = tmem_base + (uint32_t)(col0 + t * acc_stride);
-                int first = 1;
-                for (int wd = 0; wd < cw; ++wd) {
-                    for (int tap = 0; tap < L.k * L.k; ++tap) {
-                        const int r = tap / L.k, s = tap - r * L.k;
-                        const int shift = L.k == 3 ? r * Wf + s : Wf + 1;    // 1x1: the centre of the output frame
+            // consecutive MMAs go to different accumulator tiles: an MMA that accumulates onto the previous one's
+            // result waits for it (about 200 cycles), independent ones pipeline
+            for (int wd = 0; wd < cw; ++wd) {
+                for (int tap = 0; tap < L.k * L.k; ++tap) {
+                    const int r = tap / L.k, s = tap - r * L.k;
+                    const int shift = L.k == 3 ? r * Wf + s : Wf + 1;    // 1x1: the centre of the output frame
+                    const uint64_t db = umma_desc_sw32(b_base + (tap * cw + wd) * co16 * 32);
+                    for (int t = 0; t < tiles; ++t) {
                         const uint64_t da = umma_desc_interleaved(a_base + wd * cap_in * 32 + (t * UMMA_M + shift) * 16,
                                                                   (uint32_t)(cap_in * 16));
-                        const uint64_t db = umma_desc_sw32(b_base + (tap * cw + wd) * co16 * 32);
-                        umma_i8(tmem_d, da, db, idesc, first ? 0u : 1u);
-                        first = 0;
+                        umma_i8(tmem_base + (uint32_t)(col0 + t * acc_stride), da, db, idesc, (wd | tap) != 0 ? 1u : 0u);
                     }
                 }
             }
@@ -167,13 +190,16 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
         if (!mbar_wait_bounded(&mma_bar, (uint32_t)(mma_phase & 1), abortp)) { ok = false; break; }
         ++mma_phase;
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        FUSED_CLK(li, 2);
 
         // ---- epilogue (a held projection has none: the next layer reads its accumulators)
         if (!L.hold) {
-            const FusedLayer P = L.res == 2 ? layers[li - 1] : L;   // the projection whose accumulators are held
             const int qmax = (1 << L.out_bits) - 1;
             const int quarter = warp & 3;
-            for (int t = warp >> 2; t < tiles; t += 2) {
+            const bool has_cs = L.ch_scale != nullptr, has_cb = L.ch_bias != nullptr;
+            const bool p_cs = s_proj_flags & 1, p_cb = s_proj_flags & 2;
+            const float S = L.S, inv_step = L.out_inv_step, res_step = L.res_step, PS = s_proj_S;
+            for (int t = warp >> 2; t < tiles; t += FUSED_THREADS / 128) {
                 const int f = t * UMMA_M + quarter * 32 + lane;
                 const int hp = f / Wf, wp = f - hp * Wf;
                 // does this frame row have an output, and where does it go in the destination frame
@@ -185,64 +211,65 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
                 const bool in_frame = f < frame && (L.stride == 1 || valid);   // stride 1 also writes the zeros of the padding
                 const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(col0 + t * acc_stride);
                 const uint32_t prow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(FUSED_HOLD_COL + t * acc_stride);
+                uint32_t w8v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};        // the pixel's 32-channel word being assembled
+                uint32_t resw[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};      // the identity shortcut's word at the same pixel
 #pragma unroll 1
-                for (int c0 = 0; c0 < co16; c0 += 32) {
-                    int q[32];
-                    uint32_t res_lo[4] = {0, 0, 0, 0}, res_hi[4] = {0, 0, 0, 0};
-                    if (L.res == 1 && valid) {
+                for (int c0 = 0; c0 < co16; c0 += 16) {
+                    const int lane0 = (c0 & 16) >> 3;                    // byte lane of channels c0 .. c0+7 in words 0..7
+                    if (L.res == 1 && valid && (c0 & 16) == 0) {
                         const uint8_t* rp = strip_ptr(acts, L.res_buf) + (c0 >> 5) * cap_out * 32 + target * 16;
                         const uint4 a = *reinterpret_cast<const uint4*>(rp), b = *reinterpret_cast<const uint4*>(rp + cap_out * 16);
-                        res_lo[0] = a.x; res_lo[1] = a.y; res_lo[2] = a.z; res_lo[3] = a.w;
-                        res_hi[0] = b.x; res_hi[1] = b.y; res_hi[2] = b.z; res_hi[3] = b.w;
+                        resw[0] = a.x; resw[1] = a.y; resw[2] = a.z; resw[3] = a.w;
+                        resw[4] = b.x; resw[5] = b.y; resw[6] = b.z; resw[7] = b.w;
                     }
+                    uint32_t v[16], pv[16];
+                    tmem_ld16(trow + (uint32_t)c0, v);                  // whole warp, also for rows without an output
+                    if (L.res == 2) tmem_ld16(prow + (uint32_t)c0, pv);
+                    int q[16];
 #pragma unroll
-                    for (int hf = 0; hf < 2; ++hf) {
-                        uint32_t v[16], pv[16];
-                        if (c0 + 16 * hf < co16) tmem_ld16(trow + (uint32_t)(c0 + 16 * hf), v);
-                        else {
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) v[e] = 0u;
+                    for (int e = 0; e < 16; ++e) {
+                        const int c = c0 + e;
+                        float y = __fmul_rn((float)(int)v[e], S);
+                        if (has_cs) y = __fmul_rn(y, s_cs[c]);
+                        if (has_cb) y = __fadd_rn(y, s_cb[c]);
+                        if (L.res == 2) {                           // projection shortcut: its own scale and per-channel terms
+                            float r = __fmul_rn((float)(int)pv[e], PS);
+                            if (p_cs) r = __fmul_rn(r, s_pcs[c]);
+                            if (p_cb) r = __fadd_rn(r, s_pcb[c]);
+                            y = __fadd_rn(y, r);
                         }
-                        if (L.res == 2 && c0 + 16 * hf < co16) tmem_ld16(prow + (uint32_t)(c0 + 16 * hf), pv);
+                        if (L.res == 1)                             // identity shortcut: channel 8 i + k is byte i of word k
+                            y = __fadd_rn(y, __fmul_rn(res_step, (float)((resw[e & 7] >> (8 * (lane0 + (e >> 3)))) & 0xFFu)));
+                        if (L.relu && !(y > 0.0f)) y = 0.0f;
+                        int code = 0;
+                        if (valid && c < L.c_out) {
+                            if (L.dst < 0) pool_scratch[(ho * Wo + wo) * L.c_out + c] = y;
+                            else code = min(__float2int_rd(__fadd_rn(__fmul_rn(y, inv_step), 0.5f)), qmax);
+                        }
+                        q[e] = code;
+                    }
+                    if (L.dst >= 0) {
+                        // word k of the pixel = channels k, 8+k, 16+k, 24+k as bytes (negative codes saturate to 0)
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            const int c = c0 + 16 * hf + e;
-                            float y = __fmul_rn((float)(int)v[e], L.S);
-                            if (c < L.c_out) {
-                                if (L.ch_scale) y = __fmul_rn(y, __ldg(L.ch_scale + c));
-                                if (L.ch_bias) y = __fadd_rn(y, __ldg(L.ch_bias + c));
-                                if (L.res == 2) {                   // projection shortcut: its own scale and per-channel terms
-                                    float r = __fmul_rn((float)(int)pv[e], P.S);
-                                    if (P.ch_scale) r = __fmul_rn(r, __ldg(P.ch_scale + c));
-                                    if (P.ch_bias) r = __fadd_rn(r, __ldg(P.ch_bias + c));
-                                    y = __fadd_rn(y, r);
-                                }
-                                if (L.res == 1) {                   // identity shortcut: byte (c / 8) of word (c % 8)
-                                    const int cc = c & 31, k8 = cc & 7;
-                                    const uint32_t wv = k8 < 4 ? res_lo[k8] : res_hi[k8 - 4];
-                                    y = __fadd_rn(y, __fmul_rn(L.res_step, (float)((wv >> (8 * (cc >> 3))) & 0xFFu)));
+                        for (int k8 = 0; k8 < 8; ++k8) {
+                            uint32_t two;
+                            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;\n" : "=r"(two) : "r"(q[8 + k8]), "r"(q[k8]), "r"(0));
+                            w8v[k8] |= two << (8 * lane0);
+                        }
+                        if (((c0 & 16) != 0 || c0 + 16 >= co16)) {
+                            if (in_frame) {
+                                uint8_t* wp_ = dst_strip + (c0 >> 5) * cap_out * 32 + target * 16;
+                                *reinterpret_cast<uint4*>(wp_) = make_uint4(w8v[0], w8v[1], w8v[2], w8v[3]);
+                                *reinterpret_cast<uint4*>(wp_ + cap_out * 16) = make_uint4(w8v[4], w8v[5], w8v[6], w8v[7]);
+                                if (trace && L.trace_off >= 0 && valid) {
+                                    uint8_t* tp = trace + (size_t)img * trace_stride + L.trace_off + (size_t)(ho * Wo + wo) * L.c_out;
+                                    const int cb = c0 & ~31;
+                                    for (int cc = 0; cc < 32 && cb + cc < L.c_out; ++cc)
+                                        tp[cb + cc] = (uint8_t)((w8v[cc & 7] >> (8 * (cc >> 3))) & 0xFFu);
                                 }
                             }
-                            if (L.relu && !(y > 0.0f)) y = 0.0f;
-                            int code = 0;
-                            if (valid && c < L.c_out) {
-                                if (L.dst < 0) pool_scratch[(ho * Wo + wo) * L.c_out + c] = y;
-                                else code = quantize_act_code(y, L.out_inv_step, qmax);
-                            }
-                            q[16 * hf + e] = code;
-                        }
-                    }
-                    if (L.dst >= 0 && in_frame) {
-                        // word k of the pixel = channels k, 8+k, 16+k, 24+k as bytes
-                        uint32_t w8v[8];
 #pragma unroll
-                        for (int k8 = 0; k8 < 8; ++k8) w8v[k8] = pack_sat_u8x4(q[k8], q[8 + k8], q[16 + k8], q[24 + k8]);
-                        uint8_t* wp_ = dst_strip + (c0 >> 5) * cap_out * 32 + target * 16;
-                        *reinterpret_cast<uint4*>(wp_) = make_uint4(w8v[0], w8v[1], w8v[2], w8v[3]);
-                        *reinterpret_cast<uint4*>(wp_ + cap_out * 16) = make_uint4(w8v[4], w8v[5], w8v[6], w8v[7]);
-                        if (trace && L.trace_off >= 0 && valid) {
-                            uint8_t* tp = trace + (size_t)img * trace_stride + L.trace_off + (size_t)(ho * Wo + wo) * L.c_out + c0;
-                            for (int e = 0; e < 32 && c0 + e < L.c_out; ++e) tp[e] = (uint8_t)q[e];
+                            for (int k8 = 0; k8 < 8; ++k8) w8v[k8] = 0u;
                         }
                     }
                 }
@@ -254,6 +281,7 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     }
 
+    FUSED_CLK(n_layers, 0);
     // ---- pooling, 8-bit quantization, classifier
     if (ok && !abort_flag && n_layers > 0) {
         const FusedLayer L = layers[n_layers - 1];
@@ -351,3 +379,7 @@ int fused_layer_bytes() { return (int)sizeof(FusedLayer); }
 int fused_head_bytes() { return (int)sizeof(FusedHead); }
 
 }  // namespace ebs
+
+#ifdef EBS_FUSED_TRACE
+extern "C" void ebs_debug_fused_clk(long long* out) { cudaMemcpyFromSymbol(out, ebs::g_fused_clk, sizeof(ebs::g_fused_clk)); }
+#endif
