@@ -26,7 +26,7 @@
 
 namespace ebs {
 
-constexpr int FUSED_THREADS = 512;
+constexpr int FUSED_THREADS = 640;
 constexpr int FUSED_ACT_PIX = 1360;                    // pixels an activation strip holds (34 x 34 frame + halo, 128-row tiles)
 constexpr int FUSED_ACT_BYTES = FUSED_ACT_PIX * 32;    // one 32-channel word
 constexpr int FUSED_W_BYTES = 37 * 1024;               // largest weight image (3x3 64->64)
@@ -199,7 +199,10 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
             const bool has_cs = L.ch_scale != nullptr, has_cb = L.ch_bias != nullptr;
             const bool p_cs = s_proj_flags & 1, p_cb = s_proj_flags & 2;
             const float S = L.S, inv_step = L.out_inv_step, res_step = L.res_step, PS = s_proj_S;
-            for (int t = warp >> 2; t < tiles; t += FUSED_THREADS / 128) {
+            // a unit of work is (tile, 16 channels); the four warps of a TMEM lane quarter take units in turn
+            const int nb16 = co16 >> 4, units = tiles * nb16;
+            for (int u = warp >> 2; u < units; u += FUSED_THREADS / 128) {
+                const int t = u / nb16, c0 = (u - t * nb16) << 4;
                 const int f = t * UMMA_M + quarter * 32 + lane;
                 const int hp = f / Wf, wp = f - hp * Wf;
                 // does this frame row have an output, and where does it go in the destination frame
@@ -211,66 +214,55 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
                 const bool in_frame = f < frame && (L.stride == 1 || valid);   // stride 1 also writes the zeros of the padding
                 const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(col0 + t * acc_stride);
                 const uint32_t prow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(FUSED_HOLD_COL + t * acc_stride);
-                uint32_t w8v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};        // the pixel's 32-channel word being assembled
+                const int lane0 = (c0 & 16) >> 3;                        // byte lane of channels c0 .. c0+7 in words 0..7
                 uint32_t resw[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};      // the identity shortcut's word at the same pixel
-#pragma unroll 1
-                for (int c0 = 0; c0 < co16; c0 += 16) {
-                    const int lane0 = (c0 & 16) >> 3;                    // byte lane of channels c0 .. c0+7 in words 0..7
-                    if (L.res == 1 && valid && (c0 & 16) == 0) {
-                        const uint8_t* rp = strip_ptr(acts, L.res_buf) + (c0 >> 5) * cap_out * 32 + target * 16;
-                        const uint4 a = *reinterpret_cast<const uint4*>(rp), b = *reinterpret_cast<const uint4*>(rp + cap_out * 16);
-                        resw[0] = a.x; resw[1] = a.y; resw[2] = a.z; resw[3] = a.w;
-                        resw[4] = b.x; resw[5] = b.y; resw[6] = b.z; resw[7] = b.w;
+                if (L.res == 1 && valid) {
+                    const uint8_t* rp = strip_ptr(acts, L.res_buf) + (c0 >> 5) * cap_out * 32 + target * 16;
+                    const uint4 a = *reinterpret_cast<const uint4*>(rp), b = *reinterpret_cast<const uint4*>(rp + cap_out * 16);
+                    resw[0] = a.x; resw[1] = a.y; resw[2] = a.z; resw[3] = a.w;
+                    resw[4] = b.x; resw[5] = b.y; resw[6] = b.z; resw[7] = b.w;
+                }
+                uint32_t v[16], pv[16];
+                tmem_ld16(trow + (uint32_t)c0, v);                      // whole warp, also for rows without an output
+                if (L.res == 2) tmem_ld16(prow + (uint32_t)c0, pv);
+                int q[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const int c = c0 + e;
+                    float y = __fmul_rn((float)(int)v[e], S);
+                    if (has_cs) y = __fmul_rn(y, s_cs[c]);
+                    if (has_cb) y = __fadd_rn(y, s_cb[c]);
+                    if (L.res == 2) {                               // projection shortcut: its own scale and per-channel terms
+                        float r = __fmul_rn((float)(int)pv[e], PS);
+                        if (p_cs) r = __fmul_rn(r, s_pcs[c]);
+                        if (p_cb) r = __fadd_rn(r, s_pcb[c]);
+                        y = __fadd_rn(y, r);
                     }
-                    uint32_t v[16], pv[16];
-                    tmem_ld16(trow + (uint32_t)c0, v);                  // whole warp, also for rows without an output
-                    if (L.res == 2) tmem_ld16(prow + (uint32_t)c0, pv);
-                    int q[16];
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const int c = c0 + e;
-                        float y = __fmul_rn((float)(int)v[e], S);
-                        if (has_cs) y = __fmul_rn(y, s_cs[c]);
-                        if (has_cb) y = __fadd_rn(y, s_cb[c]);
-                        if (L.res == 2) {                           // projection shortcut: its own scale and per-channel terms
-                            float r = __fmul_rn((float)(int)pv[e], PS);
-                            if (p_cs) r = __fmul_rn(r, s_pcs[c]);
-                            if (p_cb) r = __fadd_rn(r, s_pcb[c]);
-                            y = __fadd_rn(y, r);
-                        }
-                        if (L.res == 1)                             // identity shortcut: channel 8 i + k is byte i of word k
-                            y = __fadd_rn(y, __fmul_rn(res_step, (float)((resw[e & 7] >> (8 * (lane0 + (e >> 3)))) & 0xFFu)));
-                        if (L.relu && !(y > 0.0f)) y = 0.0f;
-                        int code = 0;
-                        if (valid && c < L.c_out) {
-                            if (L.dst < 0) pool_scratch[(ho * Wo + wo) * L.c_out + c] = y;
-                            else code = min(__float2int_rd(__fadd_rn(__fmul_rn(y, inv_step), 0.5f)), qmax);
-                        }
-                        q[e] = code;
+                    if (L.res == 1)                                 // identity shortcut: channel 8 i + k is byte i of word k
+                        y = __fadd_rn(y, __fmul_rn(res_step, (float)((resw[e & 7] >> (8 * (lane0 + (e >> 3)))) & 0xFFu)));
+                    if (L.relu && !(y > 0.0f)) y = 0.0f;
+                    int code = 0;
+                    if (valid && c < L.c_out) {
+                        if (L.dst < 0) pool_scratch[(ho * Wo + wo) * L.c_out + c] = y;
+                        else code = min(__float2int_rd(__fadd_rn(__fmul_rn(y, inv_step), 0.5f)), qmax);
                     }
-                    if (L.dst >= 0) {
-                        // word k of the pixel = channels k, 8+k, 16+k, 24+k as bytes (negative codes saturate to 0)
+                    q[e] = code;
+                }
+                if (L.dst >= 0 && in_frame) {
+                    // word k of the pixel holds channels k, 8+k, 16+k, 24+k as bytes: these 16 channels are two
+                    // adjacent bytes of each of the eight words (negative codes saturate to 0)
+                    uint8_t* wp_ = dst_strip + (c0 >> 5) * cap_out * 32 + target * 16 + lane0;
 #pragma unroll
-                        for (int k8 = 0; k8 < 8; ++k8) {
-                            uint32_t two;
-                            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;\n" : "=r"(two) : "r"(q[8 + k8]), "r"(q[k8]), "r"(0));
-                            w8v[k8] |= two << (8 * lane0);
-                        }
-                        if (((c0 & 16) != 0 || c0 + 16 >= co16)) {
-                            if (in_frame) {
-                                uint8_t* wp_ = dst_strip + (c0 >> 5) * cap_out * 32 + target * 16;
-                                *reinterpret_cast<uint4*>(wp_) = make_uint4(w8v[0], w8v[1], w8v[2], w8v[3]);
-                                *reinterpret_cast<uint4*>(wp_ + cap_out * 16) = make_uint4(w8v[4], w8v[5], w8v[6], w8v[7]);
-                                if (trace && L.trace_off >= 0 && valid) {
-                                    uint8_t* tp = trace + (size_t)img * trace_stride + L.trace_off + (size_t)(ho * Wo + wo) * L.c_out;
-                                    const int cb = c0 & ~31;
-                                    for (int cc = 0; cc < 32 && cb + cc < L.c_out; ++cc)
-                                        tp[cb + cc] = (uint8_t)((w8v[cc & 7] >> (8 * (cc >> 3))) & 0xFFu);
-                                }
-                            }
+                    for (int k8 = 0; k8 < 8; ++k8) {
+                        uint32_t two;
+                        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;\n" : "=r"(two) : "r"(q[8 + k8]), "r"(q[k8]), "r"(0));
+                        *reinterpret_cast<uint16_t*>(wp_ + (k8 >> 2) * cap_out * 16 + (k8 & 3) * 4) = (uint16_t)two;
+                    }
+                    if (trace && L.trace_off >= 0 && valid) {
+                        uint8_t* tp = trace + (size_t)img * trace_stride + L.trace_off + (size_t)(ho * Wo + wo) * L.c_out + c0;
 #pragma unroll
-                            for (int k8 = 0; k8 < 8; ++k8) w8v[k8] = 0u;
-                        }
+                        for (int e = 0; e < 16; ++e)
+                            if (c0 + e < L.c_out) tp[e] = (uint8_t)max(q[e], 0);
                     }
                 }
             }
