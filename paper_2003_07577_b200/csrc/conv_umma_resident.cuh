@@ -208,18 +208,21 @@ __global__ void __launch_bounds__(RES_THREADS, 1) conv_umma_resident_kernel(cons
                 if (!mbar_wait_bounded(&a_full[st], (uint32_t)((g >> 1) & 1), abortp)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 if ((tid & 31) == 0) {
+                    // descriptors built once per chunk and advanced by additions: a few instructions per MMA
                     const uint32_t a_base = smem_u32(a_stages + st * a_stage_bytes);
                     const int words = min(KS, p.CW - ch * KS);
+                    const uint64_t da0 = umma_desc_interleaved(a_base, (uint32_t)(SP * 16));
+                    uint64_t db = umma_desc_sw32(b_base + (uint32_t)(ch * KS * taps * B_TILE_BYTES));
+                    uint32_t acc_flag = ch != 0 ? 1u : 0u;
                     for (int q = 0; q < words; ++q) {
-                        const int cw = ch * KS + q;
-                        int t = 0;
-                        for (int r = 0; r < p.kh; ++r)
-                            for (int s = 0; s < p.kw; ++s, ++t) {
-                                const uint64_t da = umma_desc_interleaved(a_base + q * a_word_bytes + (r * Wp + s) * 16,
-                                                                          (uint32_t)(SP * 16));
-                                const uint64_t db = umma_desc_sw32(b_base + (cw * taps + t) * B_TILE_BYTES);
-                                umma_i8(tmem_d, da, db, IDESC, (ch | q | t) != 0 ? 1u : 0u);
+                        uint64_t da_r = da0 + (uint64_t)(q * (a_word_bytes >> 4));
+                        for (int r = 0; r < p.kh; ++r, da_r += (uint64_t)Wp) {
+                            for (int s = 0; s < p.kw; ++s) {
+                                umma_i8(tmem_d, da_r + (uint64_t)s, db, IDESC, acc_flag);
+                                db += (uint64_t)(B_TILE_BYTES >> 4);
+                                acc_flag = 1u;
                             }
+                        }
                     }
                     umma_commit(&a_empty[st]);
                     if (ch == nchunks - 1) umma_commit(&acc_full[buf]);

@@ -244,17 +244,20 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
             STRIP_TRACE(5 + (ch > 0), (tid & 31) == 0);
             if ((tid & 31) == 0) {
+                // the issuing thread is the pipeline stage that feeds the tensor core: descriptors are built once
+                // and advanced by additions (start addresses are in 16-byte units), a few instructions per MMA
                 const uint32_t a_base = smem_u32(tiles + st * stage_bytes);
-                const uint32_t b_base = a_base + a_stage_bytes;
                 const int words = min(KS, p.CW - ch * KS);
+                const uint64_t da0 = umma_desc_interleaved(a_base, (uint32_t)(SP * 16));
+                uint64_t db = umma_desc_sw32(a_base + a_stage_bytes);
+                uint32_t acc_flag = ch != 0 ? 1u : 0u;
                 for (int q = 0; q < words; ++q) {
-                    int t = 0;
-                    for (int r = 0; r < p.kh; ++r) {
-                        for (int s = 0; s < p.kw; ++s, ++t) {
-                            const uint64_t da = umma_desc_interleaved(a_base + q * a_word_bytes + (r * Wp + s) * 16,
-                                                                      (uint32_t)(SP * 16));
-                            const uint64_t db = umma_desc_sw32(b_base + (q * taps + t) * B_TILE_BYTES);
-                            umma_i8(tmem_base, da, db, IDESC, (ch | q | t) != 0 ? 1u : 0u);
+                    uint64_t da_r = da0 + (uint64_t)(q * (a_word_bytes >> 4));
+                    for (int r = 0; r < p.kh; ++r, da_r += (uint64_t)Wp) {
+                        for (int s = 0; s < p.kw; ++s) {
+                            umma_i8(tmem_base, da_r + (uint64_t)s, db, IDESC, acc_flag);
+                            db += (uint64_t)(B_TILE_BYTES >> 4);
+                            acc_flag = 1u;
                         }
                     }
                 }

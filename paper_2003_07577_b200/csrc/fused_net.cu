@@ -71,7 +71,7 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
         abort_flag = 0;
         mbar_init(&w_bar[0], 1);
         mbar_init(&w_bar[1], 1);
-        mbar_init(&mma_bar, 1);
+        mbar_init(&mma_bar, 4);                                   // the four issuing threads
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (warp == 0) {
@@ -167,25 +167,34 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
         FUSED_CLK(li, 1);
         if (!mbar_wait_bounded(&w_bar[li & 1], (uint32_t)((li >> 1) & 1), abortp)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-        if (tid == 0) {
-            const uint32_t idesc = umma_idesc_i8(co16);
-            const uint8_t* a_src = L.k == 1 ? dst_strip : src_strip;   // the projection reads its subsampled copy
-            const uint32_t a_base = smem_u32(a_src), b_base = smem_u32(wbuf + (li & 1) * FUSED_W_BYTES);
-            // consecutive MMAs go to different accumulator tiles: an MMA that accumulates onto the previous one's
-            // result waits for it (about 200 cycles), independent ones pipeline
-            for (int wd = 0; wd < cw; ++wd) {
-                for (int tap = 0; tap < L.k * L.k; ++tap) {
-                    const int r = tap / L.k, s = tap - r * L.k;
-                    const int shift = L.k == 3 ? r * Wf + s : Wf + 1;    // 1x1: the centre of the output frame
-                    const uint64_t db = umma_desc_sw32(b_base + (tap * cw + wd) * co16 * 32);
-                    for (int t = 0; t < tiles; ++t) {
-                        const uint64_t da = umma_desc_interleaved(a_base + wd * cap_in * 32 + (t * UMMA_M + shift) * 16,
-                                                                  (uint32_t)(cap_in * 16));
-                        umma_i8(tmem_base + (uint32_t)(col0 + t * acc_stride), da, db, idesc, (wd | tap) != 0 ? 1u : 0u);
+        if (lane == 0 && warp < 4) {
+            // Four threads issue (lane 0 of warps 0-3, tiles dealt round-robin): the issue loop of one thread,
+            // not the tensor core, bounds a layer of many small MMAs.  Descriptors are built once and advanced
+            // by additions (start addresses are in 16-byte units).  Each thread's commit arrives once.
+            if (warp < tiles) {
+                const uint32_t idesc = umma_idesc_i8(co16);
+                const uint8_t* a_src = L.k == 1 ? dst_strip : src_strip;   // the projection reads its subsampled copy
+                const uint64_t da0 = umma_desc_interleaved(smem_u32(a_src), (uint32_t)(cap_in * 16));
+                uint64_t db = umma_desc_sw32(smem_u32(wbuf + (li & 1) * FUSED_W_BYTES));
+                const uint64_t db_step = (uint64_t)((co16 * 32) >> 4), db_word = db_step * (uint64_t)cw;
+                for (int wd = 0; wd < cw; ++wd) {
+                    const uint64_t da_w = da0 + (uint64_t)(wd * cap_in * 2);   // one word = cap_in * 32 bytes
+                    uint64_t db_t = db + db_step * (uint64_t)wd;                // weight tiles are ordered [tap][word]
+                    for (int r = 0; r < L.k; ++r) {
+                        for (int s = 0; s < L.k; ++s, db_t += db_word) {
+                            const int shift = L.k == 3 ? r * Wf + s : Wf + 1;    // 1x1: the centre of the output frame
+                            const uint32_t acc_flag = (wd | r | s) != 0 ? 1u : 0u;
+                            uint64_t da = da_w + (uint64_t)(warp * UMMA_M + shift);
+                            uint32_t tm = tmem_base + (uint32_t)(col0 + warp * acc_stride);
+                            for (int t = warp; t < tiles; t += 4, da += 4 * UMMA_M, tm += 4 * acc_stride)
+                                umma_i8(tm, da, db_t, idesc, acc_flag);
+                        }
                     }
                 }
+                umma_commit(&mma_bar);
+            } else {
+                mbar_arrive(&mma_bar);
             }
-            umma_commit(&mma_bar);
         }
         if (!mbar_wait_bounded(&mma_bar, (uint32_t)(mma_phase & 1), abortp)) { ok = false; break; }
         ++mma_phase;
