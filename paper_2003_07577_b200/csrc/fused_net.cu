@@ -26,7 +26,7 @@
 
 namespace ebs {
 
-constexpr int FUSED_THREADS = 640;
+constexpr int FUSED_THREADS = 768;
 constexpr int FUSED_ACT_PIX = 1360;                    // pixels an activation strip holds (34 x 34 frame + halo, 128-row tiles)
 constexpr int FUSED_ACT_BYTES = FUSED_ACT_PIX * 32;    // one 32-channel word
 constexpr int FUSED_W_BYTES = 37 * 1024;               // largest weight image (3x3 64->64)
