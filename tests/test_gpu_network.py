@@ -179,13 +179,14 @@ def test_resnet20_forward_matches_the_oracle(ebs, U, oracle, gen):
     assert ebs.ebs_device_wait_timeouts() == 0
 
 
-def test_fused_network_kernel_matches_the_oracle(ebs, U, oracle, gen):
-    """The one-launch whole-network kernel: every layer's codes (trace) and the logits of the sampled
-    images equal the oracle's chain bit for bit, and the logits equal the layer-by-layer run's for all images."""
+@pytest.mark.parametrize("blocks,n", [(3, 40), (5, 12)])
+def test_fused_network_kernel_matches_the_oracle(ebs, U, oracle, gen, blocks, n):
+    """The one-launch whole-network kernel (ResNet-20 and ResNet-32): every layer's codes (trace) and the logits
+    of the sampled images equal the oracle's chain bit for bit, and the logits equal the layer-by-layer run's
+    for all images."""
     from paper_2003_07577_b200.network import FusedBasicBlockNet
-    n = 40
-    sample = [0, 17, 39]
-    specs = gen.resnet20_network(0, n)
+    sample = [0, n // 2, n - 1]
+    specs = gen.resnet20_network(0, n) if blocks == 3 else gen.resnet_cifar_network(blocks, 1, n)
     imgs = gen.images_u8(0, n)
     plan, trace, logits_ref, _ = _oracle_network(oracle, gen, specs, imgs, sample)
     net = _gpu_network(ebs, U, gen, specs, plan)

@@ -139,10 +139,20 @@ def binary_ops(spec: LayerSpec, batch: Optional[int] = None) -> int:
     return 2 * n * spec.layer.macs * spec.w_bits * spec.a_bits
 
 
+def resnet_cifar_network(blocks_per_stage: int, seed: int = 0, batch: int = 128) -> List[LayerSpec]:
+    """A CIFAR ResNet (3/5/9 blocks per stage = ResNet-20/32/56) with config2's bitwidth recipe, wired as a
+    network: a projection shortcut takes the activation bitwidth of its block's first convolution."""
+    specs = _draw(seed, resnet_cifar(blocks_per_stage), [1, 2, 3, 4], batch, "uniform")
+    return _share_shortcut_inputs(specs)
+
+
 def resnet20_network(seed: int = 0, batch: int = 128) -> List[LayerSpec]:
     """The ResNet-20 stack of config2 wired as a network: a projection shortcut reads the same
     tensor as its block's first convolution, so it takes that layer's activation bitwidth."""
-    specs = config2(seed, batch)
+    return _share_shortcut_inputs(config2(seed, batch))
+
+
+def _share_shortcut_inputs(specs: List[LayerSpec]) -> List[LayerSpec]:
     by_name = {s.layer.name: s for s in specs}
     out = []
     for s in specs:
