@@ -165,9 +165,8 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
 
         // ---- MMAs of the whole layer
         FUSED_CLK(li, 1);
-        if (!mbar_wait_bounded(&w_bar[li & 1], (uint32_t)((li >> 1) & 1), abortp)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-        if (lane == 0 && warp < 4) {
+        if (lane == 0 && warp < 4 && mbar_wait_bounded(&w_bar[li & 1], (uint32_t)((li >> 1) & 1), abortp)) {
             // Four threads issue (lane 0 of warps 0-3, tiles dealt round-robin): the issue loop of one thread,
             // not the tensor core, bounds a layer of many small MMAs.  Descriptors are built once and advanced
             // by additions (start addresses are in 16-byte units).  Each thread's commit arrives once.
@@ -196,7 +195,10 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
                 mbar_arrive(&mma_bar);
             }
         }
-        if (!mbar_wait_bounded(&mma_bar, (uint32_t)(mma_phase & 1), abortp)) { ok = false; break; }
+        // one warp polls for the MMAs' completion; the others sleep in the block barrier instead of spinning
+        if (warp == 4) mbar_wait_bounded(&mma_bar, (uint32_t)(mma_phase & 1), abortp);
+        __syncthreads();
+        if (abort_flag != 0) { ok = false; break; }
         ++mma_phase;
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
         FUSED_CLK(li, 2);
