@@ -36,6 +36,8 @@ WORKLOADS = {
     "config1": ("config1: one 3x3 conv 64->64, 32x32, batch 1, W2A2, seed 0", lambda: gen.config1(0)),
     "config3": ("config3: ResNet-18 ImageNet-shaped quantized convs, batch 64, (Wb,Ab) in {2..6}^2, seed 0",
                 lambda: gen.config3(0)),
+    "config4": ("config4: 4096^3 bit-plane GEMM as a 1x1 convolution over 64x64 pixels, seven (Wb,Ab) pairs of the sweep, seed 0",
+                lambda: [gen.config4(wb, ab) for wb, ab in [(1, 1), (2, 2), (4, 4), (8, 8), (1, 8), (8, 1), (3, 5)]]),
     "config5": ("config5: ResNet-50 ImageNet-shaped bottleneck stack, batch 256, (Wb,Ab) in {2..8}^2, seed 0 "
                 "(layers run with independent inputs here; the chained run is a parity test)",
                 lambda: gen.config5(0)),
