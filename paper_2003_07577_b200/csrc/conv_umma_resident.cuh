@@ -41,9 +41,9 @@ inline ResidentGeom resident_geometry(const ConvParams& p, int tile_n, int sms) 
     const int taps = p.kh * p.kw;
     g.b_bytes = p.CW * taps * tile_n * 32;
     int ks = g.strip.ks;
-    while (ks > 1 && ks * g.strip.strip_pad * 32 > 24 * 1024) --ks;
+    while (ks > 1 && ks * strip_word_bytes(g.strip.strip_pad) > 24 * 1024) --ks;
     g.strip.ks = ks;
-    g.smem_bytes = g.b_bytes + 2 * ks * g.strip.strip_pad * 32 + 1024;
+    g.smem_bytes = g.b_bytes + 2 * (ks * strip_word_bytes(g.strip.strip_pad) + 256) + 1024;
     const long long frame = (long long)p.N * strip_frame_h(p) * strip_frame_w(p);
     const long long ftiles = (frame + UMMA_M - 1) / UMMA_M;
     const int cotiles = (p.Co + tile_n - 1) / tile_n;
@@ -74,8 +74,8 @@ __global__ void __launch_bounds__(RES_THREADS, 1) conv_umma_resident_kernel(cons
     const int ftiles = (frame + UMMA_M - 1) / UMMA_M;
     const int my_tiles = ((int)blockIdx.x < ftiles) ? (ftiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     const int co0 = blockIdx.y * TILE_N;
-    const int a_word_bytes = SP * 32;
-    const int a_stage_bytes = KS * a_word_bytes;
+    const int a_word_bytes = strip_word_bytes(SP);
+    const int a_stage_bytes = (KS * a_word_bytes + 255) & ~255;
     uint8_t* base = dyn_smem + ((1024u - (smem_u32(dyn_smem) & 1023u)) & 1023u);
     uint8_t* b_tiles = base;                                             // [CW][taps][TILE_N][32]
     uint8_t* a_stages = base + p.CW * taps * B_TILE_BYTES;               // [2][KS][2][SP][16]
@@ -119,8 +119,8 @@ __global__ void __launch_bounds__(RES_THREADS, 1) conv_umma_resident_kernel(cons
 #pragma unroll
         for (int j = 0; j < STRIP_SLOTS; ++j) {
             const int e = tid + j * UMMA_EXPANDERS;
-            const int q = e / S, s = e - q * S;
-            slot_q[j] = q < KS ? q : -1;
+            const int s = e / KS, q = e - s * KS;            // consecutive lanes: consecutive words of one pixel
+            slot_q[j] = s < S ? q : -1;
             slot_pix[j] = s;
             slot_dst[j] = q * a_word_bytes + s * 16;
         }

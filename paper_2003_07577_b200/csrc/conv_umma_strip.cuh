@@ -61,6 +61,10 @@ __host__ __device__ inline bool strip_pointwise(const ConvParams& p) {
 __host__ __device__ inline int strip_frame_h(const ConvParams& p) { return strip_pointwise(p) ? p.Ho : p.H + 2 * p.ph; }
 __host__ __device__ inline int strip_frame_w(const ConvParams& p) { return strip_pointwise(p) ? p.Wo : p.W + 2 * p.pw; }
 
+// Bytes from one reduction word of a strip to the next: two halves of strip_pad x 16 bytes plus 32 bytes, so
+// that the 16-byte stores of lanes that hold consecutive words of one pixel fall into different banks.
+__host__ __device__ inline int strip_word_bytes(int strip_pad) { return strip_pad * 32 + 32; }
+
 // Host-side geometry of a launch (also used by the library to decide whether the kernel applies).
 struct StripGeom {
     int strip_pix;      // pixels of a strip: 128 + (kh-1) * Wp + (kw-1)
@@ -75,13 +79,13 @@ inline StripGeom strip_geometry(const ConvParams& p, int tile_n) {
     g.strip_pix = UMMA_M + (p.kh - 1) * Wp + (p.kw - 1);
     g.strip_pad = (g.strip_pix + 7) & ~7;
     const long long frame = (long long)p.N * strip_frame_h(p) * Wp;
-    const int word_bytes = g.strip_pad * 32 + taps * tile_n * 32;
+    const int word_bytes = strip_word_bytes(g.strip_pad) + taps * tile_n * 32;
     int ks = STRIP_MAX_ITEMS / g.strip_pix;
     if (ks > 4) ks = 4;
     if (ks > p.CW) ks = p.CW;
     while (ks > 1 && ks * word_bytes > 48 * 1024) --ks;
     g.ks = ks;
-    g.smem_bytes = 2 * ks * word_bytes + 1024 + g.strip_pad * 4;
+    g.smem_bytes = 2 * (ks * word_bytes + 256) + 1024 + g.strip_pad * 4;
     g.ok = ((p.sh == 1 && p.sw == 1) || strip_pointwise(p)) && ks >= 1 && g.strip_pix <= STRIP_MAX_ITEMS && taps <= 64 &&
            g.smem_bytes <= 200 * 1024 && frame < (1LL << 31) - 256 && g.strip_pad * 16 < (1 << 18);
     return g;
@@ -114,8 +118,8 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
     const int frame = p.N * Hp * Wp;                          // outputs are numbered in the padded input frame
     const int f0 = blockIdx.x * UMMA_M;
     const int co0 = blockIdx.y * TILE_N;
-    const int a_word_bytes = SP * 32;                         // one reduction word of the strip: two halves of SP x 16 B
-    const int a_stage_bytes = KS * a_word_bytes;
+    const int a_word_bytes = strip_word_bytes(SP);            // one reduction word of the strip: two halves of SP x 16 B (+ skew)
+    const int a_stage_bytes = (KS * a_word_bytes + 255) & ~255;   // the weight tiles behind it keep their 256-byte alignment
     const int stage_bytes = a_stage_bytes + KS * taps * B_TILE_BYTES;
     uint8_t* tiles = dyn_smem + ((1024u - (smem_u32(dyn_smem) & 1023u)) & 1023u);
     int* csum_s = reinterpret_cast<int*>(tiles + 2 * stage_bytes);      // per strip pixel: sum of its codes (w_levels)
@@ -150,13 +154,13 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
 #pragma unroll
         for (int j = 0; j < STRIP_SLOTS; ++j) {
             const int e = tid + j * UMMA_EXPANDERS;
-            const int q = e / S, s = e - q * S;
-            slot_q[j] = q < KS ? q : -1;                      // -1: no item
+            const int s = e / KS, q = e - s * KS;            // consecutive lanes: consecutive words of one pixel (contiguous in memory)
+            slot_q[j] = s < S ? q : -1;                       // -1: no item
             slot_pix[j] = s;
             slot_dst[j] = q * a_word_bytes + s * 16;
             slot_off[j] = -1;                                 // -1: padding or past the batch -> zero bytes
             const int f = f0 + s;
-            if (q < KS && f < frame) {
+            if (s < S && f < frame) {
                 const int n = f / (Hp * Wp), rem = f - n * (Hp * Wp);
                 const int hp = rem / Wp, wp = rem - hp * Wp;
                 const int h = pointwise ? hp * p.sh : hp - p.ph, w = pointwise ? wp * p.sw : wp - p.pw;

@@ -108,7 +108,7 @@ def strip_variant_applies(d, w, tile_n):
         return False
     strip = 128 + (d.kh - 1) * (w + 2 * d.pad_w) + d.kw - 1
     pad = (strip + 7) // 8 * 8
-    return strip <= 512 and 2 * (pad * 32 + d.kh * d.kw * tile_n * 32) + 1024 + pad * 4 <= 200 * 1024
+    return strip <= 512 and 2 * (pad * 32 + 32 + d.kh * d.kw * tile_n * 32 + 256) + 1024 + pad * 4 <= 200 * 1024
 
 
 def resident_variant_applies(d, w, tile_n):
