@@ -182,7 +182,8 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
     }
     constexpr int STRIP_BASE = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS;
     constexpr int RES_BASE = STRIP_BASE + NUM_CONV_STRIP_VARIANTS;
-    if (variant >= RES_BASE + NUM_CONV_RESIDENT_VARIANTS) return EBS_ERR_INVALID_ARG;
+    constexpr int MS_BASE = RES_BASE + NUM_CONV_RESIDENT_VARIANTS;
+    if (variant >= MS_BASE + NUM_CONV_MMA_STRIP_VARIANTS) return EBS_ERR_INVALID_ARG;
 
     ConvParams p;
     memset(&p, 0, sizeof(p));
@@ -218,16 +219,22 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
         if (strip >= 0 && p.CW * d->kh * d->kw >= 8 && conv_umma_resident_applies(p, strip)) variant = RES_BASE + strip;
         else if (strip >= 0) variant = STRIP_BASE + strip;
         else if (umma >= 0) variant = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + umma;
+        // wide images with few channels and several activation planes: the warp-level strip kernel (its time does
+        // not grow with the plane count, the per-tap kernel's does)
+        else if (mma_ok && p.Co <= 16 && d->a_bits >= 3 && p.P >= (1 << 16) && conv_mma_strip_applies(p, 0)) variant = MS_BASE;
         else variant = mma_ok ? NUM_CONV_VARIANTS + choose_mma_variant(d->w_bits, d->a_bits, p.P, p.Co, sm_count())
                               : choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
     }
     if (variant >= NUM_CONV_VARIANTS && !mma_ok) return EBS_ERR_UNSUPPORTED;
-    if (variant >= RES_BASE) {
+    if (variant >= MS_BASE) {
+        if (!conv_mma_strip_applies(p, variant - MS_BASE)) return EBS_ERR_UNSUPPORTED;
+    } else if (variant >= RES_BASE) {
         if (!conv_umma_resident_applies(p, variant - RES_BASE)) return EBS_ERR_UNSUPPORTED;
     } else if (variant >= STRIP_BASE && !conv_umma_strip_applies(p, variant - STRIP_BASE)) {
         return EBS_ERR_UNSUPPORTED;
     }
     const ConvVariant* v =
+        variant >= MS_BASE ? conv_mma_strip_variant(d->a_bits, variant - MS_BASE) :
         variant >= RES_BASE ? conv_umma_resident_variant(d->a_bits, variant - RES_BASE) :
         variant >= STRIP_BASE ? conv_umma_strip_variant(d->a_bits, variant - STRIP_BASE) :
         variant >= NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS
@@ -325,7 +332,7 @@ int ebs_conv2d_mixed(const void* packed_x_dev, int n, int h, int w, const void* 
 
 int ebs_num_conv_variants(void) {
     return NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS + NUM_CONV_STRIP_VARIANTS +
-           NUM_CONV_RESIDENT_VARIANTS;
+           NUM_CONV_RESIDENT_VARIANTS + NUM_CONV_MMA_STRIP_VARIANTS;
 }
 
 long long ebs_device_wait_timeouts(void) { return (long long)conv_umma_timeouts(); }

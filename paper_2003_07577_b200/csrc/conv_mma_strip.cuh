@@ -1,0 +1,250 @@
+// Warp-level int8 MMA convolution for small stride-1 layers with every input pixel expanded ONCE per CTA.
+//
+// conv_mma_kernel rebuilds the activation fragments from the packed bits for every filter tap (two integer
+// instructions per plane and register, kh*kw times per pixel) and the weight fragments in every warp.  Here a
+// CTA owns TILE_P consecutive pixels of the zero-padded input frame (the numbering of conv_umma_strip_kernel:
+// for stride 1 a filter tap is a constant shift), expands the strip TILE_P + (kh-1) Wp + (kw-1) of pixels into
+// BYTES in shared memory once (32-byte rows per pixel and 32-channel word, byte 4b+i = channel 8i+b, the two
+// 16-byte halves swapped when (pixel >> 2) & 1 so that fragment loads are bank-conflict free), copies the weight
+// rows of its channel tile from the byte image that ebs_pack_weights appends (all taps and words: a few KB),
+// and then only loads fragments: a0/a1 = bytes 4tq..4tq+3 of rows g and g+8, a2/a3 = bytes 16+4tq.. -- one
+// 32-bit shared load per fragment register per tap.  The whole reduction of a layer fits in shared memory
+// (c_in <= 128), so there is no staging pipeline.  Layers with at most 16 (8) input channels use only byte
+// lanes 0-1 (0) of every register; there two (four) taps share one MMA step, the later tap's registers
+// shifted left by 16 (8, 16, 24) bits, for both operands alike.
+// Epilogue as in conv_mma_kernel (accumulator pairs, fp32 steps, code tile, multiply-gather pack), with the
+// output pixel of a frame row looked up in a per-CTA table (rows with hp >= Ho or wp >= Wo have none).
+#pragma once
+
+#include "conv_mma.cuh"
+#include "conv_umma_strip.cuh"   // frame helpers (strip_pointwise, strip_frame_h/w)
+
+namespace ebs {
+
+struct MmaStripGeom {
+    int strip_pix, strip_pad, smem_bytes, fold;
+    bool ok;
+};
+inline MmaStripGeom mma_strip_geometry(const ConvParams& p, int tile_p, int tile_c) {
+    MmaStripGeom g{};
+    const int Wp = strip_frame_w(p), taps = p.kh * p.kw;
+    g.strip_pix = tile_p + (p.kh - 1) * Wp + (p.kw - 1);
+    g.strip_pad = (g.strip_pix + 7) & ~7;
+    const int cin = p.CW == 1 ? p.fold_bits : 32;                 // fold_bits >= c_in for folded layers
+    g.fold = (p.CW == 1 && cin <= 8) ? 4 : ((p.CW == 1 && cin <= 16) ? 2 : 1);
+    const long long frame = (long long)p.N * strip_frame_h(p) * Wp;
+    g.smem_bytes = p.CW * g.strip_pad * 32 + taps * p.CW * tile_c * 32 + tile_p * code_row_bytes(tile_c) + tile_p * 4 + 128;
+    g.ok = ((p.sh == 1 && p.sw == 1) || strip_pointwise(p)) && p.CW <= 4 && taps * p.CW <= 64 && !p.w_levels &&
+           !p.residual && !p.res_packed && !p.y_nchw && (p.Co & 1) == 0 && p.fold <= 4 &&
+           g.smem_bytes <= 96 * 1024 && frame < (1LL << 31) - 4096;
+    return g;
+}
+
+template <int AB, int MT, int NT, int WARPS_P, int WARPS_C>
+__global__ void __launch_bounds__(32 * WARPS_P * WARPS_C)
+conv_mma_strip_kernel(const ConvParams p) {
+    constexpr int NTH = 32 * WARPS_P * WARPS_C, TILE_P = 16 * MT * WARPS_P, TILE_C = 8 * NT * WARPS_C;
+    constexpr int ROWB = code_row_bytes(TILE_C);
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, tq = lane & 3;
+    const int wp_ = warp % WARPS_P, wc = warp / WARPS_P;
+    const int S = p.strip_pix, SP = (S + 7) & ~7, taps = p.kh * p.kw;
+    const bool pointwise = strip_pointwise(p);
+    const int Wp = strip_frame_w(p), Hp = strip_frame_h(p);
+    const int frame = p.N * Hp * Wp;
+    const int f0 = blockIdx.x * TILE_P, co0 = blockIdx.y * TILE_C;
+    uint8_t* strip = smem_raw;                                       // [CW][SP][32]
+    uint8_t* wimg = strip + p.CW * SP * 32;                          // [taps * CW][TILE_C][32]
+    uint8_t* out_s = wimg + taps * p.CW * TILE_C * 32;               // [TILE_P][ROWB] requantized codes
+    int* gp_s = reinterpret_cast<int*>(out_s + TILE_P * ROWB);       // output pixel of every frame row, -1: none
+
+    // ---- output pixel of each row of the tile
+    for (int pl = tid; pl < TILE_P; pl += NTH) {
+        const int f = f0 + pl;
+        int gp = -1;
+        if (f < frame) {
+            const int n = f / (Hp * Wp), rem = f - n * (Hp * Wp);
+            const int hp = rem / Wp, wq = rem - hp * Wp;
+            if (hp < p.Ho && wq < p.Wo) gp = (n * p.Ho + hp) * p.Wo + wq;
+        }
+        gp_s[pl] = gp;
+    }
+    // ---- weight rows of this channel tile, all taps and words (rows past c_out are zero in the image)
+    for (int e = tid; e < taps * p.CW * TILE_C * 2; e += NTH) {
+        const int half = e & 1, row = (e >> 1) % TILE_C, kk = (e >> 1) / TILE_C;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (co0 + row < p.Co16) v = __ldg(reinterpret_cast<const uint4*>(p.w8 + ((size_t)kk * p.Co16 + co0 + row) * 32) + half);
+        reinterpret_cast<uint4*>(wimg + (kk * TILE_C + row) * 32)[half] = v;
+    }
+    // ---- the strip: packed words -> bytes, once per pixel and word
+    for (int e = tid; e < S * p.CW; e += NTH) {
+        const int s = e / p.CW, cw = e - s * p.CW;
+        const int f = f0 + s;
+        uint32_t r[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+        if (f < frame) {
+            const int n = f / (Hp * Wp), rem = f - n * (Hp * Wp);
+            const int hp = rem / Wp, wq = rem - hp * Wp;
+            const int h = pointwise ? hp * p.sh : hp - p.ph, w = pointwise ? wq * p.sw : wq - p.pw;
+            if ((unsigned)h < (unsigned)p.H && (unsigned)w < (unsigned)p.W) {
+                uint32_t words[AB];
+                load_words_global<AB>(p.x + (((size_t)(n * p.H + h) * p.W + w) * p.CW + cw) * AB, words);
+#pragma unroll
+                for (int k = 0; k < AB; ++k) {
+                    const uint32_t mask = 0x01010101u << k;
+#pragma unroll
+                    for (int b = 0; b < 8; ++b) r[b] |= __funnelshift_r(words[k], words[k], b - k) & mask;
+                }
+            }
+        }
+        uint4* dst = reinterpret_cast<uint4*>(strip + (cw * SP + s) * 32);
+        const int sw = (s >> 2) & 1;
+        dst[sw] = make_uint4(r[0], r[1], r[2], r[3]);
+        dst[sw ^ 1] = make_uint4(r[4], r[5], r[6], r[7]);
+    }
+    __syncthreads();
+
+    // ---- main loop: fragments are plain shared loads
+    int acc[MT][NT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0;
+
+    const int fold = p.strip_ks;                                     // taps per MMA step: 1, 2 or 4 (set by the launcher)
+    const int fshift = 32 / fold;                                    // bits a folded tap is shifted by
+    for (int cw = 0; cw < p.CW; ++cw) {
+        const uint8_t* strip_w = strip + cw * SP * 32;
+        for (int t0 = 0; t0 < taps; t0 += fold) {
+            uint32_t af[MT][4], bf[NT][2];
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) af[mt][0] = af[mt][1] = af[mt][2] = af[mt][3] = 0u;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) bf[nt][0] = bf[nt][1] = 0u;
+            for (int ft = 0; ft < fold && t0 + ft < taps; ++ft) {
+                const int t = t0 + ft, r = t / p.kw, s = t - r * p.kw;
+                const int shift = r * Wp + s, sh = ft * fshift;
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    const int pix0 = (wp_ * MT + mt) * 16 + g + shift, pix1 = pix0 + 8;
+                    const int x0 = ((pix0 >> 2) & 1) << 4, x1 = ((pix1 >> 2) & 1) << 4;
+                    const uint8_t* r0 = strip_w + pix0 * 32;
+                    const uint8_t* r1 = strip_w + pix1 * 32;
+                    af[mt][0] |= *reinterpret_cast<const uint32_t*>(r0 + ((4 * tq) ^ x0)) << sh;
+                    af[mt][1] |= *reinterpret_cast<const uint32_t*>(r1 + ((4 * tq) ^ x1)) << sh;
+                    af[mt][2] |= *reinterpret_cast<const uint32_t*>(r0 + ((16 + 4 * tq) ^ x0)) << sh;
+                    af[mt][3] |= *reinterpret_cast<const uint32_t*>(r1 + ((16 + 4 * tq) ^ x1)) << sh;
+                }
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int row = (wc * NT + nt) * 8 + g;
+                    const int xb = (((co0 + row) >> 2) & 1) << 4;     // the image swaps the halves of these rows
+                    const uint8_t* wr = wimg + ((t * p.CW + cw) * TILE_C + row) * 32;
+                    bf[nt][0] |= *reinterpret_cast<const uint32_t*>(wr + ((4 * tq) ^ xb)) << sh;
+                    bf[nt][1] |= *reinterpret_cast<const uint32_t*>(wr + ((16 + 4 * tq) ^ xb)) << sh;
+                }
+            }
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) mma_u8s8(acc[mt][nt], af[mt], bf[nt][0], bf[nt][1]);
+        }
+    }
+
+    // ---- epilogue.  Fragment element e of (mt, nt): tile row (e >> 1) * 8 + g, channel 2 * tq + (e & 1).
+    const bool want_y = p.y != nullptr, want_q = p.packed_next != nullptr;
+    const int qmax = (1 << p.next_bits) - 1;
+    float cs[NT][2], cb[NT][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
+        const bool in = co < p.Co;                                  // c_out is even: co + 1 exists with co
+        cs[nt][0] = (p.ch_scale && in) ? __ldg(p.ch_scale + co) : 1.0f;
+        cs[nt][1] = (p.ch_scale && in) ? __ldg(p.ch_scale + co + 1) : 1.0f;
+        cb[nt][0] = (p.ch_bias && in) ? __ldg(p.ch_bias + co) : 0.0f;
+        cb[nt][1] = (p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : 0.0f;
+    }
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int pl = (wp_ * MT + mt) * 16 + half * 8 + g;
+            const int gp = gp_s[pl];
+            const bool pvalid = gp >= 0;
+            const size_t row_o = (size_t)(pvalid ? gp : 0) * p.Co + co0 + wc * NT * 8 + 2 * tq;
+            uint8_t* code_row = out_s + pl * ROWB + wc * NT * 8 + 2 * tq;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
+                const int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
+                const bool valid = pvalid && co < p.Co;
+                int code0 = 0, code1 = 0;
+                if (valid && p.acc) *reinterpret_cast<int2*>(p.acc + row_o + nt * 8) = make_int2(a0, a1);
+                if (want_y || want_q) {
+                    float y0 = __fmul_rn((float)a0, p.S), y1 = __fmul_rn((float)a1, p.S);
+                    if (p.ch_scale) { y0 = __fmul_rn(y0, cs[nt][0]); y1 = __fmul_rn(y1, cs[nt][1]); }
+                    if (p.ch_bias) { y0 = __fadd_rn(y0, cb[nt][0]); y1 = __fadd_rn(y1, cb[nt][1]); }
+                    if (p.relu) { y0 = y0 > 0.0f ? y0 : 0.0f; y1 = y1 > 0.0f ? y1 : 0.0f; }
+                    if (valid && want_y) *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
+                    if (valid && want_q) {
+                        code0 = quantize_act_code(y0, p.inv_next, qmax);
+                        code1 = quantize_act_code(y1, p.inv_next, qmax);
+                    }
+                }
+                if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
+            }
+        }
+    }
+    if (want_q) {
+        __syncthreads();
+        constexpr int CWL = (TILE_C + 31) / 32;
+        constexpr int NW = TILE_C >= 32 ? 8 : TILE_C / 4;           // code words per 32-channel group
+        for (int item = tid; item < TILE_P * CWL; item += NTH) {
+            const int cwl = item / TILE_P, pl = item - cwl * TILE_P;
+            const int gp = gp_s[pl], cwg = (co0 >> 5) + cwl;
+            if (gp < 0 || cwg >= p.CWo) continue;
+            const uint32_t* row = reinterpret_cast<const uint32_t*>(out_s + pl * ROWB + cwl * 32);
+            uint32_t codes[NW];
+#pragma unroll
+            for (int k = 0; k < NW; ++k) codes[k] = row[k];
+            uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + cwg) * p.next_bits;
+            for (int j = 0; j < p.next_bits; ++j) {
+                uint32_t word = 0u;
+#pragma unroll
+                for (int k = 0; k < NW; ++k) {
+                    const uint32_t t = (codes[k] >> j) & 0x01010101u;
+                    word |= ((t * 0x01020408u) >> 24) << (4 * k);
+                }
+                dst[j] = word;
+            }
+        }
+    }
+}
+
+template <int AB, int MT, int NT, int WARPS_P, int WARPS_C>
+void launch_conv_mma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st) {
+    constexpr int TILE_P = 16 * MT * WARPS_P, TILE_C = 8 * NT * WARPS_C;
+    ConvParams p = p0;
+    const MmaStripGeom g = mma_strip_geometry(p, TILE_P, TILE_C);
+    if (!g.ok) return;                                        // callers check mma_strip_geometry first
+    p.strip_pix = g.strip_pix;
+    p.strip_ks = g.fold;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        cudaFuncSetAttribute(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             96 * 1024);
+        attr_set[dev] = true;
+    }
+    const long long frame = (long long)p.N * strip_frame_h(p) * strip_frame_w(p);
+    const dim3 grid((unsigned)((frame + TILE_P - 1) / TILE_P), (unsigned)((p.Co + TILE_C - 1) / TILE_C), 1);
+    conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C><<<grid, 32 * WARPS_P * WARPS_C, g.smem_bytes, st>>>(p);
+}
+
+// Variants: channel tile 16 / 32 / 64, 256 frame pixels per CTA (8 warps).
+constexpr int NUM_MMA_STRIP_VARIANTS = 3;
+
+}  // namespace ebs

@@ -64,7 +64,10 @@ EBS_DECLARE_WB(5) EBS_DECLARE_WB(6) EBS_DECLARE_WB(7) EBS_DECLARE_WB(8)
 #undef EBS_DECLARE_WB
 
 // 5th-generation tensor-core kernels (conv_umma_w1.cu .. conv_umma_w8.cu); variant = log2(tile_n / 16).
-enum { NUM_CONV_UMMA_VARIANTS = 5, NUM_CONV_STRIP_VARIANTS = 5, NUM_CONV_RESIDENT_VARIANTS = 5 };
+enum { NUM_CONV_UMMA_VARIANTS = 5, NUM_CONV_STRIP_VARIANTS = 5, NUM_CONV_RESIDENT_VARIANTS = 5, NUM_CONV_MMA_STRIP_VARIANTS = 3 };
+// Warp-level strip kernel for small stride-1 layers (conv_mma_strip.cu): channel tile 16 / 32 / 64.
+const ConvVariant* conv_mma_strip_variant(int a_bits, int variant);
+bool conv_mma_strip_applies(const ConvParams& p, int variant);
 // Persistent weight-resident strip kernel (conv_umma_resident.cu): variants by channel tile 16 << variant.
 const ConvVariant* conv_umma_resident_variant(int a_bits, int variant);
 bool conv_umma_resident_applies(const ConvParams& p, int variant);

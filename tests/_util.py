@@ -96,8 +96,9 @@ def run_conv(qa, qw, d, epi=None, want_acc=True, want_y=False, next_bits=0, vari
     return out
 
 
-N_STRIP = 5       # variants n-10 .. n-6: the strip kernels
-N_RESIDENT = 5    # variants n-5 .. n-1: the persistent weight-resident strip kernels
+N_STRIP = 5       # variants 24 .. 28: the strip kernels
+N_RESIDENT = 5    # variants 29 .. 33: the persistent weight-resident strip kernels
+N_MMA_STRIP = 3   # variants 34 .. 36: the warp-level strip kernels (channel tile 16, 32, 64)
 
 
 def strip_variant_applies(d, w, tile_n):
@@ -119,13 +120,28 @@ def resident_variant_applies(d, w, tile_n):
             and cw * d.kh * d.kw * tile_n * 32 <= 150 * 1024)
 
 
+def mma_strip_variant_applies(d, w, variant):
+    """Host-side rule of the warp-level strip kernel (plain or per-channel epilogue only: callers that pass a
+    shortcut or ask for NCHW output must not force it)."""
+    pointwise = d.kh == 1 and d.kw == 1 and d.pad_h == 0 and d.pad_w == 0
+    if (d.stride_h != 1 or d.stride_w != 1) and not pointwise:
+        return False
+    tile_p, tile_c = ((256, 16), (256, 32), (128, 64))[variant]
+    cw, taps = (d.c_in + 31) // 32, d.kh * d.kw
+    strip = tile_p + (d.kh - 1) * (w + 2 * d.pad_w) + d.kw - 1
+    pad = (strip + 7) // 8 * 8
+    smem = cw * pad * 32 + taps * cw * tile_c * 32 + tile_p * (tile_c + 4) + tile_p * 4 + 128
+    return (cw <= 4 and taps * cw <= 64 and not d.w_levels and d.c_out % 2 == 0 and d.c_in > 4 and smem <= 96 * 1024)
+
+
 def all_variants(d, w=16):
     """Every kernel variant that applies to descriptor d on images of width w (-1 = the library's own choice)."""
     n = ebs.ebs_num_conv_variants()
-    base = n - N_STRIP - N_RESIDENT
+    base = n - N_STRIP - N_RESIDENT - N_MMA_STRIP
     strip = [base + i for i in range(N_STRIP) if strip_variant_applies(d, w, 16 << i)]
     resident = [base + N_STRIP + i for i in range(N_RESIDENT) if resident_variant_applies(d, w, 16 << i)]
-    return list(range(-1, base)) + strip + resident
+    mma_strip = [base + N_STRIP + N_RESIDENT + i for i in range(N_MMA_STRIP) if mma_strip_variant_applies(d, w, i)]
+    return list(range(-1, base)) + strip + resident + mma_strip
 
 
 def rand_codes(rng, shape, bits, signed):

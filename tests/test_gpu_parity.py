@@ -104,6 +104,36 @@ def test_conv_all_bitwidth_pairs(ebs, U, oracle, wb, ab):
         assert np.array_equal(got, ref), f"variant {variant}"
 
 
+@pytest.mark.parametrize("ab", range(1, 9))
+@pytest.mark.parametrize("c,co,k", [(40, 22, 3), (16, 16, 3), (8, 12, 3), (64, 64, 1), (100, 34, 3)])
+def test_warp_level_strip_kernel_all_activation_bitwidths(ebs, U, oracle, ab, c, co, k):
+    """The warp-level strip variants (channel tile 16 / 32 / 64): every activation bitwidth, ragged channel tiles,
+    one, two and four taps per MMA step (c_in 40 / 16 / 8), with and without per-channel terms and packed output."""
+    rng = np.random.default_rng(100 * ab + c + co)
+    wb = 1 + (ab + c) % 8
+    pad = k // 2
+    qa = U.rand_codes(rng, (3, c, 13, 11), ab, False)
+    qw = U.rand_codes(rng, (co, c, k, k), wb, True)
+    d = U.desc_for(c, co, k, 1, pad, wb, ab, 0.03, 0.05)
+    ref = oracle.conv2d_codes(qa, qw, (1, 1), (pad, pad))
+    S = oracle.combined_scale(0.03, 0.05)
+    cs = rng.uniform(0.5, 2.0, co).astype(np.float32)
+    cb = rng.uniform(-0.3, 0.3, co).astype(np.float32)
+    to = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(U.dev())
+    px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
+    for epi, (ecs, ecb) in ((ebs.epilogue(relu=True, next_a_bits=3, next_a_scale=0.6), (None, None)),
+                            (ebs.epilogue(to(cs), to(cb), None, True, 3, 0.6), (cs, cb))):
+        y_ref, q_ref = oracle.epilogue(ref, S, ecs, ecb, None, relu=True, next_bits=3,
+                                       inv_next=np.float32(1.0) / np.float32(0.6))
+        for variant in (34, 35, 36):
+            if not U.mma_strip_variant_applies(d, 11, variant - 34) or (variant == 34 and co > 16):
+                continue                                      # 16-channel tiles cannot write packed words of wider layers
+            out = U.run_conv(qa, qw, d, epi, want_acc=True, want_y=True, next_bits=3, variant=variant, px=px, pw=pw)
+            assert np.array_equal(out["acc"], ref), f"variant {variant}"
+            assert np.array_equal(out["y"], y_ref), f"variant {variant}"
+            assert np.array_equal(oracle.unpack_acts(out["packed"], co), q_ref), f"variant {variant}"
+
+
 GEOMS = [
     # c_in, c_out, k, stride, pad, h, w
     (3, 16, 3, 1, 1, 32, 32), (3, 8, 7, 2, 3, 30, 29), (16, 16, 3, 1, 1, 17, 9), (16, 32, 1, 2, 0, 16, 16),
@@ -131,9 +161,11 @@ def test_strip_kernel_refuses_strided_layers(ebs, U):
     d = U.desc_for(32, 32, 3, 2, 1, 2, 2)
     qa, qw = np.zeros((1, 32, 8, 8), np.int32), np.zeros((32, 32, 3, 3), np.int32)
     with pytest.raises(RuntimeError):
-        U.run_conv(qa, qw, d, variant=ebs.ebs_num_conv_variants() - 6)
+        U.run_conv(qa, qw, d, variant=28)
     with pytest.raises(RuntimeError):
-        U.run_conv(qa, qw, d, variant=ebs.ebs_num_conv_variants() - 1)
+        U.run_conv(qa, qw, d, variant=33)
+    with pytest.raises(RuntimeError):
+        U.run_conv(qa, qw, d, variant=36)
 
 
 @pytest.mark.parametrize("c,co,k,s,pad,h,n,wb,ab", [(32, 64, 3, 1, 1, 30, 48, 2, 3), (64, 48, 1, 2, 0, 40, 64, 4, 2),
@@ -149,7 +181,7 @@ def test_persistent_kernel_walks_several_tiles_per_cta(ebs, U, oracle, c, co, k,
                                    inv_next=np.float32(1.0) / np.float32(0.9))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
     epi = ebs.epilogue(relu=True, next_a_bits=4, next_a_scale=0.9)
-    nv = ebs.ebs_num_conv_variants()
+    nv = ebs.ebs_num_conv_variants() - U.N_MMA_STRIP
     ran = 0
     for variant in range(nv - U.N_RESIDENT, nv):
         if not U.resident_variant_applies(d, h, 16 << (variant - (nv - U.N_RESIDENT))):
