@@ -219,9 +219,9 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
         if (strip >= 0 && p.CW * d->kh * d->kw >= 8 && conv_umma_resident_applies(p, strip)) variant = RES_BASE + strip;
         else if (strip >= 0) variant = STRIP_BASE + strip;
         else if (umma >= 0) variant = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + umma;
-        // wide images with few channels and several activation planes: the warp-level strip kernel (its time does
-        // not grow with the plane count, the per-tap kernel's does)
-        else if (mma_ok && p.Co <= 16 && d->a_bits >= 3 && p.P >= (1 << 16) && conv_mma_strip_applies(p, 0)) variant = MS_BASE;
+        // wide images with few channels: the warp-level strip kernel (its time does not grow with the plane count,
+        // and it expands every input pixel once instead of once per tap)
+        else if (mma_ok && p.Co <= 16 && p.P >= (1 << 16) && conv_mma_strip_applies(p, 0)) variant = MS_BASE;
         else variant = mma_ok ? NUM_CONV_VARIANTS + choose_mma_variant(d->w_bits, d->a_bits, p.P, p.Co, sm_count())
                               : choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
     }

@@ -16,6 +16,8 @@
 // output pixel of a frame row looked up in a per-CTA table (rows with hp >= Ho or wp >= Wo have none).
 #pragma once
 
+#include <type_traits>
+
 #include "conv_mma.cuh"
 #include "conv_umma_strip.cuh"   // frame helpers (strip_pointwise, strip_frame_h/w)
 
@@ -58,26 +60,20 @@ conv_mma_strip_kernel(const ConvParams p) {
     uint8_t* wimg = strip + p.CW * SP * 32;                          // [taps * CW][TILE_C][32]
     uint8_t* out_s = wimg + taps * p.CW * TILE_C * 32;               // [TILE_P][ROWB] requantized codes
     int* gp_s = reinterpret_cast<int*>(out_s + TILE_P * ROWB);       // output pixel of every frame row, -1: none
-
-    // ---- output pixel of each row of the tile
-    for (int pl = tid; pl < TILE_P; pl += NTH) {
-        const int f = f0 + pl;
-        int gp = -1;
-        if (f < frame) {
-            const int n = f / (Hp * Wp), rem = f - n * (Hp * Wp);
-            const int hp = rem / Wp, wq = rem - hp * Wp;
-            if (hp < p.Ho && wq < p.Wo) gp = (n * p.Ho + hp) * p.Wo + wq;
-        }
-        gp_s[pl] = gp;
-    }
-    // ---- weight rows of this channel tile, all taps and words (rows past c_out are zero in the image)
+    // ---- weight rows of this channel tile, all taps and words (rows past c_out are zero in the image): asynchronous
+    // copies issued first, so that their latency hides behind the tables and the strip expansion
     for (int e = tid; e < taps * p.CW * TILE_C * 2; e += NTH) {
         const int half = e & 1, row = (e >> 1) % TILE_C, kk = (e >> 1) / TILE_C;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (co0 + row < p.Co16) v = __ldg(reinterpret_cast<const uint4*>(p.w8 + ((size_t)kk * p.Co16 + co0 + row) * 32) + half);
-        reinterpret_cast<uint4*>(wimg + (kk * TILE_C + row) * 32)[half] = v;
+        const bool valid = co0 + row < p.Co16;
+        const uint8_t* src = valid ? p.w8 + ((size_t)kk * p.Co16 + co0 + row) * 32 + half * 16 : p.w8;
+        cp_async_bytes(wimg + (kk * TILE_C + row) * 32 + half * 16, src, 16, valid);
     }
+    cp_async_commit();
+    __shared__ int tap_shift_s[64];                                   // frame shift r * Wp + s of every tap
+    for (int t = tid; t < taps; t += NTH) tap_shift_s[t] = (t / p.kw) * Wp + (t % p.kw);
+
     // ---- the strip: packed words -> bytes, once per pixel and word
+#pragma unroll 2
     for (int e = tid; e < S * p.CW; e += NTH) {
         const int s = e / p.CW, cw = e - s * p.CW;
         const int f = f0 + s;
@@ -102,6 +98,18 @@ conv_mma_strip_kernel(const ConvParams p) {
         dst[sw] = make_uint4(r[0], r[1], r[2], r[3]);
         dst[sw ^ 1] = make_uint4(r[4], r[5], r[6], r[7]);
     }
+    // ---- output pixel of each row of the tile
+    for (int pl = tid; pl < TILE_P; pl += NTH) {
+        const int f = f0 + pl;
+        int gp = -1;
+        if (f < frame) {
+            const int n = f / (Hp * Wp), rem = f - n * (Hp * Wp);
+            const int hp = rem / Wp, wq = rem - hp * Wp;
+            if (hp < p.Ho && wq < p.Wo) gp = (n * p.Ho + hp) * p.Wo + wq;
+        }
+        gp_s[pl] = gp;
+    }
+    cp_async_wait<0>();
     __syncthreads();
 
     // ---- main loop: fragments are plain shared loads
@@ -113,45 +121,57 @@ conv_mma_strip_kernel(const ConvParams p) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0;
 
-    const int fold = p.strip_ks;                                     // taps per MMA step: 1, 2 or 4 (set by the launcher)
-    const int fshift = 32 / fold;                                    // bits a folded tap is shifted by
-    for (int cw = 0; cw < p.CW; ++cw) {
-        const uint8_t* strip_w = strip + cw * SP * 32;
-        for (int t0 = 0; t0 < taps; t0 += fold) {
-            uint32_t af[MT][4], bf[NT][2];
+    // taps per MMA step (1, 2 or 4, set by the launcher) as a compile-time constant of the loop body, so that the
+    // fragment loads of a step are independent instructions the scheduler can overlap
+    auto reduce = [&](auto fold_tag) {
+        constexpr int FOLD = decltype(fold_tag)::value;
+        constexpr int FSHIFT = 32 / FOLD;                              // bits a folded tap is shifted by
+        const int arow0 = (wp_ * MT) * 16 + g;
+        for (int cw = 0; cw < p.CW; ++cw) {
+            const uint8_t* strip_w = strip + cw * SP * 32;
+#pragma unroll 1
+            for (int t0 = 0; t0 < taps; t0 += FOLD) {
+                uint32_t af[MT][4], bf[NT][2];
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt) af[mt][0] = af[mt][1] = af[mt][2] = af[mt][3] = 0u;
+                for (int mt = 0; mt < MT; ++mt) af[mt][0] = af[mt][1] = af[mt][2] = af[mt][3] = 0u;
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) bf[nt][0] = bf[nt][1] = 0u;
-            for (int ft = 0; ft < fold && t0 + ft < taps; ++ft) {
-                const int t = t0 + ft, r = t / p.kw, s = t - r * p.kw;
-                const int shift = r * Wp + s, sh = ft * fshift;
+                for (int nt = 0; nt < NT; ++nt) bf[nt][0] = bf[nt][1] = 0u;
 #pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    const int pix0 = (wp_ * MT + mt) * 16 + g + shift, pix1 = pix0 + 8;
-                    const int x0 = ((pix0 >> 2) & 1) << 4, x1 = ((pix1 >> 2) & 1) << 4;
-                    const uint8_t* r0 = strip_w + pix0 * 32;
-                    const uint8_t* r1 = strip_w + pix1 * 32;
-                    af[mt][0] |= *reinterpret_cast<const uint32_t*>(r0 + ((4 * tq) ^ x0)) << sh;
-                    af[mt][1] |= *reinterpret_cast<const uint32_t*>(r1 + ((4 * tq) ^ x1)) << sh;
-                    af[mt][2] |= *reinterpret_cast<const uint32_t*>(r0 + ((16 + 4 * tq) ^ x0)) << sh;
-                    af[mt][3] |= *reinterpret_cast<const uint32_t*>(r1 + ((16 + 4 * tq) ^ x1)) << sh;
+                for (int ft = 0; ft < FOLD; ++ft) {
+                    const int t = t0 + ft;
+                    if (t < taps) {
+                        const int shift = tap_shift_s[t];
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt) {
+                            const int pix0 = arow0 + mt * 16 + shift, pix1 = pix0 + 8;
+                            const int x0 = ((pix0 >> 2) & 1) << 4, x1 = ((pix1 >> 2) & 1) << 4;
+                            const uint8_t* r0 = strip_w + pix0 * 32;
+                            const uint8_t* r1 = strip_w + pix1 * 32;
+                            af[mt][0] |= *reinterpret_cast<const uint32_t*>(r0 + ((4 * tq) ^ x0)) << (ft * FSHIFT);
+                            af[mt][1] |= *reinterpret_cast<const uint32_t*>(r1 + ((4 * tq) ^ x1)) << (ft * FSHIFT);
+                            af[mt][2] |= *reinterpret_cast<const uint32_t*>(r0 + ((16 + 4 * tq) ^ x0)) << (ft * FSHIFT);
+                            af[mt][3] |= *reinterpret_cast<const uint32_t*>(r1 + ((16 + 4 * tq) ^ x1)) << (ft * FSHIFT);
+                        }
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            const int row = (wc * NT + nt) * 8 + g;
+                            const int xb = (((co0 + row) >> 2) & 1) << 4;     // the image swaps the halves of these rows
+                            const uint8_t* wr = wimg + ((t * p.CW + cw) * TILE_C + row) * 32;
+                            bf[nt][0] |= *reinterpret_cast<const uint32_t*>(wr + ((4 * tq) ^ xb)) << (ft * FSHIFT);
+                            bf[nt][1] |= *reinterpret_cast<const uint32_t*>(wr + ((16 + 4 * tq) ^ xb)) << (ft * FSHIFT);
+                        }
+                    }
                 }
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const int row = (wc * NT + nt) * 8 + g;
-                    const int xb = (((co0 + row) >> 2) & 1) << 4;     // the image swaps the halves of these rows
-                    const uint8_t* wr = wimg + ((t * p.CW + cw) * TILE_C + row) * 32;
-                    bf[nt][0] |= *reinterpret_cast<const uint32_t*>(wr + ((4 * tq) ^ xb)) << sh;
-                    bf[nt][1] |= *reinterpret_cast<const uint32_t*>(wr + ((16 + 4 * tq) ^ xb)) << sh;
-                }
+                for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) mma_u8s8(acc[mt][nt], af[mt], bf[nt][0], bf[nt][1]);
             }
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) mma_u8s8(acc[mt][nt], af[mt], bf[nt][0], bf[nt][1]);
         }
-    }
+    };
+    if (p.strip_ks == 4) reduce(std::integral_constant<int, 4>{});
+    else if (p.strip_ks == 2) reduce(std::integral_constant<int, 2>{});
+    else reduce(std::integral_constant<int, 1>{});
 
     // ---- epilogue.  Fragment element e of (mt, nt): tile row (e >> 1) * 8 + g, channel 2 * tq + (e & 1).
     const bool want_y = p.y != nullptr, want_q = p.packed_next != nullptr;
