@@ -80,8 +80,9 @@ struct MmaTile {
     static constexpr int NTHREADS = 32 * WARPS_P * WARPS_C;
     static constexpr int TILE_P = 16 * MT * WARPS_P;
     static constexpr int TILE_C = 8 * NT * WARPS_C;
-    static constexpr int KW_WORDS = TILE_P * AB + TILE_C * WB;          // words per staged reduction word
-    static constexpr int KSTEP_RAW = 2048 / KW_WORDS;                    // about 8 KB per stage
+    static constexpr int KW_WORDS = TILE_P * AB + TILE_C * 8;           // words per staged reduction word: packed
+                                                                         // activation words + 32-byte weight rows
+    static constexpr int KSTEP_RAW = 4096 / KW_WORDS;                    // about 16 KB per stage
     static constexpr int KSTEP = KSTEP_RAW < 1 ? 1 : (KSTEP_RAW > 8 ? 8 : KSTEP_RAW);
     static constexpr int STAGE_WORDS = KSTEP * KW_WORDS;
     static constexpr int OUT_WORDS = TILE_P * code_row_bytes(TILE_C) / 4;
@@ -98,7 +99,7 @@ conv_mma_kernel(const ConvParams p) {
     using T = MmaTile<WB, AB, MT, NT, WARPS_P, WARPS_C>;
     constexpr int NTH = T::NTHREADS, TILE_P = T::TILE_P, TILE_C = T::TILE_C, KSTEP = T::KSTEP;
     constexpr int PPT = T::PPT, QSTRIDE = T::QSTRIDE;
-    constexpr int A_CH = chunk_bytes(AB), W_CH = chunk_bytes(WB);
+    constexpr int A_CH = chunk_bytes(AB);
 
     __shared__ __align__(16) uint32_t smem[T::SMEM_WORDS];
     __shared__ int2 ktab[MMA_KTAB];            // per reduction word: {word offset of the tap, r | s << 8}
@@ -134,11 +135,10 @@ conv_mma_kernel(const ConvParams p) {
             for (int s = 0; s < p.kw; ++s) col_ok[u] |= ((unsigned)(w0 + s) < (unsigned)p.W ? 1u : 0u) << s;
         }
     }
-    const bool w_vec_ok = ((p.Co * WB) % (W_CH / 4)) == 0;      // weight rows keep the chunk alignment
 
     auto stage = [&](int kk0, int buf) {
         uint32_t* A_s = smem + buf * T::STAGE_WORDS;                       // [KSTEP][TILE_P][AB]
-        uint32_t* W_s = A_s + KSTEP * TILE_P * AB;                         // [KSTEP][TILE_C][WB]
+        uint32_t* W_s = A_s + KSTEP * TILE_P * AB;                         // [KSTEP][TILE_C][8]
 #pragma unroll
         for (int qq = 0; qq < (KSTEP + QSTRIDE - 1) / QSTRIDE; ++qq) {
             const int q = qq * QSTRIDE + (QSTRIDE > 1 ? tid / TILE_P : 0);
@@ -158,25 +158,14 @@ conv_mma_kernel(const ConvParams p) {
                     cp_async_bytes(dst + c * (A_CH / 4), src + c * (A_CH / 4), A_CH, valid);
             }
         }
-        // weights: per reduction word a contiguous run of TILE_C*WB words (channels co0 .. co0+TILE_C)
-        if (w_vec_ok) {
-            constexpr int CHUNKS = TILE_C * WB * 4 / W_CH;
-            for (int e = tid; e < KSTEP * CHUNKS; e += NTH) {
-                const int q = e / CHUNKS, ch = e - q * CHUNKS;
-                const int word = ch * (W_CH / 4), c = word / WB;
-                const int kk = kk0 + q;
-                const bool valid = kk < p.KK && co0 + c < p.Co;
-                const uint32_t* src = valid ? p.w + ((size_t)kk * p.Co + co0) * WB + word : p.w;
-                cp_async_bytes(W_s + q * TILE_C * WB + word, src, W_CH, valid);
-            }
-        } else {
-            for (int e = tid; e < KSTEP * TILE_C * WB; e += NTH) {
-                const int q = e / (TILE_C * WB), word = e - q * (TILE_C * WB), c = word / WB;
-                const int kk = kk0 + q;
-                const bool valid = kk < p.KK && co0 + c < p.Co;
-                const uint32_t* src = valid ? p.w + ((size_t)kk * p.Co + co0) * WB + word : p.w;
-                cp_async_bytes(W_s + q * TILE_C * WB + word, src, 4, valid);
-            }
+        // weights: the 32-byte rows (one s8 code per input channel) of channels co0 .. co0+TILE_C of every staged
+        // reduction word, from the byte image; rows from c_out up to its multiple of 16 are zero there
+        for (int e = tid; e < KSTEP * TILE_C * 2; e += NTH) {
+            const int q = e / (TILE_C * 2), rem = e - q * (TILE_C * 2), c = rem >> 1, half = rem & 1;
+            const int kk = kk0 + q;
+            const bool valid = kk < p.KK && co0 + c < p.Co16;
+            const uint8_t* src = valid ? p.w8 + ((size_t)kk * p.Co16 + co0 + c) * 32 + half * 16 : p.w8;
+            cp_async_bytes(W_s + (q * TILE_C + c) * 8 + half * 4, src, 16, valid);
         }
     };
 
@@ -261,35 +250,26 @@ conv_mma_kernel(const ConvParams p) {
                         af[mt][3] |= __funnelshift_r(w1, w1, tq + 4 - k) & mask;
                     }
                 }
-                // weight fragments: the planes merged into the two's-complement code, byte = sum_m c_m 2^m bit_m.
-                // The top plane contributes -2^(WB-1) = the byte with bits WB-1 .. 7 set (sign extension).
+                // weight fragments: two words of the channel's byte row (the image holds the merged two's-complement
+                // codes, K position 4b+i = channel 8i+b, and swaps the 16-byte halves of rows with (c_out >> 2) odd)
                 uint32_t bf[NT][2];
+                const int xw = (g >> 2) << 2;
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
-                    const uint32_t* row = W_s + (q * TILE_C + (wc * NT + nt) * 8 + g) * WB;
-                    uint32_t wr[WB];
-                    load_words_shared<WB>(row, wr);
+                    const uint32_t* row = W_s + (q * TILE_C + (wc * NT + nt) * 8 + g) * 8;
+                    bf[nt][0] = row[tq ^ xw];
+                    bf[nt][1] = row[(4 + tq) ^ xw];
                     if (p.fold > 1) {
                         for (int f = 1; f < p.fold && q + f < KSTEP; ++f) {
-                            uint32_t t[WB];
-                            load_words_shared<WB>(row + f * TILE_C * WB, t);
-#pragma unroll
-                            for (int m = 0; m < WB; ++m) wr[m] |= t[m] << (f * p.fold_bits);
+                            const uint32_t* t = row + f * TILE_C * 8;
+                            if (p.fold_bits >= 8) {       // channel c + f * fold_bits: same word, byte f * fold_bits / 8 up
+                                bf[nt][0] |= t[tq ^ xw] << (f * p.fold_bits);
+                                bf[nt][1] |= t[(4 + tq) ^ xw] << (f * p.fold_bits);
+                            } else {                      // 4 channels a tap: odd taps land in the upper register
+                                const uint32_t v = t[tq ^ xw] << (8 * (f >> 1));
+                                if (f & 1) bf[nt][1] |= v; else bf[nt][0] |= v;
+                            }
                         }
-                    }
-                    bf[nt][0] = bf[nt][1] = 0u;
-#pragma unroll
-                    for (int m = 0; m < WB; ++m) {
-                        const uint32_t w = wr[m];
-                        const uint32_t mask = 0x01010101u << m;
-                        uint32_t b0 = __funnelshift_r(w, w, tq - m) & mask;
-                        uint32_t b1 = __funnelshift_r(w, w, tq + 4 - m) & mask;
-                        if (m == WB - 1 && WB < 8) {              // 2^(WB-1) * (2^(9-WB) - 1) = 256 - 2^(WB-1)
-                            b0 *= (1u << (9 - WB)) - 1u;
-                            b1 *= (1u << (9 - WB)) - 1u;
-                        }
-                        bf[nt][0] |= b0;
-                        bf[nt][1] |= b1;
                     }
                 }
 #pragma unroll
