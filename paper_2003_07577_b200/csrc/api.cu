@@ -29,15 +29,16 @@ const ConvVariant* conv_popc_variant(int w_bits, int a_bits, int variant) {
 }
 
 const ConvVariant* conv_mma_variant(int w_bits, int a_bits, int variant) {
-    switch (w_bits) {
-        case 1: return conv_mma_variant_w1(a_bits, variant);
-        case 2: return conv_mma_variant_w2(a_bits, variant);
-        case 3: return conv_mma_variant_w3(a_bits, variant);
-        case 4: return conv_mma_variant_w4(a_bits, variant);
-        case 5: return conv_mma_variant_w5(a_bits, variant);
-        case 6: return conv_mma_variant_w6(a_bits, variant);
-        case 7: return conv_mma_variant_w7(a_bits, variant);
-        case 8: return conv_mma_variant_w8(a_bits, variant);
+    if (w_bits < 1 || w_bits > 8) return nullptr;
+    switch (a_bits) {
+        case 1: return conv_mma_variant_a1(variant);
+        case 2: return conv_mma_variant_a2(variant);
+        case 3: return conv_mma_variant_a3(variant);
+        case 4: return conv_mma_variant_a4(variant);
+        case 5: return conv_mma_variant_a5(variant);
+        case 6: return conv_mma_variant_a6(variant);
+        case 7: return conv_mma_variant_a7(variant);
+        case 8: return conv_mma_variant_a8(variant);
         default: return nullptr;
     }
 }

@@ -2,26 +2,27 @@
 //
 // sm_100a has no native 1-bit AND+POPC matrix instruction: the toolchain expands
 // mma.sync...b1.and.popc into ~110 instructions that turn bits into bytes and issue eight int8
-// MMAs.  This kernel does that expansion itself, once per operand fragment instead of once per
-// MMA: a bit plane is turned into bytes that are 0 where the bit is clear and the plane's
-// coefficient where it is set (2^k for activation plane k, 2^m for weight plane m, -2^(M-1) for the
-// top weight plane), so that one int8 MMA of activation plane k against weight plane m adds
-// c_m 2^(m+k) * bitcount(AND(plane k, plane m)) -- stage 1 (Eq. 13) and stage 2 (Eq. 14) of the
-// binary decomposition at once -- into ONE int32 accumulator per output.  Every plane pair is still
-// its own binary contraction (M*K MMAs per 32 reduction bits); the matrix P never exists.
+// MMAs.  This kernel goes one step further: the planes of a 32-channel word are merged back into one
+// byte per channel -- the activation code sum_k 2^k bit_k as u8, the weight code sum_m c_m 2^m bit_m
+// as s8 (c_m = -1 for the top plane: two's complement) -- so that ONE int8 MMA per reduction word adds
+// sum_m sum_k c_m 2^(m+k) * bitcount(AND(activation plane k, weight plane m)), stage 1 (Eq. 13) and
+// stage 2 (Eq. 14) of the binary decomposition for all plane pairs at once, into one int32
+// accumulator per output.  The matrix P never exists; the result is the same integer.
 //
-// Fragments are built in registers straight from the packed 32-bit words: thread (g, tq) of a warp
-// owns reduction bits {8b + tq, 8b + 4 + tq : b = 0..3} of a word, so "rotate right by (tq - k), AND
-// with 0x01010101 << k" yields a fragment register (two instructions per register).  The same bit
-// assignment is used for both operands, which is all the MMA needs.
+// Activation fragments are built in registers straight from the packed 32-bit words: thread (g, tq)
+// of a warp owns reduction bits {8b + tq, 8b + 4 + tq : b = 0..3} of a word, so "rotate right by
+// (tq - k), AND with 0x01010101 << k" puts plane k's bits at bit k of four bytes (two instructions
+// per plane and register).  Weight fragments are two words of the channel's row of the byte image
+// the weight packer wrote (K position 4b + i = channel 8i + b, the same assignment), so the kernel
+// does not depend on the weight bit count.
 //
 // Layers with at most 16 input channels use only the low bits of each word; there 2, 4 or 8 staged
 // taps are OR-ed into one word (shifted by 16, 8 or 4 bits) while the fragments are built, for both
-// operands alike, so a 32-bit MMA step is filled with real reduction bits.
+// operands alike, so a 32-channel MMA step is filled with real reduction bits.
 //
 // Work split: a CTA owns TILE_P consecutive output pixels x TILE_C channels; a warp owns
-// 16*MT pixels x 8*NT channels.  Packed words of KSTEP reduction words are staged with cp.async
-// (zero fill for taps outside the image), double buffered.
+// 16*MT pixels x 8*NT channels.  The packed activation words and the weight rows of KSTEP reduction
+// words are staged with cp.async (zero fill for taps outside the image), double buffered.
 #pragma once
 
 #include "ebs_internal.cuh"
@@ -75,7 +76,7 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], const uint32_t (&a)[4], ui
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <int WB, int AB, int MT, int NT, int WARPS_P, int WARPS_C>
+template <int AB, int MT, int NT, int WARPS_P, int WARPS_C>
 struct MmaTile {
     static constexpr int NTHREADS = 32 * WARPS_P * WARPS_C;
     static constexpr int TILE_P = 16 * MT * WARPS_P;
@@ -93,10 +94,10 @@ struct MmaTile {
     static_assert(SMEM_WORDS * 4 + MMA_KTAB * 8 <= 47 * 1024, "static shared memory budget");
 };
 
-template <int WB, int AB, int MT, int NT, int WARPS_P, int WARPS_C>
+template <int AB, int MT, int NT, int WARPS_P, int WARPS_C>
 __global__ void __launch_bounds__(32 * WARPS_P * WARPS_C)
 conv_mma_kernel(const ConvParams p) {
-    using T = MmaTile<WB, AB, MT, NT, WARPS_P, WARPS_C>;
+    using T = MmaTile<AB, MT, NT, WARPS_P, WARPS_C>;
     constexpr int NTH = T::NTHREADS, TILE_P = T::TILE_P, TILE_C = T::TILE_C, KSTEP = T::KSTEP;
     constexpr int PPT = T::PPT, QSTRIDE = T::QSTRIDE;
     constexpr int A_CH = chunk_bytes(AB);
@@ -458,9 +459,9 @@ conv_mma_kernel(const ConvParams p) {
     }
 }
 
-template <int WB, int AB, int MT, int NT, int WARPS_P, int WARPS_C>
+template <int AB, int MT, int NT, int WARPS_P, int WARPS_C>
 void launch_conv_mma(const ConvParams& p, dim3 grid, cudaStream_t st) {
-    conv_mma_kernel<WB, AB, MT, NT, WARPS_P, WARPS_C><<<grid, 32 * WARPS_P * WARPS_C, 0, st>>>(p);
+    conv_mma_kernel<AB, MT, NT, WARPS_P, WARPS_C><<<grid, 32 * WARPS_P * WARPS_C, 0, st>>>(p);
 }
 
 // Variants: variant = size_class * 3 + tile_c_index, tile_c in {16, 32, 64}.
@@ -469,45 +470,41 @@ void launch_conv_mma(const ConvParams& p, dim3 grid, cudaStream_t st) {
 //   class 2 (small)  16 pixels x 16 channels per warp, 4 warps -- for layers that otherwise leave SMs idle
 // Every plane pair is one MMA per 16x8 output block per reduction word, so the large warp tile
 // shrinks as the pair count grows.
-template <int WB, int AB, int VARIANT>
+template <int AB, int VARIANT>
 struct MmaGeom {
-    static constexpr int PAIRS = WB * AB;
     static constexpr int CLASS = VARIANT / 3;
     static constexpr int TILE_C = 16 << (VARIANT % 3);
     static constexpr int WARPS = CLASS == 2 ? 4 : 8;
-    static constexpr int NT_PREF = (CLASS == 0 && PAIRS <= 4) ? 4 : 2;
+    static constexpr int NT_PREF = (CLASS == 0 && AB <= 4) ? 4 : 2;
     static constexpr int NT = (TILE_C / 8) < NT_PREF ? (TILE_C / 8) : NT_PREF;
     static constexpr int WARPS_C_RAW = TILE_C / (8 * NT);
     static constexpr int WARPS_C = WARPS_C_RAW > WARPS ? WARPS : WARPS_C_RAW;
     static constexpr int WARPS_P = WARPS / WARPS_C;
-    static constexpr int ACC_BUDGET = PAIRS == 1 ? 64 : (PAIRS <= 4 ? 32 : (PAIRS <= 16 ? 16 : 8));
+    static constexpr int ACC_BUDGET = AB == 1 ? 64 : (AB <= 4 ? 32 : 16);   // accumulator registers of a thread
     static constexpr int MT_RAW = ACC_BUDGET / (4 * NT);
-    static constexpr int MT_AB = AB <= 2 ? 4 : (AB <= 4 ? 2 : 1);      // activation fragments: MT*AB*4 registers
+    static constexpr int MT_AB = AB <= 2 ? 4 : (AB <= 4 ? 2 : 1);      // activation words in flight: MT*AB*2 registers
     static constexpr int MT_LARGE = MT_RAW < 1 ? 1 : (MT_RAW > MT_AB ? MT_AB : MT_RAW);
     static constexpr int MT = CLASS == 0 ? MT_LARGE : (CLASS == 1 ? (MT_AB < 2 ? MT_AB : 2) : 1);
 };
 
 constexpr int NUM_MMA_VARIANTS = 9;
 
-template <int WB, int AB, int VARIANT>
+template <int AB, int VARIANT>
 constexpr ConvVariant make_mma_variant() {
-    using G = MmaGeom<WB, AB, VARIANT>;
-    return ConvVariant{&launch_conv_mma<WB, AB, G::MT, G::NT, G::WARPS_P, G::WARPS_C>, 16 * G::MT * G::WARPS_P,
+    using G = MmaGeom<AB, VARIANT>;
+    return ConvVariant{&launch_conv_mma<AB, G::MT, G::NT, G::WARPS_P, G::WARPS_C>, 16 * G::MT * G::WARPS_P,
                        8 * G::NT * G::WARPS_C, 32 * G::WARPS_P * G::WARPS_C};
 }
 
-#define EBS_MMA_ROW(WB, AB)                                                                             \
-    {make_mma_variant<WB, AB, 0>(), make_mma_variant<WB, AB, 1>(), make_mma_variant<WB, AB, 2>(),       \
-     make_mma_variant<WB, AB, 3>(), make_mma_variant<WB, AB, 4>(), make_mma_variant<WB, AB, 5>(),       \
-     make_mma_variant<WB, AB, 6>(), make_mma_variant<WB, AB, 7>(), make_mma_variant<WB, AB, 8>()}
-
-#define EBS_DEFINE_MMA_TABLE(WB)                                                                        \
-    const ConvVariant* conv_mma_variant_w##WB(int a_bits, int variant) {                                \
-        static const ConvVariant table[8][NUM_MMA_VARIANTS] = {                                         \
-            EBS_MMA_ROW(WB, 1), EBS_MMA_ROW(WB, 2), EBS_MMA_ROW(WB, 3), EBS_MMA_ROW(WB, 4),             \
-            EBS_MMA_ROW(WB, 5), EBS_MMA_ROW(WB, 6), EBS_MMA_ROW(WB, 7), EBS_MMA_ROW(WB, 8)};            \
-        if (a_bits < 1 || a_bits > 8 || variant < 0 || variant >= NUM_MMA_VARIANTS) return nullptr;     \
-        return &table[a_bits - 1][variant];                                                             \
+// One translation unit per activation bit count (conv_mma_a1.cu .. conv_mma_a8.cu) defines its row of the table.
+#define EBS_DEFINE_MMA_ROW(AB)                                                                           \
+    const ConvVariant* conv_mma_variant_a##AB(int variant) {                                             \
+        static const ConvVariant row[NUM_MMA_VARIANTS] = {                                               \
+            make_mma_variant<AB, 0>(), make_mma_variant<AB, 1>(), make_mma_variant<AB, 2>(),             \
+            make_mma_variant<AB, 3>(), make_mma_variant<AB, 4>(), make_mma_variant<AB, 5>(),             \
+            make_mma_variant<AB, 6>(), make_mma_variant<AB, 7>(), make_mma_variant<AB, 8>()};            \
+        if (variant < 0 || variant >= NUM_MMA_VARIANTS) return nullptr;                                  \
+        return &row[variant];                                                                            \
     }
 
 }  // namespace ebs

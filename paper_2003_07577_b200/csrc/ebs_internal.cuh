@@ -55,13 +55,14 @@ EBS_DECLARE_WB(1) EBS_DECLARE_WB(2) EBS_DECLARE_WB(3) EBS_DECLARE_WB(4)
 EBS_DECLARE_WB(5) EBS_DECLARE_WB(6) EBS_DECLARE_WB(7) EBS_DECLARE_WB(8)
 #undef EBS_DECLARE_WB
 
-// Tensor-pipe kernels (conv_mma_w1.cu .. conv_mma_w8.cu); variant 0 .. NUM_CONV_MMA_VARIANTS-1.
+// Warp-level tensor-pipe kernels (conv_mma_a1.cu .. conv_mma_a8.cu, one per activation bit count; the weights come
+// as bytes, so the kernel does not depend on their bit count); variant 0 .. NUM_CONV_MMA_VARIANTS-1.
 enum { NUM_CONV_MMA_VARIANTS = 9, CONV_MMA_MAX_KK = 256 };
 const ConvVariant* conv_mma_variant(int w_bits, int a_bits, int variant);
-#define EBS_DECLARE_WB(WB) const ConvVariant* conv_mma_variant_w##WB(int a_bits, int variant);
-EBS_DECLARE_WB(1) EBS_DECLARE_WB(2) EBS_DECLARE_WB(3) EBS_DECLARE_WB(4)
-EBS_DECLARE_WB(5) EBS_DECLARE_WB(6) EBS_DECLARE_WB(7) EBS_DECLARE_WB(8)
-#undef EBS_DECLARE_WB
+#define EBS_DECLARE_AB(AB) const ConvVariant* conv_mma_variant_a##AB(int variant);
+EBS_DECLARE_AB(1) EBS_DECLARE_AB(2) EBS_DECLARE_AB(3) EBS_DECLARE_AB(4)
+EBS_DECLARE_AB(5) EBS_DECLARE_AB(6) EBS_DECLARE_AB(7) EBS_DECLARE_AB(8)
+#undef EBS_DECLARE_AB
 
 // 5th-generation tensor-core kernels (conv_umma_w1.cu .. conv_umma_w8.cu); variant = log2(tile_n / 16).
 enum { NUM_CONV_UMMA_VARIANTS = 5, NUM_CONV_STRIP_VARIANTS = 5, NUM_CONV_RESIDENT_VARIANTS = 5, NUM_CONV_MMA_STRIP_VARIANTS = 3 };
