@@ -474,7 +474,7 @@ template <int AB, int VARIANT>
 struct MmaGeom {
     static constexpr int CLASS = VARIANT / 3;
     static constexpr int TILE_C = 16 << (VARIANT % 3);
-    static constexpr int WARPS = CLASS == 2 ? 4 : 8;
+    static constexpr int WARPS = CLASS == 2 ? TILE_C / 4 : 8;          // small: 4 pixel groups x TILE_C/16 channel groups
     static constexpr int NT_PREF = (CLASS == 0 && AB <= 4) ? 4 : 2;
     static constexpr int NT = (TILE_C / 8) < NT_PREF ? (TILE_C / 8) : NT_PREF;
     static constexpr int WARPS_C_RAW = TILE_C / (8 * NT);
