@@ -42,7 +42,7 @@ inline MmaStripGeom mma_strip_geometry(const ConvParams& p, int tile_p, int tile
     return g;
 }
 
-template <int AB, int MT, int NT, int WARPS_P, int WARPS_C>
+template <int AB, int MT, int NT, int WARPS_P, int WARPS_C, bool COMPACT = false>
 __global__ void __launch_bounds__(32 * WARPS_P * WARPS_C)
 conv_mma_strip_kernel(const ConvParams p) {
     constexpr int NTH = 32 * WARPS_P * WARPS_C, TILE_P = 16 * MT * WARPS_P, TILE_C = 8 * NT * WARPS_C;
@@ -56,19 +56,36 @@ conv_mma_strip_kernel(const ConvParams p) {
     const int Wp = strip_frame_w(p), Hp = strip_frame_h(p);
     const int frame = p.N * Hp * Wp;
     const int f0 = blockIdx.x * TILE_P, co0 = blockIdx.y * TILE_C;
-    uint8_t* strip = smem_raw;                                       // [CW][SP][32]
-    uint8_t* wimg = strip + p.CW * SP * 32;                          // [taps * CW][TILE_C][32]
-    uint8_t* out_s = wimg + taps * p.CW * TILE_C * 32;               // [TILE_P][ROWB] requantized codes
+    // COMPACT (one word of at most 16 channels): 16 bytes per pixel and weight row, word j = channels j, 8+j, 4+j, 12+j;
+    // the weights get one more (zero) tap, the partner of the last tap when their number is odd
+    uint8_t* strip = smem_raw;                                       // [CW][SP][32]   | [SP][16]
+    uint8_t* wimg = strip + (COMPACT ? SP * 16 : p.CW * SP * 32);    // [taps * CW][TILE_C][32] | [taps + 1][TILE_C][16]
+    uint8_t* out_s = wimg + (COMPACT ? (taps + 1) * TILE_C * 16 : taps * p.CW * TILE_C * 32);   // [TILE_P][ROWB] codes
     int* gp_s = reinterpret_cast<int*>(out_s + TILE_P * ROWB);       // output pixel of every frame row, -1: none
     // ---- weight rows of this channel tile, all taps and words (rows past c_out are zero in the image): asynchronous
     // copies issued first, so that their latency hides behind the tables and the strip expansion
-    for (int e = tid; e < taps * p.CW * TILE_C * 2; e += NTH) {
-        const int half = e & 1, row = (e >> 1) % TILE_C, kk = (e >> 1) / TILE_C;
-        const bool valid = co0 + row < p.Co16;
-        const uint8_t* src = valid ? p.w8 + ((size_t)kk * p.Co16 + co0 + row) * 32 + half * 16 : p.w8;
-        cp_async_bytes(wimg + (kk * TILE_C + row) * 32 + half * 16, src, 16, valid);
+    if constexpr (COMPACT) {
+        for (int e = tid; e < (taps + 1) * TILE_C; e += NTH) {
+            const int t = e / TILE_C, row = e - t * TILE_C;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (t < taps && co0 + row < p.Co16) {
+                const uint4* src = reinterpret_cast<const uint4*>(p.w8 + ((size_t)t * p.Co16 + co0 + row) * 32);
+                const int sw = ((co0 + row) >> 2) & 1;                   // the image swaps the halves of these rows
+                const uint4 lo = __ldg(src + sw), hi = __ldg(src + (sw ^ 1));
+                v = make_uint4(__byte_perm(lo.x, hi.x, 0x5410), __byte_perm(lo.y, hi.y, 0x5410),
+                               __byte_perm(lo.z, hi.z, 0x5410), __byte_perm(lo.w, hi.w, 0x5410));
+            }
+            reinterpret_cast<uint4*>(wimg)[e] = v;
+        }
+    } else {
+        for (int e = tid; e < taps * p.CW * TILE_C * 2; e += NTH) {
+            const int half = e & 1, row = (e >> 1) % TILE_C, kk = (e >> 1) / TILE_C;
+            const bool valid = co0 + row < p.Co16;
+            const uint8_t* src = valid ? p.w8 + ((size_t)kk * p.Co16 + co0 + row) * 32 + half * 16 : p.w8;
+            cp_async_bytes(wimg + (kk * TILE_C + row) * 32 + half * 16, src, 16, valid);
+        }
+        cp_async_commit();
     }
-    cp_async_commit();
     __shared__ int tap_shift_s[64];                                   // frame shift r * Wp + s of every tap
     for (int t = tid; t < taps; t += NTH) tap_shift_s[t] = (t / p.kw) * Wp + (t % p.kw);
 
@@ -93,10 +110,15 @@ conv_mma_strip_kernel(const ConvParams p) {
                 }
             }
         }
-        uint4* dst = reinterpret_cast<uint4*>(strip + (cw * SP + s) * 32);
-        const int sw = (s >> 2) & 1;
-        dst[sw] = make_uint4(r[0], r[1], r[2], r[3]);
-        dst[sw ^ 1] = make_uint4(r[4], r[5], r[6], r[7]);
+        if constexpr (COMPACT) {
+            reinterpret_cast<uint4*>(strip)[s] = make_uint4(__byte_perm(r[0], r[4], 0x5410), __byte_perm(r[1], r[5], 0x5410),
+                                                            __byte_perm(r[2], r[6], 0x5410), __byte_perm(r[3], r[7], 0x5410));
+        } else {
+            uint4* dst = reinterpret_cast<uint4*>(strip + (cw * SP + s) * 32);
+            const int sw = (s >> 2) & 1;
+            dst[sw] = make_uint4(r[0], r[1], r[2], r[3]);
+            dst[sw ^ 1] = make_uint4(r[4], r[5], r[6], r[7]);
+        }
     }
     // ---- output pixel of each row of the tile
     for (int pl = tid; pl < TILE_P; pl += NTH) {
@@ -169,9 +191,39 @@ conv_mma_strip_kernel(const ConvParams p) {
             }
         }
     };
-    if (p.strip_ks == 4) reduce(std::integral_constant<int, 4>{});
-    else if (p.strip_ks == 2) reduce(std::integral_constant<int, 2>{});
-    else reduce(std::integral_constant<int, 1>{});
+    if constexpr (COMPACT) {
+        // two taps per MMA step: K positions 0-15 are the first tap's 16 channels, 16-31 the second's
+        const int arow0 = (wp_ * MT) * 16 + g;
+#pragma unroll 1
+        for (int t0 = 0; t0 < taps; t0 += 2) {
+            const int t1 = t0 + 1;                                         // == taps: the zero weight rows
+            const int sh0 = tap_shift_s[t0], sh1 = tap_shift_s[t1 < taps ? t1 : t0];
+            uint32_t af[MT][4], bf[NT][2];
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                const uint8_t* r0 = strip + (arow0 + mt * 16 + sh0) * 16 + 4 * tq;
+                const uint8_t* r1 = strip + (arow0 + mt * 16 + sh1) * 16 + 4 * tq;
+                af[mt][0] = *reinterpret_cast<const uint32_t*>(r0);
+                af[mt][1] = *reinterpret_cast<const uint32_t*>(r0 + 8 * 16);
+                af[mt][2] = *reinterpret_cast<const uint32_t*>(r1);
+                af[mt][3] = *reinterpret_cast<const uint32_t*>(r1 + 8 * 16);
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const int row = (wc * NT + nt) * 8 + g;
+                bf[nt][0] = *reinterpret_cast<const uint32_t*>(wimg + (t0 * TILE_C + row) * 16 + 4 * tq);
+                bf[nt][1] = *reinterpret_cast<const uint32_t*>(wimg + (t1 * TILE_C + row) * 16 + 4 * tq);
+            }
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) mma_u8s8(acc[mt][nt], af[mt], bf[nt][0], bf[nt][1]);
+        }
+    } else {
+        if (p.strip_ks == 4) reduce(std::integral_constant<int, 4>{});
+        else if (p.strip_ks == 2) reduce(std::integral_constant<int, 2>{});
+        else reduce(std::integral_constant<int, 1>{});
+    }
 
     // ---- epilogue.  Fragment element e of (mt, nt): tile row (e >> 1) * 8 + g, channel 2 * tq + (e & 1).
     const bool want_y = p.y != nullptr, want_q = p.packed_next != nullptr;
@@ -257,10 +309,19 @@ void launch_conv_mma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st)
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
         cudaFuncSetAttribute(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              96 * 1024);
+        if constexpr (TILE_C == 16)
+            cudaFuncSetAttribute(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, true>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
         attr_set[dev] = true;
     }
     const long long frame = (long long)p.N * strip_frame_h(p) * strip_frame_w(p);
     const dim3 grid((unsigned)((frame + TILE_P - 1) / TILE_P), (unsigned)((p.Co + TILE_C - 1) / TILE_C), 1);
+    if constexpr (TILE_C == 16) {                             // 9-16 input channels: the 16-byte-per-pixel form
+        if (g.fold == 2) {
+            conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, true><<<grid, 32 * WARPS_P * WARPS_C, g.smem_bytes, st>>>(p);
+            return;
+        }
+    }
     conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C><<<grid, 32 * WARPS_P * WARPS_C, g.smem_bytes, st>>>(p);
 }
 
