@@ -45,7 +45,7 @@ WORKLOADS = {
 SM_COUNT, POPC_LANES_PER_CLK_SM = 148, 16
 # dram__bytes_read.sum + dram__bytes_write.sum per conv launch, mean over the 20 layers, from the ncu
 # capture summarised in profiles/ (outputs stay in the 126 MB L2 while ncu replays a launch)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 721582
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 732747
 
 
 def measured_peaks():
@@ -560,8 +560,9 @@ def run_gpu(args):
                 "note": "ebs_conv2d_mixed_host per layer: pinned u8 codes in, packed next-layer planes out; layers round-robin on 3 streams; wall clock"},
         "gpu_launches": (len(layers) + 2) * args.steps, "device_wait_timeouts": ebs.ebs_device_wait_timeouts(),
         "roofline": {"bound": bound,
-                     "kernel": "bit-plane conv, the %d launches of a step (conv_umma_strip_kernel / conv_umma_kernel: "
-                               "tcgen05; conv_mma_kernel: mma.sync; planes merged to bytes in registers)" % len(layers),
+                     "kernel": "bit-plane conv, the %d launches of a step (conv_umma_strip_kernel / conv_umma_resident_kernel "
+                               "/ conv_umma_kernel: tcgen05; conv_mma_kernel / conv_mma_strip_kernel: mma.sync; planes "
+                               "merged to bytes on chip)" % len(layers),
                      "achieved": achieved, "peak": roof_peak, "unit": roof_unit, "frac": achieved / roof_peak,
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if args.workload == "config2" and not args.only else None,
                      "accounting": "achieved = algorithmic bytes (packed input planes + weight planes + int32 accumulators "
