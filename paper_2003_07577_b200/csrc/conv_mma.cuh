@@ -300,7 +300,6 @@ conv_mma_kernel(const ConvParams p) {
     // common case: even c_out and NHWC -> two-channel vectors, per-channel terms kept in registers, the
     // shortcut codes (if the shortcut comes as packed planes) staged as bytes in the code tile
     const bool simple = pair_ok && !p.y_nchw;
-    const bool plain = simple && !p.ch_scale && !p.ch_bias && !p.residual && !p.res_packed;
     if (simple && p.res_packed) {
         constexpr int GROUPS = TILE_C / 8;
         for (int e = tid; e < TILE_P * GROUPS; e += NTH) {
@@ -321,18 +320,74 @@ conv_mma_kernel(const ConvParams p) {
         }
         __syncthreads();
     }
-    float cs[NT][2], cb[NT][2];
-    if (simple && !plain) {
+    if (simple) {
+        // Per-channel terms and the shortcut default to exact identities (x * 1 and x + (-0) return x bit for bit), so
+        // the block is straight-line code with uniform predicates on its loads and stores only; the accumulators go
+        // out in a loop of their own.  (One unrolled copy instead of three keeps the kernel's code small: these
+        // launches are short enough for instruction fetch to matter.)
+        float cs[NT][2], cb[NT][2];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
             const bool in = co < p.Co;                          // c_out is even here: co + 1 exists with co
             cs[nt][0] = (p.ch_scale && in) ? __ldg(p.ch_scale + co) : 1.0f;
             cs[nt][1] = (p.ch_scale && in) ? __ldg(p.ch_scale + co + 1) : 1.0f;
-            cb[nt][0] = (p.ch_bias && in) ? __ldg(p.ch_bias + co) : 0.0f;
-            cb[nt][1] = (p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : 0.0f;
+            cb[nt][0] = (p.ch_bias && in) ? __ldg(p.ch_bias + co) : -0.0f;
+            cb[nt][1] = (p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : -0.0f;
         }
-    }
+        const int co_t = co0 + wc * NT * 8 + 2 * tq;            // this thread's first channel
+        if (p.acc) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int gp = tile_p0 + (wp * MT + mt) * 16 + half * 8 + g;
+                    int* row = p.acc + (size_t)gp * p.Co + co_t;
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+                        if (gp < p.P && co_t + nt * 8 < p.Co)
+                            *reinterpret_cast<int2*>(row + nt * 8) = make_int2(acc[mt][nt][half * 2], acc[mt][nt][half * 2 + 1]);
+                }
+        }
+        if (want_y || want_q) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int pl = (wp * MT + mt) * 16 + half * 8 + g;
+                    const int gp = tile_p0 + pl;
+                    const size_t row_o = (size_t)gp * p.Co + co_t;
+                    uint8_t* code_row = out_s + pl * ROWB + wc * NT * 8 + 2 * tq;
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const bool valid = gp < p.P && co_t + nt * 8 < p.Co;
+                        float y0 = __fmul_rn((float)acc[mt][nt][half * 2], p.S), y1 = __fmul_rn((float)acc[mt][nt][half * 2 + 1], p.S);
+                        y0 = __fadd_rn(__fmul_rn(y0, cs[nt][0]), cb[nt][0]);
+                        y1 = __fadd_rn(__fmul_rn(y1, cs[nt][1]), cb[nt][1]);
+                        float r0 = -0.0f, r1 = -0.0f;
+                        if (p.residual) {
+                            if (valid) {
+                                const float2 r = __ldg(reinterpret_cast<const float2*>(p.residual + row_o + nt * 8));
+                                r0 = r.x;
+                                r1 = r.y;
+                            }
+                        } else if (p.res_packed) {
+                            const uint32_t rc = *reinterpret_cast<const uint16_t*>(code_row + nt * 8);
+                            r0 = __fmul_rn(p.res_scale, (float)(rc & 0xFFu));
+                            r1 = __fmul_rn(p.res_scale, (float)(rc >> 8));
+                        }
+                        y0 = __fadd_rn(y0, r0);
+                        y1 = __fadd_rn(y1, r1);
+                        y0 = p.relu ? fmaxf(y0, 0.0f) : y0;
+                        y1 = p.relu ? fmaxf(y1, 0.0f) : y1;
+                        if (want_y && valid) *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
+                        const int code0 = valid ? quantize_act_code(y0, p.inv_next, qmax) : 0;
+                        const int code1 = valid ? quantize_act_code(y1, p.inv_next, qmax) : 0;
+                        if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
+                    }
+                }
+        }
+    } else {
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
@@ -340,62 +395,6 @@ conv_mma_kernel(const ConvParams p) {
             const int pl = (wp * MT + mt) * 16 + half * 8 + g;
             const int gp = tile_p0 + pl;
             const bool pvalid = gp < p.P;
-            const size_t row_o = (size_t)gp * p.Co + co0 + wc * NT * 8 + 2 * tq;
-            uint8_t* code_row = out_s + pl * ROWB + wc * NT * 8 + 2 * tq;
-            if (plain) {                                        // no per-channel terms, no shortcut
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
-                    const int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
-                    const bool valid = pvalid && co < p.Co;
-                    int code0 = 0, code1 = 0;
-                    if (valid && p.acc) *reinterpret_cast<int2*>(p.acc + row_o + nt * 8) = make_int2(a0, a1);
-                    if (want_y || want_q) {
-                        float y0 = __fmul_rn((float)a0, p.S), y1 = __fmul_rn((float)a1, p.S);
-                        if (p.relu) { y0 = y0 > 0.0f ? y0 : 0.0f; y1 = y1 > 0.0f ? y1 : 0.0f; }
-                        if (valid && want_y) *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
-                        if (valid && want_q) {
-                            code0 = quantize_act_code(y0, p.inv_next, qmax);
-                            code1 = quantize_act_code(y1, p.inv_next, qmax);
-                        }
-                    }
-                    if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
-                }
-                continue;
-            }
-            if (simple) {
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
-                    const int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
-                    const bool valid = pvalid && co < p.Co;
-                    int code0 = 0, code1 = 0;
-                    if (valid && p.acc) *reinterpret_cast<int2*>(p.acc + row_o + nt * 8) = make_int2(a0, a1);
-                    if (want_y || want_q) {
-                        float y0 = __fmul_rn((float)a0, p.S), y1 = __fmul_rn((float)a1, p.S);
-                        if (p.ch_scale) { y0 = __fmul_rn(y0, cs[nt][0]); y1 = __fmul_rn(y1, cs[nt][1]); }
-                        if (p.ch_bias) { y0 = __fadd_rn(y0, cb[nt][0]); y1 = __fadd_rn(y1, cb[nt][1]); }
-                        if (p.residual && valid) {
-                            const float2 r = __ldg(reinterpret_cast<const float2*>(p.residual + row_o + nt * 8));
-                            y0 = __fadd_rn(y0, r.x);
-                            y1 = __fadd_rn(y1, r.y);
-                        }
-                        if (p.res_packed) {
-                            const uint32_t rc = *reinterpret_cast<const uint16_t*>(code_row + nt * 8);
-                            y0 = __fadd_rn(y0, __fmul_rn(p.res_scale, (float)(rc & 0xFFu)));
-                            y1 = __fadd_rn(y1, __fmul_rn(p.res_scale, (float)(rc >> 8)));
-                        }
-                        if (p.relu) { y0 = y0 > 0.0f ? y0 : 0.0f; y1 = y1 > 0.0f ? y1 : 0.0f; }
-                        if (valid && want_y) *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
-                        if (valid && want_q) {
-                            code0 = quantize_act_code(y0, p.inv_next, qmax);
-                            code1 = quantize_act_code(y1, p.inv_next, qmax);
-                        }
-                    }
-                    if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
-                }
-                continue;
-            }
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 const int cl = (wc * NT + nt) * 8 + 2 * tq, co = co0 + cl;
@@ -452,6 +451,7 @@ conv_mma_kernel(const ConvParams p) {
                 if (want_q) *reinterpret_cast<uint16_t*>(out_s + pl * ROWB + cl) = (uint16_t)(code0 | (code1 << 8));
             }
         }
+    }
     }
     if (want_q) {
         __syncthreads();

@@ -65,6 +65,7 @@ conv_mma_strip_kernel(const ConvParams p) {
     // ---- weight rows of this channel tile, all taps and words (rows past c_out are zero in the image): asynchronous
     // copies issued first, so that their latency hides behind the tables and the strip expansion
     if constexpr (COMPACT) {
+#pragma unroll 1
         for (int e = tid; e < (taps + 1) * TILE_C; e += NTH) {
             const int t = e / TILE_C, row = e - t * TILE_C;
             uint4 v = make_uint4(0, 0, 0, 0);
@@ -78,6 +79,7 @@ conv_mma_strip_kernel(const ConvParams p) {
             reinterpret_cast<uint4*>(wimg)[e] = v;
         }
     } else {
+#pragma unroll 1
         for (int e = tid; e < taps * p.CW * TILE_C * 2; e += NTH) {
             const int half = e & 1, row = (e >> 1) % TILE_C, kk = (e >> 1) / TILE_C;
             const bool valid = co0 + row < p.Co16;
@@ -87,10 +89,11 @@ conv_mma_strip_kernel(const ConvParams p) {
         cp_async_commit();
     }
     __shared__ int tap_shift_s[64];                                   // frame shift r * Wp + s of every tap
+#pragma unroll 1
     for (int t = tid; t < taps; t += NTH) tap_shift_s[t] = (t / p.kw) * Wp + (t % p.kw);
 
     // ---- the strip: packed words -> bytes, once per pixel and word
-#pragma unroll 2
+#pragma unroll 1
     for (int e = tid; e < S * p.CW; e += NTH) {
         const int s = e / p.CW, cw = e - s * p.CW;
         const int f = f0 + s;
@@ -121,6 +124,7 @@ conv_mma_strip_kernel(const ConvParams p) {
         }
     }
     // ---- output pixel of each row of the tile
+#pragma unroll 1
     for (int pl = tid; pl < TILE_P; pl += NTH) {
         const int f = f0 + pl;
         int gp = -1;
@@ -228,6 +232,8 @@ conv_mma_strip_kernel(const ConvParams p) {
     // ---- epilogue.  Fragment element e of (mt, nt): tile row (e >> 1) * 8 + g, channel 2 * tq + (e & 1).
     const bool want_y = p.y != nullptr, want_q = p.packed_next != nullptr;
     const int qmax = (1 << p.next_bits) - 1;
+    // Per-channel terms default to exact identities (x * 1 and x + (-0) return x bit for bit), so the block below is
+    // straight-line code with uniform predicates only on its stores; accumulators go out in a loop of their own.
     float cs[NT][2], cb[NT][2];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -235,44 +241,52 @@ conv_mma_strip_kernel(const ConvParams p) {
         const bool in = co < p.Co;                                  // c_out is even: co + 1 exists with co
         cs[nt][0] = (p.ch_scale && in) ? __ldg(p.ch_scale + co) : 1.0f;
         cs[nt][1] = (p.ch_scale && in) ? __ldg(p.ch_scale + co + 1) : 1.0f;
-        cb[nt][0] = (p.ch_bias && in) ? __ldg(p.ch_bias + co) : 0.0f;
-        cb[nt][1] = (p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : 0.0f;
+        cb[nt][0] = (p.ch_bias && in) ? __ldg(p.ch_bias + co) : -0.0f;
+        cb[nt][1] = (p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : -0.0f;
     }
+    const int co_t = co0 + wc * NT * 8 + 2 * tq;                    // this thread's first channel
+    if (p.acc) {
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
+        for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int pl = (wp_ * MT + mt) * 16 + half * 8 + g;
-            const int gp = gp_s[pl];
-            const bool pvalid = gp >= 0;
-            const size_t row_o = (size_t)(pvalid ? gp : 0) * p.Co + co0 + wc * NT * 8 + 2 * tq;
-            uint8_t* code_row = out_s + pl * ROWB + wc * NT * 8 + 2 * tq;
+            for (int half = 0; half < 2; ++half) {
+                const int gp = gp_s[(wp_ * MT + mt) * 16 + half * 8 + g];
+                int* row = p.acc + (size_t)(gp < 0 ? 0 : gp) * p.Co + co_t;
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
-                const int a0 = acc[mt][nt][half * 2], a1 = acc[mt][nt][half * 2 + 1];
-                const bool valid = pvalid && co < p.Co;
-                int code0 = 0, code1 = 0;
-                if (valid && p.acc) *reinterpret_cast<int2*>(p.acc + row_o + nt * 8) = make_int2(a0, a1);
-                if (want_y || want_q) {
-                    float y0 = __fmul_rn((float)a0, p.S), y1 = __fmul_rn((float)a1, p.S);
-                    if (p.ch_scale) { y0 = __fmul_rn(y0, cs[nt][0]); y1 = __fmul_rn(y1, cs[nt][1]); }
-                    if (p.ch_bias) { y0 = __fadd_rn(y0, cb[nt][0]); y1 = __fadd_rn(y1, cb[nt][1]); }
-                    if (p.relu) { y0 = y0 > 0.0f ? y0 : 0.0f; y1 = y1 > 0.0f ? y1 : 0.0f; }
-                    if (valid && want_y) *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
-                    if (valid && want_q) {
-                        code0 = quantize_act_code(y0, p.inv_next, qmax);
-                        code1 = quantize_act_code(y1, p.inv_next, qmax);
-                    }
-                }
-                if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
+                for (int nt = 0; nt < NT; ++nt)
+                    if (gp >= 0 && co_t + nt * 8 < p.Co)
+                        *reinterpret_cast<int2*>(row + nt * 8) = make_int2(acc[mt][nt][half * 2], acc[mt][nt][half * 2 + 1]);
             }
-        }
+    }
+    if (want_y || want_q) {
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int pl = (wp_ * MT + mt) * 16 + half * 8 + g;
+                const int gp = gp_s[pl];
+                float* yrow = p.y + (size_t)(gp < 0 ? 0 : gp) * p.Co + co_t;
+                uint8_t* code_row = out_s + pl * ROWB + wc * NT * 8 + 2 * tq;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const bool valid = gp >= 0 && co_t + nt * 8 < p.Co;
+                    float y0 = __fmul_rn((float)acc[mt][nt][half * 2], p.S), y1 = __fmul_rn((float)acc[mt][nt][half * 2 + 1], p.S);
+                    y0 = __fadd_rn(__fmul_rn(y0, cs[nt][0]), cb[nt][0]);
+                    y1 = __fadd_rn(__fmul_rn(y1, cs[nt][1]), cb[nt][1]);
+                    y0 = p.relu ? fmaxf(y0, 0.0f) : y0;
+                    y1 = p.relu ? fmaxf(y1, 0.0f) : y1;
+                    if (want_y && valid) *reinterpret_cast<float2*>(yrow + nt * 8) = make_float2(y0, y1);
+                    const int code0 = valid ? quantize_act_code(y0, p.inv_next, qmax) : 0;
+                    const int code1 = valid ? quantize_act_code(y1, p.inv_next, qmax) : 0;
+                    if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
+                }
+            }
     }
     if (want_q) {
         __syncthreads();
         constexpr int CWL = (TILE_C + 31) / 32;
         constexpr int NW = TILE_C >= 32 ? 8 : TILE_C / 4;           // code words per 32-channel group
+#pragma unroll 1
         for (int item = tid; item < TILE_P * CWL; item += NTH) {
             const int cwl = item / TILE_P, pl = item - cwl * TILE_P;
             const int gp = gp_s[pl], cwg = (co0 >> 5) + cwl;
@@ -282,6 +296,7 @@ conv_mma_strip_kernel(const ConvParams p) {
 #pragma unroll
             for (int k = 0; k < NW; ++k) codes[k] = row[k];
             uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + cwg) * p.next_bits;
+#pragma unroll 1
             for (int j = 0; j < p.next_bits; ++j) {
                 uint32_t word = 0u;
 #pragma unroll
