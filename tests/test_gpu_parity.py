@@ -105,10 +105,11 @@ def test_conv_all_bitwidth_pairs(ebs, U, oracle, wb, ab):
 
 
 @pytest.mark.parametrize("ab", range(1, 9))
-@pytest.mark.parametrize("c,co,k", [(40, 22, 3), (16, 16, 3), (8, 12, 3), (64, 64, 1), (100, 34, 3)])
+@pytest.mark.parametrize("c,co,k", [(40, 22, 3), (16, 16, 3), (12, 10, 3), (16, 14, 2), (8, 12, 3), (64, 64, 1), (100, 34, 3)])
 def test_warp_level_strip_kernel_all_activation_bitwidths(ebs, U, oracle, ab, c, co, k):
     """The warp-level strip variants (channel tile 16 / 32 / 64): every activation bitwidth, ragged channel tiles,
-    one, two and four taps per MMA step (c_in 40 / 16 / 8), with and without per-channel terms and packed output."""
+    one, two and four taps per MMA step (c_in 40 / 9-16 in the 16-byte-per-pixel form, odd and even tap counts / 8),
+    with and without per-channel terms and packed output."""
     rng = np.random.default_rng(100 * ab + c + co)
     wb = 1 + (ab + c) % 8
     pad = k // 2
