@@ -112,6 +112,7 @@ conv_mma_kernel(const ConvParams p) {
     const int co0 = blockIdx.y * TILE_C;
 
     // ---- tap table (kk = tap * CW + cw)
+#pragma unroll 1
     for (int kk = tid; kk < p.KK; kk += NTH) {
         const int tap = kk / p.CW, cw = kk - tap * p.CW;
         const int r = tap / p.kw, s = tap - r * p.kw;
@@ -161,6 +162,7 @@ conv_mma_kernel(const ConvParams p) {
         }
         // weights: the 32-byte rows (one s8 code per input channel) of channels co0 .. co0+TILE_C of every staged
         // reduction word, from the byte image; rows from c_out up to its multiple of 16 are zero there
+#pragma unroll 1
         for (int e = tid; e < KSTEP * TILE_C * 2; e += NTH) {
             const int q = e / (TILE_C * 2), rem = e - q * (TILE_C * 2), c = rem >> 1, half = rem & 1;
             const int kk = kk0 + q;
@@ -302,6 +304,7 @@ conv_mma_kernel(const ConvParams p) {
     const bool simple = pair_ok && !p.y_nchw;
     if (simple && p.res_packed) {
         constexpr int GROUPS = TILE_C / 8;
+#pragma unroll 1
         for (int e = tid; e < TILE_P * GROUPS; e += NTH) {
             const int pl = e / GROUPS, grp = e - pl * GROUPS;
             const int gp = tile_p0 + pl, c = co0 + 8 * grp;

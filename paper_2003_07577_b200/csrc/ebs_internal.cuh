@@ -193,6 +193,7 @@ __device__ __forceinline__ void pack_code_tile(const uint8_t* out_s, const ConvP
     constexpr int ROWB = code_row_bytes(TILE_C);
     constexpr int CWL = (TILE_C + 31) / 32;
     constexpr int NW = TILE_C >= 32 ? 8 : TILE_C / 4;           // code words per 32-channel group
+#pragma unroll 1
     for (int item = threadIdx.x; item < TILE_P * CWL; item += NTHREADS) {
         const int cwl = item / TILE_P, pl = item - cwl * TILE_P;
         const int gp = tile_p0 + pl, cwg = (co0 >> 5) + cwl;
@@ -202,6 +203,7 @@ __device__ __forceinline__ void pack_code_tile(const uint8_t* out_s, const ConvP
 #pragma unroll
         for (int k = 0; k < NW; ++k) codes[k] = row[k];
         uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + cwg) * p.next_bits;
+#pragma unroll 1
         for (int j = 0; j < p.next_bits; ++j) {
             uint32_t word = 0u;
 #pragma unroll
