@@ -220,12 +220,14 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
         if (strip >= 0 && p.CW * d->kh * d->kw >= 8 && conv_umma_resident_applies(p, strip)) variant = RES_BASE + strip;
         else if (strip >= 0) variant = STRIP_BASE + strip;
         else if (umma >= 0) variant = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + umma;
-        // small stride-1 layers with up to 32 output channels: the warp-level strip kernel (it expands every input
+        // small stride-1 layers with up to 64 output channels: the warp-level strip kernel (it expands every input
         // pixel once instead of once per tap, and its time does not grow with the plane count); 1x1 layers have
         // nothing to save there and stay on the per-tap kernel
         else if (mma_ok && p.Co <= 16 && p.P >= (1 << 16) && conv_mma_strip_applies(p, 0)) variant = MS_BASE;
         else if (mma_ok && p.Co > 16 && p.Co <= 32 && d->kh * d->kw > 1 && p.P >= (1 << 15) && conv_mma_strip_applies(p, 1))
             variant = MS_BASE + 1;
+        else if (mma_ok && p.Co > 32 && p.Co <= 64 && d->kh * d->kw > 1 && p.P >= (1 << 13) && conv_mma_strip_applies(p, 2))
+            variant = MS_BASE + 2;
         else variant = mma_ok ? NUM_CONV_VARIANTS + choose_mma_variant(d->w_bits, d->a_bits, p.P, p.Co, sm_count())
                               : choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
     }
