@@ -5,9 +5,9 @@ namespace ebs {
 
 template <int AB, int VARIANT>
 constexpr ConvVariant make_mma_strip_variant() {
-    // tile_c 16: 8 warps x (32 pixels x 16 channels); 32: 4 warps x (32 x 32); 64: 4 x 2 warps of (16 x 32)
+    // tile_c 16: 8 warps x (32 pixels x 16 channels); 32: 4 warps x (16 x 32); 64: 4 x 2 warps of (16 x 32)
     if constexpr (VARIANT == 0) return ConvVariant{&launch_conv_mma_strip<AB, 2, 2, 8, 1>, 256, 16, 256};
-    else if constexpr (VARIANT == 1) return ConvVariant{&launch_conv_mma_strip<AB, 2, 4, 4, 1>, 128, 32, 128};
+    else if constexpr (VARIANT == 1) return ConvVariant{&launch_conv_mma_strip<AB, 1, 4, 4, 1>, 64, 32, 128};
     else return ConvVariant{&launch_conv_mma_strip<AB, 1, 4, 4, 2>, 64, 64, 256};
 }
 

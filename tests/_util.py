@@ -126,7 +126,7 @@ def mma_strip_variant_applies(d, w, variant):
     pointwise = d.kh == 1 and d.kw == 1 and d.pad_h == 0 and d.pad_w == 0
     if (d.stride_h != 1 or d.stride_w != 1) and not pointwise:
         return False
-    tile_p, tile_c = ((256, 16), (128, 32), (64, 64))[variant]
+    tile_p, tile_c = ((256, 16), (64, 32), (64, 64))[variant]
     cw, taps = (d.c_in + 31) // 32, d.kh * d.kw
     strip = tile_p + (d.kh - 1) * (w + 2 * d.pad_w) + d.kw - 1
     pad = (strip + 7) // 8 * 8
