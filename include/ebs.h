@@ -195,8 +195,8 @@ int ebs_conv2d_mixed(const void *packed_x_dev, int n, int h, int w, const void *
  *   29..33  the same as persistent CTAs that keep the weight bytes of their channel tile in
  *           shared memory and overlap expansion, MMAs and epilogue of consecutive pixel tiles
  *           (layers whose weight tiles fit in 150 KB, w_levels = 0);
- *   34..36  warp-level kernels for small stride-1 layers (c_in 5..128, even c_out, no shortcut
- *           term, NHWC): the strip of input pixels expanded to bytes once per thread block,
+ *   34..36  warp-level kernels for small stride-1 layers (c_in 5..128, even c_out, NHWC
+ *           output): the strip of input pixels expanded to bytes once per thread block,
  *           fragments loaded from shared memory, weights from the byte image; channel tile
  *           16 / 32 / 64.
  * variant = -2 lets the library choose among the integer-pipe kernels only (the literal

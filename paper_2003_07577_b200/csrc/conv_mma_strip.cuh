@@ -37,12 +37,12 @@ inline MmaStripGeom mma_strip_geometry(const ConvParams& p, int tile_p, int tile
     const long long frame = (long long)p.N * strip_frame_h(p) * Wp;
     g.smem_bytes = p.CW * g.strip_pad * 32 + taps * p.CW * tile_c * 32 + tile_p * code_row_bytes(tile_c) + tile_p * 4 + 128;
     g.ok = ((p.sh == 1 && p.sw == 1) || strip_pointwise(p)) && p.CW <= 4 && taps * p.CW <= 64 && !p.w_levels &&
-           !p.residual && !p.res_packed && !p.y_nchw && (p.Co & 1) == 0 && p.fold <= 4 &&
+           !p.y_nchw && (p.Co & 1) == 0 && p.fold <= 4 &&
            g.smem_bytes <= 96 * 1024 && frame < (1LL << 31) - 4096;
     return g;
 }
 
-template <int AB, int MT, int NT, int WARPS_P, int WARPS_C, bool COMPACT = false>
+template <int AB, int MT, int NT, int WARPS_P, int WARPS_C, bool COMPACT = false, bool RES = false>
 __global__ void __launch_bounds__(32 * WARPS_P * WARPS_C)
 conv_mma_strip_kernel(const ConvParams p) {
     constexpr int NTH = 32 * WARPS_P * WARPS_C, TILE_P = 16 * MT * WARPS_P, TILE_C = 8 * NT * WARPS_C;
@@ -245,6 +245,28 @@ conv_mma_strip_kernel(const ConvParams p) {
         cb[nt][1] = (p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : -0.0f;
     }
     const int co_t = co0 + wc * NT * 8 + 2 * tq;                    // this thread's first channel
+    if (RES && p.res_packed) {                                      // shortcut codes of the tile, one per byte, into the code tile
+        constexpr int GROUPS = TILE_C / 8;
+#pragma unroll 1
+        for (int e = tid; e < TILE_P * GROUPS; e += NTH) {
+            const int pl = e / GROUPS, grp = e - pl * GROUPS;
+            const int gp = gp_s[pl], c = co0 + 8 * grp;
+            uint32_t lo = 0u, hi = 0u;                              // channels c .. c+3 and c+4 .. c+7
+            if (gp >= 0 && c < p.Co) {
+                const uint32_t* w = p.res_packed + ((size_t)gp * p.CWo + (c >> 5)) * p.res_bits;
+#pragma unroll 1
+                for (int j = 0; j < p.res_bits; ++j) {
+                    const uint32_t byte = (__ldg(w + j) >> (c & 31)) & 0xFFu;         // plane j of the eight channels
+                    lo |= (((byte & 0xFu) * 0x00204081u) & 0x01010101u) << j;          // bit i -> bit 8 i
+                    hi |= (((byte >> 4) * 0x00204081u) & 0x01010101u) << j;
+                }
+            }
+            uint32_t* dst = reinterpret_cast<uint32_t*>(out_s + pl * ROWB + 8 * grp);
+            dst[0] = lo;
+            dst[1] = hi;
+        }
+        __syncthreads();
+    }
     if (p.acc) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
@@ -273,6 +295,23 @@ conv_mma_strip_kernel(const ConvParams p) {
                     float y0 = __fmul_rn((float)acc[mt][nt][half * 2], p.S), y1 = __fmul_rn((float)acc[mt][nt][half * 2 + 1], p.S);
                     y0 = __fadd_rn(__fmul_rn(y0, cs[nt][0]), cb[nt][0]);
                     y1 = __fadd_rn(__fmul_rn(y1, cs[nt][1]), cb[nt][1]);
+                    float r0 = -0.0f, r1 = -0.0f;                    // the shortcut, if any, after the per-channel terms
+                    if constexpr (!RES) {
+                    } else if (p.residual) {
+                        if (valid) {
+                            const float2 r = __ldg(reinterpret_cast<const float2*>(p.residual + (size_t)gp * p.Co + co_t + nt * 8));
+                            r0 = r.x;
+                            r1 = r.y;
+                        }
+                    } else if (p.res_packed) {
+                        const uint32_t rc = *reinterpret_cast<const uint16_t*>(code_row + nt * 8);
+                        r0 = __fmul_rn(p.res_scale, (float)(rc & 0xFFu));
+                        r1 = __fmul_rn(p.res_scale, (float)(rc >> 8));
+                    }
+                    if constexpr (RES) {
+                        y0 = __fadd_rn(y0, r0);
+                        y1 = __fadd_rn(y1, r1);
+                    }
                     y0 = p.relu ? fmaxf(y0, 0.0f) : y0;
                     y1 = p.relu ? fmaxf(y1, 0.0f) : y1;
                     if (want_y && valid) *reinterpret_cast<float2*>(yrow + nt * 8) = make_float2(y0, y1);
@@ -318,26 +357,31 @@ void launch_conv_mma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st)
     if (!g.ok) return;                                        // callers check mma_strip_geometry first
     p.strip_pix = g.strip_pix;
     p.strip_ks = g.fold;
-    static bool attr_set[64] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaFuncSetAttribute(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             96 * 1024);
-        if constexpr (TILE_C == 16)
-            cudaFuncSetAttribute(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, true>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-        attr_set[dev] = true;
-    }
-    const long long frame = (long long)p.N * strip_frame_h(p) * strip_frame_w(p);
-    const dim3 grid((unsigned)((frame + TILE_P - 1) / TILE_P), (unsigned)((p.Co + TILE_C - 1) / TILE_C), 1);
-    if constexpr (TILE_C == 16) {                             // 9-16 input channels: the 16-byte-per-pixel form
-        if (g.fold == 2) {
-            conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, true><<<grid, 32 * WARPS_P * WARPS_C, g.smem_bytes, st>>>(p);
+    // four forms of the kernel: with or without a shortcut term (layers without one do not pay for it), and for the
+    // 16-channel tile the 16-byte-per-pixel form when the layer has 9-16 input channels
+    const bool res = p.residual || p.res_packed;
+    const bool compact = TILE_C == 16 && g.fold == 2;
+    static bool attr_set[4][64] = {};                           // per kernel form and device
+    auto go = [&](void (*kernel)(const ConvParams), int form) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (dev >= 0 && dev < 64 && !attr_set[form][dev]) {
+            cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+            attr_set[form][dev] = true;
+        }
+        const long long frame = (long long)p.N * strip_frame_h(p) * strip_frame_w(p);
+        const dim3 grid((unsigned)((frame + TILE_P - 1) / TILE_P), (unsigned)((p.Co + TILE_C - 1) / TILE_C), 1);
+        kernel<<<grid, 32 * WARPS_P * WARPS_C, g.smem_bytes, st>>>(p);
+    };
+    if constexpr (TILE_C == 16) {
+        if (compact) {
+            if (res) go(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, true, true>, 3);
+            else go(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, true, false>, 2);
             return;
         }
     }
-    conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C><<<grid, 32 * WARPS_P * WARPS_C, g.smem_bytes, st>>>(p);
+    if (res) go(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, false, true>, 1);
+    else go(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, false, false>, 0);
 }
 
 // Variants: channel tile 16 / 32 / 64, 256 frame pixels per CTA (8 warps).

@@ -121,8 +121,7 @@ def resident_variant_applies(d, w, tile_n):
 
 
 def mma_strip_variant_applies(d, w, variant):
-    """Host-side rule of the warp-level strip kernel (plain or per-channel epilogue only: callers that pass a
-    shortcut or ask for NCHW output must not force it)."""
+    """Host-side rule of the warp-level strip kernel (NHWC output only: callers that ask for NCHW must not force it)."""
     pointwise = d.kh == 1 and d.kw == 1 and d.pad_h == 0 and d.pad_w == 0
     if (d.stride_h != 1 or d.stride_w != 1) and not pointwise:
         return False
