@@ -239,10 +239,10 @@ conv_mma_strip_kernel(const ConvParams p) {
     for (int nt = 0; nt < NT; ++nt) {
         const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
         const bool in = co < p.Co;                                  // c_out is even: co + 1 exists with co
-        cs[nt][0] = (p.ch_scale && in) ? __ldg(p.ch_scale + co) : 1.0f;
-        cs[nt][1] = (p.ch_scale && in) ? __ldg(p.ch_scale + co + 1) : 1.0f;
-        cb[nt][0] = (p.ch_bias && in) ? __ldg(p.ch_bias + co) : -0.0f;
-        cb[nt][1] = (p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : -0.0f;
+        cs[nt][0] = (RES && p.ch_scale && in) ? __ldg(p.ch_scale + co) : 1.0f;
+        cs[nt][1] = (RES && p.ch_scale && in) ? __ldg(p.ch_scale + co + 1) : 1.0f;
+        cb[nt][0] = (RES && p.ch_bias && in) ? __ldg(p.ch_bias + co) : -0.0f;
+        cb[nt][1] = (RES && p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : -0.0f;
     }
     const int co_t = co0 + wc * NT * 8 + 2 * tq;                    // this thread's first channel
     if (RES && p.res_packed) {                                      // shortcut codes of the tile, one per byte, into the code tile
@@ -293,8 +293,10 @@ conv_mma_strip_kernel(const ConvParams p) {
                 for (int nt = 0; nt < NT; ++nt) {
                     const bool valid = gp >= 0 && co_t + nt * 8 < p.Co;
                     float y0 = __fmul_rn((float)acc[mt][nt][half * 2], p.S), y1 = __fmul_rn((float)acc[mt][nt][half * 2 + 1], p.S);
-                    y0 = __fadd_rn(__fmul_rn(y0, cs[nt][0]), cb[nt][0]);
-                    y1 = __fadd_rn(__fmul_rn(y1, cs[nt][1]), cb[nt][1]);
+                    if constexpr (RES) {
+                        y0 = __fadd_rn(__fmul_rn(y0, cs[nt][0]), cb[nt][0]);
+                        y1 = __fadd_rn(__fmul_rn(y1, cs[nt][1]), cb[nt][1]);
+                    }
                     float r0 = -0.0f, r1 = -0.0f;                    // the shortcut, if any, after the per-channel terms
                     if constexpr (!RES) {
                     } else if (p.residual) {
@@ -357,9 +359,9 @@ void launch_conv_mma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st)
     if (!g.ok) return;                                        // callers check mma_strip_geometry first
     p.strip_pix = g.strip_pix;
     p.strip_ks = g.fold;
-    // four forms of the kernel: with or without a shortcut term (layers without one do not pay for it), and for the
-    // 16-channel tile the 16-byte-per-pixel form when the layer has 9-16 input channels
-    const bool res = p.residual || p.res_packed;
+    // four forms of the kernel: with or without per-channel and shortcut terms (RES; layers without any do not pay
+    // for them), and for the 16-channel tile the 16-byte-per-pixel form when the layer has 9-16 input channels
+    const bool res = p.residual || p.res_packed || p.ch_scale || p.ch_bias;
     const bool compact = TILE_C == 16 && g.fold == 2;
     static bool attr_set[4][64] = {};                           // per kernel form and device
     auto go = [&](void (*kernel)(const ConvParams), int form) {
