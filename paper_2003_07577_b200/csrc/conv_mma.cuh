@@ -94,7 +94,9 @@ struct MmaTile {
     static_assert(SMEM_WORDS * 4 + MMA_KTAB * 8 <= 47 * 1024, "static shared memory budget");
 };
 
-template <int AB, int MT, int NT, int WARPS_P, int WARPS_C>
+// FULL = false: the form for even c_out, NHWC and no per-channel or shortcut terms (chosen on the host), which leaves
+// out their instructions and the general epilogue.
+template <int AB, int MT, int NT, int WARPS_P, int WARPS_C, bool FULL>
 __global__ void __launch_bounds__(32 * WARPS_P * WARPS_C)
 conv_mma_kernel(const ConvParams p) {
     using T = MmaTile<AB, MT, NT, WARPS_P, WARPS_C>;
@@ -301,8 +303,8 @@ conv_mma_kernel(const ConvParams p) {
     }
     // common case: even c_out and NHWC -> two-channel vectors, per-channel terms kept in registers, the
     // shortcut codes (if the shortcut comes as packed planes) staged as bytes in the code tile
-    const bool simple = pair_ok && !p.y_nchw;
-    if (simple && p.res_packed) {
+    const bool simple = !FULL || (pair_ok && !p.y_nchw);
+    if (FULL && simple && p.res_packed) {
         constexpr int GROUPS = TILE_C / 8;
 #pragma unroll 1
         for (int e = tid; e < TILE_P * GROUPS; e += NTH) {
@@ -333,10 +335,10 @@ conv_mma_kernel(const ConvParams p) {
         for (int nt = 0; nt < NT; ++nt) {
             const int co = co0 + (wc * NT + nt) * 8 + 2 * tq;
             const bool in = co < p.Co;                          // c_out is even here: co + 1 exists with co
-            cs[nt][0] = (p.ch_scale && in) ? __ldg(p.ch_scale + co) : 1.0f;
-            cs[nt][1] = (p.ch_scale && in) ? __ldg(p.ch_scale + co + 1) : 1.0f;
-            cb[nt][0] = (p.ch_bias && in) ? __ldg(p.ch_bias + co) : -0.0f;
-            cb[nt][1] = (p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : -0.0f;
+            cs[nt][0] = (FULL && p.ch_scale && in) ? __ldg(p.ch_scale + co) : 1.0f;
+            cs[nt][1] = (FULL && p.ch_scale && in) ? __ldg(p.ch_scale + co + 1) : 1.0f;
+            cb[nt][0] = (FULL && p.ch_bias && in) ? __ldg(p.ch_bias + co) : -0.0f;
+            cb[nt][1] = (FULL && p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : -0.0f;
         }
         const int co_t = co0 + wc * NT * 8 + 2 * tq;            // this thread's first channel
         if (p.acc) {
@@ -365,10 +367,13 @@ conv_mma_kernel(const ConvParams p) {
                     for (int nt = 0; nt < NT; ++nt) {
                         const bool valid = gp < p.P && co_t + nt * 8 < p.Co;
                         float y0 = __fmul_rn((float)acc[mt][nt][half * 2], p.S), y1 = __fmul_rn((float)acc[mt][nt][half * 2 + 1], p.S);
-                        y0 = __fadd_rn(__fmul_rn(y0, cs[nt][0]), cb[nt][0]);
-                        y1 = __fadd_rn(__fmul_rn(y1, cs[nt][1]), cb[nt][1]);
+                        if constexpr (FULL) {
+                            y0 = __fadd_rn(__fmul_rn(y0, cs[nt][0]), cb[nt][0]);
+                            y1 = __fadd_rn(__fmul_rn(y1, cs[nt][1]), cb[nt][1]);
+                        }
                         float r0 = -0.0f, r1 = -0.0f;
-                        if (p.residual) {
+                        if constexpr (!FULL) {
+                        } else if (p.residual) {
                             if (valid) {
                                 const float2 r = __ldg(reinterpret_cast<const float2*>(p.residual + row_o + nt * 8));
                                 r0 = r.x;
@@ -379,8 +384,10 @@ conv_mma_kernel(const ConvParams p) {
                             r0 = __fmul_rn(p.res_scale, (float)(rc & 0xFFu));
                             r1 = __fmul_rn(p.res_scale, (float)(rc >> 8));
                         }
-                        y0 = __fadd_rn(y0, r0);
-                        y1 = __fadd_rn(y1, r1);
+                        if constexpr (FULL) {
+                            y0 = __fadd_rn(y0, r0);
+                            y1 = __fadd_rn(y1, r1);
+                        }
                         y0 = p.relu ? fmaxf(y0, 0.0f) : y0;
                         y1 = p.relu ? fmaxf(y1, 0.0f) : y1;
                         if (want_y && valid) *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
@@ -390,7 +397,7 @@ conv_mma_kernel(const ConvParams p) {
                     }
                 }
         }
-    } else {
+    } else if constexpr (FULL) {
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
@@ -464,7 +471,9 @@ conv_mma_kernel(const ConvParams p) {
 
 template <int AB, int MT, int NT, int WARPS_P, int WARPS_C>
 void launch_conv_mma(const ConvParams& p, dim3 grid, cudaStream_t st) {
-    conv_mma_kernel<AB, MT, NT, WARPS_P, WARPS_C><<<grid, 32 * WARPS_P * WARPS_C, 0, st>>>(p);
+    const bool full = p.ch_scale || p.ch_bias || p.residual || p.res_packed || p.y_nchw || (p.Co & 1);
+    if (full) conv_mma_kernel<AB, MT, NT, WARPS_P, WARPS_C, true><<<grid, 32 * WARPS_P * WARPS_C, 0, st>>>(p);
+    else conv_mma_kernel<AB, MT, NT, WARPS_P, WARPS_C, false><<<grid, 32 * WARPS_P * WARPS_C, 0, st>>>(p);
 }
 
 // Variants: variant = size_class * 3 + tile_c_index, tile_c in {16, 32, 64}.
