@@ -38,9 +38,15 @@ inline MmaStripGeom mma_strip_geometry(const ConvParams& p, int tile_p, int tile
     g.smem_bytes = p.CW * g.strip_pad * 32 + taps * p.CW * tile_c * 32 + tile_p * code_row_bytes(tile_c) + tile_p * 4 + 128;
     g.ok = ((p.sh == 1 && p.sw == 1) || strip_pointwise(p)) && p.CW <= 4 && taps * p.CW <= 64 && !p.w_levels &&
            !p.y_nchw && (p.Co & 1) == 0 && p.fold <= 4 &&
-           g.smem_bytes <= 96 * 1024 && frame < (1LL << 31) - 4096;
+           g.smem_bytes <= 96 * 1024 && frame < (1LL << 31) - 4096 &&
+           Wp < (1 << 15) && strip_frame_h(p) < (1 << 15) && g.strip_pix * p.CW < (1 << 15);   // small_div operands
     return g;
 }
+
+// floor(a / d) for 0 <= a < 2^20 and 1 <= d < 2^16 from the correctly rounded reciprocal of d: (a + 0.5) / d is at
+// least 0.5 / d away from every integer and the two roundings move it by less than (a + d) 2^-23, so the floor of the
+// product is the quotient (four instructions instead of a 32-bit integer division).
+__device__ __forceinline__ int small_div(int a, float rcp_d) { return __float2int_rd(__fmul_rn((float)a + 0.5f, rcp_d)); }
 
 template <int AB, int MT, int NT, int WARPS_P, int WARPS_C, bool COMPACT = false, bool RES = false>
 __global__ void __launch_bounds__(32 * WARPS_P * WARPS_C)
@@ -93,14 +99,20 @@ conv_mma_strip_kernel(const ConvParams p) {
     for (int t = tid; t < taps; t += NTH) tap_shift_s[t] = (t / p.kw) * Wp + (t % p.kw);
 
     // ---- the strip: packed words -> bytes, once per pixel and word
+    // frame coordinates of the tile's first pixel (two integer divisions a thread); the pixels after it are reached
+    // with small quotients only
+    const int n0 = f0 / (Hp * Wp), rem0 = f0 - n0 * (Hp * Wp);
+    const int hp0 = rem0 / Wp, wq0 = rem0 - hp0 * Wp;
+    const float rcp_w = __frcp_rn((float)Wp), rcp_h = __frcp_rn((float)Hp), rcp_cw = __frcp_rn((float)p.CW);
 #pragma unroll 1
     for (int e = tid; e < S * p.CW; e += NTH) {
-        const int s = e / p.CW, cw = e - s * p.CW;
+        const int s = COMPACT ? e : small_div(e, rcp_cw), cw = COMPACT ? 0 : e - s * p.CW;
         const int f = f0 + s;
         uint32_t r[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
         if (f < frame) {
-            const int n = f / (Hp * Wp), rem = f - n * (Hp * Wp);
-            const int hp = rem / Wp, wq = rem - hp * Wp;
+            const int cw_ = small_div(wq0 + s, rcp_w), wq = wq0 + s - cw_ * Wp;      // column, carry into the row
+            const int ch_ = small_div(hp0 + cw_, rcp_h), hp = hp0 + cw_ - ch_ * Hp;  // row, carry into the image
+            const int n = n0 + ch_;
             const int h = pointwise ? hp * p.sh : hp - p.ph, w = pointwise ? wq * p.sw : wq - p.pw;
             if ((unsigned)h < (unsigned)p.H && (unsigned)w < (unsigned)p.W) {
                 uint32_t words[AB];
@@ -129,8 +141,9 @@ conv_mma_strip_kernel(const ConvParams p) {
         const int f = f0 + pl;
         int gp = -1;
         if (f < frame) {
-            const int n = f / (Hp * Wp), rem = f - n * (Hp * Wp);
-            const int hp = rem / Wp, wq = rem - hp * Wp;
+            const int cw_ = small_div(wq0 + pl, rcp_w), wq = wq0 + pl - cw_ * Wp;
+            const int ch_ = small_div(hp0 + cw_, rcp_h), hp = hp0 + cw_ - ch_ * Hp;
+            const int n = n0 + ch_;
             if (hp < p.Ho && wq < p.Wo) gp = (n * p.Ho + hp) * p.Wo + wq;
         }
         gp_s[pl] = gp;
