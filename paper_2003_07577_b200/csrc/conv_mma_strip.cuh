@@ -294,6 +294,7 @@ conv_mma_strip_kernel(const ConvParams p) {
             }
     }
     if (want_y || want_q) {
+        const float relu_lo = p.relu ? 0.0f : -INFINITY;
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -327,11 +328,21 @@ conv_mma_strip_kernel(const ConvParams p) {
                         y0 = __fadd_rn(y0, r0);
                         y1 = __fadd_rn(y1, r1);
                     }
-                    y0 = p.relu ? fmaxf(y0, 0.0f) : y0;
-                    y1 = p.relu ? fmaxf(y1, 0.0f) : y1;
+                    int code0, code1;
+                    if constexpr (RES) {
+                        y0 = p.relu ? fmaxf(y0, 0.0f) : y0;
+                        y1 = p.relu ? fmaxf(y1, 0.0f) : y1;
+                        code0 = valid ? quantize_act_code(y0, p.inv_next, qmax) : 0;
+                        code1 = valid ? quantize_act_code(y1, p.inv_next, qmax) : 0;
+                    } else {
+                        // plain form: y = acc * S is finite (the host checks S), so max(y, -inf) is y; rows and channels
+                        // past the layer have zero accumulators (zero weight rows), hence zero codes, without a select
+                        y0 = fmaxf(y0, relu_lo);
+                        y1 = fmaxf(y1, relu_lo);
+                        code0 = quantize_act_code(y0, p.inv_next, qmax);
+                        code1 = quantize_act_code(y1, p.inv_next, qmax);
+                    }
                     if (want_y && valid) *reinterpret_cast<float2*>(yrow + nt * 8) = make_float2(y0, y1);
-                    const int code0 = valid ? quantize_act_code(y0, p.inv_next, qmax) : 0;
-                    const int code1 = valid ? quantize_act_code(y1, p.inv_next, qmax) : 0;
                     if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
                 }
             }
@@ -374,7 +385,7 @@ void launch_conv_mma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st)
     p.strip_ks = g.fold;
     // four forms of the kernel: with or without per-channel and shortcut terms (RES; layers without any do not pay
     // for them), and for the 16-channel tile the 16-byte-per-pixel form when the layer has 9-16 input channels
-    const bool res = p.residual || p.res_packed || p.ch_scale || p.ch_bias;
+    const bool res = p.residual || p.res_packed || p.ch_scale || p.ch_bias || !isfinite(p.S);
     const bool compact = TILE_C == 16 && g.fold == 2;
     static bool attr_set[4][64] = {};                           // per kernel form and device
     auto go = [&](void (*kernel)(const ConvParams), int form) {
