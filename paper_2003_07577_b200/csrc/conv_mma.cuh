@@ -94,8 +94,8 @@ struct MmaTile {
     static_assert(SMEM_WORDS * 4 + MMA_KTAB * 8 <= 47 * 1024, "static shared memory budget");
 };
 
-// FULL = false: the form for even c_out, NHWC and no per-channel or shortcut terms (chosen on the host), which leaves
-// out their instructions and the general epilogue.
+// FULL = false: the form for even c_out, NHWC, two's-complement weight codes and no per-channel or shortcut terms
+// (chosen on the host), which leaves out their instructions and the general epilogue.
 template <int AB, int MT, int NT, int WARPS_P, int WARPS_C, bool FULL>
 __global__ void __launch_bounds__(32 * WARPS_P * WARPS_C)
 conv_mma_kernel(const ConvParams p) {
@@ -355,6 +355,7 @@ conv_mma_kernel(const ConvParams p) {
                 }
         }
         if (want_y || want_q) {
+            const float relu_lo = p.relu ? 0.0f : -INFINITY;
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -388,11 +389,21 @@ conv_mma_kernel(const ConvParams p) {
                             y0 = __fadd_rn(y0, r0);
                             y1 = __fadd_rn(y1, r1);
                         }
-                        y0 = p.relu ? fmaxf(y0, 0.0f) : y0;
-                        y1 = p.relu ? fmaxf(y1, 0.0f) : y1;
+                        int code0, code1;
+                        if constexpr (FULL) {
+                            y0 = p.relu ? fmaxf(y0, 0.0f) : y0;
+                            y1 = p.relu ? fmaxf(y1, 0.0f) : y1;
+                            code0 = valid ? quantize_act_code(y0, p.inv_next, qmax) : 0;
+                            code1 = valid ? quantize_act_code(y1, p.inv_next, qmax) : 0;
+                        } else {
+                            // plain form: y = acc * S is finite (the host checks S), so max(y, -inf) is y; channels past
+                            // the layer have zero weight rows, hence zero codes, and pixels past it are never packed
+                            y0 = fmaxf(y0, relu_lo);
+                            y1 = fmaxf(y1, relu_lo);
+                            code0 = quantize_act_code(y0, p.inv_next, qmax);
+                            code1 = quantize_act_code(y1, p.inv_next, qmax);
+                        }
                         if (want_y && valid) *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
-                        const int code0 = valid ? quantize_act_code(y0, p.inv_next, qmax) : 0;
-                        const int code1 = valid ? quantize_act_code(y1, p.inv_next, qmax) : 0;
                         if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
                     }
                 }
@@ -471,7 +482,8 @@ conv_mma_kernel(const ConvParams p) {
 
 template <int AB, int MT, int NT, int WARPS_P, int WARPS_C>
 void launch_conv_mma(const ConvParams& p, dim3 grid, cudaStream_t st) {
-    const bool full = p.ch_scale || p.ch_bias || p.residual || p.res_packed || p.y_nchw || (p.Co & 1);
+    const bool full = p.ch_scale || p.ch_bias || p.residual || p.res_packed || p.y_nchw || (p.Co & 1) || p.w_levels ||
+                      !isfinite(p.S);
     if (full) conv_mma_kernel<AB, MT, NT, WARPS_P, WARPS_C, true><<<grid, 32 * WARPS_P * WARPS_C, 0, st>>>(p);
     else conv_mma_kernel<AB, MT, NT, WARPS_P, WARPS_C, false><<<grid, 32 * WARPS_P * WARPS_C, 0, st>>>(p);
 }
