@@ -12,8 +12,13 @@
 // (c_in <= 128), so there is no staging pipeline.  Layers with at most 16 (8) input channels use only byte
 // lanes 0-1 (0) of every register; there two (four) taps share one MMA step, the later tap's registers
 // shifted left by 16 (8, 16, 24) bits, for both operands alike.
+// COMPACT form (9-16 input channels, one word): 16 bytes per pixel and per weight row, so K positions 0-15 of an MMA
+// step are one tap and 16-31 the next -- two taps per step without shifts and half the shared loads.
 // Epilogue as in conv_mma_kernel (accumulator pairs, fp32 steps, code tile, multiply-gather pack), with the
-// output pixel of a frame row looked up in a per-CTA table (rows with hp >= Ho or wp >= Wo have none).
+// output pixel of a frame row looked up in a per-CTA table (rows with hp >= Ho or wp >= Wo have none).  The RES
+// form carries the per-channel terms and the shortcut (fp32 or packed codes); the plain form, which the host picks
+// when none of them is passed, leaves their instructions out.  These launches last a few microseconds and are
+// bound by instruction issue and fetch, so the epilogue is one straight-line block and set-up loops are not unrolled.
 #pragma once
 
 #include <type_traits>
