@@ -113,11 +113,13 @@ conv_mma_strip_kernel(const ConvParams p) {
     for (int e = tid; e < S * p.CW; e += NTH) {
         const int s = COMPACT ? e : small_div(e, rcp_cw), cw = COMPACT ? 0 : e - s * p.CW;
         const int f = f0 + s;
-        uint32_t r[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+        uint32_t r[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};          // COMPACT uses r[0..3]: the four 4-channel words
+        int gp = -1;
         if (f < frame) {
             const int cw_ = small_div(wq0 + s, rcp_w), wq = wq0 + s - cw_ * Wp;      // column, carry into the row
             const int ch_ = small_div(hp0 + cw_, rcp_h), hp = hp0 + cw_ - ch_ * Hp;  // row, carry into the image
             const int n = n0 + ch_;
+            if (hp < p.Ho && wq < p.Wo) gp = (n * p.Ho + hp) * p.Wo + wq;            // the output pixel of this frame row
             const int h = pointwise ? hp * p.sh : hp - p.ph, w = pointwise ? wq * p.sw : wq - p.pw;
             if ((unsigned)h < (unsigned)p.H && (unsigned)w < (unsigned)p.W) {
                 uint32_t words[AB];
@@ -125,33 +127,28 @@ conv_mma_strip_kernel(const ConvParams p) {
 #pragma unroll
                 for (int k = 0; k < AB; ++k) {
                     const uint32_t mask = 0x01010101u << k;
+                    if constexpr (COMPACT) {
+                        // bits 0-3 / 8-11 / 4-7 / 12-15 of the word to the low nibbles of bytes 0 / 1 / 2 / 3, then bit j
+                        // of every byte to bit k of word j: bytes = channels j, 8+j, 4+j, 12+j
+                        const uint32_t u = (words[k] & 0x0F0Fu) | ((words[k] & 0xF0F0u) << 12);
 #pragma unroll
-                    for (int b = 0; b < 8; ++b) r[b] |= __funnelshift_r(words[k], words[k], b - k) & mask;
+                        for (int j = 0; j < 4; ++j) r[j] |= __funnelshift_r(u, u, j - k) & mask;
+                    } else {
+#pragma unroll
+                        for (int b = 0; b < 8; ++b) r[b] |= __funnelshift_r(words[k], words[k], b - k) & mask;
+                    }
                 }
             }
         }
+        if (cw == 0 && s < TILE_P) gp_s[s] = gp;
         if constexpr (COMPACT) {
-            reinterpret_cast<uint4*>(strip)[s] = make_uint4(__byte_perm(r[0], r[4], 0x5410), __byte_perm(r[1], r[5], 0x5410),
-                                                            __byte_perm(r[2], r[6], 0x5410), __byte_perm(r[3], r[7], 0x5410));
+            reinterpret_cast<uint4*>(strip)[s] = make_uint4(r[0], r[1], r[2], r[3]);
         } else {
             uint4* dst = reinterpret_cast<uint4*>(strip + (cw * SP + s) * 32);
             const int sw = (s >> 2) & 1;
             dst[sw] = make_uint4(r[0], r[1], r[2], r[3]);
             dst[sw ^ 1] = make_uint4(r[4], r[5], r[6], r[7]);
         }
-    }
-    // ---- output pixel of each row of the tile
-#pragma unroll 1
-    for (int pl = tid; pl < TILE_P; pl += NTH) {
-        const int f = f0 + pl;
-        int gp = -1;
-        if (f < frame) {
-            const int cw_ = small_div(wq0 + pl, rcp_w), wq = wq0 + pl - cw_ * Wp;
-            const int ch_ = small_div(hp0 + cw_, rcp_h), hp = hp0 + cw_ - ch_ * Hp;
-            const int n = n0 + ch_;
-            if (hp < p.Ho && wq < p.Wo) gp = (n * p.Ho + hp) * p.Wo + wq;
-        }
-        gp_s[pl] = gp;
     }
     cp_async_wait<0>();
     __syncthreads();
