@@ -45,7 +45,7 @@ WORKLOADS = {
 SM_COUNT, POPC_LANES_PER_CLK_SM = 148, 16
 # dram__bytes_read.sum + dram__bytes_write.sum per conv launch, mean over the 20 layers, from the ncu
 # capture summarised in profiles/ (outputs stay in the 126 MB L2 while ncu replays a launch)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 689471
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 689207
 
 
 def measured_peaks():
