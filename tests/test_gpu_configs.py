@@ -77,6 +77,34 @@ def test_config2_resnet20_full_batch(ebs, U, oracle, gen):
         check_layer(ebs, U, oracle, spec, gen.act_codes(spec), gen.weight_codes(spec), next_bits=max(1, spec.a_bits % 5))
 
 
+def test_config2_in_the_bench_launch_configuration(ebs, U, oracle, gen):
+    """The 20 quantized layers at batch 128 exactly as bench.py launches them: no per-channel term, ReLU, int32
+    accumulators plus the next layer's planes (its bit count, step 4 * s_w * s_a * c_in), the library's own kernel
+    choice -- the form of the kernels without per-channel and shortcut terms. Every output is checked."""
+    specs = [s for s in gen.config2(0) if s.layer.quantized]
+    assert len(specs) == 20
+    for i, spec in enumerate(specs):
+        L = spec.layer
+        next_bits = specs[(i + 1) % len(specs)].a_bits
+        next_scale = np.float32(4.0 * spec.w_scale * spec.a_scale * L.c_in)
+        qa, qw = gen.act_codes(spec), gen.weight_codes(spec)
+        d = U.spec_desc(spec)
+        px, pw = U.pack_acts_codes(qa, spec.a_bits, ebs.EBS_NHWC), U.pack_weight_codes(qw, d)
+        ref = oracle.conv2d_codes(qa, qw, (L.stride, L.stride), (L.pad, L.pad))
+        S = oracle.combined_scale(spec.w_scale, spec.a_scale)
+        _, q_ref = oracle.epilogue(ref, S, None, None, None, relu=True, next_bits=next_bits,
+                                   inv_next=np.float32(1.0) / next_scale)
+        epi = ebs.epilogue(relu=True, next_a_bits=next_bits, next_a_scale=float(next_scale))
+        acc, _, pn = U.conv_on_device(px, spec.batch, L.h_in, L.w_in, pw, d, epi, True, False, next_bits)
+        torch.cuda.synchronize()
+        idx = list(range(spec.batch))
+        assert np.array_equal(U.images_nchw(acc, idx), ref), f"{L.name}: int32 accumulators"
+        got_q = oracle.unpack_acts(U.packed_images(pn, spec.batch, L.h_out, L.w_out, L.c_out, next_bits, idx), L.c_out)
+        assert np.array_equal(got_q, q_ref), f"{L.name}: requantized codes"
+        assert np.array_equal(pn.cpu().numpy().view(np.uint32).ravel(),
+                              oracle.pack_acts(q_ref, next_bits).ravel()), f"{L.name}: packed words (pad bits zero)"
+
+
 def test_config3_resnet18_batch64_sampled_images(ebs, U, oracle, gen):
     for spec in gen.config3(0):
         qa = gen.act_codes(spec)
