@@ -282,7 +282,9 @@ conv_mma_strip_kernel(const ConvParams p) {
         }
         __syncthreads();
     }
-    if (p.acc) {
+    // plain form with further outputs: the accumulators are stored from the loop below (one table look-up a row)
+    const bool acc_inline = !RES && p.acc && (want_y || want_q);
+    if (p.acc && !acc_inline) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -308,6 +310,11 @@ conv_mma_strip_kernel(const ConvParams p) {
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     const bool valid = gp >= 0 && co_t + nt * 8 < p.Co;
+                    if constexpr (!RES) {
+                        if (acc_inline && valid)
+                            *reinterpret_cast<int2*>(p.acc + (size_t)gp * p.Co + co_t + nt * 8) =
+                                make_int2(acc[mt][nt][half * 2], acc[mt][nt][half * 2 + 1]);
+                    }
                     float y0 = __fmul_rn((float)acc[mt][nt][half * 2], p.S), y1 = __fmul_rn((float)acc[mt][nt][half * 2 + 1], p.S);
                     if constexpr (RES) {
                         y0 = __fadd_rn(__fmul_rn(y0, cs[nt][0]), cb[nt][0]);
