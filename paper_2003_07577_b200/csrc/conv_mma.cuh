@@ -341,7 +341,9 @@ conv_mma_kernel(const ConvParams p) {
             cb[nt][1] = (FULL && p.ch_bias && in) ? __ldg(p.ch_bias + co + 1) : -0.0f;
         }
         const int co_t = co0 + wc * NT * 8 + 2 * tq;            // this thread's first channel
-        if (p.acc) {
+        // plain form with further outputs: the accumulators are stored from the loop below
+        const bool acc_inline = !FULL && p.acc && (want_y || want_q);
+        if (p.acc && !acc_inline) {
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -367,6 +369,11 @@ conv_mma_kernel(const ConvParams p) {
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
                         const bool valid = gp < p.P && co_t + nt * 8 < p.Co;
+                        if constexpr (!FULL) {
+                            if (acc_inline && valid)
+                                *reinterpret_cast<int2*>(p.acc + row_o + nt * 8) =
+                                    make_int2(acc[mt][nt][half * 2], acc[mt][nt][half * 2 + 1]);
+                        }
                         float y0 = __fmul_rn((float)acc[mt][nt][half * 2], p.S), y1 = __fmul_rn((float)acc[mt][nt][half * 2 + 1], p.S);
                         if constexpr (FULL) {
                             y0 = __fadd_rn(__fmul_rn(y0, cs[nt][0]), cb[nt][0]);
