@@ -1,19 +1,25 @@
 #!/usr/bin/env python
-"""Benchmark of the bit-plane mixed-precision convolution path on the CIFAR ResNet-20 stack.
+"""Benchmark of the bit-plane mixed-precision convolution path on the five workloads.
 
-A step is one pass of the whole path over one batch of 128 synthetic images: for each of the 20
-quantized convolution layers, activation quantize+pack (ebs_pack_acts), the bit-plane convolution
-with fused epilogue writing int32 accumulators and the next layer's packed planes
-(ebs_conv2d_mixed), and the stand-alone de-quantization (ebs_dequant).  Weight packing is done once
-before timing (it is off the inference path).  Prints one JSON line.
+The default run (one GPU) times all five configurations in one process and prints ONE JSON line.
+The headline (`value`, `ms_per_step`, `roofline`, `e2e`, `cpu_baseline`) is configuration 5, the
+largest single-GPU workload: the ImageNet ResNet-50 bottleneck stack at batch 256, 52 convolution
+layers chained through fused requantization.  A step is one pass of the whole path over one batch:
+ebs_pack_acts at the network entry, one ebs_conv2d_mixed per layer whose epilogue writes the next
+layer's packed planes, ebs_dequant of the last layer's accumulators at the exit; weight packing is
+done once before timing (it is off the inference path).  `per_config` holds, for each of the five
+configurations, the step time, binary and int8 TOPS, the roofline fractions in both output modes
+(raw: int32 accumulators + packed planes; fused: packed planes only), cold and warm L2, the literal
+AND+POPC path against the POPC pipe, and the CPU oracle timed on a stated sample.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload configN]
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import re
 import sys
 import threading
 import time
@@ -27,25 +33,19 @@ import torch  # noqa: E402
 
 from workloads import gen  # noqa: E402
 
-METRIC = "effective binary TOPS (2*MACs*Wb*Ab per second), ResNet-20 CIFAR quantized conv stack"
+METRIC = "effective binary TOPS (2*MACs*Wb*Ab per second) of the mixed-precision conv stack"
 UNIT = "TOPS"
-WORKLOAD = "config2: ResNet-20 CIFAR-shaped stack, 20 quantized convs, batch 128, (Wb,Ab) in {1..4}^2, seed 0"
-# other workloads of the same path, for profiling and for the results table (the default is config2)
-WORKLOADS = {
-    "config2": (WORKLOAD, lambda: [s for s in gen.config2(0) if s.layer.quantized]),
-    "config1": ("config1: one 3x3 conv 64->64, 32x32, batch 1, W2A2, seed 0", lambda: gen.config1(0)),
-    "config3": ("config3: ResNet-18 ImageNet-shaped quantized convs, batch 64, (Wb,Ab) in {2..6}^2, seed 0",
-                lambda: gen.config3(0)),
-    "config4": ("config4: 4096^3 bit-plane GEMM as a 1x1 convolution over 64x64 pixels, seven (Wb,Ab) pairs of the sweep, seed 0",
-                lambda: [gen.config4(wb, ab) for wb, ab in [(1, 1), (2, 2), (4, 4), (8, 8), (1, 8), (8, 1), (3, 5)]]),
-    "config5": ("config5: ResNet-50 ImageNet-shaped bottleneck stack, batch 256, (Wb,Ab) in {2..8}^2, seed 0 "
-                "(layers run with independent inputs here; the chained run is a parity test)",
-                lambda: gen.config5(0)),
+HEADLINE = "config5"
+WORKLOAD_TEXT = {
+    "config1": "config1: one 3x3 conv 64->64, 32x32, batch 1, W2A2, seed 0",
+    "config2": "config2: ResNet-20 CIFAR-shaped stack, 20 quantized convs, batch 128, (Wb,Ab) in {1..4}^2, seed 0",
+    "config3": "config3: ResNet-18 ImageNet-shaped quantized convs, batch 64, (Wb,Ab) in {2..6}^2, seed 0",
+    "config4": "config4: 4096^3 bit-plane GEMM as a 1x1 convolution over 64x64 pixels, all 64 (Wb,Ab) pairs, seed 0",
+    "config5": "config5: ResNet-50 ImageNet-shaped bottleneck stack, 52 convs, batch 256, (Wb,Ab) in {2..8}^2, seed 0, "
+               "chained through fused requantization",
 }
 SM_COUNT, POPC_LANES_PER_CLK_SM = 148, 16
-# dram__bytes_read.sum + dram__bytes_write.sum per conv launch, mean over the 20 layers, from the ncu
-# capture summarised in profiles/ (outputs stay in the 126 MB L2 while ncu replays a launch)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 689207
+TRAFFIC_PROFILE = os.path.join(ROOT, "profiles", "conv_dram_traffic.md")
 
 
 def measured_peaks():
@@ -61,13 +61,20 @@ def int8_tensor_peak_tops(peaks: dict) -> float:
     return 2.0 * float(peaks.get("bf16_tflops", 1590.0))
 
 
-def hbm_gbs_for_streaming(peaks: dict) -> float:
-    return float(peaks.get("hbm_gbs", 6650.0))
-
-
 def popc_pipe_peak_tops(sm_max_mhz: float) -> float:
     """Binary TOPS of the POPC pipe: 16 lanes/clk/SM x 32 bit x 148 SMs x clock, 2 ops per bit pair."""
     return 2.0 * SM_COUNT * POPC_LANES_PER_CLK_SM * 32 * sm_max_mhz * 1e6 / 1e12
+
+
+def ncu_traffic_per_launch(workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per conv launch for a workload, from the committed ncu summary
+    (a line `traffic_bytes_per_launch[<workload>] = <integer>`); None if the summary has no such line."""
+    try:
+        with open(TRAFFIC_PROFILE) as f:
+            m = re.search(r"traffic_bytes_per_launch\[%s\]\s*=\s*(\d+)" % re.escape(workload), f.read())
+        return int(m.group(1)) if m else None
+    except OSError:
+        return None
 
 
 class ClockSampler(threading.Thread):
@@ -113,53 +120,99 @@ class ClockSampler(threading.Thread):
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+# ---------------------------------------------------------------------------- workloads (layer lists, wiring)
+
+def workload_specs(name: str):
+    """(specs, chained) of a configuration; chained: layer l+1 reads layer l's packed output."""
+    if name == "config1":
+        return gen.config1(0), False
+    if name == "config2":
+        return [s for s in gen.config2(0) if s.layer.quantized], False
+    if name == "config3":
+        return gen.config3(0), False
+    if name == "config4":
+        return [gen.config4(wb, ab) for wb in range(1, 9) for ab in range(1, 9)], False
+    if name == "config5":
+        return gen.config5(0), True
+    raise KeyError(name)
+
+
+def consumer_bits(specs, i, chained):
+    """Activation bitwidth the output of layer i is requantized to: that of the layer that reads it."""
+    if not chained:
+        return specs[(i + 1) % len(specs)].a_bits
+    j = i + 1
+    while j < len(specs) and specs[j].layer.role == "shortcut":
+        j += 1
+    return specs[j].a_bits if j < len(specs) else specs[i].a_bits
+
+
 # ---------------------------------------------------------------------------- GPU arm
 
 class Layer:
     """Device buffers and descriptors of one layer (plumbing only)."""
 
-    def __init__(self, ebs, spec, next_bits, dev):
+    def __init__(self, ebs, spec, next_bits, dev, px=None, qa=None, qw_dev=None, pw=None, want_host=False):
         L = spec.layer
         self.spec, self.n, self.next_bits = spec, spec.batch, next_bits
         self.d = ebs.conv_desc(L.c_in, L.c_out, L.k, L.k, L.stride, L.stride, L.pad, L.pad, spec.w_bits, spec.a_bits,
                                spec.w_scale, spec.a_scale)
-        qa = gen.act_codes(spec).astype(np.uint8)
-        self.x_host = torch.from_numpy(np.ascontiguousarray(qa.transpose(0, 2, 3, 1))).pin_memory()   # NHWC codes
-        self.x = self.x_host.to(dev)
-        qw = torch.from_numpy(gen.weight_codes(spec).astype(np.int8)).to(dev)
-        self.pw = torch.empty(ebs.ebs_packed_weight_bytes(self.d) // 4, dtype=torch.int32, device=dev)
-        ebs.ebs_pack_weights(qw, ebs.EBS_I8_CODES, ebs.EBS_NCHW, self.d, self.pw)
-        self.px = torch.empty(ebs.ebs_packed_act_bytes(self.n, L.h_in, L.w_in, L.c_in, spec.a_bits) // 4,
-                              dtype=torch.int32, device=dev)
+        self.x = self.x_host = None
+        self.px_bytes = ebs.ebs_packed_act_bytes(self.n, L.h_in, L.w_in, L.c_in, spec.a_bits)
+        if px is None:                                              # an input of its own: generator codes, packed here
+            qa = gen.act_codes(spec).astype(np.uint8) if qa is None else qa
+            xh = torch.from_numpy(np.ascontiguousarray(qa.transpose(0, 2, 3, 1)))    # NHWC codes
+            self.x_host = xh.pin_memory() if want_host else xh
+            self.x = self.x_host.to(dev)
+            px = torch.empty(self.px_bytes // 4, dtype=torch.int32, device=dev)
+        self.px = px
+        if pw is None:
+            qw_dev = torch.from_numpy(gen.weight_codes(spec).astype(np.int8)).to(dev) if qw_dev is None else qw_dev
+            pw = torch.empty(ebs.ebs_packed_weight_bytes(self.d) // 4, dtype=torch.int32, device=dev)
+            ebs.ebs_pack_weights(qw_dev, ebs.EBS_I8_CODES, ebs.EBS_NCHW, self.d, pw)
+        self.pw = pw
         ho, wo = L.h_out, L.w_out
         self.pixels = self.n * ho * wo
-        self.acc = torch.empty((self.n, ho, wo, L.c_out), dtype=torch.int32, device=dev)
-        self.y = torch.empty((self.n, ho, wo, L.c_out), dtype=torch.float32, device=dev)
+        self.outputs = self.pixels * L.c_out
+        self.acc = None                                             # allocated by want_acc()
         self.pn_bytes = ebs.ebs_packed_act_bytes(self.n, ho, wo, L.c_out, next_bits)
         self.pn = torch.empty(self.pn_bytes // 4, dtype=torch.int32, device=dev)
-        self.pn_host = torch.empty(self.pn_bytes // 4, dtype=torch.int32).pin_memory()
-        self.epi = ebs.epilogue(relu=True, next_a_bits=next_bits, next_a_scale=4.0 * spec.w_scale * spec.a_scale * L.c_in)
+        self.next_scale = 4.0 * spec.w_scale * spec.a_scale * L.c_in
+        self.epi = ebs.epilogue(relu=True, next_a_bits=next_bits, next_a_scale=self.next_scale)
         self.S = float(np.float32(spec.w_scale) * np.float32(spec.a_scale))
         self.ops = gen.binary_ops(spec)
-        self.ws_bytes = ebs.ebs_host_workspace_bytes(self.d, self.n, L.h_in, L.w_in, ebs.EBS_U8_CODES, next_bits)
+        self.int8_ops = self.ops // (spec.w_bits * spec.a_bits)    # 2 * MACs
+        co16 = (L.c_out + 15) // 16 * 16
+        self.w_plane_bytes = ebs.ebs_packed_weight_plane_bytes(self.d)
+        self.w_image_bytes = L.k * L.k * ((L.c_in + 31) // 32) * co16 * 32
+        self.dev = dev
+
+    def want_acc(self):
+        if self.acc is None:
+            L = self.spec.layer
+            self.acc = torch.empty((self.n, L.h_out, L.w_out, L.c_out), dtype=torch.int32, device=self.dev)
+        return self.acc
+
+    def set_step(self, ebs, step: float):
+        self.next_scale = float(step)
+        self.epi = ebs.epilogue(relu=True, next_a_bits=self.next_bits, next_a_scale=self.next_scale)
 
     def run_pack(self, ebs):
         L = self.spec.layer
         ebs.ebs_pack_acts(self.x, ebs.EBS_U8_CODES, ebs.EBS_NHWC, self.n, L.c_in, L.h_in, L.w_in, self.spec.a_bits,
                           self.spec.a_scale, self.px)
 
-    def run_dequant(self, ebs):
-        ebs.ebs_dequant(self.acc, self.pixels, self.spec.layer.c_out, self.S, None, None, True, self.y)
-
-    def run_conv_only(self, ebs, variant=-1):
+    def run_conv(self, ebs, raw: bool, variant=-1):
         L = self.spec.layer
-        ebs.ebs_conv2d_mixed(self.px, self.n, L.h_in, L.w_in, self.pw, self.d, self.epi, self.acc, None, self.pn,
-                             variant=variant)
+        ebs.ebs_conv2d_mixed(self.px, self.n, L.h_in, L.w_in, self.pw, self.d, self.epi, self.want_acc() if raw else None,
+                             None, self.pn, variant=variant)
 
-    def run_host(self, ebs, ws, stream=None):
-        L = self.spec.layer
-        ebs.ebs_conv2d_mixed_host(self.x_host, ebs.EBS_U8_CODES, ebs.EBS_NHWC, self.n, L.h_in, L.w_in, self.pw, self.d,
-                                  self.epi, ws, None, None, self.pn_host, stream=stream)
+    def bytes_alg(self, raw: bool, literal: bool = False):
+        """Algorithmic bytes of one launch: packed input planes + weights as the kernel family reads them (bit planes for
+        the integer-pipe kernels, the byte image for the tensor-pipe kernels) + packed output planes (+ int32
+        accumulators in raw mode)."""
+        w = self.w_plane_bytes if literal else self.w_image_bytes
+        return self.px_bytes + w + self.pn_bytes + (4 * self.outputs if raw else 0)
 
 
 def dist_setup(n_gpus: int):
@@ -191,67 +244,336 @@ def barrier():
         dist.barrier()
 
 
-class OracleWorkload:
-    """The CPU oracle on (a batch slice of) the same workload; codes are generated outside the timing."""
+# ---------------------------------------------------------------------------- CPU oracle arm
 
-    def __init__(self, batch: int):
+ORACLE_SAMPLES = {
+    # workload: (what one pass runs, how it scales to the full workload)
+    "config1": "the layer at full size (batch 1)",
+    "config2": "all 20 quantized layers at batch {b} of 128",
+    "config3": "all 19 layers at batch {b} of 64 (scaled from subset)",
+    "config4": "the W4A4 GEMM on {b} of 4096 rows (scaled from subset; the integer oracle's time does not depend on the bitwidths)",
+    "config5": "all 52 layers at batch {b} of 256, each on generator codes (scaled from subset)",
+}
+
+
+class OracleWorkload:
+    """The CPU oracle on a bounded sample of a workload; codes are generated outside the timing."""
+
+    def __init__(self, workload: str, batch: int):
         import oracle
         oracle.build()
-        self.oracle, self.batch = oracle, batch
-        self.specs = [s for s in gen.config2(0) if s.layer.quantized]
-        self.data = [(gen.act_codes(s, batch=batch), gen.weight_codes(s)) for s in self.specs]
-        self.ops = sum(gen.binary_ops(s, batch=batch) for s in self.specs)
+        self.oracle, self.workload, self.batch = oracle, workload, batch
+        if workload == "config4":
+            spec = gen.config4(4, 4)
+            rows = batch                                       # `batch` counts GEMM rows here: 1 x rows pixels
+            qa = gen.act_codes(spec)[:, :, :1, :rows]
+            self.specs, self.data = [spec], [(np.ascontiguousarray(qa), gen.weight_codes(spec))]
+            self.ops = 2 * rows * spec.layer.c_in * spec.layer.c_out * 16
+            self.next_bits = [4]
+        else:
+            self.specs, chained = workload_specs(workload)
+            b = min(batch, self.specs[0].batch)
+            self.batch = b
+            self.data = [(gen.act_codes(s, batch=b), gen.weight_codes(s)) for s in self.specs]
+            self.ops = sum(gen.binary_ops(s, batch=b) for s in self.specs)
+            self.next_bits = [consumer_bits(self.specs, i, chained) for i in range(len(self.specs))]
 
     def step(self) -> float:
         t0 = time.perf_counter()
-        for s, (qa, qw) in zip(self.specs, self.data):
+        for s, (qa, qw), nb in zip(self.specs, self.data, self.next_bits):
             L = s.layer
             acc = self.oracle.conv2d_codes(qa, qw, (L.stride, L.stride), (L.pad, L.pad))
-            self.oracle.epilogue(acc, self.oracle.combined_scale(s.w_scale, s.a_scale), relu=True)
+            step = np.float32(4.0 * s.w_scale * s.a_scale * L.c_in)
+            self.oracle.epilogue(acc, self.oracle.combined_scale(s.w_scale, s.a_scale), relu=True, next_bits=nb,
+                                 inv_next=np.float32(1.0) / step)
         return time.perf_counter() - t0
 
+    def describe(self) -> str:
+        return ORACLE_SAMPLES[self.workload].format(b=self.batch)
 
-def oracle_batch_for(budget_s: float, n_steps: int) -> int:
-    """Largest batch (<= 128) for which n_steps oracle passes fit the time budget."""
-    probe = OracleWorkload(2)
+
+def oracle_sample_size(workload: str, budget_s: float, n_steps: int) -> int:
+    """Largest sample (images, or GEMM rows for config4) for which n_steps oracle passes fit the time budget."""
+    if workload == "config1":
+        return 1
+    # upper limits keep the generation of the sample's codes (host, untimed) and the run within minutes
+    full = {"config2": 128, "config3": 8, "config4": 256, "config5": 4}[workload]
+    small = {"config2": 2, "config3": 1, "config4": 16, "config5": 1}[workload]
+    probe = OracleWorkload(workload, small)
     probe.step()
-    per_image = probe.step() / 2
-    return int(max(1, min(128, budget_s / max(n_steps, 1) / per_image)))
+    per_unit = probe.step() / small
+    return int(max(small, min(full, budget_s / max(n_steps, 1) / per_unit)))
 
 
-def cpu_baseline_sample(budget_s: float = 15.0):
+def cpu_baseline_sample(workload: str, budget_s: float):
     """The oracle, as it stands, timed on this host's cores on a bounded sample (a reported baseline)."""
-    wl = OracleWorkload(oracle_batch_for(budget_s, 3))
+    wl = OracleWorkload(workload, oracle_sample_size(workload, budget_s, 3))
     wl.step()
-    times = [wl.step() for _ in range(2)]
+    reps = 20 if workload == "config1" else 2
+    times = [wl.step() for _ in range(reps)]
     dt = float(np.mean(times))
     return {"value": wl.ops / dt / 1e12, "unit": UNIT, "cores": wl.oracle.num_threads(), "kind": "oracle",
-            "sample": f"all 20 quantized layers at batch {wl.batch} of 128 (direct integer conv + fp32 epilogue), "
-                      f"mean of 2 passes of {dt:.2f} s"}
+            "sample": f"{wl.describe()}: direct integer conv + fp32 epilogue with requantization, "
+                      f"mean of {reps} passes of {dt:.3f} s"}
 
 
 def run_reference(args):
     rank, world, _ = dist_setup(args.gpus)
     if rank != 0:
         return
-    wl = OracleWorkload(oracle_batch_for(150.0, args.steps + args.warmup))
+    workload = HEADLINE if args.workload == "all" else args.workload
+    wl = OracleWorkload(workload, oracle_sample_size(workload, 120.0, args.steps + args.warmup))
     for _ in range(args.warmup):
         wl.step()
     times = [wl.step() for _ in range(args.steps)]
     dt = float(np.mean(times))
     value = wl.ops / dt / 1e12
     base = {"value": value, "unit": UNIT, "cores": wl.oracle.num_threads(), "kind": "oracle",
-            "sample": f"each step: all 20 quantized layers at batch {wl.batch} of 128"}
+            "sample": f"each step: {wl.describe()}"}
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "sample_batch": wl.batch},
+            "config": {"workload": WORKLOAD_TEXT[workload], "sample": wl.describe()},
             "cpu_baseline": base,
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
 
-def network_leg(ebs, dev, stream, flush, capture, reps):
+# ---------------------------------------------------------------------------- measurement helpers
+
+class Timer:
+    def __init__(self, stream, flush):
+        self.stream, self.flush = stream, flush
+
+    def graph_ms(self, graph, reps: int, cold: bool) -> float:
+        """Mean CUDA-event time of one replay; cold = the 256 MB flush buffer is rewritten before every replay."""
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        if not cold:
+            graph.replay()
+        for e0, e1 in ev:
+            if cold:
+                self.flush.zero_()
+            e0.record(self.stream)
+            graph.replay()
+            e1.record(self.stream)
+        torch.cuda.synchronize()
+        return float(np.mean([e0.elapsed_time(e1) for e0, e1 in ev]))
+
+
+def capture(fn):
+    """Records fn's launches into a CUDA graph so that replay is not bound by host launch overhead."""
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        fn()                                                    # warm-up on the capture stream
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(g):
+        fn()
+    return g
+
+
+def build_layers(ebs, name, dev, want_host=False):
+    """Layers of a workload with their device buffers; chained workloads share buffers along the chain."""
+    specs, chained = workload_specs(name)
+    layers = []
+    if name == "config4":
+        # one activation tensor per Ab and one weight tensor per Wb serve the 64 pairs
+        acts, wts = {}, {}
+        for ab in range(1, 9):
+            s = gen.config4(1, ab)
+            first = Layer(ebs, s, ab, dev)
+            first.run_pack(ebs)
+            acts[ab] = first.px
+        for wb in range(1, 9):
+            wts[wb] = torch.from_numpy(gen.weight_codes(gen.config4(wb, 1)).astype(np.int8)).to(dev)
+        for i, s in enumerate(specs):
+            layers.append(Layer(ebs, s, s.a_bits, dev, px=acts[s.a_bits], qw_dev=wts[s.w_bits]))
+        torch.cuda.synchronize()
+        return specs, layers, chained
+    block_in = None
+    for i, s in enumerate(specs):
+        nb = consumer_bits(specs, i, chained)
+        if not chained or i == 0:
+            L = Layer(ebs, s, nb, dev, want_host=want_host)
+            L.run_pack(ebs)
+        else:
+            prev = next(p for p in reversed(layers) if p.spec.layer.role != "shortcut")
+            src = block_in if s.layer.role == "shortcut" else prev.pn
+            L = Layer(ebs, s, nb, dev, px=src)
+        if chained and s.layer.name.endswith("c1"):
+            block_in = L.px
+        layers.append(L)
+    torch.cuda.synchronize()
+    return specs, layers, chained
+
+
+def calibrate_chain(ebs, layers):
+    """Requantization steps of a chained stack, fixed once before timing (set-up, untimed): each layer's step maps
+    the 99.5th percentile of its ReLU output (sampled) onto the top code, so that the codes handed down the chain
+    use their whole range.  torch is used for the percentile only."""
+    for L in layers:
+        lay = L.spec.layer
+        y = torch.empty((L.n, lay.h_out, lay.w_out, lay.c_out), dtype=torch.float32, device=L.dev)
+        epi = ebs.epilogue(relu=True)
+        ebs.ebs_conv2d_mixed(L.px, L.n, lay.h_in, lay.w_in, L.pw, L.d, epi, None, y, None)
+        flat = y.flatten()
+        sample = flat[:: max(1, flat.numel() // (1 << 20))].float()
+        top = float(torch.quantile(sample, 0.995).item())
+        L.set_step(ebs, max(top, 1e-6) / ((1 << L.next_bits) - 1))
+        del y, flat, sample
+        L.run_conv(ebs, raw=False)                              # the next layer calibrates on this output
+    torch.cuda.synchronize()
+
+
+def layer_roofs(L: Layer, raw: bool, peak_tops: float, hbm_gbs: float):
+    t_tensor = L.int8_ops / (peak_tops * 1e12)
+    t_hbm = L.bytes_alg(raw) / (hbm_gbs * 1e9)
+    return t_tensor, t_hbm
+
+
+def measure_config(ebs, name, dev, timer, peaks, args, sm_max, detail: bool):
+    """All numbers of one configuration (see the module docstring)."""
+    peak_tops, hbm_gbs = int8_tensor_peak_tops(peaks), float(peaks.get("hbm_gbs", 6650.0))
+    specs, layers, chained = build_layers(ebs, name, dev)
+    if chained:
+        calibrate_chain(ebs, layers)
+    step_raw = not chained                       # the chained stack hands packed planes down; the others also keep int32 results
+    total_ops = sum(L.ops for L in layers)
+    total_int8 = sum(L.int8_ops for L in layers)
+    n_img = specs[0].batch
+    last = layers[-1]
+    y_exit = torch.empty((last.pixels, last.spec.layer.c_out), dtype=torch.float32, device=dev)
+
+    def one_step():
+        layers[0].run_pack(ebs) if layers[0].x is not None else None
+        for L in layers[:-1]:
+            L.run_conv(ebs, raw=step_raw)
+        last.run_conv(ebs, raw=True)                            # the exit layer's accumulators feed ebs_dequant
+        ebs.ebs_dequant(last.want_acc(), last.pixels, last.spec.layer.c_out, last.S, None, None, True, y_exit)
+
+    launches_per_step = len(layers) + 1 + (1 if layers[0].x is not None else 0)
+    reps_inner = 1000 if name == "config1" else 1              # a one-layer step is timed as 1000 back-to-back launches
+    step_graph = capture(lambda: [one_step() for _ in range(reps_inner)])
+    reps = max(3, min(args.steps, 20))
+    out = {"workload": WORKLOAD_TEXT[name], "layers": len(layers), "batch": n_img,
+           "step": ("pack at the entry, %d fused conv launches (%s), dequant at the exit"
+                    % (len(layers), "int32 accumulators + packed planes" if step_raw else "packed planes only, chained")),
+           "launches_per_step": launches_per_step}
+    if name == "config1":
+        out["step"] += "; timed as 1000 back-to-back steps in one graph, per-step time reported"
+    step_ms = timer.graph_ms(step_graph, reps, cold=True) / reps_inner
+    out["ms_per_step"] = step_ms
+    out["binary_tops"] = total_ops / (step_ms * 1e-3) / 1e12
+    out["int8_tops"] = total_int8 / (step_ms * 1e-3) / 1e12
+    out["imgs_per_s"] = n_img / (step_ms * 1e-3)
+
+    # the conv launches alone, both output modes, cold (flush before every replay) and warm (replays back to back)
+    modes = {}
+    per_layer = {}
+    for mode, raw in (("raw", True), ("fused", False)):
+        g = capture(lambda raw=raw: [[L.run_conv(ebs, raw=raw) for L in layers] for _ in range(reps_inner)])
+        cold = timer.graph_ms(g, reps, cold=True) / reps_inner
+        warm = timer.graph_ms(g, reps, cold=False) / reps_inner
+        del g
+        # per-layer times: each layer's launch 10 times back to back in a graph (L2-warm)
+        lay_ms = np.zeros(len(layers))
+        for i, L in enumerate(layers):
+            gl = capture(lambda L=L, raw=raw: [L.run_conv(ebs, raw=raw) for _ in range(10)])
+            lay_ms[i] = timer.graph_ms(gl, 2, cold=False) / 10.0
+            del gl
+        roofs = [layer_roofs(L, raw, peak_tops, hbm_gbs) for L in layers]
+        roof_s = np.array([max(r) for r in roofs])
+        sum_tensor, sum_hbm = sum(r[0] for r in roofs), sum(r[1] for r in roofs)
+        fr = roof_s * 1e3 / lay_ms
+        bytes_alg = sum(L.bytes_alg(raw) for L in layers)
+        modes[mode] = {
+            "outputs": "int32 accumulators + packed planes" if raw else "packed planes only",
+            "conv_ms_cold": cold, "conv_ms_warm": warm, "sum_layer_ms_warm": float(lay_ms.sum()),
+            "sum_layer_roofs_ms": float(roof_s.sum() * 1e3),
+            "bound": "tensor" if sum_tensor >= sum_hbm else "hbm",
+            "sum_tensor_roofs_ms": sum_tensor * 1e3, "sum_hbm_roofs_ms": sum_hbm * 1e3,
+            "frac_cold": float(roof_s.sum() * 1e3 / cold), "frac_warm": float(roof_s.sum() * 1e3 / warm),
+            "frac_of_layer_roofs": float(roof_s.sum() * 1e3 / lay_ms.sum()),
+            "layer_frac_min": float(fr.min()), "layer_frac_max": float(fr.max()),
+            "layers_at_or_above_half": int((fr >= 0.5).sum()),
+            "algorithmic_bytes": int(bytes_alg), "gbs_cold": bytes_alg / (cold * 1e-3) / 1e9,
+            "int8_tops_cold": total_int8 / (cold * 1e-3) / 1e12, "binary_tops_cold": total_ops / (cold * 1e-3) / 1e12,
+        }
+        per_layer[mode] = [
+            {"name": L.spec.layer.name, "wb": L.spec.w_bits, "ab": L.spec.a_bits, "us": round(float(t) * 1e3, 2),
+             "tops": round(L.ops / (t * 1e-3) / 1e12, 1), "int8_tops": round(L.int8_ops / (t * 1e-3) / 1e12, 1),
+             "bytes": int(L.bytes_alg(raw)), "roof_us": round(float(r) * 1e6, 2),
+             "roof": "tensor" if rr[0] >= rr[1] else "hbm", "frac_of_roof": round(float(f), 3)}
+            for L, t, r, rr, f in zip(layers, lay_ms, roof_s, roofs, fr)]
+    out["modes"] = modes
+    if detail or name in ("config1", "config4"):
+        out["per_layer"] = per_layer
+    else:
+        out["per_layer"] = {m: [{k: pl[k] for k in ("name", "wb", "ab", "us", "frac_of_roof")} for pl in v]
+                            for m, v in per_layer.items()}
+
+    # the same conv launches on the integer-pipe kernels only: the plane-pair double sum evaluated literally
+    # (AND + POPC + shift-add per plane pair), held against the POPC pipe's peak
+    lit_graph = capture(lambda: [L.run_conv(ebs, raw=True, variant=-2) for L in layers])
+    lit_reps = 1 if name in ("config4", "config5") else 3
+    lit_ms = timer.graph_ms(lit_graph, lit_reps, cold=True)
+    del lit_graph
+    popc_peak = popc_pipe_peak_tops(sm_max)
+    out["literal_bitplane_path"] = {
+        "kernel": "conv_popc_kernel (variant -2: the library's choice among the integer-pipe kernels), raw outputs",
+        "conv_ms": lit_ms, "binary_tops": total_ops / (lit_ms * 1e-3) / 1e12, "popc_pipe_peak_tops": popc_peak,
+        "frac_of_popc_pipe": total_ops / (lit_ms * 1e-3) / 1e12 / popc_peak}
+    return out, layers, step_graph, one_step, launches_per_step, total_ops, total_int8
+
+
+def streaming_leg(ebs, dev, stream, hbm_gbs):
+    """The streaming kernels (rows a2 and a6, search-stage forward) on a tensor far larger than L2: achieved GB/s of
+    algorithmic bytes."""
+    sn, sh, sc, sab = 256, 56, 64, 4                                   # ResNet-50 layer-1 activations: 51 M values
+    vals = sn * sh * sh * sc
+    xf = torch.rand((sn, sh, sh, sc), dtype=torch.float32, device=dev)
+    xu = torch.randint(0, 16, (sn, sh, sh, sc), dtype=torch.uint8, device=dev)
+    pk = torch.empty(ebs.ebs_packed_act_bytes(sn, sh, sh, sc, sab) // 4, dtype=torch.int32, device=dev)
+    ai = torch.randint(-1000, 1000, (sn * sh * sh, sc), dtype=torch.int32, device=dev)
+    yo = torch.empty((sn * sh * sh, sc), dtype=torch.float32, device=dev)
+
+    def gbs(fn, nbytes, reps=10):
+        fn()
+        tot = 0.0
+        for _ in range(reps):                                       # inputs are larger than L2: no flush needed
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            tot += a.elapsed_time(b)
+        return nbytes / (tot / reps * 1e-3) / 1e9
+
+    out_b = vals * sab // 8
+    res = {
+        "tensor": f"{sn}x{sh}x{sh}x{sc} NHWC, {sab} planes", "hbm_peak_gbs": hbm_gbs,
+        "pack_acts_fp32_gbs": gbs(lambda: ebs.ebs_pack_acts(xf, ebs.EBS_F32, ebs.EBS_NHWC, sn, sc, sh, sh, sab, 0.07, pk),
+                                  vals * 4 + out_b),
+        "pack_acts_u8_gbs": gbs(lambda: ebs.ebs_pack_acts(xu, ebs.EBS_U8_CODES, ebs.EBS_NHWC, sn, sc, sh, sh, sab, 1.0, pk),
+                                vals + out_b),
+        "pack_acts_fp32_nchw_gbs": gbs(lambda: ebs.ebs_pack_acts(xf, ebs.EBS_F32, ebs.EBS_NCHW, sn, sc, sh, sh, sab, 0.07, pk),
+                                       vals * 4 + out_b),
+        "dequant_gbs": gbs(lambda: ebs.ebs_dequant(ai, sn * sh * sh, sc, 0.01, None, None, True, yo), vals * 8),
+    }
+    # search-stage forward (Eq. 6-7), five candidate bitwidths: 4 B in + 4 B out per value; the weight form
+    # reads the tensor once more for max|w|
+    cand_bits, cand_coeff = [1, 2, 3, 4, 5], [0.1, 0.15, 0.4, 0.25, 0.1]
+    scratch = torch.zeros(4, dtype=torch.int32, device=dev)
+    xo = torch.empty_like(xf)
+    res["search_act_forward_gbs"] = gbs(lambda: ebs.ebs_search_act_forward(xf, 6.0, cand_bits, cand_coeff, xo), vals * 8)
+    res["search_weight_forward_gbs"] = gbs(
+        lambda: ebs.ebs_search_weight_forward(xf, cand_bits, cand_coeff, xo, scratch), vals * 12)
+    return res
+
+
+def network_leg(ebs, dev, stream, flush, reps):
     """ResNet-20 forward passes per second at batch 128 through paper_2003_07577_b200.network."""
     from paper_2003_07577_b200.network import BasicBlockNet, FusedBasicBlockNet, calibrated_plans
     from types import SimpleNamespace
@@ -328,50 +650,32 @@ def run_gpu(args):
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
     peaks, peak_kind = measured_peaks()
-
-    workload_text, make_specs = WORKLOADS[args.workload]
-    specs = make_specs()                                            # every rank: one full batch (weak scaling)
-    if args.only:                                                   # profiling aid: a subset of the layers
-        specs = [s for s in specs if s.layer.name in args.only.split(",")]
-    layers = [Layer(ebs, s, specs[(i + 1) % len(specs)].a_bits, dev) for i, s in enumerate(specs)]
-    ws = torch.empty(max(L.ws_bytes for L in layers), dtype=torch.uint8, device=dev)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
-    total_ops = sum(L.ops for L in layers)
     stream = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
+    timer = Timer(stream, flush)
+    sm_max = float(peaks.get("sm_max_mhz", 1965.0))
+    headline = HEADLINE if args.workload == "all" else args.workload
+    others = [c for c in ("config1", "config2", "config3", "config4") if c != headline] \
+        if (args.workload == "all" and world == 1) else []
 
-    def one_step():
-        # the path as a network runs it: activations are quantized and packed once, at the entry (row a2); every
-        # layer is one fused launch whose epilogue writes the int32 accumulators and the next layer's planes
-        # (rows a3-a5); the accumulators are de-quantized once, at the exit (row a6)
-        layers[0].run_pack(ebs)
-        for L in layers:
-            L.run_conv_only(ebs)
-        layers[-1].run_dequant(ebs)
+    # ---- the other configurations first (their buffers are released before the headline workload is built)
+    per_config = {}
+    for name in others:
+        res, layers, g, _, _, _, _ = measure_config(ebs, name, dev, timer, peaks, args, sm_max, detail=False)
+        if not args.no_cpu_baseline:
+            res["cpu_baseline"] = cpu_baseline_sample(name, 4.0)
+        per_config[name] = res
+        del layers, g
+        torch.cuda.empty_cache()
 
-    def capture(fn):
-        """Records fn's launches into a CUDA graph so that replay is not bound by host launch overhead."""
-        g = torch.cuda.CUDAGraph()
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            fn()                                                    # warm-up on the capture stream
-        torch.cuda.current_stream().wait_stream(side)
-        torch.cuda.synchronize()
-        with torch.cuda.graph(g):
-            fn()
-        return g
-
-    for L in layers:                                                # every layer's resident planes (set-up, untimed)
-        L.run_pack(ebs)
+    # ---- the headline configuration: the timed steps of the contract
+    res, layers, step_graph, one_step, launches_per_step, total_ops, total_int8 = measure_config(
+        ebs, headline, dev, timer, peaks, args, sm_max, detail=True)
+    chained = headline == "config5"
+    inner = 1000 if headline == "config1" else 1
     for _ in range(max(args.warmup, 3)):
-        one_step()
-    torch.cuda.synchronize()
-    step_graph = capture(one_step)
-    conv_graph = capture(lambda: [L.run_conv_only(ebs) for L in layers])
-    for _ in range(3):
         step_graph.replay()
     torch.cuda.synchronize()
-
     sampler = ClockSampler(local)
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     barrier()
@@ -386,130 +690,69 @@ def run_gpu(args):
     torch.cuda.synchronize()
     wall = time.perf_counter() - wall0
     barrier()
-    step_ms = [e0.elapsed_time(e1) for e0, e1 in ev]
-    total_ms = max_over_ranks(float(sum(step_ms)), dev)
-    ms_per_step = total_ms / args.steps
-
-    # dominant kernel (the bit-plane convolution) alone: the 20 conv launches of a step, cold L2 per replay
-    reps = max(3, min(args.steps, 20))
-    cev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
-    for e0, e1 in cev:
-        flush.zero_()
-        e0.record(stream)
-        conv_graph.replay()
-        e1.record(stream)
-    torch.cuda.synchronize()
-    conv_total_ms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in cev]))
+    total_ms = max_over_ranks(float(sum(e0.elapsed_time(e1) for e0, e1 in ev)), dev)
+    ms_per_step = total_ms / args.steps / inner
+    # the dominant kernel family (the bit-plane convolution) alone, in the step's output mode, cold L2, timed with
+    # CUDA events on the launching stream while the clock sampler still runs
+    mode = "fused" if chained else "raw"
+    conv_graph = capture(lambda: [[L.run_conv(ebs, raw=not chained) for L in layers] for _ in range(inner)])
+    conv_ms = timer.graph_ms(conv_graph, max(3, min(args.steps, 20)), cold=True) / inner
     clocks = sampler.stop()
+    res["ms_per_step"] = ms_per_step
+    res["binary_tops"] = total_ops / (ms_per_step * 1e-3) / 1e12
+    res["int8_tops"] = total_int8 / (ms_per_step * 1e-3) / 1e12
+    res["imgs_per_s"] = layers[0].n / (ms_per_step * 1e-3)
 
-    # per-layer breakdown: each layer's conv launched 10 times back to back in a graph (L2-warm)
-    conv_ms = np.zeros(len(layers))
-    for i, L in enumerate(layers):
-        g = capture(lambda L=L: [L.run_conv_only(ebs) for _ in range(10)])
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        g.replay()
-        e0.record(stream)
-        g.replay()
-        e1.record(stream)
-        torch.cuda.synchronize()
-        conv_ms[i] = e0.elapsed_time(e1) / 10.0
-
-    # the same 20 conv launches on the integer-pipe kernels only: the plane-pair double sum evaluated
-    # literally (AND + POPC + shift-add per plane pair), held against the POPC pipe's peak
-    literal = {}
-    if world == 1:
-        lit_graph = capture(lambda: [L.run_conv_only(ebs, -2) for L in layers])
-        lev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
-        for e0, e1 in lev:
-            flush.zero_()
-            e0.record(stream)
-            lit_graph.replay()
-            e1.record(stream)
-        torch.cuda.synchronize()
-        lit_ms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in lev]))
-        literal = {"kernel": "conv_popc_kernel (variant -2: the library's choice among the integer-pipe kernels)",
-                   "conv_ms_per_step": lit_ms, "binary_tops": total_ops / (lit_ms * 1e-3) / 1e12}
-
-    # the streaming kernels (rows a2 and a6) on a tensor far larger than L2: achieved GB/s of algorithmic bytes
-    streaming = {}
-    if world == 1:
-        sn, sh, sc, sab = 256, 56, 64, 4                                   # ResNet-50 layer-1 activations: 51 M values, inputs > L2
-        vals = sn * sh * sh * sc
-        xf = torch.rand((sn, sh, sh, sc), dtype=torch.float32, device=dev)
-        xu = torch.randint(0, 16, (sn, sh, sh, sc), dtype=torch.uint8, device=dev)
-        pk = torch.empty(ebs.ebs_packed_act_bytes(sn, sh, sh, sc, sab) // 4, dtype=torch.int32, device=dev)
-        ai = torch.randint(-1000, 1000, (sn * sh * sh, sc), dtype=torch.int32, device=dev)
-        yo = torch.empty((sn * sh * sh, sc), dtype=torch.float32, device=dev)
-
-        def gbs(fn, nbytes, reps=10):
-            fn()
-            tot = 0.0
-            for _ in range(reps):                                       # inputs are larger than L2: no flush needed
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-                fn()
-                b.record(stream)
+    # ---- end to end: pinned host codes in, the stack on the device, the last layer's packed planes back on the host
+    first, last = layers[0], layers[-1]
+    e2e = None
+    if first.x is not None:
+        x_host = first.x_host if first.x_host.is_pinned() else first.x_host.pin_memory()
+        out_host = torch.empty(last.pn_bytes // 4, dtype=torch.int32).pin_memory()
+        if chained:
+            def e2e_step():
+                first.x.copy_(x_host, non_blocking=True)
+                first.run_pack(ebs)
+                for L in layers:
+                    L.run_conv(ebs, raw=False)
+                out_host.copy_(last.pn, non_blocking=True)
                 torch.cuda.synchronize()
-                tot += a.elapsed_time(b)
-            return nbytes / (tot / reps * 1e-3) / 1e9
+            h2d, d2h = x_host.numel(), last.pn_bytes
+            note = ("pinned u8 NHWC codes of the network input copied in, ebs_pack_acts, the 52 chained ebs_conv2d_mixed "
+                    "calls, the last layer's packed planes copied back; wall clock around every step")
+        else:
+            hosts = [(L, (L.x_host if L.x_host.is_pinned() else L.x_host.pin_memory()),
+                      torch.empty(L.pn_bytes // 4, dtype=torch.int32).pin_memory()) for L in layers]
+            ws = [torch.empty(max(ebs.ebs_host_workspace_bytes(L.d, L.n, L.spec.layer.h_in, L.spec.layer.w_in,
+                                                               ebs.EBS_U8_CODES, L.next_bits) for L in layers),
+                              dtype=torch.uint8, device=dev) for _ in range(3)]
+            streams = [torch.cuda.Stream() for _ in range(3)]
 
-        out_b = vals * sab // 8
-        streaming = {
-            "tensor": f"{sn}x{sh}x{sh}x{sc} NHWC, {sab} planes", "hbm_peak_gbs": hbm_gbs_for_streaming(peaks),
-            "pack_acts_fp32_gbs": gbs(lambda: ebs.ebs_pack_acts(xf, ebs.EBS_F32, ebs.EBS_NHWC, sn, sc, sh, sh, sab, 0.07, pk),
-                                      vals * 4 + out_b),
-            "pack_acts_u8_gbs": gbs(lambda: ebs.ebs_pack_acts(xu, ebs.EBS_U8_CODES, ebs.EBS_NHWC, sn, sc, sh, sh, sab, 1.0, pk),
-                                    vals + out_b),
-            "pack_acts_fp32_nchw_gbs": gbs(lambda: ebs.ebs_pack_acts(xf, ebs.EBS_F32, ebs.EBS_NCHW, sn, sc, sh, sh, sab, 0.07, pk),
-                                           vals * 4 + out_b),
-            "dequant_gbs": gbs(lambda: ebs.ebs_dequant(ai, sn * sh * sh, sc, 0.01, None, None, True, yo), vals * 8),
-        }
-        # search-stage forward (Eq. 6-7), five candidate bitwidths: 4 B in + 4 B out per value; the weight form
-        # reads the tensor once more for max|w|
-        cand_bits, cand_coeff = [1, 2, 3, 4, 5], [0.1, 0.15, 0.4, 0.25, 0.1]
-        scratch = torch.zeros(4, dtype=torch.int32, device=dev)
-        xo = torch.empty_like(xf)
-        streaming["search_act_forward_gbs"] = gbs(lambda: ebs.ebs_search_act_forward(xf, 6.0, cand_bits, cand_coeff, xo), vals * 8)
-        streaming["search_weight_forward_gbs"] = gbs(
-            lambda: ebs.ebs_search_weight_forward(xf, cand_bits, cand_coeff, xo, scratch), vals * 12)
-        del xo
-        del xf, xu, pk, ai, yo
-
-    # whole-network inference (the ResNet-20 of this workload wired with its shortcuts, pooling and
-    # classifier): one CUDA-graph replay per batch, cold L2; and the same from pinned host images to
-    # host logits
-    network = {}
-    if world == 1 and args.workload == "config2" and not args.only:
-        network = network_leg(ebs, dev, stream, flush, capture, max(5, min(args.steps, 30)))
-
-    # end to end through the host entry point: pinned host codes in, packed planes out, every step
-    # The layers of this workload have independent inputs, so they are issued round-robin on three
-    # streams (each with its own workspace): the upload of one layer overlaps the kernels of another
-    # and the download of a third.
-    e2e_steps = max(3, min(args.steps, 10))
-    e2e_streams = [torch.cuda.Stream() for _ in range(3)]
-    e2e_ws = [ws] + [torch.empty_like(ws) for _ in range(len(e2e_streams) - 1)]
-
-    def e2e_step():
-        for i, L in enumerate(layers):
-            k = i % len(e2e_streams)
-            L.run_host(ebs, e2e_ws[k], e2e_streams[k])
-        for st_ in e2e_streams:
-            st_.synchronize()
-
-    e2e_step()
-    torch.cuda.synchronize()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
+            def e2e_step():
+                for i, (L, xh, ph) in enumerate(hosts):
+                    lay = L.spec.layer
+                    ebs.ebs_conv2d_mixed_host(xh, ebs.EBS_U8_CODES, ebs.EBS_NHWC, L.n, lay.h_in, lay.w_in, L.pw, L.d,
+                                              L.epi, ws[i % 3], None, None, ph, stream=streams[i % 3])
+                for s_ in streams:
+                    s_.synchronize()
+            h2d, d2h = sum(xh.numel() for _, xh, _ in hosts), sum(L.pn_bytes for L in layers)
+            note = ("ebs_conv2d_mixed_host per layer (independent inputs): pinned u8 codes in, packed next-layer planes "
+                    "out; layers round-robin on 3 streams; wall clock")
+        e2e_steps = max(3, min(args.steps, 10))
         e2e_step()
-    e2e_s = max_over_ranks(time.perf_counter() - t0, dev) / e2e_steps
+        torch.cuda.synchronize()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e2e_s = max_over_ranks(time.perf_counter() - t0, dev) / e2e_steps
+        e2e = {"value": world * total_ops / e2e_s / 1e12, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_s * 1e3, "note": note}
 
     if rank != 0:
         return
-    sm_max = float(clocks.get("sm_max_mhz") or peaks.get("sm_max_mhz", 1965.0))
-    peak_tops = int8_tensor_peak_tops(peaks)                 # 1 bit-pair AND+bitcount = 1 byte MAC = 2 ops
-    hbm_gbs = float(peaks.get("hbm_gbs", 6650.0))
+    peak_tops, hbm_gbs = int8_tensor_peak_tops(peaks), float(peaks.get("hbm_gbs", 6650.0))
+    sm_max = float(clocks.get("sm_max_mhz") or sm_max)
     probes = {}
     if world == 1:
         try:
@@ -518,81 +761,70 @@ def run_gpu(args):
                       "and_popc_add_tops": 2 * ebs.ebs_probe_pipe(0, 500) / 1e12}
         except Exception as exc:                                 # the probes are context, never fatal
             probes = {"error": str(exc)}
-    # Roofline accounting.  The tensor-pipe kernels merge the planes of a channel back into one byte, so one
+    # Roofline of the headline: the tensor-pipe kernels merge the planes of a channel back into one byte, so one
     # int8 multiply-accumulate retires all Wb*Ab plane pairs of that channel: the work the pipe executes is
-    # 2*MACs int8 ops per layer (not 2*MACs*Wb*Ab), and that is what is held against the int8 peak.  A
-    # layer's roof is the slower of that and its packed operand + output bytes at HBM bandwidth.
-    per_layer, roof_ms, sum_tensor_s, sum_hbm_s, sum_bytes, sum_int8_ops = [], 0.0, 0.0, 0.0, 0, 0
-    for L, t in zip(layers, conv_ms):
-        lay = L.spec.layer
-        bytes_alg = (L.px.numel() * 4 + ebs.ebs_packed_weight_plane_bytes(L.d) + L.acc.numel() * 4 + L.pn_bytes)
-        int8_ops = L.ops // (L.spec.w_bits * L.spec.a_bits)                 # 2 * MACs
-        t_tensor, t_hbm = int8_ops / (peak_tops * 1e12), bytes_alg / (hbm_gbs * 1e9)
-        roof = max(t_tensor, t_hbm)
-        roof_ms += roof * 1e3
-        sum_tensor_s += t_tensor; sum_hbm_s += t_hbm; sum_bytes += bytes_alg; sum_int8_ops += int8_ops
-        per_layer.append({"name": lay.name, "wb": L.spec.w_bits, "ab": L.spec.a_bits, "us": round(float(t) * 1e3, 2),
-                          "tops": round(L.ops / (t * 1e-3) / 1e12, 1), "bytes": int(bytes_alg),
-                          "int8_tops": round(int8_ops / (t * 1e-3) / 1e12, 1),
-                          "roof_us": round(roof * 1e6, 2), "roof": "tensor" if t_tensor >= t_hbm else "hbm",
-                          "frac_of_roof": round(roof * 1e3 / float(t), 3)})
-    bound = "tensor" if sum_tensor_s >= sum_hbm_s else "hbm"
-    if bound == "tensor":
-        achieved, roof_peak, roof_unit = sum_int8_ops / (conv_total_ms * 1e-3) / 1e12, peak_tops, "TOPS"
+    # 2*MACs int8 ops per layer, held against the int8 peak; a layer's roof is the slower of that and its packed
+    # operand + output bytes at HBM bandwidth.  `bound` is whichever sum over the layers is larger.
+    m = res["modes"][mode]
+    if m["bound"] == "tensor":
+        achieved, roof_peak, roof_unit = total_int8 / (conv_ms * 1e-3) / 1e12, peak_tops, "TOPS"
     else:
-        achieved, roof_peak, roof_unit = sum_bytes / (conv_total_ms * 1e-3) / 1e9, hbm_gbs, "GB/s"
-    cpu = cpu_baseline_sample() if world == 1 and not args.no_cpu_baseline else None
+        achieved, roof_peak, roof_unit = m["algorithmic_bytes"] / (conv_ms * 1e-3) / 1e9, hbm_gbs, "GB/s"
+    streaming = streaming_leg(ebs, dev, stream, hbm_gbs) if world == 1 and not args.quick else {}
+    network = network_leg(ebs, dev, stream, flush, max(5, min(args.steps, 30))) if world == 1 and not args.quick else {}
+    cpu = cpu_baseline_sample(headline, 15.0) if world == 1 and not args.no_cpu_baseline else None
+    res_head = dict(res)
+    per_config[headline] = res_head
     line = {
         "metric": METRIC, "value": world * total_ops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-        "config": {"workload": workload_text + (f" [only {args.only}]" if args.only else ""), "global_batch": specs[0].batch * world,
-                   "imgs_per_s": world * specs[0].batch / (ms_per_step * 1e-3),
+        "config": {"workload": WORKLOAD_TEXT[headline], "global_batch": layers[0].n * world,
+                   "imgs_per_s": world * layers[0].n / (ms_per_step * 1e-3),
                    "l2": "256 MB buffer rewritten before every timed step (cold L2)",
-                   "launch": "each step is one CUDA-graph replay of its %d kernel launches" % (len(layers) + 2),
-                   "step": "ebs_pack_acts(u8 NHWC) at the entry, ebs_conv2d_mixed(acc + packed_next) per layer, "
-                           "ebs_dequant at the exit; every layer reads its own resident synthetic planes",
+                   "launch": "each step is one CUDA-graph replay of its %d kernel launches" % launches_per_step,
+                   "step": res["step"], "requantization": "per-layer steps calibrated once before timing (99.5th "
+                                                          "percentile of the ReLU output onto the top code)" if chained
+                   else "step 4*s_w*s_a*c_in per layer",
                    "parallelism": f"dp{world} (batch replicas, no data-path collective)"},
         "clocks": clocks,
-        "e2e": {"value": world * total_ops / e2e_s / 1e12, "unit": UNIT,
-                "h2d_bytes_per_step": int(sum(L.x_host.numel() for L in layers)),
-                "d2h_bytes_per_step": int(sum(L.pn_bytes for L in layers)),
-                "note": "ebs_conv2d_mixed_host per layer: pinned u8 codes in, packed next-layer planes out; layers round-robin on 3 streams; wall clock"},
-        "gpu_launches": (len(layers) + 2) * args.steps, "device_wait_timeouts": ebs.ebs_device_wait_timeouts(),
-        "roofline": {"bound": bound,
-                     "kernel": "bit-plane conv, the %d launches of a step (conv_umma_strip_kernel / conv_umma_resident_kernel "
-                               "/ conv_umma_kernel: tcgen05; conv_mma_kernel / conv_mma_strip_kernel: mma.sync; planes "
-                               "merged to bytes on chip)" % len(layers),
+        "gpu_launches": launches_per_step * args.steps * inner, "device_wait_timeouts": ebs.ebs_device_wait_timeouts(),
+        "roofline": {"bound": m["bound"],
+                     "kernel": "bit-plane conv, the %d launches of a step (tcgen05 kernels; planes merged to bytes on "
+                               "chip), output mode of the step: %s" % (len(layers), m["outputs"]),
                      "achieved": achieved, "peak": roof_peak, "unit": roof_unit, "frac": achieved / roof_peak,
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if args.workload == "config2" and not args.only else None,
-                     "accounting": "achieved = algorithmic bytes (packed input planes + weight planes + int32 accumulators "
-                                   "+ packed output planes) of the conv launches / their time when the layers' HBM roofs "
-                                   "sum to more than their tensor roofs, else executed int8 ops (2*MACs: one byte "
-                                   "multiply-accumulate retires all Wb*Ab plane pairs of a channel) / time",
-                     "effective_binary_tops_conv": total_ops / (conv_total_ms * 1e-3) / 1e12,
-                     "int8_tops_conv": sum_int8_ops / (conv_total_ms * 1e-3) / 1e12,
-                     "tensor_peak_tops": peak_tops,
+                     "traffic": ncu_traffic_per_launch(headline),
+                     "accounting": "achieved = executed int8 ops (2*MACs: one byte multiply-accumulate retires all "
+                                   "Wb*Ab plane pairs of a channel) of the conv launches / their CUDA-event time when the "
+                                   "layers' tensor roofs sum to more than their HBM roofs, else algorithmic bytes (packed "
+                                   "input planes + weight byte image + requested outputs) / time",
+                     "conv_ms_per_step": conv_ms, "conv_launches_per_step": len(layers),
+                     "avg_launch_us": conv_ms * 1e3 / len(layers),
+                     "effective_binary_tops_conv": total_ops / (conv_ms * 1e-3) / 1e12,
+                     "int8_tops_conv": total_int8 / (conv_ms * 1e-3) / 1e12,
+                     "gbs_conv": m["algorithmic_bytes"] / (conv_ms * 1e-3) / 1e9,
+                     "tensor_peak_tops": peak_tops, "hbm_peak_gbs": hbm_gbs,
                      "peak_source": f"hbm_gbs {hbm_gbs} ({peak_kind}); int8 dense = 2 x bf16 burst "
                                     f"({peaks.get('bf16_tflops')} TFLOP/s, {peak_kind})",
-                     "conv_ms_per_step": conv_total_ms, "conv_launches_per_step": len(layers),
-                     "algorithmic_bytes_per_launch": int(np.mean([pl["bytes"] for pl in per_layer])),
-                     "sum_layer_roofs_ms": roof_ms, "frac_of_layer_roofs": roof_ms / float(conv_ms.sum()),
-                     "hbm_peak_gbs": hbm_gbs, "hbm_peak_kind": peak_kind,
+                     "sum_layer_roofs_ms": m["sum_layer_roofs_ms"],
+                     "frac_of_layer_roofs_cold": m["sum_layer_roofs_ms"] / conv_ms,
+                     "frac_of_layer_roofs_warm": m["frac_of_layer_roofs"],
                      "other_pipes": dict(probes, popc_pipe_unit_count_tops=popc_pipe_peak_tops(sm_max)),
-                     "per_layer_note": "per-layer times are L2-warm (10 back-to-back launches in a graph); "
-                                       "roof = max(2*MACs / int8 tensor peak, algorithmic bytes / HBM peak)",
-                     "per_layer": per_layer},
-        "literal_bitplane_path": dict(literal, popc_pipe_peak_tops=popc_pipe_peak_tops(sm_max),
-                                      frac_of_popc_pipe=(literal["binary_tops"] / popc_pipe_peak_tops(sm_max)
-                                                         if literal else None),
+                     "per_layer_note": "per-layer times are L2-warm (10 back-to-back launches in a graph); roof = "
+                                       "max(2*MACs / int8 tensor peak, algorithmic bytes / HBM peak); see per_config"},
+        "literal_bitplane_path": dict(res["literal_bitplane_path"],
                                       note="every bit pair is one AND+POPC lane-op here, so binary ops are what this "
-                                           "pipe executes; the default path above retires Wb*Ab of them per int8 MAC"),
+                                           "pipe executes; the default path retires Wb*Ab of them per int8 MAC"),
+        "per_config": per_config,
         "streaming_kernels": streaming,
         "network": network,
         "wall_s_timed_region": wall,
     }
+    if e2e is not None:
+        line["e2e"] = e2e
     if cpu is not None:
         line["cpu_baseline"] = cpu
+        per_config[headline]["cpu_baseline"] = cpu
     print(json.dumps(line))
 
 
@@ -603,8 +835,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS), help="default: the bench workload")
-    ap.add_argument("--only", default="", help="comma-separated layer names: restrict the step to these layers (for profiling)")
+    ap.add_argument("--quick", action="store_true", help="skip the streaming-kernel and whole-network legs")
+    ap.add_argument("--workload", default="all", choices=["all"] + sorted(WORKLOAD_TEXT),
+                    help="all (default): the five configurations, headline config5; configN: that one alone")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -218,9 +218,10 @@ int ebs_conv2d_mixed_variant(const void *packed_x_dev, int n, int h, int w, cons
 long long ebs_device_wait_timeouts(void);
 
 /*
- * Stand-alone de-quantization of accumulators ("quantize_b includes the de-quantize process",
- * text after Eq. 1c): y = float(acc) * scale, then * ch_scale[co], + ch_bias[co], ReLU, each
- * optional, over n_pixels * c_out values stored pixel-major (NHWC).
+ * Stand-alone de-quantization of accumulators: the scaling by 1/(2^b - 1) that Eq. 1c folds into
+ * the quantizer (text after Eq. 1c), applied to integer results as one combined step
+ * y = float(acc) * scale, then * ch_scale[co], + ch_bias[co], ReLU, each optional, over
+ * n_pixels * c_out values stored pixel-major (NHWC).
  */
 int ebs_dequant(const int32_t *acc_dev, size_t n_pixels, int c_out, float scale,
                 const float *ch_scale_dev, const float *ch_bias_dev, int relu, float *y_dev,
@@ -349,7 +350,16 @@ int ebs_conv2d_mixed_host(const void *x_host, int dtype, int layout, int n, int 
  *    EBS_ERR_SCRATCH_TOO_SMALL before anything is enqueued; ebs_noalloc_scratch_bytes() returns the limit.
  *  - The first call on each device looks up the device address of the array (a one-time,
  *    synchronous runtime query made with that device current); make that first call outside any
- *    stream capture.  Later calls on that device only enqueue work.
+ *    stream capture.  Later calls on that device only enqueue work.  With lazy module loading that
+ *    first query is also the moment the driver loads this library's device code and sets the 32 MiB
+ *    aside; on a device whose memory is already fully claimed it fails and the call returns
+ *    EBS_ERR_CUDA (nothing enqueued).  Callers inside a pool that owns the device should make one
+ *    call early, before the pool takes everything, or load eagerly (CUDA_MODULE_LOADING=EAGER).
+ *  - The address is remembered per device ordinal and belongs to that device's primary context.  It
+ *    is wrong for a caller running on another (driver-API) context of the same device, and it is
+ *    stale after cudaDeviceReset(): neither is supported by this entry point.
+ *  - Every argument is checked before the first copy is enqueued: a call that returns an error has
+ *    not touched the shared array.
  *  - All calls on a device share the one array, and it keeps whatever the previous call left in
  *    it.  Every byte the path reads is written earlier in the same call, so nothing needs to be
  *    cleared; but two calls whose GPU work overlaps (different streams, or the same stream from

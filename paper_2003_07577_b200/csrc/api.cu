@@ -157,9 +157,16 @@ static int choose_umma_variant(const ConvParams& p, const ebs_conv_desc* d) {
     return p.Co >= 128 ? 3 : 2;             // tile_n 128 or 64
 }
 
-static int conv_impl(const void* packed_x, int n, int h, int w, const void* packed_w, const ebs_conv_desc* d,
-                     const ebs_epilogue* epi, int32_t* acc_out, float* y_out, void* packed_next, void* stream,
-                     int variant) {
+// A validated, fully decided launch: nothing has been enqueued when conv_plan returns.
+struct ConvPlan {
+    ConvParams p;
+    const ConvVariant* v;
+    dim3 grid;
+};
+
+static int conv_plan(const void* packed_x, int n, int h, int w, const void* packed_w, const ebs_conv_desc* d,
+                     const ebs_epilogue* epi, int32_t* acc_out, float* y_out, void* packed_next, int variant,
+                     ConvPlan* plan) {
     int rc = validate_desc(d);
     if (rc) return rc;
     if (!packed_x || !packed_w || n <= 0 || h <= 0 || w <= 0) return EBS_ERR_INVALID_ARG;
@@ -186,7 +193,7 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
     constexpr int MS_BASE = RES_BASE + NUM_CONV_RESIDENT_VARIANTS;
     if (variant >= MS_BASE + NUM_CONV_MMA_STRIP_VARIANTS) return EBS_ERR_INVALID_ARG;
 
-    ConvParams p;
+    ConvParams& p = plan->p;
     memset(&p, 0, sizeof(p));
     p.x = static_cast<const uint32_t*>(packed_x);
     p.w = static_cast<const uint32_t*>(packed_w);
@@ -251,8 +258,24 @@ static int conv_impl(const void* packed_x, int n, int h, int w, const void* pack
     if (packed_next && (v->tile_c % 32) != 0 && v->tile_c < p.Co) return EBS_ERR_UNSUPPORTED;
     const long long gx = (P + v->tile_p - 1) / v->tile_p, gy = (p.Co + v->tile_c - 1) / v->tile_c;
     if (gy > 65535) return EBS_ERR_UNSUPPORTED;
-    v->launch(p, dim3((unsigned)gx, (unsigned)gy, 1), static_cast<cudaStream_t>(stream));
+    plan->v = v;
+    plan->grid = dim3((unsigned)gx, (unsigned)gy, 1);
+    return EBS_OK;
+}
+
+static int conv_launch(const ConvPlan& plan, void* stream) {
+    const int rc = plan.v->launch(plan.p, plan.grid, static_cast<cudaStream_t>(stream));
+    if (rc) return rc;
     return check_cuda(cudaGetLastError());
+}
+
+static int conv_impl(const void* packed_x, int n, int h, int w, const void* packed_w, const ebs_conv_desc* d,
+                     const ebs_epilogue* epi, int32_t* acc_out, float* y_out, void* packed_next, void* stream,
+                     int variant) {
+    ConvPlan plan;
+    const int rc = conv_plan(packed_x, n, h, w, packed_w, d, epi, acc_out, y_out, packed_next, variant, &plan);
+    if (rc) return rc;
+    return conv_launch(plan, stream);
 }
 
 }  // namespace ebs
@@ -315,8 +338,8 @@ int ebs_pack_weights(const void* w_dev, int dtype, int layout, const ebs_conv_de
                                static_cast<cudaStream_t>(stream));
 }
 
-int ebs_pack_acts(const void* x_dev, int dtype, int layout, int n, int c, int h, int w, int a_bits, float a_scale,
-                  void* packed_x_dev, void* stream) {
+static int validate_pack_acts(const void* x_dev, int dtype, int layout, int n, int c, int h, int w, int a_bits,
+                              float a_scale, const void* packed_x_dev) {
     if (!x_dev || !packed_x_dev || n <= 0 || c <= 0 || h <= 0 || w <= 0) return EBS_ERR_INVALID_ARG;
     if (a_bits < 1 || a_bits > 8) return EBS_ERR_INVALID_ARG;
     if (dtype != EBS_F32 && dtype != EBS_U8_CODES) return EBS_ERR_INVALID_ARG;
@@ -324,6 +347,13 @@ int ebs_pack_acts(const void* x_dev, int dtype, int layout, int n, int c, int h,
     if (dtype == EBS_F32 && !(a_scale > 0.0f)) return EBS_ERR_INVALID_ARG;
     if (!aligned16(x_dev) || !aligned16(packed_x_dev)) return EBS_ERR_INVALID_ARG;
     if ((long long)n * h * w >= (1LL << 31)) return EBS_ERR_OVERFLOW;
+    return EBS_OK;
+}
+
+int ebs_pack_acts(const void* x_dev, int dtype, int layout, int n, int c, int h, int w, int a_bits, float a_scale,
+                  void* packed_x_dev, void* stream) {
+    const int rc = validate_pack_acts(x_dev, dtype, layout, n, c, h, w, a_bits, a_scale, packed_x_dev);
+    if (rc) return rc;
     const float inv = dtype == EBS_F32 ? 1.0f / a_scale : 1.0f;
     return launch_pack_acts(x_dev, dtype, layout, n, c, h, w, a_bits, inv, static_cast<uint32_t*>(packed_x_dev),
                             static_cast<cudaStream_t>(stream));
@@ -441,12 +471,20 @@ int ebs_conv2d_mixed_host(const void* x_host, int dtype, int layout, int n, int 
     float* y_dev = (float*)ws;        ws += round256(outs * 4);
     void* pn_dev = ws;
 
+    // every argument check of the two device calls comes first: an error return means nothing was enqueued
+    // (and, for the caller that shares one scratch between calls, that the scratch was not touched)
+    rc = validate_pack_acts(x_dev, dtype, layout, n, d->c_in, h, w, d->a_bits, d->a_scale, px_dev);
+    if (rc) return rc;
+    ConvPlan plan;
+    rc = conv_plan(px_dev, n, h, w, packed_w_dev, d, epi, acc_out_host ? acc_dev : nullptr,
+                   y_out_host ? y_dev : nullptr, packed_next_host ? pn_dev : nullptr, -1, &plan);
+    if (rc) return rc;
+
     rc = check_cuda(cudaMemcpyAsync(x_dev, x_host, elems_in * (dtype == EBS_F32 ? 4 : 1), cudaMemcpyHostToDevice, st));
     if (rc) return rc;
     rc = ebs_pack_acts(x_dev, dtype, layout, n, d->c_in, h, w, d->a_bits, d->a_scale, px_dev, stream);
     if (rc) return rc;
-    rc = conv_impl(px_dev, n, h, w, packed_w_dev, d, epi, acc_out_host ? acc_dev : nullptr,
-                   y_out_host ? y_dev : nullptr, packed_next_host ? pn_dev : nullptr, stream, -1);
+    rc = conv_launch(plan, stream);
     if (rc) return rc;
     if (acc_out_host) {
         rc = check_cuda(cudaMemcpyAsync(acc_out_host, acc_dev, outs * 4, cudaMemcpyDeviceToHost, st));

@@ -488,11 +488,12 @@ conv_mma_kernel(const ConvParams p) {
 }
 
 template <int AB, int MT, int NT, int WARPS_P, int WARPS_C>
-void launch_conv_mma(const ConvParams& p, dim3 grid, cudaStream_t st) {
+int launch_conv_mma(const ConvParams& p, dim3 grid, cudaStream_t st) {
     const bool full = p.ch_scale || p.ch_bias || p.residual || p.res_packed || p.y_nchw || (p.Co & 1) || p.w_levels ||
                       !isfinite(p.S);
     if (full) conv_mma_kernel<AB, MT, NT, WARPS_P, WARPS_C, true><<<grid, 32 * WARPS_P * WARPS_C, 0, st>>>(p);
     else conv_mma_kernel<AB, MT, NT, WARPS_P, WARPS_C, false><<<grid, 32 * WARPS_P * WARPS_C, 0, st>>>(p);
+    return EBS_OK;
 }
 
 // Variants: variant = size_class * 3 + tile_c_index, tile_c in {16, 32, 64}.

@@ -385,11 +385,11 @@ conv_mma_strip_kernel(const ConvParams p) {
 }
 
 template <int AB, int MT, int NT, int WARPS_P, int WARPS_C>
-void launch_conv_mma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st) {
+int launch_conv_mma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st) {
     constexpr int TILE_P = 16 * MT * WARPS_P, TILE_C = 8 * NT * WARPS_C;
     ConvParams p = p0;
     const MmaStripGeom g = mma_strip_geometry(p, TILE_P, TILE_C);
-    if (!g.ok) return;                                        // callers check mma_strip_geometry first
+    if (!g.ok) return EBS_ERR_UNSUPPORTED;                    // the geometry does not apply: nothing is launched
     p.strip_pix = g.strip_pix;
     p.strip_ks = g.fold;
     // four forms of the kernel: with or without per-channel and shortcut terms (RES; layers without any do not pay
@@ -412,11 +412,12 @@ void launch_conv_mma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st)
         if (compact) {
             if (res) go(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, true, true>, 3);
             else go(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, true, false>, 2);
-            return;
+            return EBS_OK;
         }
     }
     if (res) go(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, false, true>, 1);
     else go(conv_mma_strip_kernel<AB, MT, NT, WARPS_P, WARPS_C, false, false>, 0);
+    return EBS_OK;
 }
 
 // Variants: channel tile 16 / 32 / 64, 256 frame pixels per CTA (8 warps).

@@ -200,8 +200,9 @@ conv_popc_kernel(const ConvParams p) {
 }
 
 template <int WB, int AB, int TP, int TC, int WARPS_P, int WARPS_C>
-void launch_conv_popc(const ConvParams& p, dim3 grid, cudaStream_t st) {
+int launch_conv_popc(const ConvParams& p, dim3 grid, cudaStream_t st) {
     conv_popc_kernel<WB, AB, TP, TC, WARPS_P, WARPS_C><<<grid, 32 * WARPS_P * WARPS_C, 0, st>>>(p);
+    return EBS_OK;
 }
 
 // Variant table.  Every variant gives a thread TC = 8 output channels (except the small one) and

@@ -627,7 +627,7 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_kernel(const ConvParam
 }
 
 template <int WB, int AB, int TILE_N>
-void launch_conv_umma(const ConvParams& p, dim3 grid, cudaStream_t st) {
+int launch_conv_umma(const ConvParams& p, dim3 grid, cudaStream_t st) {
     using T = UmmaTile<WB, AB, TILE_N>;
     // raising the dynamic shared-memory limit is a per-device attribute of the kernel: set it once per device
     static bool attr_set[64] = {};
@@ -639,6 +639,7 @@ void launch_conv_umma(const ConvParams& p, dim3 grid, cudaStream_t st) {
         attr_set[dev] = true;
     }
     conv_umma_kernel<WB, AB, TILE_N><<<grid, UMMA_THREADS, T::SMEM_BYTES, st>>>(p);
+    return EBS_OK;
 }
 
 constexpr int NUM_UMMA_VARIANTS = 5;           // TILE_N = 16, 32, 64, 128, 256

@@ -266,10 +266,10 @@ __global__ void __launch_bounds__(RES_THREADS, 1) conv_umma_resident_kernel(cons
 int resident_sm_count();
 
 template <int AB, int TILE_N>
-void launch_conv_umma_resident(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st) {
+int launch_conv_umma_resident(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st) {
     ConvParams p = p0;
     const ResidentGeom g = resident_geometry(p, TILE_N, resident_sm_count());
-    if (!g.ok) return;                                        // callers check resident_geometry first
+    if (!g.ok) return EBS_ERR_UNSUPPORTED;                    // the geometry does not apply: nothing is launched
     p.strip_pix = g.strip.strip_pix;
     p.strip_ks = g.strip.ks;
     static bool attr_set[64] = {};
@@ -285,6 +285,7 @@ void launch_conv_umma_resident(const ConvParams& p0, dim3 /*grid*/, cudaStream_t
         conv_umma_resident_kernel<AB, TILE_N, true><<<grid, RES_THREADS, g.smem_bytes, st>>>(p);
     else
         conv_umma_resident_kernel<AB, TILE_N, false><<<grid, RES_THREADS, g.smem_bytes, st>>>(p);
+    return EBS_OK;
 }
 
 constexpr int NUM_UMMA_RESIDENT_VARIANTS = 5;      // TILE_N = 16, 32, 64, 128, 256

@@ -91,14 +91,6 @@ inline StripGeom strip_geometry(const ConvParams& p, int tile_n) {
     return g;
 }
 
-#ifdef EBS_STRIP_TRACE
-__device__ long long g_strip_trace[4][16];
-#define STRIP_TRACE(i, cond) do { const int ts_ = blockIdx.x == 0 ? 0 : (blockIdx.x == 700 ? 1 : (blockIdx.x == 1500 ? 2 : -1)); \
-    if (ts_ >= 0 && blockIdx.y == 0 && (cond)) g_strip_trace[ts_][i] = clock64(); } while (0)
-#else
-#define STRIP_TRACE(i, cond) do { } while (0)
-#endif
-
 template <int AB, int TILE_N, bool AFFINE>
 __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const ConvParams p) {
     constexpr int TMEM_COLS = TILE_N < 32 ? 32 : TILE_N;
@@ -110,7 +102,6 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
     __shared__ int abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    STRIP_TRACE(0, tid == 0);
     const int S = p.strip_pix, SP = (S + 7) & ~7, KS = p.strip_ks;
     const int taps = p.kh * p.kw;
     const bool pointwise = strip_pointwise(p);
@@ -143,7 +134,6 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const uint32_t tmem_base = tmem_slot;
-    STRIP_TRACE(1, tid == 0);
 
     const int nchunks = (p.CW + KS - 1) / KS;
 
@@ -181,8 +171,6 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
                     load_words_global<AB>(p.x + (slot_off[j] + cw * AB), a_set[set][j]);
             }
         };
-
-        STRIP_TRACE(2, tid == 0);
         load_chunk(0, 0);
         if (nchunks > 1) load_chunk(1, 1);
         bool expanders_ok = true;
@@ -230,7 +218,6 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
                 }
                 asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");  // generic writes -> tensor-core reads
                 mbar_arrive(&full_bar[st]);
-                STRIP_TRACE(3 + (ch > 0), tid == 0);
             }
         }
         if (p.w_levels) {
@@ -238,7 +225,6 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
             for (int j = 0; j < STRIP_SLOTS; ++j)
                 if (slot_q[j] >= 0 && csum[j]) atomicAdd(&csum_s[slot_pix[j]], csum[j]);
         }
-        STRIP_TRACE(8, tid == 0);
     } else {
         // =========================== issuer ===========================
         constexpr uint32_t IDESC = umma_idesc_i8(TILE_N);
@@ -246,7 +232,6 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
             const int st = ch & 1;
             if (!mbar_wait_bounded(&full_bar[st], (uint32_t)((ch >> 1) & 1), abortp)) break;
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-            STRIP_TRACE(5 + (ch > 0), (tid & 31) == 0);
             if ((tid & 31) == 0) {
                 // the issuing thread is the pipeline stage that feeds the tensor core: descriptors are built once
                 // and advanced by additions (start addresses are in 16-byte units), a few instructions per MMA
@@ -266,7 +251,6 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
                     }
                 }
                 umma_commit(&empty_bar[st]);
-                STRIP_TRACE(7, ch == nchunks - 1);
             }
             __syncwarp();
         }
@@ -279,7 +263,6 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const bool aborted = abort_flag != 0;
-    STRIP_TRACE(9, tid == 0);
 
     // ---- epilogue: expander threads read the accumulators of their own row f0 + (tid % 128)
     if (!aborted && warp < 8) {
@@ -300,7 +283,6 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
         umma_epilogue<TILE_N, AFFINE>(p, tmem_base, warp, gp, pvalid, wsum_row, co0);
     }
     if (aborted && tid == 0) atomicAdd(&g_umma_timeouts, 1ull);
-    STRIP_TRACE(10, tid == 0);
 
     // ---- release tensor memory (every path reaches this)
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
@@ -309,14 +291,13 @@ __global__ void __launch_bounds__(UMMA_THREADS) conv_umma_strip_kernel(const Con
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
                      : "memory");
     }
-    STRIP_TRACE(11, tid == 0);
 }
 
 template <int AB, int TILE_N>
-void launch_conv_umma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st) {
+int launch_conv_umma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st) {
     ConvParams p = p0;
     const StripGeom g = strip_geometry(p, TILE_N);
-    if (!g.ok) return;                                        // callers check strip_geometry first
+    if (!g.ok) return EBS_ERR_UNSUPPORTED;                    // the geometry does not apply: nothing is launched
     p.strip_pix = g.strip_pix;
     p.strip_ks = g.ks;
     const bool affine = p.ch_scale || p.ch_bias || p.residual || p.res_packed;
@@ -332,6 +313,7 @@ void launch_conv_umma_strip(const ConvParams& p0, dim3 /*grid*/, cudaStream_t st
     const dim3 grid((unsigned)((frame + UMMA_M - 1) / UMMA_M), (unsigned)((p.Co + TILE_N - 1) / TILE_N), 1);
     if (affine) conv_umma_strip_kernel<AB, TILE_N, true><<<grid, UMMA_THREADS, g.smem_bytes, st>>>(p);
     else conv_umma_strip_kernel<AB, TILE_N, false><<<grid, UMMA_THREADS, g.smem_bytes, st>>>(p);
+    return EBS_OK;
 }
 
 constexpr int NUM_UMMA_STRIP_VARIANTS = 5;      // TILE_N = 16, 32, 64, 128, 256

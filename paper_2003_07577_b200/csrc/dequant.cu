@@ -1,5 +1,5 @@
-// Stand-alone de-quantization of int32 accumulators (the "de-quantize process" of Eq. 1c and the
-// scale merge of Sec. 4.3).  Pure streaming: 4 bytes read + 4 bytes written per element.
+// Stand-alone de-quantization of int32 accumulators (the scaling back to real values that Eq. 1c
+// folds into the quantizer, and the scale merge of Sec. 4.3).  Pure streaming: 4 bytes read + 4 bytes written per element.
 #include "ebs_internal.cuh"
 
 namespace ebs {

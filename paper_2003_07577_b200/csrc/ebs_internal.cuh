@@ -41,7 +41,7 @@ struct ConvParams {
 
 // One instantiation of the popcount kernel: launch function + its tile geometry.
 struct ConvVariant {
-    void (*launch)(const ConvParams&, dim3 grid, cudaStream_t);
+    int (*launch)(const ConvParams&, dim3 grid, cudaStream_t);   // EBS_OK once the kernel is enqueued
     int tile_p, tile_c, threads;
 };
 

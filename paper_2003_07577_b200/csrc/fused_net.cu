@@ -40,13 +40,6 @@ __device__ __forceinline__ uint8_t* strip_ptr(uint8_t* acts, int buf) { return a
 // A strip holds one 32-channel word of up to 1360 frame pixels or two words of up to 680: pixels per word.
 __host__ __device__ inline int strip_cap(int channels) { return channels > 32 ? FUSED_ACT_PIX / 2 : FUSED_ACT_PIX; }
 
-#ifdef EBS_FUSED_TRACE
-__device__ long long g_fused_clk[72][4];
-#define FUSED_CLK(li, k) do { if (blockIdx.x == 0 && tid == 0) g_fused_clk[li][k] = clock64(); } while (0)
-#else
-#define FUSED_CLK(li, k) do { } while (0)
-#endif
-
 __global__ void __launch_bounds__(FUSED_THREADS, 1)
 fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, const FusedLayer* __restrict__ layers,
                     int n_layers, const FusedHead head, float* __restrict__ logits, uint8_t* __restrict__ trace,
@@ -114,7 +107,6 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
     float* pool_scratch = reinterpret_cast<float*>(strip_ptr(acts, 0));      // [pixels][c_out] of the last layer
 
     for (int li = 0; li < n_layers && ok; ++li) {
-        FUSED_CLK(li, 0);
         const FusedLayer L = layers[li];
         const int cw = (L.c_in + 31) >> 5, co16 = (L.c_out + 15) & ~15;
         const int Ho = L.stride == 2 ? L.h_in / 2 : L.h_in, Wo = L.stride == 2 ? L.w_in / 2 : L.w_in;
@@ -164,7 +156,6 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
         __syncthreads();
 
         // ---- MMAs of the whole layer
-        FUSED_CLK(li, 1);
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
         if (lane == 0 && warp < 4 && mbar_wait_bounded(&w_bar[li & 1], (uint32_t)((li >> 1) & 1), abortp)) {
             // Four threads issue (lane 0 of warps 0-3, tiles dealt round-robin): the issue loop of one thread,
@@ -201,7 +192,6 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
         if (abort_flag != 0) { ok = false; break; }
         ++mma_phase;
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-        FUSED_CLK(li, 2);
 
         // ---- epilogue (a held projection has none: the next layer reads its accumulators)
         if (!L.hold) {
@@ -283,8 +273,6 @@ fused_resnet_kernel(const uint8_t* __restrict__ images, int img_h, int img_w, co
         __syncthreads();
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     }
-
-    FUSED_CLK(n_layers, 0);
     // ---- pooling, 8-bit quantization, classifier
     if (ok && !abort_flag && n_layers > 0) {
         const FusedLayer L = layers[n_layers - 1];
@@ -383,6 +371,3 @@ int fused_head_bytes() { return (int)sizeof(FusedHead); }
 
 }  // namespace ebs
 
-#ifdef EBS_FUSED_TRACE
-extern "C" void ebs_debug_fused_clk(long long* out) { cudaMemcpyFromSymbol(out, ebs::g_fused_clk, sizeof(ebs::g_fused_clk)); }
-#endif
