@@ -52,7 +52,7 @@ typedef enum ebs_status {
     EBS_ERR_OVERFLOW = -3,    /* c_in*kh*kw*2^(w_bits-1)*(2^a_bits-1) >= 2^31 (w_levels = 1: c_in*kh*kw*(2^w_bits-1)*
                                  (2^a_bits-1)), or an index would overflow */
     EBS_ERR_CUDA = -4,        /* a CUDA runtime call failed (launch error, bad device pointer, ...) */
-    EBS_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (reserved) */
+    EBS_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (reported by ebs_check_device_status) */
     EBS_ERR_SCRATCH_TOO_SMALL = -6 /* the request needs more than the built-in scratch of the no-allocation call */
 } ebs_status;
 
@@ -198,7 +198,12 @@ int ebs_conv2d_mixed(const void *packed_x_dev, int n, int h, int w, const void *
  *   34..36  warp-level kernels for small stride-1 layers (c_in 5..128, even c_out, NHWC
  *           output): the strip of input pixels expanded to bytes once per thread block,
  *           fragments loaded from shared memory, weights from the byte image; channel tile
- *           16 / 32 / 64.
+ *           16 / 32 / 64;
+ *   37..39  persistent pipeline tcgen05 kernels for stride-1 and strided k x k layers and 1x1 layers
+ *           at any stride (stride <= 2, w_levels = 0): every input pixel expanded once per thread
+ *           block and tile, several 128-pixel accumulators per weight tile, weights resident in
+ *           shared memory or streamed, expansion / MMAs / epilogue of consecutive tiles overlapped;
+ *           channel tile 64 / 128 / 256.
  * variant = -2 lets the library choose among the integer-pipe kernels only (the literal
  * bit-plane evaluation), for comparison runs.
  * For tuning and for tests that must cover every kernel instantiation.  Returns
@@ -211,11 +216,39 @@ int ebs_conv2d_mixed_variant(const void *packed_x_dev, int n, int h, int w, cons
                              float *y_out_dev, void *packed_next_dev, void *stream, int variant);
 
 /*
+ * Which kernel family a variant number belongs to ("popc", "mma", "umma", "umma_strip", "umma_resident",
+ * "mma_strip", "umma_pipe"; "" if out of range), and whether a variant can run a layer: the full validation and
+ * kernel selection of ebs_conv2d_mixed_variant for a request with the given outputs (want_* are 0 / 1), without
+ * touching any buffer and without launching anything.  Returns EBS_OK, EBS_ERR_UNSUPPORTED, or the error the real
+ * call would return.  For tests and tuning tools that have to enumerate the variants of a layer.
+ */
+const char *ebs_conv_variant_family(int variant);
+int ebs_conv_variant_applies(const ebs_conv_desc *desc, int n, int h, int w, const ebs_epilogue *epi, int want_acc,
+                             int want_y, int want_packed_next, int variant);
+
+/*
  * Number of thread blocks that gave up a bounded device-side wait (on the tensor core's completion
  * barrier) since the library was loaded; such a block skips its outputs.  0 in a healthy run.
  * Synchronizes the device.  The paper has no counterpart.
  */
 long long ebs_device_wait_timeouts(void);
+
+/*
+ * EBS_ERR_TIMEOUT if thread blocks gave up a bounded wait since the previous call of this function (their
+ * outputs are missing: run the layer again), else EBS_OK.  Synchronizes the device.  A launch itself cannot
+ * report this: it returns before the kernel runs.  The paper has no counterpart.
+ */
+int ebs_check_device_status(void);
+
+/*
+ * Test hook for the give-up path of the tensor-core kernels (the paper has no counterpart).  `limit` = number of
+ * polls a bounded wait makes before it gives up (0 restores the default, about 2^20 polls of >= 40 ns);
+ * skip_mma = 1 makes the persistent pipeline kernel's issuing thread issue no tensor-core work at all, so that
+ * every wait for it runs out with nothing in flight: each thread block then raises its abort flag, leaves its
+ * loops, frees its tensor memory and returns, and ebs_device_wait_timeouts() rises.  Process-wide; affects the
+ * launches made afterwards.  Nothing faults or hangs by construction.
+ */
+int ebs_test_set_device_wait(unsigned int limit, int skip_mma);
 
 /*
  * Stand-alone de-quantization of accumulators: the scaling by 1/(2^b - 1) that Eq. 1c folds into

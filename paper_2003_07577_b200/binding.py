@@ -27,6 +27,7 @@ EXPORTS = [
     "ebs_conv2d_mixed_variant", "ebs_dequant", "ebs_host_workspace_bytes", "ebs_conv2d_mixed_host",
     "ebs_probe_pipe", "ebs_device_wait_timeouts", "ebs_global_avgpool", "ebs_packed_weight_plane_bytes", "ebs_search_weight_forward",
     "ebs_search_act_forward", "ebs_expected_flops", "ebs_fused_plan_upload", "ebs_resnet_cifar_forward", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
+    "ebs_conv_variant_family", "ebs_conv_variant_applies", "ebs_check_device_status", "ebs_test_set_device_wait",
 ]
 
 
@@ -97,6 +98,11 @@ def lib() -> ctypes.CDLL:
         L.ebs_noalloc_scratch_bytes.restype = z
         L.ebs_device_wait_timeouts.restype = ctypes.c_longlong
         L.ebs_conv2d_mixed_host_noalloc.argtypes = [p, i, i, i, i, i, p, D, E, p, p, p, p]
+        L.ebs_conv_variant_family.argtypes = [i]
+        L.ebs_conv_variant_family.restype = ctypes.c_char_p
+        L.ebs_conv_variant_applies.argtypes = [D, i, i, i, E, i, i, i, i]
+        L.ebs_check_device_status.restype = i
+        L.ebs_test_set_device_wait.argtypes = [ctypes.c_uint, i]
         _lib = L
     return _lib
 
@@ -284,3 +290,23 @@ def ebs_conv2d_mixed_host_noalloc(x_host, dtype, layout, n, h, w, packed_w_dev, 
                                              ctypes.byref(desc), e, _ptr(acc_out_host), _ptr(y_out_host),
                                              _ptr(packed_next_host), _stream(stream))
     _check(rc, "ebs_conv2d_mixed_host_noalloc")
+
+
+def ebs_conv_variant_family(variant: int) -> str:
+    return lib().ebs_conv_variant_family(int(variant)).decode()
+
+
+def ebs_conv_variant_applies(desc, n, h, w, epi=None, want_acc=True, want_y=False, want_packed_next=False,
+                             variant: int = -1) -> int:
+    """Status the forced-variant call would return for this request (EBS_OK / EBS_ERR_UNSUPPORTED / ...); launches nothing."""
+    e = None if epi is None else ctypes.byref(epi)
+    return lib().ebs_conv_variant_applies(ctypes.byref(desc), n, h, w, e, int(bool(want_acc)), int(bool(want_y)),
+                                          int(bool(want_packed_next)), int(variant))
+
+
+def ebs_check_device_status() -> int:
+    return int(lib().ebs_check_device_status())
+
+
+def ebs_test_set_device_wait(limit: int, skip_mma: bool) -> None:
+    _check(lib().ebs_test_set_device_wait(int(limit), int(bool(skip_mma))), "ebs_test_set_device_wait")

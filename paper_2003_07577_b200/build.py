@@ -8,6 +8,7 @@ from __future__ import annotations
 import concurrent.futures
 import glob
 import os
+import re
 import subprocess
 import sys
 
@@ -21,14 +22,27 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
 
-def _newest_header() -> float:
-    hdrs = glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
-    return max(os.path.getmtime(h) for h in hdrs)
+_INCLUDE = re.compile(r'^\s*#\s*include\s+"([^"]+)"', re.M)
+
+
+def _deps(path: str, seen: set) -> set:
+    """The file and every project header it includes, transitively (headers live in csrc/ and include/)."""
+    if path in seen:
+        return seen
+    seen.add(path)
+    with open(path) as f:
+        for name in _INCLUDE.findall(f.read()):
+            for d in (CSRC, os.path.join(ROOT, "include")):
+                cand = os.path.join(d, name)
+                if os.path.exists(cand):
+                    _deps(cand, seen)
+    return seen
 
 
 def _compile(src: str, verbose: bool) -> str:
     obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
-    if os.path.exists(obj) and os.path.getmtime(obj) >= max(os.path.getmtime(src), _newest_header()):
+    newest = max(os.path.getmtime(p) for p in _deps(src, set()))
+    if os.path.exists(obj) and os.path.getmtime(obj) >= newest:
         return obj
     cmd = ["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
     res = subprocess.run(cmd, capture_output=True, text=True)

@@ -60,8 +60,13 @@ const ConvVariant* conv_umma_variant(int w_bits, int a_bits, int variant) {
 unsigned long long conv_umma_timeouts() {
     return conv_umma_timeouts_w1() + conv_umma_timeouts_w2() + conv_umma_timeouts_w3() + conv_umma_timeouts_w4() +
            conv_umma_timeouts_w5() + conv_umma_timeouts_w6() + conv_umma_timeouts_w7() + conv_umma_timeouts_w8() +
-           conv_umma_strip_timeouts() + conv_umma_resident_timeouts() + fused_net_timeouts();
+           conv_umma_strip_timeouts() + conv_umma_resident_timeouts() + conv_umma_pipe_timeouts() + fused_net_timeouts();
 }
+
+// Polls a bounded device-side wait makes before it gives up (about 40 ns each), and test flags; process-wide,
+// changed only by ebs_test_set_device_wait.
+static unsigned g_wait_limit = 1u << 20;
+static int g_test_flags = 0;
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -148,6 +153,24 @@ static int choose_strip_variant(const ConvParams& p) {
 // The per-tap tcgen05 kernels (any stride) pay off when a CTA's 128 x tile_n accumulator sees a deep
 // reduction, the channel tile is wide enough to amortise the activation expansion, and the layer has
 // enough output tiles; smaller layers run faster on the warp-level kernels.  Returns the variant or -1.
+// The persistent pipeline kernel covers stride-1 and strided k x k layers and 1x1 layers at any stride.  It pays off
+// when the layer has at least 64 output channels and enough outputs to fill the GPU.  Channel tile: the widest of
+// 256/128/64 that divides c_out and still leaves about two tiles per SM (every tile whole: straight-line epilogue,
+// and the fewer channel tiles, the less often an input pixel is expanded); failing that the widest that applies.
+// Returns the pipeline variant (0..2) or -1.
+static int choose_pipe_variant(const ConvParams& p, int sms) {
+    if (p.Co < 64 || (long long)p.P * p.Co < (1LL << 19) || p.w_levels || p.fold != 1) return -1;
+    int fallback = -1;
+    for (int v = 2; v >= 0; --v) {
+        const int tile_n = 64 << v;
+        if (p.Co % tile_n != 0 && !(v == 0)) continue;
+        if (!conv_umma_pipe_applies(p, v)) continue;
+        if (fallback < 0) fallback = v;
+        if (conv_umma_pipe_items(p, v) >= 2LL * sms || v == 0) return v;
+    }
+    return fallback;
+}
+
 static int choose_umma_variant(const ConvParams& p, const ebs_conv_desc* d) {
     const int kwords = (p.KK + p.fold - 1) / p.fold;
     const long long outputs = (long long)p.P * p.Co;
@@ -191,7 +214,8 @@ static int conv_plan(const void* packed_x, int n, int h, int w, const void* pack
     constexpr int STRIP_BASE = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS;
     constexpr int RES_BASE = STRIP_BASE + NUM_CONV_STRIP_VARIANTS;
     constexpr int MS_BASE = RES_BASE + NUM_CONV_RESIDENT_VARIANTS;
-    if (variant >= MS_BASE + NUM_CONV_MMA_STRIP_VARIANTS) return EBS_ERR_INVALID_ARG;
+    constexpr int PIPE_BASE = MS_BASE + NUM_CONV_MMA_STRIP_VARIANTS;
+    if (variant >= PIPE_BASE + NUM_CONV_PIPE_VARIANTS) return EBS_ERR_INVALID_ARG;
 
     ConvParams& p = plan->p;
     memset(&p, 0, sizeof(p));
@@ -210,6 +234,8 @@ static int conv_plan(const void* packed_x, int n, int h, int w, const void* pack
     p.w_levels = d->w_levels;
     p.fold = d->c_in <= 4 ? 8 : (d->c_in <= 8 ? 4 : (d->c_in <= 16 ? 2 : 1));
     p.fold_bits = 32 / p.fold;
+    p.wait_limit = g_wait_limit;
+    p.test_flags = g_test_flags;
     if (epi) {
         p.ch_scale = epi->ch_scale_dev; p.ch_bias = epi->ch_bias_dev; p.residual = epi->residual_dev;
         p.res_packed = static_cast<const uint32_t*>(epi->res_packed_dev); p.res_bits = epi->res_bits; p.res_scale = epi->res_scale;
@@ -221,10 +247,12 @@ static int conv_plan(const void* packed_x, int n, int h, int w, const void* pack
     if (variant == -2) {
         variant = choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
     } else if (variant < 0) {
-        const int strip = mma_ok ? choose_strip_variant(p) : -1;
-        const int umma = (mma_ok && strip < 0) ? choose_umma_variant(p, d) : -1;
+        const int pipe = mma_ok ? choose_pipe_variant(p, sm_count()) : -1;
+        const int strip = (mma_ok && pipe < 0) ? choose_strip_variant(p) : -1;
+        const int umma = (mma_ok && strip < 0 && pipe < 0) ? choose_umma_variant(p, d) : -1;
         // deep reductions whose weight tiles fit in shared memory: the persistent form of the same tile
-        if (strip >= 0 && p.CW * d->kh * d->kw >= 8 && conv_umma_resident_applies(p, strip)) variant = RES_BASE + strip;
+        if (pipe >= 0) variant = PIPE_BASE + pipe;
+        else if (strip >= 0 && p.CW * d->kh * d->kw >= 8 && conv_umma_resident_applies(p, strip)) variant = RES_BASE + strip;
         else if (strip >= 0) variant = STRIP_BASE + strip;
         else if (umma >= 0) variant = NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + umma;
         // small stride-1 layers with up to 64 output channels: the warp-level strip kernel (it expands every input
@@ -239,7 +267,9 @@ static int conv_plan(const void* packed_x, int n, int h, int w, const void* pack
                               : choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
     }
     if (variant >= NUM_CONV_VARIANTS && !mma_ok) return EBS_ERR_UNSUPPORTED;
-    if (variant >= MS_BASE) {
+    if (variant >= PIPE_BASE) {
+        if (!conv_umma_pipe_applies(p, variant - PIPE_BASE)) return EBS_ERR_UNSUPPORTED;
+    } else if (variant >= MS_BASE) {
         if (!conv_mma_strip_applies(p, variant - MS_BASE)) return EBS_ERR_UNSUPPORTED;
     } else if (variant >= RES_BASE) {
         if (!conv_umma_resident_applies(p, variant - RES_BASE)) return EBS_ERR_UNSUPPORTED;
@@ -247,6 +277,7 @@ static int conv_plan(const void* packed_x, int n, int h, int w, const void* pack
         return EBS_ERR_UNSUPPORTED;
     }
     const ConvVariant* v =
+        variant >= PIPE_BASE ? conv_umma_pipe_variant(d->a_bits, variant - PIPE_BASE) :
         variant >= MS_BASE ? conv_mma_strip_variant(d->a_bits, variant - MS_BASE) :
         variant >= RES_BASE ? conv_umma_resident_variant(d->a_bits, variant - RES_BASE) :
         variant >= STRIP_BASE ? conv_umma_strip_variant(d->a_bits, variant - STRIP_BASE) :
@@ -368,7 +399,49 @@ int ebs_conv2d_mixed(const void* packed_x_dev, int n, int h, int w, const void* 
 
 int ebs_num_conv_variants(void) {
     return NUM_CONV_VARIANTS + NUM_CONV_MMA_VARIANTS + NUM_CONV_UMMA_VARIANTS + NUM_CONV_STRIP_VARIANTS +
-           NUM_CONV_RESIDENT_VARIANTS + NUM_CONV_MMA_STRIP_VARIANTS;
+           NUM_CONV_RESIDENT_VARIANTS + NUM_CONV_MMA_STRIP_VARIANTS + NUM_CONV_PIPE_VARIANTS;
+}
+
+const char* ebs_conv_variant_family(int variant) {
+    int v = variant;
+    if (v < 0) return "";
+    if (v < NUM_CONV_VARIANTS) return "popc";
+    v -= NUM_CONV_VARIANTS;
+    if (v < NUM_CONV_MMA_VARIANTS) return "mma";
+    v -= NUM_CONV_MMA_VARIANTS;
+    if (v < NUM_CONV_UMMA_VARIANTS) return "umma";
+    v -= NUM_CONV_UMMA_VARIANTS;
+    if (v < NUM_CONV_STRIP_VARIANTS) return "umma_strip";
+    v -= NUM_CONV_STRIP_VARIANTS;
+    if (v < NUM_CONV_RESIDENT_VARIANTS) return "umma_resident";
+    v -= NUM_CONV_RESIDENT_VARIANTS;
+    if (v < NUM_CONV_MMA_STRIP_VARIANTS) return "mma_strip";
+    v -= NUM_CONV_MMA_STRIP_VARIANTS;
+    if (v < NUM_CONV_PIPE_VARIANTS) return "umma_pipe";
+    return "";
+}
+
+int ebs_conv_variant_applies(const ebs_conv_desc* desc, int n, int h, int w, const ebs_epilogue* epi, int want_acc,
+                             int want_y, int want_packed_next, int variant) {
+    // the validation and selection of a launch with stand-in buffers (aligned, never dereferenced): nothing is enqueued
+    void* fake = reinterpret_cast<void*>(static_cast<uintptr_t>(256));
+    ConvPlan plan;
+    return conv_plan(fake, n, h, w, fake, desc, epi, want_acc ? static_cast<int32_t*>(fake) : nullptr,
+                     want_y ? static_cast<float*>(fake) : nullptr, want_packed_next ? fake : nullptr, variant, &plan);
+}
+
+int ebs_test_set_device_wait(unsigned int limit, int skip_mma) {
+    g_wait_limit = limit == 0 ? (1u << 20) : limit;
+    g_test_flags = skip_mma ? 1 : 0;
+    return EBS_OK;
+}
+
+int ebs_check_device_status(void) {
+    static long long seen = 0;
+    const long long now = (long long)conv_umma_timeouts();
+    const bool fresh = now > seen;
+    seen = now;
+    return fresh ? EBS_ERR_TIMEOUT : EBS_OK;
 }
 
 long long ebs_device_wait_timeouts(void) { return (long long)conv_umma_timeouts(); }

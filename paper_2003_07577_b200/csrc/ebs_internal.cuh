@@ -37,6 +37,9 @@ struct ConvParams {
     int fold;                         // taps OR-ed into one reduction word by the tensor-pipe kernels: 1, 2, 4, 8
     int fold_bits;                    // 32 / fold: bits each folded tap occupies (>= c_in)
     int strip_pix, strip_ks;          // strip kernel only (set by its launcher): pixels of a strip, words per stage
+    unsigned wait_limit;              // polls a bounded device-side wait makes before the CTA gives up
+    int test_flags;                   // bit 0 (tests only): the MMA issuer issues nothing, so that waits run out
+    int pipe_m_sub;                   // persistent pipeline kernel: accumulators per super-tile (0 = chosen by the library)
 };
 
 // One instantiation of the popcount kernel: launch function + its tile geometry.
@@ -65,7 +68,13 @@ EBS_DECLARE_AB(5) EBS_DECLARE_AB(6) EBS_DECLARE_AB(7) EBS_DECLARE_AB(8)
 #undef EBS_DECLARE_AB
 
 // 5th-generation tensor-core kernels (conv_umma_w1.cu .. conv_umma_w8.cu); variant = log2(tile_n / 16).
-enum { NUM_CONV_UMMA_VARIANTS = 5, NUM_CONV_STRIP_VARIANTS = 5, NUM_CONV_RESIDENT_VARIANTS = 5, NUM_CONV_MMA_STRIP_VARIANTS = 3 };
+enum { NUM_CONV_UMMA_VARIANTS = 5, NUM_CONV_STRIP_VARIANTS = 5, NUM_CONV_RESIDENT_VARIANTS = 5, NUM_CONV_MMA_STRIP_VARIANTS = 3,
+       NUM_CONV_PIPE_VARIANTS = 3 };
+// Persistent pipeline kernel for any stride (conv_umma_pipe.cu): variants by channel tile 64 << variant.
+const ConvVariant* conv_umma_pipe_variant(int a_bits, int variant);
+bool conv_umma_pipe_applies(const ConvParams& p, int variant);
+unsigned long long conv_umma_pipe_timeouts();
+long long conv_umma_pipe_items(const ConvParams& p, int variant);   // (pixel super-tile, channel tile) work items, -1 if it does not apply
 // Warp-level strip kernel for small stride-1 layers (conv_mma_strip.cu): channel tile 16 / 32 / 64.
 const ConvVariant* conv_mma_strip_variant(int a_bits, int variant);
 bool conv_mma_strip_applies(const ConvParams& p, int variant);

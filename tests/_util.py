@@ -96,51 +96,29 @@ def run_conv(qa, qw, d, epi=None, want_acc=True, want_y=False, next_bits=0, vari
     return out
 
 
-N_STRIP = 5       # variants 24 .. 28: the strip kernels
-N_RESIDENT = 5    # variants 29 .. 33: the persistent weight-resident strip kernels
-N_MMA_STRIP = 3   # variants 34 .. 36: the warp-level strip kernels (channel tile 16, 32, 64)
+def variants_of(family):
+    """Variant numbers of a kernel family, as the library names them ("popc", "mma", "umma", "umma_strip",
+    "umma_resident", "mma_strip", "umma_pipe")."""
+    return [v for v in range(ebs.ebs_num_conv_variants()) if ebs.ebs_conv_variant_family(v) == family]
 
 
-def strip_variant_applies(d, w, tile_n):
-    """Host-side rule of the strip kernel: stride 1 (or a 1x1 layer without padding), a strip
-    of at most 512 pixels, and two stages of (strip + kh*kw weight tiles) within 200 KB of shared memory."""
-    pointwise = d.kh == 1 and d.kw == 1 and d.pad_h == 0 and d.pad_w == 0    # 1x1 without padding: any stride
-    if (d.stride_h != 1 or d.stride_w != 1) and not pointwise:
-        return False
-    strip = 128 + (d.kh - 1) * (w + 2 * d.pad_w) + d.kw - 1
-    pad = (strip + 7) // 8 * 8
-    return strip <= 512 and 2 * (pad * 32 + 32 + d.kh * d.kw * tile_n * 32 + 256) + 1024 + pad * 4 <= 200 * 1024
+def applies(d, h, w, variant, n=1, epi=None, want_acc=True, want_y=False, want_packed=False):
+    """Asks the library whether a forced variant can run this request (its own rules: nothing is restated here).
+    EBS_ERR_UNSUPPORTED means no; any other error is a bug in the test's request."""
+    rc = ebs.ebs_conv_variant_applies(d, n, h, w, epi, want_acc, want_y, want_packed, variant)
+    if rc == ebs.EBS_OK:
+        return True
+    assert rc == ebs.EBS_ERR_UNSUPPORTED, f"variant {variant}: {ebs.ebs_status_string(rc)}"
+    return False
 
 
-def resident_variant_applies(d, w, tile_n):
-    """Host-side rule of the persistent kernel: the strip rule, no window-sum term, and all weight tiles
-    of a channel tile (ceil(c_in/32) * kh*kw * tile_n * 32 bytes) within 150 KB."""
-    cw = (d.c_in + 31) // 32
-    return (strip_variant_applies(d, w, tile_n) and not d.w_levels
-            and cw * d.kh * d.kw * tile_n * 32 <= 150 * 1024)
-
-
-def mma_strip_variant_applies(d, w, variant):
-    """Host-side rule of the warp-level strip kernel (NHWC output only: callers that ask for NCHW must not force it)."""
-    pointwise = d.kh == 1 and d.kw == 1 and d.pad_h == 0 and d.pad_w == 0
-    if (d.stride_h != 1 or d.stride_w != 1) and not pointwise:
-        return False
-    tile_p, tile_c = ((256, 16), (64, 32), (64, 64))[variant]
-    cw, taps = (d.c_in + 31) // 32, d.kh * d.kw
-    strip = tile_p + (d.kh - 1) * (w + 2 * d.pad_w) + d.kw - 1
-    pad = (strip + 7) // 8 * 8
-    smem = cw * pad * 32 + taps * cw * tile_c * 32 + tile_p * (tile_c + 4) + tile_p * 4 + 128
-    return (cw <= 4 and taps * cw <= 64 and not d.w_levels and d.c_out % 2 == 0 and d.c_in > 4 and smem <= 96 * 1024)
-
-
-def all_variants(d, w=16):
-    """Every kernel variant that applies to descriptor d on images of width w (-1 = the library's own choice)."""
-    n = ebs.ebs_num_conv_variants()
-    base = n - N_STRIP - N_RESIDENT - N_MMA_STRIP
-    strip = [base + i for i in range(N_STRIP) if strip_variant_applies(d, w, 16 << i)]
-    resident = [base + N_STRIP + i for i in range(N_RESIDENT) if resident_variant_applies(d, w, 16 << i)]
-    mma_strip = [base + N_STRIP + N_RESIDENT + i for i in range(N_MMA_STRIP) if mma_strip_variant_applies(d, w, i)]
-    return list(range(-1, base)) + strip + resident + mma_strip
+def all_variants(d, w=16, h=None, n=1, epi=None, want_y=False, want_packed=False, min_count=3):
+    """Every kernel variant the library accepts for this request (-1 = its own choice comes first)."""
+    h = w if h is None else h
+    out = [-1] + [v for v in range(ebs.ebs_num_conv_variants())
+                  if applies(d, h, w, v, n, epi, True, want_y, want_packed)]
+    assert len(out) >= min_count, f"only {len(out)} variants apply: the test would cover too little"
+    return out
 
 
 def rand_codes(rng, shape, bits, signed):

@@ -58,8 +58,7 @@ def test_shortcut_from_packed_codes(ebs, U, oracle, res_bits, co, next_bits):
     p_res = U.pack_acts_codes(q_res, res_bits)
     epi = ebs.epilogue(None, _to(cb, U), None, True, next_bits, float(step), ebs.EBS_NHWC, res_packed=p_res,
                        res_bits=res_bits, res_scale=res_scale)
-    ms = [v for v in (34, 35, 36) if U.mma_strip_variant_applies(d, 7, v - 34) and (v != 34 or co <= 16)]
-    for variant in [-1, 3, 6, 7, 11, 12, 14, 15, 17, 18, 20, 21, 22, 23, 25, 26, 27, 28, 30, 31, 32, 33] + ms:
+    for variant in U.all_variants(d, 7, 9, n=2, epi=epi, want_y=True, want_packed=True, min_count=12):
         out = U.run_conv(qa, qw, d, epi, want_acc=False, want_y=True, next_bits=next_bits, variant=variant)
         assert np.array_equal(out["y"], y_ref), f"variant {variant}"
         assert np.array_equal(oracle.unpack_acts(out["packed"], co), q_ref), f"variant {variant}"

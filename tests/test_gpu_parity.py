@@ -99,7 +99,10 @@ def test_conv_all_bitwidth_pairs(ebs, U, oracle, wb, ab):
     d = U.desc_for(40, 21, 3, 1, 1, wb, ab)
     ref = oracle.conv2d_codes(qa, qw, (1, 1), (1, 1))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
-    for variant in (-1, 0, 4, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28, 29, 30, 31, 32, 33):
+    variants = U.all_variants(d, 11, 13, n=3, min_count=30)    # every family has instantiations per bit count
+    for fam in ("popc", "mma", "umma", "umma_strip", "umma_resident", "umma_pipe"):
+        assert any(ebs.ebs_conv_variant_family(v) == fam for v in variants if v >= 0), fam
+    for variant in variants:
         got = U.run_conv(qa, qw, d, variant=variant, px=px, pw=pw)["acc"]
         assert np.array_equal(got, ref), f"variant {variant}"
 
@@ -126,13 +129,16 @@ def test_warp_level_strip_kernel_all_activation_bitwidths(ebs, U, oracle, ab, c,
                             (ebs.epilogue(to(cs), to(cb), None, True, 3, 0.6), (cs, cb))):
         y_ref, q_ref = oracle.epilogue(ref, S, ecs, ecb, None, relu=True, next_bits=3,
                                        inv_next=np.float32(1.0) / np.float32(0.6))
-        for variant in (34, 35, 36):
-            if not U.mma_strip_variant_applies(d, 11, variant - 34) or (variant == 34 and co > 16):
-                continue                                      # 16-channel tiles cannot write packed words of wider layers
+        ran = 0
+        for variant in U.variants_of("mma_strip"):
+            if not U.applies(d, 13, 11, variant, n=3, epi=epi, want_y=True, want_packed=True):
+                continue                                      # e.g. 16-channel tiles cannot write packed words of wider layers
+            ran += 1
             out = U.run_conv(qa, qw, d, epi, want_acc=True, want_y=True, next_bits=3, variant=variant, px=px, pw=pw)
             assert np.array_equal(out["acc"], ref), f"variant {variant}"
             assert np.array_equal(out["y"], y_ref), f"variant {variant}"
             assert np.array_equal(oracle.unpack_acts(out["packed"], co), q_ref), f"variant {variant}"
+        assert ran >= 1
 
 
 GEOMS = [
@@ -153,7 +159,7 @@ def test_conv_geometries_all_variants(ebs, U, oracle, geom):
     d = U.desc_for(c, co, k, s, pad, wb, ab)
     ref = oracle.conv2d_codes(qa, qw, (s, s), (pad, pad))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
-    for variant in U.all_variants(d, w):
+    for variant in U.all_variants(d, w, h, n=2, min_count=10):
         got = U.run_conv(qa, qw, d, variant=variant, px=px, pw=pw)["acc"]
         assert got.shape == ref.shape and np.array_equal(got, ref), f"variant {variant}"
 
@@ -161,12 +167,10 @@ def test_conv_geometries_all_variants(ebs, U, oracle, geom):
 def test_strip_kernel_refuses_strided_layers(ebs, U):
     d = U.desc_for(32, 32, 3, 2, 1, 2, 2)
     qa, qw = np.zeros((1, 32, 8, 8), np.int32), np.zeros((32, 32, 3, 3), np.int32)
-    with pytest.raises(RuntimeError):
-        U.run_conv(qa, qw, d, variant=28)
-    with pytest.raises(RuntimeError):
-        U.run_conv(qa, qw, d, variant=33)
-    with pytest.raises(RuntimeError):
-        U.run_conv(qa, qw, d, variant=36)
+    for fam in ("umma_strip", "umma_resident", "mma_strip"):
+        for variant in U.variants_of(fam):
+            with pytest.raises(RuntimeError):
+                U.run_conv(qa, qw, d, variant=variant)
 
 
 @pytest.mark.parametrize("c,co,k,s,pad,h,n,wb,ab", [(32, 64, 3, 1, 1, 30, 48, 2, 3), (64, 48, 1, 2, 0, 40, 64, 4, 2),
@@ -182,18 +186,15 @@ def test_persistent_kernel_walks_several_tiles_per_cta(ebs, U, oracle, c, co, k,
                                    inv_next=np.float32(1.0) / np.float32(0.9))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
     epi = ebs.epilogue(relu=True, next_a_bits=4, next_a_scale=0.9)
-    nv = ebs.ebs_num_conv_variants() - U.N_MMA_STRIP
     ran = 0
-    for variant in range(nv - U.N_RESIDENT, nv):
-        if not U.resident_variant_applies(d, h, 16 << (variant - (nv - U.N_RESIDENT))):
-            continue
-        if (16 << (variant - (nv - U.N_RESIDENT))) < min(co, 32):
-            continue                                          # 16-channel tiles cannot write packed words of wider layers
+    for variant in U.variants_of("umma_resident") + U.variants_of("umma_pipe"):
+        if not U.applies(d, h, h, variant, n=n, epi=epi, want_y=True, want_packed=True):
+            continue                                          # e.g. 16-channel tiles cannot write packed words of wider layers
         out = U.run_conv(qa, qw, d, epi, want_acc=True, want_y=True, next_bits=4, variant=variant, px=px, pw=pw)
         assert np.array_equal(out["acc"], ref), f"variant {variant}"
         assert np.array_equal(out["y"], y_ref) and np.array_equal(oracle.unpack_acts(out["packed"], co), q_ref)
         ran += 1
-    assert ran >= 2 and ebs.ebs_device_wait_timeouts() == 0
+    assert ran >= 4 and ebs.ebs_device_wait_timeouts() == 0
 
 
 def test_no_device_wait_timed_out(ebs):
@@ -260,9 +261,9 @@ def test_fused_epilogue_and_requantized_planes(ebs, U, oracle, next_bits, co):
     for y_layout in (ebs.EBS_NHWC, ebs.EBS_NCHW):
         epi = ebs.epilogue(to(cs), to(cb), res_nhwc, True, next_bits, float(next_scale), y_layout)
         # the warp-level strip kernels write NHWC only; their 16-channel tile cannot pack wider layers
-        ms = [v for v in (34, 35, 36) if y_layout == ebs.EBS_NHWC and U.mma_strip_variant_applies(d, 10, v - 34)
-              and (v != 34 or co <= 16)]
-        for variant in [-1, 3, 6, 7, 11, 12, 14, 15, 17, 18, 20, 21, 22, 23, 25, 26, 27, 28, 30, 31, 32, 33] + ms:
+        # every variant the library accepts for this request (e.g. the warp-level strip kernels write NHWC only and
+        # 16-channel tiles cannot pack wider layers: the library says so itself)
+        for variant in U.all_variants(d, 10, 9, n=2, epi=epi, want_y=True, want_packed=True, min_count=12):
             out = U.run_conv(qa, qw, d, epi, want_acc=True, want_y=True, next_bits=next_bits, variant=variant)
             assert np.array_equal(out["acc"], ref_acc)
             assert np.allclose(out["y"], y_ref, rtol=RTOL, atol=0.0)
@@ -371,7 +372,7 @@ def test_conv_edge_cases_all_variants(ebs, U, oracle, case):
     d = U.desc_for(c, co, k, s, pad, wb, ab)
     ref = oracle.conv2d_codes(qa, qw, (s, s), (pad, pad))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
-    for variant in U.all_variants(d, w):
+    for variant in U.all_variants(d, w, h, n=n, min_count=10):
         got = U.run_conv(qa, qw, d, variant=variant, px=px, pw=pw)["acc"]
         assert got.shape == ref.shape and np.array_equal(got, ref), f"variant {variant}"
     assert ebs.ebs_device_wait_timeouts() == 0
@@ -409,12 +410,8 @@ def test_conv_with_paper_weight_levels_all_variants(ebs, U, oracle, wb, ab, c, c
     y_ref, q_ref = oracle.epilogue(ref, S, relu=True, next_bits=3, inv_next=np.float32(1.0) / np.float32(0.4))
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qs, d)
     epi = ebs.epilogue(relu=True, next_a_bits=3, next_a_scale=0.4)
-    for variant in U.all_variants(d, 9):
-        try:
-            out = U.run_conv(qa, qs, d, epi, want_acc=True, want_y=True, next_bits=3, variant=variant, px=px, pw=pw)
-        except ebs.EbsError as exc:                      # 16-channel tiles cannot produce packed words of wider layers
-            assert exc.status == ebs.EBS_ERR_UNSUPPORTED
-            continue
+    for variant in U.all_variants(d, 9, 10, n=2, epi=epi, want_y=True, want_packed=True, min_count=8):
+        out = U.run_conv(qa, qs, d, epi, want_acc=True, want_y=True, next_bits=3, variant=variant, px=px, pw=pw)
         assert np.array_equal(out["acc"], ref), f"variant {variant}"
         assert np.array_equal(out["y"], y_ref), f"variant {variant}"
         assert np.array_equal(oracle.unpack_acts(out["packed"], co), q_ref), f"variant {variant}"

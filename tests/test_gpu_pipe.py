@@ -1,0 +1,100 @@
+"""The persistent pipeline tcgen05 kernels (family "umma_pipe") against the CPU oracle: every stride form of the
+addressing (stride 1, strided k x k as phase images, strided 1x1), several accumulators per tile, resident and
+streamed weights, many tiles per thread block, all activation bit counts, and the give-up path of its bounded waits."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ebs():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import paper_2003_07577_b200 as pkg
+    from paper_2003_07577_b200 import binding
+    if not os.path.exists(binding.LIB_PATH):
+        pkg.build()
+    binding.lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def U(ebs):
+    from tests import _util
+    return _util
+
+
+def _check(ebs, U, oracle, n, c, co, k, s, pad, h, w, wb, ab, nb, affine=False, min_variants=1):
+    rng = np.random.default_rng(n + 3 * c + 5 * co + 7 * k + 11 * s + h + w + wb * 16 + ab)
+    qa = U.rand_codes(rng, (n, c, h, w), ab, False)
+    m = (1 << (wb - 1)) - 1
+    assert m >= 1
+    qw = rng.integers(-m, m + 1, size=(co, c, k, k), dtype=np.int32)   # symmetric codes: zero-mean accumulators, half survive the ReLU
+    d = U.desc_for(c, co, k, s, pad, wb, ab, 0.03, 0.07)
+    ref = oracle.conv2d_codes(qa, qw, (s, s), (pad, pad))
+    S = oracle.combined_scale(0.03, 0.07)
+    cs = rng.uniform(0.5, 2.0, co).astype(np.float32) if affine else None
+    cb = rng.uniform(-0.3, 0.3, co).astype(np.float32) if affine else None
+    y0, _ = oracle.epilogue(ref, S, cs, cb, None, relu=True)
+    step = np.float32(max(float(np.percentile(y0, 99)), 1e-3) / ((1 << nb) - 1))
+    y_ref, q_ref = oracle.epilogue(ref, S, cs, cb, None, relu=True, next_bits=nb, inv_next=np.float32(1.0) / step)
+    to = lambda a: None if a is None else torch.from_numpy(a).to(U.dev())
+    epi = ebs.epilogue(to(cs), to(cb), None, True, nb, float(step))
+    px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
+    ran = 0
+    for variant in U.variants_of("umma_pipe"):
+        if not U.applies(d, h, w, variant, n=n, epi=epi, want_y=True, want_packed=True):
+            continue
+        out = U.run_conv(qa, qw, d, epi, want_acc=True, want_y=True, next_bits=nb, variant=variant, px=px, pw=pw)
+        assert np.array_equal(out["acc"], ref), f"variant {variant}: accumulators"
+        assert np.array_equal(out["y"], y_ref), f"variant {variant}: fp32 outputs"
+        assert np.array_equal(out["packed"], oracle.pack_acts(q_ref, nb)), f"variant {variant}: packed words"
+        # packed-only output (the mode a network runs in)
+        out = U.run_conv(qa, qw, d, epi, want_acc=False, want_y=False, next_bits=nb, variant=variant, px=px, pw=pw)
+        assert np.array_equal(out["packed"], oracle.pack_acts(q_ref, nb)), f"variant {variant}: packed only"
+        ran += 1
+    assert ran >= min_variants
+    assert q_ref.max() == (1 << nb) - 1
+    assert ebs.ebs_device_wait_timeouts() == 0
+
+
+@pytest.mark.parametrize("ab", range(1, 9))
+@pytest.mark.parametrize("nb", [1, 3, 4, 8])
+def test_pipe_all_activation_and_output_bit_counts(ebs, U, oracle, ab, nb):
+    """3x3 stride 1, 64 -> 128 channels, whole channel tiles (the straight-line epilogue), several tiles."""
+    _check(ebs, U, oracle, 5, 64, 128, 3, 1, 1, 14, 13, 2 + (ab + nb) % 7, ab, nb, min_variants=2)
+
+
+@pytest.mark.parametrize("case", [
+    # n, c, co, k, stride, pad, h, w
+    (6, 64, 64, 3, 2, 1, 15, 14),       # strided 3x3: four phase images, odd and even sizes
+    (3, 96, 128, 3, 2, 1, 16, 16),
+    (4, 64, 256, 1, 2, 0, 14, 14),      # strided 1x1: one phase
+    (2, 128, 64, 1, 1, 0, 20, 19),      # 1x1 stride 1: up to four accumulators per tile
+    (2, 40, 70, 3, 1, 1, 9, 12),        # ragged input and output channels: general epilogue
+    (3, 64, 64, 5, 2, 2, 13, 13),       # 5x5 stride 2: taps with quotients -1, 0, 1
+    (2, 32, 64, 2, 2, 0, 12, 12),       # even kernel, stride = kernel
+    (1, 64, 64, 3, 1, 0, 8, 8),         # no padding
+    (3, 64, 128, 7, 2, 3, 20, 18),      # 49 taps
+    (9, 256, 128, 3, 1, 1, 7, 7),       # small images: a strip spans several images
+])
+@pytest.mark.parametrize("affine", [False, True])
+def test_pipe_geometries(ebs, U, oracle, case, affine):
+    n, c, co, k, s, pad, h, w = case
+    _check(ebs, U, oracle, n, c, co, k, s, pad, h, w, 3, 4, 4, affine=affine)
+
+
+def test_pipe_streams_weights_that_do_not_fit_in_shared_memory(ebs, U, oracle):
+    """512 -> 256 channels, 3x3: 1.2 MB of weight bytes per 256-channel tile stream through the stage ring."""
+    _check(ebs, U, oracle, 4, 512, 256, 3, 1, 1, 9, 9, 4, 3, 3, min_variants=3)
+    _check(ebs, U, oracle, 2, 2048, 512, 1, 1, 0, 10, 10, 2, 5, 2, min_variants=3)
+
+
+def test_pipe_many_tiles_per_thread_block(ebs, U, oracle):
+    """More work items than SMs: the stage ring, both accumulator sets and the item loop wrap around several times."""
+    _check(ebs, U, oracle, 40, 64, 64, 3, 1, 1, 34, 34, 2, 2, 2, min_variants=1)
+    _check(ebs, U, oracle, 64, 64, 256, 1, 1, 0, 28, 28, 5, 6, 5, min_variants=3)
