@@ -155,20 +155,17 @@ static int choose_strip_variant(const ConvParams& p) {
 // enough output tiles; smaller layers run faster on the warp-level kernels.  Returns the variant or -1.
 // The persistent pipeline kernel covers stride-1 and strided k x k layers and 1x1 layers at any stride.  It pays off
 // when the layer has at least 64 output channels and enough outputs to fill the GPU.  Channel tile: the widest of
-// 256/128/64 that divides c_out and still leaves about two tiles per SM (every tile whole: straight-line epilogue,
-// and the fewer channel tiles, the less often an input pixel is expanded); failing that the widest that applies.
-// Returns the pipeline variant (0..2) or -1.
+// 256/128/64 that divides c_out (every tile whole: straight-line epilogue; the fewer channel tiles, the less often an
+// input pixel is expanded and the less weight traffic per multiply -- measured faster even where it leaves some SMs
+// without a tile).  Returns the pipeline variant (0..2) or -1.
 static int choose_pipe_variant(const ConvParams& p, int sms) {
+    (void)sms;
     if (p.Co < 64 || (long long)p.P * p.Co < (1LL << 19) || p.w_levels || p.fold != 1) return -1;
-    int fallback = -1;
     for (int v = 2; v >= 0; --v) {
-        const int tile_n = 64 << v;
-        if (p.Co % tile_n != 0 && !(v == 0)) continue;
-        if (!conv_umma_pipe_applies(p, v)) continue;
-        if (fallback < 0) fallback = v;
-        if (conv_umma_pipe_items(p, v) >= 2LL * sms || v == 0) return v;
+        if (p.Co % (64 << v) != 0 && v != 0) continue;
+        if (conv_umma_pipe_applies(p, v)) return v;
     }
-    return fallback;
+    return -1;
 }
 
 static int choose_umma_variant(const ConvParams& p, const ebs_conv_desc* d) {
@@ -234,6 +231,10 @@ static int conv_plan(const void* packed_x, int n, int h, int w, const void* pack
     p.w_levels = d->w_levels;
     p.fold = d->c_in <= 4 ? 8 : (d->c_in <= 8 ? 4 : (d->c_in <= 16 ? 2 : 1));
     p.fold_bits = 32 / p.fold;
+    {
+        const long long wmax = d->w_levels ? (1LL << d->w_bits) - 1 : (1LL << (d->w_bits - 1));
+        p.acc_small = (long long)d->c_in * d->kh * d->kw * wmax * ((1LL << d->a_bits) - 1) < (1LL << 22) ? 1 : 0;
+    }
     p.wait_limit = g_wait_limit;
     p.test_flags = g_test_flags;
     if (epi) {

@@ -65,6 +65,23 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     *abort_flag = 1;
     return false;
 }
+// The same wait for the single warps that feed the tensor core (issuer, weight producer): no sleep between polls (the
+// try_wait itself suspends the thread for a while), so that they react as soon as the barrier flips.
+__device__ __forceinline__ bool mbar_wait_bounded_hot(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned limit) {
+    const uint32_t addr = smem_u32(bar);
+    for (unsigned it = 0; it < limit; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}\n"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
 
 // Shared-memory matrix descriptor: K-major operand, 32-byte swizzle, rows of 32 bytes (K = 32 int8),
 // 8-row groups 256 bytes apart.
@@ -88,8 +105,8 @@ __device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t desc_a, uint64
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}\n"
-        :: "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}\n"
+        :: "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {

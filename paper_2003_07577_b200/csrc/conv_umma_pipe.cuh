@@ -41,6 +41,8 @@ constexpr int PIPE_THREADS = (PIPE_EPI_WARP0 + PIPE_EPI_WARPS) * 32;
 constexpr int PIPE_SLOTS = 2;                      // (pixel, word) items an expander thread handles per stage
 constexpr int PIPE_MAX_ITEMS = PIPE_SLOTS * PIPE_EXPANDERS;
 constexpr int PIPE_MAX_TAPS = 64, PIPE_MAX_PHASES = 4, PIPE_MAX_STAGES = 4;
+constexpr int PIPE_MAX_BSLOTS = 32;                // weight tiles in flight when the weights stream
+constexpr int PIPE_MAX_MMAS = 512;                 // MMAs of one chunk (table of their operand offsets in shared memory)
 constexpr int PIPE_SMEM_MAX = 220 * 1024;
 
 // Exact unsigned division by a run-time constant: q = (t + ((n - t) >> s1)) >> s2, t = mulhi(m, n).
@@ -69,10 +71,12 @@ struct PipeGeom {
     int m_sub, tile_pix;               // accumulators per super-tile; 128 * m_sub
     int n_ptiles, n_ctiles;
     int S, SP;                         // strip pixels (tile_pix + largest tap shift), rounded up to 8
-    int ks, nwg;                       // reduction words per stage; word groups = ceil(CW / ks)
+    int ks, nsub, kss, nwg;            // words per expander pass; passes per stage; words per stage = ks * nsub;
+                                       // word groups (stages per tile and phase) = ceil(CW / kss)
     int n_ph, nchunks;                 // phases; chunks per tile = n_ph * nwg (phase-major)
     int n_stages, a_word_bytes, a_stage_bytes, stage_bytes;
     int b_resident, b_total_bytes, taps;
+    int b_slots, b_group;              // streamed weights: ring of slots of b_group (tap, word) tiles of TILE_N x 32 bytes
     int nbuf, tmem_cols, smem_bytes;
     int grid_x, grid_y;
     int ph_a[PIPE_MAX_PHASES], ph_b[PIPE_MAX_PHASES];
@@ -140,7 +144,7 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
         if (nb == 1 && deep < 64 && !m_sub_req) continue;        // shallow reductions want the epilogue overlapped
         if (m * UMMA_M + max_shift > PIPE_MAX_ITEMS) continue;
         const long long pt = (frame + (long long)m * UMMA_M - 1) / ((long long)m * UMMA_M);
-        if (!m_sub_req && m > 1 && pt * g.n_ctiles < 2LL * sms) continue;
+        if (!m_sub_req && m > 1 && pt * g.n_ctiles < (deep >= 64 ? 1LL : 2LL) * sms) continue;
         m_sub = m;
         break;
     }
@@ -156,29 +160,49 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
     g.a_word_bytes = g.SP * 32 + 32;
     if (g.SP * 16 >= (1 << 18)) return g;
     // weights resident when they leave room for at least two activation stages
-    const int budget = PIPE_SMEM_MAX - 2048;
+    const int budget = PIPE_SMEM_MAX - 2048 - PIPE_MAX_MMAS * 8;   // the MMA table sits behind the rings
     g.b_resident = g.b_total_bytes + 2 * ((g.a_word_bytes + 255) & ~255) <= budget && g.b_total_bytes <= 160 * 1024;
     int ks = PIPE_MAX_ITEMS / g.S;
     if (ks > 4) ks = 4;
     if (ks > p.CW) ks = p.CW;
     if (ks < 1) return g;
-    auto stage_bytes = [&](int k) {
-        const int a = (k * g.a_word_bytes + 255) & ~255;
-        return a + (g.b_resident ? 0 : k * max_ph_taps * b_tile);
-    };
-    const int avail = budget - (g.b_resident ? g.b_total_bytes : 0);
+    while (ks > 1 && ks * taps * m_sub >= PIPE_MAX_MMAS) --ks;     // (the issue loop reads one entry ahead)
+    if (ks * taps * m_sub >= PIPE_MAX_MMAS) return g;
+    // Streamed weights go through a ring of their own (slots of a few consecutive (tap, word) tiles), so that copies are
+    // in flight all the time (a stage-sized unit would leave the copy engine idle while a stage's MMAs run).
+    auto stage_bytes = [&](int k) { return (k * g.a_word_bytes + 255) & ~255; };
+    const int b_ring_min = g.b_resident ? 0 : 96 * 1024;
+    const int avail = budget - (g.b_resident ? g.b_total_bytes : b_ring_min);
     while (ks > 1 && 2 * stage_bytes(ks) > avail) --ks;
     if (2 * stage_bytes(ks) > avail) return g;
-    // fewer words per stage when that buys a deeper ring (latency hiding matters more than stage size)
+    // fewer words per pass when that buys a deeper ring (latency hiding matters more than stage size)
     while (ks > 1 && avail / stage_bytes(ks) < 3) --ks;
+    // A stage is filled in nsub expander passes of ks words: the thread that issues the MMAs retires an instruction
+    // only every ten clocks or so, so its per-stage bookkeeping has to be spread over about a dozen MMAs.
+    int nsub = 1;
+    while (nsub < 4 && ks * nsub * taps * m_sub < 12 && ks * nsub < p.CW &&
+           ks * 2 * nsub * taps * m_sub < PIPE_MAX_MMAS && 3 * stage_bytes(ks * 2 * nsub) <= avail)
+        nsub *= 2;
     g.ks = ks;
-    g.nwg = (p.CW + ks - 1) / ks;
+    g.nsub = nsub;
+    g.kss = ks * nsub;
+    g.nwg = (p.CW + g.kss - 1) / g.kss;
     g.nchunks = g.n_ph * g.nwg;
-    g.a_stage_bytes = (ks * g.a_word_bytes + 255) & ~255;
-    g.stage_bytes = stage_bytes(ks);
+    g.a_stage_bytes = stage_bytes(g.kss);
+    g.stage_bytes = g.a_stage_bytes;
     g.n_stages = avail / g.stage_bytes;
-    if (g.n_stages > PIPE_MAX_STAGES) g.n_stages = PIPE_MAX_STAGES;
-    g.smem_bytes = (g.b_resident ? g.b_total_bytes : 0) + g.n_stages * g.stage_bytes + 1024;
+    if (g.n_stages > (g.b_resident ? PIPE_MAX_STAGES : 3)) g.n_stages = g.b_resident ? PIPE_MAX_STAGES : 3;
+    if (!g.b_resident) {
+        // a slot holds up to 32 KB of consecutive tiles of a chunk (one wait and one commit per slot, not per MMA)
+        g.b_group = 32768 / b_tile;
+        if (g.b_group > g.kss * max_ph_taps) g.b_group = g.kss * max_ph_taps;
+        if (g.b_group < 1) g.b_group = 1;
+        g.b_slots = (budget - g.n_stages * g.stage_bytes) / (g.b_group * b_tile);
+        if (g.b_slots > PIPE_MAX_BSLOTS) g.b_slots = PIPE_MAX_BSLOTS;
+        if (g.b_slots < 3) return g;
+    }
+    g.smem_bytes = (g.b_resident ? g.b_total_bytes : g.b_slots * g.b_group * b_tile) + g.n_stages * g.stage_bytes + 1024 +
+                   PIPE_MAX_MMAS * 8;
     if (g.b_resident) {                                        // a CTA keeps one channel tile
         g.grid_y = g.n_ctiles;
         long long gx = sms / g.n_ctiles;
@@ -196,7 +220,56 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
 
 // One 32-channel group of the plain epilogue: 32 accumulators of this thread's pixel -> stores, fp32 steps,
 // requantized codes -> plane words.
-template <bool WANT_Q>
+// tcgen05.mma with both descriptors given as (low word, high word): the start-address field sits in the low word, so
+// an operand is moved by a 32-bit addition.  The whole warp executes the call with the same operands and the
+// instruction is predicated on `leader` (non-zero in one lane): with the issue loop free of divergent branches its
+// address arithmetic stays warp-uniform, which measured faster than a loop run by one thread alone.
+__device__ __forceinline__ void umma_i8_split(uint32_t leader, uint32_t tmem_d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                              uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "setp.ne.b32 q, %7, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t}\n"
+        :: "r"(tmem_d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(leader)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_pred(uint32_t leader, uint64_t* bar) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}\n"
+        ::"r"(smem_u32(bar)), "r"(leader) : "memory");
+}
+
+// Two fp32 values in one 64-bit register for the packed fp32 instructions (one issue slot for two results; each lane is
+// an individually rounded IEEE operation, identical to the scalar instruction).
+__device__ __forceinline__ uint64_t f32x2_pack(float lo, float hi) {
+    return ((uint64_t)__float_as_uint(hi) << 32) | (uint64_t)__float_as_uint(lo);
+}
+__device__ __forceinline__ uint64_t f32x2_mul_rn(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t f32x2_add_rn(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t f32x2_add_rd(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rm.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+//
+// The float -> int conversion issues at an eighth of the fp32 rate on this machine (16 results per clock and SM against
+// 128 fp32 operations) and was what bounded the epilogue, so the floor and the clamp are done with an fp32 addition and
+// integer min / max instead (see below); the fp32 steps run as packed two-lane instructions.
+template <bool WANT_Q, bool SMALL_ACC>
 __device__ __forceinline__ void pipe_group32(const ConvParams& p, uint32_t (&v)[32], size_t o, bool pvalid, float S,
                                              float inv_next, int nb, int qmax, uint32_t* dst) {
     if (p.acc && pvalid) {
@@ -205,30 +278,51 @@ __device__ __forceinline__ void pipe_group32(const ConvParams& p, uint32_t (&v)[
             *reinterpret_cast<int4*>(p.acc + o + 4 * gq) =
                 make_int4((int)v[4 * gq], (int)v[4 * gq + 1], (int)v[4 * gq + 2], (int)v[4 * gq + 3]);
     }
-    float y[32];
+    // y = fl(float(acc) * S) for the 32 channels, two to a register: pair (h, bb) = channels 16h + bb and 16h + 8 + bb
+    uint64_t yy[2][8];
+    const uint64_t S2 = f32x2_pack(S, S);
 #pragma unroll
-    for (int e = 0; e < 32; ++e) y[e] = __fmul_rn((float)(int)v[e], S);
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int bb = 0; bb < 8; ++bb)
+            yy[h][bb] = f32x2_mul_rn(f32x2_pack((float)(int)v[16 * h + bb], (float)(int)v[16 * h + 8 + bb]), S2);
     if (p.y && pvalid) {
         const bool relu = p.relu != 0;
 #pragma unroll
         for (int gq = 0; gq < 8; ++gq) {
-            float4 t = make_float4(y[4 * gq], y[4 * gq + 1], y[4 * gq + 2], y[4 * gq + 3]);
-            if (relu) { t.x = t.x > 0.f ? t.x : 0.f; t.y = t.y > 0.f ? t.y : 0.f; t.z = t.z > 0.f ? t.z : 0.f; t.w = t.w > 0.f ? t.w : 0.f; }
-            *reinterpret_cast<float4*>(p.y + o + 4 * gq) = t;
+            float t[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int c = 4 * gq + e;                           // channel c: pair (c / 16, c % 8), upper lane if c & 8
+                const uint64_t w = yy[c >> 4][c & 7];
+                t[e] = __uint_as_float((c & 8) ? (uint32_t)(w >> 32) : (uint32_t)w);
+                if (relu) t[e] = t[e] > 0.f ? t[e] : 0.f;
+            }
+            *reinterpret_cast<float4*>(p.y + o + 4 * gq) = make_float4(t[0], t[1], t[2], t[3]);
         }
     }
     if (WANT_Q) {
         // The clamp at zero of the quantizer makes an explicit ReLU redundant here: a negative y gives
         // floor(y / step + 0.5) <= 0 and is clamped to code 0, exactly what max(y, 0) would give.
+        // floor(t) sits in the low mantissa bits of t + 2^23 added with rounding toward minus infinity; as integers the
+        // bit patterns of these sums are ordered like the sums themselves (negative ones below all others), so the
+        // clamp to 0 .. qmax is an integer clamp of the pattern to [bits(2^23), bits(2^23) + qmax].
         // Byte register bb holds the codes of channels {bb, 8 + bb, 16 + bb, 24 + bb}, rotated left by bb.
         uint32_t cr[8];
+        const uint64_t inv2 = f32x2_pack(inv_next, inv_next), half2 = f32x2_pack(0.5f, 0.5f),
+                       magic2 = f32x2_pack(8388608.0f, 8388608.0f);
+        const int m_lo = 0x4B000000, m_hi = 0x4B000000 + qmax;
 #pragma unroll
         for (int bb = 0; bb < 8; ++bb) {
-            int q[4];
+            int m[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                q[i] = min(__float2int_rd(__fadd_rn(__fmul_rn(y[8 * i + bb], inv_next), 0.5f)), qmax);
-            const uint32_t c4 = pack_sat_u8x4(q[0], q[1], q[2], q[3]);      // saturates at 0 (negative values)
+            for (int h = 0; h < 2; ++h) {
+                const uint64_t t = f32x2_add_rd(f32x2_add_rn(f32x2_mul_rn(yy[h][bb], inv2), half2), magic2);
+                m[2 * h] = min(max((int)(uint32_t)t, m_lo), m_hi);
+                m[2 * h + 1] = min(max((int)(uint32_t)(t >> 32), m_lo), m_hi);
+            }
+            const uint32_t c4 = __byte_perm(__byte_perm((uint32_t)m[0], (uint32_t)m[1], 0x0040),
+                                            __byte_perm((uint32_t)m[2], (uint32_t)m[3], 0x0040), 0x5410);
             cr[bb] = __funnelshift_l(c4, c4, bb);
         }
         uint32_t planes[8];
@@ -285,8 +379,12 @@ __device__ __forceinline__ void pipe_epilogue_plain(const ConvParams& p, uint32_
         tmem_ld16_wait(hi);
         const size_t o = (size_t)gp * p.Co + co0 + c0;
         uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + ((co0 + c0) >> 5)) * nb;
-        if (want_q) pipe_group32<true>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
-        else pipe_group32<false>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
+        if (want_q) {
+            if (p.acc_small) pipe_group32<true, true>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
+            else pipe_group32<true, false>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
+        } else {
+            pipe_group32<false, false>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
+        }
     }
 }
 
@@ -295,16 +393,52 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
     constexpr int B_TILE_BYTES = TILE_N * 32;
     extern __shared__ uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t st_full[PIPE_MAX_STAGES], st_empty[PIPE_MAX_STAGES], acc_full[2], acc_empty[2], b_full;
+    __shared__ __align__(8) uint64_t bs_full[PIPE_MAX_BSLOTS], bs_empty[PIPE_MAX_BSLOTS];   // streamed weight tiles
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ uint32_t s_tap_shift[PIPE_MAX_TAPS];     // tap tables in shared memory: indexed at run time by single threads
+    __shared__ int s_tap_id[PIPE_MAX_TAPS];
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int NST = g.n_stages, KS = g.ks, SP = g.SP, S = g.S;
+    if (tid < PIPE_MAX_TAPS) {
+        s_tap_shift[tid] = (uint32_t)g.tap_shift[tid];
+        s_tap_id[tid] = (int)g.tap_id[tid];
+    }
+    // Table of the MMAs of a chunk, per phase, in issue order (word, tap, accumulator): x = offset of the activation
+    // operand from the stage start (16-byte units: word, tap shift, 128 pixels per accumulator), y = accumulator column
+    // offset | (advance of the weight operand after this MMA) << 16.  The issuing thread then spends a load, three
+    // additions and the MMA per step; with operand addresses computed in its loop it was the slowest stage of the
+    // pipeline (a single thread retires an instruction every 5 to 10 clocks).
+    uint2* mma_tab = reinterpret_cast<uint2*>(dyn_smem + ((1024u - (smem_u32(dyn_smem) & 1023u)) & 1023u) +
+                                              (g.smem_bytes - 1024 - PIPE_MAX_MMAS * 8));
+    {
+        const int per_tap = g.kss * g.m_sub, total_e = per_tap * g.taps;
+        const uint32_t bt16 = (uint32_t)(TILE_N * 32) >> 4;
+        for (int e = tid; e < total_e; e += PIPE_THREADS) {
+            int ph = 0;
+            while (ph + 1 < g.n_ph && e >= per_tap * g.ph_tap0[ph + 1]) ++ph;
+            const int t0 = g.ph_tap0[ph], ntp = g.ph_tap0[ph + 1] - t0;
+            const int local = e - per_tap * t0;
+            const int q = local / (ntp * g.m_sub), r = local - q * (ntp * g.m_sub);
+            const int tl = r / g.m_sub, j = r - tl * g.m_sub;
+            const uint32_t a_off = (uint32_t)(q * (g.a_word_bytes >> 4) + g.tap_shift[t0 + tl] + j * UMMA_M);
+            uint32_t b_inc = 0u;
+            if (j == g.m_sub - 1)
+                b_inc = (g.b_resident && tl == ntp - 1) ? bt16 * (uint32_t)(1 + g.taps - ntp) : bt16;
+            mma_tab[e] = make_uint2(a_off, (uint32_t)(j * TILE_N) | (b_inc << 16));
+        }
+    }
+    const int NST = g.n_stages, KS = g.ks, KSS = g.kss, NSUB = g.nsub, SP = g.SP, S = g.S;
     const int nchunks = g.nchunks, nwg = g.nwg;
     const bool resident = g.b_resident != 0;
     uint8_t* base = dyn_smem + ((1024u - (smem_u32(dyn_smem) & 1023u)) & 1023u);
-    uint8_t* b_res = base;                                               // [CW][tap slots][TILE_N][32] when resident
-    uint8_t* stages = base + (resident ? g.b_total_bytes : 0);           // [NST] x ([KS][2][SP][16] A, then B tiles)
+    uint8_t* b_res = base;                                               // resident: [CW][tap slots][TILE_N][32]; else the ring of tiles
+    uint8_t* stages = base + (resident ? g.b_total_bytes : g.b_slots * g.b_group * B_TILE_BYTES);   // [NST] x [KS][2][SP][16]
+    const int NBS = g.b_slots, GB = g.b_group;
+    // Streamed weights: every CTA of a channel tile reads the same weight tiles, and CTAs that start together would ask
+    // the same few L2 slices for the same tile at the same time.  Integer accumulation is exact in any order, so each
+    // CTA starts its walk over the word groups at a different one.
+    const int wg_rot = resident ? 0 : (int)(blockIdx.x % (unsigned)nwg);
     volatile int* abortp = &abort_flag;
     const unsigned wait_limit = p.wait_limit;
 
@@ -320,8 +454,12 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
     if (tid == 0) {
         abort_flag = 0;
         for (int s = 0; s < PIPE_MAX_STAGES; ++s) {
-            mbar_init(&st_full[s], PIPE_EXPANDERS + (resident ? 0 : 1));   // expanders (+ the thread that announces the weight copies)
+            mbar_init(&st_full[s], PIPE_EXPANDERS * g.nsub);       // every expander arrives once per pass
             mbar_init(&st_empty[s], 1);
+        }
+        for (int s = 0; s < PIPE_MAX_BSLOTS; ++s) {
+            mbar_init(&bs_full[s], 1);
+            mbar_init(&bs_empty[s], 1);
         }
         mbar_init(&acc_full[0], 1);
         mbar_init(&acc_full[1], 1);
@@ -351,8 +489,8 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
             slot_pix[j] = s;
             slot_dst[j] = q * g.a_word_bytes + s * 16;
         }
-        // loader state: runs two chunks ahead of the expansion, also across tile boundaries
-        int ld_it = 0, ld_c = 0, ld_off[PIPE_SLOTS];
+        // loader state: runs several passes ahead of the expansion, also across tile boundaries
+        int ld_it = 0, ld_c = 0, ld_sub = 0, ld_off[PIPE_SLOTS];
         auto chunk_offsets = [&](int it, int ph) {
             int ptile, ctile;
             item_of(it, ptile, ctile);
@@ -372,34 +510,44 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 }
             }
         };
-        uint32_t a_set[3][PIPE_SLOTS][AB];
+        // register ring of packed words: SETS - 1 chunks of global loads in flight per thread (about 48 registers whatever
+        // the plane count: the latency of these loads, not their bandwidth, is what a deep reduction waits for)
+        constexpr int SETS = AB <= 2 ? 9 : (AB <= 4 ? 6 : (AB <= 6 ? 4 : 3));
+        uint32_t a_set[SETS][PIPE_SLOTS][AB];
+        int ld_ph = 0, ld_wg = 0;
         auto load_next = [&](int set) {
-            const int ph = ld_c / nwg, wg = ld_c - ph * nwg;
-            if (wg == 0) chunk_offsets(ld_it, ph);
+            int wg = ld_wg + wg_rot;
+            if (wg >= nwg) wg -= nwg;
+            if (ld_wg == 0 && ld_sub == 0) chunk_offsets(ld_it, ld_ph);
 #pragma unroll
             for (int j = 0; j < PIPE_SLOTS; ++j) {
 #pragma unroll
                 for (int k = 0; k < AB; ++k) a_set[set][j][k] = 0u;
-                const int cw = wg * KS + slot_q[j];
+                const int cw = wg * KSS + ld_sub * KS + slot_q[j];
                 if (slot_q[j] >= 0 && ld_off[j] >= 0 && cw < p.CW)
                     load_words_global<AB>(p.x + (ld_off[j] + cw * AB), a_set[set][j]);
             }
-            if (++ld_c == nchunks) { ld_c = 0; ++ld_it; }
+            if (++ld_sub == NSUB) {
+                ld_sub = 0;
+                if (++ld_wg == nwg) { ld_wg = 0; ++ld_ph; }
+                if (++ld_c == nchunks) { ld_c = 0; ld_ph = 0; ++ld_it; }
+            }
         };
-        const int total = my_items * nchunks;
-        if (total > 0) load_next(0);
-        if (total > 1) load_next(1);
-        bool ok = true;
-        int st = 0;
-        uint32_t st_round = 0;                                  // how many times the ring has wrapped
-        for (int g0 = 0; g0 < total && ok; g0 += 3) {
+        const int total = my_items * nchunks * NSUB;           // expander passes
 #pragma unroll
-            for (int u = 0; u < 3; ++u) {
+        for (int u = 0; u < SETS - 1; ++u)
+            if (u < total) load_next(u);
+        bool ok = true;
+        int st = 0, sub = 0;
+        uint32_t st_round = 0;                                  // how many times the ring has wrapped
+        for (int g0 = 0; g0 < total && ok; g0 += SETS) {
+#pragma unroll
+            for (int u = 0; u < SETS; ++u) {
                 const int gi = g0 + u;
                 if (gi >= total) break;
-                uint8_t* A_st = stages + st * g.stage_bytes;
-                if (gi + 2 < total) load_next((u + 2) % 3);
-                if (st_round > 0) {                             // the MMAs that read this stage one round ago must be done
+                uint8_t* A_st = stages + st * g.stage_bytes + sub * KS * g.a_word_bytes;
+                if (gi + SETS - 1 < total) load_next((u + SETS - 1) % SETS);
+                if (st_round > 0 && sub == 0) {                 // the MMAs that read this stage one round ago must be done
                     if (!mbar_wait_bounded(&st_empty[st], (st_round - 1) & 1u, abortp, wait_limit)) { ok = false; break; }
                 }
 #pragma unroll
@@ -423,52 +571,85 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 }
                 asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                 mbar_arrive(&st_full[st]);
-                if (++st == NST) { st = 0; ++st_round; }
+                if (++sub == NSUB) {
+                    sub = 0;
+                    if (++st == NST) { st = 0; ++st_round; }
+                }
             }
         }
     } else if (warp == PIPE_ISSUER_WARP) {
         // =========================== issuer ===========================
+        // The issuing thread is a pipeline stage of its own: every address is advanced by additions (descriptor start
+        // addresses are in 16-byte units), a handful of instructions per MMA.
         constexpr uint32_t IDESC = umma_idesc_i8(TILE_N);
+        constexpr uint32_t BT16 = B_TILE_BYTES >> 4;
         const bool skip_mma = (p.test_flags & 1) != 0;            // test hook: issue nothing, so that waits run out
-        bool ok = my_items == 0 || !resident || mbar_wait_bounded(&b_full, 0u, abortp, wait_limit);
-        int st = 0;
-        uint32_t st_round = 0;
+        bool ok = my_items == 0 || !resident || mbar_wait_bounded_hot(&b_full, 0u, abortp, wait_limit);
+        const uint64_t da_ring = umma_desc_interleaved(smem_u32(stages), (uint32_t)(SP * 16));
+        const uint64_t db_res = umma_desc_sw32(smem_u32(b_res));   // resident tiles, or slot 0 of the ring
+        const uint32_t da_lo = (uint32_t)da_ring, da_hi = (uint32_t)(da_ring >> 32);
+        const uint32_t db_lo = (uint32_t)db_res, db_hi = (uint32_t)(db_res >> 32);
+        const uint32_t stage16 = (uint32_t)(g.stage_bytes >> 4);
+        const int m_sub = g.m_sub;
+        const uint32_t leader = (tid & 31) == 0 ? 1u : 0u;
+        int st = 0, bs = 0;
+        uint32_t st_round = 0, bs_round = 0;
         for (int it = 0; it < my_items && ok; ++it) {
             const int buf = g.nbuf == 2 ? (it & 1) : 0;
             const int use = g.nbuf == 2 ? (it >> 1) : it;          // how often this accumulator set was used before
             if (use > 0) {                                          // its epilogue must have drained it
-                if (!mbar_wait_bounded(&acc_empty[buf], (uint32_t)((use - 1) & 1), abortp, wait_limit)) break;
+                if (!mbar_wait_bounded_hot(&acc_empty[buf], (uint32_t)((use - 1) & 1), abortp, wait_limit)) break;
             }
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-            const uint32_t tmem_d = tmem_base + (uint32_t)(buf * g.m_sub * TILE_N);
+            const uint32_t tmem_d = tmem_base + (uint32_t)(buf * m_sub * TILE_N);
+            int ph = 0, wg = 0;
             for (int c = 0; c < nchunks; ++c) {
-                if (!mbar_wait_bounded(&st_full[st], st_round & 1u, abortp, wait_limit)) { ok = false; break; }
+                if (!mbar_wait_bounded_hot(&st_full[st], st_round & 1u, abortp, wait_limit)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                if ((tid & 31) == 0 && !skip_mma) {
-                    const int ph = c / nwg, wg = c - ph * nwg;
-                    const int words = min(KS, p.CW - wg * KS);
-                    const int t0 = g.ph_tap0[ph], t1 = g.ph_tap0[ph + 1];
-                    uint8_t* stage = stages + st * g.stage_bytes;
-                    const uint64_t da0 = umma_desc_interleaved(smem_u32(stage), (uint32_t)(SP * 16));
-                    const uint32_t b_stage = smem_u32(stage + g.a_stage_bytes);
-                    for (int q = 0; q < words; ++q) {
-                        const uint64_t da_q = da0 + (uint64_t)(q * (g.a_word_bytes >> 4));
-                        for (int ts = t0; ts < t1; ++ts) {
-                            const uint32_t b_addr = resident
-                                ? smem_u32(b_res) + (uint32_t)(((wg * KS + q) * g.taps + ts) * B_TILE_BYTES)
-                                : b_stage + (uint32_t)((q * (t1 - t0) + (ts - t0)) * B_TILE_BYTES);
-                            const uint64_t db = umma_desc_sw32(b_addr);
-                            const uint64_t da_t = da_q + (uint64_t)g.tap_shift[ts];
-                            const uint32_t acc_flag = (c | q | (ts - t0)) != 0 ? 1u : 0u;
-                            for (int j = 0; j < g.m_sub; ++j)
-                                umma_i8(tmem_d + (uint32_t)(j * TILE_N), da_t + (uint64_t)(j * (UMMA_M * 16 >> 4)), db, IDESC, acc_flag);
+                if (!skip_mma) {
+                    const int wgr = wg + wg_rot >= nwg ? wg + wg_rot - nwg : wg + wg_rot;
+                    const int words = min(KSS, p.CW - wgr * KSS);
+                    const int t0 = g.ph_tap0[ph], ntp = g.ph_tap0[ph + 1] - t0;
+                    const uint2* tab = mma_tab + KSS * m_sub * t0;
+                    const int zero_n = c == 0 ? m_sub : 0;         // the first MMA into each accumulator of a tile overwrites it
+                    const uint32_t a_lo = da_lo + (uint32_t)st * stage16;
+                    if (resident) {
+                        uint32_t b_lo = db_lo + (uint32_t)((wgr * KSS) * g.taps + t0) * BT16;
+                        const int n = words * ntp * m_sub;
+                        uint2 e = tab[0];
+                        for (int i = 0; i < n; ++i) {
+                            const uint2 nxt = tab[i + 1];                 // one entry past the end is inside the table's allocation
+                            umma_i8_split(leader, tmem_d + (e.y & 0xFFFFu), a_lo + e.x, da_hi, b_lo, db_hi, IDESC, i >= zero_n ? 1u : 0u);
+                            b_lo += e.y >> 16;
+                            e = nxt;
                         }
+                    } else {
+                        // streamed weights: the chunk's (word, tap) tiles in order, GB consecutive tiles per ring slot
+                        const int ntiles = words * ntp;
+                        int i = 0;
+                        for (int i0 = 0; i0 < ntiles; i0 += GB) {
+                            if (!mbar_wait_bounded_hot(&bs_full[bs], bs_round & 1u, abortp, wait_limit)) { ok = false; break; }
+                            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                            uint32_t b_lo = db_lo + (uint32_t)(bs * GB) * BT16;
+                            const int n = i + min(GB, ntiles - i0) * m_sub;
+                            uint2 e = tab[i];
+                            for (; i < n; ++i) {
+                                const uint2 nxt = tab[i + 1];
+                                umma_i8_split(leader, tmem_d + (e.y & 0xFFFFu), a_lo + e.x, da_hi, b_lo, db_hi, IDESC, i >= zero_n ? 1u : 0u);
+                                b_lo += e.y >> 16;
+                                e = nxt;
+                            }
+                            umma_commit_pred(leader, &bs_empty[bs]);
+                            if (++bs == NBS) { bs = 0; ++bs_round; }
+                        }
+                        if (!ok) break;
                     }
-                    umma_commit(&st_empty[st]);
-                    if (c == nchunks - 1) umma_commit(&acc_full[buf]);
+                    umma_commit_pred(leader, &st_empty[st]);
+                    if (c == nchunks - 1) umma_commit_pred(leader, &acc_full[buf]);
                 }
                 __syncwarp();
                 if (++st == NST) { st = 0; ++st_round; }
+                if (++wg == nwg) { wg = 0; ++ph; }
             }
         }
     } else if (warp == PIPE_PRODUCER_WARP) {
@@ -481,31 +662,38 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 for (int cw = 0; cw < p.CW; ++cw)
                     for (int ts = 0; ts < g.taps; ++ts)
                         bulk_copy_g2s(b_res + (cw * g.taps + ts) * B_TILE_BYTES,
-                                      p.w8 + ((size_t)(g.tap_id[ts] * p.CW + cw) * p.Co16 + co0) * 32, rows * 32u, &b_full);
+                                      p.w8 + ((size_t)(s_tap_id[ts] * p.CW + cw) * p.Co16 + co0) * 32, rows * 32u, &b_full);
             } else {
-                int st = 0;
-                uint32_t st_round = 0;
+                int bs = 0;
+                uint32_t bs_round = 0;
                 bool ok = true;
                 for (int it = 0; it < my_items && ok; ++it) {
                     int ptile, ctile;
                     item_of(it, ptile, ctile);
                     const int co0 = ctile * TILE_N;
-                    const uint32_t rows = (uint32_t)min(TILE_N, p.Co16 - co0);
-                    for (int c = 0; c < nchunks; ++c) {
-                        if (st_round > 0) {
-                            if (!mbar_wait_bounded(&st_empty[st], (st_round - 1) & 1u, abortp, wait_limit)) { ok = false; break; }
-                        }
-                        const int ph = c / nwg, wg = c - ph * nwg;
-                        const int words = min(KS, p.CW - wg * KS);
+                    const uint32_t bytes = (uint32_t)min(TILE_N, p.Co16 - co0) * 32u;
+                    int ph = 0, wg = -1;
+                    for (int c = 0; c < nchunks && ok; ++c) {
+                        if (++wg == nwg) { wg = 0; ++ph; }
+                        const int wgr = wg + wg_rot >= nwg ? wg + wg_rot - nwg : wg + wg_rot;
+                        const int words = min(KSS, p.CW - wgr * KSS);
                         const int t0 = g.ph_tap0[ph], t1 = g.ph_tap0[ph + 1];
-                        uint8_t* b_stage = stages + st * g.stage_bytes + g.a_stage_bytes;
-                        mbar_arrive_expect_tx(&st_full[st], rows * 32u * (uint32_t)(words * (t1 - t0)));
-                        for (int q = 0; q < words; ++q)
-                            for (int ts = t0; ts < t1; ++ts)
-                                bulk_copy_g2s(b_stage + (q * (t1 - t0) + (ts - t0)) * B_TILE_BYTES,
-                                              p.w8 + ((size_t)(g.tap_id[ts] * p.CW + wg * KS + q) * p.Co16 + co0) * 32,
-                                              rows * 32u, &st_full[st]);
-                        if (++st == NST) { st = 0; ++st_round; }
+                        const int ntaps = t1 - t0, ntiles = words * ntaps;
+                        int q = 0, ts = t0;
+                        for (int i0 = 0; i0 < ntiles; i0 += GB) {
+                            if (bs_round > 0) {                     // the MMAs that read this slot one round ago must be done
+                                if (!mbar_wait_bounded_hot(&bs_empty[bs], (bs_round - 1) & 1u, abortp, wait_limit)) { ok = false; break; }
+                            }
+                            const int n = min(GB, ntiles - i0);
+                            mbar_arrive_expect_tx(&bs_full[bs], bytes * (uint32_t)n);
+                            for (int i = 0; i < n; ++i) {
+                                bulk_copy_g2s(b_res + (bs * GB + i) * B_TILE_BYTES,
+                                              p.w8 + ((size_t)(s_tap_id[ts] * p.CW + wgr * KSS + q) * p.Co16 + co0) * 32, bytes,
+                                              &bs_full[bs]);
+                                if (++ts == t1) { ts = t0; ++q; }
+                            }
+                            if (++bs == NBS) { bs = 0; ++bs_round; }
+                        }
                     }
                 }
             }

@@ -40,6 +40,7 @@ struct ConvParams {
     unsigned wait_limit;              // polls a bounded device-side wait makes before the CTA gives up
     int test_flags;                   // bit 0 (tests only): the MMA issuer issues nothing, so that waits run out
     int pipe_m_sub;                   // persistent pipeline kernel: accumulators per super-tile (0 = chosen by the library)
+    int acc_small;                    // 1: every accumulator of the layer is below 2^22 in magnitude (worst case of its sizes and bit counts)
 };
 
 // One instantiation of the popcount kernel: launch function + its tile geometry.
