@@ -309,15 +309,19 @@ __device__ __forceinline__ void pipe_group32(const ConvParams& p, uint32_t (&v)[
         // clamp to 0 .. qmax is an integer clamp of the pattern to [bits(2^23), bits(2^23) + qmax].
         // Byte register bb holds the codes of channels {bb, 8 + bb, 16 + bb, 24 + bb}, rotated left by bb.
         uint32_t cr[8];
-        const uint64_t inv2 = f32x2_pack(inv_next, inv_next), half2 = f32x2_pack(0.5f, 0.5f),
-                       magic2 = f32x2_pack(8388608.0f, 8388608.0f);
+        const uint64_t magic2 = f32x2_pack(8388608.0f, 8388608.0f);
         const int m_lo = 0x4B000000, m_hi = 0x4B000000 + qmax;
 #pragma unroll
         for (int bb = 0; bb < 8; ++bb) {
             int m[4];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const uint64_t t = f32x2_add_rd(f32x2_add_rn(f32x2_mul_rn(yy[h][bb], inv2), half2), magic2);
+                // (the multiply and the addition of 0.5 are scalar instructions with explicit rounding, which the assembler
+                // never contracts into a fused multiply-add; issued as a packed pair they came out fused)
+                const uint64_t w = yy[h][bb];
+                const float t_lo = __fadd_rn(__fmul_rn(__uint_as_float((uint32_t)w), inv_next), 0.5f);
+                const float t_hi = __fadd_rn(__fmul_rn(__uint_as_float((uint32_t)(w >> 32)), inv_next), 0.5f);
+                const uint64_t t = f32x2_add_rd(f32x2_pack(t_lo, t_hi), magic2);
                 m[2 * h] = min(max((int)(uint32_t)t, m_lo), m_hi);
                 m[2 * h + 1] = min(max((int)(uint32_t)(t >> 32), m_lo), m_hi);
             }

@@ -98,3 +98,39 @@ def test_pipe_many_tiles_per_thread_block(ebs, U, oracle):
     """More work items than SMs: the stage ring, both accumulator sets and the item loop wrap around several times."""
     _check(ebs, U, oracle, 40, 64, 64, 3, 1, 1, 34, 34, 2, 2, 2, min_variants=1)
     _check(ebs, U, oracle, 64, 64, 256, 1, 1, 0, 28, 28, 5, 6, 5, min_variants=3)
+
+
+def test_pipe_requantization_where_two_roundings_and_a_fused_one_differ(ebs, U, oracle):
+    """y * (1/step) + 0.5 must be a rounded multiply followed by a rounded addition.  With the step 4 * s_w * s_a * 64 of
+    the ResNet-20 bench layers the product at acc = 128 is the float just below 0.5, the sum rounds up to 1.0 (a tie, to
+    even) and the code is 1; a fused multiply-add keeps the sum below 1.0 and gives 0.  A 1x1 layer with unit weights
+    sweeps the accumulator over 0 .. 765 so that such values are present for every output bit count."""
+    spec = [s for s in __import__("workloads.gen", fromlist=["gen"]).config2(0) if s.layer.name == "s3b3c1"][0]
+    n, c, co, h, w = 4, 64, 64, 16, 12
+    qa = np.zeros((n, c, h, w), np.int32)
+    target = np.arange(n * h * w).reshape(n, h, w)                     # accumulator value wanted at each pixel
+    for ch in range(c):                                               # spread it over channels with codes 0 .. 255
+        take = np.clip(target - qa.sum(axis=1), 0, 15)
+        qa[:, ch] = take
+    qw = np.ones((co, c, 1, 1), np.int32)
+    d = U.desc_for(c, co, 1, 1, 0, 2, 4, spec.w_scale, spec.a_scale)
+    ref = oracle.conv2d_codes(qa, qw)
+    assert ref.max() >= 700 and (ref == 128).any()
+    S = oracle.combined_scale(spec.w_scale, spec.a_scale)
+    step = np.float32(4.0 * spec.w_scale * spec.a_scale * 64)
+    px, pw = U.pack_acts_codes(qa, 4), U.pack_weight_codes(qw, d)
+    fused_differs = 0
+    for nb in (1, 2, 3, 5):
+        inv = np.float32(1.0) / step
+        _, q_ref = oracle.epilogue(ref, S, relu=True, next_bits=nb, inv_next=inv)
+        y = (ref.astype(np.float32) * S).astype(np.float64)
+        q_fused = np.clip(np.floor((y * np.float64(inv) + 0.5).astype(np.float32)), 0, (1 << nb) - 1)   # one rounding
+        fused_differs += int((q_fused != q_ref).sum())
+        epi = ebs.epilogue(relu=True, next_a_bits=nb, next_a_scale=float(step))
+        for variant in [-1] + U.variants_of("umma_pipe"):
+            if variant >= 0 and not U.applies(d, h, w, variant, n=n, epi=epi, want_packed=True):
+                continue
+            out = U.run_conv(qa, qw, d, epi, want_acc=True, next_bits=nb, variant=variant, px=px, pw=pw)
+            assert np.array_equal(out["acc"], ref)
+            assert np.array_equal(oracle.unpack_acts(out["packed"], co), q_ref), f"variant {variant}, {nb} bits"
+    assert fused_differs > 0, "the case no longer separates a fused multiply-add from two rounded operations"
