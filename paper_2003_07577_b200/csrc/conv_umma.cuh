@@ -60,7 +60,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
             : "=r"(done) : "r"(addr), "r"(parity) : "memory");
         if (done) return true;
         if (*abort_flag) return false;
-        __nanosleep(40);                  // leave the issue slots to the warps that have work
+        __nanosleep(it < 8 ? 40 : 200);   // leave the issue slots to the warps that have work
     }
     *abort_flag = 1;
     return false;

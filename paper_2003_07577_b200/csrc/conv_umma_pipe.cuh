@@ -486,8 +486,11 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
         // =========================== expanders ===========================
         int slot_q[PIPE_SLOTS], slot_pix[PIPE_SLOTS], slot_dst[PIPE_SLOTS];
 #pragma unroll
+        // An even number of words per pass: a thread takes two adjacent words of one pixel, so that for an odd plane count
+        // its 2 * AB packed words still start on an 8-byte boundary and load as pairs.  Otherwise items tid and tid + 256.
+        const bool paired = (AB & 1) != 0 && (KS & 1) == 0 && (p.CW & 1) == 0;
         for (int j = 0; j < PIPE_SLOTS; ++j) {
-            const int e = tid + j * PIPE_EXPANDERS;
+            const int e = paired ? 2 * tid + j : tid + j * PIPE_EXPANDERS;
             const int s = e / KS, q = e - s * KS;            // consecutive lanes: consecutive words of one pixel
             slot_q[j] = s < S ? q : -1;                       // -1: no item
             slot_pix[j] = s;
@@ -524,12 +527,20 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
             if (wg >= nwg) wg -= nwg;
             if (ld_wg == 0 && ld_sub == 0) chunk_offsets(ld_it, ld_ph);
 #pragma unroll
-            for (int j = 0; j < PIPE_SLOTS; ++j) {
+            for (int j = 0; j < PIPE_SLOTS; ++j)
 #pragma unroll
                 for (int k = 0; k < AB; ++k) a_set[set][j][k] = 0u;
-                const int cw = wg * KSS + ld_sub * KS + slot_q[j];
-                if (slot_q[j] >= 0 && ld_off[j] >= 0 && cw < p.CW)
-                    load_words_global<AB>(p.x + (ld_off[j] + cw * AB), a_set[set][j]);
+            if (paired) {                                       // both words of the pixel in one run of 2 * AB words
+                const int cw = wg * KSS + ld_sub * KS + slot_q[0];
+                if (slot_q[0] >= 0 && ld_off[0] >= 0 && cw < p.CW)
+                    load_words_global<2 * AB>(p.x + (ld_off[0] + cw * AB), *reinterpret_cast<uint32_t(*)[2 * AB]>(&a_set[set][0][0]));
+            } else {
+#pragma unroll
+                for (int j = 0; j < PIPE_SLOTS; ++j) {
+                    const int cw = wg * KSS + ld_sub * KS + slot_q[j];
+                    if (slot_q[j] >= 0 && ld_off[j] >= 0 && cw < p.CW)
+                        load_words_global<AB>(p.x + (ld_off[j] + cw * AB), a_set[set][j]);
+                }
             }
             if (++ld_sub == NSUB) {
                 ld_sub = 0;
