@@ -514,6 +514,29 @@ def measure_config(ebs, name, dev, timer, peaks, args, sm_max, detail: bool):
         out["per_layer"] = {m: [{k: pl[k] for k in ("name", "wb", "ab", "us", "frac_of_roof")} for pl in v]
                             for m, v in per_layer.items()}
 
+    # context (not the paper's method): the same layers with the activations as unpacked u8 codes, which skips the
+    # bit-plane expansion at 8 / Ab times the activation traffic; packed output only; layers it cannot run are skipped
+    ctx_ms, ctx_ref_ms, ctx_layers = 0.0, 0.0, 0
+    for i, L in enumerate(layers):
+        lay = L.spec.layer
+        if lay.c_in % 32 != 0:
+            continue
+        xb = torch.randint(0, 1 << L.spec.a_bits, (L.n, lay.h_in, lay.w_in, lay.c_in), dtype=torch.uint8, device=dev)
+        try:
+            gl = capture(lambda L=L, lay=lay, xb=xb: [ebs.ebs_conv2d_i8(xb, L.n, lay.h_in, lay.w_in, L.pw, L.d, L.epi, None, None, L.pn)
+                                                     for _ in range(10)])
+        except ebs.EbsError:
+            del xb
+            continue
+        ctx_ms += timer.graph_ms(gl, 2, cold=False) / 10.0
+        ctx_ref_ms += float(per_layer["fused"][i]["us"]) * 1e-3
+        ctx_layers += 1
+        del gl, xb
+    out["i8_context_path"] = {
+        "what": "ebs_conv2d_i8: activations as unpacked u8 NHWC codes instead of bit planes (context, not the paper's method)",
+        "layers": ctx_layers, "sum_layer_ms_warm": ctx_ms, "bit_plane_path_same_layers_ms": ctx_ref_ms,
+        "bit_plane_over_i8": (ctx_ref_ms / ctx_ms) if ctx_ms > 0 else None}
+
     # the same conv launches on the integer-pipe kernels only: the plane-pair double sum evaluated literally
     # (AND + POPC + shift-add per plane pair), held against the POPC pipe's peak
     lit_graph = capture(lambda: [L.run_conv(ebs, raw=True, variant=-2) for L in layers])

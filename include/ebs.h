@@ -216,6 +216,20 @@ int ebs_conv2d_mixed_variant(const void *packed_x_dev, int n, int h, int w, cons
                              float *y_out_dev, void *packed_next_dev, void *stream, int variant);
 
 /*
+ * Context kernel, NOT the paper's method: the same convolution with the activations given as unpacked 8-bit codes
+ * (u8, NHWC [n][h][w][c_in], c_in a multiple of 32) instead of bit planes.  The codes go straight into the int8
+ * tensor-core operand (no bit-plane expansion); weights, epilogue, outputs and results are those of
+ * ebs_conv2d_mixed (desc->a_bits only documents the code range; the result is exact for any u8 codes within the
+ * overflow bound of desc).  It exists to measure what keeping the activations as bit planes in memory costs or
+ * saves on this machine: a_bits/8 of the activation traffic against the expansion work (the paper motivates the
+ * decomposition by hardware that has only INT8/INT4/binary operations, Sec. 1).  Runs on the persistent pipeline
+ * kernels; EBS_ERR_UNSUPPORTED where they do not apply (c_in not a multiple of 32, stride above 2, w_levels = 1).
+ */
+int ebs_conv2d_i8(const void *x_codes_dev, int n, int h, int w, const void *packed_w_dev, const ebs_conv_desc *desc,
+                  const ebs_epilogue *epi, int32_t *acc_out_dev, float *y_out_dev, void *packed_next_dev,
+                  void *stream);
+
+/*
  * Which kernel family a variant number belongs to ("popc", "mma", "umma", "umma_strip", "umma_resident",
  * "mma_strip", "umma_pipe"; "" if out of range), and whether a variant can run a layer: the full validation and
  * kernel selection of ebs_conv2d_mixed_variant for a request with the given outputs (want_* are 0 / 1), without

@@ -184,9 +184,10 @@ struct ConvPlan {
     dim3 grid;
 };
 
+// byte_acts: packed_x holds the activations as unpacked u8 NHWC codes instead of bit planes (ebs_conv2d_i8).
 static int conv_plan(const void* packed_x, int n, int h, int w, const void* packed_w, const ebs_conv_desc* d,
                      const ebs_epilogue* epi, int32_t* acc_out, float* y_out, void* packed_next, int variant,
-                     ConvPlan* plan) {
+                     ConvPlan* plan, bool byte_acts = false) {
     int rc = validate_desc(d);
     if (rc) return rc;
     if (!packed_x || !packed_w || n <= 0 || h <= 0 || w <= 0) return EBS_ERR_INVALID_ARG;
@@ -245,6 +246,19 @@ static int conv_plan(const void* packed_x, int n, int h, int w, const void* pack
         if (packed_next) { p.next_bits = epi->next_a_bits; p.inv_next = 1.0f / epi->next_a_scale; }
     }
     const bool mma_ok = mma_path_supported(p, d);
+    if (byte_acts) {
+        // the context path exists in the persistent pipeline kernels only: whole 32-channel words of byte codes
+        if ((d->c_in & 31) != 0 || d->w_levels || !mma_ok) return EBS_ERR_UNSUPPORTED;
+        int pick = -1;
+        for (int v = 2; v >= 0 && pick < 0; --v)
+            if ((p.Co % (64 << v) == 0 || v == 0) && conv_umma_pipe_applies(p, v)) pick = v;
+        if (pick < 0) return EBS_ERR_UNSUPPORTED;
+        const ConvVariant* bv = conv_umma_pipe_variant(0, pick);
+        if (!bv) return EBS_ERR_UNSUPPORTED;
+        plan->v = bv;
+        plan->grid = dim3(1, 1, 1);
+        return EBS_OK;
+    }
     if (variant == -2) {
         variant = choose_variant(d->w_bits, d->a_bits, p.P, p.Co, packed_next != nullptr, sm_count());
     } else if (variant < 0) {
@@ -396,6 +410,15 @@ int ebs_conv2d_mixed(const void* packed_x_dev, int n, int h, int w, const void* 
                      void* packed_next_dev, void* stream) {
     return conv_impl(packed_x_dev, n, h, w, packed_w_dev, desc, epi, acc_out_dev, y_out_dev, packed_next_dev,
                      stream, -1);
+}
+
+int ebs_conv2d_i8(const void* x_codes_dev, int n, int h, int w, const void* packed_w_dev, const ebs_conv_desc* desc,
+                  const ebs_epilogue* epi, int32_t* acc_out_dev, float* y_out_dev, void* packed_next_dev, void* stream) {
+    ConvPlan plan;
+    const int rc = conv_plan(x_codes_dev, n, h, w, packed_w_dev, desc, epi, acc_out_dev, y_out_dev, packed_next_dev, -1,
+                             &plan, true);
+    if (rc) return rc;
+    return conv_launch(plan, stream);
 }
 
 int ebs_num_conv_variants(void) {

@@ -6,7 +6,7 @@ namespace ebs {
 #define EBS_DECLARE_PIPE(AB)                                         \
     const ConvVariant* conv_umma_pipe_variant_a##AB(int variant);    \
     unsigned long long conv_umma_pipe_timeouts_a##AB();
-EBS_DECLARE_PIPE(1) EBS_DECLARE_PIPE(2) EBS_DECLARE_PIPE(3) EBS_DECLARE_PIPE(4)
+EBS_DECLARE_PIPE(0) EBS_DECLARE_PIPE(1) EBS_DECLARE_PIPE(2) EBS_DECLARE_PIPE(3) EBS_DECLARE_PIPE(4)
 EBS_DECLARE_PIPE(5) EBS_DECLARE_PIPE(6) EBS_DECLARE_PIPE(7) EBS_DECLARE_PIPE(8)
 #undef EBS_DECLARE_PIPE
 
@@ -18,6 +18,7 @@ int pipe_sm_count() {
 
 const ConvVariant* conv_umma_pipe_variant(int a_bits, int variant) {
     switch (a_bits) {
+        case 0: return conv_umma_pipe_variant_a0(variant);      // activations as byte codes
         case 1: return conv_umma_pipe_variant_a1(variant);
         case 2: return conv_umma_pipe_variant_a2(variant);
         case 3: return conv_umma_pipe_variant_a3(variant);
@@ -42,7 +43,7 @@ long long conv_umma_pipe_items(const ConvParams& p, int variant) {
 }
 
 unsigned long long conv_umma_pipe_timeouts() {
-    return conv_umma_pipe_timeouts_a1() + conv_umma_pipe_timeouts_a2() + conv_umma_pipe_timeouts_a3() +
+    return conv_umma_pipe_timeouts_a0() + conv_umma_pipe_timeouts_a1() + conv_umma_pipe_timeouts_a2() + conv_umma_pipe_timeouts_a3() +
            conv_umma_pipe_timeouts_a4() + conv_umma_pipe_timeouts_a5() + conv_umma_pipe_timeouts_a6() +
            conv_umma_pipe_timeouts_a7() + conv_umma_pipe_timeouts_a8();
 }

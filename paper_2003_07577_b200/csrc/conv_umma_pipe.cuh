@@ -488,7 +488,8 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
 #pragma unroll
         // An even number of words per pass: a thread takes two adjacent words of one pixel, so that for an odd plane count
         // its 2 * AB packed words still start on an 8-byte boundary and load as pairs.  Otherwise items tid and tid + 256.
-        const bool paired = (AB & 1) != 0 && (KS & 1) == 0 && (p.CW & 1) == 0;
+        constexpr int NW = AB == 0 ? 8 : AB;                  // words of one (pixel, 32-channel word) item; AB = 0: byte codes
+        const bool paired = (NW & 1) != 0 && (KS & 1) == 0 && (p.CW & 1) == 0;
         for (int j = 0; j < PIPE_SLOTS; ++j) {
             const int e = paired ? 2 * tid + j : tid + j * PIPE_EXPANDERS;
             const int s = e / KS, q = e - s * KS;            // consecutive lanes: consecutive words of one pixel
@@ -513,14 +514,14 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                     const uint32_t hq = fastdiv(rem, g.div_row), wq = rem - hq * (uint32_t)g.Wq;
                     const int h = p.sh * ((int)hq + g.q0r) + pa, w = p.sw * ((int)wq + g.q0s) + pb;
                     if ((unsigned)h < (unsigned)p.H && (unsigned)w < (unsigned)p.W)
-                        ld_off[j] = (((int)n * p.H + h) * p.W + w) * p.CW * AB;
+                        ld_off[j] = (((int)n * p.H + h) * p.W + w) * p.CW * NW;
                 }
             }
         };
         // register ring of packed words: SETS - 1 chunks of global loads in flight per thread (about 48 registers whatever
         // the plane count: the latency of these loads, not their bandwidth, is what a deep reduction waits for)
-        constexpr int SETS = AB <= 2 ? 9 : (AB <= 4 ? 6 : (AB <= 6 ? 4 : 3));
-        uint32_t a_set[SETS][PIPE_SLOTS][AB];
+        constexpr int SETS = NW <= 4 ? 4 : 3;
+        uint32_t a_set[SETS][PIPE_SLOTS][NW];
         int ld_ph = 0, ld_wg = 0;
         auto load_next = [&](int set) {
             int wg = ld_wg + wg_rot;
@@ -529,17 +530,17 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
 #pragma unroll
             for (int j = 0; j < PIPE_SLOTS; ++j)
 #pragma unroll
-                for (int k = 0; k < AB; ++k) a_set[set][j][k] = 0u;
+                for (int k = 0; k < NW; ++k) a_set[set][j][k] = 0u;
             if (paired) {                                       // both words of the pixel in one run of 2 * AB words
                 const int cw = wg * KSS + ld_sub * KS + slot_q[0];
                 if (slot_q[0] >= 0 && ld_off[0] >= 0 && cw < p.CW)
-                    load_words_global<2 * AB>(p.x + (ld_off[0] + cw * AB), *reinterpret_cast<uint32_t(*)[2 * AB]>(&a_set[set][0][0]));
+                    load_words_global<2 * NW>(p.x + (ld_off[0] + cw * NW), *reinterpret_cast<uint32_t(*)[2 * NW]>(&a_set[set][0][0]));
             } else {
 #pragma unroll
                 for (int j = 0; j < PIPE_SLOTS; ++j) {
                     const int cw = wg * KSS + ld_sub * KS + slot_q[j];
                     if (slot_q[j] >= 0 && ld_off[j] >= 0 && cw < p.CW)
-                        load_words_global<AB>(p.x + (ld_off[j] + cw * AB), a_set[set][j]);
+                        load_words_global<NW>(p.x + (ld_off[j] + cw * NW), a_set[set][j]);
                 }
             }
             if (++ld_sub == NSUB) {
@@ -569,16 +570,29 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 for (int j = 0; j < PIPE_SLOTS; ++j) {
                     if (slot_q[j] < 0) continue;
                     // v_k = rotl(w_k, k); byte register bb = rotr(OR_k v_k & (0x01010101 << ((bb + k) & 7)), bb)
-                    uint32_t v[AB];
-#pragma unroll
-                    for (int k = 0; k < AB; ++k) v[k] = __funnelshift_l(a_set[u][j][k], a_set[u][j][k], k);
                     uint32_t r[8];
+                    if constexpr (AB == 0) {
+                        // byte codes, channel c in byte c of the item: only the order changes (row byte 4b + i = channel
+                        // 8i + b, the order of the weight image): register b takes byte b % 4 of words b / 4, 2 + b / 4, ...
+                        const uint32_t (&w)[8] = a_set[u][j];
 #pragma unroll
-                    for (int bb = 0; bb < 8; ++bb) {
-                        uint32_t t = v[0] & (0x01010101u << bb);
+                        for (int bb = 0; bb < 8; ++bb) {
+                            const uint32_t sel = 0x0040u + 0x11u * (uint32_t)(bb & 3);          // byte (bb & 3) of both operands
+                            const uint32_t lo = __byte_perm(w[bb >> 2], w[2 + (bb >> 2)], sel);
+                            const uint32_t hi = __byte_perm(w[4 + (bb >> 2)], w[6 + (bb >> 2)], sel);
+                            r[bb] = __byte_perm(lo, hi, 0x5410);
+                        }
+                    } else {
+                        uint32_t v[NW];
 #pragma unroll
-                        for (int k = 1; k < AB; ++k) t |= v[k] & (0x01010101u << ((bb + k) & 7));
-                        r[bb] = __funnelshift_r(t, t, bb);
+                        for (int k = 0; k < NW; ++k) v[k] = __funnelshift_l(a_set[u][j][k], a_set[u][j][k], k);
+#pragma unroll
+                        for (int bb = 0; bb < 8; ++bb) {
+                            uint32_t t = v[0] & (0x01010101u << bb);
+#pragma unroll
+                            for (int k = 1; k < NW; ++k) t |= v[k] & (0x01010101u << ((bb + k) & 7));
+                            r[bb] = __funnelshift_r(t, t, bb);
+                        }
                     }
                     uint8_t* dst = A_st + slot_dst[j];
                     *reinterpret_cast<uint4*>(dst) = make_uint4(r[0], r[1], r[2], r[3]);

@@ -134,3 +134,44 @@ def test_pipe_requantization_where_two_roundings_and_a_fused_one_differ(ebs, U, 
             assert np.array_equal(out["acc"], ref)
             assert np.array_equal(oracle.unpack_acts(out["packed"], co), q_ref), f"variant {variant}, {nb} bits"
     assert fused_differs > 0, "the case no longer separates a fused multiply-add from two rounded operations"
+
+
+@pytest.mark.parametrize("case", [
+    # n, c, co, k, stride, pad, h, w, code bits
+    (3, 64, 64, 3, 1, 1, 14, 13, 8), (2, 128, 256, 1, 1, 0, 12, 12, 5), (4, 64, 128, 3, 2, 1, 15, 14, 3),
+    (2, 512, 128, 1, 2, 0, 10, 10, 8), (2, 96, 70, 3, 1, 1, 9, 9, 4),
+])
+def test_context_path_on_unpacked_byte_codes(ebs, U, oracle, case):
+    """ebs_conv2d_i8 (activations as u8 NHWC codes, no bit planes): same accumulators, y and packed planes as the oracle."""
+    n, c, co, k, s, pad, h, w, ab = case
+    rng = np.random.default_rng(sum(case))
+    qa = U.rand_codes(rng, (n, c, h, w), ab, False)
+    qw = rng.integers(-3, 4, size=(co, c, k, k), dtype=np.int32)
+    d = U.desc_for(c, co, k, s, pad, 3, ab, 0.03, 0.07)
+    ref = oracle.conv2d_codes(qa, qw, (s, s), (pad, pad))
+    S = oracle.combined_scale(0.03, 0.07)
+    y0, _ = oracle.epilogue(ref, S, relu=True)
+    step = np.float32(max(float(np.percentile(y0, 99)), 1e-3) / 15)
+    y_ref, q_ref = oracle.epilogue(ref, S, relu=True, next_bits=4, inv_next=np.float32(1.0) / step)
+    x = torch.from_numpy(np.ascontiguousarray(qa.astype(np.uint8).transpose(0, 2, 3, 1))).to(U.dev())
+    pw = U.pack_weight_codes(qw, d)
+    ho, wo = ebs.ebs_conv_out_shape(d, h, w)
+    acc = torch.empty((n, ho, wo, co), dtype=torch.int32, device=U.dev())
+    y = torch.empty((n, ho, wo, co), dtype=torch.float32, device=U.dev())
+    pn = torch.empty(ebs.ebs_packed_act_bytes(n, ho, wo, co, 4) // 4, dtype=torch.int32, device=U.dev())
+    epi = ebs.epilogue(relu=True, next_a_bits=4, next_a_scale=float(step))
+    ebs.ebs_conv2d_i8(x, n, h, w, pw, d, epi, acc, y, pn)
+    torch.cuda.synchronize()
+    assert np.array_equal(acc.cpu().numpy().transpose(0, 3, 1, 2), ref)
+    assert np.array_equal(y.cpu().numpy().transpose(0, 3, 1, 2), y_ref)
+    assert np.array_equal(U.as_u32(pn).reshape(n, ho, wo, (co + 31) // 32, 4), oracle.pack_acts(q_ref, 4))
+
+
+def test_context_path_refuses_what_it_cannot_run(ebs, U):
+    d = U.desc_for(48, 64, 3, 1, 1, 3, 4)                          # c_in not a multiple of 32
+    x = torch.zeros((1, 8, 8, 48), dtype=torch.uint8, device=U.dev())
+    pw = torch.zeros(ebs.ebs_packed_weight_bytes(d) // 4, dtype=torch.int32, device=U.dev())
+    acc = torch.empty((1, 8, 8, 64), dtype=torch.int32, device=U.dev())
+    with pytest.raises(ebs.EbsError) as err:
+        ebs.ebs_conv2d_i8(x, 1, 8, 8, pw, d, None, acc)
+    assert err.value.status == ebs.EBS_ERR_UNSUPPORTED
