@@ -60,18 +60,30 @@ __global__ void __launch_bounds__(256) pack_acts_nhwc_u8_kernel(const uint8_t* _
     }
 }
 
-// Plane words of 32 codes held as eight words of four code bytes each.
+// Plane words of 32 codes held as eight words of four code bytes each (word k = channels 4k .. 4k+3).
+// The codes are first regrouped with byte permutes into registers c[bb] = channels {bb, 8 + bb, 16 + bb, 24 + bb}
+// (byte i = channel 8i + bb, the spacing the plane words have); with each register rotated left by bb, plane j is then
+// rotr(OR_bb c[bb] & (0x01010101 << ((bb + j) & 7)), j): one masked merge per register and plane instead of a
+// shift, mask, multiply, shift and merge per four codes.
 __device__ __forceinline__ void store_planes(const uint32_t (&codes)[8], int AB, uint32_t* __restrict__ dst) {
+    uint32_t c[8];
+#pragma unroll
+    for (int bb = 0; bb < 8; ++bb) {
+        const uint32_t sel = 0x0040u + 0x11u * (uint32_t)(bb & 3);                      // byte (bb & 3) of both operands
+        const uint32_t lo = __byte_perm(codes[bb >> 2], codes[2 + (bb >> 2)], sel);
+        const uint32_t hi = __byte_perm(codes[4 + (bb >> 2)], codes[6 + (bb >> 2)], sel);
+        const uint32_t g = __byte_perm(lo, hi, 0x5410);
+        c[bb] = __funnelshift_l(g, g, bb);
+    }
     uint32_t w[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         uint32_t word = 0u;
         if (j < AB) {
+            uint32_t t = c[0] & (0x01010101u << j);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const uint32_t t = (codes[k] >> j) & 0x01010101u;
-                word |= ((t * 0x01020408u) >> 24) << (4 * k);
-            }
+            for (int bb = 1; bb < 8; ++bb) t |= c[bb] & (0x01010101u << ((bb + j) & 7));
+            word = __funnelshift_r(t, t, j);
         }
         w[j] = word;
     }
@@ -242,6 +254,53 @@ __global__ void __launch_bounds__(128) pack_acts_nchw_kernel(const T* __restrict
     }
 }
 
+// NCHW fp32 with a pixel count that is a multiple of four: a CTA of 256 threads takes 32 channels x 256 pixels.  Every
+// thread issues its eight 16-byte loads (four pixels of one channel each, consecutive threads consecutive pixel quads, so
+// a warp reads 512 contiguous bytes of a channel row) before it uses any of them, quantizes, and writes the codes as
+// bytes into a pixel-major tile; one thread per pixel then builds the plane words.
+__global__ void __launch_bounds__(256) pack_acts_nchw_f32_vec_kernel(const float* __restrict__ x, int N, int C, int HW,
+                                                                     int CW, int AB, float inv_scale,
+                                                                     uint32_t* __restrict__ out) {
+    constexpr int PT = 256, ROWB = 36;                       // pixels per tile; bytes per pixel row (32 codes + pad)
+    __shared__ __align__(16) uint8_t tile[PT * ROWB];
+    const int ptiles = (HW + PT - 1) / PT;
+    const long long tiles = (long long)N * CW * ptiles;
+    const int qmax = (1 << AB) - 1;
+    const int quad = threadIdx.x & 63, crow = threadIdx.x >> 6;          // pixel quad 0..63, channel row 0..3 (+ 4 per step)
+    for (long long tix = blockIdx.x; tix < tiles; tix += gridDim.x) {
+        const int pt = (int)(tix % ptiles);
+        const long long rest = tix / ptiles;
+        const int cw = (int)(rest % CW), n = (int)(rest / CW);
+        const int p0 = pt * PT, pp4 = p0 + 4 * quad;
+        float4 v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int c = cw * 32 + crow + 4 * i;
+            v[i] = (c < C && pp4 < HW) ? __ldg(reinterpret_cast<const float4*>(x + ((long long)n * C + c) * HW + pp4))
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int cl = crow + 4 * i;
+            uint8_t* col = tile + (4 * quad) * ROWB + cl;
+            col[0] = (uint8_t)quantize_act_code(v[i].x, inv_scale, qmax);
+            col[ROWB] = (uint8_t)quantize_act_code(v[i].y, inv_scale, qmax);
+            col[2 * ROWB] = (uint8_t)quantize_act_code(v[i].z, inv_scale, qmax);
+            col[3 * ROWB] = (uint8_t)quantize_act_code(v[i].w, inv_scale, qmax);
+        }
+        __syncthreads();
+        const int pp = p0 + threadIdx.x;
+        if (pp < HW) {
+            const uint32_t* row = reinterpret_cast<const uint32_t*>(tile + threadIdx.x * ROWB);
+            uint32_t codes[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) codes[k] = row[k];
+            store_planes(codes, AB, out + (((long long)n * HW + pp) * CW + cw) * AB);
+        }
+        __syncthreads();
+    }
+}
+
 // Weights: one warp per (tap, channel word, output channel); tiny and off the inference path.
 template <typename T>
 __global__ void __launch_bounds__(256) pack_weights_kernel(const T* __restrict__ wt, int layout, int Co, int C,
@@ -323,7 +382,11 @@ int launch_pack_acts(const void* x, int dtype, int layout, int n, int c, int h, 
         const long long tiles = (long long)n * CW * ((h * w + 127) / 128);
         long long grid = tiles < (long long)sms * 16 ? tiles : (long long)sms * 16;
         if (grid < 1) grid = 1;
-        if (dtype == EBS_F32)
+        if (dtype == EBS_F32 && (h * w) % 4 == 0) {
+            const long long vtiles = (long long)n * CW * ((h * w + 255) / 256);
+            long long vgrid = vtiles < (long long)sms * 16 ? vtiles : (long long)sms * 16;
+            pack_acts_nchw_f32_vec_kernel<<<(int)vgrid, 256, 0, st>>>((const float*)x, n, c, h * w, CW, a_bits, inv_scale, out);
+        } else if (dtype == EBS_F32)
             pack_acts_nchw_kernel<float><<<(int)grid, 128, 0, st>>>((const float*)x, n, c, h * w, CW, a_bits, inv_scale, out);
         else
             pack_acts_nchw_kernel<uint8_t><<<(int)grid, 128, 0, st>>>((const uint8_t*)x, n, c, h * w, CW, a_bits, inv_scale, out);
