@@ -196,6 +196,30 @@ def global_avgpool(y) -> np.ndarray:
     return (acc * (np.float32(1.0) / np.float32(h * w))).astype(np.float32)
 
 
+def maxpool_codes(q, k: int, stride: int, pad: int) -> np.ndarray:
+    """Max pooling of unsigned activation codes [N, C, H, W] (the 3x3 stride-2 pooling between the first convolution and
+    the first block of the ImageNet ResNets the paper evaluates, Sec. 5).  Codes of one tensor share one step, so the
+    maximum of the real values is the maximum of the codes; window positions outside the image are ignored, which for
+    codes (all >= 0, the image of a clipped activation) is the same as padding with the zero code.  Plain loops over the
+    window; output size floor((size + 2 pad - k) / stride) + 1."""
+    q = np.asarray(q)
+    n, c, h, w = q.shape
+    ho, wo = out_dim(h, pad, k, stride), out_dim(w, pad, k, stride)
+    out = np.zeros((n, c, ho, wo), dtype=q.dtype)
+    for i in range(ho):
+        for j in range(wo):
+            best = None
+            for r in range(k):
+                for s in range(k):
+                    hi, wi = i * stride + r - pad, j * stride + s - pad
+                    if 0 <= hi < h and 0 <= wi < w:
+                        v = q[:, :, hi, wi]
+                        best = v.copy() if best is None else np.maximum(best, v)
+            if best is not None:
+                out[:, :, i, j] = best
+    return out
+
+
 # ---------------------------------------------------------------- search stage (Sec. 4.1), plain numpy
 
 def softmax_strengths(r) -> np.ndarray:

@@ -466,3 +466,28 @@ def test_expected_flops_eq11(oracle):
     assert abs(oracle.expected_flops(1e6, bits, uniform, bits, uniform) - 9e6) < 1.0   # mean bitwidth 3 on both sides
     onehot = [0, 0, 1, 0, 0]
     assert oracle.expected_flops(40.81e6, bits, onehot, bits, [0, 1, 0, 0, 0]) == 40.81e6 * 3 * 2
+
+
+def test_maxpool_codes_pins(oracle):
+    """Max pooling of codes: brute force per output on a tiny tensor, the identity window, a hand-written case with
+    padding, and the library routine torch.nn.functional.max_pool2d (which pads with -inf: the same thing for codes)."""
+    import torch
+    rng = np.random.default_rng(5)
+    q = rng.integers(0, 16, size=(2, 3, 7, 6), dtype=np.int32)
+    for k, s, p in ((3, 2, 1), (2, 2, 0), (3, 1, 1), (1, 1, 0), (3, 2, 0)):
+        got = oracle.maxpool_codes(q, k, s, p)
+        ho, wo = (7 + 2 * p - k) // s + 1, (6 + 2 * p - k) // s + 1
+        assert got.shape == (2, 3, ho, wo)
+        for n in range(2):
+            for c in range(3):
+                for i in range(ho):
+                    for j in range(wo):
+                        vals = [q[n, c, i * s + r - p, j * s + t - p] for r in range(k) for t in range(k)
+                                if 0 <= i * s + r - p < 7 and 0 <= j * s + t - p < 6]
+                        assert got[n, c, i, j] == max(vals)
+        ref = torch.nn.functional.max_pool2d(torch.from_numpy(q.astype(np.float64)), k, s, p).numpy()
+        assert np.array_equal(got, ref.astype(np.int32))
+    assert np.array_equal(oracle.maxpool_codes(q, 1, 1, 0), q)
+    one = np.array([[[[1, 5], [7, 2]]]], np.int32)
+    assert np.array_equal(oracle.maxpool_codes(one, 3, 2, 1), np.array([[[[7]]]], np.int32))      # one window sees all
+    assert np.array_equal(oracle.maxpool_codes(one, 2, 1, 1), np.array([[[[1, 5, 5], [7, 7, 5], [7, 7, 2]]]], np.int32))
