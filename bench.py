@@ -664,6 +664,48 @@ def network_leg(ebs, dev, stream, flush, reps):
             "finite_logits": bool(torch.isfinite(out["logits"]).all().item())}
 
 
+def resnet18_leg(ebs, dev, stream, flush, reps, batch=64):
+    """ImageNet ResNet-18 forward passes per second (224x224 images) through paper_2003_07577_b200.network: 7x7 first
+    convolution at 8 bits, max pooling on packed codes, basic blocks with fused shortcuts, average pooling, classifier."""
+    from paper_2003_07577_b200.network import BasicBlockNet, calibrated_plans
+    from types import SimpleNamespace
+    specs = gen.resnet18_network(0, batch)
+    imgs_host = torch.from_numpy(np.ascontiguousarray(gen.images_u8(0, batch, 224, 224).astype(np.uint8).transpose(0, 2, 3, 1))).pin_memory()
+    imgs = imgs_host.to(dev)
+    recs = [SimpleNamespace(name=s.layer.name, role=s.layer.role, c_in=s.layer.c_in, c_out=s.layer.c_out, k=s.layer.k,
+                            stride=s.layer.stride, pad=s.layer.pad, h_in=s.layer.h_in, w_in=s.layer.w_in,
+                            w_bits=s.w_bits, a_bits=s.a_bits, w_scale=s.w_scale) for s in specs]
+    wts = {s.layer.name: torch.from_numpy(gen.weight_codes(s).astype(np.int8)).to(dev) for s in specs}
+    pool = (3, 2, 1)
+    net = BasicBlockNet(calibrated_plans(recs, wts, imgs, dev, pool=pool), dev, pool=pool)
+    out = {}
+    g = capture(lambda: out.__setitem__("logits", net.forward(imgs)))
+    ms = []
+    for _ in range(reps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        g.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    logits_host = torch.empty((batch, specs[-1].layer.c_out), dtype=torch.float32).pin_memory()
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        imgs.copy_(imgs_host, non_blocking=True)
+        g.replay()
+        logits_host.copy_(out["logits"], non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / reps
+    t = float(np.mean(ms)) * 1e-3
+    ops = sum(gen.binary_ops(s) for s in specs)
+    return {"model": "ResNet-18 (ImageNet, 224x224): 7x7 first convolution at W8A8, 3x3/2 max pooling on packed codes, basic "
+                     "blocks with fused shortcuts, average pool, classifier", "batch": batch, "ms_per_batch": t * 1e3,
+            "imgs_per_s": batch / t, "effective_tops": ops / t / 1e12, "launches_per_batch": net.launches_per_forward,
+            "l2": "cold (flushed before every replay)", "e2e_imgs_per_s": batch / e2e_s,
+            "finite_logits": bool(torch.isfinite(out["logits"]).all().item())}
+
+
 def run_gpu(args):
     from paper_2003_07577_b200 import binding as ebs
     ebs.lib()
@@ -795,6 +837,8 @@ def run_gpu(args):
         achieved, roof_peak, roof_unit = m["algorithmic_bytes"] / (conv_ms * 1e-3) / 1e9, hbm_gbs, "GB/s"
     streaming = streaming_leg(ebs, dev, stream, hbm_gbs) if world == 1 and not args.quick else {}
     network = network_leg(ebs, dev, stream, flush, max(5, min(args.steps, 30))) if world == 1 and not args.quick else {}
+    if network:
+        network["resnet18_imagenet"] = resnet18_leg(ebs, dev, stream, flush, max(3, min(args.steps, 10)))
     cpu = cpu_baseline_sample(headline, 15.0) if world == 1 and not args.no_cpu_baseline else None
     res_head = dict(res)
     per_config[headline] = res_head

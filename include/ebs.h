@@ -367,6 +367,18 @@ int ebs_resnet_cifar_forward(const unsigned char *images_dev, int n, int img_h, 
 int ebs_global_avgpool(const float *y_dev, int n, int hw, int c, float *out_dev, void *stream);
 
 /*
+ * Max pooling of packed activation planes (the 3x3 stride-2 pooling after the first convolution of the ImageNet
+ * ResNets of Sec. 5; not part of the binary decomposition itself).  All codes of a tensor share one step, so the
+ * maximum of the values is the maximum of the codes; it is taken in the bit-plane domain, 32 channels at a time.
+ * Window positions outside the image are ignored (equivalent to padding with the zero code).
+ *   packed_x_dev    u32 [n][h][w][ceil(c/32)][a_bits]
+ *   packed_out_dev  u32 [n][ho][wo][ceil(c/32)][a_bits], ho = floor((h + 2 pad - k) / stride) + 1 (likewise wo);
+ *                   must not alias the input.  pad < k.
+ */
+int ebs_maxpool_packed(const void *packed_x_dev, int n, int h, int w, int c, int a_bits, int k, int stride, int pad,
+                       void *packed_out_dev, void *stream);
+
+/*
  * One layer from HOST buffers, for callers whose data lives on the host: copies the activations
  * to the device, packs them, runs ebs_conv2d_mixed and copies the requested outputs back, all
  * enqueued on `stream` (host buffers should be pinned for the copies to be asynchronous; the

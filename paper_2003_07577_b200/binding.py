@@ -28,7 +28,7 @@ EXPORTS = [
     "ebs_probe_pipe", "ebs_device_wait_timeouts", "ebs_global_avgpool", "ebs_packed_weight_plane_bytes", "ebs_search_weight_forward",
     "ebs_search_act_forward", "ebs_expected_flops", "ebs_fused_plan_upload", "ebs_resnet_cifar_forward", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
     "ebs_conv_variant_family", "ebs_conv_variant_applies", "ebs_check_device_status", "ebs_test_set_device_wait",
-    "ebs_conv2d_i8",
+    "ebs_conv2d_i8", "ebs_maxpool_packed",
 ]
 
 
@@ -100,6 +100,7 @@ def lib() -> ctypes.CDLL:
         L.ebs_device_wait_timeouts.restype = ctypes.c_longlong
         L.ebs_conv2d_mixed_host_noalloc.argtypes = [p, i, i, i, i, i, p, D, E, p, p, p, p]
         L.ebs_conv2d_i8.argtypes = [p, i, i, i, p, D, E, p, p, p, p]
+        L.ebs_maxpool_packed.argtypes = [p, i, i, i, i, i, i, i, i, p, p]
         L.ebs_conv_variant_family.argtypes = [i]
         L.ebs_conv_variant_family.restype = ctypes.c_char_p
         L.ebs_conv_variant_applies.argtypes = [D, i, i, i, E, i, i, i, i]
@@ -320,3 +321,8 @@ def ebs_conv2d_i8(x_codes_dev, n, h, w, packed_w_dev, desc, epi=None, acc_out_de
     e = None if epi is None else ctypes.byref(epi)
     _check(lib().ebs_conv2d_i8(_ptr(x_codes_dev), n, h, w, _ptr(packed_w_dev), ctypes.byref(desc), e, _ptr(acc_out_dev),
                                _ptr(y_out_dev), _ptr(packed_next_dev), _stream(stream)), "ebs_conv2d_i8")
+
+
+def ebs_maxpool_packed(packed_x_dev, n, h, w, c, a_bits, k, stride, pad, packed_out_dev, stream=None) -> None:
+    _check(lib().ebs_maxpool_packed(_ptr(packed_x_dev), n, h, w, c, a_bits, k, stride, pad, _ptr(packed_out_dev),
+                                    _stream(stream)), "ebs_maxpool_packed")

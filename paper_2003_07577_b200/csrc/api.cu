@@ -531,6 +531,18 @@ int ebs_global_avgpool(const float* y_dev, int n, int hw, int c, float* out_dev,
     return launch_avgpool(y_dev, n, hw, c, out_dev, static_cast<cudaStream_t>(stream));
 }
 
+int ebs_maxpool_packed(const void* packed_x_dev, int n, int h, int w, int c, int a_bits, int k, int stride, int pad,
+                       void* packed_out_dev, void* stream) {
+    if (!packed_x_dev || !packed_out_dev || n <= 0 || h <= 0 || w <= 0 || c <= 0) return EBS_ERR_INVALID_ARG;
+    if (a_bits < 1 || a_bits > 8 || k < 1 || stride < 1 || pad < 0 || pad >= k) return EBS_ERR_INVALID_ARG;
+    if (!aligned16(packed_x_dev) || !aligned16(packed_out_dev) || packed_x_dev == packed_out_dev) return EBS_ERR_INVALID_ARG;
+    const int ho = out_dim(h, pad, k, stride), wo = out_dim(w, pad, k, stride);
+    if (ho <= 0 || wo <= 0) return EBS_ERR_INVALID_ARG;
+    if ((long long)n * h * w * ((c + 31) / 32) * a_bits >= (1LL << 31)) return EBS_ERR_OVERFLOW;
+    return launch_maxpool_packed(static_cast<const uint32_t*>(packed_x_dev), n, h, w, c, a_bits, k, stride, pad, ho, wo,
+                                 static_cast<uint32_t*>(packed_out_dev), static_cast<cudaStream_t>(stream));
+}
+
 static size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 size_t ebs_host_workspace_bytes(const ebs_conv_desc* d, int n, int h, int w, int dtype, int next_a_bits) {

@@ -116,6 +116,8 @@ int launch_fused_resnet(const uint8_t* images, int n, int img_h, int img_w, cons
                         const void* head_host, float* logits, uint8_t* trace, long long trace_stride, cudaStream_t st);
 unsigned long long fused_net_timeouts();
 int launch_avgpool(const float* y, int n, int hw, int c, float* out, cudaStream_t st);
+int launch_maxpool_packed(const uint32_t* x, int n, int h, int w, int c, int bits, int k, int stride, int pad, int ho,
+                          int wo, uint32_t* out, cudaStream_t st);
 
 // Records a CUDA error for ebs_last_cuda_error() and returns EBS_ERR_CUDA (or EBS_OK).
 int check_cuda(cudaError_t e);

@@ -1,4 +1,5 @@
-"""Chains the C-ABI entry points over a basic-block residual network (the CIFAR ResNets of Sec. 5).
+"""Chains the C-ABI entry points over a basic-block residual network (the CIFAR ResNets and the ImageNet ResNet-18 of
+Sec. 5; the ImageNet form has a max pooling between the first convolution and the first block).
 
 Plumbing only: this module owns device buffers and the order of the calls.  Every arithmetic step
 (quantize + pack, the plane-pair convolution, scale / bias / shortcut / ReLU / requantize, average
@@ -6,7 +7,7 @@ pooling) runs inside the library's kernels.
 
 Data flow for one batch of 8-bit images (NHWC):
 
-    pack(8 bit) -> conv1 -> x                                 x: packed planes of the block input
+    pack(8 bit) -> conv1 [-> max pool] -> x                   x: packed planes of the block input
     per block:   c1(x) -> t ; c2(t) + shortcut -> x'          t, x': packed planes
        identity shortcut:  the packed codes of x, times their step, added inside c2's epilogue
        projection shortcut: ds(x) as fp32, added inside c2's epilogue
@@ -41,8 +42,10 @@ class ConvPlan:
 class BasicBlockNet:
     """conv1, basic blocks named ``<block>c1`` / ``<block>c2`` (/ ``<block>ds``), average pool, classifier."""
 
-    def __init__(self, plans: List[ConvPlan], device=None):
+    def __init__(self, plans: List[ConvPlan], device=None, pool=None):
+        """pool: None, or (k, stride, pad) of the max pooling after the first convolution (ImageNet ResNets: (3, 2, 1))."""
         self.plans = plans
+        self.pool = pool
         self.device = torch.device("cuda:0") if device is None else device
         self.first = plans[0]
         self.fc = plans[-1]
@@ -85,8 +88,14 @@ class BasicBlockNet:
         px = self._planes(("input", "q"), n, f.h_in, f.w_in, f.desc.c_in, 8)
         ebs.ebs_pack_acts(images_u8_nhwc, ebs.EBS_U8_CODES, ebs.EBS_NHWC, n, f.desc.c_in, f.h_in, f.w_in, 8, 1.0, px,
                           stream=stream)
-        _, x, _, _ = self._conv(f, px, n, stream=stream)
+        _, x, ho1, wo1 = self._conv(f, px, n, stream=stream)
         x_bits, x_step = f.out_bits, f.out_step
+        if self.pool is not None:                                # on the packed codes; bits and step are unchanged
+            k, s, pd = self.pool
+            hp, wp = (ho1 + 2 * pd - k) // s + 1, (wo1 + 2 * pd - k) // s + 1
+            xp = self._planes(("maxpool", "q"), n, hp, wp, f.desc.c_out, x_bits)
+            ebs.ebs_maxpool_packed(x, n, ho1, wo1, f.desc.c_out, x_bits, k, s, pd, xp, stream=stream)
+            x = xp
         y_last, ho, wo = None, 0, 0
         for bi, (c1, c2, ds) in enumerate(self.blocks):
             last = bi == len(self.blocks) - 1
@@ -110,10 +119,10 @@ class BasicBlockNet:
 
     @property
     def launches_per_forward(self) -> int:
-        return 2 + len(self.plans) + 1
+        return 2 + len(self.plans) + 1 + (1 if self.pool is not None else 0)
 
 
-def calibrated_plans(layers, weight_codes, images_u8_nhwc: torch.Tensor, device=None) -> List[ConvPlan]:
+def calibrated_plans(layers, weight_codes, images_u8_nhwc: torch.Tensor, device=None, pool=None) -> List[ConvPlan]:
     """Builds the per-layer plans of a basic-block network from integer weight codes.
 
     ``layers``: records with name, role, c_in, c_out, k, stride, pad, h_in, w_in, w_bits, a_bits,
@@ -161,7 +170,13 @@ def calibrated_plans(layers, weight_codes, images_u8_nhwc: torch.Tensor, device=
                      device=device)
     ebs.ebs_pack_acts(images_u8_nhwc, ebs.EBS_U8_CODES, ebs.EBS_NHWC, n, first.c_in, first.h_in, first.w_in, 8, 1.0, px)
     x_bits = by_name[tags[0] + "c1"].a_bits
-    _, x, x_step, _ = run(first, px, 1.0 / 255.0, x_bits)
+    _, x, x_step, hw1 = run(first, px, 1.0 / 255.0, x_bits)
+    if pool is not None:
+        k, s, pd = pool
+        hp, wp = (hw1[0] + 2 * pd - k) // s + 1, (hw1[1] + 2 * pd - k) // s + 1
+        xp = torch.empty(ebs.ebs_packed_act_bytes(n, hp, wp, first.c_out, x_bits) // 4, dtype=torch.int32, device=device)
+        ebs.ebs_maxpool_packed(x, n, hw1[0], hw1[1], first.c_out, x_bits, k, s, pd, xp)
+        x = xp
     y_last, hw = None, (0, 0)
     for bi, tag in enumerate(tags):
         c1, c2, ds = by_name[tag + "c1"], by_name[tag + "c2"], by_name.get(tag + "ds")

@@ -88,7 +88,7 @@ def test_global_avgpool(ebs, U, oracle, n, hw, c):
     assert np.array_equal(out.cpu().numpy(), oracle.global_avgpool(y))
 
 
-def _oracle_network(oracle, gen, specs, imgs, sample):
+def _oracle_network(oracle, gen, specs, imgs, sample, pool=None):
     """The ResNet-20 forward pass in oracle calls on the sampled images.  Also fixes, per layer, the
     folded-BatchNorm shift and the step of the next quantizer (a calibration: any positive values
     would serve the comparison, these keep the codes spread over their range)."""
@@ -120,6 +120,9 @@ def _oracle_network(oracle, gen, specs, imgs, sample):
     first = by_name["conv1"]
     nb = by_name[blocks[0] + "c1"].a_bits
     _, qx, sx = conv(first, x, a0, nb=nb)
+    if pool is not None:
+        qx = oracle.maxpool_codes(qx, *pool)
+        trace["maxpool"] = qx
     y_last = None
     for bi, tag in enumerate(blocks):
         c1, c2, ds = by_name[tag + "c1"], by_name[tag + "c2"], by_name.get(tag + "ds")
@@ -138,7 +141,7 @@ def _oracle_network(oracle, gen, specs, imgs, sample):
     return plan, trace, logits.reshape(len(sample), -1), qp
 
 
-def _gpu_network(ebs, U, gen, specs, plan):
+def _gpu_network(ebs, U, gen, specs, plan, pool=None):
     from paper_2003_07577_b200.network import BasicBlockNet, ConvPlan
     plans = []
     for spec in specs:
@@ -147,7 +150,7 @@ def _gpu_network(ebs, U, gen, specs, plan):
                           spec.w_scale, pl["a_scale"])
         plans.append(ConvPlan(L.name, L.role, d, L.h_in, L.w_in, U.pack_weight_codes(gen.weight_codes(spec), d),
                               ch_bias=_to(pl["bias"], U), ch_scale=_to(pl["scale"], U), out_bits=pl["out_bits"], out_step=pl["out_step"]))
-    return BasicBlockNet(plans, U.dev())
+    return BasicBlockNet(plans, U.dev(), pool=pool)
 
 
 def test_resnet20_forward_matches_the_oracle(ebs, U, oracle, gen):
@@ -222,3 +225,54 @@ def test_fused_network_plan_is_validated(ebs, U):
         setattr(bad, field, value)
         with pytest.raises(RuntimeError):
             ebs.ebs_fused_plan_upload([bad], dev)
+
+
+@pytest.mark.parametrize("bits,c,h,w,k,s,p", [(4, 64, 15, 14, 3, 2, 1), (1, 32, 8, 8, 2, 2, 0), (8, 70, 9, 11, 3, 1, 1),
+                                              (3, 96, 7, 7, 3, 2, 0), (5, 33, 6, 5, 1, 1, 0), (7, 64, 12, 12, 3, 2, 1)])
+def test_maxpool_on_packed_planes(ebs, U, oracle, bits, c, h, w, k, s, p):
+    """Bit-plane-domain max pooling equals the oracle's maximum of codes, word for word (pad bits stay zero)."""
+    rng = np.random.default_rng(bits * 100 + c + h)
+    n = 3
+    q = U.rand_codes(rng, (n, c, h, w), bits, False)
+    ref = oracle.maxpool_codes(q, k, s, p)
+    px = U.pack_acts_codes(q, bits)
+    ho, wo = ref.shape[2], ref.shape[3]
+    out = torch.full((ebs.ebs_packed_act_bytes(n, ho, wo, c, bits) // 4,), -1, dtype=torch.int32, device=U.dev())
+    ebs.ebs_maxpool_packed(px, n, h, w, c, bits, k, s, p, out)
+    torch.cuda.synchronize()
+    assert np.array_equal(U.as_u32(out).reshape(n, ho, wo, (c + 31) // 32, bits), oracle.pack_acts(ref, bits))
+    with pytest.raises(ebs.EbsError):
+        ebs.ebs_maxpool_packed(px, n, h, w, c, bits, 3, 2, 3, out)          # padding as large as the window
+
+
+def test_resnet18_imagenet_forward_matches_the_oracle(ebs, U, oracle, gen):
+    """The ImageNet ResNet-18 (7x7 stride-2 first convolution at 8 bits, 3x3 stride-2 max pooling, eight basic blocks with
+    projection shortcuts, average pooling, classifier) on 224x224 images at batch 4: every layer's packed output, the
+    pooled codes and the logits of the sampled images equal the oracle chain bit for bit."""
+    n, sample, pool = 4, [0, 3], (3, 2, 1)
+    specs = gen.resnet18_network(0, n)
+    assert specs[0].layer.role == "first" and specs[0].layer.k == 7 and specs[-1].layer.role == "fc"
+    imgs = gen.images_u8(0, n, 224, 224)
+    plan, trace, logits_ref, qp_ref = _oracle_network(oracle, gen, specs, imgs, sample, pool=pool)
+    net = _gpu_network(ebs, U, gen, specs, plan, pool=pool)
+    x = _to(imgs.astype(np.uint8).transpose(0, 2, 3, 1), U)
+    logits = net.forward(x)
+    torch.cuda.synchronize()
+    first = specs[0].layer
+    got = oracle.unpack_acts(U.packed_images(net._buf[("maxpool", "q")], n, 56, 56, first.c_out, plan["conv1"]["out_bits"],
+                                             sample), first.c_out)
+    assert np.array_equal(got, trace["maxpool"]), "max pooling"
+    for spec in specs:
+        L, q_ref = spec.layer, trace[spec.layer.name]
+        if q_ref is None:
+            continue
+        bits = plan[L.name]["out_bits"]
+        got = oracle.unpack_acts(U.packed_images(net._buf[(L.name, "q")], n, L.h_out, L.w_out, L.c_out, bits, sample),
+                                 L.c_out)
+        assert np.array_equal(got, q_ref), f"{L.name} W{spec.w_bits}A{spec.a_bits}"
+        assert 0 < q_ref.mean() < (1 << bits) - 1
+    got_p = oracle.unpack_acts(U.packed_images(net._buf[("pool", "q")], n, 1, 1, 512, 8, sample), 512)
+    assert np.array_equal(got_p, qp_ref)
+    assert np.array_equal(logits[sample].cpu().numpy(), logits_ref)
+    assert np.isfinite(logits_ref).all() and logits_ref.shape == (2, 1000)
+    assert ebs.ebs_device_wait_timeouts() == 0

@@ -152,6 +152,13 @@ def resnet20_network(seed: int = 0, batch: int = 128) -> List[LayerSpec]:
     return _share_shortcut_inputs(config2(seed, batch))
 
 
+def resnet18_network(seed: int = 0, batch: int = 32) -> List[LayerSpec]:
+    """The ImageNet ResNet-18 of config3 wired as a network (first convolution and classifier at 8 bits, a projection
+    shortcut reads the same tensor as its block's first convolution); 224x224 images, a 3x3 stride-2 max pooling follows
+    the first convolution."""
+    return _share_shortcut_inputs(_draw(seed, resnet18_imagenet(), [2, 3, 4, 5, 6], batch, "gaussian"))
+
+
 def _share_shortcut_inputs(specs: List[LayerSpec]) -> List[LayerSpec]:
     by_name = {s.layer.name: s for s in specs}
     out = []
