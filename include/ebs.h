@@ -304,6 +304,14 @@ double ebs_expected_flops(double macs, const int *bits_w, const float *coeff_w, 
                           const float *coeff_x, int n_x);
 
 /*
+ * The two host-side fp32 roundings of the scale handling, exactly as the entry points above apply them:
+ * S = fl32(w_scale * a_scale) (scale merge of Sec. 4.3) and fl32(1 / step) (the quantizer multiplies by the
+ * reciprocal of its step, Eq. 1b-1c).  For callers that fill ebs_fused_layer / ebs_fused_head records.
+ */
+float ebs_combined_scale(float w_scale, float a_scale);
+float ebs_reciprocal_step(float step);
+
+/*
  * Whole-network inference of a basic-block CIFAR ResNet (Sec. 5, Table 1) in ONE launch: a thread
  * block carries one image through every layer with its activation codes resident in shared memory
  * as bytes (no bit planes, no global traffic and no launch between layers); the arithmetic of every

@@ -252,23 +252,26 @@ def search_act_forward(x, alpha, bits, coeff) -> np.ndarray:
     return (a * acc).astype(np.float32)
 
 
-def search_weight_forward(w, bits, coeff):
+def search_weight_forward(w, bits, coeff, per_candidate: bool = False):
     """Eq. 1a per candidate bitwidth, blended as in Eq. 6, in float64:
     u = tanh(w) / (2 max|tanh(w)|) + 1/2;  w_hat = sum_i coeff_i * (2 quantize_{b_i}(u) - 1).
     Also returns, per element, the smallest distance of (2^b - 1) u + 0.5 to an integer over the
-    candidates: where it is tiny, a float32 evaluation may legitimately round to the other level."""
+    candidates: where it is tiny, a float32 evaluation may legitimately round to the other level.
+    per_candidate = True returns the distances of every candidate instead ([len(bits), ...])."""
     w = np.asarray(w, dtype=np.float64)
     t = np.tanh(w)
     u = t / (2.0 * np.abs(t).max()) + 0.5
     out = np.zeros_like(u)
     margin = np.full(u.shape, 1.0)
+    each = []
     for b, c in zip(bits, coeff):
         L = float((1 << int(b)) - 1)
         v = L * u + 0.5
         code = np.clip(np.floor(v), 0.0, L)
-        margin = np.minimum(margin, np.abs(v - np.round(v)))
+        each.append(np.abs(v - np.round(v)))
+        margin = np.minimum(margin, each[-1])
         out += float(c) * (2.0 * code / L - 1.0)
-    return out, margin
+    return out, (np.stack(each) if per_candidate else margin)
 
 
 def expected_flops(macs, bits_w, coeff_w, bits_x, coeff_x) -> float:

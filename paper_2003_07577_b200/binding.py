@@ -28,7 +28,7 @@ EXPORTS = [
     "ebs_probe_pipe", "ebs_device_wait_timeouts", "ebs_global_avgpool", "ebs_packed_weight_plane_bytes", "ebs_search_weight_forward",
     "ebs_search_act_forward", "ebs_expected_flops", "ebs_fused_plan_upload", "ebs_resnet_cifar_forward", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
     "ebs_conv_variant_family", "ebs_conv_variant_applies", "ebs_check_device_status", "ebs_test_set_device_wait",
-    "ebs_conv2d_i8", "ebs_maxpool_packed",
+    "ebs_conv2d_i8", "ebs_maxpool_packed", "ebs_combined_scale", "ebs_reciprocal_step",
 ]
 
 
@@ -101,6 +101,10 @@ def lib() -> ctypes.CDLL:
         L.ebs_conv2d_mixed_host_noalloc.argtypes = [p, i, i, i, i, i, p, D, E, p, p, p, p]
         L.ebs_conv2d_i8.argtypes = [p, i, i, i, p, D, E, p, p, p, p]
         L.ebs_maxpool_packed.argtypes = [p, i, i, i, i, i, i, i, i, p, p]
+        L.ebs_combined_scale.argtypes = [f, f]
+        L.ebs_combined_scale.restype = f
+        L.ebs_reciprocal_step.argtypes = [f]
+        L.ebs_reciprocal_step.restype = f
         L.ebs_conv_variant_family.argtypes = [i]
         L.ebs_conv_variant_family.restype = ctypes.c_char_p
         L.ebs_conv_variant_applies.argtypes = [D, i, i, i, E, i, i, i, i]
@@ -326,3 +330,11 @@ def ebs_conv2d_i8(x_codes_dev, n, h, w, packed_w_dev, desc, epi=None, acc_out_de
 def ebs_maxpool_packed(packed_x_dev, n, h, w, c, a_bits, k, stride, pad, packed_out_dev, stream=None) -> None:
     _check(lib().ebs_maxpool_packed(_ptr(packed_x_dev), n, h, w, c, a_bits, k, stride, pad, _ptr(packed_out_dev),
                                     _stream(stream)), "ebs_maxpool_packed")
+
+
+def ebs_combined_scale(w_scale: float, a_scale: float) -> float:
+    return float(lib().ebs_combined_scale(w_scale, a_scale))
+
+
+def ebs_reciprocal_step(step: float) -> float:
+    return float(lib().ebs_reciprocal_step(step))

@@ -500,6 +500,9 @@ int ebs_search_act_forward(const float* x_dev, size_t n, float alpha, const int*
     return launch_search_acts(x_dev, n, alpha, bits, coeff, n_cand, x_hat_dev, static_cast<cudaStream_t>(stream));
 }
 
+float ebs_combined_scale(float w_scale, float a_scale) { return w_scale * a_scale; }        // one rounded fp32 multiply
+float ebs_reciprocal_step(float step) { return 1.0f / step; }                               // one rounded fp32 division
+
 double ebs_expected_flops(double macs, const int* bits_w, const float* coeff_w, int n_w, const int* bits_x,
                           const float* coeff_x, int n_x) {
     if (!bits_w || !coeff_w || !bits_x || !coeff_x || n_w < 1 || n_x < 1 || !(macs >= 0.0)) return -1.0;

@@ -223,8 +223,8 @@ class FusedBasicBlockNet:
                 off = trace_bytes
                 self.trace_offsets[p.name] = off
                 trace_bytes += ho * wo * d.c_out
-            S = torch.tensor(d.w_scale, dtype=torch.float32) * torch.tensor(d.a_scale, dtype=torch.float32)
-            inv = float(torch.tensor(1.0, dtype=torch.float32) / torch.tensor(p.out_step, dtype=torch.float32)) if p.out_bits else 0.0
+            S = ebs.ebs_combined_scale(d.w_scale, d.a_scale)          # the library's own fp32 roundings
+            inv = ebs.ebs_reciprocal_step(p.out_step) if p.out_bits else 0.0
             self._keep.append((p.packed_w, p.ch_scale, p.ch_bias))
             return ebs.ebs_fused_layer(
                 p.packed_w.data_ptr() + ebs.ebs_packed_weight_plane_bytes(d),
@@ -249,8 +249,8 @@ class FusedBasicBlockNet:
         self.layers_dev = torch.empty(self.n_layers * ctypes_sizeof(ebs.ebs_fused_layer), dtype=torch.uint8, device=self.device)
         ebs.ebs_fused_plan_upload(layers, self.layers_dev)
         fd = fc.desc
-        S_fc = torch.tensor(fd.w_scale, dtype=torch.float32) * torch.tensor(fd.a_scale, dtype=torch.float32)
-        a_inv = torch.tensor(1.0, dtype=torch.float32) / torch.tensor(fd.a_scale, dtype=torch.float32)
+        S_fc = ebs.ebs_combined_scale(fd.w_scale, fd.a_scale)
+        a_inv = ebs.ebs_reciprocal_step(fd.a_scale)
         self.head = ebs.ebs_fused_head(fc.packed_w.data_ptr() + ebs.ebs_packed_weight_plane_bytes(fd),
                                        None if fc.ch_scale is None else fc.ch_scale.data_ptr(),
                                        None if fc.ch_bias is None else fc.ch_bias.data_ptr(), fd.c_in, fd.c_out,

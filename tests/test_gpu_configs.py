@@ -57,6 +57,15 @@ def check_layer(ebs, U, oracle, spec, qa, qw, sample=None, next_bits=3):
     acc, y, pn = U.conv_on_device(px, n, L.h_in, L.w_in, pw, d, epi, True, True, next_bits)
     torch.cuda.synchronize()
     assert np.array_equal(U.images_nchw(acc, idx), ref), f"{L.name}: int32 accumulators"
+    if sample is not None:
+        # every image of the batch, interior ones included: the chosen kernel against the integer-pipe family on the GPU
+        # (the literal plane-pair evaluation, itself oracle-checked on the sampled images just above and in the small cases)
+        acc2 = torch.empty_like(acc)
+        pn2 = torch.empty_like(pn)
+        ebs.ebs_conv2d_mixed(px, n, L.h_in, L.w_in, pw, d, epi, acc2, None, pn2, variant=-2)
+        torch.cuda.synchronize()
+        assert torch.equal(acc, acc2), f"{L.name}: accumulators of the whole batch differ between kernel families"
+        assert torch.equal(pn, pn2), f"{L.name}: packed planes of the whole batch differ between kernel families"
     got_y = U.images_nchw(y, idx)
     assert np.allclose(got_y, y_ref, rtol=RTOL, atol=0.0), f"{L.name}: fp32 outputs"
     got_q = oracle.unpack_acts(U.packed_images(pn, n, L.h_out, L.w_out, L.c_out, next_bits, idx), L.c_out)
@@ -108,7 +117,9 @@ def test_config2_in_the_bench_launch_configuration(ebs, U, oracle, gen):
 def test_config3_resnet18_batch64_sampled_images(ebs, U, oracle, gen):
     for spec in gen.config3(0):
         qa = gen.act_codes(spec)
-        check_layer(ebs, U, oracle, spec, qa, gen.weight_codes(spec), sample=[0, qa.shape[0] - 1], next_bits=4)
+        n = qa.shape[0]
+        picks = sorted({0, n - 1, *(int(v) for v in np.random.default_rng(spec.index).integers(1, n - 1, size=2))})
+        check_layer(ebs, U, oracle, spec, qa, gen.weight_codes(spec), sample=picks, next_bits=4)
 
 
 def test_config4_bitplane_gemm_all_pairs(ebs, U, oracle, gen):
@@ -135,6 +146,11 @@ def test_config4_bitplane_gemm_all_pairs(ebs, U, oracle, gen):
             ref = oracle.conv2d_codes(sel, qw)                           # [rows, 4096, 1, 1]
             for i, (r, c) in enumerate(rows):
                 assert np.array_equal(got[0, r, c], ref[i, :, 0, 0]), f"W{wb}A{ab} row ({r},{c})"
+            if (wb, ab) in ((1, 1), (3, 5), (5, 2), (8, 8)):           # every output: against the integer-pipe family on the GPU
+                acc2 = torch.empty_like(acc)
+                ebs.ebs_conv2d_mixed(px, 1, 64, 64, pw, d, None, acc2, None, None, variant=-2)
+                torch.cuda.synchronize()
+                assert torch.equal(acc, acc2), f"W{wb}A{ab}: kernel families disagree"
             # a property that holds at any size: column sums of acc = (sum of activation rows) . weights
             if (wb, ab) in ((1, 1), (4, 4), (8, 8)):
                 colsum = got[0].reshape(-1, 4096).astype(np.int64).sum(axis=0)
@@ -148,7 +164,7 @@ def test_config5_resnet50_chain_batch256_sampled_images(ebs, U, oracle, gen):
     requantization steps; the GPU runs the full batch and must reproduce the sampled images' codes."""
     specs = gen.config5(0)
     n = specs[0].batch
-    sample = [0, n - 1]
+    sample = [0, 101, n - 1]                                 # first, an interior and the last image
     qa0 = gen.act_codes(specs[0])
     L0 = specs[0].layer
     # ---- oracle chain on the sampled images (also decides bias / next step per layer)
