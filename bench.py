@@ -468,6 +468,8 @@ def measure_config(ebs, name, dev, timer, peaks, args, sm_max, detail: bool):
     out["binary_tops"] = total_ops / (step_ms * 1e-3) / 1e12
     out["int8_tops"] = total_int8 / (step_ms * 1e-3) / 1e12
     out["imgs_per_s"] = n_img / (step_ms * 1e-3)
+    if args.step_only:
+        return out, layers, step_graph, one_step, launches_per_step, total_ops, total_int8
 
     # the conv launches alone, both output modes, cold (flush before every replay) and warm (replays back to back)
     modes = {}
@@ -757,6 +759,15 @@ def run_gpu(args):
     barrier()
     total_ms = max_over_ranks(float(sum(e0.elapsed_time(e1) for e0, e1 in ev)), dev)
     ms_per_step = total_ms / args.steps / inner
+    if args.step_only:
+        # the short form for profiler captures: the timed steps alone, none of the per-layer, per-mode or context legs
+        sampler.stop()
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": world * total_ops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT,
+                              "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+                              "ms_per_step": ms_per_step, "step_only": True, "launches_per_step": launches_per_step,
+                              "config": {"workload": WORKLOAD_TEXT[headline]}}))
+        return
     # the dominant kernel family (the bit-plane convolution) alone, in the step's output mode, cold L2, timed with
     # CUDA events on the launching stream while the clock sampler still runs
     mode = "fused" if chained else "raw"
@@ -903,6 +914,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true", help="skip the streaming-kernel and whole-network legs")
+    ap.add_argument("--step-only", action="store_true",
+                    help="time the steps of --workload and print a short line: no per-layer, per-mode or context legs "
+                         "(the command profiler captures run)")
     ap.add_argument("--workload", default="all", choices=["all"] + sorted(WORKLOAD_TEXT),
                     help="all (default): the five configurations, headline config5; configN: that one alone")
     args = ap.parse_args()

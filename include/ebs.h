@@ -255,6 +255,28 @@ long long ebs_device_wait_timeouts(void);
 int ebs_check_device_status(void);
 
 /*
+ * The range-checked build (the paper has no counterpart).  The library is built twice from the same sources:
+ * libebs.so, and libebs_checked.so with -DEBS_CHECKED, in which the convolution kernels pass the indices they
+ * compute from the run-time geometry (offsets into the operand and result buffers, into their shared-memory rings
+ * and tables) through a range test before the access.  A violation is recorded on the device -- the first one wins
+ * -- and the access is skipped: nothing traps, the kernel runs to its end, results may be incomplete.
+ * ebs_checked_build: 1 in the checked library, 0 in the normal one.
+ * ebs_checked_status: synchronizes the device; returns 1 if a violation was recorded (and stores the site code --
+ * kernel family * 16 + access, see CheckSite in csrc/ebs_internal.cuh --, the offending index and its limit in the
+ * non-null host pointers), 0 if none, EBS_ERR_UNSUPPORTED in the normal build, EBS_ERR_CUDA if a runtime call failed;
+ * clear != 0 resets the record afterwards.
+ */
+int ebs_checked_build(void);
+int ebs_checked_status(int* site, long long* index, long long* limit, int clear);
+/*
+ * Test hook of the range-checked build (EBS_ERR_UNSUPPORTED in the normal one): the convolution launches made
+ * afterwards take their accumulator / fp32 result buffers to be `elements` elements shorter than they are, so the
+ * stores of the last elements are refused and recorded although the memory is there: it shows the record working
+ * without any access out of bounds.  0 restores the true extents.  Process-wide.
+ */
+int ebs_test_checked_shrink(long long elements);
+
+/*
  * Test hook for the give-up path of the tensor-core kernels (the paper has no counterpart).  `limit` = number of
  * polls a bounded wait makes before it gives up (0 restores the default, about 2^20 polls of >= 40 ns);
  * skip_mma = 1 makes the persistent pipeline kernel's issuing thread issue no tensor-core work at all, so that

@@ -14,7 +14,8 @@ from typing import Optional
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libebs.so")
+# EBS_LIBRARY=checked selects the range-checked build of the same sources (libebs_checked.so); default: libebs.so
+LIB_PATH = os.path.join(_PKG, "libebs_checked.so" if os.environ.get("EBS_LIBRARY") == "checked" else "libebs.so")
 
 EBS_OK, EBS_ERR_INVALID_ARG, EBS_ERR_UNSUPPORTED, EBS_ERR_OVERFLOW, EBS_ERR_CUDA, EBS_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 EBS_ERR_SCRATCH_TOO_SMALL = -6
@@ -29,6 +30,7 @@ EXPORTS = [
     "ebs_search_act_forward", "ebs_expected_flops", "ebs_fused_plan_upload", "ebs_resnet_cifar_forward", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
     "ebs_conv_variant_family", "ebs_conv_variant_applies", "ebs_check_device_status", "ebs_test_set_device_wait",
     "ebs_conv2d_i8", "ebs_maxpool_packed", "ebs_combined_scale", "ebs_reciprocal_step",
+    "ebs_checked_build", "ebs_checked_status", "ebs_test_checked_shrink",
 ]
 
 
@@ -105,6 +107,9 @@ def lib() -> ctypes.CDLL:
         L.ebs_combined_scale.restype = f
         L.ebs_reciprocal_step.argtypes = [f]
         L.ebs_reciprocal_step.restype = f
+        L.ebs_checked_status.argtypes = [ctypes.POINTER(i), ctypes.POINTER(ctypes.c_longlong),
+                                         ctypes.POINTER(ctypes.c_longlong), i]
+        L.ebs_test_checked_shrink.argtypes = [ctypes.c_longlong]
         L.ebs_conv_variant_family.argtypes = [i]
         L.ebs_conv_variant_family.restype = ctypes.c_char_p
         L.ebs_conv_variant_applies.argtypes = [D, i, i, i, E, i, i, i, i]
@@ -313,6 +318,23 @@ def ebs_conv_variant_applies(desc, n, h, w, epi=None, want_acc=True, want_y=Fals
 
 def ebs_check_device_status() -> int:
     return int(lib().ebs_check_device_status())
+
+
+def ebs_checked_build() -> bool:
+    return bool(lib().ebs_checked_build())
+
+
+def ebs_checked_status(clear: bool = True):
+    """(recorded, site, index, limit) of the range-checked build; raises in the normal build."""
+    site, index, limit = ctypes.c_int(0), ctypes.c_longlong(0), ctypes.c_longlong(0)
+    rc = lib().ebs_checked_status(ctypes.byref(site), ctypes.byref(index), ctypes.byref(limit), int(bool(clear)))
+    if rc < 0:
+        _check(rc, "ebs_checked_status")
+    return bool(rc), site.value, index.value, limit.value
+
+
+def ebs_test_checked_shrink(elements: int) -> None:
+    _check(lib().ebs_test_checked_shrink(int(elements)), "ebs_test_checked_shrink")
 
 
 def ebs_test_set_device_wait(limit: int, skip_mma: bool) -> None:

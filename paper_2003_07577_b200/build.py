@@ -2,6 +2,8 @@
 
 Every translation unit under csrc/ is compiled to an object file in parallel and the objects
 are linked into ``paper_2003_07577_b200/libebs.so``.  Nothing is cached outside the tree.
+``build(checked=True)`` builds the range-checked variant of the same sources (``-DEBS_CHECKED``,
+objects under ``build_checked/``) into ``libebs_checked.so``.
 """
 from __future__ import annotations
 
@@ -39,12 +41,16 @@ def _deps(path: str, seen: set) -> set:
     return seen
 
 
-def _compile(src: str, verbose: bool) -> str:
-    obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
+LIB_CHECKED = os.path.join(PKG, "libebs_checked.so")
+
+
+def _compile(src: str, verbose: bool, checked: bool = False) -> str:
+    obj = os.path.join(OBJ + ("_checked" if checked else ""), os.path.basename(src)[:-3] + ".o")
     newest = max(os.path.getmtime(p) for p in _deps(src, set()))
     if os.path.exists(obj) and os.path.getmtime(obj) >= newest:
         return obj
-    cmd = ["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
+    cmd = ["nvcc"] + NVCC_FLAGS + (["-DEBS_CHECKED"] if checked else []) + (["-Xptxas", "-v"] if verbose else []) + \
+          ["-c", src, "-o", obj]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError(f"nvcc failed for {src}:\n{res.stdout}\n{res.stderr}")
@@ -54,22 +60,23 @@ def _compile(src: str, verbose: bool) -> str:
     return obj
 
 
-def build(force: bool = False, verbose: bool = False, jobs: int | None = None) -> str:
-    os.makedirs(OBJ, exist_ok=True)
+def build(force: bool = False, verbose: bool = False, jobs: int | None = None, checked: bool = False) -> str:
+    obj_dir, lib = OBJ + ("_checked" if checked else ""), (LIB_CHECKED if checked else LIB)
+    os.makedirs(obj_dir, exist_ok=True)
     srcs = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
     if force:
-        for o in glob.glob(os.path.join(OBJ, "*.o")):
+        for o in glob.glob(os.path.join(obj_dir, "*.o")):
             os.remove(o)
     jobs = jobs or min(len(srcs), os.cpu_count() or 4)
     with concurrent.futures.ThreadPoolExecutor(max_workers=jobs) as ex:
-        objs = list(ex.map(lambda s: _compile(s, verbose), srcs))
-    if force or not os.path.exists(LIB) or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs):
-        cmd = ["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB] + objs + ["-lcudart"]
+        objs = list(ex.map(lambda s: _compile(s, verbose, checked), srcs))
+    if force or not os.path.exists(lib) or any(os.path.getmtime(o) > os.path.getmtime(lib) for o in objs):
+        cmd = ["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", lib] + objs + ["-lcudart"]
         res = subprocess.run(cmd, capture_output=True, text=True)
         if res.returncode != 0:
             raise RuntimeError(f"link failed:\n{res.stdout}\n{res.stderr}")
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, checked="--checked" in sys.argv))

@@ -67,6 +67,18 @@ unsigned long long conv_umma_timeouts() {
 // changed only by ebs_test_set_device_wait.
 static unsigned g_wait_limit = 1u << 20;
 static int g_test_flags = 0;
+static long long g_check_shrink = 0;      // range-checked build, tests only: result extents declared this much too short
+
+// Range-checked build only: the device words the kernels record their first out-of-range index in.
+#ifdef EBS_CHECKED
+static __device__ unsigned long long g_check_words[4];
+static unsigned long long* check_status_words() {
+    void* ptr = nullptr;
+    return cudaGetSymbolAddress(&ptr, g_check_words) == cudaSuccess ? static_cast<unsigned long long*>(ptr) : nullptr;
+}
+#else
+static unsigned long long* check_status_words() { return nullptr; }
+#endif
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -238,6 +250,12 @@ static int conv_plan(const void* packed_x, int n, int h, int w, const void* pack
     }
     p.wait_limit = g_wait_limit;
     p.test_flags = g_test_flags;
+    p.lim_x = byte_acts ? in_pixels * p.CW * 8 : in_pixels * p.CW * d->a_bits;
+    p.lim_w = (long long)(packed_weight_plane_bytes(*d) / 4);
+    p.lim_w8 = (long long)d->kh * d->kw * p.CW * p.Co16 * 32;
+    p.lim_out = P * d->c_out - g_check_shrink;
+    p.lim_pn = packed_next && epi ? P * p.CWo * epi->next_a_bits : 0;
+    p.check_status = check_status_words();
     if (epi) {
         p.ch_scale = epi->ch_scale_dev; p.ch_bias = epi->ch_bias_dev; p.residual = epi->residual_dev;
         p.res_packed = static_cast<const uint32_t*>(epi->res_packed_dev); p.res_bits = epi->res_bits; p.res_scale = epi->res_scale;
@@ -466,6 +484,44 @@ int ebs_check_device_status(void) {
     const bool fresh = now > seen;
     seen = now;
     return fresh ? EBS_ERR_TIMEOUT : EBS_OK;
+}
+
+int ebs_checked_build(void) {
+#ifdef EBS_CHECKED
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+int ebs_checked_status(int* site, long long* index, long long* limit, int clear) {
+#ifdef EBS_CHECKED
+    unsigned long long w[4] = {0, 0, 0, 0};
+    if (cudaDeviceSynchronize() != cudaSuccess) return EBS_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(w, g_check_words, sizeof(w)) != cudaSuccess) return EBS_ERR_CUDA;
+    if (site) *site = (int)(w[0] >> 48);
+    if (index) *index = (long long)w[1];
+    if (limit) *limit = (long long)w[2];
+    if (clear) {
+        const unsigned long long z[4] = {0, 0, 0, 0};
+        if (cudaMemcpyToSymbol(g_check_words, z, sizeof(z)) != cudaSuccess) return EBS_ERR_CUDA;
+    }
+    return w[0] ? 1 : 0;
+#else
+    (void)site; (void)index; (void)limit; (void)clear;
+    return EBS_ERR_UNSUPPORTED;
+#endif
+}
+
+int ebs_test_checked_shrink(long long elements) {
+#ifdef EBS_CHECKED
+    if (elements < 0) return EBS_ERR_INVALID_ARG;
+    g_check_shrink = elements;
+    return EBS_OK;
+#else
+    (void)elements;
+    return EBS_ERR_UNSUPPORTED;
+#endif
 }
 
 long long ebs_device_wait_timeouts(void) { return (long long)conv_umma_timeouts(); }

@@ -154,7 +154,9 @@ conv_mma_kernel(const ConvParams p) {
 #pragma unroll
             for (int u = 0; u < PPT; ++u) {
                 const int pl = (tid % TILE_P) + u * NTH;
-                const bool valid = kvalid && ((row_ok[u] >> r) & (col_ok[u] >> s) & 1u);
+                const bool valid = kvalid && ((row_ok[u] >> r) & (col_ok[u] >> s) & 1u) &&
+                                   EBS_IN_RANGE(p, CHK_MMA_X, (long long)pix_off[u] + info.x + AB - 1, p.lim_x) &&
+                                   EBS_IN_RANGE(p, CHK_MMA_STAGE, (q * TILE_P + pl) * AB + AB - 1, KSTEP * TILE_P * AB);
                 const uint32_t* src = valid ? p.x + (pix_off[u] + info.x) : p.x;
                 uint32_t* dst = A_s + (q * TILE_P + pl) * AB;
 #pragma unroll
@@ -168,7 +170,8 @@ conv_mma_kernel(const ConvParams p) {
         for (int e = tid; e < KSTEP * TILE_C * 2; e += NTH) {
             const int q = e / (TILE_C * 2), rem = e - q * (TILE_C * 2), c = rem >> 1, half = rem & 1;
             const int kk = kk0 + q;
-            const bool valid = kk < p.KK && co0 + c < p.Co16;
+            const bool valid = kk < p.KK && co0 + c < p.Co16 &&
+                               EBS_IN_RANGE(p, CHK_MMA_W8, ((long long)kk * p.Co16 + co0 + c) * 32 + half * 16 + 15, p.lim_w8);
             const uint8_t* src = valid ? p.w8 + ((size_t)kk * p.Co16 + co0 + c) * 32 + half * 16 : p.w8;
             cp_async_bytes(W_s + (q * TILE_C + c) * 8 + half * 4, src, 16, valid);
         }
@@ -352,7 +355,7 @@ conv_mma_kernel(const ConvParams p) {
                     int* row = p.acc + (size_t)gp * p.Co + co_t;
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt)
-                        if (gp < p.P && co_t + nt * 8 < p.Co)
+                        if (gp < p.P && co_t + nt * 8 < p.Co && EBS_IN_RANGE(p, CHK_MMA_ACC, (long long)gp * p.Co + co_t + nt * 8 + 1, p.lim_out))
                             *reinterpret_cast<int2*>(row + nt * 8) = make_int2(acc[mt][nt][half * 2], acc[mt][nt][half * 2 + 1]);
                 }
         }
@@ -370,7 +373,7 @@ conv_mma_kernel(const ConvParams p) {
                     for (int nt = 0; nt < NT; ++nt) {
                         const bool valid = gp < p.P && co_t + nt * 8 < p.Co;
                         if constexpr (!FULL) {
-                            if (acc_inline && valid)
+                            if (acc_inline && valid && EBS_IN_RANGE(p, CHK_MMA_ACC, row_o + nt * 8 + 1, p.lim_out))
                                 *reinterpret_cast<int2*>(p.acc + row_o + nt * 8) =
                                     make_int2(acc[mt][nt][half * 2], acc[mt][nt][half * 2 + 1]);
                         }
@@ -410,7 +413,8 @@ conv_mma_kernel(const ConvParams p) {
                             code0 = quantize_act_code(y0, p.inv_next, qmax);
                             code1 = quantize_act_code(y1, p.inv_next, qmax);
                         }
-                        if (want_y && valid) *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
+                        if (want_y && valid && EBS_IN_RANGE(p, CHK_MMA_Y, row_o + nt * 8 + 1, p.lim_out))
+                            *reinterpret_cast<float2*>(p.y + row_o + nt * 8) = make_float2(y0, y1);
                         if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
                     }
                 }
@@ -431,7 +435,7 @@ conv_mma_kernel(const ConvParams p) {
                 if (pvalid && co < p.Co) {
                     const size_t o = (size_t)gp * p.Co + co;
                     const bool two = co + 1 < p.Co;
-                    if (p.acc) {
+                    if (p.acc && EBS_IN_RANGE(p, CHK_MMA_ACC, o + (two ? 1 : 0), p.lim_out)) {
                         if (pair_ok) *reinterpret_cast<int2*>(p.acc + o) = make_int2(a0, a1);
                         else { p.acc[o] = a0; if (two) p.acc[o + 1] = a1; }
                     }
@@ -457,7 +461,7 @@ conv_mma_kernel(const ConvParams p) {
                             if (!(y0 > 0.0f)) y0 = 0.0f;
                             if (!(y1 > 0.0f)) y1 = 0.0f;
                         }
-                        if (want_y) {
+                        if (want_y && EBS_IN_RANGE(p, CHK_MMA_Y, o + (two ? 1 : 0), p.lim_out)) {
                             if (p.y_nchw) {
                                 const int hw = p.Ho * p.Wo;
                                 const int n = gp / hw, rem = gp - n * hw;

@@ -80,7 +80,8 @@ conv_mma_strip_kernel(const ConvParams p) {
         for (int e = tid; e < (taps + 1) * TILE_C; e += NTH) {
             const int t = e / TILE_C, row = e - t * TILE_C;
             uint4 v = make_uint4(0, 0, 0, 0);
-            if (t < taps && co0 + row < p.Co16) {
+            if (t < taps && co0 + row < p.Co16 &&
+                EBS_IN_RANGE(p, CHK_MS_W8, ((long long)t * p.Co16 + co0 + row) * 32 + 31, p.lim_w8)) {
                 const uint4* src = reinterpret_cast<const uint4*>(p.w8 + ((size_t)t * p.Co16 + co0 + row) * 32);
                 const int sw = ((co0 + row) >> 2) & 1;                   // the image swaps the halves of these rows
                 const uint4 lo = __ldg(src + sw), hi = __ldg(src + (sw ^ 1));
@@ -93,7 +94,9 @@ conv_mma_strip_kernel(const ConvParams p) {
 #pragma unroll 1
         for (int e = tid; e < taps * p.CW * TILE_C * 2; e += NTH) {
             const int half = e & 1, row = (e >> 1) % TILE_C, kk = (e >> 1) / TILE_C;
-            const bool valid = co0 + row < p.Co16;
+            const bool valid = co0 + row < p.Co16 &&
+                               EBS_IN_RANGE(p, CHK_MS_W8, ((long long)kk * p.Co16 + co0 + row) * 32 + half * 16 + 15, p.lim_w8) &&
+                               EBS_IN_RANGE(p, CHK_MS_WS, (kk * TILE_C + row) * 32 + half * 16 + 15, taps * p.CW * TILE_C * 32);
             const uint8_t* src = valid ? p.w8 + ((size_t)kk * p.Co16 + co0 + row) * 32 + half * 16 : p.w8;
             cp_async_bytes(wimg + (kk * TILE_C + row) * 32 + half * 16, src, 16, valid);
         }
@@ -121,7 +124,8 @@ conv_mma_strip_kernel(const ConvParams p) {
             const int n = n0 + ch_;
             if (hp < p.Ho && wq < p.Wo) gp = (n * p.Ho + hp) * p.Wo + wq;            // the output pixel of this frame row
             const int h = pointwise ? hp * p.sh : hp - p.ph, w = pointwise ? wq * p.sw : wq - p.pw;
-            if ((unsigned)h < (unsigned)p.H && (unsigned)w < (unsigned)p.W) {
+            if ((unsigned)h < (unsigned)p.H && (unsigned)w < (unsigned)p.W &&
+                EBS_IN_RANGE(p, CHK_MS_X, (((long long)(n * p.H + h) * p.W + w) * p.CW + cw) * AB + AB - 1, p.lim_x)) {
                 uint32_t words[AB];
                 load_words_global<AB>(p.x + (((size_t)(n * p.H + h) * p.W + w) * p.CW + cw) * AB, words);
 #pragma unroll
@@ -141,6 +145,7 @@ conv_mma_strip_kernel(const ConvParams p) {
             }
         }
         if (cw == 0 && s < TILE_P) gp_s[s] = gp;
+        if (!EBS_IN_RANGE(p, CHK_MS_STRIP, COMPACT ? s * 16 + 15 : (cw * SP + s) * 32 + 31, COMPACT ? SP * 16 : p.CW * SP * 32)) continue;
         if constexpr (COMPACT) {
             reinterpret_cast<uint4*>(strip)[s] = make_uint4(r[0], r[1], r[2], r[3]);
         } else {
@@ -293,7 +298,7 @@ conv_mma_strip_kernel(const ConvParams p) {
                 int* row = p.acc + (size_t)(gp < 0 ? 0 : gp) * p.Co + co_t;
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt)
-                    if (gp >= 0 && co_t + nt * 8 < p.Co)
+                    if (gp >= 0 && co_t + nt * 8 < p.Co && EBS_IN_RANGE(p, CHK_MS_ACC, (long long)gp * p.Co + co_t + nt * 8 + 1, p.lim_out))
                         *reinterpret_cast<int2*>(row + nt * 8) = make_int2(acc[mt][nt][half * 2], acc[mt][nt][half * 2 + 1]);
             }
     }
@@ -311,7 +316,7 @@ conv_mma_strip_kernel(const ConvParams p) {
                 for (int nt = 0; nt < NT; ++nt) {
                     const bool valid = gp >= 0 && co_t + nt * 8 < p.Co;
                     if constexpr (!RES) {
-                        if (acc_inline && valid)
+                        if (acc_inline && valid && EBS_IN_RANGE(p, CHK_MS_ACC, (long long)gp * p.Co + co_t + nt * 8 + 1, p.lim_out))
                             *reinterpret_cast<int2*>(p.acc + (size_t)gp * p.Co + co_t + nt * 8) =
                                 make_int2(acc[mt][nt][half * 2], acc[mt][nt][half * 2 + 1]);
                     }
@@ -351,7 +356,8 @@ conv_mma_strip_kernel(const ConvParams p) {
                         code0 = quantize_act_code(y0, p.inv_next, qmax);
                         code1 = quantize_act_code(y1, p.inv_next, qmax);
                     }
-                    if (want_y && valid) *reinterpret_cast<float2*>(yrow + nt * 8) = make_float2(y0, y1);
+                    if (want_y && valid && EBS_IN_RANGE(p, CHK_MS_Y, (long long)gp * p.Co + co_t + nt * 8 + 1, p.lim_out))
+                        *reinterpret_cast<float2*>(yrow + nt * 8) = make_float2(y0, y1);
                     if (want_q) *reinterpret_cast<uint16_t*>(code_row + nt * 8) = (uint16_t)(code0 | (code1 << 8));
                 }
             }
@@ -370,6 +376,7 @@ conv_mma_strip_kernel(const ConvParams p) {
 #pragma unroll
             for (int k = 0; k < NW; ++k) codes[k] = row[k];
             uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + cwg) * p.next_bits;
+            if (!EBS_IN_RANGE(p, CHK_MS_PN, ((long long)gp * p.CWo + cwg) * p.next_bits + p.next_bits - 1, p.lim_pn)) continue;
 #pragma unroll 1
             for (int j = 0; j < p.next_bits; ++j) {
                 uint32_t word = 0u;

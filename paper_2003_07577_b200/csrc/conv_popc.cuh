@@ -99,7 +99,7 @@ conv_popc_kernel(const ConvParams p) {
                 const int hi = pix_h0[i] + (info & 0xff), wi = pix_w0[i] + ((info >> 8) & 0xff);
                 if ((unsigned)hi < (unsigned)p.H && (unsigned)wi < (unsigned)p.W) {
                     const size_t off = ((size_t)(base + hi * p.W + wi) * p.CW + (info >> 16)) * AB;
-                    load_words_global<AB>(p.x + off, words);
+                    if (EBS_IN_RANGE(p, CHK_POPC_X, off + AB - 1, p.lim_x)) load_words_global<AB>(p.x + off, words);
                 }
             }
 #pragma unroll
@@ -111,7 +111,8 @@ conv_popc_kernel(const ConvParams p) {
             const int c = e / WB;
             const int kk = kk0 + q;
             uint32_t v = 0u;
-            if (kk < p.KK && co0 + c < p.Co) v = __ldg(p.w + ((size_t)kk * p.Co + co0) * WB + e);
+            if (kk < p.KK && co0 + c < p.Co && EBS_IN_RANGE(p, CHK_POPC_W, ((long long)kk * p.Co + co0) * WB + e, p.lim_w))
+                v = __ldg(p.w + ((size_t)kk * p.Co + co0) * WB + e);
             (&W_s[q][0][0])[e] = v;
         }
         __syncthreads();
@@ -170,7 +171,7 @@ conv_popc_kernel(const ConvParams p) {
             if (valid) {
                 const size_t o = (size_t)gp * p.Co + co;
                 const int av = p.w_levels ? 2 * acc[t][c] + wsum[t] : acc[t][c];
-                if (p.acc) p.acc[o] = av;
+                if (p.acc && EBS_IN_RANGE(p, CHK_POPC_ACC, o, p.lim_out)) p.acc[o] = av;
                 if (want_y || want_q) {
                     float yv = __fmul_rn((float)av, p.S);
                     if (p.ch_scale) yv = __fmul_rn(yv, __ldg(p.ch_scale + co));
@@ -178,7 +179,7 @@ conv_popc_kernel(const ConvParams p) {
                     if (p.residual) yv = __fadd_rn(yv, __ldg(p.residual + o));
                     if (p.res_packed) yv = __fadd_rn(yv, packed_residual(p, gp, co));
                     if (p.relu && !(yv > 0.0f)) yv = 0.0f;
-                    if (want_y) {
+                    if (want_y && EBS_IN_RANGE(p, CHK_POPC_Y, o, p.lim_out)) {
                         if (p.y_nchw) {
                             const int hw = p.Ho * p.Wo;
                             const int n = gp / hw, rem = gp - n * hw;
@@ -190,7 +191,8 @@ conv_popc_kernel(const ConvParams p) {
                     if (want_q) code = quantize_code(yv, p.inv_next, 0, qmax);
                 }
             }
-            if (want_q) out_s[pl * code_row_bytes(TILE_C) + cl] = (uint8_t)code;
+            if (want_q && EBS_IN_RANGE(p, CHK_TILE_CODES, pl * code_row_bytes(TILE_C) + cl, TILE_P * code_row_bytes(TILE_C)))
+                out_s[pl * code_row_bytes(TILE_C) + cl] = (uint8_t)code;
         }
     }
     if (want_q) {

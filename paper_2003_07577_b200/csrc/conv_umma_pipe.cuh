@@ -272,7 +272,7 @@ __device__ __forceinline__ uint64_t f32x2_add_rd(uint64_t a, uint64_t b) {
 template <bool WANT_Q, bool SMALL_ACC>
 __device__ __forceinline__ void pipe_group32(const ConvParams& p, uint32_t (&v)[32], size_t o, bool pvalid, float S,
                                              float inv_next, int nb, int qmax, uint32_t* dst) {
-    if (p.acc && pvalid) {
+    if (p.acc && pvalid && EBS_IN_RANGE(p, CHK_PIPE_ACC, o + 31, p.lim_out)) {
 #pragma unroll
         for (int gq = 0; gq < 8; ++gq)
             *reinterpret_cast<int4*>(p.acc + o + 4 * gq) =
@@ -286,7 +286,7 @@ __device__ __forceinline__ void pipe_group32(const ConvParams& p, uint32_t (&v)[
 #pragma unroll
         for (int bb = 0; bb < 8; ++bb)
             yy[h][bb] = f32x2_mul_rn(f32x2_pack((float)(int)v[16 * h + bb], (float)(int)v[16 * h + 8 + bb]), S2);
-    if (p.y && pvalid) {
+    if (p.y && pvalid && EBS_IN_RANGE(p, CHK_PIPE_Y, o + 31, p.lim_out)) {
         const bool relu = p.relu != 0;
 #pragma unroll
         for (int gq = 0; gq < 8; ++gq) {
@@ -338,7 +338,7 @@ __device__ __forceinline__ void pipe_group32(const ConvParams& p, uint32_t (&v)[
             for (int bb = 1; bb < 8; ++bb) t |= cr[bb] & (0x01010101u << ((bb + j) & 7));
             planes[j] = __funnelshift_r(t, t, j);
         }
-        if (pvalid) {
+        if (pvalid && EBS_IN_RANGE(p, CHK_PIPE_PN, (dst - p.packed_next) + nb - 1, p.lim_pn)) {
             if (nb == 4) {
                 *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
             } else if (nb == 8) {
@@ -429,7 +429,8 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
             uint32_t b_inc = 0u;
             if (j == g.m_sub - 1)
                 b_inc = (g.b_resident && tl == ntp - 1) ? bt16 * (uint32_t)(1 + g.taps - ntp) : bt16;
-            mma_tab[e] = make_uint2(a_off, (uint32_t)(j * TILE_N) | (b_inc << 16));
+            if (EBS_IN_RANGE(p, CHK_PIPE_TAB, e, PIPE_MAX_MMAS))
+                mma_tab[e] = make_uint2(a_off, (uint32_t)(j * TILE_N) | (b_inc << 16));
         }
     }
     const int NST = g.n_stages, KS = g.ks, KSS = g.kss, NSUB = g.nsub, SP = g.SP, S = g.S;
@@ -458,7 +459,7 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
     if (tid == 0) {
         abort_flag = 0;
         for (int s = 0; s < PIPE_MAX_STAGES; ++s) {
-            mbar_init(&st_full[s], PIPE_EXPANDERS * g.nsub);       // every expander arrives once per pass
+            mbar_init(&st_full[s], (PIPE_EXPANDERS / 32) * g.nsub);  // every expander warp arrives once per pass
             mbar_init(&st_empty[s], 1);
         }
         for (int s = 0; s < PIPE_MAX_BSLOTS; ++s) {
@@ -467,8 +468,8 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
         }
         mbar_init(&acc_full[0], 1);
         mbar_init(&acc_full[1], 1);
-        mbar_init(&acc_empty[0], PIPE_EPI_WARPS * 32);
-        mbar_init(&acc_empty[1], PIPE_EPI_WARPS * 32);
+        mbar_init(&acc_empty[0], PIPE_EPI_WARPS);
+        mbar_init(&acc_empty[1], PIPE_EPI_WARPS);
         mbar_init(&b_full, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -533,13 +534,15 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 for (int k = 0; k < NW; ++k) a_set[set][j][k] = 0u;
             if (paired) {                                       // both words of the pixel in one run of 2 * AB words
                 const int cw = wg * KSS + ld_sub * KS + slot_q[0];
-                if (slot_q[0] >= 0 && ld_off[0] >= 0 && cw < p.CW)
+                if (slot_q[0] >= 0 && ld_off[0] >= 0 && cw < p.CW &&
+                    EBS_IN_RANGE(p, CHK_PIPE_X, (long long)ld_off[0] + cw * NW + 2 * NW - 1, p.lim_x))
                     load_words_global<2 * NW>(p.x + (ld_off[0] + cw * NW), *reinterpret_cast<uint32_t(*)[2 * NW]>(&a_set[set][0][0]));
             } else {
 #pragma unroll
                 for (int j = 0; j < PIPE_SLOTS; ++j) {
                     const int cw = wg * KSS + ld_sub * KS + slot_q[j];
-                    if (slot_q[j] >= 0 && ld_off[j] >= 0 && cw < p.CW)
+                    if (slot_q[j] >= 0 && ld_off[j] >= 0 && cw < p.CW &&
+                        EBS_IN_RANGE(p, CHK_PIPE_X, (long long)ld_off[j] + cw * NW + NW - 1, p.lim_x))
                         load_words_global<NW>(p.x + (ld_off[j] + cw * NW), a_set[set][j]);
                 }
             }
@@ -595,11 +598,17 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                         }
                     }
                     uint8_t* dst = A_st + slot_dst[j];
+                    if (!EBS_IN_RANGE(p, CHK_PIPE_STAGE, (dst + SP * 16 + 15) - stages, NST * g.stage_bytes) ||
+                        !EBS_IN_RANGE(p, CHK_PIPE_STAGE, dst - stages, NST * g.stage_bytes))
+                        continue;
                     *reinterpret_cast<uint4*>(dst) = make_uint4(r[0], r[1], r[2], r[3]);
                     *reinterpret_cast<uint4*>(dst + SP * 16) = make_uint4(r[4], r[5], r[6], r[7]);
                 }
+                // every lane makes its bytes visible to the tensor core's proxy, then one lane arrives for the warp (32
+                // arrivals on one barrier word would be served one after the other)
                 asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-                mbar_arrive(&st_full[st]);
+                __syncwarp();
+                if ((tid & 31) == 0) mbar_arrive(&st_full[st]);
                 if (++sub == NSUB) {
                     sub = 0;
                     if (++st == NST) { st = 0; ++st_round; }
@@ -690,6 +699,7 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 mbar_arrive_expect_tx(&b_full, rows * 32u * (uint32_t)(p.CW * g.taps));
                 for (int cw = 0; cw < p.CW; ++cw)
                     for (int ts = 0; ts < g.taps; ++ts)
+                        if (EBS_IN_RANGE(p, CHK_PIPE_W8, ((long long)(s_tap_id[ts] * p.CW + cw) * p.Co16 + co0) * 32 + rows * 32 - 1, p.lim_w8))
                         bulk_copy_g2s(b_res + (cw * g.taps + ts) * B_TILE_BYTES,
                                       p.w8 + ((size_t)(s_tap_id[ts] * p.CW + cw) * p.Co16 + co0) * 32, rows * 32u, &b_full);
             } else {
@@ -716,6 +726,9 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                             const int n = min(GB, ntiles - i0);
                             mbar_arrive_expect_tx(&bs_full[bs], bytes * (uint32_t)n);
                             for (int i = 0; i < n; ++i) {
+                                // (a copy skipped by the range-checked build leaves its barrier incomplete: the CTA then gives
+                                // up at its bounded wait, which is reported as well)
+                                if (EBS_IN_RANGE(p, CHK_PIPE_W8, ((long long)(s_tap_id[ts] * p.CW + wgr * KSS + q) * p.Co16 + co0) * 32 + bytes - 1, p.lim_w8))
                                 bulk_copy_g2s(b_res + (bs * GB + i) * B_TILE_BYTES,
                                               p.w8 + ((size_t)(s_tap_id[ts] * p.CW + wgr * KSS + q) * p.Co16 + co0) * 32, bytes,
                                               &bs_full[bs]);
@@ -759,7 +772,8 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 else umma_epilogue<TILE_N, AFFINE>(p, tmem_acc, vwarp, gp, pvalid, 0, co0);
             }
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-            mbar_arrive(&acc_empty[buf]);
+            __syncwarp();
+            if ((tid & 31) == 0) mbar_arrive(&acc_empty[buf]);
         }
     }
 

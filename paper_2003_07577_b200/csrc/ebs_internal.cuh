@@ -41,6 +41,40 @@ struct ConvParams {
     int test_flags;                   // bit 0 (tests only): the MMA issuer issues nothing, so that waits run out
     int pipe_m_sub;                   // persistent pipeline kernel: accumulators per super-tile (0 = chosen by the library)
     int acc_small;                    // 1: every accumulator of the layer is below 2^22 in magnitude (worst case of its sizes and bit counts)
+    // Extents of the buffers, for the range-checked build (EBS_CHECKED); filled in every build.
+    long long lim_x, lim_w;           // 32-bit words of the packed activations (bytes / 4 on the byte-code path) and of the weight plane words
+    long long lim_w8;                 // bytes of the weight byte image
+    long long lim_out, lim_pn;        // elements of acc / y; 32-bit words of packed_next
+    unsigned long long* check_status; // EBS_CHECKED: device words {site << 48 | 1, index, limit}; else null
+};
+
+// Range-checked build (-DEBS_CHECKED, a second library beside the normal one): the indices the kernels compute from the
+// run-time geometry -- offsets into the operand and result buffers, into the shared-memory rings and tables -- pass
+// through EBS_IN_RANGE before the access.  A violation is recorded (the first one wins: site, index, limit) and the
+// access is skipped; nothing traps or asserts, the kernel runs to its end and the host reads the record with
+// ebs_checked_status.  In the normal build the macro is the constant `true` and costs nothing.
+#ifdef EBS_CHECKED
+__device__ __forceinline__ bool check_in_range(unsigned long long* st, unsigned site, long long idx, long long limit) {
+    if (idx >= 0 && idx < limit) return true;
+    if (st && atomicCAS(&st[0], 0ull, ((unsigned long long)site << 48) | 1ull) == 0ull) {
+        st[1] = (unsigned long long)idx;
+        st[2] = (unsigned long long)limit;
+    }
+    return false;
+}
+#define EBS_IN_RANGE(p, site, idx, limit) ::ebs::check_in_range((p).check_status, (site), (long long)(idx), (long long)(limit))
+#else
+#define EBS_IN_RANGE(p, site, idx, limit) true
+#endif
+// Sites (kernel family * 16 + access): 1x pipeline kernel, 2x warp-level strip kernel, 3x warp-level per-tap kernel,
+// 4x integer-pipe kernel, 5x shared epilogue helpers.
+enum CheckSite {
+    CHK_PIPE_X = 0x10, CHK_PIPE_STAGE = 0x11, CHK_PIPE_TAB = 0x12, CHK_PIPE_ACC = 0x13, CHK_PIPE_Y = 0x14, CHK_PIPE_PN = 0x15,
+    CHK_PIPE_W8 = 0x16,
+    CHK_MS_X = 0x20, CHK_MS_STRIP = 0x21, CHK_MS_W8 = 0x22, CHK_MS_ACC = 0x23, CHK_MS_Y = 0x24, CHK_MS_PN = 0x25, CHK_MS_WS = 0x26,
+    CHK_MMA_X = 0x30, CHK_MMA_W8 = 0x31, CHK_MMA_ACC = 0x32, CHK_MMA_Y = 0x33, CHK_MMA_STAGE = 0x34,
+    CHK_POPC_X = 0x40, CHK_POPC_W = 0x41, CHK_POPC_ACC = 0x42, CHK_POPC_Y = 0x43, CHK_POPC_SMEM = 0x44,
+    CHK_TILE_PN = 0x50, CHK_TILE_CODES = 0x51,
 };
 
 // One instantiation of the popcount kernel: launch function + its tile geometry.
@@ -215,6 +249,7 @@ __device__ __forceinline__ void pack_code_tile(const uint8_t* out_s, const ConvP
 #pragma unroll
         for (int k = 0; k < NW; ++k) codes[k] = row[k];
         uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + cwg) * p.next_bits;
+        if (!EBS_IN_RANGE(p, CHK_TILE_PN, ((size_t)gp * p.CWo + cwg) * p.next_bits + p.next_bits - 1, p.lim_pn)) continue;
 #pragma unroll 1
         for (int j = 0; j < p.next_bits; ++j) {
             uint32_t word = 0u;
