@@ -22,6 +22,20 @@ __device__ __forceinline__ uint32_t act_code<uint8_t>(uint8_t v, float, int qmax
 
 __device__ __forceinline__ void store_planes(const uint32_t (&codes)[8], int AB, uint32_t* __restrict__ dst);
 
+// Four activation codes as the bytes of one word (byte i = code of v_i), identical to quantize_code on each value but
+// without the float -> int conversion, which issues at an eighth of the fp32 rate: t = fl(fl(v * inv) + 0.5) as two
+// individually rounded operations; max(t, 0) (the maximum-number operation: a NaN gives 0, like quantize_code);
+// floor(t) is then in the low mantissa bits of t + 2^23 added with rounding toward minus infinity, and the clamp at
+// qmax is an integer minimum of the sum's bit pattern with bits(2^23) + qmax; the low bytes are the codes.
+__device__ __forceinline__ uint32_t act_codes4(float v0, float v1, float v2, float v3, float inv_scale, int qmax) {
+    const int m_hi = 0x4B000000 + qmax;
+    auto pat = [&](float v) {
+        const float t = fmaxf(__fadd_rn(__fmul_rn(v, inv_scale), 0.5f), 0.0f);
+        return (uint32_t)min(__float_as_int(__fadd_rd(t, 8388608.0f)), m_hi);
+    };
+    return __byte_perm(__byte_perm(pat(v0), pat(v1), 0x0040), __byte_perm(pat(v2), pat(v3), 0x0040), 0x5410);
+}
+
 // NHWC integer codes: one thread per (pixel, 32-channel word).  The thread reads its 32 code bytes
 // as 16-byte vectors and gathers plane j of four codes at a time into a nibble with one multiply
 // (((x >> j) & 0x01010101) * 0x01020408) >> 24, so no cross-lane traffic is needed and a warp moves
@@ -126,9 +140,7 @@ __global__ void __launch_bounds__(256) pack_acts_nhwc_f32_coalesced_kernel(const
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int chunk = i * 32 + lane;
-                regroup[warp][chunk >> 3][chunk & 7] =
-                    (uint32_t)quantize_act_code(v[i].x, inv_scale, qmax) | ((uint32_t)quantize_act_code(v[i].y, inv_scale, qmax) << 8) |
-                    ((uint32_t)quantize_act_code(v[i].z, inv_scale, qmax) << 16) | ((uint32_t)quantize_act_code(v[i].w, inv_scale, qmax) << 24);
+                regroup[warp][chunk >> 3][chunk & 7] = act_codes4(v[i].x, v[i].y, v[i].z, v[i].w, inv_scale, qmax);
             }
         }
         __syncwarp();
@@ -202,8 +214,7 @@ __global__ void __launch_bounds__(256) pack_acts_nhwc_f32_kernel(const float* __
             if (vec) {
                 if (4 * k < nvalid) {
                     const float4 v = __ldg(reinterpret_cast<const float4*>(src) + k);
-                    wv = (uint32_t)quantize_act_code(v.x, inv_scale, qmax) | ((uint32_t)quantize_act_code(v.y, inv_scale, qmax) << 8) |
-                         ((uint32_t)quantize_act_code(v.z, inv_scale, qmax) << 16) | ((uint32_t)quantize_act_code(v.w, inv_scale, qmax) << 24);
+                    wv = act_codes4(v.x, v.y, v.z, v.w, inv_scale, qmax);
                 }
             } else {
 #pragma unroll
@@ -256,17 +267,21 @@ __global__ void __launch_bounds__(128) pack_acts_nchw_kernel(const T* __restrict
 
 // NCHW fp32 with a pixel count that is a multiple of four: a CTA of 256 threads takes 32 channels x 256 pixels.  Every
 // thread issues its eight 16-byte loads (four pixels of one channel each, consecutive threads consecutive pixel quads, so
-// a warp reads 512 contiguous bytes of a channel row) before it uses any of them, quantizes, and writes the codes as
-// bytes into a pixel-major tile; one thread per pixel then builds the plane words.
+// a warp reads 512 contiguous bytes of a channel row) before it uses any of them, quantizes four channels of a pixel
+// into one word of a pixel-major tile in shared memory; one thread per pixel then builds the plane words.
 __global__ void __launch_bounds__(256) pack_acts_nchw_f32_vec_kernel(const float* __restrict__ x, int N, int C, int HW,
                                                                      int CW, int AB, float inv_scale,
                                                                      uint32_t* __restrict__ out) {
-    constexpr int PT = 256, ROWB = 36;                       // pixels per tile; bytes per pixel row (32 codes + pad)
-    __shared__ __align__(16) uint8_t tile[PT * ROWB];
+    // A thread takes 4 consecutive pixels of 8 channels: the two groups of four consecutive channels 4 cg .. 4 cg + 3
+    // and 16 + 4 cg ..  Per pixel and group its four codes are one word of the pixel's row of eight code words; the row of
+    // pixel 4 quad + j sits at word 9 quad + 584 j, which makes both the stores (lanes along quad, stride 9 words) and
+    // the row reads (lanes along pixels: 9 (t / 4) + 584 (t % 4), and 584 = 8 mod 32) free of bank conflicts.
+    constexpr int PT = 256, QP = 9, JP = 584;                // pixels per tile; word pitch along quad and along j
+    __shared__ __align__(16) uint32_t tile[4 * JP];
     const int ptiles = (HW + PT - 1) / PT;
     const long long tiles = (long long)N * CW * ptiles;
     const int qmax = (1 << AB) - 1;
-    const int quad = threadIdx.x & 63, crow = threadIdx.x >> 6;          // pixel quad 0..63, channel row 0..3 (+ 4 per step)
+    const int quad = threadIdx.x & 63, cg = threadIdx.x >> 6;            // pixel quad 0..63, channel group 0..3
     for (long long tix = blockIdx.x; tix < tiles; tix += gridDim.x) {
         const int pt = (int)(tix % ptiles);
         const long long rest = tix / ptiles;
@@ -275,23 +290,22 @@ __global__ void __launch_bounds__(256) pack_acts_nchw_f32_vec_kernel(const float
         float4 v[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const int c = cw * 32 + crow + 4 * i;
+            const int c = cw * 32 + (i >> 2) * 16 + 4 * cg + (i & 3);
             v[i] = (c < C && pp4 < HW) ? __ldg(reinterpret_cast<const float4*>(x + ((long long)n * C + c) * HW + pp4))
                                        : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int cl = crow + 4 * i;
-            uint8_t* col = tile + (4 * quad) * ROWB + cl;
-            col[0] = (uint8_t)quantize_act_code(v[i].x, inv_scale, qmax);
-            col[ROWB] = (uint8_t)quantize_act_code(v[i].y, inv_scale, qmax);
-            col[2 * ROWB] = (uint8_t)quantize_act_code(v[i].z, inv_scale, qmax);
-            col[3 * ROWB] = (uint8_t)quantize_act_code(v[i].w, inv_scale, qmax);
+        for (int gq = 0; gq < 2; ++gq) {
+            uint32_t* dst = tile + quad * QP + gq * 4 + cg;
+            dst[0] = act_codes4(v[4 * gq].x, v[4 * gq + 1].x, v[4 * gq + 2].x, v[4 * gq + 3].x, inv_scale, qmax);
+            dst[JP] = act_codes4(v[4 * gq].y, v[4 * gq + 1].y, v[4 * gq + 2].y, v[4 * gq + 3].y, inv_scale, qmax);
+            dst[2 * JP] = act_codes4(v[4 * gq].z, v[4 * gq + 1].z, v[4 * gq + 2].z, v[4 * gq + 3].z, inv_scale, qmax);
+            dst[3 * JP] = act_codes4(v[4 * gq].w, v[4 * gq + 1].w, v[4 * gq + 2].w, v[4 * gq + 3].w, inv_scale, qmax);
         }
         __syncthreads();
         const int pp = p0 + threadIdx.x;
         if (pp < HW) {
-            const uint32_t* row = reinterpret_cast<const uint32_t*>(tile + threadIdx.x * ROWB);
+            const uint32_t* row = tile + (threadIdx.x >> 2) * QP + (threadIdx.x & 3) * JP;
             uint32_t codes[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) codes[k] = row[k];
