@@ -19,9 +19,11 @@
 //    m_sub MMAs and the halo of the strip is shared.
 //  * Weights stay resident in shared memory when all (tap, word) tiles of a channel tile fit, else they
 //    stream through the stage ring by cp.async.bulk, a stage ahead of the MMAs.
-//  * Roles: warps 0-7 expand (packed words -> byte strips, global loads two chunks ahead), warp 8
-//    issues the MMAs, warp 9 fetches weight tiles, warps 10-17 run the epilogue out of tensor memory
-//    while the next tile's MMAs fill the other accumulator set.
+//  * Roles (20 warps): warps 0-7 expand (packed words -> byte strips, global loads two chunks ahead), warps 8-9
+//    issue the MMAs (two warps when a tile has an even number of accumulators: each owns the accumulators of one
+//    parity; a single warp needs 140-180 clocks per MMA and was the bound of the k x k layers), warp 10 fetches weight
+//    tiles (every lane one tile of a ring slot), warps 12-19 run the epilogue out of tensor memory while the next
+//    tile's MMAs fill the other accumulator set.
 //  * Bit <-> byte transposes with one masked merge per plane and register: with v_k = rotl(w_k, k) the
 //    byte register of channels {b, 8+b, 16+b, 24+b} is rotr(OR_k v_k & (0x01010101 << ((b+k) & 7)), b);
 //    the epilogue packs requantized codes into plane words with the mirrored identity.
@@ -36,7 +38,9 @@
 namespace ebs {
 
 constexpr int PIPE_EXPANDERS = 256;
-constexpr int PIPE_ISSUER_WARP = 8, PIPE_PRODUCER_WARP = 9, PIPE_EPI_WARP0 = 10, PIPE_EPI_WARPS = 8;
+// Warps 8 and 9 issue the MMAs, warp 10 fetches weights, warp 11 has no role (20 warps cost the same registers as 18:
+// they are allotted in fours), warps 12-19 run the epilogue.
+constexpr int PIPE_ISSUER_WARP = 8, PIPE_ISSUERS = 2, PIPE_PRODUCER_WARP = 10, PIPE_EPI_WARP0 = 12, PIPE_EPI_WARPS = 8;
 constexpr int PIPE_THREADS = (PIPE_EPI_WARP0 + PIPE_EPI_WARPS) * 32;
 constexpr int PIPE_SLOTS = 2;                      // (pixel, word) items an expander thread handles per stage
 constexpr int PIPE_MAX_ITEMS = PIPE_SLOTS * PIPE_EXPANDERS;
@@ -166,8 +170,8 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
     if (ks > 4) ks = 4;
     if (ks > p.CW) ks = p.CW;
     if (ks < 1) return g;
-    while (ks > 1 && ks * taps * m_sub >= PIPE_MAX_MMAS) --ks;     // (the issue loop reads one entry ahead)
-    if (ks * taps * m_sub >= PIPE_MAX_MMAS) return g;
+    while (ks > 1 && ks * taps * m_sub >= PIPE_MAX_MMAS - 2) --ks;     // (the issue loops read up to two entries ahead)
+    if (ks * taps * m_sub >= PIPE_MAX_MMAS - 2) return g;
     // Streamed weights go through a ring of their own (slots of a few consecutive (tap, word) tiles), so that copies are
     // in flight all the time (a stage-sized unit would leave the copy engine idle while a stage's MMAs run).
     auto stage_bytes = [&](int k) { return (k * g.a_word_bytes + 255) & ~255; };
@@ -181,7 +185,7 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
     // only every ten clocks or so, so its per-stage bookkeeping has to be spread over about a dozen MMAs.
     int nsub = 1;
     while (nsub < 4 && ks * nsub * taps * m_sub < 12 && ks * nsub < p.CW &&
-           ks * 2 * nsub * taps * m_sub < PIPE_MAX_MMAS && 3 * stage_bytes(ks * 2 * nsub) <= avail)
+           ks * 2 * nsub * taps * m_sub < PIPE_MAX_MMAS - 2 && 3 * stage_bytes(ks * 2 * nsub) <= avail)
         nsub *= 2;
     g.ks = ks;
     g.nsub = nsub;
@@ -409,10 +413,10 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
         s_tap_id[tid] = (int)g.tap_id[tid];
     }
     // Table of the MMAs of a chunk, per phase, in issue order (word, tap, accumulator): x = offset of the activation
-    // operand from the stage start (16-byte units: word, tap shift, 128 pixels per accumulator), y = accumulator column
-    // offset | (advance of the weight operand after this MMA) << 16.  The issuing thread then spends a load, three
-    // additions and the MMA per step; with operand addresses computed in its loop it was the slowest stage of the
-    // pipeline (a single thread retires an instruction every 5 to 10 clocks).
+    // operand from the stage start (16-byte units: word, tap shift, 128 pixels per accumulator) | accumulator column
+    // offset << 22, y = offset of the weight tile (16-byte units) from the chunk's first tile (resident weights) or from
+    // the start of its ring slot (streamed).  An issuing warp then spends a load, three additions and the MMA per step;
+    // with operand addresses computed in its loop it was the slowest stage of the pipeline.
     uint2* mma_tab = reinterpret_cast<uint2*>(dyn_smem + ((1024u - (smem_u32(dyn_smem) & 1023u)) & 1023u) +
                                               (g.smem_bytes - 1024 - PIPE_MAX_MMAS * 8));
     {
@@ -426,11 +430,10 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
             const int q = local / (ntp * g.m_sub), r = local - q * (ntp * g.m_sub);
             const int tl = r / g.m_sub, j = r - tl * g.m_sub;
             const uint32_t a_off = (uint32_t)(q * (g.a_word_bytes >> 4) + g.tap_shift[t0 + tl] + j * UMMA_M);
-            uint32_t b_inc = 0u;
-            if (j == g.m_sub - 1)
-                b_inc = (g.b_resident && tl == ntp - 1) ? bt16 * (uint32_t)(1 + g.taps - ntp) : bt16;
+            const uint32_t b_off = g.b_resident ? (uint32_t)(q * g.taps + tl) * bt16
+                                                : (uint32_t)((q * ntp + tl) % g.b_group) * bt16;
             if (EBS_IN_RANGE(p, CHK_PIPE_TAB, e, PIPE_MAX_MMAS))
-                mma_tab[e] = make_uint2(a_off, (uint32_t)(j * TILE_N) | (b_inc << 16));
+                mma_tab[e] = make_uint2(a_off | ((uint32_t)(j * TILE_N) << 22), b_off);
         }
     }
     const int NST = g.n_stages, KS = g.ks, KSS = g.kss, NSUB = g.nsub, SP = g.SP, S = g.S;
@@ -456,18 +459,23 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
         else { ptile = idx / g.n_ctiles; ctile = idx - ptile * g.n_ctiles; }
     };
 
+    // Issuing warps: a single warp issuing every MMA of a CTA needs 140-180 clocks per MMA (measured: its busy time, not
+    // the tensor pipe, bounded the k x k layers and the GEMM), so with two or four accumulators per tile two warps share the
+    // work, each owning the accumulators of one parity -- MMAs of different warps never touch the same accumulator, so
+    // no order between the warps is needed.  One accumulator: one issuing warp.
+    const int n_iss = (g.m_sub & 1) == 0 ? PIPE_ISSUERS : 1;
     if (tid == 0) {
         abort_flag = 0;
         for (int s = 0; s < PIPE_MAX_STAGES; ++s) {
             mbar_init(&st_full[s], (PIPE_EXPANDERS / 32) * g.nsub);  // every expander warp arrives once per pass
-            mbar_init(&st_empty[s], 1);
+            mbar_init(&st_empty[s], n_iss);                         // every issuing warp commits its own MMAs
         }
         for (int s = 0; s < PIPE_MAX_BSLOTS; ++s) {
             mbar_init(&bs_full[s], 1);
-            mbar_init(&bs_empty[s], 1);
+            mbar_init(&bs_empty[s], n_iss);
         }
-        mbar_init(&acc_full[0], 1);
-        mbar_init(&acc_full[1], 1);
+        mbar_init(&acc_full[0], n_iss);
+        mbar_init(&acc_full[1], n_iss);
         mbar_init(&acc_empty[0], PIPE_EPI_WARPS);
         mbar_init(&acc_empty[1], PIPE_EPI_WARPS);
         mbar_init(&b_full, 1);
@@ -615,8 +623,9 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 }
             }
         }
-    } else if (warp == PIPE_ISSUER_WARP) {
-        // =========================== issuer ===========================
+    } else if (warp >= PIPE_ISSUER_WARP && warp < PIPE_ISSUER_WARP + n_iss) {
+        // =========================== issuers ===========================
+        const int k_iss = warp - PIPE_ISSUER_WARP;                // this warp takes the MMAs k_iss, k_iss + n_iss, ... of a chunk
         // The issuing thread is a pipeline stage of its own: every address is advanced by additions (descriptor start
         // addresses are in 16-byte units), a handful of instructions per MMA.
         constexpr uint32_t IDESC = umma_idesc_i8(TILE_N);
@@ -652,29 +661,29 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                     const int zero_n = c == 0 ? m_sub : 0;         // the first MMA into each accumulator of a tile overwrites it
                     const uint32_t a_lo = da_lo + (uint32_t)st * stage16;
                     if (resident) {
-                        uint32_t b_lo = db_lo + (uint32_t)((wgr * KSS) * g.taps + t0) * BT16;
+                        const uint32_t b_lo = db_lo + (uint32_t)((wgr * KSS) * g.taps + t0) * BT16;
                         const int n = words * ntp * m_sub;
-                        uint2 e = tab[0];
-                        for (int i = 0; i < n; ++i) {
-                            const uint2 nxt = tab[i + 1];                 // one entry past the end is inside the table's allocation
-                            umma_i8_split(leader, tmem_d + (e.y & 0xFFFFu), a_lo + e.x, da_hi, b_lo, db_hi, IDESC, i >= zero_n ? 1u : 0u);
-                            b_lo += e.y >> 16;
+                        uint2 e = tab[k_iss];
+                        for (int i = k_iss; i < n; i += n_iss) {
+                            const uint2 nxt = tab[i + n_iss];             // (past the end: inside the table's allocation)
+                            umma_i8_split(leader, tmem_d + (e.x >> 22), a_lo + (e.x & 0x3FFFFFu), da_hi, b_lo + e.y, db_hi, IDESC,
+                                          i >= zero_n ? 1u : 0u);
                             e = nxt;
                         }
                     } else {
                         // streamed weights: the chunk's (word, tap) tiles in order, GB consecutive tiles per ring slot
                         const int ntiles = words * ntp;
-                        int i = 0;
+                        int i = k_iss;
                         for (int i0 = 0; i0 < ntiles; i0 += GB) {
                             if (!mbar_wait_bounded_hot(&bs_full[bs], bs_round & 1u, abortp, wait_limit)) { ok = false; break; }
                             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                            uint32_t b_lo = db_lo + (uint32_t)(bs * GB) * BT16;
-                            const int n = i + min(GB, ntiles - i0) * m_sub;
+                            const uint32_t b_lo = db_lo + (uint32_t)(bs * GB) * BT16;
+                            const int n = (i0 + min(GB, ntiles - i0)) * m_sub;
                             uint2 e = tab[i];
-                            for (; i < n; ++i) {
-                                const uint2 nxt = tab[i + 1];
-                                umma_i8_split(leader, tmem_d + (e.y & 0xFFFFu), a_lo + e.x, da_hi, b_lo, db_hi, IDESC, i >= zero_n ? 1u : 0u);
-                                b_lo += e.y >> 16;
+                            for (; i < n; i += n_iss) {
+                                const uint2 nxt = tab[i + n_iss];
+                                umma_i8_split(leader, tmem_d + (e.x >> 22), a_lo + (e.x & 0x3FFFFFu), da_hi, b_lo + e.y, db_hi, IDESC,
+                                              i >= zero_n ? 1u : 0u);
                                 e = nxt;
                             }
                             umma_commit_pred(leader, &bs_empty[bs]);
@@ -692,16 +701,24 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
         }
     } else if (warp == PIPE_PRODUCER_WARP) {
         // =========================== weight tiles ===========================
-        if ((tid & 31) == 0 && my_items > 0) {
+        // The whole warp runs the loops with uniform control flow and every lane issues the copy of one tile of a slot
+        // (its own address arithmetic, side by side with the other lanes'): a single lane working through the tiles one
+        // after the other retired an instruction every dozen clocks and needed about 360 clocks per tile -- more than
+        // the two MMAs that consume a 256-channel tile -- which bounded every layer whose weights stream.
+        const int lane = tid & 31;
+        if (my_items > 0) {
             if (resident) {                                      // all tiles of this CTA's channel tile, once
                 const int co0 = (int)blockIdx.y * TILE_N;
                 const uint32_t rows = (uint32_t)min(TILE_N, p.Co16 - co0);
-                mbar_arrive_expect_tx(&b_full, rows * 32u * (uint32_t)(p.CW * g.taps));
-                for (int cw = 0; cw < p.CW; ++cw)
-                    for (int ts = 0; ts < g.taps; ++ts)
-                        if (EBS_IN_RANGE(p, CHK_PIPE_W8, ((long long)(s_tap_id[ts] * p.CW + cw) * p.Co16 + co0) * 32 + rows * 32 - 1, p.lim_w8))
-                        bulk_copy_g2s(b_res + (cw * g.taps + ts) * B_TILE_BYTES,
+                const int total_tiles = p.CW * g.taps;
+                if (lane == 0) mbar_arrive_expect_tx(&b_full, rows * 32u * (uint32_t)total_tiles);
+                __syncwarp();
+                for (int t = lane; t < total_tiles; t += 32) {
+                    const int cw = t / g.taps, ts = t - cw * g.taps;
+                    if (EBS_IN_RANGE(p, CHK_PIPE_W8, ((long long)(s_tap_id[ts] * p.CW + cw) * p.Co16 + co0) * 32 + rows * 32 - 1, p.lim_w8))
+                        bulk_copy_g2s(b_res + t * B_TILE_BYTES,
                                       p.w8 + ((size_t)(s_tap_id[ts] * p.CW + cw) * p.Co16 + co0) * 32, rows * 32u, &b_full);
+                }
             } else {
                 int bs = 0;
                 uint32_t bs_round = 0;
@@ -716,23 +733,23 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                         if (++wg == nwg) { wg = 0; ++ph; }
                         const int wgr = wg + wg_rot >= nwg ? wg + wg_rot - nwg : wg + wg_rot;
                         const int words = min(KSS, p.CW - wgr * KSS);
-                        const int t0 = g.ph_tap0[ph], t1 = g.ph_tap0[ph + 1];
-                        const int ntaps = t1 - t0, ntiles = words * ntaps;
-                        int q = 0, ts = t0;
+                        const int t0 = g.ph_tap0[ph], ntaps = g.ph_tap0[ph + 1] - t0, ntiles = words * ntaps;
                         for (int i0 = 0; i0 < ntiles; i0 += GB) {
                             if (bs_round > 0) {                     // the MMAs that read this slot one round ago must be done
-                                if (!mbar_wait_bounded_hot(&bs_empty[bs], (bs_round - 1) & 1u, abortp, wait_limit)) { ok = false; break; }
+                                const bool free = mbar_wait_bounded_hot(&bs_empty[bs], (bs_round - 1) & 1u, abortp, wait_limit);
+                                if (!__all_sync(0xffffffffu, free)) { ok = false; break; }
                             }
                             const int n = min(GB, ntiles - i0);
-                            mbar_arrive_expect_tx(&bs_full[bs], bytes * (uint32_t)n);
-                            for (int i = 0; i < n; ++i) {
+                            if (lane == 0) mbar_arrive_expect_tx(&bs_full[bs], bytes * (uint32_t)n);
+                            __syncwarp();
+                            if (lane < n) {
+                                const int t = i0 + lane;                          // tile of the chunk: word-major, taps inside
+                                const int q = t / ntaps, ts = t0 + (t - q * ntaps);
+                                const size_t src = ((size_t)(s_tap_id[ts] * p.CW + wgr * KSS + q) * p.Co16 + co0) * 32;
                                 // (a copy skipped by the range-checked build leaves its barrier incomplete: the CTA then gives
                                 // up at its bounded wait, which is reported as well)
-                                if (EBS_IN_RANGE(p, CHK_PIPE_W8, ((long long)(s_tap_id[ts] * p.CW + wgr * KSS + q) * p.Co16 + co0) * 32 + bytes - 1, p.lim_w8))
-                                bulk_copy_g2s(b_res + (bs * GB + i) * B_TILE_BYTES,
-                                              p.w8 + ((size_t)(s_tap_id[ts] * p.CW + wgr * KSS + q) * p.Co16 + co0) * 32, bytes,
-                                              &bs_full[bs]);
-                                if (++ts == t1) { ts = t0; ++q; }
+                                if (EBS_IN_RANGE(p, CHK_PIPE_W8, src + bytes - 1, p.lim_w8))
+                                    bulk_copy_g2s(b_res + (bs * GB + lane) * B_TILE_BYTES, p.w8 + src, bytes, &bs_full[bs]);
                             }
                             if (++bs == NBS) { bs = 0; ++bs_round; }
                         }
@@ -740,7 +757,7 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 }
             }
         }
-    } else {
+    } else if (warp >= PIPE_EPI_WARP0) {
         // =========================== epilogue ===========================
         const int half = (warp - PIPE_EPI_WARP0) >> 2;           // which half of the channels
         const int vwarp = (warp & 3) + 4 * half;                 // TMEM lane quarter = warp % 4 (hardware rule)
