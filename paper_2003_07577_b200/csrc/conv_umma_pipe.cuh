@@ -365,6 +365,63 @@ __device__ __forceinline__ void pipe_group32(const ConvParams& p, uint32_t (&v)[
     }
 }
 
+// The same group when only packed planes are asked for (a chained network: no accumulator and no fp32 output): the
+// four channels of a byte register go from accumulator to code in one short chain, so that nothing but the 32
+// accumulators and the finished code registers is alive at a time -- the general form above keeps the 32 fp32 images
+// as well, which at 96 registers costs spills and the parallelism of the instruction stream.
+__device__ __forceinline__ void pipe_group32_packed(const uint32_t (&v)[32], bool pvalid, float S, float inv_next, int nb, int qmax,
+                                                    uint32_t* dst, const ConvParams& p) {
+    uint32_t cr[8];
+    const uint64_t S2 = f32x2_pack(S, S);
+    const uint64_t magic2 = f32x2_pack(8388608.0f, 8388608.0f);
+    const int m_lo = 0x4B000000, m_hi = 0x4B000000 + qmax;
+#pragma unroll
+    for (int bb = 0; bb < 8; ++bb) {
+        int m[4];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint64_t w = f32x2_mul_rn(f32x2_pack((float)(int)v[16 * h + bb], (float)(int)v[16 * h + 8 + bb]), S2);
+            const float t_lo = __fadd_rn(__fmul_rn(__uint_as_float((uint32_t)w), inv_next), 0.5f);
+            const float t_hi = __fadd_rn(__fmul_rn(__uint_as_float((uint32_t)(w >> 32)), inv_next), 0.5f);
+            const uint64_t t = f32x2_add_rd(f32x2_pack(t_lo, t_hi), magic2);
+            m[2 * h] = min(max((int)(uint32_t)t, m_lo), m_hi);
+            m[2 * h + 1] = min(max((int)(uint32_t)(t >> 32), m_lo), m_hi);
+        }
+        const uint32_t c4 = __byte_perm(__byte_perm((uint32_t)m[0], (uint32_t)m[1], 0x0040),
+                                        __byte_perm((uint32_t)m[2], (uint32_t)m[3], 0x0040), 0x5410);
+        cr[bb] = __funnelshift_l(c4, c4, bb);
+    }
+    uint32_t planes[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        if (j >= nb) break;
+        uint32_t t = cr[0] & (0x01010101u << (j & 7));
+#pragma unroll
+        for (int bb = 1; bb < 8; ++bb) t |= cr[bb] & (0x01010101u << ((bb + j) & 7));
+        planes[j] = __funnelshift_r(t, t, j);
+    }
+    if (pvalid && EBS_IN_RANGE(p, CHK_PIPE_PN, (dst - p.packed_next) + nb - 1, p.lim_pn)) {
+        if (nb == 4) {
+            *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
+        } else if (nb == 8) {
+            *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
+            *reinterpret_cast<uint4*>(dst + 4) = make_uint4(planes[4], planes[5], planes[6], planes[7]);
+        } else if (nb == 2) {
+            *reinterpret_cast<uint2*>(dst) = make_uint2(planes[0], planes[1]);
+        } else if (nb == 6) {
+            *reinterpret_cast<uint2*>(dst) = make_uint2(planes[0], planes[1]);
+            *reinterpret_cast<uint2*>(dst + 2) = make_uint2(planes[2], planes[3]);
+            *reinterpret_cast<uint2*>(dst + 4) = make_uint2(planes[4], planes[5]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (j >= nb) break;
+                dst[j] = planes[j];
+            }
+        }
+    }
+}
+
 // Plain epilogue (no per-channel terms, no shortcut, NHWC, whole channel tile, c_out % 4 == 0) of one
 // 128-pixel accumulator.  vwarp 0..7: TMEM lane quarter vwarp % 4, channel half vwarp / 4.
 template <int TILE_N>
@@ -387,7 +444,9 @@ __device__ __forceinline__ void pipe_epilogue_plain(const ConvParams& p, uint32_
         tmem_ld16_wait(hi);
         const size_t o = (size_t)gp * p.Co + co0 + c0;
         uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + ((co0 + c0) >> 5)) * nb;
-        if (want_q) {
+        if (want_q && !p.acc && !p.y) {
+            pipe_group32_packed(v, pvalid, S, inv_next, nb, qmax, dst, p);
+        } else if (want_q) {
             if (p.acc_small) pipe_group32<true, true>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
             else pipe_group32<true, false>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
         } else {
@@ -491,7 +550,18 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const uint32_t tmem_base = tmem_slot;
 
+    // Registers follow the roles (warpgroups of four warps: 0-7 expanders, 8-11 issuers / producer / no role, 12-19
+    // epilogue): each role's branch opens with a setmaxnreg executed by all four warps of its warpgroups, and the
+    // assembler allocates each branch for its own count.  The epilogue's 32 accumulators, their fp32 images and the code
+    // registers want about 126 registers; with the 96 a CTA of 20 warps starts with it spilled and its instruction stream
+    // lost its parallelism (wide 1x1 layers 15-20% slower, and no better with twelve epilogue warps).  The other roles
+    // need fewer than 96.  The increase waits in hardware until the CTA's pool has the registers, so the counts must fit
+    // into what the launch allots: checked at compile time.  (80 / 56 / 128 measured best of three splits.)
+    constexpr int REG_LAUNCH = 96, REG_EXP = 80, REG_MID = 56, REG_EPI = 128;
+    static_assert(8 * REG_EXP + 4 * REG_MID + 8 * REG_EPI <= 20 * REG_LAUNCH, "setmaxnreg: the roles' registers exceed the CTA's pool");
+    static_assert(PIPE_EPI_WARP0 == 12 && PIPE_EPI_WARPS == 8 && PIPE_THREADS == 640, "role layout changed: revisit the register split");
     if (warp < 8) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(REG_EXP));
         // =========================== expanders ===========================
         int slot_q[PIPE_SLOTS], slot_pix[PIPE_SLOTS], slot_dst[PIPE_SLOTS];
 #pragma unroll
@@ -623,7 +693,9 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 }
             }
         }
-    } else if (warp >= PIPE_ISSUER_WARP && warp < PIPE_ISSUER_WARP + n_iss) {
+    } else if (warp < PIPE_EPI_WARP0) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(REG_MID));
+      if (warp >= PIPE_ISSUER_WARP && warp < PIPE_ISSUER_WARP + n_iss) {
         // =========================== issuers ===========================
         const int k_iss = warp - PIPE_ISSUER_WARP;                // this warp takes the MMAs k_iss, k_iss + n_iss, ... of a chunk
         // The issuing thread is a pipeline stage of its own: every address is advanced by additions (descriptor start
@@ -757,7 +829,9 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 }
             }
         }
-    } else if (warp >= PIPE_EPI_WARP0) {
+      }
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(REG_EPI));
         // =========================== epilogue ===========================
         const int half = (warp - PIPE_EPI_WARP0) >> 2;           // which half of the channels
         const int vwarp = (warp & 3) + 4 * half;                 // TMEM lane quarter = warp % 4 (hardware rule)
