@@ -422,6 +422,107 @@ __device__ __forceinline__ void pipe_group32_packed(const uint32_t (&v)[32], boo
     }
 }
 
+// The packed-only group of a layer with per-channel terms and / or a shortcut (a folded batch normalisation, the
+// second convolution of a residual block): the same chain per byte register with the terms applied in the library's
+// order -- per-channel scale, per-channel shift, fp32 shortcut, shortcut from packed codes -- each an individually
+// rounded fp32 operation.  The shortcut codes come out of their planes with the rotate-merge of the expanders, which
+// leaves them in exactly the byte registers (channels bb, 8 + bb, 16 + bb, 24 + bb) this loop works on.  The ReLU is
+// not applied: the quantizer's clamp at zero gives the same codes.
+__device__ __forceinline__ void pipe_group32_affine(const uint32_t (&v)[32], const ConvParams& p, size_t o, int cbase, int gp,
+                                                    bool pvalid, int nb, int qmax, uint32_t* dst) {
+    const float S = p.S, inv_next = p.inv_next;
+    uint32_t rbyte[8];
+    const bool has_rp = p.res_packed != nullptr;
+    if (has_rp) {
+        const uint32_t* rw = p.res_packed + ((size_t)gp * p.CWo + (cbase >> 5)) * p.res_bits;
+        uint32_t rv[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t w = (pvalid && j < p.res_bits) ? __ldg(rw + j) : 0u;
+            rv[j] = __funnelshift_l(w, w, j);
+        }
+#pragma unroll
+        for (int bb = 0; bb < 8; ++bb) {
+            uint32_t t = rv[0] & (0x01010101u << bb);
+#pragma unroll
+            for (int j = 1; j < 8; ++j) t |= rv[j] & (0x01010101u << ((bb + j) & 7));
+            rbyte[bb] = __funnelshift_r(t, t, bb);
+        }
+    }
+    uint32_t cr[8];
+    const int m_lo = 0x4B000000, m_hi = 0x4B000000 + qmax;
+#pragma unroll
+    for (int bb = 0; bb < 8; ++bb) {
+        int m[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c = 8 * i + bb;
+            float t = __fmul_rn((float)(int)v[c], S);
+            if (p.ch_scale) t = __fmul_rn(t, __ldg(p.ch_scale + cbase + c));
+            if (p.ch_bias) t = __fadd_rn(t, __ldg(p.ch_bias + cbase + c));
+            if (p.residual && pvalid) t = __fadd_rn(t, __ldg(p.residual + o + c));
+            if (has_rp) t = __fadd_rn(t, __fmul_rn(p.res_scale, (float)((rbyte[bb] >> (8 * i)) & 0xFFu)));
+            const float u = __fadd_rn(__fmul_rn(t, inv_next), 0.5f);
+            m[i] = min(max(__float_as_int(__fadd_rd(u, 8388608.0f)), m_lo), m_hi);
+        }
+        const uint32_t c4 = __byte_perm(__byte_perm((uint32_t)m[0], (uint32_t)m[1], 0x0040),
+                                        __byte_perm((uint32_t)m[2], (uint32_t)m[3], 0x0040), 0x5410);
+        cr[bb] = __funnelshift_l(c4, c4, bb);
+    }
+    uint32_t planes[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        if (j >= nb) break;
+        uint32_t t = cr[0] & (0x01010101u << (j & 7));
+#pragma unroll
+        for (int bb = 1; bb < 8; ++bb) t |= cr[bb] & (0x01010101u << ((bb + j) & 7));
+        planes[j] = __funnelshift_r(t, t, j);
+    }
+    if (pvalid && EBS_IN_RANGE(p, CHK_PIPE_PN, (dst - p.packed_next) + nb - 1, p.lim_pn)) {
+        if (nb == 4) {
+            *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
+        } else if (nb == 8) {
+            *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
+            *reinterpret_cast<uint4*>(dst + 4) = make_uint4(planes[4], planes[5], planes[6], planes[7]);
+        } else if (nb == 2) {
+            *reinterpret_cast<uint2*>(dst) = make_uint2(planes[0], planes[1]);
+        } else if (nb == 6) {
+            *reinterpret_cast<uint2*>(dst) = make_uint2(planes[0], planes[1]);
+            *reinterpret_cast<uint2*>(dst + 2) = make_uint2(planes[2], planes[3]);
+            *reinterpret_cast<uint2*>(dst + 4) = make_uint2(planes[4], planes[5]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (j >= nb) break;
+                dst[j] = planes[j];
+            }
+        }
+    }
+}
+
+// Packed-only epilogue with per-channel terms / shortcut of one 128-pixel accumulator (whole channel tile, NHWC).
+template <int TILE_N>
+__device__ __forceinline__ void pipe_epilogue_affine(const ConvParams& p, uint32_t tmem_acc, int vwarp, int gp, bool pvalid,
+                                                     int co0) {
+    constexpr int COLS = TILE_N / 2;
+    const uint32_t trow = tmem_acc + ((uint32_t)((vwarp & 3) * 32) << 16);
+    const int cbeg = (vwarp >> 2) * COLS;
+    const int nb = p.next_bits, qmax = (1 << p.next_bits) - 1;
+    uint32_t v[32];
+#pragma unroll 1
+    for (int c0 = cbeg; c0 < cbeg + COLS; c0 += 32) {
+        uint32_t (&lo)[16] = *reinterpret_cast<uint32_t(*)[16]>(&v[0]);
+        uint32_t (&hi)[16] = *reinterpret_cast<uint32_t(*)[16]>(&v[16]);
+        tmem_ld16_issue(trow + (uint32_t)c0, lo);
+        tmem_ld16_issue(trow + (uint32_t)(c0 + 16), hi);
+        tmem_ld16_wait(lo);
+        tmem_ld16_wait(hi);
+        const size_t o = (size_t)gp * p.Co + co0 + c0;
+        uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + ((co0 + c0) >> 5)) * nb;
+        pipe_group32_affine(v, p, o, co0 + c0, gp, pvalid, nb, qmax, dst);
+    }
+}
+
 // Plain epilogue (no per-channel terms, no shortcut, NHWC, whole channel tile, c_out % 4 == 0) of one
 // 128-pixel accumulator.  vwarp 0..7: TMEM lane quarter vwarp % 4, channel half vwarp / 4.
 template <int TILE_N>
@@ -838,6 +939,8 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
         const int row = (warp & 3) * 32 + (tid & 31);
         const bool plain_ok = !AFFINE && !p.ch_scale && !p.ch_bias && !p.residual && !p.res_packed && !p.y_nchw &&
                               (p.Co & 3) == 0;
+        // layers with per-channel terms or a shortcut that only hand packed planes on (the usual layer of a network)
+        const bool affine_ok = AFFINE && p.packed_next && !p.y && !p.acc && !p.w_levels && (p.Co & 31) == 0;
         for (int it = 0; it < my_items; ++it) {
             const int buf = g.nbuf == 2 ? (it & 1) : 0;
             const int use = g.nbuf == 2 ? (it >> 1) : it;
@@ -860,6 +963,7 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 if (!__any_sync(0xffffffffu, pvalid)) continue;   // 32 frame pixels without an output
                 const uint32_t tmem_acc = tmem_base + (uint32_t)((buf * g.m_sub + j) * TILE_N);
                 if (plain_ok && co0 + TILE_N <= p.Co) pipe_epilogue_plain<TILE_N>(p, tmem_acc, vwarp, gp, pvalid, co0);
+                else if (affine_ok && co0 + TILE_N <= p.Co) pipe_epilogue_affine<TILE_N>(p, tmem_acc, vwarp, gp, pvalid, co0);
                 else umma_epilogue<TILE_N, AFFINE>(p, tmem_acc, vwarp, gp, pvalid, 0, co0);
             }
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
