@@ -154,6 +154,33 @@ __global__ void __launch_bounds__(256) pack_acts_nhwc_f32_coalesced_kernel(const
     }
 }
 
+// Integer codes, channels a multiple of 32, 32-byte aligned tensor: a thread reads the 32 code bytes of its items with one
+// 256-bit load each (a warp instruction reads 1 KB of consecutive memory: no regrouping through shared memory is needed)
+// and builds the plane words.  UNROLL items per thread are loaded before any is used.
+template <int UNROLL>
+__global__ void __launch_bounds__(256) pack_acts_nhwc_u8_v8_kernel(const uint8_t* __restrict__ x, long long items, int AB,
+                                                                   uint32_t* __restrict__ out) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long item0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; item0 < items; item0 += stride * UNROLL) {
+        uint32_t codes[UNROLL][8];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const long long item = item0 + u * stride;
+            if (item < items) {
+                asm volatile("ld.global.nc.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                             : "=r"(codes[u][0]), "=r"(codes[u][1]), "=r"(codes[u][2]), "=r"(codes[u][3]), "=r"(codes[u][4]),
+                               "=r"(codes[u][5]), "=r"(codes[u][6]), "=r"(codes[u][7])
+                             : "l"(x + item * 32));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const long long item = item0 + u * stride;
+            if (item < items) store_planes(codes[u], AB, out + item * AB);
+        }
+    }
+}
+
 // Same for integer codes; a warp takes 128 items (4 KB) per iteration so that enough loads are in flight.
 __global__ void __launch_bounds__(256) pack_acts_nhwc_u8_coalesced_kernel(const uint8_t* __restrict__ x, long long items,
                                                                           int AB, uint32_t* __restrict__ out) {
@@ -383,7 +410,11 @@ int launch_pack_acts(const void* x, int dtype, int layout, int n, int c, int h, 
             if (wblocks > (long long)sms * 32) wblocks = (long long)sms * 32;
             if (dtype == EBS_F32)
                 pack_acts_nhwc_f32_coalesced_kernel<<<(int)wblocks, 256, 0, st>>>((const float*)x, items, a_bits, inv_scale, out);
-            else {
+            else if ((reinterpret_cast<uintptr_t>(x) & 31u) == 0) {
+                long long vblocks = (items + 256 * 4 - 1) / (256 * 4);
+                if (vblocks > (long long)sms * 16) vblocks = (long long)sms * 16;
+                pack_acts_nhwc_u8_v8_kernel<4><<<(int)vblocks, 256, 0, st>>>((const uint8_t*)x, items, a_bits, out);
+            } else {
                 long long ublocks = ((items + 127) / 128 + 7) / 8;
                 if (ublocks > (long long)sms * 16) ublocks = (long long)sms * 16;
                 pack_acts_nhwc_u8_coalesced_kernel<<<(int)ublocks, 256, 0, st>>>((const uint8_t*)x, items, a_bits, out);
