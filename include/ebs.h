@@ -163,6 +163,22 @@ int ebs_pack_acts(const void *x_dev, int dtype, int layout, int n, int c, int h,
                   float a_scale, void *packed_x_dev, void *stream);
 
 /*
+ * Space-to-depth packing for a stride-2 first layer with few input channels (the paper has no counterpart: it leaves
+ * the first layer unquantized; networks run it at 8 bits through this library).  x_dev: u8 codes, NHWC [n][h][w][c],
+ * device memory, 4 * c <= 32, h and w even.  Output: bit planes in the packed activation layout of a tensor
+ * [n][hs][ws] with 4 * c channels, hs = (h + offset) / 2 + offset (likewise ws): pixel (i, j) holds the 2 x 2 block of
+ * input pixels (2 i - offset + dy, 2 j - offset + dx), dy, dx in {0, 1}, as channel (2 dy + dx) * c + ch; positions
+ * outside the image are code 0.  A k x k, stride-2, pad-p convolution (k odd) over x equals a ((k + 1) / 2)-square,
+ * stride-1, pad-((p - offset) / 2) convolution over this tensor with offset = p mod 2 and the weights regrouped as
+ * w2[co][(2 dy + dx) * c + ch][bi][bj] = w[co][ch][2 bi + dy][2 bj + dx] (zero where 2 bi + dy or 2 bj + dx reaches
+ * k): a quarter of the reduction words, four times as full.  packed_x_dev: ebs_packed_act_bytes(n, hs, ws, 4 * c,
+ * a_bits) bytes, 16-byte aligned, caller-owned.  Asynchronous on `stream`.  Returns EBS_ERR_UNSUPPORTED for 4 * c > 32
+ * or odd h / w, EBS_ERR_INVALID_ARG for null pointers, sizes <= 0, a_bits outside 1..8, offset outside {0, 1}.
+ */
+int ebs_pack_acts_s2d(const void* x_dev, int n, int c, int h, int w, int offset, int a_bits, void* packed_x_dev,
+                      void* stream);
+
+/*
  * The mixed-precision convolution by binary decomposition (Eq. 13-14): for every output
  * (n, ho, wo, co)
  *   acc = sum_{m<M} sum_{k<K} c_m 2^(m+k) * sum_{taps, channel words} popcount(A_k AND W_m),

@@ -30,7 +30,7 @@ EXPORTS = [
     "ebs_search_act_forward", "ebs_expected_flops", "ebs_fused_plan_upload", "ebs_resnet_cifar_forward", "ebs_noalloc_scratch_bytes", "ebs_conv2d_mixed_host_noalloc",
     "ebs_conv_variant_family", "ebs_conv_variant_applies", "ebs_check_device_status", "ebs_test_set_device_wait",
     "ebs_conv2d_i8", "ebs_maxpool_packed", "ebs_combined_scale", "ebs_reciprocal_step",
-    "ebs_checked_build", "ebs_checked_status", "ebs_test_checked_shrink",
+    "ebs_checked_build", "ebs_checked_status", "ebs_test_checked_shrink", "ebs_pack_acts_s2d",
 ]
 
 
@@ -110,6 +110,7 @@ def lib() -> ctypes.CDLL:
         L.ebs_checked_status.argtypes = [ctypes.POINTER(i), ctypes.POINTER(ctypes.c_longlong),
                                          ctypes.POINTER(ctypes.c_longlong), i]
         L.ebs_test_checked_shrink.argtypes = [ctypes.c_longlong]
+        L.ebs_pack_acts_s2d.argtypes = [p, i, i, i, i, i, i, p, p]
         L.ebs_conv_variant_family.argtypes = [i]
         L.ebs_conv_variant_family.restype = ctypes.c_char_p
         L.ebs_conv_variant_applies.argtypes = [D, i, i, i, E, i, i, i, i]
@@ -331,6 +332,11 @@ def ebs_checked_status(clear: bool = True):
     if rc < 0:
         _check(rc, "ebs_checked_status")
     return bool(rc), site.value, index.value, limit.value
+
+
+def ebs_pack_acts_s2d(x_dev, n, c, h, w, offset, a_bits, packed_x_dev, stream=None) -> None:
+    _check(lib().ebs_pack_acts_s2d(_ptr(x_dev), int(n), int(c), int(h), int(w), int(offset), int(a_bits),
+                                   _ptr(packed_x_dev), _stream(stream)), "ebs_pack_acts_s2d")
 
 
 def ebs_test_checked_shrink(elements: int) -> None:

@@ -428,6 +428,17 @@ int ebs_pack_acts(const void* x_dev, int dtype, int layout, int n, int c, int h,
                             static_cast<cudaStream_t>(stream));
 }
 
+int ebs_pack_acts_s2d(const void* x_dev, int n, int c, int h, int w, int offset, int a_bits, void* packed_x_dev,
+                      void* stream) {
+    if (!x_dev || !packed_x_dev || n <= 0 || c <= 0 || h <= 0 || w <= 0) return EBS_ERR_INVALID_ARG;
+    if (a_bits < 1 || a_bits > 8 || (offset != 0 && offset != 1)) return EBS_ERR_INVALID_ARG;
+    if (4 * c > 32 || (h & 1) || (w & 1)) return EBS_ERR_UNSUPPORTED;
+    if (!aligned16(packed_x_dev)) return EBS_ERR_INVALID_ARG;
+    if (h > 32000 || w > 32000 || (long long)n * h * w >= (1LL << 31)) return EBS_ERR_OVERFLOW;
+    return launch_pack_acts_s2d(x_dev, n, c, h, w, offset, a_bits, static_cast<uint32_t*>(packed_x_dev),
+                                static_cast<cudaStream_t>(stream));
+}
+
 int ebs_conv2d_mixed(const void* packed_x_dev, int n, int h, int w, const void* packed_w_dev,
                      const ebs_conv_desc* desc, const ebs_epilogue* epi, int32_t* acc_out_dev, float* y_out_dev,
                      void* packed_next_dev, void* stream) {

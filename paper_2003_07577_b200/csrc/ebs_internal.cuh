@@ -131,6 +131,7 @@ EBS_DECLARE_WB(5) EBS_DECLARE_WB(6) EBS_DECLARE_WB(7) EBS_DECLARE_WB(8)
 #undef EBS_DECLARE_WB
 
 // pack.cu
+int launch_pack_acts_s2d(const void* x, int n, int c, int h, int w, int off, int a_bits, uint32_t* out, cudaStream_t st);
 int launch_pack_acts(const void* x, int dtype, int layout, int n, int c, int h, int w, int a_bits,
                      float inv_scale, uint32_t* out, cudaStream_t st);
 int launch_pack_weights(const void* wt, int dtype, int layout, const ebs_conv_desc& d, float inv_scale,

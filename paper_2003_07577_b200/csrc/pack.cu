@@ -342,6 +342,41 @@ __global__ void __launch_bounds__(256) pack_acts_nchw_f32_vec_kernel(const float
     }
 }
 
+// Space-to-depth packing for a stride-2 first layer with few channels (u8 NHWC codes, 4 * C <= 32): output pixel (i, j)
+// of the [N][Hs][Ws] tensor holds the 2 x 2 block of input pixels (2i - off + dy, 2j - off + dx), channel slot
+// (2 dy + dx) * C + c, zero outside the image; off = 1 shifts the blocks by one pixel so that an odd padding of the
+// original convolution becomes a whole number of blocks.  A k x k stride-2 convolution over the image is then a
+// ceil(k/2) x ceil(k/2) stride-1 convolution over this tensor with the weights regrouped the same way: its reduction
+// words are a quarter as many and four times as full.  One thread per output pixel.
+__global__ void __launch_bounds__(256) pack_acts_s2d_u8_kernel(const uint8_t* __restrict__ x, int N, int C, int H, int W, int Hs,
+                                                               int Ws, int off, int AB, uint32_t* __restrict__ out) {
+    const long long total = (long long)N * Hs * Ws;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const uint32_t code_mask = (1u << AB) - 1u;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += stride) {
+        const int j = (int)(t % Ws);
+        const long long r = t / Ws;
+        const int i = (int)(r % Hs), n = (int)(r / Hs);
+        uint32_t codes[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int dy = 0; dy < 2; ++dy) {
+            const int h = 2 * i - off + dy;
+            if ((unsigned)h >= (unsigned)H) continue;
+#pragma unroll
+            for (int dx = 0; dx < 2; ++dx) {
+                const int w = 2 * j - off + dx;
+                if ((unsigned)w >= (unsigned)W) continue;
+                const uint8_t* src = x + (((long long)n * H + h) * W + w) * C;
+                for (int c = 0; c < C; ++c) {
+                    const int slot = (2 * dy + dx) * C + c;
+                    codes[slot >> 2] |= ((uint32_t)__ldg(src + c) & code_mask) << (8 * (slot & 3));
+                }
+            }
+        }
+        store_planes(codes, AB, out + t * AB);
+    }
+}
+
 // Weights: one warp per (tap, channel word, output channel); tiny and off the inference path.
 template <typename T>
 __global__ void __launch_bounds__(256) pack_weights_kernel(const T* __restrict__ wt, int layout, int Co, int C,
@@ -391,6 +426,17 @@ static int sm_count() {
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
     return n > 0 ? n : 148;
 }
+
+int launch_pack_acts_s2d(const void* x, int n, int c, int h, int w, int off, int a_bits, uint32_t* out, cudaStream_t st) {
+    const int Hs = (h + off) / 2 + off, Ws = (w + off) / 2 + off;
+    const long long total = (long long)n * Hs * Ws;
+    long long blocks = (total + 255) / 256;
+    const long long cap = (long long)sm_count() * 32;
+    if (blocks > cap) blocks = cap;
+    pack_acts_s2d_u8_kernel<<<(int)blocks, 256, 0, st>>>((const uint8_t*)x, n, c, h, w, Hs, Ws, off, a_bits, out);
+    return check_cuda(cudaGetLastError());
+}
+
 
 int launch_pack_acts(const void* x, int dtype, int layout, int n, int c, int h, int w, int a_bits,
                      float inv_scale, uint32_t* out, cudaStream_t st) {

@@ -37,6 +37,47 @@ class ConvPlan:
     ch_scale: Optional[torch.Tensor] = None
     out_bits: int = 0             # bitwidth of the packed output (0: fp32 output only)
     out_step: float = 0.0         # quantization step of the packed output
+    # first layer in space-to-depth form (space_to_depth_stem): block offset, and the image the packing reads
+    s2d_offset: int = -1
+    src_c: int = 0
+    src_h: int = 0
+    src_w: int = 0
+
+
+def space_to_depth_weights(weight_codes: torch.Tensor) -> torch.Tensor:
+    """[c_out, c, k, k] -> [c_out, 4 c, ceil(k/2), ceil(k/2)]: w2[co][(2 dy + dx) c + ch][bi][bj] = w[co][ch][2 bi + dy][2 bj + dx],
+    zero where 2 bi + dy or 2 bj + dx reaches k (slices only)."""
+    co, c, k, _ = weight_codes.shape
+    k2 = (k + 1) // 2
+    w2 = torch.zeros((co, 4 * c, k2, k2), dtype=weight_codes.dtype, device=weight_codes.device)
+    for dy in (0, 1):
+        for dx in (0, 1):
+            sub = weight_codes[:, :, dy::2, dx::2]
+            w2[:, (2 * dy + dx) * c:(2 * dy + dx + 1) * c, :sub.shape[2], :sub.shape[3]] = sub
+    return w2.contiguous()
+
+
+def space_to_depth_stem(plan: ConvPlan, weight_codes: torch.Tensor) -> ConvPlan:
+    """The first layer of an ImageNet network (k x k, k odd, stride 2, few input channels, even image sides) as the
+    equivalent stride-1 layer over the space-to-depth image that ebs_pack_acts_s2d writes: ceil(k/2)-square kernel, four
+    times the channels, weights regrouped as w2[co][(2 dy + dx) c + ch][bi][bj] = w[co][ch][2 bi + dy][2 bj + dx]
+    (slices of the code tensor: no arithmetic).  Returns `plan` itself when the layer does not have that shape.
+    weight_codes: int8 [c_out, c_in, k, k] on the device."""
+    d = plan.desc
+    c, k = d.c_in, d.kh
+    if not (plan.role == "first" and d.kh == d.kw and k % 2 == 1 and d.stride_h == 2 and d.stride_w == 2 and
+            d.pad_h == d.pad_w and 4 * c <= 32 and plan.h_in % 2 == 0 and plan.w_in % 2 == 0):
+        return plan
+    off, k2 = d.pad_h & 1, (k + 1) // 2
+    pb = (d.pad_h - off) // 2
+    hs, ws = (plan.h_in + off) // 2 + off, (plan.w_in + off) // 2 + off
+    w2 = space_to_depth_weights(weight_codes)
+    d2 = ebs.conv_desc(4 * c, d.c_out, k2, k2, 1, 1, pb, pb, d.w_bits, d.a_bits, d.w_scale, d.a_scale)
+    assert ebs.ebs_conv_out_shape(d2, hs, ws) == ebs.ebs_conv_out_shape(d, plan.h_in, plan.w_in)
+    pw2 = torch.empty(ebs.ebs_packed_weight_bytes(d2) // 4, dtype=torch.int32, device=weight_codes.device)
+    ebs.ebs_pack_weights(w2, ebs.EBS_I8_CODES, ebs.EBS_NCHW, d2, pw2)
+    return ConvPlan(plan.name, plan.role, d2, hs, ws, pw2, plan.ch_bias, plan.ch_scale, plan.out_bits, plan.out_step,
+                    s2d_offset=off, src_c=c, src_h=plan.h_in, src_w=plan.w_in)
 
 
 class BasicBlockNet:
@@ -86,8 +127,11 @@ class BasicBlockNet:
         n = images_u8_nhwc.shape[0]
         f = self.first
         px = self._planes(("input", "q"), n, f.h_in, f.w_in, f.desc.c_in, 8)
-        ebs.ebs_pack_acts(images_u8_nhwc, ebs.EBS_U8_CODES, ebs.EBS_NHWC, n, f.desc.c_in, f.h_in, f.w_in, 8, 1.0, px,
-                          stream=stream)
+        if f.s2d_offset >= 0:                                    # stride-2 first layer in space-to-depth form
+            ebs.ebs_pack_acts_s2d(images_u8_nhwc, n, f.src_c, f.src_h, f.src_w, f.s2d_offset, 8, px, stream=stream)
+        else:
+            ebs.ebs_pack_acts(images_u8_nhwc, ebs.EBS_U8_CODES, ebs.EBS_NHWC, n, f.desc.c_in, f.h_in, f.w_in, 8, 1.0, px,
+                              stream=stream)
         _, x, ho1, wo1 = self._conv(f, px, n, stream=stream)
         x_bits, x_step = f.out_bits, f.out_step
         if self.pool is not None:                                # on the packed codes; bits and step are unchanged
@@ -122,7 +166,8 @@ class BasicBlockNet:
         return 2 + len(self.plans) + 1 + (1 if self.pool is not None else 0)
 
 
-def calibrated_plans(layers, weight_codes, images_u8_nhwc: torch.Tensor, device=None, pool=None) -> List[ConvPlan]:
+def calibrated_plans(layers, weight_codes, images_u8_nhwc: torch.Tensor, device=None, pool=None,
+                     stem_s2d: bool = True) -> List[ConvPlan]:
     """Builds the per-layer plans of a basic-block network from integer weight codes.
 
     ``layers``: records with name, role, c_in, c_out, k, stride, pad, h_in, w_in, w_bits, a_bits,
@@ -196,7 +241,10 @@ def calibrated_plans(layers, weight_codes, images_u8_nhwc: torch.Tensor, device=
     ebs.ebs_pack_acts(pooled, ebs.EBS_F32, ebs.EBS_NHWC, n, c_last, 1, 1, fc.a_bits, s_fc, pq)
     run(fc, pq, s_fc, 0, relu=False)
     torch.cuda.synchronize(device)
-    return [plans[L.name] for L in layers]
+    out = [plans[L.name] for L in layers]
+    if stem_s2d:
+        out[0] = space_to_depth_stem(out[0], weight_codes[first.name])
+    return out
 
 
 class FusedBasicBlockNet:

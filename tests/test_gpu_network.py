@@ -141,8 +141,8 @@ def _oracle_network(oracle, gen, specs, imgs, sample, pool=None):
     return plan, trace, logits.reshape(len(sample), -1), qp
 
 
-def _gpu_network(ebs, U, gen, specs, plan, pool=None):
-    from paper_2003_07577_b200.network import BasicBlockNet, ConvPlan
+def _gpu_network(ebs, U, gen, specs, plan, pool=None, stem_s2d=False):
+    from paper_2003_07577_b200.network import BasicBlockNet, ConvPlan, space_to_depth_stem
     plans = []
     for spec in specs:
         L, pl = spec.layer, plan[spec.layer.name]
@@ -150,6 +150,10 @@ def _gpu_network(ebs, U, gen, specs, plan, pool=None):
                           spec.w_scale, pl["a_scale"])
         plans.append(ConvPlan(L.name, L.role, d, L.h_in, L.w_in, U.pack_weight_codes(gen.weight_codes(spec), d),
                               ch_bias=_to(pl["bias"], U), ch_scale=_to(pl["scale"], U), out_bits=pl["out_bits"], out_step=pl["out_step"]))
+    if stem_s2d:
+        converted = space_to_depth_stem(plans[0], _to(gen.weight_codes(specs[0]).astype(np.int8), U))
+        assert converted.s2d_offset >= 0, "the first layer did not qualify for the space-to-depth form"
+        plans[0] = converted
     return BasicBlockNet(plans, U.dev(), pool=pool)
 
 
@@ -227,6 +231,49 @@ def test_fused_network_plan_is_validated(ebs, U):
             ebs.ebs_fused_plan_upload([bad], dev)
 
 
+def _space_to_depth(x, off):
+    """numpy form of the block layout: [N, C, H, W] -> [N, 4 C, Hs, Ws], channel (2 dy + dx) C + c of block (i, j) =
+    pixel (2 i - off + dy, 2 j - off + dx), zero outside."""
+    n, c, h, w = x.shape
+    hs, ws = (h + off) // 2 + off, (w + off) // 2 + off
+    out = np.zeros((n, 4 * c, hs, ws), dtype=x.dtype)
+    for dy in (0, 1):
+        for dx in (0, 1):
+            for i in range(hs):
+                hh = 2 * i - off + dy
+                if not 0 <= hh < h:
+                    continue
+                for j in range(ws):
+                    ww = 2 * j - off + dx
+                    if 0 <= ww < w:
+                        out[:, (2 * dy + dx) * c:(2 * dy + dx + 1) * c, i, j] = x[:, :, hh, ww]
+    return out
+
+
+@pytest.mark.parametrize("n,c,h,w,off,bits", [(2, 3, 16, 12, 1, 8), (1, 3, 8, 8, 0, 8), (3, 8, 10, 14, 1, 4), (2, 1, 6, 6, 0, 1),
+                                              (1, 5, 12, 10, 1, 6)])
+def test_space_to_depth_packing(ebs, U, oracle, n, c, h, w, off, bits):
+    """ebs_pack_acts_s2d against the block layout written out in numpy, packed by the oracle."""
+    rng = np.random.default_rng(n * 100 + c)
+    x = rng.integers(0, 1 << bits, size=(n, c, h, w), dtype=np.int32)
+    ref = _space_to_depth(x, off)
+    hs, ws = ref.shape[2], ref.shape[3]
+    xd = _to(x.astype(np.uint8).transpose(0, 2, 3, 1), U)
+    out = torch.zeros(ebs.ebs_packed_act_bytes(n, hs, ws, 4 * c, bits) // 4, dtype=torch.int32, device=U.dev())
+    ebs.ebs_pack_acts_s2d(xd, n, c, h, w, off, bits, out)
+    torch.cuda.synchronize()
+    got = oracle.unpack_acts(U.packed_images(out, n, hs, ws, 4 * c, bits, list(range(n))), 4 * c)
+    assert np.array_equal(got, ref)
+
+
+def test_space_to_depth_argument_checks(ebs, U):
+    x = torch.zeros((1, 8, 8, 3), dtype=torch.uint8, device=U.dev())
+    out = torch.zeros(4096, dtype=torch.int32, device=U.dev())
+    for args in [(1, 9, 8, 8, 1, 8), (1, 3, 7, 8, 1, 8), (1, 3, 8, 8, 2, 8), (1, 3, 8, 8, 1, 9), (0, 3, 8, 8, 1, 8)]:
+        with pytest.raises(ebs.EbsError):
+            ebs.ebs_pack_acts_s2d(x, *args, out)
+
+
 @pytest.mark.parametrize("bits,c,h,w,k,s,p", [(4, 64, 15, 14, 3, 2, 1), (1, 32, 8, 8, 2, 2, 0), (8, 70, 9, 11, 3, 1, 1),
                                               (3, 96, 7, 7, 3, 2, 0), (5, 33, 6, 5, 1, 1, 0), (7, 64, 12, 12, 3, 2, 1)])
 def test_maxpool_on_packed_planes(ebs, U, oracle, bits, c, h, w, k, s, p):
@@ -254,10 +301,14 @@ def test_resnet18_imagenet_forward_matches_the_oracle(ebs, U, oracle, gen):
     assert specs[0].layer.role == "first" and specs[0].layer.k == 7 and specs[-1].layer.role == "fc"
     imgs = gen.images_u8(0, n, 224, 224)
     plan, trace, logits_ref, qp_ref = _oracle_network(oracle, gen, specs, imgs, sample, pool=pool)
-    net = _gpu_network(ebs, U, gen, specs, plan, pool=pool)
     x = _to(imgs.astype(np.uint8).transpose(0, 2, 3, 1), U)
+    # the first layer as given (7x7 stride 2 over the image) and in its space-to-depth form (4x4 stride 1 over 2x2 pixel
+    # blocks): the same codes, so the same logits
+    logits_plain = _gpu_network(ebs, U, gen, specs, plan, pool=pool).forward(x).clone()
+    net = _gpu_network(ebs, U, gen, specs, plan, pool=pool, stem_s2d=True)
     logits = net.forward(x)
     torch.cuda.synchronize()
+    assert torch.equal(logits, logits_plain)
     first = specs[0].layer
     got = oracle.unpack_acts(U.packed_images(net._buf[("maxpool", "q")], n, 56, 56, first.c_out, plan["conv1"]["out_bits"],
                                              sample), first.c_out)

@@ -491,3 +491,31 @@ def test_maxpool_codes_pins(oracle):
     one = np.array([[[[1, 5], [7, 2]]]], np.int32)
     assert np.array_equal(oracle.maxpool_codes(one, 3, 2, 1), np.array([[[[7]]]], np.int32))      # one window sees all
     assert np.array_equal(oracle.maxpool_codes(one, 2, 1, 1), np.array([[[[1, 5, 5], [7, 7, 5], [7, 7, 2]]]], np.int32))
+
+
+
+@pytest.mark.parametrize("c,k,pad,h,w", [(3, 7, 3, 12, 10), (3, 5, 2, 8, 8), (2, 3, 1, 6, 8), (4, 3, 0, 8, 6), (1, 7, 2, 10, 10)])
+def test_stride2_first_layer_equals_its_space_to_depth_form(oracle, c, k, pad, h, w):
+    """A k x k stride-2 convolution equals the ceil(k/2)-square stride-1 convolution over 2 x 2 pixel blocks with the
+    weights regrouped the same way (the form the network runner gives an ImageNet stem): both evaluated by the oracle's
+    direct definition.  The block layout is written out here; the weight regrouping is the runner's own function."""
+    import torch
+    from paper_2003_07577_b200.network import space_to_depth_weights
+    rng = np.random.default_rng(k * 10 + pad)
+    x = rng.integers(0, 256, size=(2, c, h, w), dtype=np.int32)
+    wt = rng.integers(-128, 128, size=(5, c, k, k), dtype=np.int32)
+    ref = oracle.conv2d_codes(x, wt, (2, 2), (pad, pad))
+    off, pb = pad & 1, (pad - (pad & 1)) // 2
+    hs, ws = (h + off) // 2 + off, (w + off) // 2 + off
+    xs = np.zeros((2, 4 * c, hs, ws), dtype=np.int32)
+    for dy in (0, 1):
+        for dx in (0, 1):
+            for i in range(hs):
+                for j in range(ws):
+                    hh, ww = 2 * i - off + dy, 2 * j - off + dx
+                    if 0 <= hh < h and 0 <= ww < w:
+                        xs[:, (2 * dy + dx) * c:(2 * dy + dx + 1) * c, i, j] = x[:, :, hh, ww]
+    w2 = space_to_depth_weights(torch.from_numpy(wt)).numpy()
+    assert w2.shape == (5, 4 * c, (k + 1) // 2, (k + 1) // 2)
+    got = oracle.conv2d_codes(xs, w2, (1, 1), (pb, pb))
+    assert got.shape == ref.shape and np.array_equal(got, ref)
