@@ -61,10 +61,11 @@ def run_checked(args, timeout):
 
 def test_kernel_parity_tests_pass_on_the_range_checked_library(checked_library):
     """The small parity cases of every kernel family (all variants that apply, odd sizes, strides, padding, shortcut
-    forms) on the checked library: results identical to the oracle and, after every test, an empty record
-    (tests/conftest.py checks it when EBS_LIBRARY=checked)."""
+    forms) and the whole-network runs (per-channel terms, shortcuts, pooling, the space-to-depth first layer) on the
+    checked library: results identical to the oracle and, after every test, an empty record (tests/conftest.py checks
+    it when EBS_LIBRARY=checked)."""
     res = run_checked(["-m", "pytest", "-x", "-q", "-m", "gpu", "tests/test_gpu_parity.py", "tests/test_gpu_pipe.py",
-                       "-p", "no:cacheprovider"], timeout=1500)
+                       "tests/test_gpu_network.py", "-p", "no:cacheprovider"], timeout=1500)
     assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
 
 
