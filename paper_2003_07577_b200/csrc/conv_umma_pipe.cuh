@@ -365,12 +365,83 @@ __device__ __forceinline__ void pipe_group32(const ConvParams& p, uint32_t (&v)[
     }
 }
 
+// Plane words of consecutive 32-channel groups of one pixel, held back until their run can leave in wide stores.  A
+// group's nb plane words are contiguous in memory, but for an odd nb their start is only 4-byte aligned and 32 lanes
+// each storing nb single words scatter 32 sectors per instruction (the wide 1x1 layers of a chain were up to 1.7 times
+// slower with nb = 7 than with nb = 8).  A warp handles G consecutive groups of its pixel (G = 4 for the 256-channel tile, 2
+// for the 128-channel one): their G * nb words are one contiguous run that starts on a 4 * G-byte boundary, stored as nb
+// vectors of G words.  The hold is a shift register (static indices only); last = the run's last group.
+template <int G>
+struct PlaneHold {
+    uint32_t w[G > 1 ? G : 1][8];
+    int filled;
+};
+template <int NB, int G>
+__device__ __forceinline__ void pipe_store_run(const uint32_t (&w)[G][8], uint32_t* run) {
+    static_assert(G == 2 || G == 4, "two or four groups to a run");
+#pragma unroll
+    for (int t = 0; t < NB; ++t) {                       // vector t = words G t .. G t + G - 1 of the run; word i = group i / NB, plane i % NB
+        if constexpr (G == 4)
+            *reinterpret_cast<uint4*>(run + 4 * t) = make_uint4(w[(4 * t) / NB][(4 * t) % NB], w[(4 * t + 1) / NB][(4 * t + 1) % NB],
+                                                                 w[(4 * t + 2) / NB][(4 * t + 2) % NB], w[(4 * t + 3) / NB][(4 * t + 3) % NB]);
+        else
+            *reinterpret_cast<uint2*>(run + 2 * t) = make_uint2(w[(2 * t) / NB][(2 * t) % NB], w[(2 * t + 1) / NB][(2 * t + 1) % NB]);
+    }
+}
+template <int G>
+__device__ __forceinline__ void pipe_store_planes(const uint32_t (&planes)[8], int nb, uint32_t* dst, bool pvalid, PlaneHold<G>& hold,
+                                                  const ConvParams& p) {
+    if constexpr (G > 1) {
+        if ((nb & 1) && (p.CWo % G) == 0) {               // odd: hold the group; store the run with its last group (rows of
+                                                          // CWo * nb words keep the run's alignment only if G divides CWo)
+#pragma unroll
+            for (int gi = 0; gi + 1 < G; ++gi)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) hold.w[gi][j] = hold.w[gi + 1][j];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) hold.w[G - 1][j] = planes[j];
+            if (++hold.filled == G) {
+                hold.filled = 0;
+                uint32_t* run = dst - (G - 1) * nb;          // the first group of the run
+                if (pvalid && EBS_IN_RANGE(p, CHK_PIPE_PN, (dst - p.packed_next) + nb - 1, p.lim_pn)) {
+                    if (nb == 7) pipe_store_run<7, G>(hold.w, run);
+                    else if (nb == 5) pipe_store_run<5, G>(hold.w, run);
+                    else if (nb == 3) pipe_store_run<3, G>(hold.w, run);
+                    else pipe_store_run<1, G>(hold.w, run);
+                }
+            }
+            return;
+        }
+    }
+    if (pvalid && EBS_IN_RANGE(p, CHK_PIPE_PN, (dst - p.packed_next) + nb - 1, p.lim_pn)) {
+        if (nb == 4) {
+            *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
+        } else if (nb == 8) {
+            *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
+            *reinterpret_cast<uint4*>(dst + 4) = make_uint4(planes[4], planes[5], planes[6], planes[7]);
+        } else if (nb == 2) {
+            *reinterpret_cast<uint2*>(dst) = make_uint2(planes[0], planes[1]);
+        } else if (nb == 6) {
+            *reinterpret_cast<uint2*>(dst) = make_uint2(planes[0], planes[1]);
+            *reinterpret_cast<uint2*>(dst + 2) = make_uint2(planes[2], planes[3]);
+            *reinterpret_cast<uint2*>(dst + 4) = make_uint2(planes[4], planes[5]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (j >= nb) break;
+                dst[j] = planes[j];
+            }
+        }
+    }
+}
+
 // The same group when only packed planes are asked for (a chained network: no accumulator and no fp32 output): the
 // four channels of a byte register go from accumulator to code in one short chain, so that nothing but the 32
 // accumulators and the finished code registers is alive at a time -- the general form above keeps the 32 fp32 images
 // as well, which at 96 registers costs spills and the parallelism of the instruction stream.
+template <int G>
 __device__ __forceinline__ void pipe_group32_packed(const uint32_t (&v)[32], bool pvalid, float S, float inv_next, int nb, int qmax,
-                                                    uint32_t* dst, const ConvParams& p) {
+                                                    uint32_t* dst, const ConvParams& p, PlaneHold<G>& hold) {
     uint32_t cr[8];
     const uint64_t S2 = f32x2_pack(S, S);
     const uint64_t magic2 = f32x2_pack(8388608.0f, 8388608.0f);
@@ -400,26 +471,7 @@ __device__ __forceinline__ void pipe_group32_packed(const uint32_t (&v)[32], boo
         for (int bb = 1; bb < 8; ++bb) t |= cr[bb] & (0x01010101u << ((bb + j) & 7));
         planes[j] = __funnelshift_r(t, t, j);
     }
-    if (pvalid && EBS_IN_RANGE(p, CHK_PIPE_PN, (dst - p.packed_next) + nb - 1, p.lim_pn)) {
-        if (nb == 4) {
-            *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
-        } else if (nb == 8) {
-            *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
-            *reinterpret_cast<uint4*>(dst + 4) = make_uint4(planes[4], planes[5], planes[6], planes[7]);
-        } else if (nb == 2) {
-            *reinterpret_cast<uint2*>(dst) = make_uint2(planes[0], planes[1]);
-        } else if (nb == 6) {
-            *reinterpret_cast<uint2*>(dst) = make_uint2(planes[0], planes[1]);
-            *reinterpret_cast<uint2*>(dst + 2) = make_uint2(planes[2], planes[3]);
-            *reinterpret_cast<uint2*>(dst + 4) = make_uint2(planes[4], planes[5]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if (j >= nb) break;
-                dst[j] = planes[j];
-            }
-        }
-    }
+    pipe_store_planes(planes, nb, dst, pvalid, hold, p);
 }
 
 // The packed-only group of a layer with per-channel terms and / or a shortcut (a folded batch normalisation, the
@@ -428,8 +480,9 @@ __device__ __forceinline__ void pipe_group32_packed(const uint32_t (&v)[32], boo
 // rounded fp32 operation.  The shortcut codes come out of their planes with the rotate-merge of the expanders, which
 // leaves them in exactly the byte registers (channels bb, 8 + bb, 16 + bb, 24 + bb) this loop works on.  The ReLU is
 // not applied: the quantizer's clamp at zero gives the same codes.
+template <int G>
 __device__ __forceinline__ void pipe_group32_affine(const uint32_t (&v)[32], const ConvParams& p, size_t o, int cbase, int gp,
-                                                    bool pvalid, int nb, int qmax, uint32_t* dst) {
+                                                    bool pvalid, int nb, int qmax, uint32_t* dst, PlaneHold<G>& hold) {
     const float S = p.S, inv_next = p.inv_next;
     uint32_t rbyte[8];
     const bool has_rp = p.res_packed != nullptr;
@@ -478,37 +531,20 @@ __device__ __forceinline__ void pipe_group32_affine(const uint32_t (&v)[32], con
         for (int bb = 1; bb < 8; ++bb) t |= cr[bb] & (0x01010101u << ((bb + j) & 7));
         planes[j] = __funnelshift_r(t, t, j);
     }
-    if (pvalid && EBS_IN_RANGE(p, CHK_PIPE_PN, (dst - p.packed_next) + nb - 1, p.lim_pn)) {
-        if (nb == 4) {
-            *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
-        } else if (nb == 8) {
-            *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
-            *reinterpret_cast<uint4*>(dst + 4) = make_uint4(planes[4], planes[5], planes[6], planes[7]);
-        } else if (nb == 2) {
-            *reinterpret_cast<uint2*>(dst) = make_uint2(planes[0], planes[1]);
-        } else if (nb == 6) {
-            *reinterpret_cast<uint2*>(dst) = make_uint2(planes[0], planes[1]);
-            *reinterpret_cast<uint2*>(dst + 2) = make_uint2(planes[2], planes[3]);
-            *reinterpret_cast<uint2*>(dst + 4) = make_uint2(planes[4], planes[5]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if (j >= nb) break;
-                dst[j] = planes[j];
-            }
-        }
-    }
+    pipe_store_planes(planes, nb, dst, pvalid, hold, p);
 }
 
 // Packed-only epilogue with per-channel terms / shortcut of one 128-pixel accumulator (whole channel tile, NHWC).
-template <int TILE_N>
-__device__ __forceinline__ void pipe_epilogue_affine(const ConvParams& p, uint32_t tmem_acc, int vwarp, int gp, bool pvalid,
-                                                     int co0) {
+template <int TILE_N, int G>
+__device__ __forceinline__ void pipe_epilogue_affine_g(const ConvParams& p, uint32_t tmem_acc, int vwarp, int gp, bool pvalid,
+                                                       int co0) {
     constexpr int COLS = TILE_N / 2;
     const uint32_t trow = tmem_acc + ((uint32_t)((vwarp & 3) * 32) << 16);
     const int cbeg = (vwarp >> 2) * COLS;
     const int nb = p.next_bits, qmax = (1 << p.next_bits) - 1;
     uint32_t v[32];
+    PlaneHold<G> hold;
+    hold.filled = 0;
 #pragma unroll 1
     for (int c0 = cbeg; c0 < cbeg + COLS; c0 += 32) {
         uint32_t (&lo)[16] = *reinterpret_cast<uint32_t(*)[16]>(&v[0]);
@@ -519,15 +555,15 @@ __device__ __forceinline__ void pipe_epilogue_affine(const ConvParams& p, uint32
         tmem_ld16_wait(hi);
         const size_t o = (size_t)gp * p.Co + co0 + c0;
         uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + ((co0 + c0) >> 5)) * nb;
-        pipe_group32_affine(v, p, o, co0 + c0, gp, pvalid, nb, qmax, dst);
+        pipe_group32_affine(v, p, o, co0 + c0, gp, pvalid, nb, qmax, dst, hold);
     }
 }
 
 // Plain epilogue (no per-channel terms, no shortcut, NHWC, whole channel tile, c_out % 4 == 0) of one
 // 128-pixel accumulator.  vwarp 0..7: TMEM lane quarter vwarp % 4, channel half vwarp / 4.
-template <int TILE_N>
-__device__ __forceinline__ void pipe_epilogue_plain(const ConvParams& p, uint32_t tmem_acc, int vwarp, int gp, bool pvalid,
-                                                    int co0) {
+template <int TILE_N, int G>
+__device__ __forceinline__ void pipe_epilogue_plain_g(const ConvParams& p, uint32_t tmem_acc, int vwarp, int gp, bool pvalid,
+                                                      int co0) {
     constexpr int COLS = TILE_N / 2;
     const uint32_t trow = tmem_acc + ((uint32_t)((vwarp & 3) * 32) << 16);
     const int cbeg = (vwarp >> 2) * COLS;
@@ -535,6 +571,8 @@ __device__ __forceinline__ void pipe_epilogue_plain(const ConvParams& p, uint32_
     const int nb = want_q ? p.next_bits : 0, qmax = (1 << p.next_bits) - 1;
     const float S = p.S, inv_next = p.inv_next;
     uint32_t v[32];
+    PlaneHold<G> hold;
+    hold.filled = 0;
 #pragma unroll 1
     for (int c0 = cbeg; c0 < cbeg + COLS; c0 += 32) {
         uint32_t (&lo)[16] = *reinterpret_cast<uint32_t(*)[16]>(&v[0]);
@@ -546,7 +584,7 @@ __device__ __forceinline__ void pipe_epilogue_plain(const ConvParams& p, uint32_
         const size_t o = (size_t)gp * p.Co + co0 + c0;
         uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + ((co0 + c0) >> 5)) * nb;
         if (want_q && !p.acc && !p.y) {
-            pipe_group32_packed(v, pvalid, S, inv_next, nb, qmax, dst, p);
+            pipe_group32_packed(v, pvalid, S, inv_next, nb, qmax, dst, p, hold);
         } else if (want_q) {
             if (p.acc_small) pipe_group32<true, true>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
             else pipe_group32<true, false>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
@@ -556,8 +594,19 @@ __device__ __forceinline__ void pipe_epilogue_plain(const ConvParams& p, uint32_
     }
 }
 
-template <int AB, int TILE_N, bool AFFINE>
+// Odd plane counts of the packed output take the form that holds the groups of a run back: a kernel instantiation of
+// its own (HOLD), chosen by the launcher, because the shift register costs the other layers registers and time even
+// as an untaken branch of the same kernel (even counts 15-25% slower when both forms were compiled into one kernel).
+inline bool pipe_hold_applies(const ConvParams& p, int tile_n) {
+    const int G = tile_n / 64;
+    // (5 and 7 planes; with 1 or 3 the single-word stores are few and the held form measured slower)
+    return G > 1 && p.packed_next && (p.next_bits == 5 || p.next_bits == 7) && (p.CWo % G) == 0 && !p.acc && !p.y && !p.y_nchw &&
+           (p.Co & 31) == 0 && !p.w_levels;
+}
+
+template <int AB, int TILE_N, bool AFFINE, bool HOLD>
 __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const ConvParams p, const PipeGeom g) {
+    constexpr int EPI_G = HOLD ? TILE_N / 64 : 1;              // groups of an output run held back (odd plane counts)
     constexpr int B_TILE_BYTES = TILE_N * 32;
     extern __shared__ uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t st_full[PIPE_MAX_STAGES], st_empty[PIPE_MAX_STAGES], acc_full[2], acc_empty[2], b_full;
@@ -962,8 +1011,8 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 }
                 if (!__any_sync(0xffffffffu, pvalid)) continue;   // 32 frame pixels without an output
                 const uint32_t tmem_acc = tmem_base + (uint32_t)((buf * g.m_sub + j) * TILE_N);
-                if (plain_ok && co0 + TILE_N <= p.Co) pipe_epilogue_plain<TILE_N>(p, tmem_acc, vwarp, gp, pvalid, co0);
-                else if (affine_ok && co0 + TILE_N <= p.Co) pipe_epilogue_affine<TILE_N>(p, tmem_acc, vwarp, gp, pvalid, co0);
+                if (plain_ok && co0 + TILE_N <= p.Co) pipe_epilogue_plain_g<TILE_N, EPI_G>(p, tmem_acc, vwarp, gp, pvalid, co0);
+                else if (affine_ok && co0 + TILE_N <= p.Co) pipe_epilogue_affine_g<TILE_N, EPI_G>(p, tmem_acc, vwarp, gp, pvalid, co0);
                 else umma_epilogue<TILE_N, AFFINE>(p, tmem_acc, vwarp, gp, pvalid, 0, co0);
             }
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
@@ -988,24 +1037,32 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
 
 int pipe_sm_count();
 
-template <int AB, int TILE_N>
-int launch_conv_umma_pipe(const ConvParams& p, dim3 /*grid*/, cudaStream_t st) {
-    const PipeGeom g = pipe_geometry(p, TILE_N, pipe_sm_count(), p.pipe_m_sub);
-    if (!g.ok) return EBS_ERR_UNSUPPORTED;                    // the geometry does not apply: nothing is launched
+template <int AB, int TILE_N, bool HOLD>
+int launch_conv_umma_pipe_form(const ConvParams& p, const PipeGeom& g, cudaStream_t st) {
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaFuncSetAttribute(conv_umma_pipe_kernel<AB, TILE_N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE_SMEM_MAX);
-        cudaFuncSetAttribute(conv_umma_pipe_kernel<AB, TILE_N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE_SMEM_MAX);
+        cudaFuncSetAttribute(conv_umma_pipe_kernel<AB, TILE_N, false, HOLD>, cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE_SMEM_MAX);
+        cudaFuncSetAttribute(conv_umma_pipe_kernel<AB, TILE_N, true, HOLD>, cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE_SMEM_MAX);
         attr_set[dev] = true;
     }
     const dim3 grid((unsigned)g.grid_x, (unsigned)g.grid_y, 1);
     if (p.ch_scale || p.ch_bias || p.residual || p.res_packed)
-        conv_umma_pipe_kernel<AB, TILE_N, true><<<grid, PIPE_THREADS, g.smem_bytes, st>>>(p, g);
+        conv_umma_pipe_kernel<AB, TILE_N, true, HOLD><<<grid, PIPE_THREADS, g.smem_bytes, st>>>(p, g);
     else
-        conv_umma_pipe_kernel<AB, TILE_N, false><<<grid, PIPE_THREADS, g.smem_bytes, st>>>(p, g);
+        conv_umma_pipe_kernel<AB, TILE_N, false, HOLD><<<grid, PIPE_THREADS, g.smem_bytes, st>>>(p, g);
     return EBS_OK;
+}
+
+template <int AB, int TILE_N>
+int launch_conv_umma_pipe(const ConvParams& p, dim3 /*grid*/, cudaStream_t st) {
+    const PipeGeom g = pipe_geometry(p, TILE_N, pipe_sm_count(), p.pipe_m_sub);
+    if (!g.ok) return EBS_ERR_UNSUPPORTED;                    // the geometry does not apply: nothing is launched
+    if constexpr (TILE_N >= 128) {
+        if (pipe_hold_applies(p, TILE_N)) return launch_conv_umma_pipe_form<AB, TILE_N, true>(p, g, st);
+    }
+    return launch_conv_umma_pipe_form<AB, TILE_N, false>(p, g, st);
 }
 
 constexpr int NUM_UMMA_PIPE_VARIANTS = 3;          // TILE_N = 64, 128, 256
