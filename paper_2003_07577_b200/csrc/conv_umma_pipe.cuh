@@ -594,9 +594,41 @@ __device__ __forceinline__ void pipe_epilogue_plain_g(const ConvParams& p, uint3
     }
 }
 
+// Packed-only epilogue without per-channel terms of one 128-pixel accumulator (whole channel tile): nothing but the lean
+// group, for the kernel forms that are launched only for such layers.
+template <int TILE_N, int G>
+__device__ __forceinline__ void pipe_epilogue_packed_g(const ConvParams& p, uint32_t tmem_acc, int vwarp, int gp, bool pvalid,
+                                                       int co0) {
+    constexpr int COLS = TILE_N / 2;
+    const uint32_t trow = tmem_acc + ((uint32_t)((vwarp & 3) * 32) << 16);
+    const int cbeg = (vwarp >> 2) * COLS;
+    const int nb = p.next_bits, qmax = (1 << p.next_bits) - 1;
+    const float S = p.S, inv_next = p.inv_next;
+    uint32_t v[32];
+    PlaneHold<G> hold;
+    hold.filled = 0;
+#pragma unroll 1
+    for (int c0 = cbeg; c0 < cbeg + COLS; c0 += 32) {
+        uint32_t (&lo)[16] = *reinterpret_cast<uint32_t(*)[16]>(&v[0]);
+        uint32_t (&hi)[16] = *reinterpret_cast<uint32_t(*)[16]>(&v[16]);
+        tmem_ld16_issue(trow + (uint32_t)c0, lo);
+        tmem_ld16_issue(trow + (uint32_t)(c0 + 16), hi);
+        tmem_ld16_wait(lo);
+        tmem_ld16_wait(hi);
+        uint32_t* dst = p.packed_next + ((size_t)gp * p.CWo + ((co0 + c0) >> 5)) * nb;
+        pipe_group32_packed(v, pvalid, S, inv_next, nb, qmax, dst, p, hold);
+    }
+}
+
 // Odd plane counts of the packed output take the form that holds the groups of a run back: a kernel instantiation of
 // its own (HOLD), chosen by the launcher, because the shift register costs the other layers registers and time even
 // as an untaken branch of the same kernel (even counts 15-25% slower when both forms were compiled into one kernel).
+// Kernel form for a layer: 0 = every output mode and ragged channel tiles; 1 = packed planes only, whole channel tiles
+// (the usual layer of a network: its epilogue holds nothing but the lean group, or the group with per-channel terms);
+// 2 = form 1 with the held-back runs.
+inline bool pipe_packed_only(const ConvParams& p, int tile_n) {
+    return p.packed_next && !p.acc && !p.y && !p.w_levels && (p.Co % tile_n) == 0;
+}
 inline bool pipe_hold_applies(const ConvParams& p, int tile_n) {
     const int G = tile_n / 64;
     // (5 and 7 planes; with 1 or 3 the single-word stores are few and the held form measured slower)
@@ -604,9 +636,9 @@ inline bool pipe_hold_applies(const ConvParams& p, int tile_n) {
            (p.Co & 31) == 0 && !p.w_levels;
 }
 
-template <int AB, int TILE_N, bool AFFINE, bool HOLD>
+template <int AB, int TILE_N, bool AFFINE, int FORM>
 __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const ConvParams p, const PipeGeom g) {
-    constexpr int EPI_G = HOLD ? TILE_N / 64 : 1;              // groups of an output run held back (odd plane counts)
+    constexpr int EPI_G = FORM == 2 ? TILE_N / 64 : 1;         // groups of an output run held back (odd plane counts)
     constexpr int B_TILE_BYTES = TILE_N * 32;
     extern __shared__ uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t st_full[PIPE_MAX_STAGES], st_empty[PIPE_MAX_STAGES], acc_full[2], acc_empty[2], b_full;
@@ -1011,9 +1043,14 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 }
                 if (!__any_sync(0xffffffffu, pvalid)) continue;   // 32 frame pixels without an output
                 const uint32_t tmem_acc = tmem_base + (uint32_t)((buf * g.m_sub + j) * TILE_N);
-                if (plain_ok && co0 + TILE_N <= p.Co) pipe_epilogue_plain_g<TILE_N, EPI_G>(p, tmem_acc, vwarp, gp, pvalid, co0);
-                else if (affine_ok && co0 + TILE_N <= p.Co) pipe_epilogue_affine_g<TILE_N, EPI_G>(p, tmem_acc, vwarp, gp, pvalid, co0);
-                else umma_epilogue<TILE_N, AFFINE>(p, tmem_acc, vwarp, gp, pvalid, 0, co0);
+                if constexpr (FORM != 0) {
+                    if constexpr (AFFINE) pipe_epilogue_affine_g<TILE_N, EPI_G>(p, tmem_acc, vwarp, gp, pvalid, co0);
+                    else pipe_epilogue_packed_g<TILE_N, EPI_G>(p, tmem_acc, vwarp, gp, pvalid, co0);
+                } else {
+                    if (plain_ok && co0 + TILE_N <= p.Co) pipe_epilogue_plain_g<TILE_N, 1>(p, tmem_acc, vwarp, gp, pvalid, co0);
+                    else if (affine_ok && co0 + TILE_N <= p.Co) pipe_epilogue_affine_g<TILE_N, 1>(p, tmem_acc, vwarp, gp, pvalid, co0);
+                    else umma_epilogue<TILE_N, AFFINE>(p, tmem_acc, vwarp, gp, pvalid, 0, co0);
+                }
             }
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
             __syncwarp();
@@ -1037,7 +1074,7 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
 
 int pipe_sm_count();
 
-template <int AB, int TILE_N, bool HOLD>
+template <int AB, int TILE_N, int HOLD>
 int launch_conv_umma_pipe_form(const ConvParams& p, const PipeGeom& g, cudaStream_t st) {
     static bool attr_set[64] = {};
     int dev = 0;
@@ -1059,10 +1096,13 @@ template <int AB, int TILE_N>
 int launch_conv_umma_pipe(const ConvParams& p, dim3 /*grid*/, cudaStream_t st) {
     const PipeGeom g = pipe_geometry(p, TILE_N, pipe_sm_count(), p.pipe_m_sub);
     if (!g.ok) return EBS_ERR_UNSUPPORTED;                    // the geometry does not apply: nothing is launched
-    if constexpr (TILE_N >= 128) {
-        if (pipe_hold_applies(p, TILE_N)) return launch_conv_umma_pipe_form<AB, TILE_N, true>(p, g, st);
+    if (pipe_packed_only(p, TILE_N)) {
+        if constexpr (TILE_N >= 128) {
+            if (pipe_hold_applies(p, TILE_N)) return launch_conv_umma_pipe_form<AB, TILE_N, 2>(p, g, st);
+        }
+        return launch_conv_umma_pipe_form<AB, TILE_N, 1>(p, g, st);
     }
-    return launch_conv_umma_pipe_form<AB, TILE_N, false>(p, g, st);
+    return launch_conv_umma_pipe_form<AB, TILE_N, 0>(p, g, st);
 }
 
 constexpr int NUM_UMMA_PIPE_VARIANTS = 3;          // TILE_N = 64, 128, 256
