@@ -273,7 +273,7 @@ __device__ __forceinline__ uint64_t f32x2_add_rd(uint64_t a, uint64_t b) {
 // The float -> int conversion issues at an eighth of the fp32 rate on this machine (16 results per clock and SM against
 // 128 fp32 operations) and was what bounded the epilogue, so the floor and the clamp are done with an fp32 addition and
 // integer min / max instead (see below); the fp32 steps run as packed two-lane instructions.
-template <bool WANT_Q, bool SMALL_ACC>
+template <bool WANT_Q>
 __device__ __forceinline__ void pipe_group32(const ConvParams& p, uint32_t (&v)[32], size_t o, bool pvalid, float S,
                                              float inv_next, int nb, int qmax, uint32_t* dst) {
     if (p.acc && pvalid && EBS_IN_RANGE(p, CHK_PIPE_ACC, o + 31, p.lim_out)) {
@@ -586,10 +586,9 @@ __device__ __forceinline__ void pipe_epilogue_plain_g(const ConvParams& p, uint3
         if (want_q && !p.acc && !p.y) {
             pipe_group32_packed(v, pvalid, S, inv_next, nb, qmax, dst, p, hold);
         } else if (want_q) {
-            if (p.acc_small) pipe_group32<true, true>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
-            else pipe_group32<true, false>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
+            pipe_group32<true>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
         } else {
-            pipe_group32<false, false>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
+            pipe_group32<false>(p, v, o, pvalid, S, inv_next, nb, qmax, dst);
         }
     }
 }
