@@ -59,13 +59,12 @@ def run_checked(args, timeout):
     return subprocess.run([sys.executable] + args, capture_output=True, text=True, env=env, cwd=ROOT, timeout=timeout)
 
 
-def test_kernel_parity_tests_pass_on_the_range_checked_library(checked_library):
-    """The small parity cases of every kernel family (all variants that apply, odd sizes, strides, padding, shortcut
-    forms) and the whole-network runs (per-channel terms, shortcuts, pooling, the space-to-depth first layer) on the
-    checked library: results identical to the oracle and, after every test, an empty record (tests/conftest.py checks
-    it when EBS_LIBRARY=checked)."""
-    res = run_checked(["-m", "pytest", "-x", "-q", "-m", "gpu", "tests/test_gpu_parity.py", "tests/test_gpu_pipe.py",
-                       "tests/test_gpu_network.py", "-p", "no:cacheprovider"], timeout=1500)
+def test_the_gpu_suite_passes_on_the_range_checked_library(checked_library):
+    """Every GPU test of the repository (all kernel families and variants, odd sizes, strides, paddings, shortcut forms,
+    the full-size configurations, the whole-network runs, the host calls) on the checked library: results identical to
+    the oracle and, after every test, an empty record (tests/conftest.py checks it when EBS_LIBRARY=checked)."""
+    res = run_checked(["-m", "pytest", "-x", "-q", "-m", "gpu", "tests", "--deselect", "tests/test_gpu_checked_build.py",
+                       "-p", "no:cacheprovider"], timeout=1800)
     assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
 
 
