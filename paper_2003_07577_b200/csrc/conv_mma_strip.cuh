@@ -112,47 +112,77 @@ conv_mma_strip_kernel(const ConvParams p) {
     const int n0 = f0 / (Hp * Wp), rem0 = f0 - n0 * (Hp * Wp);
     const int hp0 = rem0 / Wp, wq0 = rem0 - hp0 * Wp;
     const float rcp_w = __frcp_rn((float)Wp), rcp_h = __frcp_rn((float)Hp), rcp_cw = __frcp_rn((float)p.CW);
+    // Two items per thread and round: both items' packed words are requested before either is used, so a strip of up
+    // to 2 * NTH (pixel, word) items costs one round trip to memory, not two (the small layers this kernel serves are
+    // a few microseconds long: a second dependent load is a tenth of that).
+    constexpr int PF = 2;
+    const int n_items = S * p.CW;
 #pragma unroll 1
-    for (int e = tid; e < S * p.CW; e += NTH) {
-        const int s = COMPACT ? e : small_div(e, rcp_cw), cw = COMPACT ? 0 : e - s * p.CW;
-        const int f = f0 + s;
-        uint32_t r[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};          // COMPACT uses r[0..3]: the four 4-channel words
-        int gp = -1;
-        if (f < frame) {
-            const int cw_ = small_div(wq0 + s, rcp_w), wq = wq0 + s - cw_ * Wp;      // column, carry into the row
-            const int ch_ = small_div(hp0 + cw_, rcp_h), hp = hp0 + cw_ - ch_ * Hp;  // row, carry into the image
-            const int n = n0 + ch_;
-            if (hp < p.Ho && wq < p.Wo) gp = (n * p.Ho + hp) * p.Wo + wq;            // the output pixel of this frame row
-            const int h = pointwise ? hp * p.sh : hp - p.ph, w = pointwise ? wq * p.sw : wq - p.pw;
-            if ((unsigned)h < (unsigned)p.H && (unsigned)w < (unsigned)p.W &&
-                EBS_IN_RANGE(p, CHK_MS_X, (((long long)(n * p.H + h) * p.W + w) * p.CW + cw) * AB + AB - 1, p.lim_x)) {
-                uint32_t words[AB];
-                load_words_global<AB>(p.x + (((size_t)(n * p.H + h) * p.W + w) * p.CW + cw) * AB, words);
+    for (int e0 = tid; e0 < n_items; e0 += PF * NTH) {
+        uint32_t words[PF][AB];
+        int s_[PF], cw_[PF], gp_[PF];
+#pragma unroll
+        for (int u = 0; u < PF; ++u) {
+            const int e = e0 + u * NTH;
+            s_[u] = -1;
+            cw_[u] = 0;
+            gp_[u] = -1;
+#pragma unroll
+            for (int k = 0; k < AB; ++k) words[u][k] = 0u;
+            if (e >= n_items) continue;
+            const int s = COMPACT ? e : small_div(e, rcp_cw), cw = COMPACT ? 0 : e - s * p.CW;
+            s_[u] = s;
+            cw_[u] = cw;
+            const int f = f0 + s;
+            if (f < frame) {
+                const int cwq = small_div(wq0 + s, rcp_w), wq = wq0 + s - cwq * Wp;      // column, carry into the row
+                const int chq = small_div(hp0 + cwq, rcp_h), hp = hp0 + cwq - chq * Hp;  // row, carry into the image
+                const int n = n0 + chq;
+                if (hp < p.Ho && wq < p.Wo) gp_[u] = (n * p.Ho + hp) * p.Wo + wq;        // the output pixel of this frame row
+                const int h = pointwise ? hp * p.sh : hp - p.ph, w = pointwise ? wq * p.sw : wq - p.pw;
+                if ((unsigned)h < (unsigned)p.H && (unsigned)w < (unsigned)p.W &&
+                    EBS_IN_RANGE(p, CHK_MS_X, (((long long)(n * p.H + h) * p.W + w) * p.CW + cw) * AB + AB - 1, p.lim_x))
+                    load_words_global<AB>(p.x + (((size_t)(n * p.H + h) * p.W + w) * p.CW + cw) * AB, words[u]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < PF; ++u) {
+            const int s = s_[u], cw = cw_[u];
+            if (s < 0) continue;
+            uint32_t r[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};          // COMPACT uses r[0..3]: the four 4-channel words
+            if constexpr (COMPACT) {
 #pragma unroll
                 for (int k = 0; k < AB; ++k) {
                     const uint32_t mask = 0x01010101u << k;
-                    if constexpr (COMPACT) {
-                        // bits 0-3 / 8-11 / 4-7 / 12-15 of the word to the low nibbles of bytes 0 / 1 / 2 / 3, then bit j
-                        // of every byte to bit k of word j: bytes = channels j, 8+j, 4+j, 12+j
-                        const uint32_t u = (words[k] & 0x0F0Fu) | ((words[k] & 0xF0F0u) << 12);
+                    // bits 0-3 / 8-11 / 4-7 / 12-15 of the word to the low nibbles of bytes 0 / 1 / 2 / 3, then bit j
+                    // of every byte to bit k of word j: bytes = channels j, 8+j, 4+j, 12+j
+                    const uint32_t u4 = (words[u][k] & 0x0F0Fu) | ((words[u][k] & 0xF0F0u) << 12);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) r[j] |= __funnelshift_r(u, u, j - k) & mask;
-                    } else {
+                    for (int j = 0; j < 4; ++j) r[j] |= __funnelshift_r(u4, u4, j - k) & mask;
+                }
+            } else {
+                // v_k = rotl(w_k, k); byte register b = rotr(OR_k v_k & (0x01010101 << ((b + k) & 7)), b)
+                uint32_t v[AB];
 #pragma unroll
-                        for (int b = 0; b < 8; ++b) r[b] |= __funnelshift_r(words[k], words[k], b - k) & mask;
-                    }
+                for (int k = 0; k < AB; ++k) v[k] = __funnelshift_l(words[u][k], words[u][k], k);
+#pragma unroll
+                for (int b8 = 0; b8 < 8; ++b8) {
+                    uint32_t t = v[0] & (0x01010101u << b8);
+#pragma unroll
+                    for (int k = 1; k < AB; ++k) t |= v[k] & (0x01010101u << ((b8 + k) & 7));
+                    r[b8] = __funnelshift_r(t, t, b8);
                 }
             }
-        }
-        if (cw == 0 && s < TILE_P) gp_s[s] = gp;
-        if (!EBS_IN_RANGE(p, CHK_MS_STRIP, COMPACT ? s * 16 + 15 : (cw * SP + s) * 32 + 31, COMPACT ? SP * 16 : p.CW * SP * 32)) continue;
-        if constexpr (COMPACT) {
-            reinterpret_cast<uint4*>(strip)[s] = make_uint4(r[0], r[1], r[2], r[3]);
-        } else {
-            uint4* dst = reinterpret_cast<uint4*>(strip + (cw * SP + s) * 32);
-            const int sw = (s >> 2) & 1;
-            dst[sw] = make_uint4(r[0], r[1], r[2], r[3]);
-            dst[sw ^ 1] = make_uint4(r[4], r[5], r[6], r[7]);
+            if (cw == 0 && s < TILE_P) gp_s[s] = gp_[u];
+            if (!EBS_IN_RANGE(p, CHK_MS_STRIP, COMPACT ? s * 16 + 15 : (cw * SP + s) * 32 + 31, COMPACT ? SP * 16 : p.CW * SP * 32)) continue;
+            if constexpr (COMPACT) {
+                reinterpret_cast<uint4*>(strip)[s] = make_uint4(r[0], r[1], r[2], r[3]);
+            } else {
+                uint4* dst = reinterpret_cast<uint4*>(strip + (cw * SP + s) * 32);
+                const int sw = (s >> 2) & 1;
+                dst[sw] = make_uint4(r[0], r[1], r[2], r[3]);
+                dst[sw ^ 1] = make_uint4(r[4], r[5], r[6], r[7]);
+            }
         }
     }
     cp_async_wait<0>();
@@ -175,7 +205,7 @@ conv_mma_strip_kernel(const ConvParams p) {
         const int arow0 = (wp_ * MT) * 16 + g;
         for (int cw = 0; cw < p.CW; ++cw) {
             const uint8_t* strip_w = strip + cw * SP * 32;
-#pragma unroll 1
+#pragma unroll 3           // (three taps' fragment loads in flight; nine made the ResNet-20 step 8% slower: code size)
             for (int t0 = 0; t0 < taps; t0 += FOLD) {
                 uint32_t af[MT][4], bf[NT][2];
 #pragma unroll
