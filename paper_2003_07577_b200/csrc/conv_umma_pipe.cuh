@@ -161,7 +161,7 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
     g.n_ptiles = (int)((frame + g.tile_pix - 1) / g.tile_pix);
     g.S = g.tile_pix + max_shift;
     g.SP = (g.S + 7) & ~7;
-    g.a_word_bytes = g.SP * 32 + 32;
+    g.a_word_bytes = g.SP * 32 + 64;                           // sized with the largest skew; fixed once ks is known
     if (g.SP * 16 >= (1 << 18)) return g;
     // weights resident when they leave room for at least two activation stages
     const int budget = PIPE_SMEM_MAX - 2048 - PIPE_MAX_MMAS * 8;   // the MMA table sits behind the rings
@@ -187,6 +187,9 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
     while (nsub < 4 && ks * nsub * taps * m_sub < 12 && ks * nsub < p.CW &&
            ks * 2 * nsub * taps * m_sub < PIPE_MAX_MMAS - 2 && 3 * stage_bytes(ks * 2 * nsub) <= avail)
         nsub *= 2;
+    // Skew between the word tiles of a pass: the 8 lanes of a quarter warp store 16 bytes each for ks words of 8 / ks
+    // pixels; a skew of 128 / ks bytes (48 for three words) puts them on eight different 16-byte bank groups.
+    g.a_word_bytes = g.SP * 32 + (ks == 4 ? 32 : ks == 3 ? 48 : 64);
     g.ks = ks;
     g.nsub = nsub;
     g.kss = ks * nsub;
@@ -220,6 +223,94 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
     }
     g.ok = g.n_stages >= 2 && g.smem_bytes <= PIPE_SMEM_MAX && g.grid_y <= 65535 && g.n_ctiles <= 65535;
     return g;
+}
+
+// NW plane words of one (pixel, 32-channel word) item -> eight registers of four channel bytes (row byte 4b + i = channel
+// 8i + b).  With v_k = rotl(w_k, k), register b is rotr(t_b, b) where byte position (b + k) & 7 of t_b holds plane k.  The
+// eight t_b pick the planes in eight cyclic orders, and orders that agree modulo 2 (modulo 4) share their pairs (quads)
+// of planes: one bit-select per pair and parity, one per quad and residue, one per register - 24 selects for eight
+// planes where a merge per (register, plane) takes 64.
+__device__ __forceinline__ uint32_t bit_select(uint32_t a, uint32_t b, uint32_t m) { return (a & m) | (b & ~m); }
+
+template <int NW>
+__device__ __forceinline__ void planes_to_bytes(const uint32_t (&w)[NW], uint32_t (&r)[8]) {
+    uint32_t v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v[k] = k < NW ? __funnelshift_l(w[k < NW ? k : 0], w[k < NW ? k : 0], k) : 0u;
+    if constexpr (NW == 1) {
+#pragma unroll
+        for (int bb = 0; bb < 8; ++bb) {
+            const uint32_t t = v[0] & (0x01010101u << bb);
+            r[bb] = __funnelshift_r(t, t, bb);
+        }
+    } else {
+        // pairs: plane 2j on the even bit positions and plane 2j + 1 on the odd ones (parity 0), or the reverse
+        uint32_t pr[4][2];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            pr[j][0] = bit_select(v[2 * j], v[2 * j + 1], 0x55555555u);
+            pr[j][1] = bit_select(v[2 * j + 1], v[2 * j], 0x55555555u);
+        }
+        if constexpr (NW == 2) {
+#pragma unroll
+            for (int bb = 0; bb < 8; ++bb) {
+                const uint32_t t = pr[0][bb & 1] & ((0x01010101u << bb) | (0x01010101u << ((bb + 1) & 7)));
+                r[bb] = __funnelshift_r(t, t, bb);
+            }
+        } else {
+            // quads: the pair 2i on the positions = c, c + 1 (mod 4), the pair 2i + 1 on the other two
+            uint32_t qd[2][4];
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t m2 = c == 0 ? 0x33333333u : c == 1 ? 0x66666666u : c == 2 ? 0xCCCCCCCCu : 0x99999999u;
+                    qd[i][c] = bit_select(pr[2 * i][c & 1], pr[2 * i + 1][c & 1], m2);
+                }
+#pragma unroll
+            for (int bb = 0; bb < 8; ++bb) {
+                const uint32_t m3 = 0x01010101u * (uint32_t)(((0x0Fu << bb) | (0x0Fu >> (8 - bb))) & 0xFFu);
+                const uint32_t t = bit_select(qd[0][bb & 3], qd[1][bb & 3], m3);   // planes 0-3 on positions bb .. bb + 3
+                r[bb] = __funnelshift_r(t, t, bb);
+            }
+        }
+    }
+}
+
+// Eight registers of four channel bytes (byte i of register b = channel 8i + b) -> plane words: the mirror image of
+// planes_to_bytes.  With c_b = rotl(bytes_b, b), plane j is rotr(t_j, j) where byte position (b + j) & 7 of t_j comes from
+// register b; the pair and quad selects are shared between the planes (16 + nb selects where a merge per (plane,
+// register) takes 8 * nb).
+__device__ __forceinline__ void bytes_to_planes(const uint32_t (&cr)[8], int nb, uint32_t (&planes)[8]) {
+    uint32_t pr[4][2], qd[2][4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        pr[j][0] = bit_select(cr[2 * j], cr[2 * j + 1], 0x55555555u);
+        pr[j][1] = bit_select(cr[2 * j + 1], cr[2 * j], 0x55555555u);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint32_t m2 = c == 0 ? 0x33333333u : c == 1 ? 0x66666666u : c == 2 ? 0xCCCCCCCCu : 0x99999999u;
+            qd[i][c] = bit_select(pr[2 * i][c & 1], pr[2 * i + 1][c & 1], m2);
+        }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        if (j >= nb) break;
+        const uint32_t m3 = 0x01010101u * (uint32_t)(((0x0Fu << j) | (0x0Fu >> (8 - j))) & 0xFFu);
+        const uint32_t t = bit_select(qd[0][j & 3], qd[1][j & 3], m3);
+        planes[j] = __funnelshift_r(t, t, j);
+    }
+}
+
+// fl(t) -> the bit pattern 0x4B000000 + clamp(floor(t), 0, qmax) without the conversion pipe and with one logic-pipe
+// instruction: t + |t| is 2 * max(t, 0) exactly, the minimum with 2 * qmax + 1 bounds it (floor and clamp commute for
+// integer bounds: floor(min(max(t, 0), qmax + 1/2)) = min(max(floor(t), 0), qmax)), and the halving and the 2^23 go into
+// one multiply-add rounded toward -inf, whose low mantissa bits are the floor.
+__device__ __forceinline__ uint32_t code_pattern(float t, float hi2) {
+    const float a = __fadd_rn(t, fabsf(t));
+    return __float_as_uint(__fmaf_rd(fminf(a, hi2), 0.5f, 8388608.0f));
 }
 
 // One 32-channel group of the plain epilogue: 32 accumulators of this thread's pixel -> stores, fp32 steps,
@@ -308,40 +399,26 @@ __device__ __forceinline__ void pipe_group32(const ConvParams& p, uint32_t (&v)[
     if (WANT_Q) {
         // The clamp at zero of the quantizer makes an explicit ReLU redundant here: a negative y gives
         // floor(y / step + 0.5) <= 0 and is clamped to code 0, exactly what max(y, 0) would give.
-        // floor(t) sits in the low mantissa bits of t + 2^23 added with rounding toward minus infinity; as integers the
-        // bit patterns of these sums are ordered like the sums themselves (negative ones below all others), so the
-        // clamp to 0 .. qmax is an integer clamp of the pattern to [bits(2^23), bits(2^23) + qmax].
+        // Floor and clamp without the conversion pipe: code_pattern above.
         // Byte register bb holds the codes of channels {bb, 8 + bb, 16 + bb, 24 + bb}, rotated left by bb.
         uint32_t cr[8];
-        const uint64_t magic2 = f32x2_pack(8388608.0f, 8388608.0f);
-        const int m_lo = 0x4B000000, m_hi = 0x4B000000 + qmax;
+        const float hi2 = (float)(2 * qmax + 1);
 #pragma unroll
         for (int bb = 0; bb < 8; ++bb) {
-            int m[4];
+            uint32_t m[4];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 // (the multiply and the addition of 0.5 are scalar instructions with explicit rounding, which the assembler
                 // never contracts into a fused multiply-add; issued as a packed pair they came out fused)
                 const uint64_t w = yy[h][bb];
-                const float t_lo = __fadd_rn(__fmul_rn(__uint_as_float((uint32_t)w), inv_next), 0.5f);
-                const float t_hi = __fadd_rn(__fmul_rn(__uint_as_float((uint32_t)(w >> 32)), inv_next), 0.5f);
-                const uint64_t t = f32x2_add_rd(f32x2_pack(t_lo, t_hi), magic2);
-                m[2 * h] = min(max((int)(uint32_t)t, m_lo), m_hi);
-                m[2 * h + 1] = min(max((int)(uint32_t)(t >> 32), m_lo), m_hi);
+                m[2 * h] = code_pattern(__fadd_rn(__fmul_rn(__uint_as_float((uint32_t)w), inv_next), 0.5f), hi2);
+                m[2 * h + 1] = code_pattern(__fadd_rn(__fmul_rn(__uint_as_float((uint32_t)(w >> 32)), inv_next), 0.5f), hi2);
             }
-            const uint32_t c4 = __byte_perm(__byte_perm((uint32_t)m[0], (uint32_t)m[1], 0x0040),
-                                            __byte_perm((uint32_t)m[2], (uint32_t)m[3], 0x0040), 0x5410);
+            const uint32_t c4 = __byte_perm(__byte_perm(m[0], m[1], 0x0040), __byte_perm(m[2], m[3], 0x0040), 0x5410);
             cr[bb] = __funnelshift_l(c4, c4, bb);
         }
         uint32_t planes[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            if (j >= nb) break;
-            uint32_t t = cr[0] & (0x01010101u << (j & 7));
-#pragma unroll
-            for (int bb = 1; bb < 8; ++bb) t |= cr[bb] & (0x01010101u << ((bb + j) & 7));
-            planes[j] = __funnelshift_r(t, t, j);
-        }
+        bytes_to_planes(cr, nb, planes);
         if (pvalid && EBS_IN_RANGE(p, CHK_PIPE_PN, (dst - p.packed_next) + nb - 1, p.lim_pn)) {
             if (nb == 4) {
                 *reinterpret_cast<uint4*>(dst) = make_uint4(planes[0], planes[1], planes[2], planes[3]);
@@ -444,33 +521,21 @@ __device__ __forceinline__ void pipe_group32_packed(const uint32_t (&v)[32], boo
                                                     uint32_t* dst, const ConvParams& p, PlaneHold<G>& hold) {
     uint32_t cr[8];
     const uint64_t S2 = f32x2_pack(S, S);
-    const uint64_t magic2 = f32x2_pack(8388608.0f, 8388608.0f);
-    const int m_lo = 0x4B000000, m_hi = 0x4B000000 + qmax;
+    const float hi2 = (float)(2 * qmax + 1);
 #pragma unroll
     for (int bb = 0; bb < 8; ++bb) {
-        int m[4];
+        uint32_t m[4];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const uint64_t w = f32x2_mul_rn(f32x2_pack((float)(int)v[16 * h + bb], (float)(int)v[16 * h + 8 + bb]), S2);
-            const float t_lo = __fadd_rn(__fmul_rn(__uint_as_float((uint32_t)w), inv_next), 0.5f);
-            const float t_hi = __fadd_rn(__fmul_rn(__uint_as_float((uint32_t)(w >> 32)), inv_next), 0.5f);
-            const uint64_t t = f32x2_add_rd(f32x2_pack(t_lo, t_hi), magic2);
-            m[2 * h] = min(max((int)(uint32_t)t, m_lo), m_hi);
-            m[2 * h + 1] = min(max((int)(uint32_t)(t >> 32), m_lo), m_hi);
+            m[2 * h] = code_pattern(__fadd_rn(__fmul_rn(__uint_as_float((uint32_t)w), inv_next), 0.5f), hi2);
+            m[2 * h + 1] = code_pattern(__fadd_rn(__fmul_rn(__uint_as_float((uint32_t)(w >> 32)), inv_next), 0.5f), hi2);
         }
-        const uint32_t c4 = __byte_perm(__byte_perm((uint32_t)m[0], (uint32_t)m[1], 0x0040),
-                                        __byte_perm((uint32_t)m[2], (uint32_t)m[3], 0x0040), 0x5410);
+        const uint32_t c4 = __byte_perm(__byte_perm(m[0], m[1], 0x0040), __byte_perm(m[2], m[3], 0x0040), 0x5410);
         cr[bb] = __funnelshift_l(c4, c4, bb);
     }
     uint32_t planes[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        if (j >= nb) break;
-        uint32_t t = cr[0] & (0x01010101u << (j & 7));
-#pragma unroll
-        for (int bb = 1; bb < 8; ++bb) t |= cr[bb] & (0x01010101u << ((bb + j) & 7));
-        planes[j] = __funnelshift_r(t, t, j);
-    }
+    bytes_to_planes(cr, nb, planes);
     pipe_store_planes(planes, nb, dst, pvalid, hold, p);
 }
 
@@ -488,25 +553,16 @@ __device__ __forceinline__ void pipe_group32_affine(const uint32_t (&v)[32], con
     const bool has_rp = p.res_packed != nullptr;
     if (has_rp) {
         const uint32_t* rw = p.res_packed + ((size_t)gp * p.CWo + (cbase >> 5)) * p.res_bits;
-        uint32_t rv[8];
+        uint32_t rw8[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const uint32_t w = (pvalid && j < p.res_bits) ? __ldg(rw + j) : 0u;
-            rv[j] = __funnelshift_l(w, w, j);
-        }
-#pragma unroll
-        for (int bb = 0; bb < 8; ++bb) {
-            uint32_t t = rv[0] & (0x01010101u << bb);
-#pragma unroll
-            for (int j = 1; j < 8; ++j) t |= rv[j] & (0x01010101u << ((bb + j) & 7));
-            rbyte[bb] = __funnelshift_r(t, t, bb);
-        }
+        for (int j = 0; j < 8; ++j) rw8[j] = (pvalid && j < p.res_bits) ? __ldg(rw + j) : 0u;
+        planes_to_bytes<8>(rw8, rbyte);
     }
     uint32_t cr[8];
-    const int m_lo = 0x4B000000, m_hi = 0x4B000000 + qmax;
+    const float hi2 = (float)(2 * qmax + 1);
 #pragma unroll
     for (int bb = 0; bb < 8; ++bb) {
-        int m[4];
+        uint32_t m[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int c = 8 * i + bb;
@@ -515,22 +571,13 @@ __device__ __forceinline__ void pipe_group32_affine(const uint32_t (&v)[32], con
             if (p.ch_bias) t = __fadd_rn(t, __ldg(p.ch_bias + cbase + c));
             if (p.residual && pvalid) t = __fadd_rn(t, __ldg(p.residual + o + c));
             if (has_rp) t = __fadd_rn(t, __fmul_rn(p.res_scale, (float)((rbyte[bb] >> (8 * i)) & 0xFFu)));
-            const float u = __fadd_rn(__fmul_rn(t, inv_next), 0.5f);
-            m[i] = min(max(__float_as_int(__fadd_rd(u, 8388608.0f)), m_lo), m_hi);
+            m[i] = code_pattern(__fadd_rn(__fmul_rn(t, inv_next), 0.5f), hi2);
         }
-        const uint32_t c4 = __byte_perm(__byte_perm((uint32_t)m[0], (uint32_t)m[1], 0x0040),
-                                        __byte_perm((uint32_t)m[2], (uint32_t)m[3], 0x0040), 0x5410);
+        const uint32_t c4 = __byte_perm(__byte_perm(m[0], m[1], 0x0040), __byte_perm(m[2], m[3], 0x0040), 0x5410);
         cr[bb] = __funnelshift_l(c4, c4, bb);
     }
     uint32_t planes[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        if (j >= nb) break;
-        uint32_t t = cr[0] & (0x01010101u << (j & 7));
-#pragma unroll
-        for (int bb = 1; bb < 8; ++bb) t |= cr[bb] & (0x01010101u << ((bb + j) & 7));
-        planes[j] = __funnelshift_r(t, t, j);
-    }
+    bytes_to_planes(cr, nb, planes);
     pipe_store_planes(planes, nb, dst, pvalid, hold, p);
 }
 
@@ -845,16 +892,7 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                             r[bb] = __byte_perm(lo, hi, 0x5410);
                         }
                     } else {
-                        uint32_t v[NW];
-#pragma unroll
-                        for (int k = 0; k < NW; ++k) v[k] = __funnelshift_l(a_set[u][j][k], a_set[u][j][k], k);
-#pragma unroll
-                        for (int bb = 0; bb < 8; ++bb) {
-                            uint32_t t = v[0] & (0x01010101u << bb);
-#pragma unroll
-                            for (int k = 1; k < NW; ++k) t |= v[k] & (0x01010101u << ((bb + k) & 7));
-                            r[bb] = __funnelshift_r(t, t, bb);
-                        }
+                        planes_to_bytes<NW>(a_set[u][j], r);
                     }
                     uint8_t* dst = A_st + slot_dst[j];
                     if (!EBS_IN_RANGE(p, CHK_PIPE_STAGE, (dst + SP * 16 + 15) - stages, NST * g.stage_bytes) ||
