@@ -323,8 +323,11 @@ int ebs_dequant(const int32_t *acc_dev, size_t n_pixels, int c_out, float scale,
  *   quantize_b(u) = fl32(1/(2^b - 1)) * floor((2^b - 1) u + 0.5)   (Eq. 1c, round half up)
  * `bits` (each 1..16) and `coeff` are HOST arrays of n_cand <= EBS_MAX_CANDIDATES entries; coeff is
  * the softmax of the strengths (deterministic search) or the Gumbel-softmax sample (stochastic
- * search, Eq. 8), computed by the caller.  Every fp32 operation is rounded on its own, candidates
- * are accumulated in array order.  src/dst are device tensors of n floats (16-byte aligned; dst
+ * search, Eq. 8), computed by the caller.  Activations: every fp32 operation is rounded on its own
+ * and candidates are accumulated in array order (bit-exact against that chain).  Weights: fp32 with
+ * tanhf, the blend evaluated as sum_i fl32(2 coeff[i] / (2^b[i] - 1)) * code_i - sum_i coeff[i] with
+ * fused multiply-adds (within 1e-5 of the formula in double precision away from rounding ties of
+ * the codes).  src/dst are device tensors of n floats (16-byte aligned; dst
  * may alias src); scratch_dev is 16 bytes of device memory the weight call uses for max|w|.
  */
 #define EBS_MAX_CANDIDATES 8

@@ -9,6 +9,8 @@ struct SearchParams {
     float coeff[EBS_MAX_CANDIDATES];   // blend coefficients (softmax of the strengths, or Gumbel-softmax)
     float levels[EBS_MAX_CANDIDATES];  // 2^b - 1 as float
     float inv_levels[EBS_MAX_CANDIDATES];  // fl32(1 / (2^b - 1))
+    float w_gain[EBS_MAX_CANDIDATES];  // weights: fl32(2 coeff / (2^b - 1)), the weight of one code step in the blend
+    float w_offset;                    // weights: -sum of the coefficients
     int n_cand;
 };
 
@@ -44,15 +46,27 @@ __global__ void __launch_bounds__(256) abs_max_kernel(const float* __restrict__ 
     if ((threadIdx.x & 31) == 0 && m > 0.0f) atomicMax(out, __float_as_uint(m));
 }
 
-// Eq. 1a per candidate, blended (Eq. 6): w_hat = sum_i coeff_i * (2 * quantize_b_i(tanh(w) / (2 max|tanh|) + 1/2) - 1)
+// tanh(w) = sign(w) (1 - 2 / (exp(2|w|) + 1)) with the hardware exponential and reciprocal: absolute error below 3e-7
+// (the cancellation for small |w| costs relative, not absolute accuracy, and the blend needs the latter); tanhf spends
+// twice the instructions on a relative bound.
+__device__ __forceinline__ float tanh_fast(float w) {
+    const float e = __expf(2.0f * fabsf(w));                   // +inf for large |w|: 2 / inf = 0, tanh = 1
+    return copysignf(1.0f - __fdividef(2.0f, e + 1.0f), w);
+}
+
+// Eq. 1a per candidate, blended (Eq. 6): w_hat = sum_i coeff_i * (2 * quantize_b_i(tanh(w) / (2 max|tanh|) + 1/2) - 1),
+// evaluated as sum_i (2 coeff_i / L_i) * code_i - sum_i coeff_i with code_i = floor(L_i u + 1/2): a multiply-add, a
+// floor and a multiply-add per candidate.  The floor is taken on the fp32 pipe (u L + 1/2 is in [0.5, 2^16), so adding
+// 2^23 with rounding toward -inf leaves it in the low mantissa bits): the conversion pipe, which tanhf already loads
+// with an exponential and a reciprocal, retires 16 results per clock and SM and bounded this kernel.
 template <int NC>
 __device__ __forceinline__ float blend_weight(float w, float inv_2max, const SearchParams& sp) {
-    const float u = __fadd_rn(__fmul_rn(tanhf(w), inv_2max), 0.5f);
-    float acc = 0.0f;
+    const float u = fmaf(tanh_fast(w), inv_2max, 0.5f);
+    float acc = sp.w_offset;
 #pragma unroll
     for (int i = 0; i < NC; ++i) {
-        const float lvl = __fadd_rn(__fmul_rn(2.0f, quantize_unit(u, sp.levels[i], sp.inv_levels[i])), -1.0f);
-        acc = __fadd_rn(acc, __fmul_rn(sp.coeff[i], lvl));
+        const float code = __fadd_rn(__fadd_rd(fmaf(u, sp.levels[i], 0.5f), 8388608.0f), -8388608.0f);
+        acc = fmaf(sp.w_gain[i], code, acc);
     }
     return acc;
 }
@@ -73,7 +87,7 @@ __global__ void __launch_bounds__(256) search_forward_kernel(const float* __rest
                                                              const SearchParams sp, float* __restrict__ dst) {
     float k = 1.0f / alpha;                      // fl32(1 / alpha), one rounded division
     if (WEIGHTS) {                               // 1 / (2 max|tanh(w)|); tanh is monotonic, so max|tanh(w)| = tanh(max|w|)
-        const float mt = tanhf(__uint_as_float(__ldg(abs_max_bits)));
+        const float mt = tanh_fast(__uint_as_float(__ldg(abs_max_bits)));   // the same tanh as the elements: u <= 1
         k = mt > 0.0f ? __fdiv_rn(1.0f, __fmul_rn(2.0f, mt)) : 0.0f;
     }
     const size_t stride = (size_t)gridDim.x * blockDim.x;
@@ -117,7 +131,11 @@ static int fill_params(SearchParams& sp, const int* bits, const float* coeff, in
         sp.coeff[i] = coeff[i];
         sp.levels[i] = (float)((1 << bits[i]) - 1);
         sp.inv_levels[i] = 1.0f / sp.levels[i];
+        sp.w_gain[i] = (float)(2.0 * (double)coeff[i] / (double)sp.levels[i]);
     }
+    double csum = 0.0;
+    for (int i = 0; i < n_cand; ++i) csum += (double)coeff[i];
+    sp.w_offset = (float)-csum;
     return EBS_OK;
 }
 
