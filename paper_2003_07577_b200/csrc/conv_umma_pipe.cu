@@ -32,13 +32,14 @@ const ConvVariant* conv_umma_pipe_variant(int a_bits, int variant) {
 }
 
 bool conv_umma_pipe_applies(const ConvParams& p, int variant) {
-    return variant >= 0 && variant < NUM_UMMA_PIPE_VARIANTS &&
-           pipe_geometry(p, 64 << variant, pipe_sm_count(), p.pipe_m_sub).ok;
+    if (variant == 3) return pipe_pair_request_ok(p) && pipe_geometry(p, 256, pipe_sm_count(), p.pipe_m_sub, true).ok;
+    return variant >= 0 && variant < 3 && pipe_geometry(p, 64 << variant, pipe_sm_count(), p.pipe_m_sub).ok;
 }
 
 long long conv_umma_pipe_items(const ConvParams& p, int variant) {
     if (variant < 0 || variant >= NUM_UMMA_PIPE_VARIANTS) return -1;
-    const PipeGeom g = pipe_geometry(p, 64 << variant, pipe_sm_count(), p.pipe_m_sub);
+    const PipeGeom g = variant == 3 ? pipe_geometry(p, 256, pipe_sm_count(), p.pipe_m_sub, true)
+                                    : pipe_geometry(p, 64 << variant, pipe_sm_count(), p.pipe_m_sub);
     return g.ok ? (long long)g.n_ptiles * g.n_ctiles : -1;
 }
 

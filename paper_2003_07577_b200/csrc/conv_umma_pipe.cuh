@@ -24,13 +24,17 @@
 //    parity; a single warp needs 140-180 clocks per MMA and was the bound of the k x k layers), warp 10 fetches weight
 //    tiles (every lane one tile of a ring slot), warps 12-19 run the epilogue out of tensor memory while the next
 //    tile's MMAs fill the other accumulator set.
-//  * Bit <-> byte transposes with one masked merge per plane and register: with v_k = rotl(w_k, k) the
-//    byte register of channels {b, 8+b, 16+b, 24+b} is rotr(OR_k v_k & (0x01010101 << ((b+k) & 7)), b);
-//    the epilogue packs requantized codes into plane words with the mirrored identity.
+//  * Bit <-> byte transposes by rotate and bit-select: with v_k = rotl(w_k, k) the byte register of
+//    channels {b, 8+b, 16+b, 24+b} is rotr(t_b, b), byte position (b+k) & 7 of t_b taken from v_k; the
+//    selects of plane pairs and quads are shared between the eight registers (planes_to_bytes), and the
+//    epilogue packs requantized codes into plane words with the mirrored tree (bytes_to_planes).
+//  * PAIR form (the 256-channel tile on a cluster of two CTAs): one MMA of M = 256 per (tap, word) over
+//    both CTAs' shared and tensor memory (cta_group::2), each CTA fetching the weight rows of half the
+//    channel tile; see the kernel.  No load is multicast; only tcgen05.commit signals both CTAs.
 //
 // Every wait on an mbarrier is bounded (ConvParams::wait_limit polls); on a timeout the CTA raises a
 // shared abort flag, all its loops end, it records the event in a device counter, frees its tensor
-// memory and returns.  No clusters, no multicast.
+// memory and returns.  The single-CTA forms use no clusters.
 #pragma once
 
 #include "conv_umma_strip.cuh"
@@ -82,6 +86,7 @@ struct PipeGeom {
     int b_resident, b_total_bytes, taps;
     int b_slots, b_group;              // streamed weights: ring of slots of b_group (tap, word) tiles of TILE_N x 32 bytes
     int nbuf, tmem_cols, smem_bytes;
+    int pair;                          // 1: two CTAs of a cluster share every MMA (256 pixels x 256 channels, half a weight tile each)
     int grid_x, grid_y;
     int ph_a[PIPE_MAX_PHASES], ph_b[PIPE_MAX_PHASES];
     int ph_tap0[PIPE_MAX_PHASES + 1];  // tap slots of phase i: [ph_tap0[i], ph_tap0[i + 1])
@@ -93,8 +98,12 @@ struct PipeGeom {
 inline int floordiv_int(int a, int b) { return (a >= 0) ? a / b : -((-a + b - 1) / b); }
 
 // m_sub_req / ks_req = 0: chosen here.  Returns ok = false when the kernel does not apply.
-inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_sub_req = 0) {
+inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_sub_req = 0, bool pair = false) {
     PipeGeom g{};
+    if (pair && (tile_n != 256 || (p.Co % 256) != 0 || sms < 2)) return g;
+    const int pw = pair ? 2 : 1;                               // CTAs that share a pixel pair-tile
+    g.pair = pair ? 1 : 0;
+    sms /= pw;                                                 // the unit that takes work items: a CTA, or a pair
     const int taps = p.kh * p.kw;
     if (p.w_levels || p.sh > 2 || p.sw > 2 || taps > PIPE_MAX_TAPS || p.kh > 16 || p.kw > 16) return g;
     if (tile_n != 64 && tile_n != 128 && tile_n != 256) return g;
@@ -135,7 +144,7 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
     int max_ph_taps = 0;
     for (int i = 0; i < g.n_ph; ++i) max_ph_taps = max_ph_taps > g.ph_tap0[i + 1] - g.ph_tap0[i] ? max_ph_taps : g.ph_tap0[i + 1] - g.ph_tap0[i];
     g.n_ctiles = (p.Co + tile_n - 1) / tile_n;
-    const int b_tile = tile_n * 32;
+    const int b_tile = tile_n * 32 / pw;                       // a pair: each CTA holds the rows of half the channels
     g.b_total_bytes = p.CW * taps * b_tile;
     const int deep = p.CW * taps;                               // MMAs per accumulator and tile
     // candidates for the super-tile, largest first: it must leave the strip within the expanders' items and give
@@ -147,7 +156,7 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
         const int nb = (2 * m * tile_n <= 512) ? 2 : 1;
         if (nb == 1 && deep < 64 && !m_sub_req) continue;        // shallow reductions want the epilogue overlapped
         if (m * UMMA_M + max_shift > PIPE_MAX_ITEMS) continue;
-        const long long pt = (frame + (long long)m * UMMA_M - 1) / ((long long)m * UMMA_M);
+        const long long pt = (frame + (long long)m * UMMA_M * pw - 1) / ((long long)m * UMMA_M * pw);
         if (!m_sub_req && m > 1 && pt * g.n_ctiles < (deep >= 64 ? 1LL : 2LL) * sms) continue;
         m_sub = m;
         break;
@@ -158,7 +167,7 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
     g.nbuf = (2 * m_sub * tile_n <= 512) ? 2 : 1;
     g.tmem_cols = g.nbuf * m_sub * tile_n;
     if (g.tmem_cols < 32) g.tmem_cols = 32;
-    g.n_ptiles = (int)((frame + g.tile_pix - 1) / g.tile_pix);
+    g.n_ptiles = (int)((frame + (long long)g.tile_pix * pw - 1) / ((long long)g.tile_pix * pw));   // pair-tiles for a pair
     g.S = g.tile_pix + max_shift;
     g.SP = (g.S + 7) & ~7;
     g.a_word_bytes = g.SP * 32 + 64;                           // sized with the largest skew; fixed once ks is known
@@ -175,7 +184,7 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
     // Streamed weights go through a ring of their own (slots of a few consecutive (tap, word) tiles), so that copies are
     // in flight all the time (a stage-sized unit would leave the copy engine idle while a stage's MMAs run).
     auto stage_bytes = [&](int k) { return (k * g.a_word_bytes + 255) & ~255; };
-    const int b_ring_min = g.b_resident ? 0 : 96 * 1024;
+    const int b_ring_min = g.b_resident ? 0 : 96 * 1024 / pw;
     const int avail = budget - (g.b_resident ? g.b_total_bytes : b_ring_min);
     while (ks > 1 && 2 * stage_bytes(ks) > avail) --ks;
     if (2 * stage_bytes(ks) > avail) return g;
@@ -198,7 +207,8 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
     g.a_stage_bytes = stage_bytes(g.kss);
     g.stage_bytes = g.a_stage_bytes;
     g.n_stages = avail / g.stage_bytes;
-    if (g.n_stages > (g.b_resident ? PIPE_MAX_STAGES : 3)) g.n_stages = g.b_resident ? PIPE_MAX_STAGES : 3;
+    const int st_cap = g.b_resident ? PIPE_MAX_STAGES : (pair ? PIPE_MAX_STAGES : 3);
+    if (g.n_stages > st_cap) g.n_stages = st_cap;
     if (!g.b_resident) {
         // a slot holds up to 32 KB of consecutive tiles of a chunk (one wait and one commit per slot, not per MMA)
         g.b_group = 32768 / b_tile;
@@ -215,11 +225,11 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
         long long gx = sms / g.n_ctiles;
         if (gx < 1) gx = 1;
         if (gx > g.n_ptiles) gx = g.n_ptiles;
-        g.grid_x = (int)gx;
+        g.grid_x = (int)gx * pw;
     } else {
         g.grid_y = 1;
         const long long items = (long long)g.n_ptiles * g.n_ctiles;
-        g.grid_x = (int)(items < sms ? items : sms);
+        g.grid_x = (int)(items < sms ? items : sms) * pw;
     }
     g.ok = g.n_stages >= 2 && g.smem_bytes <= PIPE_SMEM_MAX && g.grid_y <= 65535 && g.n_ctiles <= 65535;
     return g;
@@ -330,6 +340,56 @@ __device__ __forceinline__ void umma_i8_split(uint32_t leader, uint32_t tmem_d, 
         "@q tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t}\n"
         :: "r"(tmem_d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(leader)
         : "memory");
+}
+// The same for a CTA pair: M = 256 over the two CTAs' tensor memory, issued by the even CTA; the commit arrives on the
+// barrier at this offset in both CTAs.
+__device__ __forceinline__ void umma_i8_split_pair(uint32_t leader, uint32_t tmem_d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                                   uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "setp.ne.b32 q, %7, 0;\n\t"
+        "@q tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %5, p;\n\t}\n"
+        :: "r"(tmem_d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(leader)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_pred_pair(uint32_t leader, uint64_t* bar) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t.reg .b16 m;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "mov.b16 m, 3;\n\t"
+        "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}\n"
+        ::"r"(smem_u32(bar)), "r"(leader) : "memory");
+}
+// Address of the same shared-memory object in the CTA of the given rank of this cluster.
+__device__ __forceinline__ uint32_t cluster_addr(const void* ptr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(smem_u32(ptr)), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_address) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];\n" ::"r"(cluster_address) : "memory");
+}
+// Bounded wait on a barrier another CTA of the cluster arrives on.
+__device__ __forceinline__ bool mbar_wait_cluster_hot(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned limit) {
+    const uint32_t addr = smem_u32(bar);
+    for (unsigned it = 0; it < limit; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}\n"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;\n" ::: "memory");
 }
 __device__ __forceinline__ void umma_commit_pred(uint32_t leader, uint64_t* bar) {
     asm volatile(
@@ -682,10 +742,19 @@ inline bool pipe_hold_applies(const ConvParams& p, int tile_n) {
            (p.Co & 31) == 0 && !p.w_levels;
 }
 
-template <int AB, int TILE_N, bool AFFINE, int FORM>
+template <int AB, int TILE_N, bool AFFINE, int FORM, bool PAIR = false>
 __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const ConvParams p, const PipeGeom g) {
     constexpr int EPI_G = FORM == 2 ? TILE_N / 64 : 1;         // groups of an output run held back (odd plane counts)
-    constexpr int B_TILE_BYTES = TILE_N * 32;
+    // PAIR: the two CTAs of a cluster work as one.  Each expands its own 128 * m_sub pixels and holds the weight rows of
+    // half the channel tile; the even CTA issues MMAs of M = 256 (cta_group::2) that read both CTAs' shared memory and
+    // write both CTAs' tensor memory, so a weight byte is fetched from L2 once per 256 pixels instead of once per 128.
+    // The odd CTA's issuing warp only reports to the even CTA when its stages, weight slots and accumulators are ready.
+    constexpr int B_ROWS = PAIR ? TILE_N / 2 : TILE_N;
+    constexpr int B_TILE_BYTES = B_ROWS * 32;
+    static_assert(!PAIR || TILE_N == 256, "a CTA pair works on 256-channel tiles");
+    __shared__ __align__(8) uint64_t st_peer[PAIR ? PIPE_MAX_STAGES : 1], bs_peer[PAIR ? PIPE_MAX_BSLOTS : 1], acc_peer[2], b_peer;
+    const int crank = PAIR ? (int)(blockIdx.x & 1u) : 0;       // rank in the pair (cluster of 2 along x)
+    const int bx = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, gx = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     extern __shared__ uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t st_full[PIPE_MAX_STAGES], st_empty[PIPE_MAX_STAGES], acc_full[2], acc_empty[2], b_full;
     __shared__ __align__(8) uint64_t bs_full[PIPE_MAX_BSLOTS], bs_empty[PIPE_MAX_BSLOTS];   // streamed weight tiles
@@ -708,7 +777,7 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                                               (g.smem_bytes - 1024 - PIPE_MAX_MMAS * 8));
     {
         const int per_tap = g.kss * g.m_sub, total_e = per_tap * g.taps;
-        const uint32_t bt16 = (uint32_t)(TILE_N * 32) >> 4;
+        const uint32_t bt16 = (uint32_t)B_TILE_BYTES >> 4;
         for (int e = tid; e < total_e; e += PIPE_THREADS) {
             int ph = 0;
             while (ph + 1 < g.n_ph && e >= per_tap * g.ph_tap0[ph + 1]) ++ph;
@@ -733,15 +802,15 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
     // Streamed weights: every CTA of a channel tile reads the same weight tiles, and CTAs that start together would ask
     // the same few L2 slices for the same tile at the same time.  Integer accumulation is exact in any order, so each
     // CTA starts its walk over the word groups at a different one.
-    const int wg_rot = resident ? 0 : (int)(blockIdx.x % (unsigned)nwg);
+    const int wg_rot = resident ? 0 : bx % nwg;
     volatile int* abortp = &abort_flag;
     const unsigned wait_limit = p.wait_limit;
 
     // work items of this CTA: (pixel super-tile, channel tile)
     const int n_items = resident ? g.n_ptiles : g.n_ptiles * g.n_ctiles;
-    const int my_items = ((int)blockIdx.x < n_items) ? (n_items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int my_items = (bx < n_items) ? (n_items - 1 - bx) / gx + 1 : 0;
     auto item_of = [&](int it, int& ptile, int& ctile) {
-        const int idx = (int)blockIdx.x + it * (int)gridDim.x;
+        const int idx = bx + it * gx;
         if (resident) { ptile = idx; ctile = (int)blockIdx.y; }
         else { ptile = idx / g.n_ctiles; ctile = idx - ptile * g.n_ctiles; }
     };
@@ -766,15 +835,29 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
         mbar_init(&acc_empty[0], PIPE_EPI_WARPS);
         mbar_init(&acc_empty[1], PIPE_EPI_WARPS);
         mbar_init(&b_full, 1);
+        if constexpr (PAIR) {
+            for (int s = 0; s < PIPE_MAX_STAGES; ++s) mbar_init(&st_peer[s], 1);
+            for (int s = 0; s < PIPE_MAX_BSLOTS; ++s) mbar_init(&bs_peer[s], 1);
+            mbar_init(&acc_peer[0], 1);
+            mbar_init(&acc_peer[1], 1);
+            mbar_init(&b_peer, 1);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (warp == PIPE_ISSUER_WARP) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&tmem_slot)),
-                     "r"((uint32_t)g.tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+        if constexpr (PAIR) {                                 // the same warp of both CTAs, the same slot address
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&tmem_slot)),
+                         "r"((uint32_t)g.tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;\n" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&tmem_slot)),
+                         "r"((uint32_t)g.tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();                   // the other CTA's barriers exist before anything arrives on them
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const uint32_t tmem_base = tmem_slot;
 
@@ -809,7 +892,7 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
         auto chunk_offsets = [&](int it, int ph) {
             int ptile, ctile;
             item_of(it, ptile, ctile);
-            const int f0 = ptile * g.tile_pix;
+            const int f0 = (PAIR ? 2 * ptile + crank : ptile) * g.tile_pix;
             const int pa = g.ph_a[ph], pb = g.ph_b[ph];
 #pragma unroll
             for (int j = 0; j < PIPE_SLOTS; ++j) {
@@ -914,15 +997,58 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
         }
     } else if (warp < PIPE_EPI_WARP0) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(REG_MID));
-      if (warp >= PIPE_ISSUER_WARP && warp < PIPE_ISSUER_WARP + n_iss) {
+      if (PAIR && crank == 1 && warp < PIPE_PRODUCER_WARP) {
+        // =========================== the odd CTA of a pair: reports ===========================
+        // One warp follows this CTA's own barriers in the order the even CTA's issuing warps wait for them and passes
+        // each completion on with one arrival on the even CTA's barrier of the same name.
+        if (warp == PIPE_ISSUER_WARP) {
+            const bool lane0 = (tid & 31) == 0;
+            const uint32_t r_st = cluster_addr(&st_peer[0], 0), r_bs = cluster_addr(&bs_peer[0], 0);
+            const uint32_t r_acc = cluster_addr(&acc_peer[0], 0), r_b = cluster_addr(&b_peer, 0);
+            bool ok = true;
+            if (my_items > 0 && resident) {
+                ok = mbar_wait_bounded_hot(&b_full, 0u, abortp, wait_limit);
+                if (ok && lane0) mbar_arrive_cluster(r_b);
+            }
+            int st = 0, bs = 0;
+            uint32_t st_round = 0, bs_round = 0;
+            for (int it = 0; it < my_items && ok; ++it) {
+                const int buf = g.nbuf == 2 ? (it & 1) : 0;
+                const int use = g.nbuf == 2 ? (it >> 1) : it;
+                if (use > 0) {
+                    if (!mbar_wait_bounded_hot(&acc_empty[buf], (uint32_t)((use - 1) & 1), abortp, wait_limit)) break;
+                    if (lane0) mbar_arrive_cluster(r_acc + 8u * (uint32_t)buf);
+                }
+                int ph = 0, wg = 0;
+                for (int c = 0; c < nchunks && ok; ++c) {
+                    if (!mbar_wait_bounded_hot(&st_full[st], st_round & 1u, abortp, wait_limit)) { ok = false; break; }
+                    if (lane0) mbar_arrive_cluster(r_st + 8u * (uint32_t)st);
+                    if (!resident) {
+                        const int wgr = wg + wg_rot >= nwg ? wg + wg_rot - nwg : wg + wg_rot;
+                        const int words = min(KSS, p.CW - wgr * KSS);
+                        const int ntiles = words * (g.ph_tap0[ph + 1] - g.ph_tap0[ph]);
+                        for (int i0 = 0; i0 < ntiles; i0 += GB) {
+                            if (!mbar_wait_bounded_hot(&bs_full[bs], bs_round & 1u, abortp, wait_limit)) { ok = false; break; }
+                            if (lane0) mbar_arrive_cluster(r_bs + 8u * (uint32_t)bs);
+                            if (++bs == NBS) { bs = 0; ++bs_round; }
+                        }
+                    }
+                    __syncwarp();
+                    if (++st == NST) { st = 0; ++st_round; }
+                    if (++wg == nwg) { wg = 0; ++ph; }
+                }
+            }
+        }
+      } else if (warp >= PIPE_ISSUER_WARP && warp < PIPE_ISSUER_WARP + n_iss) {
         // =========================== issuers ===========================
         const int k_iss = warp - PIPE_ISSUER_WARP;                // this warp takes the MMAs k_iss, k_iss + n_iss, ... of a chunk
         // The issuing thread is a pipeline stage of its own: every address is advanced by additions (descriptor start
         // addresses are in 16-byte units), a handful of instructions per MMA.
-        constexpr uint32_t IDESC = umma_idesc_i8(TILE_N);
+        constexpr uint32_t IDESC = PAIR ? (umma_idesc_i8(TILE_N) & ~(0x1Fu << 24)) | ((256u >> 4) << 24) : umma_idesc_i8(TILE_N);
         constexpr uint32_t BT16 = B_TILE_BYTES >> 4;
         const bool skip_mma = (p.test_flags & 1) != 0;            // test hook: issue nothing, so that waits run out
         bool ok = my_items == 0 || !resident || mbar_wait_bounded_hot(&b_full, 0u, abortp, wait_limit);
+        if (PAIR && ok && my_items > 0 && resident) ok = mbar_wait_cluster_hot(&b_peer, 0u, abortp, wait_limit);
         const uint64_t da_ring = umma_desc_interleaved(smem_u32(stages), (uint32_t)(SP * 16));
         const uint64_t db_res = umma_desc_sw32(smem_u32(b_res));   // resident tiles, or slot 0 of the ring
         const uint32_t da_lo = (uint32_t)da_ring, da_hi = (uint32_t)(da_ring >> 32);
@@ -930,6 +1056,14 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
         const uint32_t stage16 = (uint32_t)(g.stage_bytes >> 4);
         const int m_sub = g.m_sub;
         const uint32_t leader = (tid & 31) == 0 ? 1u : 0u;
+        auto mma_issue = [](uint32_t ld, uint32_t d, uint32_t al, uint32_t ah, uint32_t bl, uint32_t bh, uint32_t idesc, uint32_t accu) {
+            if constexpr (PAIR) umma_i8_split_pair(ld, d, al, ah, bl, bh, idesc, accu);
+            else umma_i8_split(ld, d, al, ah, bl, bh, idesc, accu);
+        };
+        auto mma_commit = [](uint32_t ld, uint64_t* bar) {
+            if constexpr (PAIR) umma_commit_pred_pair(ld, bar);
+            else umma_commit_pred(ld, bar);
+        };
         int st = 0, bs = 0;
         uint32_t st_round = 0, bs_round = 0;
         for (int it = 0; it < my_items && ok; ++it) {
@@ -937,12 +1071,14 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
             const int use = g.nbuf == 2 ? (it >> 1) : it;          // how often this accumulator set was used before
             if (use > 0) {                                          // its epilogue must have drained it
                 if (!mbar_wait_bounded_hot(&acc_empty[buf], (uint32_t)((use - 1) & 1), abortp, wait_limit)) break;
+                if (PAIR && !mbar_wait_cluster_hot(&acc_peer[buf], (uint32_t)((use - 1) & 1), abortp, wait_limit)) break;
             }
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
             const uint32_t tmem_d = tmem_base + (uint32_t)(buf * m_sub * TILE_N);
             int ph = 0, wg = 0;
             for (int c = 0; c < nchunks; ++c) {
                 if (!mbar_wait_bounded_hot(&st_full[st], st_round & 1u, abortp, wait_limit)) { ok = false; break; }
+                if (PAIR && !mbar_wait_cluster_hot(&st_peer[st], st_round & 1u, abortp, wait_limit)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 if (!skip_mma) {
                     const int wgr = wg + wg_rot >= nwg ? wg + wg_rot - nwg : wg + wg_rot;
@@ -957,7 +1093,7 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                         uint2 e = tab[k_iss];
                         for (int i = k_iss; i < n; i += n_iss) {
                             const uint2 nxt = tab[i + n_iss];             // (past the end: inside the table's allocation)
-                            umma_i8_split(leader, tmem_d + (e.x >> 22), a_lo + (e.x & 0x3FFFFFu), da_hi, b_lo + e.y, db_hi, IDESC,
+                            mma_issue(leader, tmem_d + (e.x >> 22), a_lo + (e.x & 0x3FFFFFu), da_hi, b_lo + e.y, db_hi, IDESC,
                                           i >= zero_n ? 1u : 0u);
                             e = nxt;
                         }
@@ -967,23 +1103,24 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                         int i = k_iss;
                         for (int i0 = 0; i0 < ntiles; i0 += GB) {
                             if (!mbar_wait_bounded_hot(&bs_full[bs], bs_round & 1u, abortp, wait_limit)) { ok = false; break; }
+                            if (PAIR && !mbar_wait_cluster_hot(&bs_peer[bs], bs_round & 1u, abortp, wait_limit)) { ok = false; break; }
                             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                             const uint32_t b_lo = db_lo + (uint32_t)(bs * GB) * BT16;
                             const int n = (i0 + min(GB, ntiles - i0)) * m_sub;
                             uint2 e = tab[i];
                             for (; i < n; i += n_iss) {
                                 const uint2 nxt = tab[i + n_iss];
-                                umma_i8_split(leader, tmem_d + (e.x >> 22), a_lo + (e.x & 0x3FFFFFu), da_hi, b_lo + e.y, db_hi, IDESC,
+                                mma_issue(leader, tmem_d + (e.x >> 22), a_lo + (e.x & 0x3FFFFFu), da_hi, b_lo + e.y, db_hi, IDESC,
                                               i >= zero_n ? 1u : 0u);
                                 e = nxt;
                             }
-                            umma_commit_pred(leader, &bs_empty[bs]);
+                            mma_commit(leader, &bs_empty[bs]);
                             if (++bs == NBS) { bs = 0; ++bs_round; }
                         }
                         if (!ok) break;
                     }
-                    umma_commit_pred(leader, &st_empty[st]);
-                    if (c == nchunks - 1) umma_commit_pred(leader, &acc_full[buf]);
+                    mma_commit(leader, &st_empty[st]);
+                    if (c == nchunks - 1) mma_commit(leader, &acc_full[buf]);
                 }
                 __syncwarp();
                 if (++st == NST) { st = 0; ++st_round; }
@@ -999,8 +1136,8 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
         const int lane = tid & 31;
         if (my_items > 0) {
             if (resident) {                                      // all tiles of this CTA's channel tile, once
-                const int co0 = (int)blockIdx.y * TILE_N;
-                const uint32_t rows = (uint32_t)min(TILE_N, p.Co16 - co0);
+                const int co0 = (int)blockIdx.y * TILE_N + crank * B_ROWS;   // a pair: this CTA's half of the channel tile
+                const uint32_t rows = (uint32_t)min(B_ROWS, p.Co16 - co0);
                 const int total_tiles = p.CW * g.taps;
                 if (lane == 0) mbar_arrive_expect_tx(&b_full, rows * 32u * (uint32_t)total_tiles);
                 __syncwarp();
@@ -1017,8 +1154,8 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
                 for (int it = 0; it < my_items && ok; ++it) {
                     int ptile, ctile;
                     item_of(it, ptile, ctile);
-                    const int co0 = ctile * TILE_N;
-                    const uint32_t bytes = (uint32_t)min(TILE_N, p.Co16 - co0) * 32u;
+                    const int co0 = ctile * TILE_N + crank * B_ROWS;
+                    const uint32_t bytes = (uint32_t)min(B_ROWS, p.Co16 - co0) * 32u;
                     int ph = 0, wg = -1;
                     for (int c = 0; c < nchunks && ok; ++c) {
                         if (++wg == nwg) { wg = 0; ++ph; }
@@ -1068,7 +1205,7 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
             item_of(it, ptile, ctile);
             const int co0 = ctile * TILE_N;
             for (int j = 0; j < g.m_sub; ++j) {
-                const int f = ptile * g.tile_pix + j * UMMA_M + row;
+                const int f = (PAIR ? 2 * ptile + crank : ptile) * g.tile_pix + j * UMMA_M + row;
                 bool pvalid = false;
                 int gp = 0;
                 if (f < g.frame) {
@@ -1102,10 +1239,15 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
     }
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();                   // neither CTA leaves while the other may still arrive on its barriers
     if (abort_flag != 0 && tid == 0) atomicAdd(&g_umma_timeouts, 1ull);
     if (warp == PIPE_ISSUER_WARP) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols)
-                     : "memory");
+        if constexpr (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols)
+                         : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols)
+                         : "memory");
     }
 }
 
@@ -1129,6 +1271,46 @@ int launch_conv_umma_pipe_form(const ConvParams& p, const PipeGeom& g, cudaStrea
     return EBS_OK;
 }
 
+// The CTA-pair form: clusters of two CTAs along x; packed-only whole tiles (form 1) or every output mode (form 0),
+// no per-channel terms.
+template <int AB, int FORM>
+int launch_conv_umma_pipe_pair_form(const ConvParams& p, const PipeGeom& g, cudaStream_t st) {
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    auto kern = conv_umma_pipe_kernel<AB, 256, false, FORM, true>;
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PIPE_SMEM_MAX);
+        attr_set[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)g.grid_x, (unsigned)g.grid_y, 1);
+    cfg.blockDim = dim3(PIPE_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)g.smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, p, g) == cudaSuccess ? EBS_OK : EBS_ERR_CUDA;
+}
+
+inline bool pipe_pair_request_ok(const ConvParams& p) {
+    return !p.ch_scale && !p.ch_bias && !p.residual && !p.res_packed && !p.w_levels && (p.Co % 256) == 0;
+}
+
+template <int AB>
+int launch_conv_umma_pipe_pair(const ConvParams& p, dim3 /*grid*/, cudaStream_t st) {
+    if (!pipe_pair_request_ok(p)) return EBS_ERR_UNSUPPORTED;
+    const PipeGeom g = pipe_geometry(p, 256, pipe_sm_count(), p.pipe_m_sub, true);
+    if (!g.ok) return EBS_ERR_UNSUPPORTED;
+    if (pipe_packed_only(p, 256)) return launch_conv_umma_pipe_pair_form<AB, 1>(p, g, st);
+    return launch_conv_umma_pipe_pair_form<AB, 0>(p, g, st);
+}
+
 template <int AB, int TILE_N>
 int launch_conv_umma_pipe(const ConvParams& p, dim3 /*grid*/, cudaStream_t st) {
     const PipeGeom g = pipe_geometry(p, TILE_N, pipe_sm_count(), p.pipe_m_sub);
@@ -1142,7 +1324,7 @@ int launch_conv_umma_pipe(const ConvParams& p, dim3 /*grid*/, cudaStream_t st) {
     return launch_conv_umma_pipe_form<AB, TILE_N, 0>(p, g, st);
 }
 
-constexpr int NUM_UMMA_PIPE_VARIANTS = 3;          // TILE_N = 64, 128, 256
+constexpr int NUM_UMMA_PIPE_VARIANTS = 4;          // TILE_N = 64, 128, 256; 256 on a CTA pair
 
 // One translation unit per activation bit count (conv_umma_pipe_a1.cu .. a8.cu): its three channel tiles and
 // its share of the give-up counter.
@@ -1151,7 +1333,8 @@ constexpr int NUM_UMMA_PIPE_VARIANTS = 3;          // TILE_N = 64, 128, 256
         static const ConvVariant row[NUM_UMMA_PIPE_VARIANTS] = {                                            \
             ConvVariant{&launch_conv_umma_pipe<AB, 64>, UMMA_M, 64, PIPE_THREADS},                          \
             ConvVariant{&launch_conv_umma_pipe<AB, 128>, UMMA_M, 128, PIPE_THREADS},                        \
-            ConvVariant{&launch_conv_umma_pipe<AB, 256>, UMMA_M, 256, PIPE_THREADS}};                       \
+            ConvVariant{&launch_conv_umma_pipe<AB, 256>, UMMA_M, 256, PIPE_THREADS},                        \
+            ConvVariant{&launch_conv_umma_pipe_pair<AB>, UMMA_M, 256, PIPE_THREADS}};                       \
         if (variant < 0 || variant >= NUM_UMMA_PIPE_VARIANTS) return nullptr;                               \
         return &row[variant];                                                                               \
     }                                                                                                       \

@@ -104,8 +104,9 @@ EBS_DECLARE_AB(5) EBS_DECLARE_AB(6) EBS_DECLARE_AB(7) EBS_DECLARE_AB(8)
 
 // 5th-generation tensor-core kernels (conv_umma_w1.cu .. conv_umma_w8.cu); variant = log2(tile_n / 16).
 enum { NUM_CONV_UMMA_VARIANTS = 5, NUM_CONV_STRIP_VARIANTS = 5, NUM_CONV_RESIDENT_VARIANTS = 5, NUM_CONV_MMA_STRIP_VARIANTS = 3,
-       NUM_CONV_PIPE_VARIANTS = 3 };
-// Persistent pipeline kernel for any stride (conv_umma_pipe.cu): variants by channel tile 64 << variant.
+       NUM_CONV_PIPE_VARIANTS = 4 };
+// Persistent pipeline kernel for any stride (conv_umma_pipe.cu): variants 0-2 by channel tile 64 << variant, variant 3 the
+// 256-channel tile on a pair of CTAs (a cluster of two sharing every MMA).
 const ConvVariant* conv_umma_pipe_variant(int a_bits, int variant);
 bool conv_umma_pipe_applies(const ConvParams& p, int variant);
 unsigned long long conv_umma_pipe_timeouts();

@@ -46,7 +46,7 @@ def test_sizes_and_shapes(ebs):
     assert ebs.ebs_conv_out_shape(d, 32, 32) == (32, 32)
     d2 = ebs.conv_desc(3, 64, 7, 7, 2, 2, 3, 3, 8, 8, 0.05, 0.05)
     assert ebs.ebs_conv_out_shape(d2, 224, 224) == (112, 112)
-    assert ebs.ebs_version() >= 100 and ebs.ebs_num_conv_variants() == 40
+    assert ebs.ebs_version() >= 100 and ebs.ebs_num_conv_variants() == 41
     assert ebs.ebs_status_string(0) == "ok" and "overflow" in ebs.ebs_status_string(-3)
     assert ebs.ebs_host_workspace_bytes(d, 1, 32, 32, ebs.EBS_U8_CODES, 2) >= 65536 + 16384 + 2 * 262144 + 16384
 

@@ -28,7 +28,7 @@ def U(ebs):
     return _util
 
 
-def _check(ebs, U, oracle, n, c, co, k, s, pad, h, w, wb, ab, nb, affine=False, min_variants=1):
+def _check(ebs, U, oracle, n, c, co, k, s, pad, h, w, wb, ab, nb, affine=False, min_variants=1, only=None):
     rng = np.random.default_rng(n + 3 * c + 5 * co + 7 * k + 11 * s + h + w + wb * 16 + ab)
     qa = U.rand_codes(rng, (n, c, h, w), ab, False)
     m = (1 << (wb - 1)) - 1
@@ -47,6 +47,8 @@ def _check(ebs, U, oracle, n, c, co, k, s, pad, h, w, wb, ab, nb, affine=False, 
     px, pw = U.pack_acts_codes(qa, ab), U.pack_weight_codes(qw, d)
     ran = 0
     for variant in U.variants_of("umma_pipe"):
+        if only is not None and variant != only:
+            continue
         if not U.applies(d, h, w, variant, n=n, epi=epi, want_y=True, want_packed=True):
             continue
         out = U.run_conv(qa, qw, d, epi, want_acc=True, want_y=True, next_bits=nb, variant=variant, px=px, pw=pw)
@@ -86,6 +88,33 @@ def test_pipe_all_activation_and_output_bit_counts(ebs, U, oracle, ab, nb):
 def test_pipe_geometries(ebs, U, oracle, case, affine):
     n, c, co, k, s, pad, h, w = case
     _check(ebs, U, oracle, n, c, co, k, s, pad, h, w, 3, 4, 4, affine=affine)
+
+
+@pytest.mark.parametrize("case", [
+    # n, c, co, k, stride, pad, h, w, ab
+    (3, 64, 256, 1, 1, 0, 20, 19, 6),     # resident weights, one pair-tile and a ragged second one
+    (4, 512, 256, 3, 1, 1, 9, 9, 3),      # streamed weights through the ring, strip halo across images
+    (2, 1024, 512, 1, 1, 0, 24, 24, 8),   # deep reduction, two channel tiles, two accumulators per CTA
+    (5, 128, 256, 3, 2, 1, 17, 16, 5),    # strided 3x3: four phase images
+    (70, 64, 256, 1, 1, 0, 28, 28, 2),    # more pair-tiles than CTA pairs: the rings and both accumulator sets wrap
+])
+def test_pipe_cta_pair(ebs, U, oracle, case):
+    """The 256-channel tile on a pair of CTAs (one MMA of 256 pixels over two SMs, half a weight tile each): the last
+    variant of the family, forced."""
+    n, c, co, k, s, pad, h, w, ab = case
+    pair = U.variants_of("umma_pipe")[-1]
+    _check(ebs, U, oracle, n, c, co, k, s, pad, h, w, 4, ab, 4, min_variants=1, only=pair)
+
+
+def test_pipe_cta_pair_declines_what_it_does_not_cover(ebs, U):
+    pair = U.variants_of("umma_pipe")[-1]
+    d = U.desc_for(64, 128, 3, 1, 1, 4, 4, 0.03, 0.07)                 # 128 output channels: no whole 256-channel tile
+    assert not U.applies(d, 16, 16, pair, n=2)
+    d = U.desc_for(64, 256, 3, 1, 1, 4, 4, 0.03, 0.07)
+    assert U.applies(d, 16, 16, pair, n=2)
+    cs = torch.ones(256, device=U.dev())
+    epi = ebs.epilogue(cs, None, None, True, 4, 1.0)                   # per-channel terms: the other variants
+    assert not U.applies(d, 16, 16, pair, n=2, epi=epi, want_packed=True)
 
 
 def test_pipe_streams_weights_that_do_not_fit_in_shared_memory(ebs, U, oracle):

@@ -27,17 +27,20 @@ def U(ebs):
     return _util
 
 
-def test_pipe_bounded_waits_give_up_and_recover(ebs, U, oracle):
+@pytest.mark.parametrize("form", ["single", "pair"])
+def test_pipe_bounded_waits_give_up_and_recover(ebs, U, oracle, form):
     """The give-up path, made to run on purpose without faulting anything: with the wait limit at a few polls and the
     issuing thread told to issue no tensor-core work, every wait for the tensor core runs out with nothing in flight;
     each thread block raises its abort flag, leaves its loops, frees its tensor memory and returns.  The counter rises,
     ebs_check_device_status reports EBS_ERR_TIMEOUT once, and the next healthy launch is bit-exact."""
     rng = np.random.default_rng(5)
     qa = U.rand_codes(rng, (4, 64, 12, 12), 3, False)
-    qw = U.rand_codes(rng, (64, 64, 3, 3), 2, True)
-    d = U.desc_for(64, 64, 3, 1, 1, 2, 3)
+    co = 64 if form == "single" else 256                      # the pair of CTAs works on whole 256-channel tiles
+    qw = U.rand_codes(rng, (co, 64, 3, 3), 2, True)
+    d = U.desc_for(64, co, 3, 1, 1, 2, 3)
     ref = oracle.conv2d_codes(qa, qw, (1, 1), (1, 1))
-    variant = U.variants_of("umma_pipe")[0]
+    variant = U.variants_of("umma_pipe")[0 if form == "single" else -1]
+    assert U.applies(d, 12, 12, variant, n=4)
     assert ebs.ebs_check_device_status() == ebs.EBS_OK
     before = ebs.ebs_device_wait_timeouts()
     ebs.ebs_test_set_device_wait(64, True)
