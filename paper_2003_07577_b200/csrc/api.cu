@@ -80,6 +80,20 @@ static unsigned long long* check_status_words() {
 static unsigned long long* check_status_words() { return nullptr; }
 #endif
 
+// A page of zero words on the device (what the pipeline kernel's expanders read where a layer pads); its address is
+// looked up once per device.
+static __device__ __align__(256) uint32_t g_zero_words[PIPE_ZERO_WORDS];
+static const uint32_t* zero_words_ptr() {
+    static const uint32_t* cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cached[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_zero_words) == cudaSuccess) cached[dev] = static_cast<const uint32_t*>(ptr);
+    }
+    return cached[dev];
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static int out_dim(int in, int pad, int k, int stride) {
@@ -258,6 +272,7 @@ static int conv_plan(const void* packed_x, int n, int h, int w, const void* pack
     p.lim_out = P * d->c_out - g_check_shrink;
     p.lim_pn = packed_next && epi ? P * p.CWo * epi->next_a_bits : 0;
     p.check_status = check_status_words();
+    p.zero_words = zero_words_ptr();
     if (epi) {
         p.ch_scale = epi->ch_scale_dev; p.ch_bias = epi->ch_bias_dev; p.residual = epi->residual_dev;
         p.res_packed = static_cast<const uint32_t*>(epi->res_packed_dev); p.res_bits = epi->res_bits; p.res_scale = epi->res_scale;

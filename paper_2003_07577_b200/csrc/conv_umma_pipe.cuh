@@ -107,6 +107,7 @@ inline PipeGeom pipe_geometry(const ConvParams& p, int tile_n, int sms, int m_su
     const int taps = p.kh * p.kw;
     if (p.w_levels || p.sh > 2 || p.sw > 2 || taps > PIPE_MAX_TAPS || p.kh > 16 || p.kw > 16) return g;
     if (tile_n != 64 && tile_n != 128 && tile_n != 256) return g;
+    if ((long long)p.CW * 8 > PIPE_ZERO_WORDS) return g;      // the zero page covers a pixel's words at 8 planes (byte codes: 8 words a word)
     g.q0r = floordiv_int(-p.ph, p.sh);
     g.q0s = floordiv_int(-p.pw, p.sw);
     const int qr_max = floordiv_int(p.kh - 1 - p.ph, p.sh), qs_max = floordiv_int(p.kw - 1 - p.pw, p.sw);
@@ -887,8 +888,17 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
             slot_pix[j] = s;
             slot_dst[j] = q * g.a_word_bytes + s * 16;
         }
-        // loader state: runs several passes ahead of the expansion, also across tile boundaries
-        int ld_it = 0, ld_c = 0, ld_sub = 0, ld_off[PIPE_SLOTS];
+        // Loader state: runs several passes ahead of the expansion, also across tile boundaries.  Per (tile, phase) a
+        // thread keeps one pointer per slot -- its pixel's words at its word position, or a page of zero words for
+        // padding, pixels past the batch and threads without an item -- so that a pass adds one warp-uniform word offset,
+        // bounded per thread so that the ragged last word group stays inside the pixel (those words feed no MMA).
+        int ld_it = 0, ld_c = 0, ld_sub = 0, ld_lim[PIPE_SLOTS];
+        const uint32_t* ld_src[PIPE_SLOTS];
+#ifdef EBS_CHECKED
+        bool ld_real[PIPE_SLOTS];
+#endif
+#pragma unroll
+        for (int j = 0; j < PIPE_SLOTS; ++j) ld_lim[j] = p.CW - ((paired && j == 0) ? 2 : 1) - max(slot_q[j], 0);
         auto chunk_offsets = [&](int it, int ph) {
             int ptile, ctile;
             item_of(it, ptile, ctile);
@@ -896,15 +906,23 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
             const int pa = g.ph_a[ph], pb = g.ph_b[ph];
 #pragma unroll
             for (int j = 0; j < PIPE_SLOTS; ++j) {
-                ld_off[j] = -1;                                 // -1: padding or past the batch -> zero bytes
+                const int qn = max(slot_q[j], 0) * NW;
+                ld_src[j] = p.zero_words + qn;                  // padding or past the batch -> zero bytes
+#ifdef EBS_CHECKED
+                ld_real[j] = false;
+#endif
                 const int f = f0 + slot_pix[j];
                 if (slot_q[j] >= 0 && f < g.frame) {
                     const uint32_t n = fastdiv((uint32_t)f, g.div_img);
                     const uint32_t rem = (uint32_t)f - n * (uint32_t)(g.Hq * g.Wq);
                     const uint32_t hq = fastdiv(rem, g.div_row), wq = rem - hq * (uint32_t)g.Wq;
                     const int h = p.sh * ((int)hq + g.q0r) + pa, w = p.sw * ((int)wq + g.q0s) + pb;
-                    if ((unsigned)h < (unsigned)p.H && (unsigned)w < (unsigned)p.W)
-                        ld_off[j] = (((int)n * p.H + h) * p.W + w) * p.CW * NW;
+                    if ((unsigned)h < (unsigned)p.H && (unsigned)w < (unsigned)p.W) {
+                        ld_src[j] = p.x + ((size_t)((((int)n * p.H + h) * p.W + w) * p.CW) * NW + qn);
+#ifdef EBS_CHECKED
+                        ld_real[j] = true;
+#endif
+                    }
                 }
             }
         };
@@ -917,22 +935,23 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
             int wg = ld_wg + wg_rot;
             if (wg >= nwg) wg -= nwg;
             if (ld_wg == 0 && ld_sub == 0) chunk_offsets(ld_it, ld_ph);
-#pragma unroll
-            for (int j = 0; j < PIPE_SLOTS; ++j)
-#pragma unroll
-                for (int k = 0; k < NW; ++k) a_set[set][j][k] = 0u;
+            const int base = wg * KSS + ld_sub * KS;            // first word of the pass (warp-uniform)
+#ifdef EBS_CHECKED
+            auto load_ok = [&](int j, const uint32_t* a, int n) {
+                return ld_real[j] ? EBS_IN_RANGE(p, CHK_PIPE_X, (a - p.x) + n - 1, p.lim_x)
+                                  : EBS_IN_RANGE(p, CHK_PIPE_X, (a - p.zero_words) + n - 1, PIPE_ZERO_WORDS);
+            };
+#else
+            auto load_ok = [](int, const uint32_t*, int) { return true; };
+#endif
             if (paired) {                                       // both words of the pixel in one run of 2 * AB words
-                const int cw = wg * KSS + ld_sub * KS + slot_q[0];
-                if (slot_q[0] >= 0 && ld_off[0] >= 0 && cw < p.CW &&
-                    EBS_IN_RANGE(p, CHK_PIPE_X, (long long)ld_off[0] + cw * NW + 2 * NW - 1, p.lim_x))
-                    load_words_global<2 * NW>(p.x + (ld_off[0] + cw * NW), *reinterpret_cast<uint32_t(*)[2 * NW]>(&a_set[set][0][0]));
+                const uint32_t* a = ld_src[0] + min(base, ld_lim[0]) * NW;
+                if (load_ok(0, a, 2 * NW)) load_words_global<2 * NW>(a, *reinterpret_cast<uint32_t(*)[2 * NW]>(&a_set[set][0][0]));
             } else {
 #pragma unroll
                 for (int j = 0; j < PIPE_SLOTS; ++j) {
-                    const int cw = wg * KSS + ld_sub * KS + slot_q[j];
-                    if (slot_q[j] >= 0 && ld_off[j] >= 0 && cw < p.CW &&
-                        EBS_IN_RANGE(p, CHK_PIPE_X, (long long)ld_off[j] + cw * NW + NW - 1, p.lim_x))
-                        load_words_global<NW>(p.x + (ld_off[j] + cw * NW), a_set[set][j]);
+                    const uint32_t* a = ld_src[j] + min(base, ld_lim[j]) * NW;
+                    if (load_ok(j, a, NW)) load_words_global<NW>(a, a_set[set][j]);
                 }
             }
             if (++ld_sub == NSUB) {
@@ -1307,6 +1326,7 @@ int launch_conv_umma_pipe_pair(const ConvParams& p, dim3 /*grid*/, cudaStream_t 
     if (!pipe_pair_request_ok(p)) return EBS_ERR_UNSUPPORTED;
     const PipeGeom g = pipe_geometry(p, 256, pipe_sm_count(), p.pipe_m_sub, true);
     if (!g.ok) return EBS_ERR_UNSUPPORTED;
+    if (!p.zero_words) return EBS_ERR_CUDA;                   // the device's zero page could not be found
     if (pipe_packed_only(p, 256)) return launch_conv_umma_pipe_pair_form<AB, 1>(p, g, st);
     return launch_conv_umma_pipe_pair_form<AB, 0>(p, g, st);
 }
@@ -1315,6 +1335,7 @@ template <int AB, int TILE_N>
 int launch_conv_umma_pipe(const ConvParams& p, dim3 /*grid*/, cudaStream_t st) {
     const PipeGeom g = pipe_geometry(p, TILE_N, pipe_sm_count(), p.pipe_m_sub);
     if (!g.ok) return EBS_ERR_UNSUPPORTED;                    // the geometry does not apply: nothing is launched
+    if (!p.zero_words) return EBS_ERR_CUDA;                   // the device's zero page could not be found
     if (pipe_packed_only(p, TILE_N)) {
         if constexpr (TILE_N >= 128) {
             if (pipe_hold_applies(p, TILE_N)) return launch_conv_umma_pipe_form<AB, TILE_N, 2>(p, g, st);

@@ -8,6 +8,8 @@
 
 namespace ebs {
 
+constexpr int PIPE_ZERO_WORDS = 8192;   // words of the zero page (ConvParams::zero_words): >= CW * planes of a layer on the pipeline kernel
+
 // Everything the convolution kernels need, passed by value as a kernel argument.
 struct ConvParams {
     const uint32_t* __restrict__ x;   // packed activations [N][H][W][CW][AB]
@@ -45,6 +47,7 @@ struct ConvParams {
     long long lim_x, lim_w;           // 32-bit words of the packed activations (bytes / 4 on the byte-code path) and of the weight plane words
     long long lim_w8;                 // bytes of the weight byte image
     long long lim_out, lim_pn;        // elements of acc / y; 32-bit words of packed_next
+    const uint32_t* zero_words;       // device page of zero words (pipeline kernel: what its expanders read for padding)
     unsigned long long* check_status; // EBS_CHECKED: device words {site << 48 | 1, index, limit}; else null
 };
 
