@@ -888,7 +888,9 @@ def run_gpu(args):
         try:
             probes = {"imma_mma_sync_tops": 2 * ebs.ebs_probe_pipe(3, 500) / 1e12,
                       "b1_mma_sync_tops": 2 * ebs.ebs_probe_pipe(1, 200) / 1e12,
-                      "and_popc_add_tops": 2 * ebs.ebs_probe_pipe(0, 500) / 1e12}
+                      "and_popc_add_tops": 2 * ebs.ebs_probe_pipe(0, 500) / 1e12,
+                      # the instruction the conv kernels issue, from shared memory, nothing else running on the SM
+                      "tcgen05_i8_m128n256k32_tops": 2 * ebs.ebs_probe_pipe(4, 2000) / 1e12}
         except Exception as exc:                                 # the probes are context, never fatal
             probes = {"error": str(exc)}
     # Roofline of the headline: the tensor-pipe kernels merge the planes of a channel back into one byte, so one
@@ -936,6 +938,9 @@ def run_gpu(args):
                      "int8_tops_conv": total_int8 / (conv_ms * 1e-3) / 1e12,
                      "gbs_conv": m["algorithmic_bytes"] / (conv_ms * 1e-3) / 1e9,
                      "tensor_peak_tops": peak_tops, "hbm_peak_gbs": hbm_gbs,
+                     # context: the same work against the rate the library's own tcgen05 int8 probe reaches on this GPU
+                     "frac_of_tcgen05_i8_probe": (total_int8 / (conv_ms * 1e-3) / 1e12 / probes["tcgen05_i8_m128n256k32_tops"]
+                                                  if probes.get("tcgen05_i8_m128n256k32_tops") else None),
                      "peak_source": f"hbm_gbs {hbm_gbs} ({peak_kind}); int8 dense = 2 x bf16 burst "
                                     f"({peaks.get('bf16_tflops')} TFLOP/s, {peak_kind})",
                      "sum_layer_roofs_ms": m["sum_layer_roofs_ms"],

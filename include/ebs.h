@@ -489,6 +489,9 @@ int ebs_conv2d_mixed_host_noalloc(const void *x_host, int dtype, int layout, int
  *   kind 1: mma.sync m16n8k256 b1 AND.POPC                      -> bit-AND-popcounts per second
  *   kind 2: POPC alone                                          -> bit-popcounts per second
  *   kind 3: mma.sync m16n8k32 u8 x s8 (one byte per bit)        -> byte multiply-accumulates per second
+ *   kind 4: tcgen05.mma kind::i8, M 128 x N 256 x K 32 from shared memory into tensor memory, 16 * iters
+ *           instructions per SM issued by one thread (iters <= 16384)  -> byte multiply-accumulates per second;
+ *           EBS_ERR_TIMEOUT if the bounded wait for their completion ran out
  * The paper has no counterpart; this is measurement support.
  */
 int ebs_probe_pipe(int kind, int iters, double *bit_ops_per_second);

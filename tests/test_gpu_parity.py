@@ -428,3 +428,12 @@ def test_pack_weights_fp32_to_paper_levels(ebs, U, oracle):
     out = torch.empty(ebs.ebs_packed_weight_bytes(d) // 4, dtype=torch.int32, device=U.dev())
     ebs.ebs_pack_weights(torch.from_numpy(w).to(U.dev()), ebs.EBS_F32, ebs.EBS_NCHW, d, out)
     assert np.array_equal(U.weight_planes(out, d), oracle.pack_weights(qs, wb))
+
+
+def test_tensor_core_probe_runs_and_is_in_range(ebs):
+    """ebs_probe_pipe kind 4 (tcgen05.mma kind::i8 from shared memory): returns, its bounded wait does not run out, and
+    the rate lies between the warp-level int8 MMA's and twice the nominal dense int8 figure."""
+    umma = 2 * ebs.ebs_probe_pipe(4, 500) / 1e12
+    imma = 2 * ebs.ebs_probe_pipe(3, 200) / 1e12
+    assert imma < umma < 9000.0, (imma, umma)
+    assert ebs.ebs_device_wait_timeouts() == 0
