@@ -30,7 +30,8 @@
 //    epilogue packs requantized codes into plane words with the mirrored tree (bytes_to_planes).
 //  * PAIR form (the 256-channel tile on a cluster of two CTAs): one MMA of M = 256 per (tap, word) over
 //    both CTAs' shared and tensor memory (cta_group::2), each CTA fetching the weight rows of half the
-//    channel tile; see the kernel.  No load is multicast; only tcgen05.commit signals both CTAs.
+//    channel tile; see the kernel.  Every copy into shared memory is a plain per-CTA copy; the MMAs' completion is
+//    signalled to both CTAs by one tcgen05.commit each.
 //
 // Every wait on an mbarrier is bounded (ConvParams::wait_limit polls); on a timeout the CTA raises a
 // shared abort flag, all its loops end, it records the event in a device counter, frees its tensor
@@ -356,13 +357,16 @@ __device__ __forceinline__ void umma_i8_split_pair(uint32_t leader, uint32_t tme
         :: "r"(tmem_d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(leader)
         : "memory");
 }
-__device__ __forceinline__ void umma_commit_pred_pair(uint32_t leader, uint64_t* bar) {
+// Completion of the pair's MMAs issued so far, signalled to the barrier at this offset in both CTAs: one commit on the
+// issuing (even) CTA's barrier and one on the odd CTA's, whose address in the cluster window is passed in.
+__device__ __forceinline__ void umma_commit_pred_pair(uint32_t leader, uint64_t* bar, uint32_t peer_delta) {
+    const uint32_t own = smem_u32(bar);
     asm volatile(
-        "{\n\t.reg .pred q;\n\t.reg .b16 m;\n\t"
-        "setp.ne.b32 q, %1, 0;\n\t"
-        "mov.b16 m, 3;\n\t"
-        "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}\n"
-        ::"r"(smem_u32(bar)), "r"(leader) : "memory");
+        "{\n\t.reg .pred q;\n\t"
+        "setp.ne.b32 q, %2, 0;\n\t"
+        "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t"
+        "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%1];\n\t}\n"
+        ::"r"(own), "r"(own + peer_delta), "r"(leader) : "memory");
 }
 // Address of the same shared-memory object in the CTA of the given rank of this cluster.
 __device__ __forceinline__ uint32_t cluster_addr(const void* ptr, uint32_t rank) {
@@ -1079,8 +1083,10 @@ __global__ void __launch_bounds__(PIPE_THREADS, 1) conv_umma_pipe_kernel(const C
             if constexpr (PAIR) umma_i8_split_pair(ld, d, al, ah, bl, bh, idesc, accu);
             else umma_i8_split(ld, d, al, ah, bl, bh, idesc, accu);
         };
-        auto mma_commit = [](uint32_t ld, uint64_t* bar) {
-            if constexpr (PAIR) umma_commit_pred_pair(ld, bar);
+        // (a pair: the odd CTA's shared window lies at a fixed distance from this one's in the cluster window)
+        const uint32_t peer_delta = PAIR ? cluster_addr(&abort_flag, 1) - smem_u32(&abort_flag) : 0u;
+        auto mma_commit = [peer_delta](uint32_t ld, uint64_t* bar) {
+            if constexpr (PAIR) umma_commit_pred_pair(ld, bar, peer_delta);
             else umma_commit_pred(ld, bar);
         };
         int st = 0, bs = 0;
