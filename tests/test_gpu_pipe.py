@@ -204,3 +204,17 @@ def test_context_path_refuses_what_it_cannot_run(ebs, U):
     with pytest.raises(ebs.EbsError) as err:
         ebs.ebs_conv2d_i8(x, 1, 8, 8, pw, d, None, acc)
     assert err.value.status == ebs.EBS_ERR_UNSUPPORTED
+
+
+def test_pipe_declines_layers_wider_than_its_zero_page(ebs, U, oracle):
+    """The expanders read padding from a page of 8192 zero words, which has to cover a pixel's words at 8 planes: a layer
+    with more than 32768 input channels goes to another kernel family, and the library's own choice stays exact."""
+    c, co = 32768 + 64, 64
+    d = U.desc_for(c, co, 1, 1, 0, 2, 2, 0.03, 0.07)
+    for variant in U.variants_of("umma_pipe"):
+        assert not U.applies(d, 4, 4, variant, n=1)
+    rng = np.random.default_rng(11)
+    qa = U.rand_codes(rng, (1, c, 4, 4), 2, False)
+    qw = rng.integers(-1, 2, size=(co, c, 1, 1), dtype=np.int32)
+    out = U.run_conv(qa, qw, d, None, want_acc=True)
+    assert np.array_equal(out["acc"], oracle.conv2d_codes(qa, qw, (1, 1), (0, 0)))
