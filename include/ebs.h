@@ -492,6 +492,7 @@ int ebs_conv2d_mixed_host_noalloc(const void *x_host, int dtype, int layout, int
  *   kind 4: tcgen05.mma kind::i8, M 128 x N 256 x K 32 from shared memory into tensor memory, 16 * iters
  *           instructions per SM issued by one thread (iters <= 16384)  -> byte multiply-accumulates per second;
  *           EBS_ERR_TIMEOUT if the bounded wait for their completion ran out
+ *   kind 5: the same with N 64 (a quarter of the work per instruction: what one issuing thread sustains)
  * The paper has no counterpart; this is measurement support.
  */
 int ebs_probe_pipe(int kind, int iters, double *bit_ops_per_second);

@@ -93,14 +93,14 @@ __global__ void __launch_bounds__(256) probe_imma_kernel(uint32_t* out, int iter
     out[blockIdx.x * blockDim.x + threadIdx.x] = (uint32_t)s;
 }
 
-int probe_umma_i8(int iters, double* macs_per_second);     // probe_umma.cu
+int probe_umma_i8(int iters, double* macs_per_second, int n_cols);     // probe_umma.cu
 
 }  // namespace ebs
 
 extern "C" int ebs_probe_pipe(int kind, int iters, double* bit_ops_per_second) {
     using namespace ebs;
-    if (kind < 0 || kind > 4 || iters < 1 || iters > (1 << 22) || !bit_ops_per_second) return EBS_ERR_INVALID_ARG;
-    if (kind == 4) return iters > (1 << 14) ? EBS_ERR_INVALID_ARG : probe_umma_i8(iters, bit_ops_per_second);
+    if (kind < 0 || kind > 5 || iters < 1 || iters > (1 << 22) || !bit_ops_per_second) return EBS_ERR_INVALID_ARG;
+    if (kind >= 4) return iters > (1 << 14) ? EBS_ERR_INVALID_ARG : probe_umma_i8(iters, bit_ops_per_second, kind == 4 ? 256 : 64);
     int dev = 0, sms = 0;
     if (check_cuda(cudaGetDevice(&dev))) return EBS_ERR_CUDA;
     if (check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev))) return EBS_ERR_CUDA;

@@ -11,6 +11,7 @@ constexpr int PROBE_UMMA_TILES = 8;
 constexpr int PROBE_UMMA_A_BYTES = 128 * 32, PROBE_UMMA_B_BYTES = 256 * 32;
 constexpr int PROBE_UMMA_SMEM = PROBE_UMMA_TILES * (PROBE_UMMA_A_BYTES + PROBE_UMMA_B_BYTES) + 1024;
 
+template <int N>
 __global__ void __launch_bounds__(128, 1) probe_umma_i8_kernel(int iters, unsigned wait_limit, unsigned* gave_up) {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t done_bar;
@@ -38,7 +39,7 @@ __global__ void __launch_bounds__(128, 1) probe_umma_i8_kernel(int iters, unsign
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const uint32_t tmem_base = tmem_slot;
     if (tid == 0) {
-        constexpr uint32_t IDESC = umma_idesc_i8(256);
+        constexpr uint32_t IDESC = umma_idesc_i8(N);
         const uint64_t da0 = umma_desc_interleaved(smem_u32(a_tiles), 128u * 16u);
         const uint64_t db0 = umma_desc_sw32(smem_u32(b_tiles));
         for (int it = 0; it < iters; ++it) {
@@ -59,11 +60,12 @@ __global__ void __launch_bounds__(128, 1) probe_umma_i8_kernel(int iters, unsign
 }
 
 // Byte multiply-accumulates per second over all SMs; EBS_ERR_TIMEOUT if a CTA's wait ran out.
-int probe_umma_i8(int iters, double* macs_per_second) {
+template <int N>
+static int probe_umma_i8_n(int iters, double* macs_per_second) {
     int dev = 0, sms = 0;
     if (check_cuda(cudaGetDevice(&dev))) return EBS_ERR_CUDA;
     if (check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev))) return EBS_ERR_CUDA;
-    if (check_cuda(cudaFuncSetAttribute(probe_umma_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PROBE_UMMA_SMEM)))
+    if (check_cuda(cudaFuncSetAttribute(probe_umma_i8_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, PROBE_UMMA_SMEM)))
         return EBS_ERR_CUDA;
     unsigned* gave_up = nullptr;
     if (check_cuda(cudaMalloc(&gave_up, sizeof(unsigned)))) return EBS_ERR_CUDA;
@@ -73,9 +75,9 @@ int probe_umma_i8(int iters, double* macs_per_second) {
     cudaEventCreate(&e1);
     // the wait covers the whole run: 16 * iters MMAs of at least 128 clocks, polled every 40-200 ns
     const unsigned limit = 1u << 22;
-    probe_umma_i8_kernel<<<sms, 128, PROBE_UMMA_SMEM>>>(iters, limit, gave_up);     // warm-up
+    probe_umma_i8_kernel<N><<<sms, 128, PROBE_UMMA_SMEM>>>(iters, limit, gave_up);     // warm-up
     cudaEventRecord(e0);
-    probe_umma_i8_kernel<<<sms, 128, PROBE_UMMA_SMEM>>>(iters, limit, gave_up);
+    probe_umma_i8_kernel<N><<<sms, 128, PROBE_UMMA_SMEM>>>(iters, limit, gave_up);
     cudaEventRecord(e1);
     int rc = check_cuda(cudaDeviceSynchronize());
     float ms = 0.f;
@@ -87,8 +89,14 @@ int probe_umma_i8(int iters, double* macs_per_second) {
     cudaFree(gave_up);
     if (rc) return rc;
     if (n_gave_up) return EBS_ERR_TIMEOUT;
-    *macs_per_second = 2.0 * PROBE_UMMA_TILES * iters * (128.0 * 256.0 * 32.0) * sms / (ms * 1e-3);
+    *macs_per_second = 2.0 * PROBE_UMMA_TILES * iters * (128.0 * N * 32.0) * sms / (ms * 1e-3);
     return EBS_OK;
+}
+
+// n_cols: 256 (the widest channel tile) or 64 (the narrowest: the same instruction count at a quarter of the work, which
+// shows what one issuing thread can sustain)
+int probe_umma_i8(int iters, double* macs_per_second, int n_cols) {
+    return n_cols == 64 ? probe_umma_i8_n<64>(iters, macs_per_second) : probe_umma_i8_n<256>(iters, macs_per_second);
 }
 
 }  // namespace ebs
